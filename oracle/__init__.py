@@ -1,0 +1,189 @@
+"""numpy front end of the CPU oracle for the BigMac DCCA MoE layer.  TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes marshalling over oracle/bigmac_oracle.cpp (fp64, per token / per row, written from
+Eq. 2 and Eq. 4 of the paper).  Nothing under the product package may import this module; only the
+tests, the smoke check and the benchmark's CPU-baseline leg do.
+
+Float inputs are float32 arrays holding values exactly representable in the workload dtype; every
+result is float64 or int32.  Weights are [out_features, in_features].
+"""
+from __future__ import annotations
+
+import ctypes as C
+from dataclasses import dataclass
+from typing import Dict, Optional
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(_build.build())
+    return _lib
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+@dataclass
+class Routing:
+    logits: np.ndarray        # [T,E] f64
+    topk_idx: np.ndarray      # [T,k] int32, slots in descending-logit order
+    topk_p: np.ndarray        # [T,k] f64, softmax over the k selected logits
+    counts: np.ndarray        # [E]   int32
+    offsets: np.ndarray       # [E+1] int32, exclusive prefix sum of counts
+    row_of_slot: np.ndarray   # [T*k] int32
+    slot_of_row: np.ndarray   # [T*k] int32
+
+
+def gate_logits(x, w_gate, b_gate=None) -> np.ndarray:
+    x, w_gate = _f32(x), _f32(w_gate)
+    b = None if b_gate is None else _f32(b_gate)
+    T, d = x.shape
+    E = w_gate.shape[0]
+    out = np.empty((T, E), dtype=np.float64)
+    lib().oracle_gate_logits(_p(x), _p(w_gate), _p(b), C.c_int(T), C.c_int(d), C.c_int(E), _p(out))
+    return out
+
+
+def topk(logits: np.ndarray, k: int):
+    logits = np.ascontiguousarray(logits, dtype=np.float64)
+    T, E = logits.shape
+    assert 1 <= k <= E
+    idx = np.empty((T, k), dtype=np.int32)
+    p = np.empty((T, k), dtype=np.float64)
+    lib().oracle_topk(_p(logits), C.c_int(T), C.c_int(E), C.c_int(k), _p(idx), _p(p))
+    return idx, p
+
+
+def tables(topk_idx: np.ndarray, E: int):
+    topk_idx = np.ascontiguousarray(topk_idx, dtype=np.int32)
+    T, k = topk_idx.shape
+    counts = np.empty(E, dtype=np.int32)
+    offsets = np.empty(E + 1, dtype=np.int32)
+    row_of_slot = np.empty(T * k, dtype=np.int32)
+    slot_of_row = np.empty(T * k, dtype=np.int32)
+    lib().oracle_tables(_p(topk_idx), C.c_int(T), C.c_int(k), C.c_int(E), _p(counts), _p(offsets),
+                        _p(row_of_slot), _p(slot_of_row))
+    return counts, offsets, row_of_slot, slot_of_row
+
+
+def route(inp: Dict[str, np.ndarray], k: int) -> Routing:
+    logits = gate_logits(inp["x"], inp["w_gate"], inp.get("b_gate"))
+    idx, p = topk(logits, k)
+    counts, offsets, ros, sor = tables(idx, logits.shape[1])
+    return Routing(logits, idx, p, counts, offsets, ros, sor)
+
+
+def _dims(inp):
+    T, d = inp["x"].shape
+    E, h, r = inp["w1"].shape
+    return T, d, r, h, E
+
+
+def _tokens(tokens, T):
+    if tokens is None:
+        return None, T
+    tok = np.ascontiguousarray(tokens, dtype=np.int32)
+    assert tok.ndim == 1 and (tok.size == 0 or (tok.min() >= 0 and tok.max() < T))
+    return tok, tok.size
+
+
+def forward_tokens(inp, routing: Routing, act: int, tokens=None, want_slots: bool = False):
+    """Per-token evaluation of Eq. 2.  Returns x_lo [n,r], y_lo [n,r], y [n,d] (+ z [n,k,h], u [n,k,r])."""
+    T, d, r, h, E = _dims(inp)
+    k = routing.topk_idx.shape[1]
+    tok, n = _tokens(tokens, T)
+    x_lo = np.empty((n, r)); y_lo = np.empty((n, r)); y = np.empty((n, d))
+    z = np.empty((n, k, h)) if want_slots else None
+    u = np.empty((n, k, r)) if want_slots else None
+    lib().oracle_forward_tokens(_p(_f32(inp["x"])), _p(_f32(inp["w_down"])), _p(_f32(inp["w1"])),
+                                _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])), _p(routing.topk_idx),
+                                _p(routing.topk_p), _p(tok), C.c_int(n), C.c_int(d), C.c_int(r), C.c_int(h),
+                                C.c_int(E), C.c_int(k), C.c_int(act), _p(x_lo), _p(y_lo), _p(y), _p(z), _p(u))
+    out = {"x_lo": x_lo, "y_lo": y_lo, "y": y}
+    if want_slots:
+        out["z"], out["u"] = z, u
+    return out
+
+
+def forward_grouped(inp, routing: Routing, act: int):
+    """Dispatch / per-expert segments / combine evaluation; must equal forward_tokens."""
+    T, d, r, h, E = _dims(inp)
+    k = routing.topk_idx.shape[1]
+    xg = np.empty((T * k, r)); y_lo = np.empty((T, r)); y = np.empty((T, d))
+    lib().oracle_forward_grouped(_p(_f32(inp["x"])), _p(_f32(inp["w_down"])), _p(_f32(inp["w1"])),
+                                 _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])), _p(routing.topk_p),
+                                 _p(routing.offsets), _p(routing.row_of_slot), _p(routing.slot_of_row),
+                                 C.c_int(T), C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(E), C.c_int(k),
+                                 C.c_int(act), _p(xg), _p(y_lo), _p(y))
+    return {"xg": xg, "y_lo": y_lo, "y": y}
+
+
+def backward_tokens(inp, routing: Routing, act: int, tokens=None):
+    """Per-token gradients of L = sum(y*dy): dx [n,d], dx_lo [n,r], dlogit [n,k] (top-k slots), dy_lo [n,r]."""
+    T, d, r, h, E = _dims(inp)
+    k = routing.topk_idx.shape[1]
+    tok, n = _tokens(tokens, T)
+    dx = np.empty((n, d)); dx_lo = np.empty((n, r)); dlogit = np.empty((n, k)); dy_lo = np.empty((n, r))
+    lib().oracle_backward_tokens(_p(_f32(inp["x"])), _p(_f32(inp["dy"])), _p(_f32(inp["w_gate"])),
+                                 _p(_f32(inp["w_down"])), _p(_f32(inp["w1"])), _p(_f32(inp["w2"])),
+                                 _p(_f32(inp["w_up"])), _p(routing.topk_idx), _p(routing.topk_p), _p(tok),
+                                 C.c_int(n), C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(E), C.c_int(k),
+                                 C.c_int(act), _p(dx), _p(dx_lo), _p(dlogit), _p(dy_lo))
+    return {"dx": dx, "dx_lo": dx_lo, "dlogit": dlogit, "dy_lo": dy_lo}
+
+
+def backward_expert(inp, routing: Routing, act: int, e: int):
+    """dW1[e] [h,r] and dW2[e] [r,h], summed over the rows of expert e's segment."""
+    T, d, r, h, E = _dims(inp)
+    k = routing.topk_idx.shape[1]
+    dw1 = np.empty((h, r)); dw2 = np.empty((r, h))
+    lib().oracle_backward_expert(_p(_f32(inp["x"])), _p(_f32(inp["dy"])), _p(_f32(inp["w_down"])),
+                                 _p(_f32(inp["w1"])), _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])),
+                                 _p(routing.topk_p), _p(routing.offsets), _p(routing.slot_of_row), C.c_int(e),
+                                 C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(k), C.c_int(act), _p(dw1), _p(dw2))
+    return dw1, dw2
+
+
+def backward_full(inp, routing: Routing, act: int, experts=None):
+    """All gradients: dx and every weight gradient (dw1/dw2 for `experts`, default all)."""
+    T, d, r, h, E = _dims(inp)
+    k = routing.topk_idx.shape[1]
+    fwd = forward_tokens(inp, routing, act)
+    bwd = backward_tokens(inp, routing, act)
+    dw_up = np.empty((d, r)); dw_down = np.empty((r, d)); dw_gate = np.empty((E, d)); db_gate = np.empty(E)
+    lib().oracle_backward_shared(_p(_f32(inp["x"])), _p(_f32(inp["dy"])), _p(fwd["y_lo"]), _p(bwd["dx_lo"]),
+                                 _p(routing.topk_idx), _p(bwd["dlogit"]), C.c_int(T), C.c_int(d), C.c_int(r),
+                                 C.c_int(E), C.c_int(k), _p(dw_up), _p(dw_down), _p(dw_gate), _p(db_gate))
+    experts = range(E) if experts is None else experts
+    dw1, dw2 = {}, {}
+    for e in experts:
+        dw1[e], dw2[e] = backward_expert(inp, routing, act, e)
+    out = {"y": fwd["y"], "y_lo": fwd["y_lo"], "x_lo": fwd["x_lo"], "dx": bwd["dx"], "dx_lo": bwd["dx_lo"],
+           "dlogit": bwd["dlogit"], "dw_up": dw_up, "dw_down": dw_down, "dw_gate": dw_gate,
+           "db_gate": db_gate, "dw1": dw1, "dw2": dw2}
+    return out
+
+
+def rel_err(a, b) -> float:
+    """max_i |a_i - b_i| / max(|b_i|, rms(b)): elementwise relative error with the denominator
+    floored at the reference tensor's RMS, so near-zero elements do not dominate."""
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    if b.size == 0:
+        return 0.0
+    rms = float(np.sqrt(np.mean(b * b)))
+    if rms == 0.0:
+        return float(np.max(np.abs(a))) if a.size else 0.0
+    return float(np.max(np.abs(a - b) / np.maximum(np.abs(b), rms)))

@@ -1,0 +1,356 @@
+// CPU oracle for the BigMac DCCA Mixture-of-Experts layer.  TEST INFRASTRUCTURE ONLY.
+//
+// A plain, slow, per-token / per-row evaluation in fp64 of what the layer computes, written
+// from the paper's equations.  It shares no code with the CUDA library and must never sit on
+// the product path: only the tests, the smoke check and the benchmark's CPU-baseline leg call it.
+//
+// The layer (Eq. 2 with the BigMac expert of Eq. 4; the gate reads the full-width token x, as the
+// text after Eq. 2 chooses):
+//     x' = x W'_down ;   y' = sum_{i in T} p_i(x) E_i(x') ;   y = y' W'_up ;
+//     E_i(v) = sigma(v W_{i,up}) W_{i,down}
+// Storage convention: every weight is [out_features, in_features], row-major, so "v W" above is
+// out[o] = sum_i v[i] * W[o][i].  Names: w_down [r,d], w1 = W_{i,up} [E,h,r], w2 = W_{i,down} [E,r,h],
+// w_up [d,r], w_gate [E,d], b_gate [E] (optional).
+//
+// Readings where the paper is silent (all listed in the design notes): linear gate; top-k by
+// (logit descending, expert id ascending); gate weights = softmax over the k selected logits;
+// dropless routing; no biases except the optional gate bias; rows of an expert's segment in
+// ascending slot id (slot s = t*k + j).
+//
+// Inputs are float arrays holding values exactly representable in the workload dtype; they are
+// widened to double before any arithmetic and nothing is rounded afterwards.
+//
+// Parity pins (tests, CPU only): top-k against a full library sort, gate weights against a library
+// softmax, tables against a library stable argsort and a brute-force count, E=1/k=1 and
+// shared-expert special cases against a 4-matmul MLP, identity-expert case against the two
+// projections alone, per-token against grouped evaluation, gradients against central finite
+// differences and the adjoint identity.  Float values of y and of the gradients on random data
+// have no printed example in the paper: "parity unpinned" by the paper for those, pinned only by
+// the special cases above.
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <numeric>
+#include <vector>
+
+namespace {
+
+enum { ACT_RELU = 0, ACT_GELU_ERF = 1, ACT_GELU_TANH = 2, ACT_IDENTITY = 3 };
+
+const double kSqrt2 = 1.41421356237309504880;
+const double kSqrt2OverPi = 0.79788456080286535588;
+const double kInvSqrt2Pi = 0.39894228040143267794;
+
+// sigma of Eq. 4.
+double act_f(int act, double z) {
+    switch (act) {
+        case ACT_RELU: return z > 0.0 ? z : 0.0;
+        case ACT_GELU_ERF: return 0.5 * z * (1.0 + std::erf(z / kSqrt2));
+        case ACT_GELU_TANH: return 0.5 * z * (1.0 + std::tanh(kSqrt2OverPi * (z + 0.044715 * z * z * z)));
+        default: return z;
+    }
+}
+
+// d sigma / dz.  ReLU' is 0 at z = 0.
+double act_df(int act, double z) {
+    switch (act) {
+        case ACT_RELU: return z > 0.0 ? 1.0 : 0.0;
+        case ACT_GELU_ERF: {
+            double Phi = 0.5 * (1.0 + std::erf(z / kSqrt2));
+            double phi = kInvSqrt2Pi * std::exp(-0.5 * z * z);
+            return Phi + z * phi;
+        }
+        case ACT_GELU_TANH: {
+            double w = kSqrt2OverPi * (z + 0.044715 * z * z * z);
+            double th = std::tanh(w);
+            double dw = kSqrt2OverPi * (1.0 + 3.0 * 0.044715 * z * z);
+            return 0.5 * (1.0 + th) + 0.5 * z * (1.0 - th * th) * dw;
+        }
+        default: return 1.0;
+    }
+}
+
+// out[o] = sum_i v[i] * W[o][i]      (W is [n_out, n_in] floats, widened per element)
+void matvec(const double* v, const float* W, int n_out, int n_in, double* out) {
+    for (int o = 0; o < n_out; ++o) {
+        const float* row = W + (size_t)o * n_in;
+        double acc = 0.0;
+        for (int i = 0; i < n_in; ++i) acc += v[i] * (double)row[i];
+        out[o] = acc;
+    }
+}
+
+// out[i] = sum_o g[o] * W[o][i]      (the transpose product, for gradients w.r.t. the input)
+void matvec_t(const double* g, const float* W, int n_out, int n_in, double* out) {
+    for (int i = 0; i < n_in; ++i) out[i] = 0.0;
+    for (int o = 0; o < n_out; ++o) {
+        const float* row = W + (size_t)o * n_in;
+        double go = g[o];
+        for (int i = 0; i < n_in; ++i) out[i] += go * (double)row[i];
+    }
+}
+
+void widen(const float* src, int n, double* dst) {
+    for (int i = 0; i < n; ++i) dst[i] = (double)src[i];
+}
+
+// One routed slot of one token through expert e (Eq. 4):  z = x' W1_e^T, a = sigma(z), u = a W2_e^T.
+void expert_forward(const double* x_lo, const float* w1_e, const float* w2_e, int r, int h, int act,
+                    double* z, double* a, double* u) {
+    matvec(x_lo, w1_e, h, r, z);
+    for (int q = 0; q < h; ++q) a[q] = act_f(act, z[q]);
+    matvec(a, w2_e, r, h, u);
+}
+
+}  // namespace
+
+extern "C" {
+
+// Gate logits: l[t,e] = sum_c x[t,c] W_g[e,c] (+ b_g[e]).  The gate reads x, not x' (text after Eq. 2).
+void oracle_gate_logits(const float* x, const float* w_gate, const float* b_gate, int T, int d, int E,
+                        double* logits) {
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < T; ++t) {
+        std::vector<double> xt(d);
+        widen(x + (size_t)t * d, d, xt.data());
+        matvec(xt.data(), w_gate, E, d, logits + (size_t)t * E);
+        if (b_gate)
+            for (int e = 0; e < E; ++e) logits[(size_t)t * E + e] += (double)b_gate[e];
+    }
+}
+
+// Top-k set T of Eq. 2 and the gate values p_i: experts ordered by (logit descending, id ascending),
+// first k kept in that order; p = softmax over the k kept logits (so the p of a token sum to 1).
+void oracle_topk(const double* logits, int T, int E, int k, int32_t* topk_idx, double* topk_p) {
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < T; ++t) {
+        const double* l = logits + (size_t)t * E;
+        std::vector<int> order(E);
+        std::iota(order.begin(), order.end(), 0);
+        std::stable_sort(order.begin(), order.end(), [l](int a, int b) { return l[a] > l[b]; });
+        double m = l[order[0]], denom = 0.0;
+        for (int j = 0; j < k; ++j) denom += std::exp(l[order[j]] - m);
+        for (int j = 0; j < k; ++j) {
+            topk_idx[(size_t)t * k + j] = order[j];
+            topk_p[(size_t)t * k + j] = std::exp(l[order[j]] - m) / denom;
+        }
+    }
+}
+
+// Dropless dispatch layout (the on-device stand-in for the first All-to-All): a stable counting sort
+// of slot ids s = t*k + j by expert id.
+void oracle_tables(const int32_t* topk_idx, int T, int k, int E, int32_t* counts, int32_t* offsets,
+                   int32_t* row_of_slot, int32_t* slot_of_row) {
+    const int64_t N = (int64_t)T * k;
+    for (int e = 0; e < E; ++e) counts[e] = 0;
+    for (int64_t s = 0; s < N; ++s) counts[topk_idx[s]] += 1;
+    offsets[0] = 0;
+    for (int e = 0; e < E; ++e) offsets[e + 1] = offsets[e] + counts[e];
+    std::vector<int32_t> seen(E, 0);   // slots already placed per expert = #{s' < s : idx[s'] = e}
+    for (int64_t s = 0; s < N; ++s) {
+        int e = topk_idx[s];
+        int32_t row = offsets[e] + seen[e];
+        seen[e] += 1;
+        row_of_slot[s] = row;
+        slot_of_row[row] = (int32_t)s;
+    }
+}
+
+// Forward, token by token, exactly as Eq. 2 is written.  `tokens` selects n token ids (NULL = 0..n-1).
+// Outputs are indexed by position in `tokens`.  z_out / u_out may be NULL.
+void oracle_forward_tokens(const float* x, const float* w_down, const float* w1, const float* w2,
+                           const float* w_up, const int32_t* topk_idx, const double* topk_p,
+                           const int32_t* tokens, int n, int d, int r, int h, int E, int k, int act,
+                           double* x_lo_out, double* y_lo_out, double* y_out, double* z_out, double* u_out) {
+    (void)E;
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int i = 0; i < n; ++i) {
+        const int t = tokens ? tokens[i] : i;
+        std::vector<double> xt(d), x_lo(r), z(h), a(h), u(r), y_lo(r, 0.0);
+        widen(x + (size_t)t * d, d, xt.data());
+        matvec(xt.data(), w_down, r, d, x_lo.data());                       // x' = x W'_down
+        for (int j = 0; j < k; ++j) {                                       // sum over i in T
+            const int e = topk_idx[(size_t)t * k + j];
+            const double p = topk_p[(size_t)t * k + j];
+            expert_forward(x_lo.data(), w1 + (size_t)e * h * r, w2 + (size_t)e * r * h, r, h, act,
+                           z.data(), a.data(), u.data());
+            for (int c = 0; c < r; ++c) y_lo[c] += p * u[c];               // p_i(x) E_i(x')
+            if (z_out) std::memcpy(z_out + ((size_t)i * k + j) * h, z.data(), sizeof(double) * h);
+            if (u_out) std::memcpy(u_out + ((size_t)i * k + j) * r, u.data(), sizeof(double) * r);
+        }
+        if (x_lo_out) std::memcpy(x_lo_out + (size_t)i * r, x_lo.data(), sizeof(double) * r);
+        if (y_lo_out) std::memcpy(y_lo_out + (size_t)i * r, y_lo.data(), sizeof(double) * r);
+        if (y_out) matvec(y_lo.data(), w_up, d, r, y_out + (size_t)i * d);  // y = y' W'_up
+    }
+}
+
+// Forward the way a dispatching implementation evaluates it: descend all tokens, gather the r-wide
+// rows into expert segments (dispatch), run every expert over its segment, combine by slot with the
+// gate weights, ascend.  Must agree with oracle_forward_tokens; it also exercises the tables.
+void oracle_forward_grouped(const float* x, const float* w_down, const float* w1, const float* w2,
+                            const float* w_up, const double* topk_p, const int32_t* offsets,
+                            const int32_t* row_of_slot, const int32_t* slot_of_row, int T, int d, int r,
+                            int h, int E, int k, int act, double* xg_out, double* y_lo_out, double* y_out) {
+    const int64_t N = (int64_t)T * k;
+    std::vector<double> x_lo((size_t)T * r), xg((size_t)N * r), ug((size_t)N * r);
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < T; ++t) {
+        std::vector<double> xt(d);
+        widen(x + (size_t)t * d, d, xt.data());
+        matvec(xt.data(), w_down, r, d, &x_lo[(size_t)t * r]);
+    }
+    for (int64_t row = 0; row < N; ++row) {                                 // dispatch
+        const int t = slot_of_row[row] / k;
+        std::memcpy(&xg[(size_t)row * r], &x_lo[(size_t)t * r], sizeof(double) * r);
+    }
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int e = 0; e < E; ++e) {                                           // experts over segments
+        std::vector<double> z(h), a(h);
+        for (int row = offsets[e]; row < offsets[e + 1]; ++row)
+            expert_forward(&xg[(size_t)row * r], w1 + (size_t)e * h * r, w2 + (size_t)e * r * h, r, h, act,
+                           z.data(), a.data(), &ug[(size_t)row * r]);
+    }
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < T; ++t) {                                           // combine + ascend
+        std::vector<double> y_lo(r, 0.0);
+        for (int j = 0; j < k; ++j) {
+            const int64_t s = (int64_t)t * k + j;
+            const double p = topk_p[s];
+            const double* u = &ug[(size_t)row_of_slot[s] * r];
+            for (int c = 0; c < r; ++c) y_lo[c] += p * u[c];
+        }
+        if (y_lo_out) std::memcpy(y_lo_out + (size_t)t * r, y_lo.data(), sizeof(double) * r);
+        if (y_out) matvec(y_lo.data(), w_up, d, r, y_out + (size_t)t * d);
+    }
+    if (xg_out) std::memcpy(xg_out, xg.data(), sizeof(double) * xg.size());
+}
+
+// Backward of the scalar L = sum(y * dy), token by token (chain rule through Eq. 2 / Eq. 4; the
+// discrete top-k choice carries no gradient, the gate weights do).  Per selected token i (id t):
+//   dy' = dy W_up ; per slot j: dp_j = <dy', u_j>, du_j = p_j dy', da_j = du_j W2, dz_j = da_j * sigma'(z_j),
+//   dx' = sum_j dz_j W1 ; softmax-over-k: g = sum_i p_i dp_i, dl_j = p_j (dp_j - g) ;
+//   dx = dx' W_down + sum_j dl_j W_g[e_j].
+// Outputs (any may be NULL) are indexed by position in `tokens`.
+void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate, const float* w_down,
+                            const float* w1, const float* w2, const float* w_up, const int32_t* topk_idx,
+                            const double* topk_p, const int32_t* tokens, int n, int d, int r, int h, int E,
+                            int k, int act, double* dx_out, double* dx_lo_out, double* dlogit_out,
+                            double* dy_lo_out) {
+    (void)E;
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int i = 0; i < n; ++i) {
+        const int t = tokens ? tokens[i] : i;
+        std::vector<double> xt(d), dyt(d), x_lo(r), dy_lo(r), z(h), a(h), u(r), du(r), da(h), dz(h), tmp(r),
+            dx_lo(r, 0.0), dp(k), dl(k), dx(d), gate_part(d, 0.0);
+        widen(x + (size_t)t * d, d, xt.data());
+        widen(dy + (size_t)t * d, d, dyt.data());
+        matvec(xt.data(), w_down, r, d, x_lo.data());
+        matvec_t(dyt.data(), w_up, d, r, dy_lo.data());
+        for (int j = 0; j < k; ++j) {
+            const int e = topk_idx[(size_t)t * k + j];
+            const double p = topk_p[(size_t)t * k + j];
+            const float* w1_e = w1 + (size_t)e * h * r;
+            const float* w2_e = w2 + (size_t)e * r * h;
+            expert_forward(x_lo.data(), w1_e, w2_e, r, h, act, z.data(), a.data(), u.data());
+            double acc = 0.0;
+            for (int c = 0; c < r; ++c) acc += dy_lo[c] * u[c];
+            dp[j] = acc;
+            for (int c = 0; c < r; ++c) du[c] = p * dy_lo[c];
+            matvec_t(du.data(), w2_e, r, h, da.data());
+            for (int q = 0; q < h; ++q) dz[q] = da[q] * act_df(act, z[q]);
+            matvec_t(dz.data(), w1_e, h, r, tmp.data());
+            for (int c = 0; c < r; ++c) dx_lo[c] += tmp[c];
+        }
+        double g = 0.0;
+        for (int j = 0; j < k; ++j) g += topk_p[(size_t)t * k + j] * dp[j];
+        for (int j = 0; j < k; ++j) dl[j] = topk_p[(size_t)t * k + j] * (dp[j] - g);
+        matvec_t(dx_lo.data(), w_down, r, d, dx.data());
+        for (int j = 0; j < k; ++j) {
+            const float* wg = w_gate + (size_t)topk_idx[(size_t)t * k + j] * d;
+            for (int c = 0; c < d; ++c) gate_part[c] += dl[j] * (double)wg[c];
+        }
+        for (int c = 0; c < d; ++c) dx[c] += gate_part[c];
+        if (dx_out) std::memcpy(dx_out + (size_t)i * d, dx.data(), sizeof(double) * d);
+        if (dx_lo_out) std::memcpy(dx_lo_out + (size_t)i * r, dx_lo.data(), sizeof(double) * r);
+        if (dlogit_out) std::memcpy(dlogit_out + (size_t)i * k, dl.data(), sizeof(double) * k);
+        if (dy_lo_out) std::memcpy(dy_lo_out + (size_t)i * r, dy_lo.data(), sizeof(double) * r);
+    }
+}
+
+// Weight gradients of one expert e over its segment of rows [offsets[e], offsets[e+1]):
+//   dW2_e[c,q] = sum_rows du[c] a[q] ;  dW1_e[q,c] = sum_rows dz[q] x'[c].
+// An expert that received no rows gets exactly zero gradients.
+void oracle_backward_expert(const float* x, const float* dy, const float* w_down, const float* w1,
+                            const float* w2, const float* w_up, const double* topk_p, const int32_t* offsets,
+                            const int32_t* slot_of_row, int e, int d, int r, int h, int k, int act,
+                            double* dw1_e, double* dw2_e) {
+    std::fill(dw1_e, dw1_e + (size_t)h * r, 0.0);
+    std::fill(dw2_e, dw2_e + (size_t)r * h, 0.0);
+    const float* w1_e = w1 + (size_t)e * h * r;
+    const float* w2_e = w2 + (size_t)e * r * h;
+    std::vector<double> xt(d), dyt(d), x_lo(r), dy_lo(r), z(h), a(h), u(r), du(r), da(h), dz(h);
+    for (int row = offsets[e]; row < offsets[e + 1]; ++row) {
+        const int s = slot_of_row[row];
+        const int t = s / k;
+        const double p = topk_p[s];
+        widen(x + (size_t)t * d, d, xt.data());
+        widen(dy + (size_t)t * d, d, dyt.data());
+        matvec(xt.data(), w_down, r, d, x_lo.data());
+        matvec_t(dyt.data(), w_up, d, r, dy_lo.data());
+        expert_forward(x_lo.data(), w1_e, w2_e, r, h, act, z.data(), a.data(), u.data());
+        for (int c = 0; c < r; ++c) du[c] = p * dy_lo[c];
+        matvec_t(du.data(), w2_e, r, h, da.data());
+        for (int q = 0; q < h; ++q) dz[q] = da[q] * act_df(act, z[q]);
+        for (int c = 0; c < r; ++c)
+            for (int q = 0; q < h; ++q) dw2_e[(size_t)c * h + q] += du[c] * a[q];
+        for (int q = 0; q < h; ++q)
+            for (int c = 0; c < r; ++c) dw1_e[(size_t)q * r + c] += dz[q] * x_lo[c];
+    }
+}
+
+// Gradients of the shared matrices, as sums over all tokens of outer products of per-token vectors
+// (which the caller obtains from oracle_forward_tokens / oracle_backward_tokens):
+//   dW_up[c,c'] = sum_t dy[t,c] y'[t,c'] ;  dW_down[c',c] = sum_t dx'[t,c'] x[t,c] ;
+//   dW_g[e,c]   = sum_t dl[t,e] x[t,c]   ;  db_g[e]      = sum_t dl[t,e]   (dl is zero off the top-k set).
+void oracle_backward_shared(const float* x, const float* dy, const double* y_lo, const double* dx_lo,
+                            const int32_t* topk_idx, const double* dlogit, int T, int d, int r, int E, int k,
+                            double* dw_up, double* dw_down, double* dw_gate, double* db_gate) {
+#pragma omp parallel for schedule(static)
+    for (int c = 0; c < d; ++c) {
+        double* out = dw_up + (size_t)c * r;
+        for (int cc = 0; cc < r; ++cc) out[cc] = 0.0;
+        for (int t = 0; t < T; ++t) {
+            const double g = (double)dy[(size_t)t * d + c];
+            const double* yl = y_lo + (size_t)t * r;
+            for (int cc = 0; cc < r; ++cc) out[cc] += g * yl[cc];
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (int cc = 0; cc < r; ++cc) {
+        double* out = dw_down + (size_t)cc * d;
+        for (int c = 0; c < d; ++c) out[c] = 0.0;
+        for (int t = 0; t < T; ++t) {
+            const double g = dx_lo[(size_t)t * r + cc];
+            const float* xt = x + (size_t)t * d;
+            for (int c = 0; c < d; ++c) out[c] += g * (double)xt[c];
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (int e = 0; e < E; ++e) {
+        double* out = dw_gate + (size_t)e * d;
+        for (int c = 0; c < d; ++c) out[c] = 0.0;
+        double bsum = 0.0;
+        for (int t = 0; t < T; ++t)
+            for (int j = 0; j < k; ++j) {
+                if (topk_idx[(size_t)t * k + j] != e) continue;
+                const double g = dlogit[(size_t)t * k + j];
+                const float* xt = x + (size_t)t * d;
+                for (int c = 0; c < d; ++c) out[c] += g * (double)xt[c];
+                bsum += g;
+            }
+        if (db_gate) db_gate[e] = bsum;
+    }
+}
+
+}  // extern "C"
