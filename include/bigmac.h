@@ -1,0 +1,169 @@
+/* bigmac.h - C ABI of the BigMac DCCA Mixture-of-Experts layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer (paper, Eq. 2, with the BigMac expert of Eq. 4; the gate reads the full-width token x,
+ * as the text following Eq. 2 chooses):
+ *
+ *     x' = x W'_down ;   y' = sum_{i in T} p_i(x) E_i(x') ;   y = y' W'_up ;
+ *     E_i(v) = sigma(v W_{i,up}) W_{i,down}
+ *
+ * T is the set of the top_k experts of the token, p_i its gate values.  Tokens travel between the
+ * shared projections and the experts at the low width r; on one GPU the two All-to-All exchanges of
+ * Fig. 2c become a dispatch into expert-grouped row segments and a gate-weighted combine back to
+ * token order.  Routing is dropless (section "Enabling Dropless Token Routing"): every token reaches
+ * exactly k experts and segments have variable length.
+ *
+ * Symbols (paper's Table 2 in brackets): T tokens [b*s], d model width [h], r low width [r*h],
+ * h expert hidden width, E experts [e], k experts per token [top_k], N = T*k routed rows.
+ *
+ * Conventions
+ *  - Every tensor pointer is CALLER-OWNED DEVICE memory, 16-byte aligned, row-major, dense, and is
+ *    borrowed only for the stream-ordered duration of the call.  Configuration structs and the
+ *    output-size pointers are HOST memory.
+ *  - Weights are stored [out_features, in_features] (the contraction index is contiguous):
+ *    w_gate [E,d], w_down [r,d], w1 [E,h,r] (W_{i,up}), w2 [E,r,h] (W_{i,down}), w_up [d,r].
+ *  - dtype BIGMAC_F32: all float tensors are fp32 and all arithmetic is fp32 FMA.
+ *    dtype BIGMAC_BF16: x, y, dy, dx, weights, weight gradients and intermediates are bf16, products
+ *    accumulate in fp32 on the tensor cores; gate logits, gate weights and the gate bias stay fp32.
+ *    The BF16 path requires d, r and h to be multiples of 64.
+ *  - Where the paper is silent: the gate is linear, l = x w_gate^T (+ b_gate); the k experts are
+ *    chosen by (logit descending, expert id ascending); p is the softmax over the k chosen logits,
+ *    so the p of one token sum to 1; there are no biases other than the optional gate bias.
+ *  - The library never allocates device memory in route/forward/backward, never synchronises the
+ *    stream (bigmac_device_status excepted) and launches everything on the stream passed in
+ *    (a cudaStream_t as void*).  One handle serves one stream at a time.
+ *  - Return value: BIGMAC_OK (0) or a negative bigmac_status_t.  On an argument error nothing is
+ *    launched.  Nothing throws, aborts or traps; problems detected on the device (a bounded wait that
+ *    ran out) are recorded in a status word read by bigmac_device_status.
+ */
+#ifndef BIGMAC_H_
+#define BIGMAC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bigmac_layer bigmac_layer_t; /* opaque, library-owned */
+
+typedef enum {
+    BIGMAC_OK = 0,
+    BIGMAC_ERR_INVALID_ARG = -1,
+    BIGMAC_ERR_UNSUPPORTED = -2,
+    BIGMAC_ERR_WORKSPACE = -3,
+    BIGMAC_ERR_CUDA = -4,
+    BIGMAC_ERR_TIMEOUT = -5,
+    BIGMAC_ERR_STATE = -6
+} bigmac_status_t;
+
+typedef enum { BIGMAC_F32 = 0, BIGMAC_BF16 = 1 } bigmac_dtype_t;
+
+/* sigma of Eq. 4.  GELU_ERF: z/2 (1 + erf(z/sqrt 2)); GELU_TANH: the tanh approximation with
+ * coefficient 0.044715; IDENTITY exists for tests. */
+typedef enum {
+    BIGMAC_ACT_RELU = 0,
+    BIGMAC_ACT_GELU_ERF = 1,
+    BIGMAC_ACT_GELU_TANH = 2,
+    BIGMAC_ACT_IDENTITY = 3
+} bigmac_act_t;
+
+/* flags */
+#define BIGMAC_FLAG_SIMT_GEMM 1u /* BF16 only: run every contraction on the plain FMA kernels (debug aid) */
+
+typedef struct {
+    int32_t d, r, h, E, k; /* 1 <= k <= E */
+    int32_t max_tokens;    /* largest T any call will pass */
+    int32_t dtype;         /* bigmac_dtype_t */
+    int32_t act;           /* bigmac_act_t */
+    uint32_t flags;
+} bigmac_config_t;
+
+typedef struct {
+    const void *w_gate;   /* [E,d]   */
+    const float *b_gate;  /* [E] fp32, or NULL */
+    const void *w_down;   /* [r,d]   W'_down of Eq. 2 */
+    const void *w1;       /* [E,h,r] W_{i,up} of Eq. 4 */
+    const void *w2;       /* [E,r,h] W_{i,down} of Eq. 4 */
+    const void *w_up;     /* [d,r]   W'_up of Eq. 2 */
+} bigmac_weights_t;
+
+/* Gradient buffers, same shapes and dtype as the weights; db_gate fp32 [E] or NULL. */
+typedef struct {
+    void *dw_gate;
+    float *db_gate;
+    void *dw_down, *dw1, *dw2, *dw_up;
+} bigmac_grads_t;
+
+/* Routing tables.  Flat slot id s = t*k + j (j-th choice of token t).
+ *   topk_idx[s]    expert of slot s, slots of a token in descending-logit order
+ *   topk_w[s]      gate value p of slot s (fp32)
+ *   counts[e]      rows routed to expert e;  offsets = exclusive prefix sum, offsets[E] = T*k
+ *   row_of_slot[s] = offsets[e] + #{s' < s : topk_idx[s'] = e}  (stable counting sort by expert)
+ *   slot_of_row    its inverse
+ * Any member may be NULL if the caller does not want that table. */
+typedef struct {
+    int32_t *topk_idx;    /* [T*k] */
+    float *topk_w;        /* [T*k] */
+    int32_t *counts;      /* [E]   */
+    int32_t *offsets;     /* [E+1] */
+    int32_t *row_of_slot; /* [T*k] */
+    int32_t *slot_of_row; /* [T*k] */
+} bigmac_routing_t;
+
+/* Validate the configuration and create a handle on the current CUDA device.  Allocates one small
+ * device status word; no other device memory is owned by the handle.
+ * Errors: INVALID_ARG (null pointers, non-positive sizes, k > E, unknown enums), UNSUPPORTED (BF16
+ * with d, r or h not a multiple of 64; E > 1024), CUDA. */
+int bigmac_layer_create(const bigmac_config_t *cfg, bigmac_layer_t **out);
+int bigmac_layer_destroy(bigmac_layer_t *L);
+
+/* Bytes the caller must provide for a call with T tokens: `scratch_bytes` of scratch (contents
+ * undefined before and after a call) and, for a training forward and its backward, `saved_bytes`
+ * of saved state.  Both pointers must be 256-byte aligned.  training: 0 = inference forward,
+ * 1 = training forward / backward. */
+int bigmac_workspace_bytes(const bigmac_layer_t *L, int32_t T, int training, size_t *scratch_bytes,
+                           size_t *saved_bytes);
+
+/* Routing only: gate logits on x (text after Eq. 2), top-k, gate values, and the dispatch layout that
+ * stands in for the first All-to-All (dropless).  x [T,d].  Integer tables have exactly one correct
+ * value.  T = 0 is a no-op. */
+int bigmac_route(bigmac_layer_t *L, const void *x, int32_t T, const bigmac_weights_t *W,
+                 bigmac_routing_t *out, void *scratch, size_t scratch_bytes, void *stream);
+
+/* Forward of Eq. 2 / Eq. 4: y [T,d] from x [T,d].  routing_out (nullable) receives the tables.
+ * saved = NULL runs the inference forward; otherwise `saved` (saved_bytes of the training query)
+ * receives what bigmac_backward needs. */
+int bigmac_forward(bigmac_layer_t *L, const void *x, int32_t T, const bigmac_weights_t *W, void *y,
+                   bigmac_routing_t *routing_out, void *saved, void *scratch, size_t scratch_bytes,
+                   void *stream);
+
+/* Backward of the same layer for an upstream gradient dy [T,d] (chain rule through Eq. 2 / Eq. 4):
+ * dx [T,d] (through both the projections and the gate weights; the discrete top-k choice carries no
+ * gradient) and every weight gradient in G (members may be NULL to skip one).  `x`, `W`, `T` and
+ * `saved` must be those of the training forward.  accumulate = 0 overwrites the gradients (experts
+ * that received no token get zeros), 1 adds to them.  `saved` may be modified. */
+int bigmac_backward(bigmac_layer_t *L, const void *x, const void *dy, int32_t T, const bigmac_weights_t *W,
+                    void *saved, void *dx, const bigmac_grads_t *G, int accumulate, void *scratch,
+                    size_t scratch_bytes, void *stream);
+
+/* Synchronise `stream` and return the device status word (BIGMAC_OK, or BIGMAC_ERR_TIMEOUT if a
+ * bounded wait inside a kernel ran out, in which case outputs of that call are undefined).  The word
+ * is cleared by the call. */
+int bigmac_device_status(bigmac_layer_t *L, void *stream);
+
+const char *bigmac_status_string(int status);
+
+/* Measurement aid for the dispatch/combine stage (Eq. 1: bytes through the exchange are proportional
+ * to the row width): run the standalone dispatch and combine kernels on rows of `width` elements of
+ * the layer's dtype.  width = r is BigMac's exchange; width = d is what a fine-grained layer of equal
+ * E and k moves.  src [T,width] -> grouped [rows_padded,width] -> dst [T,width] with the gate values
+ * of the routing held in `saved` (from a training forward of the same T).  which: 0 = dispatch only,
+ * 1 = combine only (grouped must hold data), 2 = both. */
+int bigmac_exchange_rows(bigmac_layer_t *L, const void *saved, int32_t T, int32_t width, const void *src,
+                         void *grouped, size_t grouped_bytes, void *dst, int which, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BIGMAC_H_ */

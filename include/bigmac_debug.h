@@ -1,0 +1,36 @@
+/* bigmac_debug.h - unit-test entry point of libbigmac: run ONE contraction of the layer in isolation.
+ * Not needed to use the layer.  The paper has no counterpart; the contractions it implies are the
+ * matrix products of Eq. 2 and Eq. 4 and of their chain-rule gradients.
+ *
+ *   C[m,n] (+)= epilogue( sum_k A(m,k) * B(n,k) ),  fp32 accumulation
+ *   a_kmajor: A(m,k) = A[m*lda + k], else A[k*lda + m];  b_kmajor: B(n,k) = B[n*ldb + k], else B[k*ldb + n].
+ *   group 0: dense.  group 1: rows are expert-grouped segments padded to 128 rows, row tile i belongs to
+ *   expert tile_expert[i], only *n_tiles tiles exist, B of expert e at B + e*b_stride.  group 2: one
+ *   problem per expert with k running over rows [poffsets[e], poffsets[e+1]), C of expert e at C + e*c_stride.
+ *   epilogue 0: none; 1: Z = acc (if Z), C = sigma(acc); 2: C = acc * sigma'(Z).
+ * All pointers are device memory (tables included), 16-byte aligned.  use_tensor_cores = 1 requires a
+ * BF16 handle.  Returns a bigmac_status_t.
+ */
+#ifndef BIGMAC_DEBUG_H_
+#define BIGMAC_DEBUG_H_
+#include "bigmac.h"
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct {
+    const void *A, *B;
+    void *C, *Z;
+    int64_t lda, ldb, ldc;
+    int32_t M, N, K;
+    int32_t a_kmajor, b_kmajor, out_f32, accumulate, epilogue, act, group, num_experts;
+    int64_t b_stride, c_stride;
+    const int32_t *tile_expert, *n_tiles, *poffsets;
+} bigmac_debug_gemm_t;
+
+int bigmac_debug_gemm(bigmac_layer_t *L, const bigmac_debug_gemm_t *q, int use_tensor_cores, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BIGMAC_DEBUG_H_ */

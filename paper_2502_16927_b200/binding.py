@@ -1,0 +1,230 @@
+"""ctypes binding of libbigmac's C ABI (include/bigmac.h): same names, argument marshalling only.
+
+Every step of the layer runs inside the library's CUDA kernels; torch is used here for device
+memory and streams.  There is no fallback: if the shared library is missing or a call fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libbigmac.so")
+
+BIGMAC_OK = 0
+BIGMAC_F32, BIGMAC_BF16 = 0, 1
+BIGMAC_FLAG_SIMT_GEMM = 1
+
+
+class bigmac_config_t(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("d", "r", "h", "E", "k", "max_tokens", "dtype", "act")] + [("flags", C.c_uint32)]
+
+
+class bigmac_weights_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_gate", "b_gate", "w_down", "w1", "w2", "w_up")]
+
+
+class bigmac_grads_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("dw_gate", "db_gate", "dw_down", "dw1", "dw2", "dw_up")]
+
+
+class bigmac_routing_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("topk_idx", "topk_w", "counts", "offsets", "row_of_slot", "slot_of_row")]
+
+
+class bigmac_debug_gemm_t(C.Structure):
+    _fields_ = ([(n, C.c_void_p) for n in ("A", "B", "C", "Z")] + [(n, C.c_int64) for n in ("lda", "ldb", "ldc")] +
+                [(n, C.c_int32) for n in ("M", "N", "K", "a_kmajor", "b_kmajor", "out_f32", "accumulate", "epilogue",
+                                          "act", "group", "num_experts")] +
+                [(n, C.c_int64) for n in ("b_stride", "c_stride")] +
+                [(n, C.c_void_p) for n in ("tile_expert", "n_tiles", "poffsets")])
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """Load libbigmac.so (built in-tree by paper_2502_16927_b200/build.py); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2502_16927_b200.build` first")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+        L.bigmac_layer_create.argtypes = [C.POINTER(bigmac_config_t), C.POINTER(vp)]
+        L.bigmac_layer_destroy.argtypes = [vp]
+        L.bigmac_workspace_bytes.argtypes = [vp, i32, C.c_int, C.POINTER(sz), C.POINTER(sz)]
+        L.bigmac_route.argtypes = [vp, vp, i32, C.POINTER(bigmac_weights_t), C.POINTER(bigmac_routing_t), vp, sz, vp]
+        L.bigmac_forward.argtypes = [vp, vp, i32, C.POINTER(bigmac_weights_t), vp, C.POINTER(bigmac_routing_t), vp,
+                                     vp, sz, vp]
+        L.bigmac_backward.argtypes = [vp, vp, vp, i32, C.POINTER(bigmac_weights_t), vp, vp, C.POINTER(bigmac_grads_t),
+                                      C.c_int, vp, sz, vp]
+        L.bigmac_device_status.argtypes = [vp, vp]
+        L.bigmac_status_string.argtypes = [C.c_int]
+        L.bigmac_status_string.restype = C.c_char_p
+        L.bigmac_exchange_rows.argtypes = [vp, vp, i32, i32, vp, vp, sz, vp, C.c_int, vp]
+        L.bigmac_debug_gemm.argtypes = [vp, C.POINTER(bigmac_debug_gemm_t), C.c_int, vp]
+        for name in ("bigmac_layer_create", "bigmac_layer_destroy", "bigmac_workspace_bytes", "bigmac_route",
+                     "bigmac_forward", "bigmac_backward", "bigmac_device_status", "bigmac_exchange_rows",
+                     "bigmac_debug_gemm"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+class BigmacError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib().bigmac_status_string(status).decode()} ({status})")
+
+
+def _check(status: int, where: str) -> None:
+    if status != BIGMAC_OK:
+        raise BigmacError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors passed to libbigmac must be contiguous CUDA tensors"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+# ---- the C ABI, name for name -------------------------------------------------------------------------
+
+def bigmac_layer_create(d, r, h, E, k, max_tokens, dtype, act, flags=0) -> C.c_void_p:
+    cfg = bigmac_config_t(d, r, h, E, k, max_tokens, dtype, act, flags)
+    handle = C.c_void_p()
+    _check(lib().bigmac_layer_create(C.byref(cfg), C.byref(handle)), "bigmac_layer_create")
+    return handle
+
+
+def bigmac_layer_destroy(handle) -> None:
+    _check(lib().bigmac_layer_destroy(handle), "bigmac_layer_destroy")
+
+
+def bigmac_workspace_bytes(handle, T: int, training: bool):
+    s, v = C.c_size_t(), C.c_size_t()
+    _check(lib().bigmac_workspace_bytes(handle, T, int(training), C.byref(s), C.byref(v)), "bigmac_workspace_bytes")
+    return s.value, v.value
+
+
+def _weights(W: Dict[str, torch.Tensor]) -> bigmac_weights_t:
+    return bigmac_weights_t(_ptr(W["w_gate"]), _ptr(W.get("b_gate")), _ptr(W["w_down"]), _ptr(W["w1"]), _ptr(W["w2"]),
+                            _ptr(W["w_up"]))
+
+
+def _routing(R: Optional[Dict[str, torch.Tensor]]):
+    if R is None:
+        return None
+    return C.byref(bigmac_routing_t(*[_ptr(R.get(n)) for n in ("topk_idx", "topk_w", "counts", "offsets",
+                                                                  "row_of_slot", "slot_of_row")]))
+
+
+def bigmac_route(handle, x, T, W, routing, scratch) -> None:
+    _check(lib().bigmac_route(handle, _ptr(x), T, C.byref(_weights(W)), _routing(routing), _ptr(scratch),
+                              scratch.numel() * scratch.element_size(), _stream()), "bigmac_route")
+
+
+def bigmac_forward(handle, x, T, W, y, routing, saved, scratch) -> None:
+    _check(lib().bigmac_forward(handle, _ptr(x), T, C.byref(_weights(W)), _ptr(y), _routing(routing), _ptr(saved),
+                                _ptr(scratch), scratch.numel() * scratch.element_size(), _stream()), "bigmac_forward")
+
+
+def bigmac_backward(handle, x, dy, T, W, saved, dx, G, accumulate, scratch) -> None:
+    grads = bigmac_grads_t(*[_ptr(G.get(n)) for n in ("dw_gate", "db_gate", "dw_down", "dw1", "dw2", "dw_up")])
+    _check(lib().bigmac_backward(handle, _ptr(x), _ptr(dy), T, C.byref(_weights(W)), _ptr(saved), _ptr(dx),
+                                 C.byref(grads), int(accumulate), _ptr(scratch),
+                                 scratch.numel() * scratch.element_size(), _stream()), "bigmac_backward")
+
+
+def bigmac_device_status(handle) -> int:
+    return lib().bigmac_device_status(handle, _stream())
+
+
+def bigmac_exchange_rows(handle, saved, T, width, src, grouped, dst, which) -> None:
+    _check(lib().bigmac_exchange_rows(handle, _ptr(saved), T, width, _ptr(src), _ptr(grouped),
+                                      grouped.numel() * grouped.element_size(), _ptr(dst), which, _stream()),
+           "bigmac_exchange_rows")
+
+
+def bigmac_debug_gemm(handle, q: bigmac_debug_gemm_t, use_tensor_cores: bool) -> None:
+    _check(lib().bigmac_debug_gemm(handle, C.byref(q), int(use_tensor_cores), _stream()), "bigmac_debug_gemm")
+
+
+# ---- a small convenience wrapper: owns the handle and the workspaces ------------------------------------
+
+class Layer:
+    """One BigMac layer handle plus torch-allocated workspaces.  Marshalling only."""
+
+    def __init__(self, d, r, h, E, k, max_tokens, dtype, act, flags=0, device="cuda"):
+        self.cfg = dict(d=d, r=r, h=h, E=E, k=k, max_tokens=max_tokens, dtype=dtype, act=act, flags=flags)
+        self.device = torch.device(device)
+        with torch.cuda.device(self.device):
+            self.handle = bigmac_layer_create(d, r, h, E, k, max_tokens, dtype, act, flags)
+        self.tdtype = torch.bfloat16 if dtype == BIGMAC_BF16 else torch.float32
+        self._scratch = None
+        self._saved = None
+        self._T = None
+
+    def close(self):
+        if self.handle is not None:
+            bigmac_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _workspaces(self, T, training):
+        s, v = bigmac_workspace_bytes(self.handle, T, training)
+        if self._scratch is None or self._scratch.numel() < s:
+            self._scratch = torch.empty(max(s, 256), dtype=torch.uint8, device=self.device)
+        if training and (self._saved is None or self._saved.numel() < v):
+            self._saved = torch.empty(max(v, 256), dtype=torch.uint8, device=self.device)
+
+    def empty_routing(self, T):
+        E, k = self.cfg["E"], self.cfg["k"]
+        i32 = dict(dtype=torch.int32, device=self.device)
+        return {"topk_idx": torch.empty(T * k, **i32), "topk_w": torch.empty(T * k, dtype=torch.float32, device=self.device),
+                "counts": torch.empty(E, **i32), "offsets": torch.empty(E + 1, **i32),
+                "row_of_slot": torch.empty(T * k, **i32), "slot_of_row": torch.empty(T * k, **i32)}
+
+    def route(self, x, W):
+        T = x.shape[0]
+        self._workspaces(T, False)
+        R = self.empty_routing(T)
+        bigmac_route(self.handle, x, T, W, R, self._scratch)
+        return R
+
+    def forward(self, x, W, y=None, training=False, want_routing=False):
+        T = x.shape[0]
+        self._workspaces(T, training)
+        if y is None:
+            y = torch.empty_like(x)
+        R = self.empty_routing(T) if want_routing else None
+        bigmac_forward(self.handle, x, T, W, y, R, self._saved if training else None, self._scratch)
+        self._T = T if training else None
+        return (y, R) if want_routing else y
+
+    def backward(self, x, dy, W, G, dx=None, accumulate=False):
+        T = x.shape[0]
+        if self._T != T:
+            raise RuntimeError("backward needs a training forward of the same batch first")
+        if dx is None:
+            dx = torch.empty_like(x)
+        bigmac_backward(self.handle, x, dy, T, W, self._saved, dx, G, accumulate, self._scratch)
+        return dx
+
+    def status(self) -> int:
+        return bigmac_device_status(self.handle)

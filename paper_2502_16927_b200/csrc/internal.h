@@ -1,0 +1,103 @@
+// Internal declarations shared by the translation units of libbigmac (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "bigmac.h"
+
+namespace bigmac {
+
+constexpr int kPad = 128;          // expert segments are padded to multiples of this many rows internally
+constexpr int kMaxExperts = 1024;
+
+// ---------------------------------------------------------------------------------------------
+// GEMM request:  C[m,n] (+)= epilogue( sum_k A(m,k) * B(n,k) )
+//   a_kmajor: A(m,k) = A[m*lda + k], else A[k*lda + m].   b_kmajor: B(n,k) = B[n*ldb + k], else B[k*ldb + n].
+//   C is row-major [M, ldc].
+// Grouping (the experts' variable-length row segments, padded to kPad rows; tables live on the device):
+//   GROUP_NONE  one dense problem.
+//   GROUP_M     rows of A and C are the padded grouped rows; row tile i (kPad rows) belongs to expert
+//               tile_expert[i] (only the first *n_tiles tiles exist); B of expert e starts at B + e*b_stride.
+//   GROUP_K     one problem per expert e with the contraction running over its padded rows
+//               [poffsets[e], poffsets[e+1]) of A and B; C of expert e starts at C + e*c_stride.
+// ---------------------------------------------------------------------------------------------
+enum GroupMode { GROUP_NONE = 0, GROUP_M = 1, GROUP_K = 2 };
+enum Epilogue {
+    EPI_NONE = 0,   // C = acc
+    EPI_ACT = 1,    // Z = acc (if Z != nullptr), C = sigma(acc)
+    EPI_DACT = 2,   // C = acc * sigma'(Z[m,n])      (C may alias Z)
+};
+
+struct GemmArgs {
+    const void* A = nullptr; const void* B = nullptr; void* C = nullptr;
+    void* Z = nullptr;                  // activation input, [M, ldc] like C, element type = input dtype
+    int64_t lda = 0, ldb = 0, ldc = 0;
+    int M = 0, N = 0, K = 0;            // GROUP_M: M = upper bound on padded rows; GROUP_K: K = row extent of A and B
+    bool a_kmajor = true, b_kmajor = true;
+    bool out_f32 = false;               // C is fp32 regardless of the input dtype
+    bool accumulate = false;            // C += result
+    int epilogue = EPI_NONE;
+    int act = 0;
+    int group = GROUP_NONE;
+    int num_experts = 0;
+    int64_t b_stride = 0, c_stride = 0; // elements
+    const int32_t* tile_expert = nullptr;
+    const int32_t* n_tiles = nullptr;
+    const int32_t* poffsets = nullptr;
+};
+
+// fp32-FMA GEMM for either dtype (dtype: bigmac_dtype_t of A, B, Z and - unless out_f32 - C).
+cudaError_t gemm_simt(const GemmArgs& g, int dtype, cudaStream_t stream);
+// tcgen05 / TMEM / TMA GEMM, bf16 inputs, fp32 accumulation.  `status` is the device status word.
+cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream);
+bool gemm_tc_available();
+
+// ---------------------------------------------------------------------------------------------
+// Routing tables held in device memory (internal superset of bigmac_routing_t).
+// ---------------------------------------------------------------------------------------------
+struct Tables {
+    int32_t* topk_idx;      // [N]
+    float* topk_w;          // [N]
+    int32_t* counts;        // [E]
+    int32_t* offsets;       // [E+1]   canonical (unpadded)
+    int32_t* poffsets;      // [E+1]   padded to kPad
+    int32_t* row_of_slot;   // [N]     canonical
+    int32_t* slot_of_row;   // [N]
+    int32_t* prow_of_slot;  // [N]     row in the padded grouped buffers
+    int32_t* slot_of_prow;  // [P]     -1 on padding rows
+    int32_t* tile_expert;   // [P/kPad]
+    int32_t* n_tiles;       // [1]     number of kPad-row tiles in use
+    int32_t* block_counts;  // [n_blocks, E] scratch of the counting sort
+};
+
+inline int64_t padded_rows_max(int64_t N, int E) { return ((N + kPad - 1) / kPad + E) * (int64_t)kPad; }
+constexpr int kSortChunk = 1024;   // slots per block of the counting sort
+inline int sort_blocks(int64_t N) { return (int)((N + kSortChunk - 1) / kSortChunk); }
+
+// logits [T,E] fp32 (+ b_gate) -> topk_idx, topk_w.
+cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, int k, int32_t* topk_idx,
+                        float* topk_w, cudaStream_t stream);
+// topk_idx -> every other table (deterministic stable counting sort of slots by expert).
+cudaError_t launch_tables(const Tables& tb, int T, int E, int k, cudaStream_t stream);
+
+// Row moves.  `width` elements of the dtype per row; all row pointers 16-byte aligned.
+// grouped[prow,:] = src[slot_of_prow[prow]/k,:], zeros on padding rows, for prow < n_tiles*kPad.
+cudaError_t launch_dispatch(const void* src, void* grouped, const Tables& tb, int k, int width, int dtype,
+                            int64_t max_prows, cudaStream_t stream);
+// dst[t,:] = sum_j w[t*k+j] * grouped[prow_of_slot[t*k+j],:]   (w == nullptr: unit weights), fp32 accumulation.
+cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const int32_t* prow_of_slot, int T,
+                           int k, int width, int dtype, cudaStream_t stream);
+// Backward of the combine: du[prow,:] = p[s] * dy_lo[t,:] (zeros on padding), dp[s] = <dy_lo[t,:], u[prow,:]>.
+cudaError_t launch_combine_bwd(const void* dy_lo, const void* u, void* du, float* dp, const Tables& tb, int k,
+                               int width, int dtype, int64_t max_prows, cudaStream_t stream);
+// Softmax-over-k backward: g = sum_i p_i dp_i, dl_j = p_j (dp_j - g); writes the dense [T,E] matrix
+// (zeros off the top-k set, and in the padding columns E..ld-1) in the dtype, rows `ld` elements apart.
+cudaError_t launch_gate_bwd(const float* dp, const Tables& tb, void* dlogits, int T, int E, int ld, int k, int dtype,
+                            cudaStream_t stream);
+// db[e] (+)= sum_t dlogits[t,e]
+cudaError_t launch_colsum(const void* dlogits, float* db, int T, int E, int ld, int dtype, bool accumulate,
+                          cudaStream_t stream);
+
+}  // namespace bigmac

@@ -1,0 +1,480 @@
+// C-ABI entry points of libbigmac: argument checks, workspace carving and the launch sequence of the
+// BigMac DCCA MoE layer (Eq. 2 / Eq. 4), forward and backward.  No device allocation, no stream
+// synchronisation and no host-visible data dependence inside route / forward / backward: segment sizes
+// stay on the device.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+#include "bigmac_debug.h"
+
+using namespace bigmac;
+
+struct bigmac_layer {
+    bigmac_config_t cfg;
+    int device;
+    int* status;        // device status word
+    bool use_tc;        // bf16 contractions on tcgen05
+    unsigned tc_mask;   // debug: bit i set = contraction i runs on tcgen05 (BIGMAC_TC_MASK)
+};
+
+namespace {
+
+// Contraction ids (bits of tc_mask).
+enum { G_LOGITS = 0, G_DESCEND, G_EXPERT1, G_EXPERT2, G_ASCEND, G_DY_LO, G_DW_UP, G_DZ, G_DW2, G_DXG, G_DW1,
+       G_DX, G_DX_GATE, G_DW_DOWN, G_DW_GATE };
+
+inline size_t esize(int dtype) { return dtype == BIGMAC_BF16 ? 2 : 4; }
+
+// Hands out 256-byte-aligned regions of one buffer; with base == nullptr it only measures.
+struct Carver {
+    char* base;
+    size_t used = 0;
+    explicit Carver(void* b) : base((char*)b) {}
+    template <typename T> T* take(size_t count) {
+        used = (used + 255) & ~(size_t)255;
+        T* p = base ? (T*)(base + used) : nullptr;
+        used += count * sizeof(T);
+        return p;
+    }
+    void* take_bytes(size_t bytes) { return take<char>(bytes); }
+    size_t total() const { return (used + 255) & ~(size_t)255; }
+};
+
+struct Buffers {
+    Tables tb;
+    float* logits;
+    void *x_lo, *xg, *z, *a, *u, *y_lo;                 // forward intermediates
+    void *dy_lo, *du, *dxg, *dx_lo, *dlogits; float* dp; // backward intermediates
+};
+
+struct Dims {
+    int T, d, r, h, E, k, dtype;
+    int64_t N, P;
+    int E64;   // leading dimension of the dense [T,E] gate-gradient matrix (E rounded up to 64)
+};
+
+Dims dims_of(const bigmac_config_t& c, int T) {
+    Dims m{T, c.d, c.r, c.h, c.E, c.k, c.dtype, (int64_t)T * c.k, 0};
+    m.P = padded_rows_max(m.N, c.E);
+    m.E64 = (c.E + 63) / 64 * 64;
+    return m;
+}
+
+// What a training forward hands to its backward.
+void carve_saved(Carver& cv, const Dims& m, Buffers& b, bool with_z) {
+    const size_t es = esize(m.dtype);
+    b.tb.topk_idx = cv.take<int32_t>(m.N);
+    b.tb.topk_w = cv.take<float>(m.N);
+    b.tb.counts = cv.take<int32_t>(m.E);
+    b.tb.offsets = cv.take<int32_t>(m.E + 1);
+    b.tb.poffsets = cv.take<int32_t>(m.E + 1);
+    b.tb.row_of_slot = cv.take<int32_t>(m.N);
+    b.tb.slot_of_row = cv.take<int32_t>(m.N);
+    b.tb.prow_of_slot = cv.take<int32_t>(m.N);
+    b.tb.slot_of_prow = cv.take<int32_t>(m.P);
+    b.tb.tile_expert = cv.take<int32_t>(m.P / kPad);
+    b.tb.n_tiles = cv.take<int32_t>(1);
+    b.x_lo = cv.take_bytes((size_t)m.T * m.r * es);
+    b.xg = cv.take_bytes((size_t)m.P * m.r * es);
+    b.z = with_z ? cv.take_bytes((size_t)m.P * m.h * es) : nullptr;
+    b.a = cv.take_bytes((size_t)m.P * m.h * es);
+    b.u = cv.take_bytes((size_t)m.P * m.r * es);
+    b.y_lo = cv.take_bytes((size_t)m.T * m.r * es);
+}
+
+void carve_route_scratch(Carver& cv, const Dims& m, Buffers& b) {
+    b.logits = cv.take<float>((size_t)m.T * m.E);
+    b.tb.block_counts = cv.take<int32_t>((size_t)(sort_blocks(m.N) + 1) * m.E);
+}
+
+void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
+    const size_t es = esize(m.dtype);
+    b.dy_lo = cv.take_bytes((size_t)m.T * m.r * es);
+    b.du = cv.take_bytes((size_t)m.P * m.r * es);
+    b.dxg = cv.take_bytes((size_t)m.P * m.r * es);
+    b.dx_lo = cv.take_bytes((size_t)m.T * m.r * es);
+    b.dlogits = cv.take_bytes((size_t)m.T * m.E64 * es);
+    b.dp = cv.take<float>(m.N);
+}
+
+size_t forward_scratch_bytes(const Dims& m, bool training) {
+    Carver cv(nullptr);
+    Buffers b{};
+    carve_route_scratch(cv, m, b);
+    if (!training) carve_saved(cv, m, b, false);
+    return cv.total();
+}
+size_t backward_scratch_bytes(const Dims& m) {
+    Carver cv(nullptr);
+    Buffers b{};
+    carve_backward_scratch(cv, m, b);
+    return cv.total();
+}
+size_t saved_bytes_of(const Dims& m) {
+    Carver cv(nullptr);
+    Buffers b{};
+    carve_saved(cv, m, b, true);
+    return cv.total();
+}
+
+bool aligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
+
+int check_weights(const bigmac_weights_t* W) {
+    if (!W || !W->w_gate || !W->w_down || !W->w1 || !W->w2 || !W->w_up) return BIGMAC_ERR_INVALID_ARG;
+    if (!aligned(W->w_gate, 16) || !aligned(W->w_down, 16) || !aligned(W->w1, 16) || !aligned(W->w2, 16) ||
+        !aligned(W->w_up, 16) || !aligned(W->b_gate, 4))
+        return BIGMAC_ERR_INVALID_ARG;
+    return BIGMAC_OK;
+}
+
+int gemm(const bigmac_layer* L, int id, const GemmArgs& g, cudaStream_t st) {
+    cudaError_t err;
+    if (L->cfg.dtype == BIGMAC_BF16 && L->use_tc && ((L->tc_mask >> id) & 1u))
+        err = gemm_tc(g, L->status, st);
+    else
+        err = gemm_simt(g, L->cfg.dtype, st);
+    return err == cudaSuccess ? BIGMAC_OK : BIGMAC_ERR_CUDA;
+}
+
+#define BIGMAC_TRY(expr)                        \
+    do {                                        \
+        int _s = (expr);                        \
+        if (_s != BIGMAC_OK) return _s;         \
+    } while (0)
+#define BIGMAC_CUDA(expr)                                   \
+    do {                                                    \
+        if ((expr) != cudaSuccess) return BIGMAC_ERR_CUDA;  \
+    } while (0)
+
+// Steps F1-F3: gate logits on x, top-k with softmax gate values, dispatch layout.
+int run_routing(const bigmac_layer* L, const Dims& m, const void* x, const bigmac_weights_t* W, Buffers& b,
+                cudaStream_t st) {
+    GemmArgs g;
+    g.A = x; g.lda = m.d; g.B = W->w_gate; g.ldb = m.d; g.C = b.logits; g.ldc = m.E;
+    g.M = m.T; g.N = m.E; g.K = m.d; g.out_f32 = true;
+    BIGMAC_TRY(gemm(L, G_LOGITS, g, st));
+    BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st));
+    BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, st));
+    return BIGMAC_OK;
+}
+
+int export_routing(const Dims& m, const Buffers& b, bigmac_routing_t* out, cudaStream_t st) {
+    if (!out) return BIGMAC_OK;
+    const cudaMemcpyKind kind = cudaMemcpyDeviceToDevice;
+    if (out->topk_idx) BIGMAC_CUDA(cudaMemcpyAsync(out->topk_idx, b.tb.topk_idx, sizeof(int32_t) * m.N, kind, st));
+    if (out->topk_w) BIGMAC_CUDA(cudaMemcpyAsync(out->topk_w, b.tb.topk_w, sizeof(float) * m.N, kind, st));
+    if (out->counts) BIGMAC_CUDA(cudaMemcpyAsync(out->counts, b.tb.counts, sizeof(int32_t) * m.E, kind, st));
+    if (out->offsets) BIGMAC_CUDA(cudaMemcpyAsync(out->offsets, b.tb.offsets, sizeof(int32_t) * (m.E + 1), kind, st));
+    if (out->row_of_slot)
+        BIGMAC_CUDA(cudaMemcpyAsync(out->row_of_slot, b.tb.row_of_slot, sizeof(int32_t) * m.N, kind, st));
+    if (out->slot_of_row)
+        BIGMAC_CUDA(cudaMemcpyAsync(out->slot_of_row, b.tb.slot_of_row, sizeof(int32_t) * m.N, kind, st));
+    return BIGMAC_OK;
+}
+
+int check_call(const bigmac_layer* L, int32_t T) {
+    if (!L) return BIGMAC_ERR_INVALID_ARG;
+    if (T < 0 || T > L->cfg.max_tokens) return BIGMAC_ERR_INVALID_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return BIGMAC_ERR_CUDA;
+    if (dev != L->device) return BIGMAC_ERR_STATE;
+    return BIGMAC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
+    if (!cfg || !out) return BIGMAC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->d <= 0 || cfg->r <= 0 || cfg->h <= 0 || cfg->E <= 0 || cfg->k <= 0 || cfg->max_tokens < 0)
+        return BIGMAC_ERR_INVALID_ARG;
+    if (cfg->k > cfg->E) return BIGMAC_ERR_INVALID_ARG;
+    if (cfg->dtype != BIGMAC_F32 && cfg->dtype != BIGMAC_BF16) return BIGMAC_ERR_INVALID_ARG;
+    if (cfg->act < BIGMAC_ACT_RELU || cfg->act > BIGMAC_ACT_IDENTITY) return BIGMAC_ERR_INVALID_ARG;
+    if (cfg->flags & ~BIGMAC_FLAG_SIMT_GEMM) return BIGMAC_ERR_INVALID_ARG;
+    if (cfg->E > kMaxExperts) return BIGMAC_ERR_UNSUPPORTED;
+    if ((int64_t)cfg->max_tokens * cfg->k > (int64_t)1 << 30) return BIGMAC_ERR_UNSUPPORTED;
+    const int vec = cfg->dtype == BIGMAC_BF16 ? 8 : 4;     // rows move as 16-byte vectors
+    if (cfg->d % vec || cfg->r % vec || cfg->h % vec) return BIGMAC_ERR_UNSUPPORTED;
+    if (cfg->dtype == BIGMAC_BF16 && (cfg->d % 64 || cfg->r % 64 || cfg->h % 64)) return BIGMAC_ERR_UNSUPPORTED;
+    bigmac_layer* L = new (std::nothrow) bigmac_layer();
+    if (!L) return BIGMAC_ERR_CUDA;
+    L->cfg = *cfg;
+    L->use_tc = cfg->dtype == BIGMAC_BF16 && !(cfg->flags & BIGMAC_FLAG_SIMT_GEMM);
+    L->tc_mask = ~0u;
+    if (const char* env = std::getenv("BIGMAC_TC_MASK")) L->tc_mask = (unsigned)std::strtoul(env, nullptr, 0);
+    if (cudaGetDevice(&L->device) != cudaSuccess || cudaMalloc((void**)&L->status, sizeof(int)) != cudaSuccess ||
+        cudaMemset(L->status, 0, sizeof(int)) != cudaSuccess) {
+        delete L;
+        return BIGMAC_ERR_CUDA;
+    }
+    if (L->use_tc && !gemm_tc_available()) {
+        cudaFree(L->status);
+        delete L;
+        return BIGMAC_ERR_UNSUPPORTED;
+    }
+    *out = L;
+    return BIGMAC_OK;
+}
+
+int bigmac_layer_destroy(bigmac_layer_t* L) {
+    if (!L) return BIGMAC_ERR_INVALID_ARG;
+    cudaFree(L->status);
+    delete L;
+    return BIGMAC_OK;
+}
+
+int bigmac_workspace_bytes(const bigmac_layer_t* L, int32_t T, int training, size_t* scratch_bytes,
+                           size_t* saved_bytes) {
+    if (!L || !scratch_bytes || !saved_bytes || T < 0 || T > L->cfg.max_tokens) return BIGMAC_ERR_INVALID_ARG;
+    const Dims m = dims_of(L->cfg, T);
+    size_t s = forward_scratch_bytes(m, training != 0);
+    if (training) {
+        const size_t bw = backward_scratch_bytes(m);
+        if (bw > s) s = bw;
+    }
+    *scratch_bytes = s;
+    *saved_bytes = training ? saved_bytes_of(m) : 0;
+    return BIGMAC_OK;
+}
+
+int bigmac_route(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_weights_t* W, bigmac_routing_t* out,
+                 void* scratch, size_t scratch_bytes, void* stream) {
+    BIGMAC_TRY(check_call(L, T));
+    if (!out) return BIGMAC_ERR_INVALID_ARG;
+    BIGMAC_TRY(check_weights(W));
+    if (T == 0) return BIGMAC_OK;
+    if (!x || !aligned(x, 16) || !scratch || !aligned(scratch, 256)) return BIGMAC_ERR_INVALID_ARG;
+    const Dims m = dims_of(L->cfg, T);
+    if (scratch_bytes < forward_scratch_bytes(m, false)) return BIGMAC_ERR_WORKSPACE;
+    Carver cv(scratch);
+    Buffers b{};
+    carve_route_scratch(cv, m, b);
+    carve_saved(cv, m, b, false);
+    cudaStream_t st = (cudaStream_t)stream;
+    BIGMAC_TRY(run_routing(L, m, x, W, b, st));
+    return export_routing(m, b, out, st);
+}
+
+int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_weights_t* W, void* y,
+                   bigmac_routing_t* routing_out, void* saved, void* scratch, size_t scratch_bytes, void* stream) {
+    BIGMAC_TRY(check_call(L, T));
+    BIGMAC_TRY(check_weights(W));
+    if (T == 0) return BIGMAC_OK;
+    if (!x || !y || !aligned(x, 16) || !aligned(y, 16) || !scratch || !aligned(scratch, 256) ||
+        !aligned(saved, 256))
+        return BIGMAC_ERR_INVALID_ARG;
+    const bool training = saved != nullptr;
+    const Dims m = dims_of(L->cfg, T);
+    if (scratch_bytes < forward_scratch_bytes(m, training)) return BIGMAC_ERR_WORKSPACE;
+    Buffers b{};
+    Carver cs(scratch);
+    carve_route_scratch(cs, m, b);
+    if (training) {
+        Carver cv(saved);
+        carve_saved(cv, m, b, true);
+    } else {
+        carve_saved(cs, m, b, false);
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    const bigmac_config_t& c = L->cfg;
+
+    BIGMAC_TRY(run_routing(L, m, x, W, b, st));                                   // F1-F3
+    BIGMAC_TRY(export_routing(m, b, routing_out, st));
+    {                                                                             // F4 descend: x' = x W'_down
+        GemmArgs g;
+        g.A = x; g.lda = m.d; g.B = W->w_down; g.ldb = m.d; g.C = b.x_lo; g.ldc = m.r;
+        g.M = m.T; g.N = m.r; g.K = m.d;
+        BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
+    }
+    BIGMAC_CUDA(launch_dispatch(b.x_lo, b.xg, b.tb, m.k, m.r, m.dtype, m.P, st)); // F5 dispatch at width r
+    {                                                                             // F6 a = sigma(xg W1_e^T)
+        GemmArgs g;
+        g.A = b.xg; g.lda = m.r; g.B = W->w1; g.ldb = m.r; g.b_stride = (int64_t)m.h * m.r;
+        g.C = b.a; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
+        g.epilogue = EPI_ACT; g.act = c.act; g.group = GROUP_M; g.num_experts = m.E;
+        g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles;
+        BIGMAC_TRY(gemm(L, G_EXPERT1, g, st));
+    }
+    {                                                                             // F7 u = a W2_e^T
+        GemmArgs g;
+        g.A = b.a; g.lda = m.h; g.B = W->w2; g.ldb = m.h; g.b_stride = (int64_t)m.r * m.h;
+        g.C = b.u; g.ldc = m.r; g.M = (int)m.P; g.N = m.r; g.K = m.h;
+        g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles;
+        BIGMAC_TRY(gemm(L, G_EXPERT2, g, st));
+    }
+    BIGMAC_CUDA(launch_combine(b.u, b.y_lo, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st));  // F8
+    {                                                                             // F9 ascend: y = y' W'_up
+        GemmArgs g;
+        g.A = b.y_lo; g.lda = m.r; g.B = W->w_up; g.ldb = m.r; g.C = y; g.ldc = m.d;
+        g.M = m.T; g.N = m.d; g.K = m.r;
+        BIGMAC_TRY(gemm(L, G_ASCEND, g, st));
+    }
+    return BIGMAC_OK;
+}
+
+int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T, const bigmac_weights_t* W,
+                    void* saved, void* dx, const bigmac_grads_t* G, int accumulate, void* scratch,
+                    size_t scratch_bytes, void* stream) {
+    BIGMAC_TRY(check_call(L, T));
+    BIGMAC_TRY(check_weights(W));
+    if (!G) return BIGMAC_ERR_INVALID_ARG;
+    if (T == 0) return BIGMAC_OK;
+    if (!x || !dy || !dx || !saved || !scratch || !aligned(x, 16) || !aligned(dy, 16) || !aligned(dx, 16) ||
+        !aligned(saved, 256) || !aligned(scratch, 256))
+        return BIGMAC_ERR_INVALID_ARG;
+    if (!aligned(G->dw_gate, 16) || !aligned(G->dw_down, 16) || !aligned(G->dw1, 16) || !aligned(G->dw2, 16) ||
+        !aligned(G->dw_up, 16) || !aligned(G->db_gate, 4))
+        return BIGMAC_ERR_INVALID_ARG;
+    const Dims m = dims_of(L->cfg, T);
+    if (scratch_bytes < backward_scratch_bytes(m)) return BIGMAC_ERR_WORKSPACE;
+    Buffers b{};
+    {
+        Carver cv(saved);
+        carve_saved(cv, m, b, true);
+        Carver cs(scratch);
+        carve_backward_scratch(cs, m, b);
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    const bigmac_config_t& c = L->cfg;
+    const bool acc = accumulate != 0;
+
+    {   // dy' = dy W_up                                   [T,d] x [d,r]
+        GemmArgs g;
+        g.A = dy; g.lda = m.d; g.B = W->w_up; g.ldb = m.r; g.b_kmajor = false; g.C = b.dy_lo; g.ldc = m.r;
+        g.M = m.T; g.N = m.r; g.K = m.d;
+        BIGMAC_TRY(gemm(L, G_DY_LO, g, st));
+    }
+    if (G->dw_up) {   // dW_up[c,c'] = sum_t dy[t,c] y'[t,c']
+        GemmArgs g;
+        g.A = dy; g.lda = m.d; g.a_kmajor = false; g.B = b.y_lo; g.ldb = m.r; g.b_kmajor = false;
+        g.C = G->dw_up; g.ldc = m.r; g.M = m.d; g.N = m.r; g.K = m.T; g.accumulate = acc;
+        BIGMAC_TRY(gemm(L, G_DW_UP, g, st));
+    }
+    // du = p dy'[t], dp = <dy'[t], u>; then the softmax-over-k backward
+    BIGMAC_CUDA(launch_combine_bwd(b.dy_lo, b.u, b.du, b.dp, b.tb, m.k, m.r, m.dtype, m.P, st));
+    BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, m.k, m.dtype, st));
+    {   // dz = (du W2_e) * sigma'(z), written over z
+        GemmArgs g;
+        g.A = b.du; g.lda = m.r; g.B = W->w2; g.ldb = m.h; g.b_kmajor = false; g.b_stride = (int64_t)m.r * m.h;
+        g.C = b.z; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
+        g.epilogue = EPI_DACT; g.act = c.act; g.group = GROUP_M; g.num_experts = m.E;
+        g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles;
+        BIGMAC_TRY(gemm(L, G_DZ, g, st));
+    }
+    void* dz = b.z;
+    if (G->dw2) {   // dW2_e[c',q] = sum_rows du[row,c'] a[row,q]
+        GemmArgs g;
+        g.A = b.du; g.lda = m.r; g.a_kmajor = false; g.B = b.a; g.ldb = m.h; g.b_kmajor = false;
+        g.C = G->dw2; g.ldc = m.h; g.c_stride = (int64_t)m.r * m.h; g.M = m.r; g.N = m.h; g.K = (int)m.P;
+        g.group = GROUP_K; g.num_experts = m.E; g.poffsets = b.tb.poffsets; g.accumulate = acc;
+        BIGMAC_TRY(gemm(L, G_DW2, g, st));
+    }
+    {   // dxg = dz W1_e
+        GemmArgs g;
+        g.A = dz; g.lda = m.h; g.B = W->w1; g.ldb = m.r; g.b_kmajor = false; g.b_stride = (int64_t)m.h * m.r;
+        g.C = b.dxg; g.ldc = m.r; g.M = (int)m.P; g.N = m.r; g.K = m.h;
+        g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles;
+        BIGMAC_TRY(gemm(L, G_DXG, g, st));
+    }
+    if (G->dw1) {   // dW1_e[q,c'] = sum_rows dz[row,q] xg[row,c']
+        GemmArgs g;
+        g.A = dz; g.lda = m.h; g.a_kmajor = false; g.B = b.xg; g.ldb = m.r; g.b_kmajor = false;
+        g.C = G->dw1; g.ldc = m.r; g.c_stride = (int64_t)m.h * m.r; g.M = m.h; g.N = m.r; g.K = (int)m.P;
+        g.group = GROUP_K; g.num_experts = m.E; g.poffsets = b.tb.poffsets; g.accumulate = acc;
+        BIGMAC_TRY(gemm(L, G_DW1, g, st));
+    }
+    // dx'[t] = sum_j dxg[row of slot (t,j)]   (the transpose of the dispatch gather)
+    BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st));
+    {   // dx = dx' W_down
+        GemmArgs g;
+        g.A = b.dx_lo; g.lda = m.r; g.B = W->w_down; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
+        g.M = m.T; g.N = m.d; g.K = m.r;
+        BIGMAC_TRY(gemm(L, G_DX, g, st));
+    }
+    {   // dx += dl W_gate
+        GemmArgs g;
+        g.A = b.dlogits; g.lda = m.E64; g.B = W->w_gate; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
+        g.M = m.T; g.N = m.d; g.K = m.E; g.accumulate = true;
+        BIGMAC_TRY(gemm(L, G_DX_GATE, g, st));
+    }
+    if (G->dw_down) {   // dW_down[c',c] = sum_t dx'[t,c'] x[t,c]
+        GemmArgs g;
+        g.A = b.dx_lo; g.lda = m.r; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
+        g.C = G->dw_down; g.ldc = m.d; g.M = m.r; g.N = m.d; g.K = m.T; g.accumulate = acc;
+        BIGMAC_TRY(gemm(L, G_DW_DOWN, g, st));
+    }
+    if (G->dw_gate) {   // dW_gate[e,c] = sum_t dl[t,e] x[t,c]
+        GemmArgs g;
+        g.A = b.dlogits; g.lda = m.E64; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
+        g.C = G->dw_gate; g.ldc = m.d; g.M = m.E; g.N = m.d; g.K = m.T; g.accumulate = acc;
+        BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
+    }
+    if (G->db_gate) BIGMAC_CUDA(launch_colsum(b.dlogits, G->db_gate, m.T, m.E, m.E64, m.dtype, acc, st));
+    return BIGMAC_OK;
+}
+
+int bigmac_device_status(bigmac_layer_t* L, void* stream) {
+    if (!L) return BIGMAC_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    int word = 0;
+    if (cudaMemcpyAsync(&word, L->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemsetAsync(L->status, 0, sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+        return BIGMAC_ERR_CUDA;
+    return word == 0 ? BIGMAC_OK : BIGMAC_ERR_TIMEOUT;
+}
+
+const char* bigmac_status_string(int status) {
+    switch (status) {
+        case BIGMAC_OK: return "ok";
+        case BIGMAC_ERR_INVALID_ARG: return "invalid argument";
+        case BIGMAC_ERR_UNSUPPORTED: return "unsupported configuration";
+        case BIGMAC_ERR_WORKSPACE: return "workspace too small";
+        case BIGMAC_ERR_CUDA: return "CUDA error";
+        case BIGMAC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case BIGMAC_ERR_STATE: return "handle used on the wrong device";
+        default: return "unknown status";
+    }
+}
+
+int bigmac_exchange_rows(bigmac_layer_t* L, const void* saved, int32_t T, int32_t width, const void* src,
+                         void* grouped, size_t grouped_bytes, void* dst, int which, void* stream) {
+    BIGMAC_TRY(check_call(L, T));
+    if (!saved || !grouped || width <= 0 || which < 0 || which > 2 || !aligned(saved, 256) ||
+        !aligned(grouped, 16) || !aligned(src, 16) || !aligned(dst, 16))
+        return BIGMAC_ERR_INVALID_ARG;
+    if ((which != 1 && !src) || (which != 0 && !dst)) return BIGMAC_ERR_INVALID_ARG;
+    const size_t es = esize(L->cfg.dtype);
+    if ((width * es) % 16) return BIGMAC_ERR_UNSUPPORTED;
+    if (T == 0) return BIGMAC_OK;
+    const Dims m = dims_of(L->cfg, T);
+    if (grouped_bytes < (size_t)m.P * width * es) return BIGMAC_ERR_WORKSPACE;
+    Buffers b{};
+    Carver cv(const_cast<void*>(saved));
+    carve_saved(cv, m, b, true);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (which != 1) BIGMAC_CUDA(launch_dispatch(src, grouped, b.tb, m.k, width, m.dtype, m.P, st));
+    if (which != 0)
+        BIGMAC_CUDA(launch_combine(grouped, dst, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, width, m.dtype, st));
+    return BIGMAC_OK;
+}
+
+// ---- debug / unit-test entry point (declared in bigmac_debug.h) --------------------------------------
+int bigmac_debug_gemm(bigmac_layer_t* L, const bigmac_debug_gemm_t* q, int use_tensor_cores, void* stream) {
+    if (!L || !q) return BIGMAC_ERR_INVALID_ARG;
+    GemmArgs g;
+    g.A = q->A; g.B = q->B; g.C = q->C; g.Z = q->Z; g.lda = q->lda; g.ldb = q->ldb; g.ldc = q->ldc;
+    g.M = q->M; g.N = q->N; g.K = q->K; g.a_kmajor = q->a_kmajor != 0; g.b_kmajor = q->b_kmajor != 0;
+    g.out_f32 = q->out_f32 != 0; g.accumulate = q->accumulate != 0; g.epilogue = q->epilogue; g.act = q->act;
+    g.group = q->group; g.num_experts = q->num_experts; g.b_stride = q->b_stride; g.c_stride = q->c_stride;
+    g.tile_expert = q->tile_expert; g.n_tiles = q->n_tiles; g.poffsets = q->poffsets;
+    cudaError_t err = use_tensor_cores ? gemm_tc(g, L->status, (cudaStream_t)stream)
+                                       : gemm_simt(g, L->cfg.dtype, (cudaStream_t)stream);
+    return err == cudaSuccess ? BIGMAC_OK : BIGMAC_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,226 @@
+// Row-move kernels of the exchange stage: dispatch (token rows -> expert-grouped rows), combine
+// (gate-weighted return to token order) and their backward twins.  All rows move as 16-byte vectors;
+// one warp owns one destination row, so every output element is written once and summed in a fixed
+// order (deterministic, no atomics).
+#include "internal.h"
+
+namespace bigmac {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+template <typename T> struct Vec;          // 16 bytes of T
+template <> struct Vec<float> {
+    static constexpr int kElems = 4;
+    static __device__ __forceinline__ void unpack(const uint4& v, float* f) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+    static __device__ __forceinline__ uint4 pack(const float* f) {
+        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+    }
+};
+template <> struct Vec<__nv_bfloat16> {
+    static constexpr int kElems = 8;
+    static __device__ __forceinline__ void unpack(const uint4& v, float* f) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    static __device__ __forceinline__ uint4 pack(const float* f) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t*>(&p);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+__device__ __forceinline__ int warp_global_id() { return blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); }
+
+__global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__ src, uint4* __restrict__ grouped,
+                                                       const int32_t* __restrict__ slot_of_prow,
+                                                       const int32_t* __restrict__ n_tiles, int k, int vecs_per_row,
+                                                       int64_t max_prows) {
+    const int64_t prow = warp_global_id();
+    int64_t live = (int64_t)(*n_tiles) * kPad;
+    if (live > max_prows) live = max_prows;
+    if (prow >= live) return;
+    const int lane = threadIdx.x & 31;
+    const int s = slot_of_prow[prow];
+    uint4* out = grouped + prow * vecs_per_row;
+    if (s < 0) {
+        for (int c = lane; c < vecs_per_row; c += 32) out[c] = make_uint4(0, 0, 0, 0);
+    } else {
+        const uint4* in = src + (int64_t)(s / k) * vecs_per_row;
+        for (int c = lane; c < vecs_per_row; c += 32) out[c] = in[c];
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ grouped, uint4* __restrict__ dst,
+                                                      const float* __restrict__ w,
+                                                      const int32_t* __restrict__ prow_of_slot, int n_tokens, int k,
+                                                      int vecs_per_row) {
+    constexpr int V = Vec<T>::kElems;
+    const int t = warp_global_id();
+    if (t >= n_tokens) return;
+    const int lane = threadIdx.x & 31;
+    for (int c = lane; c < vecs_per_row; c += 32) {
+        float acc[V];
+#pragma unroll
+        for (int i = 0; i < V; ++i) acc[i] = 0.0f;
+        for (int j = 0; j < k; ++j) {                      // slot order: fixed summation order
+            const int64_t s = (int64_t)t * k + j;
+            const float p = w ? w[s] : 1.0f;
+            float f[V];
+            Vec<T>::unpack(grouped[(int64_t)prow_of_slot[s] * vecs_per_row + c], f);
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc[i] = fmaf(p, f[i], acc[i]);
+        }
+        dst[(int64_t)t * vecs_per_row + c] = Vec<T>::pack(acc);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) combine_bwd_kernel(const uint4* __restrict__ dy_lo, const uint4* __restrict__ u,
+                                                          uint4* __restrict__ du, float* __restrict__ dp,
+                                                          const int32_t* __restrict__ slot_of_prow,
+                                                          const float* __restrict__ topk_w,
+                                                          const int32_t* __restrict__ n_tiles, int k, int vecs_per_row,
+                                                          int64_t max_prows) {
+    constexpr int V = Vec<T>::kElems;
+    const int64_t prow = warp_global_id();
+    int64_t live = (int64_t)(*n_tiles) * kPad;
+    if (live > max_prows) live = max_prows;
+    if (prow >= live) return;
+    const int lane = threadIdx.x & 31;
+    const int s = slot_of_prow[prow];
+    uint4* out = du + prow * vecs_per_row;
+    if (s < 0) {
+        for (int c = lane; c < vecs_per_row; c += 32) out[c] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    const float p = topk_w[s];
+    const uint4* g = dy_lo + (int64_t)(s / k) * vecs_per_row;
+    const uint4* ur = u + prow * vecs_per_row;
+    float dot = 0.0f;
+    for (int c = lane; c < vecs_per_row; c += 32) {
+        float a[V], b[V], o[V];
+        Vec<T>::unpack(g[c], a);
+        Vec<T>::unpack(ur[c], b);
+#pragma unroll
+        for (int i = 0; i < V; ++i) { dot = fmaf(a[i], b[i], dot); o[i] = p * a[i]; }
+        out[c] = Vec<T>::pack(o);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(kFull, dot, off);
+    if (lane == 0) dp[s] = dot;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) gate_bwd_kernel(const float* __restrict__ dp, const float* __restrict__ topk_w,
+                                                       const int32_t* __restrict__ topk_idx, T* __restrict__ dlogits,
+                                                       int n_tokens, int E, int ld, int k) {
+    const int t = warp_global_id();
+    if (t >= n_tokens) return;
+    const int lane = threadIdx.x & 31;
+    const float* p = topk_w + (int64_t)t * k;
+    const float* g = dp + (int64_t)t * k;
+    float part = 0.0f;
+    for (int j = lane; j < k; j += 32) part = fmaf(p[j], g[j], part);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
+    T* row = dlogits + (int64_t)t * ld;
+    for (int e = lane; e < ld; e += 32) row[e] = (T)0.0f;
+    __syncwarp();
+    for (int j = lane; j < k; j += 32) row[topk_idx[(int64_t)t * k + j]] = (T)(p[j] * (g[j] - part));
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ m, float* __restrict__ out, int rows, int cols,
+                                                     int ld, int accumulate) {
+    __shared__ float part[8][33];
+    const int c = blockIdx.x * 32 + (threadIdx.x & 31);
+    const int g = threadIdx.x >> 5;
+    float acc = 0.0f;
+    if (c < cols)
+        for (int r = g; r < rows; r += 8) acc += (float)m[(int64_t)r * ld + c];
+    part[g][threadIdx.x & 31] = acc;
+    __syncthreads();
+    if (g == 0 && c < cols) {
+        float total = 0.0f;
+        for (int i = 0; i < 8; ++i) total += part[i][threadIdx.x];
+        out[c] = accumulate ? out[c] + total : total;
+    }
+}
+
+inline int elem_bytes(int dtype) { return dtype == BIGMAC_BF16 ? 2 : 4; }
+inline unsigned warp_blocks(int64_t warps) { return (unsigned)((warps + 7) / 8); }
+
+}  // namespace
+
+cudaError_t launch_dispatch(const void* src, void* grouped, const Tables& tb, int k, int width, int dtype,
+                            int64_t max_prows, cudaStream_t stream) {
+    if (max_prows == 0) return cudaSuccess;
+    const int vecs = width * elem_bytes(dtype) / 16;
+    dispatch_kernel<<<warp_blocks(max_prows), 256, 0, stream>>>((const uint4*)src, (uint4*)grouped, tb.slot_of_prow,
+                                                                tb.n_tiles, k, vecs, max_prows);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const int32_t* prow_of_slot, int T, int k,
+                           int width, int dtype, cudaStream_t stream) {
+    if (T == 0) return cudaSuccess;
+    const int vecs = width * elem_bytes(dtype) / 16;
+    if (dtype == BIGMAC_BF16)
+        combine_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, stream>>>((const uint4*)grouped, (uint4*)dst, w,
+                                                                         prow_of_slot, T, k, vecs);
+    else
+        combine_kernel<float><<<warp_blocks(T), 256, 0, stream>>>((const uint4*)grouped, (uint4*)dst, w, prow_of_slot,
+                                                                 T, k, vecs);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine_bwd(const void* dy_lo, const void* u, void* du, float* dp, const Tables& tb, int k,
+                               int width, int dtype, int64_t max_prows, cudaStream_t stream) {
+    if (max_prows == 0) return cudaSuccess;
+    const int vecs = width * elem_bytes(dtype) / 16;
+    if (dtype == BIGMAC_BF16)
+        combine_bwd_kernel<__nv_bfloat16><<<warp_blocks(max_prows), 256, 0, stream>>>(
+            (const uint4*)dy_lo, (const uint4*)u, (uint4*)du, dp, tb.slot_of_prow, tb.topk_w, tb.n_tiles, k, vecs,
+            max_prows);
+    else
+        combine_bwd_kernel<float><<<warp_blocks(max_prows), 256, 0, stream>>>(
+            (const uint4*)dy_lo, (const uint4*)u, (uint4*)du, dp, tb.slot_of_prow, tb.topk_w, tb.n_tiles, k, vecs,
+            max_prows);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gate_bwd(const float* dp, const Tables& tb, void* dlogits, int T, int E, int ld, int k, int dtype,
+                            cudaStream_t stream) {
+    if (T == 0) return cudaSuccess;
+    if (dtype == BIGMAC_BF16)
+        gate_bwd_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, stream>>>(dp, tb.topk_w, tb.topk_idx,
+                                                                          (__nv_bfloat16*)dlogits, T, E, ld, k);
+    else
+        gate_bwd_kernel<float><<<warp_blocks(T), 256, 0, stream>>>(dp, tb.topk_w, tb.topk_idx, (float*)dlogits, T, E, ld, k);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_colsum(const void* dlogits, float* db, int T, int E, int ld, int dtype, bool accumulate,
+                          cudaStream_t stream) {
+    const unsigned blocks = (unsigned)((E + 31) / 32);
+    if (dtype == BIGMAC_BF16)
+        colsum_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)dlogits, db, T, E, ld, accumulate);
+    else
+        colsum_kernel<float><<<blocks, 256, 0, stream>>>((const float*)dlogits, db, T, E, ld, accumulate);
+    return cudaGetLastError();
+}
+
+}  // namespace bigmac

@@ -1,0 +1,210 @@
+// Routing kernels: per-token top-k with softmax gate values, and the deterministic stable counting
+// sort of routed slots by expert that lays out the dropless dispatch (the on-device stand-in for the
+// send layout of the first All-to-All).
+#include "internal.h"
+
+namespace bigmac {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+// One warp per token.  Lane l holds experts l, l+32, ...  k rounds of warp arg-max under the order
+// (logit descending, expert id ascending); gate values are the softmax over the k winners.
+template <int VPL>
+__global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ logits, const float* __restrict__ b_gate,
+                                                   int T, int E, int k, int32_t* __restrict__ topk_idx,
+                                                   float* __restrict__ topk_w) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const float* row = logits + (size_t)t * E;
+    float v[VPL];
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+        const int e = lane + 32 * i;
+        v[i] = e < E ? row[e] + (b_gate ? b_gate[e] : 0.0f) : -INFINITY;
+    }
+    int32_t* out_idx = topk_idx + (size_t)t * k;
+    float* out_w = topk_w + (size_t)t * k;
+    for (int j = 0; j < k; ++j) {
+        float best = -INFINITY;
+        int best_e = 0x7fffffff;
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) {            // ascending expert id within the lane: strict > keeps the lowest id
+            const int e = lane + 32 * i;
+            if (e < E && v[i] > best) { best = v[i]; best_e = e; }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(kFull, best, off);
+            const int oe = __shfl_xor_sync(kFull, best_e, off);
+            if (ov > best || (ov == best && oe < best_e)) { best = ov; best_e = oe; }
+        }
+        if ((best_e & 31) == lane) {
+#pragma unroll
+            for (int i = 0; i < VPL; ++i)
+                if (lane + 32 * i == best_e) v[i] = -INFINITY;
+        }
+        if (lane == 0) { out_idx[j] = best_e; out_w[j] = best; }   // raw logit for now
+    }
+    __syncwarp();
+    const float top = out_w[0];
+    float part = 0.0f;
+    for (int j = lane; j < k; j += 32) part += expf(out_w[j] - top);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
+    for (int j = lane; j < k; j += 32) out_w[j] = expf(out_w[j] - top) / part;
+}
+
+// Pass 1 of the counting sort.  Block b owns slots [b*kSortChunk, (b+1)*kSortChunk); it writes, per
+// slot, the number of earlier slots of the same block routed to the same expert, and per expert the
+// block's count.  Warps own consecutive sub-chunks, so the order is the slot order.
+__global__ void __launch_bounds__(256) sort_local_kernel(const int32_t* __restrict__ topk_idx, int64_t N, int E,
+                                                         int32_t* __restrict__ local_rank,
+                                                         int32_t* __restrict__ block_counts) {
+    extern __shared__ int32_t warp_run[];            // [8][E]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < 8 * E; i += blockDim.x) warp_run[i] = 0;
+    __syncthreads();
+    const int64_t base = (int64_t)blockIdx.x * kSortChunk + warp * (kSortChunk / 8);
+    int32_t my_rank[kSortChunk / 256];
+#pragma unroll
+    for (int it = 0; it < kSortChunk / 256; ++it) {
+        const int64_t s = base + it * 32 + lane;
+        const int e = s < N ? topk_idx[s] : -1;
+        const unsigned peers = __match_any_sync(kFull, e);
+        const int leader = __ffs(peers) - 1;
+        int old = 0;
+        if (lane == leader && e >= 0) {
+            old = warp_run[warp * E + e];
+            warp_run[warp * E + e] = old + __popc(peers);
+        }
+        old = __shfl_sync(kFull, old, leader);
+        my_rank[it] = old + __popc(peers & ((1u << lane) - 1u));
+        __syncwarp();
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {   // exclusive scan over the 8 warps
+        int run = 0;
+        for (int w = 0; w < 8; ++w) {
+            const int c = warp_run[w * E + e];
+            warp_run[w * E + e] = run;
+            run += c;
+        }
+        block_counts[(size_t)blockIdx.x * E + e] = run;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int it = 0; it < kSortChunk / 256; ++it) {
+        const int64_t s = base + it * 32 + lane;
+        if (s < N) local_rank[s] = warp_run[warp * E + topk_idx[s]] + my_rank[it];
+    }
+}
+
+// Pass 2 (one block): per expert an exclusive scan of the block counts, then offsets, padded offsets
+// and the tile -> expert map.
+__global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ block_counts, int n_blocks, int E,
+                                                         int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+                                                         int32_t* __restrict__ poffsets,
+                                                         int32_t* __restrict__ tile_expert,
+                                                         int32_t* __restrict__ n_tiles) {
+    __shared__ int32_t s_cnt[kMaxExperts];
+    __shared__ int32_t s_poff[kMaxExperts + 1];
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        int run = 0;
+        int b = 0;
+        for (; b + 8 <= n_blocks; b += 8) {
+            int c[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) c[i] = block_counts[(size_t)(b + i) * E + e];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { block_counts[(size_t)(b + i) * E + e] = run; run += c[i]; }
+        }
+        for (; b < n_blocks; ++b) {
+            const int c = block_counts[(size_t)b * E + e];
+            block_counts[(size_t)b * E + e] = run;
+            run += c;
+        }
+        s_cnt[e] = run;
+        counts[e] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int off = 0, poff = 0;
+        for (int e = 0; e < E; ++e) {
+            offsets[e] = off;
+            s_poff[e] = poff;
+            off += s_cnt[e];
+            poff += (s_cnt[e] + kPad - 1) / kPad * kPad;
+        }
+        offsets[E] = off;
+        s_poff[E] = poff;
+        *n_tiles = poff / kPad;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e <= E; e += blockDim.x) poffsets[e] = s_poff[e];
+    for (int e = threadIdx.x; e < E; e += blockDim.x)
+        for (int tile = s_poff[e] / kPad; tile < s_poff[e + 1] / kPad; ++tile) tile_expert[tile] = e;
+}
+
+// Pass 3: final positions.
+__global__ void __launch_bounds__(256) sort_place_kernel(const int32_t* __restrict__ topk_idx, int64_t N, int E,
+                                                         const int32_t* __restrict__ block_base,
+                                                         const int32_t* __restrict__ offsets,
+                                                         const int32_t* __restrict__ poffsets,
+                                                         int32_t* __restrict__ prow_of_slot /* in: local rank */,
+                                                         int32_t* __restrict__ row_of_slot,
+                                                         int32_t* __restrict__ slot_of_row,
+                                                         int32_t* __restrict__ slot_of_prow) {
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= N) return;
+    const int e = topk_idx[s];
+    const int within = block_base[(size_t)(s / kSortChunk) * E + e] + prow_of_slot[s];
+    const int row = offsets[e] + within;
+    const int prow = poffsets[e] + within;
+    row_of_slot[s] = row;
+    slot_of_row[row] = (int32_t)s;
+    prow_of_slot[s] = prow;
+    slot_of_prow[prow] = (int32_t)s;
+}
+
+}  // namespace
+
+cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, int k, int32_t* topk_idx,
+                        float* topk_w, cudaStream_t stream) {
+    if (T == 0) return cudaSuccess;
+    const int warps = 8;
+    dim3 grid((T + warps - 1) / warps), block(warps * 32);
+    const int vpl = (E + 31) / 32;
+#define BIGMAC_TOPK(V) topk_kernel<V><<<grid, block, 0, stream>>>(logits, b_gate, T, E, k, topk_idx, topk_w)
+    if (vpl <= 1) BIGMAC_TOPK(1);
+    else if (vpl <= 2) BIGMAC_TOPK(2);
+    else if (vpl <= 4) BIGMAC_TOPK(4);
+    else if (vpl <= 8) BIGMAC_TOPK(8);
+    else if (vpl <= 16) BIGMAC_TOPK(16);
+    else BIGMAC_TOPK(32);
+#undef BIGMAC_TOPK
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tables(const Tables& tb, int T, int E, int k, cudaStream_t stream) {
+    const int64_t N = (int64_t)T * k;
+    const int64_t P = padded_rows_max(N, E);
+    cudaError_t err = cudaMemsetAsync(tb.slot_of_prow, 0xff, sizeof(int32_t) * P, stream);
+    if (err != cudaSuccess) return err;
+    const int nb = sort_blocks(N);
+    if (nb > 0)
+        sort_local_kernel<<<nb, 256, sizeof(int32_t) * 8 * E, stream>>>(tb.topk_idx, N, E, tb.prow_of_slot,
+                                                                      tb.block_counts);
+    sort_scan_kernel<<<1, 1024, 0, stream>>>(tb.block_counts, nb, E, tb.counts, tb.offsets, tb.poffsets,
+                                             tb.tile_expert, tb.n_tiles);
+    if (N > 0)
+        sort_place_kernel<<<(unsigned)((N + 255) / 256), 256, 0, stream>>>(tb.topk_idx, N, E, tb.block_counts,
+                                                                          tb.offsets, tb.poffsets, tb.prow_of_slot,
+                                                                          tb.row_of_slot, tb.slot_of_row,
+                                                                          tb.slot_of_prow);
+    return cudaGetLastError();
+}
+
+}  // namespace bigmac

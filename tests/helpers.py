@@ -22,3 +22,52 @@ def small_workload(T=24, d=16, r=8, h=12, E=4, k=2, act=wl.ACT_GELU_ERF, seed=7,
 
 def regrid(w, inp, grid=2.0 ** -10):
     inp["x"] = (np.round(inp["x"] / grid) * grid).astype(np.float32)
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU side: move a generated workload to the device and run it through the C ABI binding.
+# ---------------------------------------------------------------------------------------------
+
+def to_device(w, inp, device="cuda"):
+    """numpy float32 arrays (dtype-representable values) -> torch tensors of the workload dtype."""
+    import torch
+
+    out = {}
+    for key, val in inp.items():
+        if val is None:
+            continue
+        if key == "b_gate" or w.dtype == wl.DTYPE_F32:
+            out[key] = torch.from_numpy(np.ascontiguousarray(val, dtype=np.float32)).to(device)
+        else:
+            bits = torch.from_numpy(wl.to_bf16_bits(val).view(np.int16)).to(device)
+            out[key] = bits.view(torch.bfloat16)
+    return out
+
+
+def to_numpy(t):
+    """torch tensor (fp32 / bf16 / int32) -> numpy float64 or int32."""
+    import torch
+
+    if t.dtype in (torch.int32, torch.int64):
+        return t.cpu().numpy()
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def make_layer(w, flags=0, max_tokens=None):
+    from paper_2502_16927_b200 import binding
+
+    return binding.Layer(w.d, w.r, w.h, w.E, w.k, max_tokens or max(w.T, 1), w.dtype, w.act, flags)
+
+
+def empty_grads(w, dev, fill=None):
+    import torch
+
+    dt = torch.float32 if w.dtype == wl.DTYPE_F32 else torch.bfloat16
+    shapes = {"dw_gate": (w.E, w.d), "dw_down": (w.r, w.d), "dw1": (w.E, w.h, w.r), "dw2": (w.E, w.r, w.h),
+              "dw_up": (w.d, w.r)}
+    G = {}
+    for key, shp in shapes.items():
+        G[key] = torch.empty(shp, dtype=dt, device="cuda") if fill is None else torch.full(shp, fill, dtype=dt, device="cuda")
+    G["db_gate"] = (torch.empty(w.E, dtype=torch.float32, device="cuda") if fill is None
+                    else torch.full((w.E,), fill, dtype=torch.float32, device="cuda"))
+    return G
