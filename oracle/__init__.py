@@ -130,8 +130,11 @@ def forward_grouped(inp, routing: Routing, act: int):
     return {"xg": xg, "y_lo": y_lo, "y": y}
 
 
-def backward_tokens(inp, routing: Routing, act: int, tokens=None):
-    """Per-token gradients of L = sum(y*dy): dx [n,d], dx_lo [n,r], dlogit [n,k] (top-k slots), dy_lo [n,r]."""
+def backward_tokens(inp, routing: Routing, act: int, tokens=None, decide_bf16: bool = False):
+    """Per-token gradients of L = sum(y*dy): dx [n,d], dx_lo [n,r], dlogit [n,k] (top-k slots), dy_lo [n,r].
+
+    decide_bf16: take the ReLU' decision (z > 0) from x' rounded to bf16, as the BF16 kernels do; a
+    discrete decision has to be taken on the same numbers on both sides.  No effect on other activations."""
     T, d, r, h, E = _dims(inp)
     k = routing.topk_idx.shape[1]
     tok, n = _tokens(tokens, T)
@@ -140,11 +143,11 @@ def backward_tokens(inp, routing: Routing, act: int, tokens=None):
                                  _p(_f32(inp["w_down"])), _p(_f32(inp["w1"])), _p(_f32(inp["w2"])),
                                  _p(_f32(inp["w_up"])), _p(routing.topk_idx), _p(routing.topk_p), _p(tok),
                                  C.c_int(n), C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(E), C.c_int(k),
-                                 C.c_int(act), _p(dx), _p(dx_lo), _p(dlogit), _p(dy_lo))
+                                 C.c_int(act), C.c_int(int(decide_bf16)), _p(dx), _p(dx_lo), _p(dlogit), _p(dy_lo))
     return {"dx": dx, "dx_lo": dx_lo, "dlogit": dlogit, "dy_lo": dy_lo}
 
 
-def backward_expert(inp, routing: Routing, act: int, e: int):
+def backward_expert(inp, routing: Routing, act: int, e: int, decide_bf16: bool = False):
     """dW1[e] [h,r] and dW2[e] [r,h], summed over the rows of expert e's segment."""
     T, d, r, h, E = _dims(inp)
     k = routing.topk_idx.shape[1]
@@ -152,16 +155,17 @@ def backward_expert(inp, routing: Routing, act: int, e: int):
     lib().oracle_backward_expert(_p(_f32(inp["x"])), _p(_f32(inp["dy"])), _p(_f32(inp["w_down"])),
                                  _p(_f32(inp["w1"])), _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])),
                                  _p(routing.topk_p), _p(routing.offsets), _p(routing.slot_of_row), C.c_int(e),
-                                 C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(k), C.c_int(act), _p(dw1), _p(dw2))
+                                 C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(k), C.c_int(act), C.c_int(int(decide_bf16)),
+                                 _p(dw1), _p(dw2))
     return dw1, dw2
 
 
-def backward_full(inp, routing: Routing, act: int, experts=None):
+def backward_full(inp, routing: Routing, act: int, experts=None, decide_bf16: bool = False):
     """All gradients: dx and every weight gradient (dw1/dw2 for `experts`, default all)."""
     T, d, r, h, E = _dims(inp)
     k = routing.topk_idx.shape[1]
     fwd = forward_tokens(inp, routing, act)
-    bwd = backward_tokens(inp, routing, act)
+    bwd = backward_tokens(inp, routing, act, decide_bf16=decide_bf16)
     dw_up = np.empty((d, r)); dw_down = np.empty((r, d)); dw_gate = np.empty((E, d)); db_gate = np.empty(E)
     lib().oracle_backward_shared(_p(_f32(inp["x"])), _p(_f32(inp["dy"])), _p(fwd["y_lo"]), _p(bwd["dx_lo"]),
                                  _p(routing.topk_idx), _p(bwd["dlogit"]), C.c_int(T), C.c_int(d), C.c_int(r),
@@ -169,11 +173,31 @@ def backward_full(inp, routing: Routing, act: int, experts=None):
     experts = range(E) if experts is None else experts
     dw1, dw2 = {}, {}
     for e in experts:
-        dw1[e], dw2[e] = backward_expert(inp, routing, act, e)
+        dw1[e], dw2[e] = backward_expert(inp, routing, act, e, decide_bf16)
     out = {"y": fwd["y"], "y_lo": fwd["y_lo"], "x_lo": fwd["x_lo"], "dx": bwd["dx"], "dx_lo": bwd["dx_lo"],
            "dlogit": bwd["dlogit"], "dw_up": dw_up, "dw_down": dw_down, "dw_gate": dw_gate,
            "db_gate": db_gate, "dw1": dw1, "dw2": dw2}
     return out
+
+
+def max_rel_err(a, b) -> float:
+    """max_i |a_i - b_i| / max_i |b_i|: the largest error relative to the largest reference magnitude."""
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    if b.size == 0:
+        return 0.0
+    top = float(np.max(np.abs(b)))
+    if top == 0.0:
+        return float(np.max(np.abs(a)))
+    return float(np.max(np.abs(a - b))) / top
+
+
+def fro_rel_err(a, b) -> float:
+    """||a - b||_F / ||b||_F."""
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    nb = float(np.linalg.norm(b))
+    return float(np.linalg.norm(a - b)) / nb if nb > 0 else float(np.linalg.norm(a))
 
 
 def rel_err(a, b) -> float:

@@ -91,6 +91,30 @@ void matvec_t(const double* g, const float* W, int n_out, int n_in, double* out)
     }
 }
 
+// Round to the nearest bf16 value (ties to even), via float.
+double round_bf16(double v) {
+    float f = (float)v;
+    uint32_t bits;
+    std::memcpy(&bits, &f, 4);
+    bits = (bits + 0x7fffu + ((bits >> 16) & 1u)) & 0xffff0000u;
+    std::memcpy(&f, &bits, 4);
+    return (double)f;
+}
+
+// The pre-activation at which sigma' is evaluated in the backward pass.  ReLU' is a discrete decision
+// (z > 0): when `decide_bf16` is set it is taken the way the BF16 kernels take it, from x' rounded to
+// bf16, so that both sides decide on the same numbers; every other quantity stays exact.
+void decision_preact(const double* x_lo, const double* z_exact, const float* w1_e, int r, int h, int act,
+                     int decide_bf16, double* z_dec) {
+    if (!decide_bf16 || act != ACT_RELU) {
+        std::memcpy(z_dec, z_exact, sizeof(double) * h);
+        return;
+    }
+    std::vector<double> xr(r);
+    for (int c = 0; c < r; ++c) xr[c] = round_bf16(x_lo[c]);
+    matvec(xr.data(), w1_e, h, r, z_dec);
+}
+
 void widen(const float* src, int n, double* dst) {
     for (int i = 0; i < n; ++i) dst[i] = (double)src[i];
 }
@@ -235,13 +259,13 @@ void oracle_forward_grouped(const float* x, const float* w_down, const float* w1
 void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate, const float* w_down,
                             const float* w1, const float* w2, const float* w_up, const int32_t* topk_idx,
                             const double* topk_p, const int32_t* tokens, int n, int d, int r, int h, int E,
-                            int k, int act, double* dx_out, double* dx_lo_out, double* dlogit_out,
-                            double* dy_lo_out) {
+                            int k, int act, int decide_bf16, double* dx_out, double* dx_lo_out,
+                            double* dlogit_out, double* dy_lo_out) {
     (void)E;
 #pragma omp parallel for schedule(dynamic, 4)
     for (int i = 0; i < n; ++i) {
         const int t = tokens ? tokens[i] : i;
-        std::vector<double> xt(d), dyt(d), x_lo(r), dy_lo(r), z(h), a(h), u(r), du(r), da(h), dz(h), tmp(r),
+        std::vector<double> xt(d), dyt(d), x_lo(r), dy_lo(r), z(h), zd(h), a(h), u(r), du(r), da(h), dz(h), tmp(r),
             dx_lo(r, 0.0), dp(k), dl(k), dx(d), gate_part(d, 0.0);
         widen(x + (size_t)t * d, d, xt.data());
         widen(dy + (size_t)t * d, d, dyt.data());
@@ -258,7 +282,8 @@ void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate
             dp[j] = acc;
             for (int c = 0; c < r; ++c) du[c] = p * dy_lo[c];
             matvec_t(du.data(), w2_e, r, h, da.data());
-            for (int q = 0; q < h; ++q) dz[q] = da[q] * act_df(act, z[q]);
+            decision_preact(x_lo.data(), z.data(), w1_e, r, h, act, decide_bf16, zd.data());
+            for (int q = 0; q < h; ++q) dz[q] = da[q] * act_df(act, zd[q]);
             matvec_t(dz.data(), w1_e, h, r, tmp.data());
             for (int c = 0; c < r; ++c) dx_lo[c] += tmp[c];
         }
@@ -284,12 +309,12 @@ void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate
 void oracle_backward_expert(const float* x, const float* dy, const float* w_down, const float* w1,
                             const float* w2, const float* w_up, const double* topk_p, const int32_t* offsets,
                             const int32_t* slot_of_row, int e, int d, int r, int h, int k, int act,
-                            double* dw1_e, double* dw2_e) {
+                            int decide_bf16, double* dw1_e, double* dw2_e) {
     std::fill(dw1_e, dw1_e + (size_t)h * r, 0.0);
     std::fill(dw2_e, dw2_e + (size_t)r * h, 0.0);
     const float* w1_e = w1 + (size_t)e * h * r;
     const float* w2_e = w2 + (size_t)e * r * h;
-    std::vector<double> xt(d), dyt(d), x_lo(r), dy_lo(r), z(h), a(h), u(r), du(r), da(h), dz(h);
+    std::vector<double> xt(d), dyt(d), x_lo(r), dy_lo(r), z(h), zd(h), a(h), u(r), du(r), da(h), dz(h);
     for (int row = offsets[e]; row < offsets[e + 1]; ++row) {
         const int s = slot_of_row[row];
         const int t = s / k;
@@ -301,7 +326,8 @@ void oracle_backward_expert(const float* x, const float* dy, const float* w_down
         expert_forward(x_lo.data(), w1_e, w2_e, r, h, act, z.data(), a.data(), u.data());
         for (int c = 0; c < r; ++c) du[c] = p * dy_lo[c];
         matvec_t(du.data(), w2_e, r, h, da.data());
-        for (int q = 0; q < h; ++q) dz[q] = da[q] * act_df(act, z[q]);
+        decision_preact(x_lo.data(), z.data(), w1_e, r, h, act, decide_bf16, zd.data());
+        for (int q = 0; q < h; ++q) dz[q] = da[q] * act_df(act, zd[q]);
         for (int c = 0; c < r; ++c)
             for (int q = 0; q < h; ++q) dw2_e[(size_t)c * h + q] += du[c] * a[q];
         for (int q = 0; q < h; ++q)
