@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the BigMac DCCA MoE layer on B200: tokens/s of one training step (forward + backward,
+all weight gradients) of one layer, and the fraction of the tensor-core roofline its contractions reach.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config large] [--impl ours|reference]
+
+A step is one pass of the whole hot path (routing, descend, dispatch, expert GEMMs, combine, ascend and
+the matching backward) over one batch of synthetic input.  The default workload is the largest
+configuration (T=32768, d=4096, r=512, E=128, k=8, h=2048, GELU, BF16), which is the one the layer's
+target is stated on.  With N > 1 (launched by torch.distributed.run) every rank runs its own batch on
+its own GPU - the layer has no exchange step on one GPU per rank, so there is no data-path collective -
+and the reported value is the total over ranks divided by the slowest rank's device time ("weak").
+
+`--impl reference` times the CPU oracle (plain fp64 loops, as it stands) on a bounded token sample of the
+same workload on the host cores; it is the reported baseline, not a target.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2502_16927_b200 import workloads as wl
+
+METRIC = "bigmac_layer_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# ------------------------------------------------------------------------------------------------ counts
+def forward_flops(w) -> float:
+    """Algorithmic forward FLOPs of one call: gate logits + descend + ascend + the two expert GEMMs over the
+    N = T*k routed rows (no padding rows, no dense every-expert work)."""
+    return 2.0 * w.T * w.d * (w.E + 2 * w.r) + 4.0 * w.N * w.r * w.h
+
+
+GEMM_FLOPS = {   # per launch, algorithmic (unpadded rows)
+    "gemm_logits": lambda w: 2.0 * w.T * w.d * w.E, "gemm_descend": lambda w: 2.0 * w.T * w.d * w.r,
+    "gemm_expert1": lambda w: 2.0 * w.N * w.r * w.h, "gemm_expert2": lambda w: 2.0 * w.N * w.r * w.h,
+    "gemm_ascend": lambda w: 2.0 * w.T * w.d * w.r, "gemm_dy_lo": lambda w: 2.0 * w.T * w.d * w.r,
+    "gemm_dw_up": lambda w: 2.0 * w.T * w.d * w.r, "gemm_dz": lambda w: 2.0 * w.N * w.r * w.h,
+    "gemm_dw2": lambda w: 2.0 * w.N * w.r * w.h, "gemm_dxg": lambda w: 2.0 * w.N * w.r * w.h,
+    "gemm_dw1": lambda w: 2.0 * w.N * w.r * w.h, "gemm_dx": lambda w: 2.0 * w.T * w.d * w.r,
+    "gemm_dx_gate": lambda w: 2.0 * w.T * w.d * w.E, "gemm_dw_down": lambda w: 2.0 * w.T * w.d * w.r,
+    "gemm_dw_gate": lambda w: 2.0 * w.T * w.d * w.E,
+}
+ROW_MOVE_BYTES = {   # per launch, algorithmic: rows read + rows written (+ the 4-byte tables)
+    "dispatch": lambda w, b: (w.T * w.r + w.N * w.r) * b + 4.0 * w.N,
+    "combine": lambda w, b: (w.N * w.r + w.T * w.r) * b + 8.0 * w.N,
+    "dxlo_gather": lambda w, b: (w.N * w.r + w.T * w.r) * b + 4.0 * w.N,
+    "combine_bwd": lambda w, b: (2.0 * w.N * w.r + w.N * w.r) * b + 12.0 * w.N,
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "tflops_burst": p["bf16_tflops"],
+                "tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops_burst": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.thread = [], None, None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append((time.time(), parts))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        inside = [r for t, r in self.rows if t0 is None or (t0 <= t <= t1 + 0.15)]
+        window = "timed region"
+        if not inside:                      # region shorter than the sampling period: use the loaded run
+            inside, window = [r for _, r in self.rows], "warm-up and timed region"
+        sm, mx, reasons = [], 0.0, set()
+        for r in inside:
+            try:
+                sm.append(float(r[0])); mx = max(mx, float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm), "window": window}
+
+
+# ------------------------------------------------------------------------------------------------ oracle leg
+def oracle_sample_rate(w, inp, sample_tokens: int):
+    """tokens/s of the CPU oracle (routing + forward + backward with every gradient) on the first
+    `sample_tokens` tokens of the workload; cost is linear in T, so the rate carries over."""
+    import oracle
+
+    S = min(sample_tokens, w.T)
+    sub = dict(inp, x=np.ascontiguousarray(inp["x"][:S]), dy=np.ascontiguousarray(inp["dy"][:S]))
+    t0 = time.perf_counter()
+    rt = oracle.route(sub, w.k)
+    oracle.backward_full(sub, rt, w.act)
+    dt = time.perf_counter() - t0
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    threads = int(os.environ.get("OMP_NUM_THREADS", cores))
+    return S / dt, dt, S, min(threads, cores)
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = wl.make_inputs(w)
+    S = args.ref_tokens
+    rates = []
+    for i in range(args.warmup + args.steps):
+        rate, dt, S_used, cores = oracle_sample_rate(w, inp, S)
+        if i >= args.warmup:
+            rates.append((rate, dt))
+    total_t = sum(dt for _, dt in rates)
+    value = S_used * len(rates) / total_t
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / len(rates),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(w, args),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"first {S_used} tokens of the workload, all experts and gradients, per step"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def config_dict(w, args):
+    return {"workload": w.name, "T": w.T, "d": w.d, "r": w.r, "h": w.h, "E": w.E, "k": w.k,
+            "act": {0: "relu", 1: "gelu_erf", 2: "gelu_tanh", 3: "identity"}[w.act],
+            "gate_bias": w.gate_bias, "tokens_per_gpu": w.T,
+            "l2": "inputs larger than L2 (x, dy 268 MB each, weights 546 MB at the large workload)"}
+
+
+# ------------------------------------------------------------------------------------------------ ours
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_16927_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the layer has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+
+    wr = w.with_tokens(w.T, seed=w.seed + 1000 * rank)          # every rank draws its own batch
+    inp = wl.make_inputs(wr)
+    tdt = torch.bfloat16 if w.dtype == wl.DTYPE_BF16 else torch.float32
+
+    def host(a):
+        if w.dtype == wl.DTYPE_BF16:
+            t = torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).view(torch.bfloat16)
+        else:
+            t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
+        return t.pin_memory()
+
+    hx, hdy = host(inp["x"]), host(inp["dy"])
+    dev = {k: host(inp[k]).cuda() for k in ("w_gate", "w_down", "w1", "w2", "w_up")}
+    if inp["b_gate"] is not None:
+        dev["b_gate"] = torch.from_numpy(inp["b_gate"]).cuda()
+    x, dy = hx.cuda(), hdy.cuda()
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    G = {"dw_gate": torch.empty_like(dev["w_gate"]), "dw_down": torch.empty_like(dev["w_down"]),
+         "dw1": torch.empty_like(dev["w1"]), "dw2": torch.empty_like(dev["w2"]), "dw_up": torch.empty_like(dev["w_up"]),
+         "db_gate": torch.empty(w.E, dtype=torch.float32, device="cuda")}
+    hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+    layer = binding.Layer(w.d, w.r, w.h, w.E, w.k, w.T, w.dtype, w.act)
+    if rank != 0:
+        del inp
+
+    def step():
+        layer.forward(x, dev, y=y, training=True)
+        layer.backward(x, dy, dev, G, dx=dx)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        start.record()
+        for _ in range(steps):
+            fn()
+        stop.record()
+        barrier()
+        ms = torch.tensor([start.elapsed_time(stop)], device="cuda")
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    t_warm = time.time()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    if layer.status() != 0:
+        raise RuntimeError("device status word reports a timed-out wait")
+    while sampler and not sampler.rows and time.time() - t_warm < 3.0:   # let nvidia-smi come up, under load
+        step()
+        torch.cuda.synchronize()
+
+    # ---- timed region: K steps, device-timed, max over ranks; per-stage events recorded inside it
+    binding.bigmac_profile_enable(layer.handle, True)
+    t0 = time.time()
+    ms_total = timed(step, args.steps)
+    t1 = time.time()
+    prof = binding.bigmac_profile_read(layer.handle)
+    binding.bigmac_profile_enable(layer.handle, False)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    ms_step = ms_total / args.steps
+    value = world * w.T / (ms_step * 1e-3)
+
+    # forward only (inference forward: nothing saved)
+    def fwd_only():
+        layer.forward(x, dev, y=y, training=False)
+    for _ in range(3):
+        fwd_only()
+    ms_fwd = timed(fwd_only, args.steps) / args.steps
+
+    # ---- end to end through the same calls with HOST buffers: x, dy in; y, dx out, every step
+    def e2e_step():
+        x.copy_(hx, non_blocking=True)
+        dy.copy_(hdy, non_blocking=True)
+        step()
+        hy.copy_(y, non_blocking=True)
+        hdx.copy_(dx, non_blocking=True)
+    for _ in range(2):
+        e2e_step()
+    e2e_steps = max(2, min(args.steps, 10))
+    ms_e2e = timed(e2e_step, e2e_steps) / e2e_steps
+    if layer.status() != 0:
+        raise RuntimeError("device status word reports a timed-out wait")
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    esz = 2 if w.dtype == wl.DTYPE_BF16 else 4
+    stages = {}
+    gemm_ms = gemm_flops = 0.0
+    for name, (ms, calls) in prof["stages"].items():
+        per = ms / calls
+        entry = {"ms": round(per, 4), "launches_per_step": calls // args.steps}
+        if name in GEMM_FLOPS:
+            fl = GEMM_FLOPS[name](w)
+            entry["tflops"] = round(fl / (per * 1e-3) / 1e12, 1)
+            entry["frac_of_measured_sustained"] = round(entry["tflops"] / peaks["tflops_sustained"], 3)
+            gemm_ms += ms
+            gemm_flops += fl * calls
+        elif name in ROW_MOVE_BYTES:
+            by = ROW_MOVE_BYTES[name](w, esz)
+            entry["gbs"] = round(by / (per * 1e-3) / 1e9, 1)
+            entry["frac_of_measured_hbm"] = round(entry["gbs"] / peaks["hbm_gbs"], 3)
+        stages[name] = entry
+    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    fwd_fl = forward_flops(w)
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (tcgen05 contractions, all 15 launches of a step)",
+                "achieved": round(achieved, 1), "peak": peaks["tflops_sustained"], "unit": "TFLOP/s",
+                "frac": round(achieved / peaks["tflops_sustained"], 4), "traffic": None,
+                "peak_source": f"{peaks['source']}: sustained bf16 (kernels timed inside a long step)",
+                "frac_of_burst_peak": round(achieved / peaks["tflops_burst"], 4),
+                "step_frac": round(3.0 * fwd_fl / (ms_step * 1e-3) / 1e12 / peaks["tflops_sustained"], 4)}
+
+    rate, dt, S_used, cores = oracle_sample_rate(w, inp, args.ref_tokens)
+    bytes_io = 2 * w.T * w.d * esz
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == wl.DTYPE_BF16 else "f32", "data": "synthetic",
+            "config": config_dict(w, args), "clocks": clocks,
+            "e2e": {"value": world * w.T / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": bytes_io,
+                    "d2h_bytes_per_step": bytes_io, "ms_per_step": ms_e2e},
+            "gpu_launches": prof["launches"],
+            "forward_only": {"tokens_per_s": world * w.T / (ms_fwd * 1e-3), "ms": ms_fwd,
+                             "frac_of_tensor_roofline": round(fwd_fl / (ms_fwd * 1e-3) / 1e12 / peaks["tflops_sustained"], 4)},
+            "roofline": roofline,
+            "cpu_baseline": {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"first {S_used} tokens of the workload, routing + forward + backward with "
+                                       f"every gradient, {dt:.1f} s"},
+            "exchange_bytes": {"bigmac_width_r": 2 * (w.T + w.N) * w.r * esz, "cdac_width_d": 2 * (w.T + w.N) * w.d * esz},
+            "stages": stages}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="large", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--tokens", type=int, default=0, help="override T (per GPU)")
+    ap.add_argument("--ref-tokens", type=int, default=64, help="token sample of the CPU-oracle leg")
+    args = ap.parse_args()
+    w = wl.WORKLOADS[args.config]
+    if args.tokens:
+        w = w.with_tokens(args.tokens)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -163,6 +163,23 @@ const char *bigmac_status_string(int status);
 int bigmac_exchange_rows(bigmac_layer_t *L, const void *saved, int32_t T, int32_t width, const void *src,
                          void *grouped, size_t grouped_bytes, void *dst, int which, void *stream);
 
+/* Measurement aid: per-stage device timing and a launch counter.  While enabled, every kernel the
+ * library launches is bracketed by a pair of CUDA events on the caller's stream (no synchronisation) and
+ * counted.  bigmac_profile_read synchronises `stream`, adds the elapsed time of every bracket recorded
+ * since the last read to its stage's slot and returns the totals; the bracket pool holds 8192 launches
+ * between reads, later ones are counted in `dropped` and not timed.  The paper has no counterpart. */
+#define BIGMAC_PROFILE_SLOTS 32
+typedef struct {
+    uint64_t launches;                      /* kernels launched since enable */
+    uint32_t dropped;                       /* launches not timed because the pool was full */
+    int32_t n_slots;                        /* slots in use */
+    float ms[BIGMAC_PROFILE_SLOTS];         /* summed device time per stage */
+    uint32_t calls[BIGMAC_PROFILE_SLOTS];   /* launches per stage */
+} bigmac_profile_t;
+int bigmac_profile_enable(bigmac_layer_t *L, int on);
+int bigmac_profile_read(bigmac_layer_t *L, void *stream, bigmac_profile_t *out);
+const char *bigmac_profile_slot_name(int slot);
+
 #ifdef __cplusplus
 }
 #endif

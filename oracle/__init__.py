@@ -170,10 +170,19 @@ def backward_full(inp, routing: Routing, act: int, experts=None, decide_bf16: bo
     lib().oracle_backward_shared(_p(_f32(inp["x"])), _p(_f32(inp["dy"])), _p(fwd["y_lo"]), _p(bwd["dx_lo"]),
                                  _p(routing.topk_idx), _p(bwd["dlogit"]), C.c_int(T), C.c_int(d), C.c_int(r),
                                  C.c_int(E), C.c_int(k), _p(dw_up), _p(dw_down), _p(dw_gate), _p(db_gate))
-    experts = range(E) if experts is None else experts
     dw1, dw2 = {}, {}
-    for e in experts:
-        dw1[e], dw2[e] = backward_expert(inp, routing, act, e, decide_bf16)
+    if experts is None:
+        all1 = np.empty((E, h, r)); all2 = np.empty((E, r, h))
+        lib().oracle_backward_all_experts(_p(_f32(inp["x"])), _p(_f32(inp["dy"])), _p(_f32(inp["w_down"])),
+                                          _p(_f32(inp["w1"])), _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])),
+                                          _p(routing.topk_p), _p(routing.offsets), _p(routing.slot_of_row),
+                                          C.c_int(E), C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(k), C.c_int(act),
+                                          C.c_int(int(decide_bf16)), _p(all1), _p(all2))
+        for e in range(E):
+            dw1[e], dw2[e] = all1[e], all2[e]
+    else:
+        for e in experts:
+            dw1[e], dw2[e] = backward_expert(inp, routing, act, e, decide_bf16)
     out = {"y": fwd["y"], "y_lo": fwd["y_lo"], "x_lo": fwd["x_lo"], "dx": bwd["dx"], "dx_lo": bwd["dx_lo"],
            "dlogit": bwd["dlogit"], "dw_up": dw_up, "dw_down": dw_down, "dw_gate": dw_gate,
            "db_gate": db_gate, "dw1": dw1, "dw2": dw2}

@@ -335,6 +335,17 @@ void oracle_backward_expert(const float* x, const float* dy, const float* w_down
     }
 }
 
+// dW1 [E,h,r] and dW2 [E,r,h] of every expert (experts are independent: one thread each).
+void oracle_backward_all_experts(const float* x, const float* dy, const float* w_down, const float* w1,
+                                 const float* w2, const float* w_up, const double* topk_p, const int32_t* offsets,
+                                 const int32_t* slot_of_row, int E, int d, int r, int h, int k, int act,
+                                 int decide_bf16, double* dw1, double* dw2) {
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int e = 0; e < E; ++e)
+        oracle_backward_expert(x, dy, w_down, w1, w2, w_up, topk_p, offsets, slot_of_row, e, d, r, h, k, act,
+                               decide_bf16, dw1 + (size_t)e * h * r, dw2 + (size_t)e * r * h);
+}
+
 // Gradients of the shared matrices, as sums over all tokens of outer products of per-token vectors
 // (which the caller obtains from oracle_forward_tokens / oracle_backward_tokens):
 //   dW_up[c,c'] = sum_t dy[t,c] y'[t,c'] ;  dW_down[c',c] = sum_t dx'[t,c'] x[t,c] ;

@@ -44,6 +44,14 @@ class bigmac_debug_gemm_t(C.Structure):
                 [(n, C.c_void_p) for n in ("tile_expert", "n_tiles", "poffsets")])
 
 
+BIGMAC_PROFILE_SLOTS = 32
+
+
+class bigmac_profile_t(C.Structure):
+    _fields_ = [("launches", C.c_uint64), ("dropped", C.c_uint32), ("n_slots", C.c_int32),
+                ("ms", C.c_float * BIGMAC_PROFILE_SLOTS), ("calls", C.c_uint32 * BIGMAC_PROFILE_SLOTS)]
+
+
 _lib: Optional[C.CDLL] = None
 
 
@@ -68,7 +76,11 @@ def lib() -> C.CDLL:
         L.bigmac_status_string.restype = C.c_char_p
         L.bigmac_exchange_rows.argtypes = [vp, vp, i32, i32, vp, vp, sz, vp, C.c_int, vp]
         L.bigmac_debug_gemm.argtypes = [vp, C.POINTER(bigmac_debug_gemm_t), C.c_int, vp]
-        for name in ("bigmac_layer_create", "bigmac_layer_destroy", "bigmac_workspace_bytes", "bigmac_route",
+        L.bigmac_profile_enable.argtypes = [vp, C.c_int]
+        L.bigmac_profile_read.argtypes = [vp, vp, C.POINTER(bigmac_profile_t)]
+        L.bigmac_profile_slot_name.argtypes = [C.c_int]
+        L.bigmac_profile_slot_name.restype = C.c_char_p
+        for name in ("bigmac_profile_enable", "bigmac_profile_read", "bigmac_layer_create", "bigmac_layer_destroy", "bigmac_workspace_bytes", "bigmac_route",
                      "bigmac_forward", "bigmac_backward", "bigmac_device_status", "bigmac_exchange_rows",
                      "bigmac_debug_gemm"):
             getattr(L, name).restype = C.c_int
@@ -154,6 +166,19 @@ def bigmac_exchange_rows(handle, saved, T, width, src, grouped, dst, which) -> N
     _check(lib().bigmac_exchange_rows(handle, _ptr(saved), T, width, _ptr(src), _ptr(grouped),
                                       grouped.numel() * grouped.element_size(), _ptr(dst), which, _stream()),
            "bigmac_exchange_rows")
+
+
+def bigmac_profile_enable(handle, on: bool) -> None:
+    _check(lib().bigmac_profile_enable(handle, int(on)), "bigmac_profile_enable")
+
+
+def bigmac_profile_read(handle) -> Dict[str, object]:
+    """Synchronises the current stream; returns {"launches", "dropped", "stages": {name: (ms, calls)}}."""
+    prof = bigmac_profile_t()
+    _check(lib().bigmac_profile_read(handle, _stream(), C.byref(prof)), "bigmac_profile_read")
+    stages = {lib().bigmac_profile_slot_name(i).decode(): (float(prof.ms[i]), int(prof.calls[i]))
+              for i in range(prof.n_slots) if prof.calls[i]}
+    return {"launches": int(prof.launches), "dropped": int(prof.dropped), "stages": stages}
 
 
 def bigmac_debug_gemm(handle, q: bigmac_debug_gemm_t, use_tensor_cores: bool) -> None:

@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "internal.h"
 #include "bigmac_debug.h"
@@ -17,13 +18,46 @@ struct bigmac_layer {
     int* status;        // device status word
     bool use_tc;        // bf16 contractions on tcgen05
     unsigned tc_mask;   // debug: bit i set = contraction i runs on tcgen05 (BIGMAC_TC_MASK)
+    // measurement aid
+    bool prof_on = false;
+    uint64_t launches = 0;
+    uint32_t dropped = 0;
+    std::vector<cudaEvent_t> ev;       // pool of start/stop pairs
+    std::vector<int> ev_slot;          // stage of each recorded pair
+    float ms[BIGMAC_PROFILE_SLOTS] = {};
+    uint32_t calls[BIGMAC_PROFILE_SLOTS] = {};
 };
 
 namespace {
 
 // Contraction ids (bits of tc_mask).
 enum { G_LOGITS = 0, G_DESCEND, G_EXPERT1, G_EXPERT2, G_ASCEND, G_DY_LO, G_DW_UP, G_DZ, G_DW2, G_DXG, G_DW1,
-       G_DX, G_DX_GATE, G_DW_DOWN, G_DW_GATE };
+       G_DX, G_DX_GATE, G_DW_DOWN, G_DW_GATE,
+       S_TOPK, S_TABLES, S_DISPATCH, S_COMBINE, S_COMBINE_BWD, S_GATE_BWD, S_DXLO_GATHER, S_COLSUM, S_COUNT };
+const char* const kSlotNames[S_COUNT] = {
+    "gemm_logits", "gemm_descend", "gemm_expert1", "gemm_expert2", "gemm_ascend", "gemm_dy_lo", "gemm_dw_up",
+    "gemm_dz", "gemm_dw2", "gemm_dxg", "gemm_dw1", "gemm_dx", "gemm_dx_gate", "gemm_dw_down", "gemm_dw_gate",
+    "topk", "tables", "dispatch", "combine", "combine_bwd", "gate_bwd", "dxlo_gather", "colsum"};
+constexpr size_t kEventPairs = 8192;
+
+// Counts the launches of one stage and, while profiling, brackets them with an event pair.
+struct Stage {
+    bigmac_layer* L;
+    cudaStream_t st;
+    cudaEvent_t stop = nullptr;
+    Stage(const bigmac_layer* layer, int slot, cudaStream_t stream, int kernels = 1)
+        : L(const_cast<bigmac_layer*>(layer)), st(stream) {
+        L->launches += kernels;
+        if (!L->prof_on) return;
+        const size_t i = L->ev_slot.size();
+        if (i >= kEventPairs) { L->dropped += kernels; return; }
+        L->ev_slot.push_back(slot);
+        L->calls[slot] += kernels;
+        cudaEventRecord(L->ev[2 * i], st);
+        stop = L->ev[2 * i + 1];
+    }
+    ~Stage() { if (stop) cudaEventRecord(stop, st); }
+};
 
 inline size_t esize(int dtype) { return dtype == BIGMAC_BF16 ? 2 : 4; }
 
@@ -130,6 +164,7 @@ int check_weights(const bigmac_weights_t* W) {
 }
 
 int gemm(const bigmac_layer* L, int id, const GemmArgs& g, cudaStream_t st) {
+    Stage stage(L, id, st);
     cudaError_t err;
     if (L->cfg.dtype == BIGMAC_BF16 && L->use_tc && ((L->tc_mask >> id) & 1u))
         err = gemm_tc(g, L->status, st);
@@ -155,8 +190,8 @@ int run_routing(const bigmac_layer* L, const Dims& m, const void* x, const bigma
     g.A = x; g.lda = m.d; g.B = W->w_gate; g.ldb = m.d; g.C = b.logits; g.ldc = m.E;
     g.M = m.T; g.N = m.E; g.K = m.d; g.out_f32 = true;
     BIGMAC_TRY(gemm(L, G_LOGITS, g, st));
-    BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st));
-    BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, st));
+    { Stage s(L, S_TOPK, st); BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st)); }
+    { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, st)); }
     return BIGMAC_OK;
 }
 
@@ -223,6 +258,7 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
 
 int bigmac_layer_destroy(bigmac_layer_t* L) {
     if (!L) return BIGMAC_ERR_INVALID_ARG;
+    for (cudaEvent_t e : L->ev) cudaEventDestroy(e);
     cudaFree(L->status);
     delete L;
     return BIGMAC_OK;
@@ -291,7 +327,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         g.M = m.T; g.N = m.r; g.K = m.d;
         BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
     }
-    BIGMAC_CUDA(launch_dispatch(b.x_lo, b.xg, b.tb, m.k, m.r, m.dtype, m.P, st)); // F5 dispatch at width r
+    { Stage s(L, S_DISPATCH, st); BIGMAC_CUDA(launch_dispatch(b.x_lo, b.xg, b.tb, m.k, m.r, m.dtype, m.P, st)); }  // F5 dispatch at width r
     {                                                                             // F6 a = sigma(xg W1_e^T)
         GemmArgs g;
         g.A = b.xg; g.lda = m.r; g.B = W->w1; g.ldb = m.r; g.b_stride = (int64_t)m.h * m.r;
@@ -307,7 +343,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles;
         BIGMAC_TRY(gemm(L, G_EXPERT2, g, st));
     }
-    BIGMAC_CUDA(launch_combine(b.u, b.y_lo, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st));  // F8
+    { Stage s(L, S_COMBINE, st); BIGMAC_CUDA(launch_combine(b.u, b.y_lo, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st)); }  // F8
     {                                                                             // F9 ascend: y = y' W'_up
         GemmArgs g;
         g.A = b.y_lo; g.lda = m.r; g.B = W->w_up; g.ldb = m.r; g.C = y; g.ldc = m.d;
@@ -356,8 +392,8 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         BIGMAC_TRY(gemm(L, G_DW_UP, g, st));
     }
     // du = p dy'[t], dp = <dy'[t], u>; then the softmax-over-k backward
-    BIGMAC_CUDA(launch_combine_bwd(b.dy_lo, b.u, b.du, b.dp, b.tb, m.k, m.r, m.dtype, m.P, st));
-    BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, m.k, m.dtype, st));
+    { Stage s(L, S_COMBINE_BWD, st); BIGMAC_CUDA(launch_combine_bwd(b.dy_lo, b.u, b.du, b.dp, b.tb, m.k, m.r, m.dtype, m.P, st)); }
+    { Stage s(L, S_GATE_BWD, st); BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, m.k, m.dtype, st)); }
     {   // dz = (du W2_e) * sigma'(z), written over z
         GemmArgs g;
         g.A = b.du; g.lda = m.r; g.B = W->w2; g.ldb = m.h; g.b_kmajor = false; g.b_stride = (int64_t)m.r * m.h;
@@ -389,7 +425,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         BIGMAC_TRY(gemm(L, G_DW1, g, st));
     }
     // dx'[t] = sum_j dxg[row of slot (t,j)]   (the transpose of the dispatch gather)
-    BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st));
+    { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st)); }
     {   // dx = dx' W_down
         GemmArgs g;
         g.A = b.dx_lo; g.lda = m.r; g.B = W->w_down; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
@@ -414,7 +450,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.C = G->dw_gate; g.ldc = m.d; g.M = m.E; g.N = m.d; g.K = m.T; g.accumulate = acc;
         BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
     }
-    if (G->db_gate) BIGMAC_CUDA(launch_colsum(b.dlogits, G->db_gate, m.T, m.E, m.E64, m.dtype, acc, st));
+    if (G->db_gate) { Stage s(L, S_COLSUM, st); BIGMAC_CUDA(launch_colsum(b.dlogits, G->db_gate, m.T, m.E, m.E64, m.dtype, acc, st)); }
     return BIGMAC_OK;
 }
 
@@ -457,11 +493,47 @@ int bigmac_exchange_rows(bigmac_layer_t* L, const void* saved, int32_t T, int32_
     Carver cv(const_cast<void*>(saved));
     carve_saved(cv, m, b, true);
     cudaStream_t st = (cudaStream_t)stream;
-    if (which != 1) BIGMAC_CUDA(launch_dispatch(src, grouped, b.tb, m.k, width, m.dtype, m.P, st));
-    if (which != 0)
+    if (which != 1) { Stage s(L, S_DISPATCH, st); BIGMAC_CUDA(launch_dispatch(src, grouped, b.tb, m.k, width, m.dtype, m.P, st)); }
+    if (which != 0) {
+        Stage s(L, S_COMBINE, st);
         BIGMAC_CUDA(launch_combine(grouped, dst, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, width, m.dtype, st));
+    }
     return BIGMAC_OK;
 }
+
+int bigmac_profile_enable(bigmac_layer_t* L, int on) {
+    if (!L) return BIGMAC_ERR_INVALID_ARG;
+    if (on && L->ev.empty()) {
+        L->ev.resize(2 * kEventPairs);
+        for (cudaEvent_t& e : L->ev)
+            if (cudaEventCreate(&e) != cudaSuccess) return BIGMAC_ERR_CUDA;
+    }
+    L->prof_on = on != 0;
+    L->launches = 0;
+    L->dropped = 0;
+    L->ev_slot.clear();
+    std::memset(L->ms, 0, sizeof(L->ms));
+    std::memset(L->calls, 0, sizeof(L->calls));
+    return BIGMAC_OK;
+}
+
+int bigmac_profile_read(bigmac_layer_t* L, void* stream, bigmac_profile_t* out) {
+    if (!L || !out) return BIGMAC_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BIGMAC_ERR_CUDA;
+    for (size_t i = 0; i < L->ev_slot.size(); ++i) {
+        float ms = 0.0f;
+        if (cudaEventElapsedTime(&ms, L->ev[2 * i], L->ev[2 * i + 1]) == cudaSuccess) L->ms[L->ev_slot[i]] += ms;
+    }
+    L->ev_slot.clear();
+    out->launches = L->launches;
+    out->dropped = L->dropped;
+    out->n_slots = S_COUNT;
+    std::memcpy(out->ms, L->ms, sizeof(L->ms));
+    std::memcpy(out->calls, L->calls, sizeof(L->calls));
+    return BIGMAC_OK;
+}
+
+const char* bigmac_profile_slot_name(int slot) { return slot >= 0 && slot < S_COUNT ? kSlotNames[slot] : ""; }
 
 // ---- debug / unit-test entry point (declared in bigmac_debug.h) --------------------------------------
 int bigmac_debug_gemm(bigmac_layer_t* L, const bigmac_debug_gemm_t* q, int use_tensor_cores, void* stream) {
@@ -472,6 +544,7 @@ int bigmac_debug_gemm(bigmac_layer_t* L, const bigmac_debug_gemm_t* q, int use_t
     g.out_f32 = q->out_f32 != 0; g.accumulate = q->accumulate != 0; g.epilogue = q->epilogue; g.act = q->act;
     g.group = q->group; g.num_experts = q->num_experts; g.b_stride = q->b_stride; g.c_stride = q->c_stride;
     g.tile_expert = q->tile_expert; g.n_tiles = q->n_tiles; g.poffsets = q->poffsets;
+    L->launches += 1;
     cudaError_t err = use_tensor_cores ? gemm_tc(g, L->status, (cudaStream_t)stream)
                                        : gemm_simt(g, L->cfg.dtype, (cudaStream_t)stream);
     return err == cudaSuccess ? BIGMAC_OK : BIGMAC_ERR_CUDA;

@@ -24,6 +24,8 @@ from __future__ import annotations
 from dataclasses import dataclass, replace
 from typing import Dict, Optional
 
+import os
+
 import numpy as np
 
 ACT_RELU, ACT_GELU_ERF, ACT_GELU_TANH, ACT_IDENTITY = 0, 1, 2, 3
@@ -70,13 +72,29 @@ DECODE_TOKEN_COUNTS = (1, 8, 64, 512)
 _TAGS = {"x": 1, "dy": 2, "w_gate": 3, "w_down": 4, "w1": 5, "w2": 6, "w_up": 7}
 
 
-def bf16_round(a: np.ndarray) -> np.ndarray:
+def _round_chunk_inplace(bits: np.ndarray) -> None:
+    step = 1 << 20                                  # cache-sized pieces, no full-size temporaries
+    for i in range(0, bits.size, step):
+        b = bits[i:i + step]
+        lsb = (b >> np.uint32(16)) & np.uint32(1)
+        b += np.uint32(0x7FFF)
+        b += lsb
+        b &= np.uint32(0xFFFF0000)
+
+
+def bf16_round(a: np.ndarray, inplace: bool = False) -> np.ndarray:
     """Round float32 values to the nearest bf16 value (ties to even); result stays float32."""
-    a = np.ascontiguousarray(a, dtype=np.float32)
-    bits = a.view(np.uint32)
-    lsb = (bits >> np.uint32(16)) & np.uint32(1)
-    rounded = (bits + np.uint32(0x7FFF) + lsb) & np.uint32(0xFFFF0000)
-    return rounded.view(np.float32)
+    out = a if inplace and a.dtype == np.float32 and a.flags.c_contiguous else np.array(a, dtype=np.float32, order="C", copy=True)
+    flat = out.reshape(-1).view(np.uint32)
+    if flat.size < (1 << 22):
+        _round_chunk_inplace(flat)
+    else:                                           # numpy releases the GIL inside ufuncs
+        from concurrent.futures import ThreadPoolExecutor
+        n = min(16, os.cpu_count() or 1)
+        bounds = np.linspace(0, flat.size, n + 1).astype(np.int64)
+        with ThreadPoolExecutor(n) as pool:
+            list(pool.map(lambda i: _round_chunk_inplace(flat[bounds[i]:bounds[i + 1]]), range(n)))
+    return out
 
 
 def to_bf16_bits(a: np.ndarray) -> np.ndarray:
@@ -95,7 +113,7 @@ def _normal(seed: int, tag: int, attempt: int, shape, std: float, dtype: int) ->
     a = gen.standard_normal(size=shape, dtype=np.float32)
     if std != 1.0:
         a *= np.float32(std)
-    return bf16_round(a) if dtype == DTYPE_BF16 else a
+    return bf16_round(a, inplace=True) if dtype == DTYPE_BF16 else a
 
 
 def zipf_log_popularity(E: int, s: float = 1.1) -> np.ndarray:
