@@ -233,6 +233,15 @@ def run_ours(args, w):
             dist.all_reduce(ms, op=dist.ReduceOp.MAX)
         return float(ms.item())
 
+    if args.profile_run:                    # bare loop for a profiler: warm-up and K steps, nothing else
+        for _ in range(args.warmup + args.steps):
+            step()
+        torch.cuda.synchronize()
+        if layer.status() != 0:
+            raise RuntimeError("device status word reports a timed-out wait")
+        print(json.dumps({"profile_run": True, "config": config_dict(w, args), "steps": args.steps,
+                          "warmup": args.warmup}))
+        return
     sampler = ClockSampler(local) if rank == 0 else None
     t_warm = time.time()
     for _ in range(max(args.warmup, 3)):
@@ -337,6 +346,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="large", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0, help="override T (per GPU)")
+    ap.add_argument("--profile-run", action="store_true",
+                    help="only run warm-up + K steps (for a kernel-list or counter capture); prints no bench line")
     ap.add_argument("--ref-tokens", type=int, default=64, help="token sample of the CPU-oracle leg")
     args = ap.parse_args()
     w = wl.WORKLOADS[args.config]
