@@ -54,7 +54,8 @@ typedef enum {
     BIGMAC_ERR_WORKSPACE = -3,
     BIGMAC_ERR_CUDA = -4,
     BIGMAC_ERR_TIMEOUT = -5,
-    BIGMAC_ERR_STATE = -6
+    BIGMAC_ERR_STATE = -6,
+    BIGMAC_ERR_TOO_LARGE = -7 /* problem exceeds the fixed scratch of bigmac_route_static */
 } bigmac_status_t;
 
 typedef enum { BIGMAC_F32 = 0, BIGMAC_BF16 = 1 } bigmac_dtype_t;
@@ -162,6 +163,31 @@ const char *bigmac_status_string(int status);
  * 1 = combine only (grouped must hold data), 2 = both. */
 int bigmac_exchange_rows(bigmac_layer_t *L, const void *saved, int32_t T, int32_t width, const void *src,
                          void *grouped, size_t grouped_bytes, void *dst, int which, void *stream);
+
+/* bigmac_route for callers that cannot provide scratch memory.  (The paper has no counterpart: this is
+ * a deployment variant of the routing step, not part of the method.)
+ *
+ * Who needs it: a host program that has handed all free device memory to its own pool, a latency-critical
+ * loop that must not run into cudaMalloc's implicit device synchronisation, or a plug-in that is given
+ * nothing but input and output pointers and has no allocator to ask.  Such callers cannot size and
+ * allocate the `scratch` buffer that bigmac_route wants.  This entry point computes exactly the same tables
+ * from the same inputs, but keeps its intermediates (gate logits, counting-sort counters, the internal
+ * padded tables) in a fixed array of BIGMAC_STATIC_SCRATCH_BYTES that is part of the library image: every
+ * GPU that loads the library holds that much memory until the process exits.
+ *
+ *  - It allocates nothing: no cudaMalloc / cudaFree, no allocating library routine.  The caller still passes
+ *    x, the weights and the output tables (device memory, as for bigmac_route).
+ *  - Limit: the routing intermediates of (T, E, k) must fit the array, roughly
+ *    4*T*E + 20*T*k + 5*E*(T*k/1024 + 130) bytes; a larger problem is rejected with BIGMAC_ERR_TOO_LARGE and
+ *    nothing is launched.
+ *  - The first call on a device resolves the array's device address (once per device, with that device
+ *    current); make that first call before any stream capture.
+ *  - All calls share the one array, and it keeps the previous call's contents (everything a call reads it
+ *    has written itself first).  Two calls that overlap on the GPU - different streams, or different
+ *    handles - race on it: serialise them. */
+#define BIGMAC_STATIC_SCRATCH_BYTES (8u << 20)
+int bigmac_route_static(bigmac_layer_t *L, const void *x, int32_t T, const bigmac_weights_t *W,
+                        bigmac_routing_t *out, void *stream);
 
 /* Measurement aid: per-stage device timing and a launch counter.  While enabled, every kernel the
  * library launches is bracketed by a pair of CUDA events on the caller's stream (no synchronisation) and

@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
         L.bigmac_status_string.restype = C.c_char_p
         L.bigmac_exchange_rows.argtypes = [vp, vp, i32, i32, vp, vp, sz, vp, C.c_int, vp]
         L.bigmac_debug_gemm.argtypes = [vp, C.POINTER(bigmac_debug_gemm_t), C.c_int, vp]
+        L.bigmac_route_static.argtypes = [vp, vp, i32, C.POINTER(bigmac_weights_t), C.POINTER(bigmac_routing_t), vp]
+        L.bigmac_route_static.restype = C.c_int
         L.bigmac_profile_enable.argtypes = [vp, C.c_int]
         L.bigmac_profile_read.argtypes = [vp, vp, C.POINTER(bigmac_profile_t)]
         L.bigmac_profile_slot_name.argtypes = [C.c_int]
@@ -144,6 +146,14 @@ def _routing(R: Optional[Dict[str, torch.Tensor]]):
 def bigmac_route(handle, x, T, W, routing, scratch) -> None:
     _check(lib().bigmac_route(handle, _ptr(x), T, C.byref(_weights(W)), _routing(routing), _ptr(scratch),
                               scratch.numel() * scratch.element_size(), _stream()), "bigmac_route")
+
+
+def bigmac_route_static(handle, x, T, W, routing) -> None:
+    """bigmac_route without a scratch buffer: intermediates live in the library's fixed device array
+    (BIGMAC_STATIC_SCRATCH_BYTES).  For callers that cannot allocate device memory; raises BigmacError with
+    status -7 if (T, E, k) does not fit.  Calls must not overlap on the GPU (they share the array)."""
+    _check(lib().bigmac_route_static(handle, _ptr(x), T, C.byref(_weights(W)), _routing(routing), _stream()),
+           "bigmac_route_static")
 
 
 def bigmac_forward(handle, x, T, W, y, routing, saved, scratch) -> None:

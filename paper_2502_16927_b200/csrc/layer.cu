@@ -4,6 +4,7 @@
 // stay on the device.
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -473,6 +474,7 @@ const char* bigmac_status_string(int status) {
         case BIGMAC_ERR_CUDA: return "CUDA error";
         case BIGMAC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
         case BIGMAC_ERR_STATE: return "handle used on the wrong device";
+        case BIGMAC_ERR_TOO_LARGE: return "problem exceeds the fixed scratch array of bigmac_route_static";
         default: return "unknown status";
     }
 }
@@ -499,6 +501,77 @@ int bigmac_exchange_rows(bigmac_layer_t* L, const void* saved, int32_t T, int32_
         BIGMAC_CUDA(launch_combine(grouped, dst, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, width, m.dtype, st));
     }
     return BIGMAC_OK;
+}
+
+}  // extern "C"
+
+// ---- routing without caller-provided scratch ----------------------------------------------------------
+// The intermediates of the routing step live in this file-scope device array.  In host code its name is
+// only a stand-in for the symbol, never a device address: the address is resolved once per device with
+// cudaGetSymbolAddress (with that device current) and that pointer is what the kernels are given.
+static __device__ __align__(256) unsigned char g_route_static_scratch[BIGMAC_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};
+
+// Device address of the array on the current device (which the caller has checked to be `device`).
+int static_scratch_address(int device, void** ptr) {
+    if (device < 0 || device >= kMaxDevices) return BIGMAC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_route_static_scratch) != cudaSuccess || !p) return BIGMAC_ERR_CUDA;
+        g_static_ptr[device] = p;
+    }
+    *ptr = g_static_ptr[device];
+    return BIGMAC_OK;
+}
+
+// Only what routing needs: logits, counting-sort counters and the tables (no float intermediates).
+void carve_route_only(Carver& cv, const Dims& m, Buffers& b) {
+    carve_route_scratch(cv, m, b);
+    b.tb.topk_idx = cv.take<int32_t>(m.N);
+    b.tb.topk_w = cv.take<float>(m.N);
+    b.tb.counts = cv.take<int32_t>(m.E);
+    b.tb.offsets = cv.take<int32_t>(m.E + 1);
+    b.tb.poffsets = cv.take<int32_t>(m.E + 1);
+    b.tb.row_of_slot = cv.take<int32_t>(m.N);
+    b.tb.slot_of_row = cv.take<int32_t>(m.N);
+    b.tb.prow_of_slot = cv.take<int32_t>(m.N);
+    b.tb.slot_of_prow = cv.take<int32_t>(m.P);
+    b.tb.tile_expert = cv.take<int32_t>(m.P / kPad);
+    b.tb.n_tiles = cv.take<int32_t>(1);
+}
+
+}  // namespace
+
+extern "C" {
+
+int bigmac_route_static(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_weights_t* W,
+                        bigmac_routing_t* out, void* stream) {
+    BIGMAC_TRY(check_call(L, T));
+    if (!out) return BIGMAC_ERR_INVALID_ARG;
+    BIGMAC_TRY(check_weights(W));
+    if (T == 0) return BIGMAC_OK;
+    if (!x || !aligned(x, 16)) return BIGMAC_ERR_INVALID_ARG;
+    const Dims m = dims_of(L->cfg, T);
+    {
+        Carver measure(nullptr);
+        Buffers b{};
+        carve_route_only(measure, m, b);
+        if (measure.total() > (size_t)BIGMAC_STATIC_SCRATCH_BYTES) return BIGMAC_ERR_TOO_LARGE;
+    }
+    void* base = nullptr;
+    BIGMAC_TRY(static_scratch_address(L->device, &base));
+    Carver cv(base);
+    Buffers b{};
+    carve_route_only(cv, m, b);
+    cudaStream_t st = (cudaStream_t)stream;
+    BIGMAC_TRY(run_routing(L, m, x, W, b, st));
+    return export_routing(m, b, out, st);
 }
 
 int bigmac_profile_enable(bigmac_layer_t* L, int on) {
