@@ -82,10 +82,10 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
             const int64_t off = c_base + (int64_t)gm * g.ldc + gn;
             float v = acc[i][j];
             if (g.epilogue == EPI_ACT) {
-                if (g.Z) ((T*)g.Z)[off] = (T)v;
+                if (g.Z) ((T*)g.Z)[off] = (T)act_grad(g.act, v);
                 v = act_apply(g.act, v);
             } else if (g.epilogue == EPI_DACT) {
-                v *= act_grad(g.act, (float)((const T*)g.Z)[off]);
+                v *= (float)((const T*)g.Z)[off];
             }
             if (g.out_f32) {
                 float* C = (float*)g.C;

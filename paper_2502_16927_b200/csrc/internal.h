@@ -26,13 +26,13 @@ constexpr int kMaxExperts = 1024;
 enum GroupMode { GROUP_NONE = 0, GROUP_M = 1, GROUP_K = 2 };
 enum Epilogue {
     EPI_NONE = 0,   // C = acc
-    EPI_ACT = 1,    // Z = acc (if Z != nullptr), C = sigma(acc)
-    EPI_DACT = 2,   // C = acc * sigma'(Z[m,n])      (C may alias Z)
+    EPI_ACT = 1,    // Z = sigma'(acc) (if Z != nullptr), C = sigma(acc)
+    EPI_DACT = 2,   // C = acc * Z[m,n]               (Z holds sigma'(z) from the forward; C may alias Z)
 };
 
 struct GemmArgs {
     const void* A = nullptr; const void* B = nullptr; void* C = nullptr;
-    void* Z = nullptr;                  // activation input, [M, ldc] like C, element type = input dtype
+    void* Z = nullptr;                  // sigma'(z), [M, ldc] like C, element type = input dtype
     int64_t lda = 0, ldb = 0, ldc = 0;
     int M = 0, N = 0, K = 0;            // GROUP_M: M = upper bound on padded rows; GROUP_K: K = row extent of A and B
     bool a_kmajor = true, b_kmajor = true;
@@ -46,6 +46,11 @@ struct GemmArgs {
     const int32_t* tile_expert = nullptr;
     const int32_t* n_tiles = nullptr;
     const int32_t* poffsets = nullptr;
+    // Tensor-core path only, dense problems only:
+    const void* B2 = nullptr;           // second MN-major B: contraction rows k >= b2_first_k read B2[(k - b2_first_k)*ldb2 + n]
+    int64_t ldb2 = 0;
+    int b2_first_k = 0;                 // multiple of 64
+    int split_k = 1;                    // > 1: part s of the contraction writes its partial result (fp32) to C + s*M*ldc
 };
 
 // fp32-FMA GEMM for either dtype (dtype: bigmac_dtype_t of A, B, Z and - unless out_f32 - C).
@@ -53,6 +58,7 @@ cudaError_t gemm_simt(const GemmArgs& g, int dtype, cudaStream_t stream);
 // tcgen05 / TMEM / TMA GEMM, bf16 inputs, fp32 accumulation.  `status` is the device status word.
 cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream);
 bool gemm_tc_available();
+int gemm_tc_sm_count();
 
 // ---------------------------------------------------------------------------------------------
 // Routing tables held in device memory (internal superset of bigmac_routing_t).
@@ -87,17 +93,24 @@ cudaError_t launch_tables(const Tables& tb, int T, int E, int k, cudaStream_t st
 cudaError_t launch_dispatch(const void* src, void* grouped, const Tables& tb, int k, int width, int dtype,
                             int64_t max_prows, cudaStream_t stream);
 // dst[t,:] = sum_j w[t*k+j] * grouped[prow_of_slot[t*k+j],:]   (w == nullptr: unit weights), fp32 accumulation.
+// dst rows are `dst_ld` elements apart (0: dense, = width).
 cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const int32_t* prow_of_slot, int T,
-                           int k, int width, int dtype, cudaStream_t stream);
+                           int k, int width, int dtype, cudaStream_t stream, int dst_ld = 0);
 // Backward of the combine: du[prow,:] = p[s] * dy_lo[t,:] (zeros on padding), dp[s] = <dy_lo[t,:], u[prow,:]>.
 cudaError_t launch_combine_bwd(const void* dy_lo, const void* u, void* du, float* dp, const Tables& tb, int k,
                                int width, int dtype, int64_t max_prows, cudaStream_t stream);
 // Softmax-over-k backward: g = sum_i p_i dp_i, dl_j = p_j (dp_j - g); writes the dense [T,E] matrix
-// (zeros off the top-k set, and in the padding columns E..ld-1) in the dtype, rows `ld` elements apart.
-cudaError_t launch_gate_bwd(const float* dp, const Tables& tb, void* dlogits, int T, int E, int ld, int k, int dtype,
-                            cudaStream_t stream);
-// db[e] (+)= sum_t dlogits[t,e]
-cudaError_t launch_colsum(const void* dlogits, float* db, int T, int E, int ld, int dtype, bool accumulate,
-                          cudaStream_t stream);
+// (zeros off the top-k set, and in the padding columns E..width-1) in the dtype, rows `ld` elements apart.
+cudaError_t launch_gate_bwd(const float* dp, const Tables& tb, void* dlogits, int T, int E, int width, int ld, int k,
+                            int dtype, cudaStream_t stream);
+// db[e] (+)= sum_t dlogits[t,e]; `partial` holds kColsumChunks * E floats of scratch.
+constexpr int kColsumChunks = 64;
+cudaError_t launch_colsum(const void* dlogits, float* db, float* partial, int T, int E, int ld, int dtype,
+                          bool accumulate, cudaStream_t stream);
+// Sum the `parts` fp32 partial results ws[s][m][n] of a split contraction in the order s = 0, 1, ... and write
+// rows [0, m_split) to dst1 [m_split, N] and rows [m_split, m_split + m2) to dst2 [m2, N] (dst2 may be null),
+// in the dtype, adding to the destination if `accumulate`.
+cudaError_t launch_splitk_reduce(const float* ws, int parts, int M, int N, void* dst1, int m_split, void* dst2, int m2,
+                                 int dtype, bool accumulate, cudaStream_t stream);
 
 }  // namespace bigmac

@@ -34,12 +34,15 @@ namespace {
 // Contraction ids (bits of tc_mask).
 enum { G_LOGITS = 0, G_DESCEND, G_EXPERT1, G_EXPERT2, G_ASCEND, G_DY_LO, G_DW_UP, G_DZ, G_DW2, G_DXG, G_DW1,
        G_DX, G_DX_GATE, G_DW_DOWN, G_DW_GATE,
-       S_TOPK, S_TABLES, S_DISPATCH, S_COMBINE, S_COMBINE_BWD, S_GATE_BWD, S_DXLO_GATHER, S_COLSUM, S_COUNT };
+       S_TOPK, S_TABLES, S_DISPATCH, S_COMBINE, S_COMBINE_BWD, S_GATE_BWD, S_DXLO_GATHER, S_COLSUM, S_SPLITK_REDUCE,
+       S_COUNT };
 const char* const kSlotNames[S_COUNT] = {
     "gemm_logits", "gemm_descend", "gemm_expert1", "gemm_expert2", "gemm_ascend", "gemm_dy_lo", "gemm_dw_up",
     "gemm_dz", "gemm_dw2", "gemm_dxg", "gemm_dw1", "gemm_dx", "gemm_dx_gate", "gemm_dw_down", "gemm_dw_gate",
-    "topk", "tables", "dispatch", "combine", "combine_bwd", "gate_bwd", "dxlo_gather", "colsum"};
+    "topk", "tables", "dispatch", "combine", "combine_bwd", "gate_bwd", "dxlo_gather", "colsum",
+    "splitk_reduce"};
 constexpr size_t kEventPairs = 8192;
+constexpr int kMaxSplitK = 8;
 
 // Counts the launches of one stage and, while profiling, brackets them with an event pair.
 struct Stage {
@@ -81,7 +84,11 @@ struct Buffers {
     Tables tb;
     float* logits;
     void *x_lo, *xg, *z, *a, *u, *y_lo;                 // forward intermediates
-    void *dy_lo, *du, *dxg, *dx_lo, *dlogits; float* dp; // backward intermediates
+    void *dy_lo, *du, *dxg; float* dp;                   // backward intermediates
+    void* dcat;          // [T, r + E64]: dx' in columns [0, r), the dense gate gradient dl in columns [r, r + E64)
+    void *dx_lo, *dlogits;                               // views into dcat (row stride r + E64)
+    float* colsum_part;  // [kColsumChunks, E]
+    float* splitk_ws;    // fp32 partial results of the split weight-gradient contractions
 };
 
 struct Dims {
@@ -129,9 +136,12 @@ void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
     b.dy_lo = cv.take_bytes((size_t)m.T * m.r * es);
     b.du = cv.take_bytes((size_t)m.P * m.r * es);
     b.dxg = cv.take_bytes((size_t)m.P * m.r * es);
-    b.dx_lo = cv.take_bytes((size_t)m.T * m.r * es);
-    b.dlogits = cv.take_bytes((size_t)m.T * m.E64 * es);
+    b.dcat = cv.take_bytes((size_t)m.T * (m.r + m.E64) * es);
+    b.dx_lo = b.dcat;
+    b.dlogits = b.dcat ? (char*)b.dcat + (size_t)m.r * es : nullptr;
     b.dp = cv.take<float>(m.N);
+    b.colsum_part = cv.take<float>((size_t)kColsumChunks * m.E);
+    b.splitk_ws = cv.take<float>((size_t)kMaxSplitK * (m.r + m.E64) * m.d);
 }
 
 size_t forward_scratch_bytes(const Dims& m, bool training) {
@@ -172,6 +182,21 @@ int gemm(const bigmac_layer* L, int id, const GemmArgs& g, cudaStream_t st) {
     else
         err = gemm_simt(g, L->cfg.dtype, st);
     return err == cudaSuccess ? BIGMAC_OK : BIGMAC_ERR_CUDA;
+}
+
+// Number of parts to cut a dense contraction of `num_kb` k slices into so that tiles * parts fills the SMs:
+// minimises waves * slices-per-part (ties: fewer parts).
+int choose_split_k(int M, int N, int K) {
+    const int bn = N >= 256 ? 256 : 128;
+    const int64_t tiles = (int64_t)((M + 127) / 128) * ((N + bn - 1) / bn);
+    const int num_kb = (K + 63) / 64, sms = gemm_tc_sm_count();
+    int best = 1;
+    int64_t best_cost = -1;
+    for (int s = 1; s <= kMaxSplitK && s <= num_kb; ++s) {
+        const int64_t cost = ((tiles * s + sms - 1) / sms) * ((num_kb + s - 1) / s);
+        if (best_cost < 0 || cost < best_cost) { best = s; best_cost = cost; }
+    }
+    return best;
 }
 
 #define BIGMAC_TRY(expr)                        \
@@ -329,7 +354,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
     }
     { Stage s(L, S_DISPATCH, st); BIGMAC_CUDA(launch_dispatch(b.x_lo, b.xg, b.tb, m.k, m.r, m.dtype, m.P, st)); }  // F5 dispatch at width r
-    {                                                                             // F6 a = sigma(xg W1_e^T)
+    {                                                                             // F6 a = sigma(xg W1_e^T); saves sigma'(z)
         GemmArgs g;
         g.A = b.xg; g.lda = m.r; g.B = W->w1; g.ldb = m.r; g.b_stride = (int64_t)m.h * m.r;
         g.C = b.a; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
@@ -386,16 +411,25 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.M = m.T; g.N = m.r; g.K = m.d;
         BIGMAC_TRY(gemm(L, G_DY_LO, g, st));
     }
+    const bool fused = L->cfg.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u;
+    const int ldcat = m.r + m.E64;
     if (G->dw_up) {   // dW_up[c,c'] = sum_t dy[t,c] y'[t,c']
         GemmArgs g;
         g.A = dy; g.lda = m.d; g.a_kmajor = false; g.B = b.y_lo; g.ldb = m.r; g.b_kmajor = false;
         g.C = G->dw_up; g.ldc = m.r; g.M = m.d; g.N = m.r; g.K = m.T; g.accumulate = acc;
-        BIGMAC_TRY(gemm(L, G_DW_UP, g, st));
+        if (fused) {   // contraction over all tokens, few output tiles: split it, reduce the parts in order
+            g.split_k = choose_split_k(g.M, g.N, g.K); g.C = b.splitk_ws; g.out_f32 = true; g.accumulate = false;
+            BIGMAC_TRY(gemm(L, G_DW_UP, g, st));
+            Stage s(L, S_SPLITK_REDUCE, st);
+            BIGMAC_CUDA(launch_splitk_reduce(b.splitk_ws, g.split_k, m.d, m.r, G->dw_up, m.d, nullptr, 0, m.dtype, acc, st));
+        } else {
+            BIGMAC_TRY(gemm(L, G_DW_UP, g, st));
+        }
     }
     // du = p dy'[t], dp = <dy'[t], u>; then the softmax-over-k backward
     { Stage s(L, S_COMBINE_BWD, st); BIGMAC_CUDA(launch_combine_bwd(b.dy_lo, b.u, b.du, b.dp, b.tb, m.k, m.r, m.dtype, m.P, st)); }
-    { Stage s(L, S_GATE_BWD, st); BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, m.k, m.dtype, st)); }
-    {   // dz = (du W2_e) * sigma'(z), written over z
+    { Stage s(L, S_GATE_BWD, st); BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, ldcat, m.k, m.dtype, st)); }
+    {   // dz = (du W2_e) * sigma'(z); the forward saved sigma'(z) in the z buffer, dz is written over it
         GemmArgs g;
         g.A = b.du; g.lda = m.r; g.B = W->w2; g.ldb = m.h; g.b_kmajor = false; g.b_stride = (int64_t)m.r * m.h;
         g.C = b.z; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
@@ -426,32 +460,52 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         BIGMAC_TRY(gemm(L, G_DW1, g, st));
     }
     // dx'[t] = sum_j dxg[row of slot (t,j)]   (the transpose of the dispatch gather)
-    { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st)); }
-    {   // dx = dx' W_down
-        GemmArgs g;
-        g.A = b.dx_lo; g.lda = m.r; g.B = W->w_down; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
-        g.M = m.T; g.N = m.d; g.K = m.r;
-        BIGMAC_TRY(gemm(L, G_DX, g, st));
+    { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st, ldcat)); }
+    if (fused) {
+        {   // dx = [dx' | dl] [W_down ; W_gate]: one contraction over r + E
+            GemmArgs g;
+            g.A = b.dcat; g.lda = ldcat; g.B = W->w_down; g.ldb = m.d; g.b_kmajor = false;
+            g.B2 = W->w_gate; g.ldb2 = m.d; g.b2_first_k = m.r;
+            g.C = dx; g.ldc = m.d; g.M = m.T; g.N = m.d; g.K = m.r + m.E;
+            BIGMAC_TRY(gemm(L, G_DX, g, st));
+        }
+        if (G->dw_down || G->dw_gate) {   // [dW_down ; dW_gate] = [dx' | dl]^T x: x is read once for both
+            GemmArgs g;
+            g.A = b.dcat; g.lda = ldcat; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
+            g.C = b.splitk_ws; g.ldc = m.d; g.out_f32 = true; g.M = ldcat; g.N = m.d; g.K = m.T;
+            g.split_k = choose_split_k(g.M, g.N, g.K);
+            BIGMAC_TRY(gemm(L, G_DW_DOWN, g, st));
+            Stage s(L, S_SPLITK_REDUCE, st);
+            BIGMAC_CUDA(launch_splitk_reduce(b.splitk_ws, g.split_k, ldcat, m.d, G->dw_down, m.r, G->dw_gate, m.E, m.dtype,
+                                             acc, st));
+        }
+    } else {
+        {   // dx = dx' W_down
+            GemmArgs g;
+            g.A = b.dx_lo; g.lda = ldcat; g.B = W->w_down; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
+            g.M = m.T; g.N = m.d; g.K = m.r;
+            BIGMAC_TRY(gemm(L, G_DX, g, st));
+        }
+        {   // dx += dl W_gate
+            GemmArgs g;
+            g.A = b.dlogits; g.lda = ldcat; g.B = W->w_gate; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
+            g.M = m.T; g.N = m.d; g.K = m.E; g.accumulate = true;
+            BIGMAC_TRY(gemm(L, G_DX_GATE, g, st));
+        }
+        if (G->dw_down) {   // dW_down[c',c] = sum_t dx'[t,c'] x[t,c]
+            GemmArgs g;
+            g.A = b.dx_lo; g.lda = ldcat; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
+            g.C = G->dw_down; g.ldc = m.d; g.M = m.r; g.N = m.d; g.K = m.T; g.accumulate = acc;
+            BIGMAC_TRY(gemm(L, G_DW_DOWN, g, st));
+        }
+        if (G->dw_gate) {   // dW_gate[e,c] = sum_t dl[t,e] x[t,c]
+            GemmArgs g;
+            g.A = b.dlogits; g.lda = ldcat; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
+            g.C = G->dw_gate; g.ldc = m.d; g.M = m.E; g.N = m.d; g.K = m.T; g.accumulate = acc;
+            BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
+        }
     }
-    {   // dx += dl W_gate
-        GemmArgs g;
-        g.A = b.dlogits; g.lda = m.E64; g.B = W->w_gate; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
-        g.M = m.T; g.N = m.d; g.K = m.E; g.accumulate = true;
-        BIGMAC_TRY(gemm(L, G_DX_GATE, g, st));
-    }
-    if (G->dw_down) {   // dW_down[c',c] = sum_t dx'[t,c'] x[t,c]
-        GemmArgs g;
-        g.A = b.dx_lo; g.lda = m.r; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
-        g.C = G->dw_down; g.ldc = m.d; g.M = m.r; g.N = m.d; g.K = m.T; g.accumulate = acc;
-        BIGMAC_TRY(gemm(L, G_DW_DOWN, g, st));
-    }
-    if (G->dw_gate) {   // dW_gate[e,c] = sum_t dl[t,e] x[t,c]
-        GemmArgs g;
-        g.A = b.dlogits; g.lda = m.E64; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
-        g.C = G->dw_gate; g.ldc = m.d; g.M = m.E; g.N = m.d; g.K = m.T; g.accumulate = acc;
-        BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
-    }
-    if (G->db_gate) { Stage s(L, S_COLSUM, st); BIGMAC_CUDA(launch_colsum(b.dlogits, G->db_gate, m.T, m.E, m.E64, m.dtype, acc, st)); }
+    if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_colsum(b.dlogits, G->db_gate, b.colsum_part, m.T, m.E, ldcat, m.dtype, acc, st)); }
     return BIGMAC_OK;
 }
 

@@ -66,7 +66,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ grouped, uint4* __restrict__ dst,
                                                       const float* __restrict__ w,
                                                       const int32_t* __restrict__ prow_of_slot, int n_tokens, int k,
-                                                      int vecs_per_row) {
+                                                      int vecs_per_row, int dst_vecs_per_row) {
     constexpr int V = Vec<T>::kElems;
     const int t = warp_global_id();
     if (t >= n_tokens) return;
@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
 #pragma unroll
             for (int i = 0; i < V; ++i) acc[i] = fmaf(p, f[i], acc[i]);
         }
-        dst[(int64_t)t * vecs_per_row + c] = Vec<T>::pack(acc);
+        dst[(int64_t)t * dst_vecs_per_row + c] = Vec<T>::pack(acc);
     }
 }
 
@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const uint4* __restric
 template <typename T>
 __global__ void __launch_bounds__(256) gate_bwd_kernel(const float* __restrict__ dp, const float* __restrict__ topk_w,
                                                        const int32_t* __restrict__ topk_idx, T* __restrict__ dlogits,
-                                                       int n_tokens, int E, int ld, int k) {
+                                                       int n_tokens, int E, int width, int ld, int k) {
     const int t = warp_global_id();
     if (t >= n_tokens) return;
     const int lane = threadIdx.x & 31;
@@ -137,27 +137,58 @@ __global__ void __launch_bounds__(256) gate_bwd_kernel(const float* __restrict__
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
     T* row = dlogits + (int64_t)t * ld;
-    for (int e = lane; e < ld; e += 32) row[e] = (T)0.0f;
+    for (int e = lane; e < width; e += 32) row[e] = (T)0.0f;
     __syncwarp();
     for (int j = lane; j < k; j += 32) row[topk_idx[(int64_t)t * k + j]] = (T)(p[j] * (g[j] - part));
 }
 
+// Column sums in two deterministic stages: blockIdx.y owns a contiguous chunk of rows and writes its partial
+// sums; a second kernel adds the chunks in order.
 template <typename T>
-__global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ m, float* __restrict__ out, int rows, int cols,
-                                                     int ld, int accumulate) {
+__global__ void __launch_bounds__(256) colsum_partial_kernel(const T* __restrict__ m, float* __restrict__ partial, int rows,
+                                                             int cols, int ld) {
     __shared__ float part[8][33];
     const int c = blockIdx.x * 32 + (threadIdx.x & 31);
     const int g = threadIdx.x >> 5;
+    const int per = (rows + gridDim.y - 1) / gridDim.y;
+    const int r0 = blockIdx.y * per, r1 = min(rows, r0 + per);
     float acc = 0.0f;
     if (c < cols)
-        for (int r = g; r < rows; r += 8) acc += (float)m[(int64_t)r * ld + c];
+        for (int r = r0 + g; r < r1; r += 8) acc += (float)m[(int64_t)r * ld + c];
     part[g][threadIdx.x & 31] = acc;
     __syncthreads();
     if (g == 0 && c < cols) {
         float total = 0.0f;
         for (int i = 0; i < 8; ++i) total += part[i][threadIdx.x];
-        out[c] = accumulate ? out[c] + total : total;
+        partial[(int64_t)blockIdx.y * cols + c] = total;
     }
+}
+
+__global__ void __launch_bounds__(256) colsum_final_kernel(const float* __restrict__ partial, float* __restrict__ out, int chunks,
+                                                           int cols, int accumulate) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= cols) return;
+    float total = 0.0f;
+    for (int i = 0; i < chunks; ++i) total += partial[(int64_t)i * cols + c];
+    out[c] = accumulate ? out[c] + total : total;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ ws, int parts, int M, int N,
+                                                            T* __restrict__ dst1, int m_split, T* __restrict__ dst2, int m2,
+                                                            int accumulate) {
+    const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;     // N is a multiple of 4
+    if (i >= (int64_t)(m_split + m2) * N) return;
+    const int m = (int)(i / N);
+    float4 acc = *(const float4*)(ws + i);
+    for (int s = 1; s < parts; ++s) {
+        const float4 v = *(const float4*)(ws + (int64_t)s * M * N + i);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    T* dst = m < m_split ? dst1 + i : dst2 + (i - (int64_t)m_split * N);
+    if (!(m < m_split ? dst1 : dst2)) return;
+    if (accumulate) { acc.x += (float)dst[0]; acc.y += (float)dst[1]; acc.z += (float)dst[2]; acc.w += (float)dst[3]; }
+    dst[0] = (T)acc.x; dst[1] = (T)acc.y; dst[2] = (T)acc.z; dst[3] = (T)acc.w;
 }
 
 inline int elem_bytes(int dtype) { return dtype == BIGMAC_BF16 ? 2 : 4; }
@@ -175,15 +206,16 @@ cudaError_t launch_dispatch(const void* src, void* grouped, const Tables& tb, in
 }
 
 cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const int32_t* prow_of_slot, int T, int k,
-                           int width, int dtype, cudaStream_t stream) {
+                           int width, int dtype, cudaStream_t stream, int dst_ld) {
     if (T == 0) return cudaSuccess;
     const int vecs = width * elem_bytes(dtype) / 16;
+    const int dvecs = (dst_ld ? dst_ld : width) * elem_bytes(dtype) / 16;
     if (dtype == BIGMAC_BF16)
         combine_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, stream>>>((const uint4*)grouped, (uint4*)dst, w,
-                                                                         prow_of_slot, T, k, vecs);
+                                                                         prow_of_slot, T, k, vecs, dvecs);
     else
         combine_kernel<float><<<warp_blocks(T), 256, 0, stream>>>((const uint4*)grouped, (uint4*)dst, w, prow_of_slot,
-                                                                 T, k, vecs);
+                                                                 T, k, vecs, dvecs);
     return cudaGetLastError();
 }
 
@@ -202,24 +234,39 @@ cudaError_t launch_combine_bwd(const void* dy_lo, const void* u, void* du, float
     return cudaGetLastError();
 }
 
-cudaError_t launch_gate_bwd(const float* dp, const Tables& tb, void* dlogits, int T, int E, int ld, int k, int dtype,
-                            cudaStream_t stream) {
+cudaError_t launch_gate_bwd(const float* dp, const Tables& tb, void* dlogits, int T, int E, int width, int ld, int k,
+                            int dtype, cudaStream_t stream) {
     if (T == 0) return cudaSuccess;
     if (dtype == BIGMAC_BF16)
         gate_bwd_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, stream>>>(dp, tb.topk_w, tb.topk_idx,
-                                                                          (__nv_bfloat16*)dlogits, T, E, ld, k);
+                                                                          (__nv_bfloat16*)dlogits, T, E, width, ld, k);
     else
-        gate_bwd_kernel<float><<<warp_blocks(T), 256, 0, stream>>>(dp, tb.topk_w, tb.topk_idx, (float*)dlogits, T, E, ld, k);
+        gate_bwd_kernel<float><<<warp_blocks(T), 256, 0, stream>>>(dp, tb.topk_w, tb.topk_idx, (float*)dlogits, T, E, width, ld, k);
     return cudaGetLastError();
 }
 
-cudaError_t launch_colsum(const void* dlogits, float* db, int T, int E, int ld, int dtype, bool accumulate,
-                          cudaStream_t stream) {
-    const unsigned blocks = (unsigned)((E + 31) / 32);
+cudaError_t launch_colsum(const void* dlogits, float* db, float* partial, int T, int E, int ld, int dtype,
+                          bool accumulate, cudaStream_t stream) {
+    dim3 grid((unsigned)((E + 31) / 32), kColsumChunks);
     if (dtype == BIGMAC_BF16)
-        colsum_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)dlogits, db, T, E, ld, accumulate);
+        colsum_partial_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)dlogits, partial, T, E, ld);
     else
-        colsum_kernel<float><<<blocks, 256, 0, stream>>>((const float*)dlogits, db, T, E, ld, accumulate);
+        colsum_partial_kernel<float><<<grid, 256, 0, stream>>>((const float*)dlogits, partial, T, E, ld);
+    colsum_final_kernel<<<(unsigned)((E + 255) / 256), 256, 0, stream>>>(partial, db, kColsumChunks, E, accumulate);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_splitk_reduce(const float* ws, int parts, int M, int N, void* dst1, int m_split, void* dst2, int m2,
+                                 int dtype, bool accumulate, cudaStream_t stream) {
+    const int64_t quads = (int64_t)(m_split + m2) * N / 4;
+    if (quads == 0) return cudaSuccess;
+    const unsigned blocks = (unsigned)((quads + 255) / 256);
+    if (dtype == BIGMAC_BF16)
+        splitk_reduce_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(ws, parts, M, N, (__nv_bfloat16*)dst1, m_split,
+                                                                      (__nv_bfloat16*)dst2, m2, accumulate);
+    else
+        splitk_reduce_kernel<float><<<blocks, 256, 0, stream>>>(ws, parts, M, N, (float*)dst1, m_split, (float*)dst2, m2,
+                                                               accumulate);
     return cudaGetLastError();
 }
 

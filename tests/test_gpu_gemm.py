@@ -144,11 +144,11 @@ def test_grouped_rows_forward_and_backward_epilogues():
     for e, c in enumerate(counts):
         rows = slice(poff[e], poff[e + 1])
         z = A[rows].astype(np.float64) @ W[e].astype(np.float64).T
-        _close(got_z[rows], z)
+        _close(got_z[rows], _dgelu(z))
         _close(got_c[rows], _gelu(z))
     assert np.isnan(got_c[poff[-1]:]).all()                     # nothing beyond the live tiles is touched
 
-    # input-gradient form: K-major A, MN-major per-expert weights, multiply by sigma'(Z) in place over Z
+    # input-gradient form: K-major A, MN-major per-expert weights, multiply by the saved sigma' in place over Z
     G = np.zeros((P, N), dtype=np.float32)                       # "du": [P, N] now the contraction side
     for e, c in enumerate(counts):
         G[poff[e]:poff[e] + c] = _rand((c, N), 40 + e)
@@ -161,7 +161,7 @@ def test_grouped_rows_forward_and_backward_epilogues():
     got = _np(Zd)
     for e in range(E):
         rows = slice(poff[e], poff[e + 1])
-        ref = (G[rows].astype(np.float64) @ Wt[e].astype(np.float64)) * _dgelu(Zin[rows].astype(np.float64))
+        ref = (G[rows].astype(np.float64) @ Wt[e].astype(np.float64)) * Zin[rows].astype(np.float64)
         _close(got[rows], ref)
 
 
