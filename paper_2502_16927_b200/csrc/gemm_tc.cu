@@ -76,6 +76,9 @@ __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void ld_shared_16B(const void* ptr, uint32_t* w) {
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(smem_u32(ptr)));
+}
 __device__ __forceinline__ void st_shared_16B(void* ptr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(smem_u32(ptr)), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -211,6 +214,29 @@ __device__ __forceinline__ void act_pair(int act, float z, float& a, float& g) {
     }
 }
 
+// Activation of 32 accumulator values in place; with WITH_G the 32 sigma' values are packed to bf16 pairs in wg.
+// The activation is a compile-time constant here so that the switch is taken once per chunk, not per element.
+template <int ACT, bool WITH_G>
+__device__ __forceinline__ void act_chunk(float* v, uint32_t* wg) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        float a0, g0, a1, g1;
+        act_pair(ACT, v[2 * i], a0, g0);
+        act_pair(ACT, v[2 * i + 1], a1, g1);
+        v[2 * i] = a0; v[2 * i + 1] = a1;
+        if (WITH_G) wg[i] = pack_bf16(g0, g1);
+    }
+}
+template <bool WITH_G>
+__device__ __forceinline__ void act_chunk_any(int act, float* v, uint32_t* wg) {
+    switch (act) {
+        case BIGMAC_ACT_GELU_ERF: act_chunk<BIGMAC_ACT_GELU_ERF, WITH_G>(v, wg); break;
+        case BIGMAC_ACT_RELU: act_chunk<BIGMAC_ACT_RELU, WITH_G>(v, wg); break;
+        case BIGMAC_ACT_GELU_TANH: act_chunk<BIGMAC_ACT_GELU_TANH, WITH_G>(v, wg); break;
+        default: act_chunk<BIGMAC_ACT_IDENTITY, WITH_G>(v, wg); break;
+    }
+}
+
 // Epilogue for 32 consecutive columns [col0, col0+32) of one output row held in v[0..31].
 __device__ __forceinline__ void store_row_chunk(const TcParams& p, float* v, int64_t row_off, int col0, bool vec_ok) {
     const int ncols = min(32, p.N - col0);
@@ -221,19 +247,11 @@ __device__ __forceinline__ void store_row_chunk(const TcParams& p, float* v, int
         if (p.epilogue == EPI_ACT) {
             if (Zb) {
                 uint32_t w[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float a0, g0, a1, g1;
-                    act_pair(p.act, v[2 * i], a0, g0);
-                    act_pair(p.act, v[2 * i + 1], a1, g1);
-                    v[2 * i] = a0; v[2 * i + 1] = a1;
-                    w[i] = pack_bf16(g0, g1);
-                }
+                act_chunk_any<true>(p.act, v, w);
                 st_global_32B(Zb + off, w);
                 st_global_32B(Zb + off + 16, w + 8);
             } else {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) { float g; act_pair(p.act, v[i], v[i], g); }
+                act_chunk_any<false>(p.act, v, nullptr);
             }
         } else if (p.epilogue == EPI_DACT) {
             uint32_t w[16];
@@ -311,28 +329,12 @@ __device__ __forceinline__ void stage_row_chunk(const TcParams& p, float* v, uin
     uint32_t w[16];
     if (p.epilogue == EPI_ACT) {
         if (p.Z) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                float a0, g0, a1, g1;
-                act_pair(p.act, v[2 * i], a0, g0);
-                act_pair(p.act, v[2 * i + 1], a1, g1);
-                v[2 * i] = a0; v[2 * i + 1] = a1;
-                w[i] = pack_bf16(g0, g1);
-            }
+            act_chunk_any<true>(p.act, v, w);
             stage_row_bf16(box_z, lane, w);
         } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) { float g; act_pair(p.act, v[i], v[i], g); }
+            act_chunk_any<false>(p.act, v, nullptr);
         }
-    } else if (p.epilogue == EPI_DACT) {
-        if (row_ok) {
-            const __nv_bfloat16* zp = (const __nv_bfloat16*)p.Z + row_off + col0;
-            ld_global_32B(zp, w);
-            ld_global_32B(zp + 16, w + 8);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) { v[2 * i] *= bf16_lo(w[i]); v[2 * i + 1] *= bf16_hi(w[i]); }
-        }
-    }
+    }   // EPI_DACT: the caller has already multiplied by the prefetched sigma'
 #pragma unroll
     for (int i = 0; i < 16; ++i) w[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
     stage_row_bf16(box_c, lane, w);
@@ -387,7 +389,7 @@ constexpr int kThreadsV2 = (2 + kEpiWarps) * 32;
 // Persistent kernel: gridDim.x CTAs (one per SM) walk the tile list with stride gridDim.x.  The
 // accumulator is double-buffered in tensor memory (2 x BN columns), so the epilogue of tile i overlaps
 // the MMAs of tile i+1.
-template <int BN, int STAGES, bool A_KMAJOR, bool B_KMAJOR>
+template <int BN, int STAGES, bool A_KMAJOR, bool B_KMAJOR, bool TMA_EPI>
 __global__ void __launch_bounds__(kThreadsV2, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_z,
@@ -396,7 +398,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     constexpr uint32_t B_BYTES = BN * BK * 2;
     constexpr uint32_t CHUNK_BYTES = 64 * BK * 2;            // one 64-wide MN-major box
     constexpr uint32_t TMEM_COLS = 2 * BN;
-    constexpr uint32_t STAGING_BYTES = kEpiWarps * 2 * kBoxBytes;   // per epilogue warp: one box for C, one for Z
+    constexpr uint32_t STAGING_BYTES = TMA_EPI ? kEpiWarps * 2 * kBoxBytes : 0;   // per epilogue warp: a box for C, one for Z
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -407,7 +409,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint64_t* empty_bar = full_bar + STAGES;
     uint64_t* tmem_full_bar = empty_bar + STAGES;            // [2]
     uint64_t* tmem_empty_bar = tmem_full_bar + 2;            // [2]
-    uint32_t* tmem_slot = (uint32_t*)(tmem_empty_bar + 2);
+    uint64_t* z_bar = tmem_empty_bar + 2;                    // [kEpiWarps]: sigma' boxes prefetched by TMA (EPI_DACT)
+    uint32_t* tmem_slot = (uint32_t*)(z_bar + kEpiWarps);
     volatile int* dead = (volatile int*)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -417,6 +420,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], kEpiWarps); }
+        for (int s = 0; s < kEpiWarps; ++s) mbar_init(&z_bar[s], 1);
         *dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -506,6 +510,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int esz = p.out_f32 ? 4 : 2;
         const bool vec_ok = ((p.ldc * esz) % 32 == 0) && ((p.c_stride * esz) % 32 == 0) && (p.ldc % 16 == 0) &&
                             (((uintptr_t)p.C) % 32 == 0) && (((uintptr_t)p.Z) % 32 == 0);
+        // EPI_DACT with staged stores: the saved sigma' box of the next chunk is fetched by TMA into box_z one
+        // chunk ahead (across tiles too), so its DRAM latency is hidden behind the MMAs and the previous chunk.
+        const bool z_prefetch = TMA_EPI && p.epilogue == EPI_DACT;
+        uint64_t* my_z_bar = &z_bar[warp - 2];
+        uint32_t z_count = 0;
+        auto issue_z = [&](const Tile& tile, int c) {
+            if (lane == 0) {
+                mbar_expect_tx(my_z_bar, kBoxBytes);
+                tma_load_2d(box_z, &map_z, my_z_bar, tile.n0 + part * COLS_PER_WARP + c * 32, tile.m0 + quad * 32);
+            }
+        };
+        if (z_prefetch && (int)blockIdx.x < total) issue_z(get_tile(p, BN, blockIdx.x, tiles_m, tiles_n), 0);
         uint32_t local = 0;
         for (int t = blockIdx.x; t < total; t += gridDim.x, ++local) {
             const Tile tl = get_tile(p, BN, t, tiles_m, tiles_n);
@@ -533,9 +549,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 const int col0 = tl.n0 + part * COLS_PER_WARP + c * 32;
                 if (col0 >= p.N) continue;             // uniform across the warp
-                if (p.tma_store) {
+                if (TMA_EPI) {
                     if (lane == 0) tma_store_wait_read();        // previous boxes of this warp have left smem
                     __syncwarp();
+                    if (z_prefetch) {
+                        mbar_wait(my_z_bar, z_count & 1, dead, p.status);
+                        ++z_count;
+                        uint32_t w[16];
+                        const uint8_t* zrow = box_z + lane * 64;
+                        const int sw = (lane >> 1) & 3;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) ld_shared_16B(zrow + ((j ^ sw) << 4), w + 4 * j);
+                        fence_async_smem();
+                        __syncwarp();
+                        if (c + 1 < CHUNKS) issue_z(tl, c + 1);
+                        else if (t + (int)gridDim.x < total) issue_z(get_tile(p, BN, t + gridDim.x, tiles_m, tiles_n), 0);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { v[2 * i] *= bf16_lo(w[i]); v[2 * i + 1] *= bf16_hi(w[i]); }
+                    }
                     stage_row_chunk(p, v, box_c, box_z, lane, row_off, col0, row_ok);
                     fence_async_smem();
                     __syncwarp();
@@ -550,7 +581,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
             }
         }
-        if (lane == 0) tma_store_wait_all();
+        if (TMA_EPI && lane == 0) tma_store_wait_all();
     }
     tc_fence_before();
     __syncthreads();
@@ -602,12 +633,13 @@ int sm_count() {
     return n;
 }
 
-template <int BN, int STAGES, bool AK, bool BKM>
+template <int BN, int STAGES, bool AK, bool BKM, bool TMA_EPI>
 cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mz,
                    const CUtensorMap& mb2, const TcParams& p, int max_tiles, cudaStream_t stream) {
-    constexpr size_t smem = STAGES * (BM * BK * 2 + BN * BK * 2) + kEpiWarps * 2 * kBoxBytes + (2 * STAGES + 4) * 8 + 16 + 1024;
+    constexpr size_t smem = STAGES * (BM * BK * 2 + BN * BK * 2) + (TMA_EPI ? kEpiWarps * 2 * kBoxBytes : 0) +
+                            (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + 1024;
     static bool configured = false;
-    auto kernel = gemm_tc_kernel<BN, STAGES, AK, BKM>;
+    auto kernel = gemm_tc_kernel<BN, STAGES, AK, BKM, TMA_EPI>;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -618,7 +650,7 @@ cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorM
     return cudaGetLastError();
 }
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, bool TMA_EPI>
 cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
     const int E = g.group == GROUP_NONE ? 1 : g.num_experts;
     CUtensorMap ma, mb;
@@ -645,13 +677,15 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
     }
     // Outputs through TMA stores: bf16, no read-modify-write, 16-byte aligned rows; per-expert outputs (GROUP_K)
     // only when a row tile cannot run into the next expert's rows.
-    const bool tma_store = !g.out_f32 && !g.accumulate && g.split_k <= 1 && (g.ldc % 8 == 0) && ((uintptr_t)g.C % 16 == 0) &&
+    const bool tma_store = TMA_EPI;
+    const bool tma_possible = !g.out_f32 && !g.accumulate && g.split_k <= 1 && (g.ldc % 8 == 0) && ((uintptr_t)g.C % 16 == 0) &&
                            ((uintptr_t)g.Z % 16 == 0) && (g.group != GROUP_K || (g.M % BM == 0 && g.c_stride == (int64_t)g.M * g.ldc));
+    if (TMA_EPI && !tma_possible) return cudaErrorInvalidValue;
     CUtensorMap mc = ma, mz = ma;
     if (tma_store) {
         const uint64_t c_rows = g.group == GROUP_K ? (uint64_t)g.M * E : (uint64_t)g.M;
         ok &= make_map(&mc, g.C, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
-        if (g.epilogue == EPI_ACT && g.Z)
+        if ((g.epilogue == EPI_ACT && g.Z) || g.epilogue == EPI_DACT)
             ok &= make_map(&mz, g.Z, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
     }
     if (!ok) return cudaErrorInvalidValue;
@@ -664,9 +698,9 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
     p.num_experts = E; p.tile_expert = g.tile_expert; p.n_tiles = g.n_tiles; p.poffsets = g.poffsets; p.status = status;
     const int64_t tiles = (int64_t)((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * (g.group == GROUP_K ? E : p.split_k);
     const int max_tiles = tiles > (1 << 30) ? (1 << 30) : (int)tiles;
-    if (g.a_kmajor && g.b_kmajor) return launch<BN, STAGES, true, true>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
-    if (g.a_kmajor && !g.b_kmajor) return launch<BN, STAGES, true, false>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
-    if (!g.a_kmajor && !g.b_kmajor) return launch<BN, STAGES, false, false>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
+    if (g.a_kmajor && g.b_kmajor) return launch<BN, STAGES, true, true, TMA_EPI>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
+    if (g.a_kmajor && !g.b_kmajor) return launch<BN, STAGES, true, false, TMA_EPI>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
+    if (!g.a_kmajor && !g.b_kmajor) return launch<BN, STAGES, false, false, TMA_EPI>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
     return cudaErrorNotSupported;
 }
 
@@ -675,12 +709,20 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
 bool gemm_tc_available() { return encode_fn() != nullptr; }
 int gemm_tc_sm_count() { return sm_count(); }
 
+// Can this problem's output leave through shared memory and TMA stores?
+bool tma_epilogue_possible(const GemmArgs& g) {
+    return !g.out_f32 && !g.accumulate && g.split_k <= 1 && (g.ldc % 8 == 0) && ((uintptr_t)g.C % 16 == 0) &&
+           ((uintptr_t)g.Z % 16 == 0) &&
+           (g.group != GROUP_K || (g.M % BM == 0 && g.c_stride == (int64_t)g.M * g.ldc));
+}
+
 cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
-    // 128 x 256 tiles (3 stages of 48 KB) when the output is at least 256 wide, else 128 x 128 (5 stages);
-    // 64 KB of shared memory stage the epilogue's TMA stores.
-    if (g.N >= 256) return dispatch<256, 3>(g, status, stream);
-    return dispatch<128, 5>(g, status, stream);
+    // Output-heavy problems (wide rows: activations, ascend, dx) stage their stores through shared memory and
+    // TMA, which costs one pipeline stage; contraction-heavy ones keep the deeper pipeline and store directly.
+    const bool staged = tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 && (g.epilogue != EPI_DACT || g.group != GROUP_K);
+    if (g.N >= 256) return staged ? dispatch<256, 3, true>(g, status, stream) : dispatch<256, 4, false>(g, status, stream);
+    return dispatch<128, 6, false>(g, status, stream);
 }
 
 }  // namespace bigmac

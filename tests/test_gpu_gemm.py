@@ -57,7 +57,8 @@ def _run(layer, q, tc=True):
     assert layer.status() == 0
 
 
-@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (300, 192, 256), (1000, 64, 4096), (77, 320, 128)])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (300, 192, 256), (1000, 64, 4096), (77, 320, 128), (333, 1024, 192),
+                                   (20000, 2048, 64)])
 def test_dense_kmajor_kmajor(M, N, K):
     import torch
     A, B = _rand((M, K), 1), _rand((N, K), 2, K ** -0.5)
@@ -123,10 +124,11 @@ def _dgelu(z):
     return 0.5 * (1.0 + erf(z / np.sqrt(2.0))) + z * np.exp(-0.5 * z * z) / np.sqrt(2 * np.pi)
 
 
-def test_grouped_rows_forward_and_backward_epilogues():
+@pytest.mark.parametrize("N", [192, 1024])       # 1024: wide outputs leave through shared memory and TMA stores
+def test_grouped_rows_forward_and_backward_epilogues(N):
     import torch
     counts = [130, 0, 5, 256, 1]
-    E, K, N = len(counts), 128, 192
+    E, K = len(counts), 128
     poff, tile_expert = _segments(counts)
     P = int(poff[-1]) + 256                                     # buffer larger than the live tiles
     A = np.zeros((P, K), dtype=np.float32)
@@ -152,7 +154,7 @@ def test_grouped_rows_forward_and_backward_epilogues():
     G = np.zeros((P, N), dtype=np.float32)                       # "du": [P, N] now the contraction side
     for e, c in enumerate(counts):
         G[poff[e]:poff[e] + c] = _rand((c, N), 40 + e)
-    N2 = K                                                       # output width
+    N2 = K if N == 192 else 1024                                 # output width
     Wt = _rand((E, N, N2), 12, N ** -0.5)                        # B(n2, k=n) = Wt[e][n, n2]
     Zin = _rand((P, N2), 13)
     Zd = _dev_bf16(Zin)
