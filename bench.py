@@ -166,6 +166,29 @@ def config_dict(w, args):
             "l2": "inputs larger than L2 (x, dy 268 MB each, weights 546 MB at the large workload)"}
 
 
+# ------------------------------------------------------------------------------------------------ ranks
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Every rank draws its own batch (independent data-parallel replicas, replicated shapes)."""
+    return base_seed + 1000 * rank
+
+
+def slowest_rank_ms(ms_local: float, device: str = "cpu") -> float:
+    """Device time of the slowest rank (MAX all-reduce); the identity without a process group."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms_local)
+    t = torch.tensor([float(ms_local)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Weak scaling: every rank processes tokens_per_rank tokens per step; the job is as fast as its slowest rank."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------------ ours
 def run_ours(args, w):
     import torch
@@ -185,7 +208,7 @@ def run_ours(args, w):
     if world > 1:
         dist.barrier()
 
-    wr = w.with_tokens(w.T, seed=w.seed + 1000 * rank)          # every rank draws its own batch
+    wr = w.with_tokens(w.T, seed=rank_seed(w.seed, rank))
     inp = wl.make_inputs(wr)
     tdt = torch.bfloat16 if w.dtype == wl.DTYPE_BF16 else torch.float32
 
@@ -228,10 +251,7 @@ def run_ours(args, w):
             fn()
         stop.record()
         barrier()
-        ms = torch.tensor([start.elapsed_time(stop)], device="cuda")
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return slowest_rank_ms(start.elapsed_time(stop), device="cuda")
 
     if args.profile_run:                    # bare loop for a profiler: warm-up and K steps, nothing else
         for _ in range(args.warmup + args.steps):
@@ -261,7 +281,7 @@ def run_ours(args, w):
     binding.bigmac_profile_enable(layer.handle, False)
     clocks = sampler.stop(t0, t1) if sampler else None
     ms_step = ms_total / args.steps
-    value = world * w.T / (ms_step * 1e-3)
+    value = whole_job_tokens_per_s(w.T, world, ms_step)
 
     # forward only (inference forward: nothing saved)
     def fwd_only():
