@@ -43,22 +43,37 @@ template <> struct Vec<__nv_bfloat16> {
 
 __device__ __forceinline__ int warp_global_id() { return blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); }
 
+// Each warp moves kDispatchRows consecutive grouped rows: all row indices are read first, then every
+// 16-byte load of the rows is issued before the first store, so many loads are in flight per lane.
+constexpr int kDispatchRows = 4;
 __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__ src, uint4* __restrict__ grouped,
                                                        const int32_t* __restrict__ slot_of_prow,
                                                        const int32_t* __restrict__ n_tiles, int k, int vecs_per_row,
                                                        int64_t max_prows) {
-    const int64_t prow = warp_global_id();
-    int64_t live = (int64_t)(*n_tiles) * kPad;
+    const int64_t prow0 = (int64_t)warp_global_id() * kDispatchRows;
+    int64_t live = (int64_t)(*n_tiles) * kPad;              // a multiple of kDispatchRows
     if (live > max_prows) live = max_prows;
-    if (prow >= live) return;
+    if (prow0 >= live) return;
     const int lane = threadIdx.x & 31;
-    const int s = slot_of_prow[prow];
-    uint4* out = grouped + prow * vecs_per_row;
-    if (s < 0) {
-        for (int c = lane; c < vecs_per_row; c += 32) out[c] = make_uint4(0, 0, 0, 0);
-    } else {
-        const uint4* in = src + (int64_t)(s / k) * vecs_per_row;
-        for (int c = lane; c < vecs_per_row; c += 32) out[c] = in[c];
+    int s[kDispatchRows];
+#pragma unroll
+    for (int i = 0; i < kDispatchRows; ++i) s[i] = slot_of_prow[prow0 + i];
+    for (int c0 = 0; c0 < vecs_per_row; c0 += 64) {
+        uint4 v[kDispatchRows][2];
+#pragma unroll
+        for (int i = 0; i < kDispatchRows; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int c = c0 + lane + 32 * j;
+                v[i][j] = (s[i] >= 0 && c < vecs_per_row) ? src[(int64_t)(s[i] / k) * vecs_per_row + c] : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+        for (int i = 0; i < kDispatchRows; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int c = c0 + lane + 32 * j;
+                if (c < vecs_per_row) grouped[(prow0 + i) * vecs_per_row + c] = v[i][j];
+            }
     }
 }
 
@@ -200,7 +215,7 @@ cudaError_t launch_dispatch(const void* src, void* grouped, const Tables& tb, in
                             int64_t max_prows, cudaStream_t stream) {
     if (max_prows == 0) return cudaSuccess;
     const int vecs = width * elem_bytes(dtype) / 16;
-    dispatch_kernel<<<warp_blocks(max_prows), 256, 0, stream>>>((const uint4*)src, (uint4*)grouped, tb.slot_of_prow,
+    dispatch_kernel<<<warp_blocks((max_prows + kDispatchRows - 1) / kDispatchRows), 256, 0, stream>>>((const uint4*)src, (uint4*)grouped, tb.slot_of_prow,
                                                                 tb.n_tiles, k, vecs, max_prows);
     return cudaGetLastError();
 }
