@@ -136,12 +136,20 @@ def oracle_sample_rate(w, inp, sample_tokens: int):
     return S / dt, dt, S, min(threads, cores)
 
 
+def sample_size_for(w, inp, seconds: float, repeats: int = 1, cap: int = 0) -> int:
+    """Tokens per oracle run so that `repeats` runs take about `seconds` in total (calibrated on 32 tokens)."""
+    rate, _, _, _ = oracle_sample_rate(w, inp, 32)
+    s = int(seconds * rate / max(repeats, 1))
+    s = max(8, min(w.T, s))
+    return min(s, cap) if cap else s
+
+
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     inp = wl.make_inputs(w)
-    S = args.ref_tokens
+    S = args.ref_tokens or sample_size_for(w, inp, 90.0, repeats=args.warmup + args.steps)
     rates = []
     for i in range(args.warmup + args.steps):
         rate, dt, S_used, cores = oracle_sample_rate(w, inp, S)
@@ -290,6 +298,32 @@ def run_ours(args, w):
         fwd_only()
     ms_fwd = timed(fwd_only, args.steps) / args.steps
 
+    # ---- the exchange stage alone at width r (BigMac) and at width d (a fine-grained CDAC layer of equal E, k
+    # dispatches and combines full-width rows, Eq. 1): same kernels, same routing, rank 0's GPU only
+    exchange = None
+    if rank == 0:
+        layer.forward(x, dev, y=y, training=True)                  # leaves the routing tables in `saved`
+        P = ((w.N + 127) // 128 + w.E) * 128
+        exchange = {}
+        for label, width, src in (("bigmac_width_r", w.r, x[:, : w.r].contiguous()), ("cdac_width_d", w.d, x)):
+            grouped = torch.empty((P, width), dtype=tdt, device="cuda")
+            dst = torch.empty((w.T, width), dtype=tdt, device="cuda")
+            run = lambda: binding.bigmac_exchange_rows(layer.handle, layer._saved, w.T, width, src, grouped, dst, 2)
+            for _ in range(3):
+                run()
+            start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            start.record()
+            for _ in range(10):
+                run()
+            stop.record()
+            torch.cuda.synchronize()
+            ms = start.elapsed_time(stop) / 10
+            nbytes = 2 * (w.T + w.N) * width * (2 if w.dtype == wl.DTYPE_BF16 else 4)
+            exchange[label] = {"bytes": nbytes, "ms": round(ms, 4), "gbs": round(nbytes / ms / 1e6, 1)}
+            del grouped, dst
+        exchange["time_ratio_d_over_r"] = round(exchange["cdac_width_d"]["ms"] / exchange["bigmac_width_r"]["ms"], 2)
+
     # ---- end to end through the same calls with HOST buffers: x, dy in; y, dx out, every step
     def e2e_step():
         x.copy_(hx, non_blocking=True)
@@ -341,7 +375,7 @@ def run_ours(args, w):
                 "frac_of_burst_peak": round(achieved / peaks["tflops_burst"], 4),
                 "step_frac": round(3.0 * fwd_fl / (ms_step * 1e-3) / 1e12 / peaks["tflops_sustained"], 4)}
 
-    rate, dt, S_used, cores = oracle_sample_rate(w, inp, args.ref_tokens)
+    rate, dt, S_used, cores = oracle_sample_rate(w, inp, args.ref_tokens or sample_size_for(w, inp, 15.0))
     bytes_io = 2 * w.T * w.d * esz
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -356,7 +390,7 @@ def run_ours(args, w):
             "cpu_baseline": {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": f"first {S_used} tokens of the workload, routing + forward + backward with "
                                        f"every gradient, {dt:.1f} s"},
-            "exchange_bytes": {"bigmac_width_r": 2 * (w.T + w.N) * w.r * esz, "cdac_width_d": 2 * (w.T + w.N) * w.d * esz},
+            "exchange": exchange,
             "stages": stages}
     print(json.dumps(line))
     if world > 1:
@@ -373,7 +407,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="override T (per GPU)")
     ap.add_argument("--profile-run", action="store_true",
                     help="only run warm-up + K steps (for a kernel-list or counter capture); prints no bench line")
-    ap.add_argument("--ref-tokens", type=int, default=64, help="token sample of the CPU-oracle leg")
+    ap.add_argument("--ref-tokens", type=int, default=0,
+                    help="token sample of the CPU-oracle leg (0: sized for about 15 s; reference arm: about 90 s in total)")
     args = ap.parse_args()
     w = wl.WORKLOADS[args.config]
     if args.tokens:
