@@ -12,379 +12,15 @@
 //
 // Every wait on an mbarrier is bounded: when the bound is hit the CTA records BIGMAC_ERR_TIMEOUT in the
 // status word, stops waiting, and still releases its tensor memory before it exits.
-#include <cuda.h>
+#include <cstdlib>
 
-#include "internal.h"
-#include "act.cuh"
+#include "tc_common.cuh"
 
 namespace bigmac {
 
+using namespace tc;
+
 namespace {
-
-constexpr int BM = 128;          // UMMA M
-constexpr int BK = 64;           // bf16 elements per k slice = one 128-byte swizzle row
-constexpr int UMMA_K = 16;
-constexpr uint32_t kWaitLimit = 1u << 22;
-
-// ------------------------------------------------------------------------------------------ PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return done != 0;
-}
-// Bounded wait.  `dead` is a CTA-wide flag in shared memory: once any wait ran out nobody waits again.
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile int* dead, int* status) {
-    if (*dead) return;
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return;
-        if ((i & 1023u) == 1023u && *dead) return;
-    }
-    *dead = 1;
-    atomicExch(status, 1);
-}
-
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
-        : "memory");
-}
-
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* src, int c0, int c1) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                 ::"l"(map), "r"(c0), "r"(c1), "r"(smem_u32(src))
-                 : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void ld_shared_16B(const void* ptr, uint32_t* w) {
-    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(smem_u32(ptr)));
-}
-__device__ __forceinline__ void st_shared_16B(void* ptr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(smem_u32(ptr)), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-__device__ __forceinline__ void tmem_load_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_load_32_nowait(uint32_t taddr, uint32_t* v) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_load_32(uint32_t taddr, uint32_t* v) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
-//   K-major tile:  rows of 128 bytes (64 k), 8-row groups 1024 bytes apart (SBO); LBO unused.
-//   MN-major tile: k rows of 128 bytes (64 m/n), 8-k groups 1024 bytes apart (SBO), consecutive
-//                  64-wide m/n chunks `lbo_bytes` apart (LBO).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3ffff) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fff) << 32;
-    d |= (uint64_t)1 << 46;          // version
-    d |= (uint64_t)2 << 61;          // SWIZZLE_128B
-    return d;
-}
-
-// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M = 128, N = bn.
-__host__ __device__ constexpr uint32_t instr_desc(int bn, bool a_mn_major, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
-           ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-
-struct TcParams {
-    void* C;
-    void* Z;
-    int64_t ldc, c_stride;
-    int M, N, K;
-    int b_rows_per_expert;       // rows of the B tensor map per expert (GROUP_M); 0 if dense
-    int out_f32, accumulate, epilogue, act, group, num_experts;
-    int tma_store;               // bf16 outputs leave through shared memory and TMA stores (map_c / map_z)
-    int c_rows_per_expert;       // rows of the C tensor map per expert (GROUP_K); 0 otherwise
-    int split_k;                 // dense only: the contraction is cut into split_k parts, part s writes C + s*M*ldc
-    int b2_first_kb;             // k slices from this one on come from the second B tensor (map_b2); <0: none
-    const int32_t* tile_expert;
-    const int32_t* n_tiles;
-    const int32_t* poffsets;
-    int* status;
-};
-
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-    __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
-    return *reinterpret_cast<uint32_t*>(&p);
-}
-__device__ __forceinline__ void st_global_32B(void* ptr, const uint32_t* w) {
-    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(ptr), "r"(w[0]), "r"(w[1]), "r"(w[2]),
-                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
-                 : "memory");
-}
-__device__ __forceinline__ void ld_global_32B(const void* ptr, uint32_t* w) {
-    asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
-                 : "l"(ptr));
-}
-
-__device__ __forceinline__ float fast_rcp(float x) { float y; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
-__device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
-
-// sigma(z) and sigma'(z) together.  For GELU(erf) the two share one exponential: with s = |z|/sqrt2,
-// erf(s) = 1 - (a1 t + ... + a5 t^5) exp(-s^2), t = 1/(1 + 0.3275911 s) (absolute error below 1.5e-7, far
-// inside bf16 resolution), Phi(z) = 1 - q or q with q = poly * exp(-z^2/2) / 2, phi(z) = exp(-z^2/2)/sqrt(2 pi).
-__device__ __forceinline__ void act_pair(int act, float z, float& a, float& g) {
-    if (act == BIGMAC_ACT_GELU_ERF) {
-        const float t = fast_rcp(fmaf(0.23164190f, fabsf(z), 1.0f));          // 0.3275911 / sqrt 2
-        float poly = fmaf(t, 0.5307027145f, -0.7265760135f);                    // coefficients halved
-        poly = fmaf(t, poly, 0.7107068705f);
-        poly = fmaf(t, poly, -0.142248368f);
-        poly = fmaf(t, poly, 0.127414796f);
-        const float e = fast_ex2(-0.72134752f * z * z);                            // exp(-z^2 / 2)
-        const float q = poly * t * e;
-        const float cdf = z >= 0.0f ? 1.0f - q : q;
-        a = z * cdf;
-        g = fmaf(z * e, 0.39894228f, cdf);
-    } else if (act == BIGMAC_ACT_RELU) {
-        a = z > 0.0f ? z : 0.0f;
-        g = z > 0.0f ? 1.0f : 0.0f;
-    } else {
-        a = act_apply(act, z);
-        g = act_grad(act, z);
-    }
-}
-
-// Activation of 32 accumulator values in place; with WITH_G the 32 sigma' values are packed to bf16 pairs in wg.
-// The activation is a compile-time constant here so that the switch is taken once per chunk, not per element.
-template <int ACT, bool WITH_G>
-__device__ __forceinline__ void act_chunk(float* v, uint32_t* wg) {
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        float a0, g0, a1, g1;
-        act_pair(ACT, v[2 * i], a0, g0);
-        act_pair(ACT, v[2 * i + 1], a1, g1);
-        v[2 * i] = a0; v[2 * i + 1] = a1;
-        if (WITH_G) wg[i] = pack_bf16(g0, g1);
-    }
-}
-template <bool WITH_G>
-__device__ __forceinline__ void act_chunk_any(int act, float* v, uint32_t* wg) {
-    switch (act) {
-        case BIGMAC_ACT_GELU_ERF: act_chunk<BIGMAC_ACT_GELU_ERF, WITH_G>(v, wg); break;
-        case BIGMAC_ACT_RELU: act_chunk<BIGMAC_ACT_RELU, WITH_G>(v, wg); break;
-        case BIGMAC_ACT_GELU_TANH: act_chunk<BIGMAC_ACT_GELU_TANH, WITH_G>(v, wg); break;
-        default: act_chunk<BIGMAC_ACT_IDENTITY, WITH_G>(v, wg); break;
-    }
-}
-
-// Epilogue for 32 consecutive columns [col0, col0+32) of one output row held in v[0..31].
-__device__ __forceinline__ void store_row_chunk(const TcParams& p, float* v, int64_t row_off, int col0, bool vec_ok) {
-    const int ncols = min(32, p.N - col0);
-    if (ncols <= 0) return;
-    __nv_bfloat16* Zb = (__nv_bfloat16*)p.Z;
-    if (vec_ok && ncols == 32) {
-        const int64_t off = row_off + col0;
-        if (p.epilogue == EPI_ACT) {
-            if (Zb) {
-                uint32_t w[16];
-                act_chunk_any<true>(p.act, v, w);
-                st_global_32B(Zb + off, w);
-                st_global_32B(Zb + off + 16, w + 8);
-            } else {
-                act_chunk_any<false>(p.act, v, nullptr);
-            }
-        } else if (p.epilogue == EPI_DACT) {
-            uint32_t w[16];
-            ld_global_32B(Zb + off, w);
-            ld_global_32B(Zb + off + 16, w + 8);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) { v[2 * i] *= bf16_lo(w[i]); v[2 * i + 1] *= bf16_hi(w[i]); }
-        }
-        if (p.out_f32) {
-            float* cp = (float*)p.C + off;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t w[8];
-                if (p.accumulate) {
-                    ld_global_32B(cp + 8 * i, w);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) v[8 * i + j] += __uint_as_float(w[j]);
-                }
-#pragma unroll
-                for (int j = 0; j < 8; ++j) w[j] = __float_as_uint(v[8 * i + j]);
-                st_global_32B(cp + 8 * i, w);
-            }
-        } else {
-            __nv_bfloat16* cp = (__nv_bfloat16*)p.C + off;
-            uint32_t w[16];
-            if (p.accumulate) {
-                ld_global_32B(cp, w);
-                ld_global_32B(cp + 16, w + 8);
-#pragma unroll
-                for (int i = 0; i < 16; ++i) { v[2 * i] += bf16_lo(w[i]); v[2 * i + 1] += bf16_hi(w[i]); }
-            }
-#pragma unroll
-            for (int i = 0; i < 16; ++i) w[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
-            st_global_32B(cp, w);
-            st_global_32B(cp + 16, w + 8);
-        }
-        return;
-    }
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {           // ragged edge or unaligned rows: scalar (unrolled: v stays in registers)
-        if (i >= ncols) break;
-        const int64_t off = row_off + col0 + i;
-        float x = v[i];
-        if (p.epilogue == EPI_ACT) {
-            float g;
-            act_pair(p.act, x, x, g);
-            if (Zb) Zb[off] = __float2bfloat16(g);
-        } else if (p.epilogue == EPI_DACT) {
-            x *= __bfloat162float(Zb[off]);
-        }
-        if (p.out_f32) {
-            float* C = (float*)p.C;
-            C[off] = p.accumulate ? C[off] + x : x;
-        } else {
-            __nv_bfloat16* C = (__nv_bfloat16*)p.C;
-            C[off] = __float2bfloat16(p.accumulate ? __bfloat162float(C[off]) + x : x);
-        }
-    }
-}
-
-// One 32-row x 32-column bf16 box of an output in shared memory, laid out for a TMA store with the 64-byte
-// swizzle: row `lane` occupies 64 bytes, its 16-byte piece j sits at piece j ^ ((lane >> 1) & 3), which makes
-// the 32 lanes' 16-byte stores conflict-free.
-__device__ __forceinline__ void stage_row_bf16(uint8_t* box, int lane, const uint32_t* w /*16 packed pairs*/) {
-    uint8_t* row = box + lane * 64;
-    const int sw = (lane >> 1) & 3;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) st_shared_16B(row + ((j ^ sw) << 4), w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-}
-
-// Epilogue of 32 columns through shared memory: v -> (sigma', sigma) or v * Z or v, packed to bf16 into the
-// warp's staging boxes.  Returns nothing; the caller fences and issues the TMA stores.
-__device__ __forceinline__ void stage_row_chunk(const TcParams& p, float* v, uint8_t* box_c, uint8_t* box_z, int lane,
-                                                int64_t row_off, int col0, bool row_ok) {
-    uint32_t w[16];
-    if (p.epilogue == EPI_ACT) {
-        if (p.Z) {
-            act_chunk_any<true>(p.act, v, w);
-            stage_row_bf16(box_z, lane, w);
-        } else {
-            act_chunk_any<false>(p.act, v, nullptr);
-        }
-    }   // EPI_DACT: the caller has already multiplied by the prefetched sigma'
-#pragma unroll
-    for (int i = 0; i < 16; ++i) w[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
-    stage_row_bf16(box_c, lane, w);
-}
-
-// What one CTA works on next: output tile (m0, n0) of problem `expert`, contraction rows
-// [k_row0, k_row0 + 64*num_kb).
-struct Tile {
-    int m0, n0, expert, k_row0, num_kb, m_limit;
-    int64_t c_base;
-};
-
-__device__ __forceinline__ int total_tiles(const TcParams& p, int BN, int& tiles_m, int& tiles_n) {
-    tiles_n = (p.N + BN - 1) / BN;
-    tiles_m = p.group == GROUP_M ? min(*p.n_tiles, (p.M + BM - 1) / BM) : (p.M + BM - 1) / BM;
-    return tiles_m * tiles_n * (p.group == GROUP_K ? p.num_experts : p.split_k);
-}
-
-__device__ __forceinline__ Tile get_tile(const TcParams& p, int BN, int t, int tiles_m, int tiles_n) {
-    Tile tl;
-    const int per = tiles_m * tiles_n;
-    const int e = (p.group == GROUP_K || p.split_k > 1) ? t / per : 0;     // expert, or part of a split contraction
-    const int r = t - e * per;
-    tl.m0 = (r / tiles_n) * BM;
-    tl.n0 = (r % tiles_n) * BN;
-    tl.expert = p.group == GROUP_K ? e : 0;
-    tl.k_row0 = 0;
-    tl.num_kb = (p.K + BK - 1) / BK;
-    tl.m_limit = p.M;
-    tl.c_base = 0;
-    if (p.group != GROUP_K && p.split_k > 1) {
-        const int per_part = (tl.num_kb + p.split_k - 1) / p.split_k;
-        tl.k_row0 = e * per_part * BK;
-        tl.num_kb = max(0, min(per_part, tl.num_kb - e * per_part));
-        tl.c_base = (int64_t)e * p.M * p.ldc;
-    }
-    if (p.group == GROUP_M) {
-        tl.expert = p.tile_expert[r / tiles_n];
-        tl.m_limit = min(p.M, tiles_m * kPad);
-    } else if (p.group == GROUP_K) {
-        tl.k_row0 = p.poffsets[e];
-        tl.num_kb = (p.poffsets[e + 1] - tl.k_row0) / BK;
-        tl.c_base = (int64_t)e * p.c_stride;
-    }
-    return tl;
-}
-
-constexpr int kEpiWarps = 16;
-constexpr uint32_t kBoxBytes = 32 * 64;                  // 32 rows x 32 bf16 columns
-constexpr int kThreadsV2 = (2 + kEpiWarps) * 32;
 
 // Persistent kernel: gridDim.x CTAs (one per SM) walk the tile list with stride gridDim.x.  The
 // accumulator is double-buffered in tensor memory (2 x BN columns), so the epilogue of tile i overlaps
@@ -591,48 +227,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 }
 
-// ------------------------------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = []() -> EncodeTiledFn {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            return nullptr;
-        return (EncodeTiledFn)sym;
-    }();
-    return fn;
-}
-
-// 2-D bf16 tensor map: `inner` contiguous elements per row, `rows` rows `ld` elements apart.
-bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner,
-              uint32_t box_rows, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {inner, rows};
-    const cuuint64_t strides[1] = {ld * 2};
-    const cuuint32_t box[2] = {box_inner, box_rows};
-    const cuuint32_t elem[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int sm_count() {
-    static int n = []() {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
-            return 148;
-        return v;
-    }();
-    return n;
-}
-
 template <int BN, int STAGES, bool AK, bool BKM, bool TMA_EPI>
 cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mz,
                    const CUtensorMap& mb2, const TcParams& p, int max_tiles, cudaStream_t stream) {
@@ -709,15 +303,13 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
 bool gemm_tc_available() { return encode_fn() != nullptr; }
 int gemm_tc_sm_count() { return sm_count(); }
 
-// Can this problem's output leave through shared memory and TMA stores?
-bool tma_epilogue_possible(const GemmArgs& g) {
-    return !g.out_f32 && !g.accumulate && g.split_k <= 1 && (g.ldc % 8 == 0) && ((uintptr_t)g.C % 16 == 0) &&
-           ((uintptr_t)g.Z % 16 == 0) &&
-           (g.group != GROUP_K || (g.M % BM == 0 && g.c_stride == (int64_t)g.M * g.ldc));
-}
-
 cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
+    // Where it pays, the problem runs on CTA pairs (each SM stages half of B); BIGMAC_TC_PAIR=0 disables that.
+    static const bool pair_enabled = []() { const char* e = std::getenv("BIGMAC_TC_PAIR"); return !(e && e[0] == '0'); }();
+    const bool want_pair = g.force_kernel == 2 ? gemm_tc_pair_supported(g)
+                           : g.force_kernel == 1 ? false : (pair_enabled && gemm_tc_pair_preferred(g));
+    if (want_pair) return gemm_tc_pair(g, status, stream);
     // Output-heavy problems (wide rows: activations, ascend, dx) stage their stores through shared memory and
     // TMA, which costs one pipeline stage; contraction-heavy ones keep the deeper pipeline and store directly.
     const bool staged = tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 && (g.epilogue != EPI_DACT || g.group != GROUP_K);

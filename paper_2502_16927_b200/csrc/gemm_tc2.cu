@@ -1,0 +1,446 @@
+// Tensor-core GEMM on CTA pairs (tcgen05 cta_group::2): C[m,n] (+)= epilogue(sum_k A(m,k) B(n,k)).
+//
+// Two CTAs of a cluster (two neighbouring SMs) own one 256 x BN output tile: CTA r holds rows 128r..128r+127
+// of A and columns (BN/2)r.. of B in its shared memory, and the 128 x BN accumulator of its rows in its own
+// tensor memory.  One tcgen05.mma.cta_group::2 (M=256, N=BN, K=16), issued by the pair's leader (CTA 0),
+// multiplies both CTAs' A rows with the B halves of both, so every SM stages only half of B: 32 KB instead of
+// 48 KB per 64-deep k slice for the same tensor-core work, which is what bounds the one-CTA kernel.
+// Protocol per k slice: each CTA's producer waits for its own "empty" barrier and issues its TMA loads, which
+// all complete on the LEADER's "full" barrier (armed by the leader with the bytes of both CTAs); the leader's
+// MMA warp waits there, issues the MMAs and commits with a multicast arrive onto the "empty" barrier of both
+// CTAs.  Accumulators are double-buffered: "tmem_full" is signalled in both CTAs by a multicast commit, and the
+// epilogue warps of both CTAs arrive on the leader's "tmem_empty" when they have read their half.
+// No TMA multicast is used.  Everything else (epilogues, grouping, split contraction) is as in gemm_tc.cu.
+#include "tc_common.cuh"
+
+namespace bigmac {
+
+using namespace tc;
+
+namespace {
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(const void* local, uint32_t rank) {
+    uint32_t out;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(smem_u32(local)), "r"(rank));
+    return out;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory that completes on a barrier of the pair's leader CTA.
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, uint32_t leader_bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(leader_bar)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive (when all MMAs issued so far have completed) on the barrier at this offset in both CTAs of the pair.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(smem_u32(bar)), "h"((uint16_t)3)
+        : "memory");
+}
+
+// Instruction descriptor for the pair MMA: M = 256 (128 rows per CTA), N = bn.
+__host__ __device__ constexpr uint32_t instr_desc_pair(int bn, bool a_mn_major, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+           ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+// Work item of one CTA pair: rows m0.. (CTA 0) and m0+128.. (CTA 1) of problem `expert`.
+struct PairTile {
+    int m0, n0, expert, k_row0, num_kb, m_limit, halves;
+    int64_t c_base;
+};
+
+// pairs of 128-row tiles: dense problems pair consecutive row tiles; expert-grouped rows pair tiles inside one
+// expert (an expert with an odd number of tiles ends with a half-used pair).  s_pp[e] = pairs before expert e.
+__device__ __forceinline__ PairTile get_pair_tile(const TcParams& p, int BN, int w, int pairs_m, int tiles_n, const int32_t* s_pp) {
+    PairTile t;
+    const int per = pairs_m * tiles_n;
+    const int e = (p.group == GROUP_K || p.split_k > 1) ? w / per : 0;
+    const int r = w - e * per;
+    const int pair = r / tiles_n;
+    t.n0 = (r % tiles_n) * BN;
+    t.m0 = pair * 2 * BM;
+    t.expert = p.group == GROUP_K ? e : 0;
+    t.k_row0 = 0;
+    t.num_kb = (p.K + BK - 1) / BK;
+    t.m_limit = p.M;
+    t.halves = 2;
+    t.c_base = 0;
+    if (p.group == GROUP_NONE && p.split_k > 1) {
+        const int per_part = (t.num_kb + p.split_k - 1) / p.split_k;
+        t.k_row0 = e * per_part * BK;
+        t.num_kb = max(0, min(per_part, t.num_kb - e * per_part));
+        t.c_base = (int64_t)e * p.M * p.ldc;
+    } else if (p.group == GROUP_M) {
+        int lo = 0, hi = p.num_experts;                        // largest x with s_pp[x] <= pair
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_pp[mid] <= pair) lo = mid; else hi = mid;
+        }
+        const int first = p.poffsets[lo] / kPad, count = (p.poffsets[lo + 1] - p.poffsets[lo]) / kPad;
+        const int j = pair - s_pp[lo];
+        t.expert = lo;
+        t.m0 = (first + 2 * j) * BM;
+        t.halves = min(2, count - 2 * j);
+    } else if (p.group == GROUP_K) {
+        t.k_row0 = p.poffsets[e];
+        t.num_kb = (p.poffsets[e + 1] - t.k_row0) / BK;
+        t.c_base = (int64_t)e * p.c_stride;
+    }
+    return t;
+}
+
+template <int BN, int STAGES, bool A_KMAJOR, bool B_KMAJOR, bool TMA_EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsV2, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_z,
+                    const __grid_constant__ CUtensorMap map_b2, const TcParams p) {
+    constexpr int BH = BN / 2;                               // B rows (output columns) staged by each CTA
+    constexpr uint32_t A_BYTES = BM * BK * 2;
+    constexpr uint32_t B_BYTES = BH * BK * 2;
+    constexpr uint32_t CHUNK_BYTES = 64 * BK * 2;            // one 64-wide MN-major box
+    constexpr uint32_t TMEM_COLS = 2 * BN;
+    constexpr uint32_t STAGING_BYTES = TMA_EPI ? kEpiWarps * 2 * kBoxBytes : 0;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* smem_a = smem;
+    uint8_t* smem_b = smem + STAGES * A_BYTES;
+    uint8_t* staging = smem + STAGES * (A_BYTES + B_BYTES);
+    uint64_t* full_bar = (uint64_t*)(staging + STAGING_BYTES);   // waited on in the leader only
+    uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* tmem_full_bar = empty_bar + STAGES;            // [2]
+    uint64_t* tmem_empty_bar = tmem_full_bar + 2;            // [2], the leader's are used
+    uint64_t* z_bar = tmem_empty_bar + 2;                    // [kEpiWarps]
+    uint32_t* tmem_slot = (uint32_t*)(z_bar + kEpiWarps);
+    volatile int* dead = (volatile int*)(tmem_slot + 1);
+    int32_t* s_pp = (int32_t*)(tmem_slot + 4);               // [num_experts + 1] pair prefix (GROUP_M)
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+
+    // ---- work list
+    const int tiles_n = (p.N + BN - 1) / BN;
+    int pairs_m = (p.M + 2 * BM - 1) / (2 * BM);
+    if (p.group == GROUP_M) {
+        if (threadIdx.x == 0) {
+            int run = 0;
+            for (int e = 0; e < p.num_experts; ++e) {
+                s_pp[e] = run;
+                run += ((p.poffsets[e + 1] - p.poffsets[e]) / kPad + 1) / 2;
+            }
+            s_pp[p.num_experts] = run;
+        }
+    }
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], 2 * kEpiWarps); }
+        for (int s = 0; s < kEpiWarps; ++s) mbar_init(&z_bar[s], 1);
+        *dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(tmem_slot, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                      // the peer's barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    if (p.group == GROUP_M) pairs_m = s_pp[p.num_experts];
+    const int total = pairs_m * tiles_n * (p.group == GROUP_K ? p.num_experts : p.split_k);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int w = cluster_id; w < total; w += num_clusters) {
+                const PairTile tl = get_pair_tile(p, BN, w, pairs_m, tiles_n, s_pp);
+                const int my_m0 = tl.m0 + (int)rank * BM;
+                const int my_n0 = tl.n0 + (int)rank * BH;
+                for (int kb = 0; kb < tl.num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, dead, p.status);
+                    if (leader) mbar_expect_tx(&full_bar[s], 2 * (A_BYTES + B_BYTES));
+                    const uint32_t bar = map_to_cta(&full_bar[s], 0);
+                    const int k0 = tl.k_row0 + kb * BK;
+                    uint8_t* a_dst = smem_a + s * A_BYTES;
+                    uint8_t* b_dst = smem_b + s * B_BYTES;
+                    if (A_KMAJOR) {
+                        tma_load_2d_pair(a_dst, &map_a, bar, k0, my_m0);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < BM / 64; ++c) tma_load_2d_pair(a_dst + c * CHUNK_BYTES, &map_a, bar, my_m0 + 64 * c, k0);
+                    }
+                    if (B_KMAJOR) {
+                        tma_load_2d_pair(b_dst, &map_b, bar, k0, tl.expert * p.b_rows_per_expert + my_n0);
+                    } else {
+                        const bool second = p.b2_first_kb >= 0 && kb >= p.b2_first_kb;     // dense only
+                        const CUtensorMap* mb = second ? &map_b2 : &map_b;
+                        const int kb_row = second ? (kb - p.b2_first_kb) * BK : tl.expert * p.b_rows_per_expert + k0;
+#pragma unroll
+                        for (int c = 0; c < BH / 64; ++c) tma_load_2d_pair(b_dst + c * CHUNK_BYTES, mb, bar, my_n0 + 64 * c, kb_row);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (leader) {
+            constexpr uint32_t idesc = instr_desc_pair(BN, !A_KMAJOR, !B_KMAJOR);
+            uint32_t it = 0, local = 0;
+            for (int w = cluster_id; w < total; w += num_clusters, ++local) {
+                const PairTile tl = get_pair_tile(p, BN, w, pairs_m, tiles_n, s_pp);
+                const uint32_t acc = local & 1;
+                mbar_wait(&tmem_empty_bar[acc], ((local >> 1) & 1) ^ 1, dead, p.status);
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < tl.num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    mbar_wait(&full_bar[s], (it / STAGES) & 1, dead, p.status);
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t a_addr = smem_u32(smem_a + s * A_BYTES);
+                        const uint32_t b_addr = smem_u32(smem_b + s * B_BYTES);
+#pragma unroll
+                        for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                            const uint64_t da = A_KMAJOR ? smem_desc(a_addr + kk * UMMA_K * 2, 16, 1024)
+                                                         : smem_desc(a_addr + kk * UMMA_K * 128, CHUNK_BYTES, 1024);
+                            const uint64_t db = B_KMAJOR ? smem_desc(b_addr + kk * UMMA_K * 2, 16, 1024)
+                                                         : smem_desc(b_addr + kk * UMMA_K * 128, CHUNK_BYTES, 1024);
+                            umma_bf16_pair(d_tmem, da, db, idesc, (kb | kk) != 0);
+                        }
+                        umma_commit_pair(&empty_bar[s]);
+                    }
+                    __syncwarp();
+                }
+                if (lane == 0) {
+                    if (tl.num_kb > 0) {
+                        umma_commit_pair(&tmem_full_bar[acc]);
+                    } else {                                   // nothing to contract: zero accumulators, signal directly
+                        mbar_arrive(&tmem_full_bar[acc]);
+                        mbar_arrive_cluster(map_to_cta(&tmem_full_bar[acc], 1));
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..17, both CTAs)
+        const int quad = warp & 3;
+        constexpr int COLS_PER_WARP = BN / (kEpiWarps / 4);
+        constexpr int CHUNKS = COLS_PER_WARP / 32;
+        const int part = (warp - 2) >> 2;
+        uint8_t* box_c = staging + (warp - 2) * 2 * kBoxBytes;
+        uint8_t* box_z = box_c + kBoxBytes;
+        const int esz = p.out_f32 ? 4 : 2;
+        const bool vec_ok = ((p.ldc * esz) % 32 == 0) && ((p.c_stride * esz) % 32 == 0) && (p.ldc % 16 == 0) &&
+                            (((uintptr_t)p.C) % 32 == 0) && (((uintptr_t)p.Z) % 32 == 0);
+        const uint32_t leader_tmem_empty[2] = {map_to_cta(&tmem_empty_bar[0], 0), map_to_cta(&tmem_empty_bar[1], 0)};
+        const bool z_prefetch = TMA_EPI && p.epilogue == EPI_DACT;
+        uint64_t* my_z_bar = &z_bar[warp - 2];
+        uint32_t z_count = 0;
+        auto issue_z = [&](const PairTile& tile, int c) {
+            if (lane == 0) {
+                mbar_expect_tx(my_z_bar, kBoxBytes);
+                tma_load_2d(box_z, &map_z, my_z_bar, tile.n0 + part * COLS_PER_WARP + c * 32,
+                            tile.m0 + (int)rank * BM + quad * 32);
+            }
+        };
+        if (z_prefetch && cluster_id < total) issue_z(get_pair_tile(p, BN, cluster_id, pairs_m, tiles_n, s_pp), 0);
+        uint32_t local = 0;
+        for (int w = cluster_id; w < total; w += num_clusters, ++local) {
+            const PairTile tl = get_pair_tile(p, BN, w, pairs_m, tiles_n, s_pp);
+            const uint32_t acc = local & 1;
+            mbar_wait(&tmem_full_bar[acc], (local >> 1) & 1, dead, p.status);
+            tc_fence_after();
+            const int my_m0 = tl.m0 + (int)rank * BM;
+            const int row = my_m0 + quad * 32 + lane;
+            const bool half_ok = (int)rank < tl.halves;
+            const bool row_ok = half_ok && row < tl.m_limit;
+            const int64_t row_off = tl.c_base + (int64_t)row * p.ldc;
+            const uint32_t t_addr = tmem_base + acc * BN + ((uint32_t)(quad * 32) << 16) + (uint32_t)(part * COLS_PER_WARP);
+#pragma unroll 1
+            for (int c = 0; c < CHUNKS; ++c) {
+                float v[32];
+                if (tl.num_kb > 0) {
+                    tmem_load_32_nowait(t_addr + c * 32, (uint32_t*)v);
+                    tmem_load_wait();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0.0f;
+                }
+                if (c == CHUNKS - 1) {                 // accumulator half fully read: tell the leader's MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(leader_tmem_empty[acc]);
+                }
+                const int col0 = tl.n0 + part * COLS_PER_WARP + c * 32;
+                if (col0 >= p.N) continue;             // uniform across the warp
+                if (TMA_EPI) {
+                    if (lane == 0) tma_store_wait_read();
+                    __syncwarp();
+                    if (z_prefetch) {
+                        mbar_wait(my_z_bar, z_count & 1, dead, p.status);
+                        ++z_count;
+                        uint32_t wz[16];
+                        const uint8_t* zrow = box_z + lane * 64;
+                        const int sw = (lane >> 1) & 3;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) ld_shared_16B(zrow + ((j ^ sw) << 4), wz + 4 * j);
+                        fence_async_smem();
+                        __syncwarp();
+                        if (c + 1 < CHUNKS) issue_z(tl, c + 1);
+                        else if (w + num_clusters < total) issue_z(get_pair_tile(p, BN, w + num_clusters, pairs_m, tiles_n, s_pp), 0);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) { v[2 * i] *= bf16_lo(wz[i]); v[2 * i + 1] *= bf16_hi(wz[i]); }
+                    }
+                    stage_row_chunk(p, v, box_c, box_z, lane, row_off, col0, row_ok);
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && half_ok && my_m0 < tl.m_limit) {
+                        const int row0 = tl.expert * p.c_rows_per_expert + my_m0 + quad * 32;
+                        tma_store_2d(&map_c, box_c, col0, row0);
+                        if (p.epilogue == EPI_ACT && p.Z) tma_store_2d(&map_z, box_z, col0, row0);
+                        tma_store_commit();
+                    }
+                } else if (row_ok) {
+                    store_row_chunk(p, v, row_off, col0, vec_ok);
+                }
+            }
+        }
+        if (TMA_EPI && lane == 0) tma_store_wait_all();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                      // nobody leaves while the peer may still touch this CTA
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+template <int BN, int STAGES, bool AK, bool BKM, bool TMA_EPI>
+cudaError_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mz,
+                        const CUtensorMap& mb2, const TcParams& p, int64_t max_items, cudaStream_t stream) {
+    constexpr size_t kMaxSmem = 232448;                      // 227 KB: the most a CTA can have on sm_100
+    const size_t smem = STAGES * (BM * BK * 2 + (BN / 2) * BK * 2) + (TMA_EPI ? kEpiWarps * 2 * kBoxBytes : 0) +
+                        (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + (size_t)(p.num_experts + 1) * 4 + 1024;
+    if (smem > kMaxSmem) return cudaErrorInvalidConfiguration;
+    static bool configured = false;
+    auto kernel = gemm_tc_pair_kernel<BN, STAGES, AK, BKM, TMA_EPI>;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    int64_t clusters = sm_count() / 2;
+    if (max_items < clusters) clusters = max_items;
+    if (clusters < 1) clusters = 1;
+    kernel<<<(unsigned)(2 * clusters), kThreadsV2, smem, stream>>>(ma, mb, mc, mz, mb2, p);
+    return cudaGetLastError();
+}
+
+template <int BN, int STAGES, bool TMA_EPI>
+cudaError_t dispatch_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
+    constexpr int BH = BN / 2;
+    const int E = g.group == GROUP_NONE ? 1 : g.num_experts;
+    CUtensorMap ma, mb;
+    bool ok = true;
+    TcParams p{};
+    if (g.a_kmajor) ok &= make_map(&ma, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.lda, BK, BM);
+    else ok &= make_map(&ma, g.A, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.lda, 64, BK);
+    const uint64_t rows_per = g.group == GROUP_M ? (uint64_t)(g.b_stride / g.ldb) : 0;
+    if (g.b_kmajor)
+        ok &= make_map(&mb, g.B, (uint64_t)g.K, g.group == GROUP_M ? rows_per * E : (uint64_t)g.N, (uint64_t)g.ldb, BK, BH);
+    else
+        ok &= make_map(&mb, g.B, (uint64_t)g.N, g.group == GROUP_M ? rows_per * E : (uint64_t)g.K, (uint64_t)g.ldb, 64, BK);
+    CUtensorMap mb2 = mb;
+    p.b2_first_kb = -1;
+    if (g.B2) {
+        if (g.b_kmajor || g.group != GROUP_NONE || g.b2_first_k % BK) return cudaErrorInvalidValue;
+        ok &= make_map(&mb2, g.B2, (uint64_t)g.N, (uint64_t)(g.K - g.b2_first_k), (uint64_t)g.ldb2, 64, BK);
+        ok &= make_map(&mb, g.B, (uint64_t)g.N, (uint64_t)g.b2_first_k, (uint64_t)g.ldb, 64, BK);
+        p.b2_first_kb = g.b2_first_k / BK;
+    }
+    if (TMA_EPI && !tma_epilogue_possible(g)) return cudaErrorInvalidValue;
+    CUtensorMap mc = ma, mz = ma;
+    if (TMA_EPI) {
+        const uint64_t c_rows = g.group == GROUP_K ? (uint64_t)g.M * E : (uint64_t)g.M;
+        ok &= make_map(&mc, g.C, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+        if ((g.epilogue == EPI_ACT && g.Z) || g.epilogue == EPI_DACT)
+            ok &= make_map(&mz, g.Z, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+    }
+    if (!ok) return cudaErrorInvalidValue;
+    p.tma_store = TMA_EPI ? 1 : 0;
+    p.split_k = (g.group == GROUP_NONE && g.split_k > 1) ? g.split_k : 1;
+    p.c_rows_per_expert = g.group == GROUP_K ? g.M : 0;
+    p.b_rows_per_expert = (int)rows_per;
+    p.C = g.C; p.Z = g.Z; p.ldc = g.ldc; p.c_stride = g.c_stride; p.M = g.M; p.N = g.N; p.K = g.K;
+    p.out_f32 = g.out_f32; p.accumulate = g.accumulate; p.epilogue = g.epilogue; p.act = g.act; p.group = g.group;
+    p.num_experts = E; p.tile_expert = g.tile_expert; p.n_tiles = g.n_tiles; p.poffsets = g.poffsets; p.status = status;
+    // upper bound on work items (the kernel derives the exact count on the device for grouped rows)
+    const int64_t pairs = g.group == GROUP_M ? ((g.M + BM - 1) / BM + 1) / 2 + E : (g.M + 2 * BM - 1) / (2 * BM);
+    const int64_t items = pairs * ((g.N + BN - 1) / BN) * (g.group == GROUP_K ? E : p.split_k);
+    if (g.a_kmajor && g.b_kmajor) return launch_pair<BN, STAGES, true, true, TMA_EPI>(ma, mb, mc, mz, mb2, p, items, stream);
+    if (g.a_kmajor && !g.b_kmajor) return launch_pair<BN, STAGES, true, false, TMA_EPI>(ma, mb, mc, mz, mb2, p, items, stream);
+    if (!g.a_kmajor && !g.b_kmajor) return launch_pair<BN, STAGES, false, false, TMA_EPI>(ma, mb, mc, mz, mb2, p, items, stream);
+    return cudaErrorNotSupported;
+}
+
+}  // namespace
+
+// GROUP_M needs the padded offsets (to pair row tiles inside an expert).
+bool gemm_tc_pair_supported(const GemmArgs& g) {
+    if (g.N < 256) return false;                                  // narrow outputs stay on the one-CTA kernel
+    if (g.group == GROUP_M && !g.poffsets) return false;
+    return true;
+}
+
+// Measured on B200 (interleaved A/B at the large workload's shapes): pairs win 5-10 % when B is MN-major (half
+// as many TMA boxes per SM) and on wide dense outputs; K-major/K-major expert GEMMs are a few % faster alone.
+bool gemm_tc_pair_preferred(const GemmArgs& g) {
+    return gemm_tc_pair_supported(g) && (!g.b_kmajor || (g.group == GROUP_NONE && g.N >= 1024));
+}
+
+cudaError_t gemm_tc_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
+    if (g.M <= 0 || g.N <= 0) return cudaSuccess;
+    const bool staged = tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 &&
+                        (g.epilogue != EPI_DACT || g.group != GROUP_K);
+    // 32 KB per stage and CTA: 5 stages beside the 64 KB store staging (4 if the expert table is long), 6 without it
+    if (!staged) return dispatch_pair<256, 6, false>(g, status, stream);
+    const int E = g.group == GROUP_NONE ? 1 : g.num_experts;
+    return E <= 256 ? dispatch_pair<256, 5, true>(g, status, stream) : dispatch_pair<256, 4, true>(g, status, stream);
+}
+
+}  // namespace bigmac

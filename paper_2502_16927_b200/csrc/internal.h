@@ -51,6 +51,7 @@ struct GemmArgs {
     int64_t ldb2 = 0;
     int b2_first_k = 0;                 // multiple of 64
     int split_k = 1;                    // > 1: part s of the contraction writes its partial result (fp32) to C + s*M*ldc
+    int force_kernel = 0;               // measurement aid: 1 = one-CTA kernel, 2 = CTA-pair kernel, 0 = default choice
 };
 
 // fp32-FMA GEMM for either dtype (dtype: bigmac_dtype_t of A, B, Z and - unless out_f32 - C).
@@ -58,6 +59,10 @@ cudaError_t gemm_simt(const GemmArgs& g, int dtype, cudaStream_t stream);
 // tcgen05 / TMEM / TMA GEMM, bf16 inputs, fp32 accumulation.  `status` is the device status word.
 cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream);
 bool gemm_tc_available();
+// CTA-pair variant (tcgen05 cta_group::2) for outputs at least 256 wide.
+bool gemm_tc_pair_supported(const GemmArgs& g);
+bool gemm_tc_pair_preferred(const GemmArgs& g);
+cudaError_t gemm_tc_pair(const GemmArgs& g, int* status, cudaStream_t stream);
 int gemm_tc_sm_count();
 
 // ---------------------------------------------------------------------------------------------

@@ -187,13 +187,15 @@ int gemm(const bigmac_layer* L, int id, const GemmArgs& g, cudaStream_t st) {
 // Number of parts to cut a dense contraction of `num_kb` k slices into so that tiles * parts fills the SMs:
 // minimises waves * slices-per-part (ties: fewer parts).
 int choose_split_k(int M, int N, int K) {
-    const int bn = N >= 256 ? 256 : 128;
-    const int64_t tiles = (int64_t)((M + 127) / 128) * ((N + bn - 1) / bn);
-    const int num_kb = (K + 63) / 64, sms = gemm_tc_sm_count();
+    // the weight-gradient contractions (both operands MN-major, N >= 256) run on CTA pairs: 256-row tiles, SMs/2 units
+    const bool pairs = N >= 256;
+    const int bn = N >= 256 ? 256 : 128, bm = pairs ? 256 : 128;
+    const int64_t tiles = (int64_t)((M + bm - 1) / bm) * ((N + bn - 1) / bn);
+    const int num_kb = (K + 63) / 64, units = pairs ? gemm_tc_sm_count() / 2 : gemm_tc_sm_count();
     int best = 1;
     int64_t best_cost = -1;
     for (int s = 1; s <= kMaxSplitK && s <= num_kb; ++s) {
-        const int64_t cost = ((tiles * s + sms - 1) / sms) * ((num_kb + s - 1) / s);
+        const int64_t cost = ((tiles * s + units - 1) / units) * ((num_kb + s - 1) / s);
         if (best_cost < 0 || cost < best_cost) { best = s; best_cost = cost; }
     }
     return best;
@@ -359,14 +361,14 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         g.A = b.xg; g.lda = m.r; g.B = W->w1; g.ldb = m.r; g.b_stride = (int64_t)m.h * m.r;
         g.C = b.a; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
         g.epilogue = EPI_ACT; g.act = c.act; g.group = GROUP_M; g.num_experts = m.E;
-        g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles;
+        g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
         BIGMAC_TRY(gemm(L, G_EXPERT1, g, st));
     }
     {                                                                             // F7 u = a W2_e^T
         GemmArgs g;
         g.A = b.a; g.lda = m.h; g.B = W->w2; g.ldb = m.h; g.b_stride = (int64_t)m.r * m.h;
         g.C = b.u; g.ldc = m.r; g.M = (int)m.P; g.N = m.r; g.K = m.h;
-        g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles;
+        g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
         BIGMAC_TRY(gemm(L, G_EXPERT2, g, st));
     }
     { Stage s(L, S_COMBINE, st); BIGMAC_CUDA(launch_combine(b.u, b.y_lo, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st)); }  // F8
@@ -434,7 +436,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.A = b.du; g.lda = m.r; g.B = W->w2; g.ldb = m.h; g.b_kmajor = false; g.b_stride = (int64_t)m.r * m.h;
         g.C = b.z; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
         g.epilogue = EPI_DACT; g.act = c.act; g.group = GROUP_M; g.num_experts = m.E;
-        g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles;
+        g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
         BIGMAC_TRY(gemm(L, G_DZ, g, st));
     }
     void* dz = b.z;
@@ -449,7 +451,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         GemmArgs g;
         g.A = dz; g.lda = m.h; g.B = W->w1; g.ldb = m.r; g.b_kmajor = false; g.b_stride = (int64_t)m.h * m.r;
         g.C = b.dxg; g.ldc = m.r; g.M = (int)m.P; g.N = m.r; g.K = m.h;
-        g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles;
+        g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
         BIGMAC_TRY(gemm(L, G_DXG, g, st));
     }
     if (G->dw1) {   // dW1_e[q,c'] = sum_rows dz[row,q] xg[row,c']
@@ -672,6 +674,7 @@ int bigmac_debug_gemm(bigmac_layer_t* L, const bigmac_debug_gemm_t* q, int use_t
     g.group = q->group; g.num_experts = q->num_experts; g.b_stride = q->b_stride; g.c_stride = q->c_stride;
     g.tile_expert = q->tile_expert; g.n_tiles = q->n_tiles; g.poffsets = q->poffsets;
     L->launches += 1;
+    g.force_kernel = use_tensor_cores == 2 ? 1 : use_tensor_cores == 3 ? 2 : 0;
     cudaError_t err = use_tensor_cores ? gemm_tc(g, L->status, (cudaStream_t)stream)
                                        : gemm_simt(g, L->cfg.dtype, (cudaStream_t)stream);
     return err == cudaSuccess ? BIGMAC_OK : BIGMAC_ERR_CUDA;

@@ -137,11 +137,12 @@ def test_grouped_rows_forward_and_backward_epilogues(N):
     W = _rand((E, N, K), 11, K ** -0.5)                          # K-major weights [E,N,K]
     d_te = torch.from_numpy(np.concatenate([tile_expert, np.full(8, 99, np.int32)])).cuda()
     d_nt = torch.tensor([len(tile_expert)], dtype=torch.int32, device="cuda")
+    d_po = torch.from_numpy(poff).cuda()
     C = torch.full((P, N), float("nan"), dtype=torch.bfloat16, device="cuda")
     Z = torch.full((P, N), float("nan"), dtype=torch.bfloat16, device="cuda")
     layer = _layer()
     _run(layer, _q(A=_dev_bf16(A), B=_dev_bf16(W), C=C, Z=Z, lda=K, ldb=K, ldc=N, M=P, N=N, K=K, a_kmajor=1, b_kmajor=1,
-                   epilogue=1, act=1, group=1, num_experts=E, b_stride=N * K, tile_expert=d_te, n_tiles=d_nt))
+                   epilogue=1, act=1, group=1, num_experts=E, b_stride=N * K, tile_expert=d_te, n_tiles=d_nt, poffsets=d_po))
     got_c, got_z = _np(C), _np(Z)
     for e, c in enumerate(counts):
         rows = slice(poff[e], poff[e + 1])
@@ -159,7 +160,7 @@ def test_grouped_rows_forward_and_backward_epilogues(N):
     Zin = _rand((P, N2), 13)
     Zd = _dev_bf16(Zin)
     _run(layer, _q(A=_dev_bf16(G), B=_dev_bf16(Wt), C=Zd, Z=Zd, lda=N, ldb=N2, ldc=N2, M=P, N=N2, K=N, a_kmajor=1,
-                   b_kmajor=0, epilogue=2, act=1, group=1, num_experts=E, b_stride=N * N2, tile_expert=d_te, n_tiles=d_nt))
+                   b_kmajor=0, epilogue=2, act=1, group=1, num_experts=E, b_stride=N * N2, tile_expert=d_te, n_tiles=d_nt, poffsets=d_po))
     got = _np(Zd)
     for e in range(E):
         rows = slice(poff[e], poff[e + 1])
