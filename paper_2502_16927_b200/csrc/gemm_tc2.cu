@@ -34,7 +34,7 @@ __device__ __forceinline__ uint32_t map_to_cta(const void* local, uint32_t rank)
     return out;
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // TMA load into this CTA's shared memory that completes on a barrier of the pair's leader CTA.
 __device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, uint32_t leader_bar, int c0, int c1) {
@@ -427,10 +427,11 @@ bool gemm_tc_pair_supported(const GemmArgs& g) {
     return true;
 }
 
-// Measured on B200 (interleaved A/B at the large workload's shapes): pairs win 5-10 % when B is MN-major (half
-// as many TMA boxes per SM) and on wide dense outputs; K-major/K-major expert GEMMs are a few % faster alone.
+// Measured on B200 (interleaved A/B at the large workload's shapes): pairs win 5-12 % when B is MN-major (half
+// as many TMA boxes per SM) and on wide, output-heavy problems (expert GEMM1, dz, ascend, dx); the K-major /
+// K-major contraction-heavy GEMMs (expert GEMM2, descend) are 1-2 % faster on single CTAs.
 bool gemm_tc_pair_preferred(const GemmArgs& g) {
-    return gemm_tc_pair_supported(g) && (!g.b_kmajor || (g.group == GROUP_NONE && g.N >= 1024));
+    return gemm_tc_pair_supported(g) && (!g.b_kmajor || g.N >= 1024);
 }
 
 cudaError_t gemm_tc_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
