@@ -348,6 +348,8 @@ def run_ours(args, w):
     stages = {}
     gemm_ms = gemm_flops = 0.0
     flops_of = {name: fn(w) for name, fn in GEMM_FLOPS.items()}
+    if "gemm_logits" not in prof["stages"]:         # gate logits computed by the descend launch
+        flops_of["gemm_descend"] += flops_of["gemm_logits"]
     if "gemm_dx_gate" not in prof["stages"]:        # gate part fused into the dx contraction
         flops_of["gemm_dx"] += flops_of["gemm_dx_gate"]
     if "gemm_dw_gate" not in prof["stages"]:        # dW_gate computed together with dW_down

@@ -88,7 +88,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             tma_load_2d(a_dst + c * CHUNK_BYTES, &map_a, &full_bar[s], tl.m0 + 64 * c, k0);
                     }
                     if (B_KMAJOR) {
-                        tma_load_2d(b_dst, &map_b, &full_bar[s], k0, tl.expert * p.b_rows_per_expert + tl.n0);
+                        if (p.n_split >= 0 && tl.n0 >= p.n_split) tma_load_2d(b_dst, &map_b2, &full_bar[s], k0, tl.n0 - p.n_split);
+                        else tma_load_2d(b_dst, &map_b, &full_bar[s], k0, tl.expert * p.b_rows_per_expert + tl.n0);
                     } else {
                         const bool second = p.b2_first_kb >= 0 && kb >= p.b2_first_kb;     // dense only
                         const CUtensorMap* mb = second ? &map_b2 : &map_b;
@@ -213,7 +214,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         tma_store_commit();
                     }
                 } else if (row_ok) {
-                    store_row_chunk(p, v, row_off, col0, vec_ok);
+                    if (p.n_split >= 0 && tl.n0 >= p.n_split) {          // second output: fp32, its own leading dimension
+                        TcParams p2 = p;
+                        p2.C = p.C2; p2.ldc = p.ldc2; p2.N = p.N2; p2.out_f32 = 1; p2.epilogue = EPI_NONE; p2.accumulate = 0;
+                        const bool vec2 = (p.ldc2 % 8 == 0) && (((uintptr_t)p.C2) % 32 == 0);
+                        store_row_chunk(p2, v, (int64_t)row * p.ldc2, col0 - p.n_split, vec2);
+                    } else {
+                        store_row_chunk(p, v, row_off, col0, vec_ok);
+                    }
                 }
             }
         }
@@ -262,12 +270,20 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
     // Optional second B tensor (MN-major only): contraction rows k >= b2_first_k come from B2[k - b2_first_k, :].
     CUtensorMap mb2 = mb;
     p.b2_first_kb = -1;
-    if (g.B2) {
+    if (g.B2 && !g.C2) {
         if (g.b_kmajor || g.group != GROUP_NONE || g.b2_first_k % BK) return cudaErrorInvalidValue;
         ok &= make_map(&mb2, g.B2, (uint64_t)g.N, (uint64_t)(g.K - g.b2_first_k), (uint64_t)g.ldb2, 64, BK);
         // the first tensor ends where the second begins
         ok &= make_map(&mb, g.B, (uint64_t)g.N, (uint64_t)g.b2_first_k, (uint64_t)g.ldb, 64, BK);
         p.b2_first_kb = g.b2_first_k / BK;
+    }
+    p.n_split = -1;
+    if (g.C2) {      // second K-major B tensor feeding a second (fp32) output
+        if (!g.b_kmajor || g.group != GROUP_NONE || g.n_split % BN || TMA_EPI || g.B2 == nullptr || g.split_k > 1)
+            return cudaErrorInvalidValue;
+        ok &= make_map(&mb2, g.B2, (uint64_t)g.K, (uint64_t)g.N2, (uint64_t)g.ldb2, BK, BN);
+        ok &= make_map(&mb, g.B, (uint64_t)g.K, (uint64_t)g.n_split, (uint64_t)g.ldb, BK, BN);
+        p.n_split = g.n_split; p.C2 = g.C2; p.ldc2 = g.ldc2; p.N2 = g.N2;
     }
     // Outputs through TMA stores: bf16, no read-modify-write, 16-byte aligned rows; per-expert outputs (GROUP_K)
     // only when a row tile cannot run into the next expert's rows.
@@ -307,12 +323,12 @@ cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
     // Where it pays, the problem runs on CTA pairs (each SM stages half of B); BIGMAC_TC_PAIR=0 disables that.
     static const bool pair_enabled = []() { const char* e = std::getenv("BIGMAC_TC_PAIR"); return !(e && e[0] == '0'); }();
-    const bool want_pair = g.force_kernel == 2 ? gemm_tc_pair_supported(g)
+    const bool want_pair = g.C2 ? false : g.force_kernel == 2 ? gemm_tc_pair_supported(g)
                            : g.force_kernel == 1 ? false : (pair_enabled && gemm_tc_pair_preferred(g));
     if (want_pair) return gemm_tc_pair(g, status, stream);
     // Output-heavy problems (wide rows: activations, ascend, dx) stage their stores through shared memory and
     // TMA, which costs one pipeline stage; contraction-heavy ones keep the deeper pipeline and store directly.
-    const bool staged = tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 && (g.epilogue != EPI_DACT || g.group != GROUP_K);
+    const bool staged = !g.C2 && tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 && (g.epilogue != EPI_DACT || g.group != GROUP_K);
     if (g.N >= 256) return staged ? dispatch<256, 3, true>(g, status, stream) : dispatch<256, 4, false>(g, status, stream);
     return dispatch<128, 6, false>(g, status, stream);
 }

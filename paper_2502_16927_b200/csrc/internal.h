@@ -50,6 +50,12 @@ struct GemmArgs {
     const void* B2 = nullptr;           // second MN-major B: contraction rows k >= b2_first_k read B2[(k - b2_first_k)*ldb2 + n]
     int64_t ldb2 = 0;
     int b2_first_k = 0;                 // multiple of 64
+    // ... or, with K-major B: output columns n >= n_split use rows of B2 (n - n_split) and are written as fp32 to
+    // C2[m*ldc2 + n - n_split] for n - n_split < N2 (n_split a multiple of the tile width; N = n_split + N2).
+    int n_split = -1;
+    float* C2 = nullptr;
+    int64_t ldc2 = 0;
+    int N2 = 0;
     int split_k = 1;                    // > 1: part s of the contraction writes its partial result (fp32) to C + s*M*ldc
     int force_kernel = 0;               // measurement aid: 1 = one-CTA kernel, 2 = CTA-pair kernel, 0 = default choice
 };

@@ -347,9 +347,22 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     cudaStream_t st = (cudaStream_t)stream;
     const bigmac_config_t& c = L->cfg;
 
-    BIGMAC_TRY(run_routing(L, m, x, W, b, st));                                   // F1-F3
+    // F1 + F4 in one pass over x when the tile grid allows it: [x' | logits] = x [W'_down ; W_gate]^T, logits in fp32
+    const int bn_desc = (m.r + m.E) >= 256 ? 256 : 128;
+    const bool fuse_gate = c.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u && m.r % bn_desc == 0;
+    if (fuse_gate) {
+        GemmArgs g;
+        g.A = x; g.lda = m.d; g.B = W->w_down; g.ldb = m.d; g.C = b.x_lo; g.ldc = m.r;
+        g.B2 = W->w_gate; g.ldb2 = m.d; g.n_split = m.r; g.C2 = b.logits; g.ldc2 = m.E; g.N2 = m.E;
+        g.M = m.T; g.N = m.r + m.E; g.K = m.d;
+        BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
+        { Stage s(L, S_TOPK, st); BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st)); }
+        { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, st)); }
+    } else {
+        BIGMAC_TRY(run_routing(L, m, x, W, b, st));                               // F1-F3
+    }
     BIGMAC_TRY(export_routing(m, b, routing_out, st));
-    {                                                                             // F4 descend: x' = x W'_down
+    if (!fuse_gate) {                                                             // F4 descend: x' = x W'_down
         GemmArgs g;
         g.A = x; g.lda = m.d; g.B = W->w_down; g.ldb = m.d; g.C = b.x_lo; g.ldc = m.r;
         g.M = m.T; g.N = m.r; g.K = m.d;

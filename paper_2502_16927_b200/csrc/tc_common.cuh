@@ -152,6 +152,10 @@ struct TcParams {
     int c_rows_per_expert;       // rows of the C tensor map per expert (GROUP_K); 0 otherwise
     int split_k;                 // dense only: the contraction is cut into split_k parts, part s writes C + s*M*ldc
     int b2_first_kb;             // k slices from this one on come from the second B tensor (map_b2); <0: none
+    int n_split;                 // output columns from this one on come from map_b2 (K-major) and go to C2 (fp32); <0: none
+    float* C2;
+    int64_t ldc2;
+    int N2;
     const int32_t* tile_expert;
     const int32_t* n_tiles;
     const int32_t* poffsets;
