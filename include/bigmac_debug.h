@@ -7,7 +7,8 @@
  *   group 0: dense.  group 1: rows are expert-grouped segments padded to 128 rows, row tile i belongs to
  *   expert tile_expert[i], only *n_tiles tiles exist, B of expert e at B + e*b_stride.  group 2: one
  *   problem per expert with k running over rows [poffsets[e], poffsets[e+1]), C of expert e at C + e*c_stride.
- *   epilogue 0: none; 1: Z = sigma'(acc) (if Z), C = sigma(acc); 2: C = acc * Z.
+ *   epilogue 0: none; 1: Z = sigma'(acc) (if Z), C = sigma(acc); 2: C = acc * Z.  On the tensor-core kernels Z holds
+ *   sigma' as one byte per element, q = round(200 sigma' + 27); on the plain FMA kernel Z has the layer's dtype.
  * All pointers are device memory (tables included), 16-byte aligned.  use_tensor_cores: 0 = plain FMA kernel,
  * 1 = tensor cores (default kernel choice), 2 = force the one-CTA kernel, 3 = force the CTA-pair kernel; non-zero
  * values require a BF16 handle.  Returns a bigmac_status_t.

@@ -265,14 +265,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         uint8_t* box_z = box_c + kBoxBytes;
         const int esz = p.out_f32 ? 4 : 2;
         const bool vec_ok = ((p.ldc * esz) % 32 == 0) && ((p.c_stride * esz) % 32 == 0) && (p.ldc % 16 == 0) &&
-                            (((uintptr_t)p.C) % 32 == 0) && (((uintptr_t)p.Z) % 32 == 0);
+                            (((uintptr_t)p.C) % 32 == 0) && (((uintptr_t)p.Z) % 32 == 0) && (p.Z == nullptr || p.ldc % 32 == 0);
         const uint32_t leader_tmem_empty[2] = {map_to_cta(&tmem_empty_bar[0], 0), map_to_cta(&tmem_empty_bar[1], 0)};
         const bool z_prefetch = TMA_EPI && p.epilogue == EPI_DACT;
         uint64_t* my_z_bar = &z_bar[warp - 2];
         uint32_t z_count = 0;
         auto issue_z = [&](const PairTile& tile, int c) {
             if (lane == 0) {
-                mbar_expect_tx(my_z_bar, kBoxBytes);
+                mbar_expect_tx(my_z_bar, kBoxBytesZ);
                 tma_load_2d(box_z, &map_z, my_z_bar, tile.n0 + part * COLS_PER_WARP + c * 32,
                             tile.m0 + (int)rank * BM + quad * 32);
             }
@@ -313,17 +313,15 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     if (z_prefetch) {
                         mbar_wait(my_z_bar, z_count & 1, dead, p.status);
                         ++z_count;
-                        uint32_t wz[16];
-                        const uint8_t* zrow = box_z + lane * 64;
-                        const int sw = (lane >> 1) & 3;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) ld_shared_16B(zrow + ((j ^ sw) << 4), wz + 4 * j);
+                        uint32_t wz[8];
+                        const uint8_t* zrow = box_z + lane * 32;
+                        ld_shared_16B(zrow, wz);
+                        ld_shared_16B(zrow + 16, wz + 4);
                         fence_async_smem();
                         __syncwarp();
                         if (c + 1 < CHUNKS) issue_z(tl, c + 1);
                         else if (w + num_clusters < total) issue_z(get_pair_tile(p, BN, w + num_clusters, pairs_m, tiles_n, s_pp), 0);
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) { v[2 * i] *= bf16_lo(wz[i]); v[2 * i + 1] *= bf16_hi(wz[i]); }
+                        mul_by_sig32(v, wz);
                     }
                     stage_row_chunk(p, v, box_c, box_z, lane, row_off, col0, row_ok);
                     fence_async_smem();
@@ -399,7 +397,7 @@ cudaError_t dispatch_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
         const uint64_t c_rows = g.group == GROUP_K ? (uint64_t)g.M * E : (uint64_t)g.M;
         ok &= make_map(&mc, g.C, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
         if ((g.epilogue == EPI_ACT && g.Z) || g.epilogue == EPI_DACT)
-            ok &= make_map(&mz, g.Z, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+            ok &= make_map_u8(&mz, g.Z, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32);
     }
     if (!ok) return cudaErrorInvalidValue;
     p.tma_store = TMA_EPI ? 1 : 0;

@@ -85,6 +85,7 @@ struct Buffers {
     float* logits;
     void *x_lo, *xg, *z, *a, *u, *y_lo;                 // forward intermediates
     void *dy_lo, *du, *dxg; float* dp;                   // backward intermediates
+    void* dz;            // [P,h]: its own buffer when sigma' is saved as bytes, else written over sigma'
     void* dcat;          // [T, r + E64]: dx' in columns [0, r), the dense gate gradient dl in columns [r, r + E64)
     void *dx_lo, *dlogits;                               // views into dcat (row stride r + E64)
     float* colsum_part;  // [kColsumChunks, E]
@@ -95,12 +96,18 @@ struct Dims {
     int T, d, r, h, E, k, dtype;
     int64_t N, P;
     int E64;   // leading dimension of the dense [T,E] gate-gradient matrix (E rounded up to 64)
+    int z_es;  // bytes per saved sigma'(z) element: 1 on the tensor-core path (quantised), else the dtype's
 };
 
-Dims dims_of(const bigmac_config_t& c, int T) {
+// The tensor-core kernels save sigma' as one byte per element; that needs expert GEMM1 and dz on the same side.
+bool sigma_as_bytes(const bigmac_layer* L) { return L->cfg.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u; }
+
+Dims dims_of(const bigmac_layer* L, int T) {
+    const bigmac_config_t& c = L->cfg;
     Dims m{T, c.d, c.r, c.h, c.E, c.k, c.dtype, (int64_t)T * c.k, 0};
     m.P = padded_rows_max(m.N, c.E);
     m.E64 = (c.E + 63) / 64 * 64;
+    m.z_es = sigma_as_bytes(L) ? 1 : (int)esize(c.dtype);
     return m;
 }
 
@@ -120,7 +127,7 @@ void carve_saved(Carver& cv, const Dims& m, Buffers& b, bool with_z) {
     b.tb.n_tiles = cv.take<int32_t>(1);
     b.x_lo = cv.take_bytes((size_t)m.T * m.r * es);
     b.xg = cv.take_bytes((size_t)m.P * m.r * es);
-    b.z = with_z ? cv.take_bytes((size_t)m.P * m.h * es) : nullptr;
+    b.z = with_z ? cv.take_bytes((size_t)m.P * m.h * m.z_es) : nullptr;
     b.a = cv.take_bytes((size_t)m.P * m.h * es);
     b.u = cv.take_bytes((size_t)m.P * m.r * es);
     b.y_lo = cv.take_bytes((size_t)m.T * m.r * es);
@@ -136,6 +143,7 @@ void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
     b.dy_lo = cv.take_bytes((size_t)m.T * m.r * es);
     b.du = cv.take_bytes((size_t)m.P * m.r * es);
     b.dxg = cv.take_bytes((size_t)m.P * m.r * es);
+    b.dz = m.z_es == 1 ? cv.take_bytes((size_t)m.P * m.h * es) : nullptr;
     b.dcat = cv.take_bytes((size_t)m.T * (m.r + m.E64) * es);
     b.dx_lo = b.dcat;
     b.dlogits = b.dcat ? (char*)b.dcat + (size_t)m.r * es : nullptr;
@@ -177,7 +185,8 @@ int check_weights(const bigmac_weights_t* W) {
 int gemm(const bigmac_layer* L, int id, const GemmArgs& g, cudaStream_t st) {
     Stage stage(L, id, st);
     cudaError_t err;
-    if (L->cfg.dtype == BIGMAC_BF16 && L->use_tc && ((L->tc_mask >> id) & 1u))
+    const bool sigma_pair = id == G_EXPERT1 || id == G_DZ;      // these two must agree on the sigma' format
+    if (L->cfg.dtype == BIGMAC_BF16 && L->use_tc && ((L->tc_mask >> id) & 1u) && (!sigma_pair || L->tc_mask == ~0u))
         err = gemm_tc(g, L->status, st);
     else
         err = gemm_simt(g, L->cfg.dtype, st);
@@ -295,7 +304,7 @@ int bigmac_layer_destroy(bigmac_layer_t* L) {
 int bigmac_workspace_bytes(const bigmac_layer_t* L, int32_t T, int training, size_t* scratch_bytes,
                            size_t* saved_bytes) {
     if (!L || !scratch_bytes || !saved_bytes || T < 0 || T > L->cfg.max_tokens) return BIGMAC_ERR_INVALID_ARG;
-    const Dims m = dims_of(L->cfg, T);
+    const Dims m = dims_of(L, T);
     size_t s = forward_scratch_bytes(m, training != 0);
     if (training) {
         const size_t bw = backward_scratch_bytes(m);
@@ -313,7 +322,7 @@ int bigmac_route(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_weigh
     BIGMAC_TRY(check_weights(W));
     if (T == 0) return BIGMAC_OK;
     if (!x || !aligned(x, 16) || !scratch || !aligned(scratch, 256)) return BIGMAC_ERR_INVALID_ARG;
-    const Dims m = dims_of(L->cfg, T);
+    const Dims m = dims_of(L, T);
     if (scratch_bytes < forward_scratch_bytes(m, false)) return BIGMAC_ERR_WORKSPACE;
     Carver cv(scratch);
     Buffers b{};
@@ -333,7 +342,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         !aligned(saved, 256))
         return BIGMAC_ERR_INVALID_ARG;
     const bool training = saved != nullptr;
-    const Dims m = dims_of(L->cfg, T);
+    const Dims m = dims_of(L, T);
     if (scratch_bytes < forward_scratch_bytes(m, training)) return BIGMAC_ERR_WORKSPACE;
     Buffers b{};
     Carver cs(scratch);
@@ -407,7 +416,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     if (!aligned(G->dw_gate, 16) || !aligned(G->dw_down, 16) || !aligned(G->dw1, 16) || !aligned(G->dw2, 16) ||
         !aligned(G->dw_up, 16) || !aligned(G->db_gate, 4))
         return BIGMAC_ERR_INVALID_ARG;
-    const Dims m = dims_of(L->cfg, T);
+    const Dims m = dims_of(L, T);
     if (scratch_bytes < backward_scratch_bytes(m)) return BIGMAC_ERR_WORKSPACE;
     Buffers b{};
     {
@@ -447,12 +456,12 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     {   // dz = (du W2_e) * sigma'(z); the forward saved sigma'(z) in the z buffer, dz is written over it
         GemmArgs g;
         g.A = b.du; g.lda = m.r; g.B = W->w2; g.ldb = m.h; g.b_kmajor = false; g.b_stride = (int64_t)m.r * m.h;
-        g.C = b.z; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
+        g.C = b.dz ? b.dz : b.z; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
         g.epilogue = EPI_DACT; g.act = c.act; g.group = GROUP_M; g.num_experts = m.E;
         g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
         BIGMAC_TRY(gemm(L, G_DZ, g, st));
     }
-    void* dz = b.z;
+    void* dz = b.dz ? b.dz : b.z;
     if (G->dw2) {   // dW2_e[c',q] = sum_rows du[row,c'] a[row,q]
         GemmArgs g;
         g.A = b.du; g.lda = m.r; g.a_kmajor = false; g.B = b.a; g.ldb = m.h; g.b_kmajor = false;
@@ -558,7 +567,7 @@ int bigmac_exchange_rows(bigmac_layer_t* L, const void* saved, int32_t T, int32_
     const size_t es = esize(L->cfg.dtype);
     if ((width * es) % 16) return BIGMAC_ERR_UNSUPPORTED;
     if (T == 0) return BIGMAC_OK;
-    const Dims m = dims_of(L->cfg, T);
+    const Dims m = dims_of(L, T);
     if (grouped_bytes < (size_t)m.P * width * es) return BIGMAC_ERR_WORKSPACE;
     Buffers b{};
     Carver cv(const_cast<void*>(saved));
@@ -626,7 +635,7 @@ int bigmac_route_static(bigmac_layer_t* L, const void* x, int32_t T, const bigma
     BIGMAC_TRY(check_weights(W));
     if (T == 0) return BIGMAC_OK;
     if (!x || !aligned(x, 16)) return BIGMAC_ERR_INVALID_ARG;
-    const Dims m = dims_of(L->cfg, T);
+    const Dims m = dims_of(L, T);
     {
         Carver measure(nullptr);
         Buffers b{};

@@ -206,17 +206,82 @@ __device__ __forceinline__ void act_pair(int act, float z, float& a, float& g) {
     }
 }
 
-// Activation of 32 accumulator values in place; with WITH_G the 32 sigma' values are packed to bf16 pairs in wg.
+// Packed fp32 pairs (sm_100 f32x2 arithmetic): one instruction issue for two elements.
+typedef unsigned long long f32x2_t;
+__device__ __forceinline__ f32x2_t pk2(float a, float b) { f32x2_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ void upk2(f32x2_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ f32x2_t fma2(f32x2_t a, f32x2_t b, f32x2_t c) { f32x2_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+__device__ __forceinline__ f32x2_t mul2(f32x2_t a, f32x2_t b) { f32x2_t d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2_t add2(f32x2_t a, f32x2_t b) { f32x2_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+
+// GELU(erf) and its derivative for two elements at once; same formulas as act_pair (A&S 7.1.26, one ex2 and one
+// rcp per element), with every multiply-add issued as a packed pair and the sign handled by bit operations:
+// Phi(z) = 1/2 + copysign(1/2 - q, z).
+__device__ __forceinline__ void gelu_pair2(float z0, float z1, float& a0, float& a1, float& g0, float& g1) {
+    const f32x2_t z = pk2(z0, z1);
+    const f32x2_t az = z & 0x7fffffff7fffffffull;
+    const f32x2_t den = fma2(az, pk2(0.23164190f, 0.23164190f), pk2(1.0f, 1.0f));
+    float d0, d1;
+    upk2(den, d0, d1);
+    const f32x2_t t = pk2(fast_rcp(d0), fast_rcp(d1));
+    f32x2_t poly = fma2(t, pk2(0.5307027145f, 0.5307027145f), pk2(-0.7265760135f, -0.7265760135f));
+    poly = fma2(t, poly, pk2(0.7107068705f, 0.7107068705f));
+    poly = fma2(t, poly, pk2(-0.142248368f, -0.142248368f));
+    poly = fma2(t, poly, pk2(0.127414796f, 0.127414796f));
+    const f32x2_t arg = mul2(mul2(z, z), pk2(-0.72134752f, -0.72134752f));
+    float x0, x1;
+    upk2(arg, x0, x1);
+    const f32x2_t e = pk2(fast_ex2(x0), fast_ex2(x1));
+    const f32x2_t q = mul2(mul2(poly, t), e);
+    const f32x2_t h = fma2(q, pk2(-1.0f, -1.0f), pk2(0.5f, 0.5f));               // 1/2 - q >= 0
+    const f32x2_t cdf = add2(h | (z & 0x8000000080000000ull), pk2(0.5f, 0.5f));
+    upk2(mul2(z, cdf), a0, a1);
+    upk2(fma2(mul2(z, e), pk2(0.39894228f, 0.39894228f), cdf), g0, g1);
+}
+
+// sigma' is saved as one byte per element: q = round(200 sigma' + 27), i.e. sigma' = (q - 27) / 200 on [-0.135, 1.14]
+// (GELU' lies in [-0.129, 1.129]; 0 and 1, all that ReLU needs, are exact).  The step 0.005 gives an absolute error
+// of at most 0.0025 (rms 0.0014, about 0.23 % of sigma's rms - the size of a bf16 rounding) at half the bytes.
+// Rounding uses the 2^23 trick: the low byte of float(2^23 + 27 + 200 g) is q.
+constexpr float kSigScale = 200.0f, kSigMagic = 8388608.0f + 27.0f, kSigStep = 0.005f;
+__device__ __forceinline__ uint32_t sig_quant4(float g0, float g1, float g2, float g3) {
+    const uint32_t b0 = __float_as_uint(fmaf(g0, kSigScale, kSigMagic)), b1 = __float_as_uint(fmaf(g1, kSigScale, kSigMagic));
+    const uint32_t b2 = __float_as_uint(fmaf(g2, kSigScale, kSigMagic)), b3 = __float_as_uint(fmaf(g3, kSigScale, kSigMagic));
+    return __byte_perm(__byte_perm(b0, b1, 0x0040), __byte_perm(b2, b3, 0x0040), 0x5410);
+}
+__device__ __forceinline__ uint8_t sig_quant1(float g) { return (uint8_t)(__float_as_uint(fmaf(g, kSigScale, kSigMagic)) & 0xffu); }
+template <int I>
+__device__ __forceinline__ float sig_dequant(uint32_t word) {     // byte I of word -> sigma'
+    const uint32_t bits = __byte_perm(word, 0x4B000000u, 0x7650 + I);
+    return (__uint_as_float(bits) - kSigMagic) * kSigStep;
+}
+__device__ __forceinline__ float sig_dequant1(uint8_t q) { return ((float)q - 27.0f) * kSigStep; }
+// v[0..31] *= sigma' from 8 words of 4 bytes
+__device__ __forceinline__ void mul_by_sig32(float* v, const uint32_t* w) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        v[4 * i] *= sig_dequant<0>(w[i]); v[4 * i + 1] *= sig_dequant<1>(w[i]);
+        v[4 * i + 2] *= sig_dequant<2>(w[i]); v[4 * i + 3] *= sig_dequant<3>(w[i]);
+    }
+}
+
+// Activation of 32 accumulator values in place; with WITH_G the 32 sigma' values are packed, one byte each, in wg[0..7].
 // The activation is a compile-time constant here so that the switch is taken once per chunk, not per element.
 template <int ACT, bool WITH_G>
 __device__ __forceinline__ void act_chunk(float* v, uint32_t* wg) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        float a0, g0, a1, g1;
-        act_pair(ACT, v[2 * i], a0, g0);
-        act_pair(ACT, v[2 * i + 1], a1, g1);
-        v[2 * i] = a0; v[2 * i + 1] = a1;
-        if (WITH_G) wg[i] = pack_bf16(g0, g1);
+    for (int i = 0; i < 8; ++i) {
+        float a[4], g[4];
+        if (ACT == BIGMAC_ACT_GELU_ERF) {
+            gelu_pair2(v[4 * i], v[4 * i + 1], a[0], a[1], g[0], g[1]);
+            gelu_pair2(v[4 * i + 2], v[4 * i + 3], a[2], a[3], g[2], g[3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) act_pair(ACT, v[4 * i + j], a[j], g[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[4 * i + j] = a[j];
+        if (WITH_G) wg[i] = sig_quant4(g[0], g[1], g[2], g[3]);
     }
 }
 template <bool WITH_G>
@@ -233,24 +298,21 @@ __device__ __forceinline__ void act_chunk_any(int act, float* v, uint32_t* wg) {
 __device__ __forceinline__ void store_row_chunk(const TcParams& p, float* v, int64_t row_off, int col0, bool vec_ok) {
     const int ncols = min(32, p.N - col0);
     if (ncols <= 0) return;
-    __nv_bfloat16* Zb = (__nv_bfloat16*)p.Z;
+    uint8_t* Zb = (uint8_t*)p.Z;                 // sigma', one byte per element
     if (vec_ok && ncols == 32) {
         const int64_t off = row_off + col0;
         if (p.epilogue == EPI_ACT) {
             if (Zb) {
-                uint32_t w[16];
+                uint32_t w[8];
                 act_chunk_any<true>(p.act, v, w);
                 st_global_32B(Zb + off, w);
-                st_global_32B(Zb + off + 16, w + 8);
             } else {
                 act_chunk_any<false>(p.act, v, nullptr);
             }
         } else if (p.epilogue == EPI_DACT) {
-            uint32_t w[16];
+            uint32_t w[8];
             ld_global_32B(Zb + off, w);
-            ld_global_32B(Zb + off + 16, w + 8);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) { v[2 * i] *= bf16_lo(w[i]); v[2 * i + 1] *= bf16_hi(w[i]); }
+            mul_by_sig32(v, w);
         }
         if (p.out_f32) {
             float* cp = (float*)p.C + off;
@@ -290,9 +352,9 @@ __device__ __forceinline__ void store_row_chunk(const TcParams& p, float* v, int
         if (p.epilogue == EPI_ACT) {
             float g;
             act_pair(p.act, x, x, g);
-            if (Zb) Zb[off] = __float2bfloat16(g);
+            if (Zb) Zb[off] = sig_quant1(g);
         } else if (p.epilogue == EPI_DACT) {
-            x *= __bfloat162float(Zb[off]);
+            x *= sig_dequant1(Zb[off]);
         }
         if (p.out_f32) {
             float* C = (float*)p.C;
@@ -314,6 +376,13 @@ __device__ __forceinline__ void stage_row_bf16(uint8_t* box, int lane, const uin
     for (int j = 0; j < 4; ++j) st_shared_16B(row + ((j ^ sw) << 4), w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
 }
 
+// 32 rows x 32 sigma' bytes for a TMA store without swizzle: row `lane` occupies 32 bytes.
+__device__ __forceinline__ void stage_row_u8(uint8_t* box, int lane, const uint32_t* w /*8 words*/) {
+    uint8_t* row = box + lane * 32;
+    st_shared_16B(row, w[0], w[1], w[2], w[3]);
+    st_shared_16B(row + 16, w[4], w[5], w[6], w[7]);
+}
+
 // Epilogue of 32 columns through shared memory: v -> (sigma', sigma) or v * Z or v, packed to bf16 into the
 // warp's staging boxes.  Returns nothing; the caller fences and issues the TMA stores.
 __device__ __forceinline__ void stage_row_chunk(const TcParams& p, float* v, uint8_t* box_c, uint8_t* box_z, int lane,
@@ -322,7 +391,7 @@ __device__ __forceinline__ void stage_row_chunk(const TcParams& p, float* v, uin
     if (p.epilogue == EPI_ACT) {
         if (p.Z) {
             act_chunk_any<true>(p.act, v, w);
-            stage_row_bf16(box_z, lane, w);
+            stage_row_u8(box_z, lane, w);
         } else {
             act_chunk_any<false>(p.act, v, nullptr);
         }
@@ -376,6 +445,7 @@ __device__ __forceinline__ Tile get_tile(const TcParams& p, int BN, int t, int t
 
 constexpr int kEpiWarps = 16;
 constexpr uint32_t kBoxBytes = 32 * 64;                  // 32 rows x 32 bf16 columns
+constexpr uint32_t kBoxBytesZ = 32 * 32;                 // 32 rows x 32 sigma' bytes
 constexpr int kThreadsV2 = (2 + kEpiWarps) * 32;
 
 
@@ -397,6 +467,20 @@ inline EncodeTiledFn encode_fn() {
 }
 
 // 2-D bf16 tensor map: `inner` contiguous elements per row, `rows` rows `ld` elements apart.
+// 2-D byte tensor map (the saved sigma'): `inner` bytes per row, rows `ld` bytes apart, no swizzle.
+inline bool make_map_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner,
+                        uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {inner, rows};
+    const cuuint64_t strides[1] = {ld};
+    const cuuint32_t box[2] = {box_inner, box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 inline bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner,
               uint32_t box_rows, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     EncodeTiledFn fn = encode_fn();
@@ -425,7 +509,7 @@ inline int sm_count() {
 // Can this problem's output leave through shared memory and TMA stores?
 inline bool tma_epilogue_possible(const GemmArgs& g) {
     return !g.out_f32 && !g.accumulate && g.split_k <= 1 && (g.ldc % 8 == 0) && ((uintptr_t)g.C % 16 == 0) &&
-           ((uintptr_t)g.Z % 16 == 0) &&
+           ((uintptr_t)g.Z % 16 == 0) && (g.Z == nullptr || g.ldc % 16 == 0) &&
            (g.group != GROUP_K || (g.M % BM == 0 && g.c_stride == (int64_t)g.M * g.ldc));
 }
 

@@ -139,29 +139,32 @@ def test_grouped_rows_forward_and_backward_epilogues(N):
     d_nt = torch.tensor([len(tile_expert)], dtype=torch.int32, device="cuda")
     d_po = torch.from_numpy(poff).cuda()
     C = torch.full((P, N), float("nan"), dtype=torch.bfloat16, device="cuda")
-    Z = torch.full((P, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Z = torch.full((P, N), 255, dtype=torch.uint8, device="cuda")     # tensor-core path: sigma' as bytes, (q - 27) / 200
     layer = _layer()
     _run(layer, _q(A=_dev_bf16(A), B=_dev_bf16(W), C=C, Z=Z, lda=K, ldb=K, ldc=N, M=P, N=N, K=K, a_kmajor=1, b_kmajor=1,
                    epilogue=1, act=1, group=1, num_experts=E, b_stride=N * K, tile_expert=d_te, n_tiles=d_nt, poffsets=d_po))
-    got_c, got_z = _np(C), _np(Z)
+    got_c, got_z = _np(C), (Z.cpu().numpy().astype(np.float64) - 27.0) / 200.0
     for e, c in enumerate(counts):
         rows = slice(poff[e], poff[e + 1])
         z = A[rows].astype(np.float64) @ W[e].astype(np.float64).T
-        _close(got_z[rows], _dgelu(z))
+        if z.size:
+            assert np.max(np.abs(got_z[rows] - _dgelu(z))) <= 0.0026       # half a quantisation step (+ fp32 noise)
         _close(got_c[rows], _gelu(z))
     assert np.isnan(got_c[poff[-1]:]).all()                     # nothing beyond the live tiles is touched
 
-    # input-gradient form: K-major A, MN-major per-expert weights, multiply by the saved sigma' in place over Z
+    # input-gradient form: K-major A, MN-major per-expert weights, multiply by the saved sigma' bytes
     G = np.zeros((P, N), dtype=np.float32)                       # "du": [P, N] now the contraction side
     for e, c in enumerate(counts):
         G[poff[e]:poff[e] + c] = _rand((c, N), 40 + e)
     N2 = K if N == 192 else 1024                                 # output width
     Wt = _rand((E, N, N2), 12, N ** -0.5)                        # B(n2, k=n) = Wt[e][n, n2]
-    Zin = _rand((P, N2), 13)
-    Zd = _dev_bf16(Zin)
-    _run(layer, _q(A=_dev_bf16(G), B=_dev_bf16(Wt), C=Zd, Z=Zd, lda=N, ldb=N2, ldc=N2, M=P, N=N2, K=N, a_kmajor=1,
+    q_in = np.random.default_rng(13).integers(0, 256, size=(P, N2)).astype(np.uint8)
+    Zin = (q_in.astype(np.float64) - 27.0) / 200.0
+    Zd = torch.from_numpy(q_in).cuda()
+    Cd = torch.full((P, N2), float("nan"), dtype=torch.bfloat16, device="cuda")
+    _run(layer, _q(A=_dev_bf16(G), B=_dev_bf16(Wt), C=Cd, Z=Zd, lda=N, ldb=N2, ldc=N2, M=P, N=N2, K=N, a_kmajor=1,
                    b_kmajor=0, epilogue=2, act=1, group=1, num_experts=E, b_stride=N * N2, tile_expert=d_te, n_tiles=d_nt, poffsets=d_po))
-    got = _np(Zd)
+    got = _np(Cd)
     for e in range(E):
         rows = slice(poff[e], poff[e + 1])
         ref = (G[rows].astype(np.float64) @ Wt[e].astype(np.float64)) * Zin[rows].astype(np.float64)
