@@ -298,6 +298,23 @@ def run_ours(args, w):
         fwd_only()
     ms_fwd = timed(fwd_only, args.steps) / args.steps
 
+    # small batches are launch-bound: also time the same forward replayed from a CUDA graph (the C ABI neither
+    # allocates nor synchronises, so a caller can capture it)
+    ms_fwd_graph = None
+    if w.T <= 1024:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fwd_only()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            fwd_only()
+        for _ in range(3):
+            graph.replay()
+        ms_fwd_graph = timed(graph.replay, args.steps) / args.steps
+
     # ---- the exchange stage alone at width r (BigMac) and at width d (a fine-grained CDAC layer of equal E, k
     # dispatches and combines full-width rows, Eq. 1): same kernels, same routing, rank 0's GPU only
     exchange = None
@@ -387,7 +404,8 @@ def run_ours(args, w):
                     "d2h_bytes_per_step": bytes_io, "ms_per_step": ms_e2e},
             "gpu_launches": prof["launches"],
             "forward_only": {"tokens_per_s": world * w.T / (ms_fwd * 1e-3), "ms": ms_fwd,
-                             "frac_of_tensor_roofline": round(fwd_fl / (ms_fwd * 1e-3) / 1e12 / peaks["tflops_sustained"], 4)},
+                             "frac_of_tensor_roofline": round(fwd_fl / (ms_fwd * 1e-3) / 1e12 / peaks["tflops_sustained"], 4),
+                             "cuda_graph_ms": ms_fwd_graph},
             "roofline": roofline,
             "cpu_baseline": {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": f"first {S_used} tokens of the workload, routing + forward + backward with "

@@ -124,4 +124,11 @@ cudaError_t launch_colsum(const void* dlogits, float* db, float* partial, int T,
 cudaError_t launch_splitk_reduce(const float* ws, int parts, int M, int N, void* dst1, int m_split, void* dst2, int m2,
                                  int dtype, bool accumulate, cudaStream_t stream);
 
+// Small-batch inference forward in one cooperative kernel (bf16, T <= 16): scratch logits [T,E], x_lo [T,r],
+// a [T*k,h], u [T*k,r] fp32; writes y, topk_idx, topk_w.  `barrier` is one device word owned by the handle.
+bool decode_forward_supported(int T, int d, int r, int h, int E, int k, int dtype);
+cudaError_t launch_decode_forward(const void* x, const bigmac_weights_t* W, void* y, float* logits, float* x_lo, float* a,
+                                  float* u, int32_t* topk_idx, float* topk_w, unsigned* barrier, int* status, int T, int d,
+                                  int r, int h, int E, int k, int act, int num_sms, cudaStream_t stream);
+
 }  // namespace bigmac

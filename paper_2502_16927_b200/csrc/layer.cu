@@ -16,7 +16,7 @@ using namespace bigmac;
 struct bigmac_layer {
     bigmac_config_t cfg;
     int device;
-    int* status;        // device status word
+    int* status;        // device status word; status[1] is the grid-barrier counter of the small-batch kernel
     bool use_tc;        // bf16 contractions on tcgen05
     unsigned tc_mask;   // debug: bit i set = contraction i runs on tcgen05 (BIGMAC_TC_MASK)
     // measurement aid
@@ -35,12 +35,12 @@ namespace {
 enum { G_LOGITS = 0, G_DESCEND, G_EXPERT1, G_EXPERT2, G_ASCEND, G_DY_LO, G_DW_UP, G_DZ, G_DW2, G_DXG, G_DW1,
        G_DX, G_DX_GATE, G_DW_DOWN, G_DW_GATE,
        S_TOPK, S_TABLES, S_DISPATCH, S_COMBINE, S_COMBINE_BWD, S_GATE_BWD, S_DXLO_GATHER, S_COLSUM, S_SPLITK_REDUCE,
-       S_COUNT };
+       S_DECODE, S_COUNT };
 const char* const kSlotNames[S_COUNT] = {
     "gemm_logits", "gemm_descend", "gemm_expert1", "gemm_expert2", "gemm_ascend", "gemm_dy_lo", "gemm_dw_up",
     "gemm_dz", "gemm_dw2", "gemm_dxg", "gemm_dw1", "gemm_dx", "gemm_dx_gate", "gemm_dw_down", "gemm_dw_gate",
     "topk", "tables", "dispatch", "combine", "combine_bwd", "gate_bwd", "dxlo_gather", "colsum",
-    "splitk_reduce"};
+    "splitk_reduce", "decode_forward"};
 constexpr size_t kEventPairs = 8192;
 constexpr int kMaxSplitK = 8;
 
@@ -279,8 +279,8 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
     L->use_tc = cfg->dtype == BIGMAC_BF16 && !(cfg->flags & BIGMAC_FLAG_SIMT_GEMM);
     L->tc_mask = ~0u;
     if (const char* env = std::getenv("BIGMAC_TC_MASK")) L->tc_mask = (unsigned)std::strtoul(env, nullptr, 0);
-    if (cudaGetDevice(&L->device) != cudaSuccess || cudaMalloc((void**)&L->status, sizeof(int)) != cudaSuccess ||
-        cudaMemset(L->status, 0, sizeof(int)) != cudaSuccess) {
+    if (cudaGetDevice(&L->device) != cudaSuccess || cudaMalloc((void**)&L->status, 2 * sizeof(int)) != cudaSuccess ||
+        cudaMemset(L->status, 0, 2 * sizeof(int)) != cudaSuccess) {
         delete L;
         return BIGMAC_ERR_CUDA;
     }
@@ -356,6 +356,20 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     cudaStream_t st = (cudaStream_t)stream;
     const bigmac_config_t& c = L->cfg;
 
+    // A few tokens, inference: the whole forward in one cooperative kernel (weight streaming, no tensor cores)
+    if (!training && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
+        {
+            Stage s(L, S_DECODE, st);
+            BIGMAC_CUDA(launch_decode_forward(x, W, y, b.logits, (float*)b.xg, (float*)b.a, (float*)b.u, b.tb.topk_idx,
+                                              b.tb.topk_w, (unsigned*)(L->status + 1), L->status, m.T, m.d, m.r, m.h, m.E,
+                                              m.k, c.act, gemm_tc_sm_count(), st));
+        }
+        if (routing_out) {
+            { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, st)); }
+            BIGMAC_TRY(export_routing(m, b, routing_out, st));
+        }
+        return BIGMAC_OK;
+    }
     // F1 + F4 in one pass over x when the tile grid allows it: [x' | logits] = x [W'_down ; W_gate]^T, logits in fp32
     const int bn_desc = (m.r + m.E) >= 256 ? 256 : 128;
     const bool fuse_gate = c.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u && m.r % bn_desc == 0;

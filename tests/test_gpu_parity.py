@@ -240,3 +240,31 @@ def binding_exchange(layer, w, width, src, grouped, dst):
     from paper_2502_16927_b200 import binding
 
     binding.bigmac_exchange_rows(layer.handle, layer._saved, w.T, width, src, grouped, dst, 2)
+
+
+@pytest.mark.parametrize("T", [1, 3, 8, 16])
+@pytest.mark.parametrize("shape", [
+    dict(d=2048, r=256, h=1024, E=64, k=8),        # the decode configuration
+    dict(d=192, r=64, h=320, E=5, k=5),            # k = E, ragged widths
+    dict(d=64, r=128, h=64, E=40, k=1),
+])
+def test_small_batch_inference_forward(T, shape):
+    """Inference forward at a handful of tokens (one fused kernel): y and the routing tables against the oracle."""
+    import torch
+
+    w = wl.Workload("decode", T=T, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=300 + T, **shape)
+    inp = conditioned(w)
+    inp["b_gate"] = (np.linspace(-0.2, 0.2, w.E)).astype(np.float32)
+    margin.enforce_margin(w, inp, 1e-3)
+    dev = to_device(w, inp)
+    layer = make_layer(w)
+    y, R = layer.forward(dev["x"], dev, training=False, want_routing=True)
+    y2 = layer.forward(dev["x"], dev, training=False)            # no tables requested: same kernel, same result
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    rt = oracle.route(inp, w.k)
+    check_routing(R, rt)
+    ref = oracle.forward_tokens(inp, rt, w.act)["y"]
+    assert_within(w, float_errors(w, {"y": to_numpy(y)}, {"y": ref}))
+    assert torch.equal(y, y2)
+    layer.close()
