@@ -259,11 +259,12 @@ cudaError_t launch_decode_forward(const void* x, const bigmac_weights_t* W, void
     p.topk_idx = topk_idx; p.topk_w = topk_w; p.barrier = barrier; p.status = status;
     p.T = T; p.d = d; p.r = r; p.h = h; p.E = E; p.k = k; p.act = act;
     const size_t smem = sizeof(float) * (size_t)T * (d > r ? d : r);
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce once;
+    int dev;
+    if (once.needed(&dev)) {
         cudaError_t e = cudaFuncSetAttribute(decode_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
         if (e != cudaSuccess) return e;
-        configured = true;
+        once.mark(dev);
     }
     cudaError_t err = cudaMemsetAsync(barrier, 0, sizeof(unsigned), stream);
     if (err != cudaSuccess) return err;

@@ -238,12 +238,13 @@ cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorM
                    const CUtensorMap& mb2, const TcParams& p, int max_tiles, cudaStream_t stream) {
     constexpr size_t smem = STAGES * (BM * BK * 2 + BN * BK * 2) + (TMA_EPI ? kEpiWarps * 2 * kBoxBytes : 0) +
                             (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + 1024;
-    static bool configured = false;
+    static PerDeviceOnce once;
     auto kernel = gemm_tc_kernel<BN, STAGES, AK, BKM, TMA_EPI>;
-    if (!configured) {
+    int dev;
+    if (once.needed(&dev)) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured = true;
+        once.mark(dev);
     }
     const int grid = max_tiles < sm_count() ? max_tiles : sm_count();
     kernel<<<grid, kThreadsV2, smem, stream>>>(ma, mb, mc, mz, mb2, p);

@@ -355,12 +355,13 @@ cudaError_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUte
     const size_t smem = STAGES * (BM * BK * 2 + (BN / 2) * BK * 2) + (TMA_EPI ? kEpiWarps * 2 * kBoxBytes : 0) +
                         (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + (size_t)(p.num_experts + 1) * 4 + 1024;
     if (smem > kMaxSmem) return cudaErrorInvalidConfiguration;
-    static bool configured = false;
+    static PerDeviceOnce once;
     auto kernel = gemm_tc_pair_kernel<BN, STAGES, AK, BKM, TMA_EPI>;
-    if (!configured) {
+    int dev;
+    if (once.needed(&dev)) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
         if (e != cudaSuccess) return e;
-        configured = true;
+        once.mark(dev);
     }
     int64_t clusters = sm_count() / 2;
     if (max_items < clusters) clusters = max_items;

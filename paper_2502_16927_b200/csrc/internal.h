@@ -89,6 +89,19 @@ struct Tables {
     int32_t* block_counts;  // [n_blocks, E] scratch of the counting sort
 };
 
+// Per-device one-time launch configuration (function attributes are per device; a process may use several).
+struct PerDeviceOnce {
+    unsigned long long done = 0;           // bit d: configured on device d (d < 64)
+    // true if `fn` still has to run on the current device
+    bool needed(int* device_out) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *device_out = -1; return true; }
+        *device_out = dev;
+        return !((done >> dev) & 1ull);
+    }
+    void mark(int dev) { if (dev >= 0) done |= 1ull << dev; }
+};
+
 inline int64_t padded_rows_max(int64_t N, int E) { return ((N + kPad - 1) / kPad + E) * (int64_t)kPad; }
 constexpr int kSortChunk = 1024;   // slots per block of the counting sort
 inline int sort_blocks(int64_t N) { return (int)((N + kSortChunk - 1) / kSortChunk); }

@@ -495,16 +495,14 @@ inline bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_
 }
 
 inline int sm_count() {
-    static int n = []() {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
-            return 148;
-        return v;
-    }();
-    return n;
+    static int cached[64] = {};
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] > 0) return cached[dev];
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+    cached[dev] = v;
+    return v;
 }
-
 
 // Can this problem's output leave through shared memory and TMA stores?
 inline bool tma_epilogue_possible(const GemmArgs& g) {
