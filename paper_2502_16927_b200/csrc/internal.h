@@ -124,13 +124,15 @@ cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const
 cudaError_t launch_combine_bwd(const void* dy_lo, const void* u, void* du, float* dp, const Tables& tb, int k,
                                int width, int dtype, int64_t max_prows, cudaStream_t stream);
 // Softmax-over-k backward: g = sum_i p_i dp_i, dl_j = p_j (dp_j - g); writes the dense [T,E] matrix
-// (zeros off the top-k set, and in the padding columns E..width-1) in the dtype, rows `ld` elements apart.
-cudaError_t launch_gate_bwd(const float* dp, const Tables& tb, void* dlogits, int T, int E, int width, int ld, int k,
+// (zeros off the top-k set, and in the padding columns E..width-1) in the dtype, rows `ld` elements apart, and
+// leaves the fp32 dl_j in dp[slot].
+cudaError_t launch_gate_bwd(float* dp, const Tables& tb, void* dlogits, int T, int E, int width, int ld, int k,
                             int dtype, cudaStream_t stream);
-// db[e] (+)= sum_t dlogits[t,e]; `partial` holds kColsumChunks * E floats of scratch.
-constexpr int kColsumChunks = 64;
-cudaError_t launch_colsum(const void* dlogits, float* db, float* partial, int T, int E, int ld, int dtype,
-                          bool accumulate, cudaStream_t stream);
+// db[e] (+)= sum over the slots routed to e of dl_slot[slot] (the fp32 per-slot gate gradients launch_gate_bwd
+// leaves in dp); `partial` holds kColsumChunks * E floats of scratch.  Deterministic summation order.
+constexpr int kColsumChunks = 296;
+cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db, float* partial, int64_t N, int E,
+                               bool accumulate, cudaStream_t stream);
 // Sum the `parts` fp32 partial results ws[s][m][n] of a split contraction in the order s = 0, 1, ... and write
 // rows [0, m_split) to dst1 [m_split, N] and rows [m_split, m_split + m2) to dst2 [m2, N] (dst2 may be null),
 // in the dtype, adding to the destination if `accumulate`.

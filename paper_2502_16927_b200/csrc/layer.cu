@@ -543,7 +543,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
             BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
         }
     }
-    if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_colsum(b.dlogits, G->db_gate, b.colsum_part, m.T, m.E, ldcat, m.dtype, acc, st)); }
+    if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st)); }
     return BIGMAC_OK;
 }
 

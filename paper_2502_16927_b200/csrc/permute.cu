@@ -139,14 +139,14 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const uint4* __restric
 }
 
 template <typename T>
-__global__ void __launch_bounds__(256) gate_bwd_kernel(const float* __restrict__ dp, const float* __restrict__ topk_w,
+__global__ void __launch_bounds__(256) gate_bwd_kernel(float* __restrict__ dp, const float* __restrict__ topk_w,
                                                        const int32_t* __restrict__ topk_idx, T* __restrict__ dlogits,
                                                        int n_tokens, int E, int width, int ld, int k) {
     const int t = warp_global_id();
     if (t >= n_tokens) return;
     const int lane = threadIdx.x & 31;
     const float* p = topk_w + (int64_t)t * k;
-    const float* g = dp + (int64_t)t * k;
+    float* g = dp + (int64_t)t * k;
     float part = 0.0f;
     for (int j = lane; j < k; j += 32) part = fmaf(p[j], g[j], part);
 #pragma unroll
@@ -154,28 +154,43 @@ __global__ void __launch_bounds__(256) gate_bwd_kernel(const float* __restrict__
     T* row = dlogits + (int64_t)t * ld;
     for (int e = lane; e < width; e += 32) row[e] = (T)0.0f;
     __syncwarp();
-    for (int j = lane; j < k; j += 32) row[topk_idx[(int64_t)t * k + j]] = (T)(p[j] * (g[j] - part));
+    for (int j = lane; j < k; j += 32) {
+        const float dl = p[j] * (g[j] - part);
+        row[topk_idx[(int64_t)t * k + j]] = (T)dl;
+        g[j] = dl;                                   // fp32 copy per slot, for the bias gradient
+    }
 }
 
-// Column sums in two deterministic stages: blockIdx.y owns a contiguous chunk of rows and writes its partial
-// sums; a second kernel adds the chunks in order.
-template <typename T>
-__global__ void __launch_bounds__(256) colsum_partial_kernel(const T* __restrict__ m, float* __restrict__ partial, int rows,
-                                                             int cols, int ld) {
-    __shared__ float part[8][33];
-    const int c = blockIdx.x * 32 + (threadIdx.x & 31);
-    const int g = threadIdx.x >> 5;
-    const int per = (rows + gridDim.y - 1) / gridDim.y;
-    const int r0 = blockIdx.y * per, r1 = min(rows, r0 + per);
-    float acc = 0.0f;
-    if (c < cols)
-        for (int r = r0 + g; r < r1; r += 8) acc += (float)m[(int64_t)r * ld + c];
-    part[g][threadIdx.x & 31] = acc;
+// Bias gradient db[e] = sum over slots routed to e of dl[slot], from the fp32 per-slot values, in two
+// deterministic stages.  Block b owns a contiguous range of slots, its warps contiguous sub-ranges; a warp walks
+// its range 32 slots at a time and lane l adds, in slot order, the values of the experts e with e % 32 == l into
+// the warp's row of shared memory.  The block then adds its warps' rows in order.
+__global__ void __launch_bounds__(256) colsum_slots_kernel(const float* __restrict__ dl, const int32_t* __restrict__ topk_idx,
+                                                           float* __restrict__ partial, int64_t N, int E) {
+    extern __shared__ float warp_acc[];              // [8][E]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < 8 * E; i += blockDim.x) warp_acc[i] = 0.0f;
     __syncthreads();
-    if (g == 0 && c < cols) {
+    const int64_t per_warp = ((N + (int64_t)gridDim.x * 8 - 1) / ((int64_t)gridDim.x * 8) + 31) / 32 * 32;
+    const int64_t s0 = ((int64_t)blockIdx.x * 8 + warp) * per_warp;
+    const int64_t s1 = s0 + per_warp < N ? s0 + per_warp : N;
+    float* mine = warp_acc + warp * E;
+    for (int64_t base = s0; base < s1; base += 32) {
+        const int64_t s = base + lane;
+        const int e = s < s1 ? topk_idx[s] : -1;
+        const float v = s < s1 ? dl[s] : 0.0f;
+#pragma unroll 8
+        for (int i = 0; i < 32; ++i) {
+            const int ei = __shfl_sync(kFull, e, i);
+            const float vi = __shfl_sync(kFull, v, i);
+            if (ei >= 0 && (ei & 31) == lane) mine[ei] += vi;
+        }
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
         float total = 0.0f;
-        for (int i = 0; i < 8; ++i) total += part[i][threadIdx.x];
-        partial[(int64_t)blockIdx.y * cols + c] = total;
+        for (int w = 0; w < 8; ++w) total += warp_acc[w * E + e];
+        partial[(int64_t)blockIdx.x * E + e] = total;
     }
 }
 
@@ -249,7 +264,7 @@ cudaError_t launch_combine_bwd(const void* dy_lo, const void* u, void* du, float
     return cudaGetLastError();
 }
 
-cudaError_t launch_gate_bwd(const float* dp, const Tables& tb, void* dlogits, int T, int E, int width, int ld, int k,
+cudaError_t launch_gate_bwd(float* dp, const Tables& tb, void* dlogits, int T, int E, int width, int ld, int k,
                             int dtype, cudaStream_t stream) {
     if (T == 0) return cudaSuccess;
     if (dtype == BIGMAC_BF16)
@@ -260,13 +275,9 @@ cudaError_t launch_gate_bwd(const float* dp, const Tables& tb, void* dlogits, in
     return cudaGetLastError();
 }
 
-cudaError_t launch_colsum(const void* dlogits, float* db, float* partial, int T, int E, int ld, int dtype,
-                          bool accumulate, cudaStream_t stream) {
-    dim3 grid((unsigned)((E + 31) / 32), kColsumChunks);
-    if (dtype == BIGMAC_BF16)
-        colsum_partial_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)dlogits, partial, T, E, ld);
-    else
-        colsum_partial_kernel<float><<<grid, 256, 0, stream>>>((const float*)dlogits, partial, T, E, ld);
+cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db, float* partial, int64_t N, int E,
+                               bool accumulate, cudaStream_t stream) {
+    colsum_slots_kernel<<<kColsumChunks, 256, sizeof(float) * 8 * E, stream>>>(dl_slot, tb.topk_idx, partial, N, E);
     colsum_final_kernel<<<(unsigned)((E + 255) / 256), 256, 0, stream>>>(partial, db, kColsumChunks, E, accumulate);
     return cudaGetLastError();
 }

@@ -157,6 +157,44 @@ def test_bf16_edge_shapes(shape, act):
     compare_full(w, inp, run_full(w, inp))
 
 
+@pytest.mark.parametrize("case", [
+    # one expert takes a slot of nearly every token
+    dict(shape=dict(T=6000, d=256, r=256, h=512, E=16, k=2), bias="one_hot"),
+    # graded popularity: expert loads from thousands of rows down to none
+    dict(shape=dict(T=6000, d=256, r=256, h=256, E=24, k=3), bias="graded"),
+    # balanced, many row tiles per expert
+    dict(shape=dict(T=20000, d=256, r=256, h=256, E=24, k=2), bias=None),
+])
+def test_bf16_skewed_routing(case):
+    """Expert-load skew (dropless routing keeps every slot, so one expert may hold most rows and others none):
+    results must match the oracle as for balanced routing, also when accumulating into existing gradients."""
+    import torch
+
+    w = wl.Workload("skew", dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=311, **case["shape"])
+    inp = conditioned(w)
+    if case["bias"] == "one_hot":
+        b = np.zeros(w.E, dtype=np.float32)
+        b[3] = 8.0
+        inp["b_gate"] = b
+    elif case["bias"] == "graded":
+        inp["b_gate"] = (2.5 * np.linspace(1.0, -1.0, w.E) ** 3).astype(np.float32)
+    margin.enforce_margin(w, inp, 1e-3)
+    got = run_full(w, inp)
+    compare_full(w, inp, got)
+    if case["bias"] == "one_hot":
+        assert got["routing"]["counts"][3].item() >= 0.9 * w.T
+        dev = to_device(w, inp)
+        layer = make_layer(w)
+        layer.forward(dev["x"], dev, training=True)
+        G1 = empty_grads(w, "cuda", fill=0.5)
+        layer.backward(dev["x"], dev["dy"], dev, G1, accumulate=True)
+        torch.cuda.synchronize()
+        for key in ("dw1", "dw2"):
+            ref = got[key] + 0.5
+            assert np.max(np.abs(to_numpy(G1[key]) - ref)) <= 2.0 ** -7 * np.max(np.abs(ref)), key
+        layer.close()
+
+
 def test_route_matches_forward_tables_and_zero_tokens_is_a_noop():
     import torch
 
