@@ -197,6 +197,70 @@ def whole_job_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float)
     return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
+def run_cdac_twin(w, x, dy, dev, ms_step, ms_fwd, steps, peaks, esz):
+    """The conventional fine-grained layer (Eq. 3) with the same E, k, d and expert parameter count (experts
+    d -> m -> d, m = r h / d), same x, dy, gate and routing, through the same entry points and kernels: what one
+    GPU pays for the layer when tokens travel at width d and there are no shared projections."""
+    import torch
+    from paper_2502_16927_b200 import binding
+
+    if w.dtype != wl.DTYPE_BF16 or (w.r * w.h) % w.d or (w.r * w.h // w.d) % 64:
+        return None
+    t = w.cdac_twin()
+    gen = torch.Generator(device="cuda").manual_seed(w.seed)
+    tw = {"w_gate": dev["w_gate"],
+          "w1": (torch.randn((t.E, t.h, t.d), generator=gen, device="cuda") * t.d ** -0.5).to(torch.bfloat16),
+          "w2": (torch.randn((t.E, t.d, t.h), generator=gen, device="cuda") * t.h ** -0.5).to(torch.bfloat16)}
+    if "b_gate" in dev:
+        tw["b_gate"] = dev["b_gate"]
+    G = {"dw_gate": torch.empty_like(tw["w_gate"]), "dw1": torch.empty_like(tw["w1"]), "dw2": torch.empty_like(tw["w2"]),
+         "db_gate": torch.empty(t.E, dtype=torch.float32, device="cuda")}
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    layer = binding.Layer(t.d, t.r, t.h, t.E, t.k, t.T, t.dtype, t.act, wl.FLAG_CDAC)
+
+    def step():
+        layer.forward(x, tw, y=y, training=True)
+        layer.backward(x, dy, tw, G, dx=dx)
+
+    def timed(fn, n):
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(n):
+            fn()
+        stop.record()
+        torch.cuda.synchronize()
+        return start.elapsed_time(stop) / n
+
+    for _ in range(3):
+        step()
+    binding.bigmac_profile_enable(layer.handle, True)
+    ms = timed(step, steps)
+    prof = binding.bigmac_profile_read(layer.handle)
+    binding.bigmac_profile_enable(layer.handle, False)
+    fwd = lambda: layer.forward(x, tw, y=y, training=False)
+    for _ in range(3):
+        fwd()
+    ms_f = timed(fwd, steps)
+    if layer.status() != 0:
+        raise RuntimeError("device status word reports a timed-out wait")
+    stages = {}
+    for name, (tot, calls) in prof["stages"].items():
+        per = tot / calls
+        entry = {"ms": round(per, 4)}
+        if name in GEMM_FLOPS:
+            entry["tflops"] = round(GEMM_FLOPS[name](t) / (per * 1e-3) / 1e12, 1)
+        elif name in ROW_MOVE_BYTES:
+            entry["gbs"] = round(ROW_MOVE_BYTES[name](t, esz) / (per * 1e-3) / 1e9, 1)
+        stages[name] = entry
+    layer.close()
+    return {"config": {"workload": t.name, "T": t.T, "d": t.d, "expert_hidden_m": t.h, "E": t.E, "k": t.k,
+                       "expert_parameters": 2 * t.E * t.d * t.h, "bigmac_expert_parameters": 2 * w.E * w.r * w.h},
+            "ms_per_step": ms, "tokens_per_s": t.T / (ms * 1e-3), "forward_ms": ms_f,
+            "bigmac_over_cdac_time": {"fwd_bwd": round(ms_step / ms, 3), "fwd": round(ms_fwd / ms_f, 3)},
+            "stages": stages}
+
+
 # ------------------------------------------------------------------------------------------------ ours
 def run_ours(args, w):
     import torch
@@ -362,6 +426,7 @@ def run_ours(args, w):
 
     peaks = measured_peaks()
     esz = 2 if w.dtype == wl.DTYPE_BF16 else 4
+    twin = run_cdac_twin(w, x, dy, dev, ms_step, ms_fwd, max(3, min(args.steps, 10)), peaks, esz)
     stages = {}
     gemm_ms = gemm_flops = 0.0
     flops_of = {name: fn(w) for name, fn in GEMM_FLOPS.items()}
@@ -414,6 +479,7 @@ def run_ours(args, w):
                              "sample": f"first {S_used} tokens of the workload, routing + forward + backward with "
                                        f"every gradient, {dt:.1f} s"},
             "exchange": exchange,
+            "cdac_twin": twin,
             "stages": stages}
     print(json.dumps(line))
     if world > 1:

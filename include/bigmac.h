@@ -71,6 +71,13 @@ typedef enum {
 
 /* flags */
 #define BIGMAC_FLAG_SIMT_GEMM 1u /* BF16 only: run every contraction on the plain FMA kernels (debug aid) */
+/* The conventional fine-grained MoE layer the paper compares with (Eq. 3, the communicate-descend-ascend-
+ * communicate structure): y = sum_{i in T} p_i(x) E_i(x) with experts that map d -> h -> d themselves, so tokens are
+ * dispatched and combined at the full width d and there are no shared projections.  Requires r == d; w_down, w_up,
+ * dw_down and dw_up are ignored (may be NULL); w1 is [E,h,d], w2 is [E,d,h].  Same routing, same kernels, same
+ * entry points: the like-for-like single-GPU counterpart of the BigMac layer (parameter parity: h = r'h'/d for a
+ * BigMac layer with low width r' and expert hidden width h'). */
+#define BIGMAC_FLAG_CDAC 2u
 
 typedef struct {
     int32_t d, r, h, E, k; /* 1 <= k <= E */

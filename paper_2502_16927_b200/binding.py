@@ -132,8 +132,9 @@ def bigmac_workspace_bytes(handle, T: int, training: bool):
 
 
 def _weights(W: Dict[str, torch.Tensor]) -> bigmac_weights_t:
-    return bigmac_weights_t(_ptr(W["w_gate"]), _ptr(W.get("b_gate")), _ptr(W["w_down"]), _ptr(W["w1"]), _ptr(W["w2"]),
-                            _ptr(W["w_up"]))
+    # w_down / w_up are absent for the projection-free layer (BIGMAC_FLAG_CDAC)
+    return bigmac_weights_t(_ptr(W["w_gate"]), _ptr(W.get("b_gate")), _ptr(W.get("w_down")), _ptr(W["w1"]), _ptr(W["w2"]),
+                            _ptr(W.get("w_up")))
 
 
 def _routing(R: Optional[Dict[str, torch.Tensor]]):

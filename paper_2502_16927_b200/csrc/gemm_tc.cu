@@ -147,18 +147,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int esz = p.out_f32 ? 4 : 2;
         const bool vec_ok = ((p.ldc * esz) % 32 == 0) && ((p.c_stride * esz) % 32 == 0) && (p.ldc % 16 == 0) &&
                             (((uintptr_t)p.C) % 32 == 0) && (((uintptr_t)p.Z) % 32 == 0) && (p.Z == nullptr || p.ldc % 32 == 0);
-        // EPI_DACT with staged stores: the saved sigma' box of the next chunk is fetched by TMA into box_z one
-        // chunk ahead (across tiles too), so its DRAM latency is hidden behind the MMAs and the previous chunk.
+        // EPI_DACT with staged stores: the warp's saved sigma' box (32 rows x its 64 columns) of the next tile is
+        // fetched by TMA into box_z one tile ahead, so its DRAM latency is hidden behind the MMAs and the stores.
+        static_assert(!TMA_EPI || CHUNKS == 2, "the sigma' box holds two 32-column chunks");
         const bool z_prefetch = TMA_EPI && p.epilogue == EPI_DACT;
         uint64_t* my_z_bar = &z_bar[warp - 2];
         uint32_t z_count = 0;
-        auto issue_z = [&](const Tile& tile, int c) {
+        auto issue_z = [&](const Tile& tile) {
             if (lane == 0) {
                 mbar_expect_tx(my_z_bar, kBoxBytesZ);
-                tma_load_2d(box_z, &map_z, my_z_bar, tile.n0 + part * COLS_PER_WARP + c * 32, tile.m0 + quad * 32);
+                tma_load_2d(box_z, &map_z, my_z_bar, tile.n0 + part * COLS_PER_WARP, tile.m0 + quad * 32);
             }
         };
-        if (z_prefetch && (int)blockIdx.x < total) issue_z(get_tile(p, BN, blockIdx.x, tiles_m, tiles_n), 0);
+        if (z_prefetch && (int)blockIdx.x < total) issue_z(get_tile(p, BN, blockIdx.x, tiles_m, tiles_n));
         uint32_t local = 0;
         for (int t = blockIdx.x; t < total; t += gridDim.x, ++local) {
             const Tile tl = get_tile(p, BN, t, tiles_m, tiles_n);
@@ -190,25 +191,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (lane == 0) tma_store_wait_read();        // previous boxes of this warp have left smem
                     __syncwarp();
                     if (z_prefetch) {
-                        mbar_wait(my_z_bar, z_count & 1, dead, p.status);
-                        ++z_count;
+                        if (c == 0) {
+                            mbar_wait(my_z_bar, z_count & 1, dead, p.status);
+                            ++z_count;
+                        }
                         uint32_t w[8];
-                        const uint8_t* zrow = box_z + lane * 32;
-                        ld_shared_16B(zrow, w);
-                        ld_shared_16B(zrow + 16, w + 4);
-                        fence_async_smem();
-                        __syncwarp();
-                        if (c + 1 < CHUNKS) issue_z(tl, c + 1);
-                        else if (t + (int)gridDim.x < total) issue_z(get_tile(p, BN, t + gridDim.x, tiles_m, tiles_n), 0);
+                        load_row_u8(box_z, lane, c, w);
+                        if (c == CHUNKS - 1) {             // box read by every lane: fetch the next tile's
+                            fence_async_smem();
+                            __syncwarp();
+                            if (t + (int)gridDim.x < total) issue_z(get_tile(p, BN, t + gridDim.x, tiles_m, tiles_n));
+                        }
                         mul_by_sig32(v, w);
                     }
-                    stage_row_chunk(p, v, box_c, box_z, lane, row_off, col0, row_ok);
+                    stage_row_chunk(p, v, box_c, box_z, lane, c);
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) {
                         const int row0 = tl.expert * p.c_rows_per_expert + tl.m0 + quad * 32;
                         tma_store_2d(&map_c, box_c, col0, row0);
-                        if (p.epilogue == EPI_ACT && p.Z) tma_store_2d(&map_z, box_z, col0, row0);
+                        if (p.epilogue == EPI_ACT && p.Z && c == CHUNKS - 1) tma_store_2d(&map_z, box_z, col0 - 32, row0);
                         tma_store_commit();
                     }
                 } else if (row_ok) {
@@ -295,7 +297,7 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
         const uint64_t c_rows = g.group == GROUP_K ? (uint64_t)g.M * E : (uint64_t)g.M;
         ok &= make_map(&mc, g.C, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
         if ((g.epilogue == EPI_ACT && g.Z) || g.epilogue == EPI_DACT)
-            ok &= make_map_u8(&mz, g.Z, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32);
+            ok &= make_map_u8(&mz, g.Z, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B);
     }
     if (!ok) return cudaErrorInvalidValue;
     p.tma_store = tma_store ? 1 : 0;

@@ -270,14 +270,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const bool z_prefetch = TMA_EPI && p.epilogue == EPI_DACT;
         uint64_t* my_z_bar = &z_bar[warp - 2];
         uint32_t z_count = 0;
-        auto issue_z = [&](const PairTile& tile, int c) {
+        static_assert(!TMA_EPI || CHUNKS == 2, "the sigma' box holds two 32-column chunks");
+        auto issue_z = [&](const PairTile& tile) {           // the warp's 32 rows x 64 columns of saved sigma'
             if (lane == 0) {
                 mbar_expect_tx(my_z_bar, kBoxBytesZ);
-                tma_load_2d(box_z, &map_z, my_z_bar, tile.n0 + part * COLS_PER_WARP + c * 32,
-                            tile.m0 + (int)rank * BM + quad * 32);
+                tma_load_2d(box_z, &map_z, my_z_bar, tile.n0 + part * COLS_PER_WARP, tile.m0 + (int)rank * BM + quad * 32);
             }
         };
-        if (z_prefetch && cluster_id < total) issue_z(get_pair_tile(p, BN, cluster_id, pairs_m, tiles_n, s_pp), 0);
+        if (z_prefetch && cluster_id < total) issue_z(get_pair_tile(p, BN, cluster_id, pairs_m, tiles_n, s_pp));
         uint32_t local = 0;
         for (int w = cluster_id; w < total; w += num_clusters, ++local) {
             const PairTile tl = get_pair_tile(p, BN, w, pairs_m, tiles_n, s_pp);
@@ -311,25 +311,26 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     if (lane == 0) tma_store_wait_read();
                     __syncwarp();
                     if (z_prefetch) {
-                        mbar_wait(my_z_bar, z_count & 1, dead, p.status);
-                        ++z_count;
+                        if (c == 0) {
+                            mbar_wait(my_z_bar, z_count & 1, dead, p.status);
+                            ++z_count;
+                        }
                         uint32_t wz[8];
-                        const uint8_t* zrow = box_z + lane * 32;
-                        ld_shared_16B(zrow, wz);
-                        ld_shared_16B(zrow + 16, wz + 4);
-                        fence_async_smem();
-                        __syncwarp();
-                        if (c + 1 < CHUNKS) issue_z(tl, c + 1);
-                        else if (w + num_clusters < total) issue_z(get_pair_tile(p, BN, w + num_clusters, pairs_m, tiles_n, s_pp), 0);
+                        load_row_u8(box_z, lane, c, wz);
+                        if (c == CHUNKS - 1) {             // box read by every lane: fetch the next tile's
+                            fence_async_smem();
+                            __syncwarp();
+                            if (w + num_clusters < total) issue_z(get_pair_tile(p, BN, w + num_clusters, pairs_m, tiles_n, s_pp));
+                        }
                         mul_by_sig32(v, wz);
                     }
-                    stage_row_chunk(p, v, box_c, box_z, lane, row_off, col0, row_ok);
+                    stage_row_chunk(p, v, box_c, box_z, lane, c);
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0 && half_ok && my_m0 < tl.m_limit) {
                         const int row0 = tl.expert * p.c_rows_per_expert + my_m0 + quad * 32;
                         tma_store_2d(&map_c, box_c, col0, row0);
-                        if (p.epilogue == EPI_ACT && p.Z) tma_store_2d(&map_z, box_z, col0, row0);
+                        if (p.epilogue == EPI_ACT && p.Z && c == CHUNKS - 1) tma_store_2d(&map_z, box_z, col0 - 32, row0);
                         tma_store_commit();
                     }
                 } else if (row_ok) {
@@ -398,7 +399,7 @@ cudaError_t dispatch_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
         const uint64_t c_rows = g.group == GROUP_K ? (uint64_t)g.M * E : (uint64_t)g.M;
         ok &= make_map(&mc, g.C, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
         if ((g.epilogue == EPI_ACT && g.Z) || g.epilogue == EPI_DACT)
-            ok &= make_map_u8(&mz, g.Z, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 32, 32);
+            ok &= make_map_u8(&mz, g.Z, (uint64_t)g.N, c_rows, (uint64_t)g.ldc, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B);
     }
     if (!ok) return cudaErrorInvalidValue;
     p.tma_store = TMA_EPI ? 1 : 0;

@@ -97,6 +97,8 @@ struct Dims {
     int64_t N, P;
     int E64;   // leading dimension of the dense [T,E] gate-gradient matrix (E rounded up to 64)
     int z_es;  // bytes per saved sigma'(z) element: 1 on the tensor-core path (quantised), else the dtype's
+    bool cdac; // Eq. 3 layer: no descend / ascend projections, r == d
+    int ldcat; // row stride of dcat: r + E64, or E64 alone without projections (dx' then goes straight to dx)
 };
 
 // The tensor-core kernels save sigma' as one byte per element; that needs expert GEMM1 and dz on the same side.
@@ -108,6 +110,8 @@ Dims dims_of(const bigmac_layer* L, int T) {
     m.P = padded_rows_max(m.N, c.E);
     m.E64 = (c.E + 63) / 64 * 64;
     m.z_es = sigma_as_bytes(L) ? 1 : (int)esize(c.dtype);
+    m.cdac = (c.flags & BIGMAC_FLAG_CDAC) != 0;
+    m.ldcat = m.cdac ? m.E64 : m.r + m.E64;
     return m;
 }
 
@@ -125,12 +129,12 @@ void carve_saved(Carver& cv, const Dims& m, Buffers& b, bool with_z) {
     b.tb.slot_of_prow = cv.take<int32_t>(m.P);
     b.tb.tile_expert = cv.take<int32_t>(m.P / kPad);
     b.tb.n_tiles = cv.take<int32_t>(1);
-    b.x_lo = cv.take_bytes((size_t)m.T * m.r * es);
+    b.x_lo = m.cdac ? nullptr : cv.take_bytes((size_t)m.T * m.r * es);     // without projections x' is x itself
     b.xg = cv.take_bytes((size_t)m.P * m.r * es);
     b.z = with_z ? cv.take_bytes((size_t)m.P * m.h * m.z_es) : nullptr;
     b.a = cv.take_bytes((size_t)m.P * m.h * es);
     b.u = cv.take_bytes((size_t)m.P * m.r * es);
-    b.y_lo = cv.take_bytes((size_t)m.T * m.r * es);
+    b.y_lo = m.cdac ? nullptr : cv.take_bytes((size_t)m.T * m.r * es);     // ... and y' is y
 }
 
 void carve_route_scratch(Carver& cv, const Dims& m, Buffers& b) {
@@ -140,16 +144,16 @@ void carve_route_scratch(Carver& cv, const Dims& m, Buffers& b) {
 
 void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
     const size_t es = esize(m.dtype);
-    b.dy_lo = cv.take_bytes((size_t)m.T * m.r * es);
+    b.dy_lo = m.cdac ? nullptr : cv.take_bytes((size_t)m.T * m.r * es);
     b.du = cv.take_bytes((size_t)m.P * m.r * es);
     b.dxg = cv.take_bytes((size_t)m.P * m.r * es);
     b.dz = m.z_es == 1 ? cv.take_bytes((size_t)m.P * m.h * es) : nullptr;
-    b.dcat = cv.take_bytes((size_t)m.T * (m.r + m.E64) * es);
-    b.dx_lo = b.dcat;
-    b.dlogits = b.dcat ? (char*)b.dcat + (size_t)m.r * es : nullptr;
+    b.dcat = cv.take_bytes((size_t)m.T * m.ldcat * es);
+    b.dx_lo = m.cdac ? nullptr : b.dcat;
+    b.dlogits = (b.dcat && !m.cdac) ? (char*)b.dcat + (size_t)m.r * es : b.dcat;
     b.dp = cv.take<float>(m.N);
     b.colsum_part = cv.take<float>((size_t)kColsumChunks * m.E);
-    b.splitk_ws = cv.take<float>((size_t)kMaxSplitK * (m.r + m.E64) * m.d);
+    b.splitk_ws = cv.take<float>((size_t)kMaxSplitK * m.ldcat * m.d);
 }
 
 size_t forward_scratch_bytes(const Dims& m, bool training) {
@@ -174,11 +178,12 @@ size_t saved_bytes_of(const Dims& m) {
 
 bool aligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
 
-int check_weights(const bigmac_weights_t* W) {
-    if (!W || !W->w_gate || !W->w_down || !W->w1 || !W->w2 || !W->w_up) return BIGMAC_ERR_INVALID_ARG;
-    if (!aligned(W->w_gate, 16) || !aligned(W->w_down, 16) || !aligned(W->w1, 16) || !aligned(W->w2, 16) ||
-        !aligned(W->w_up, 16) || !aligned(W->b_gate, 4))
+int check_weights(const bigmac_layer* L, const bigmac_weights_t* W) {
+    if (!W || !W->w_gate || !W->w1 || !W->w2) return BIGMAC_ERR_INVALID_ARG;
+    if (!aligned(W->w_gate, 16) || !aligned(W->w1, 16) || !aligned(W->w2, 16) || !aligned(W->b_gate, 4))
         return BIGMAC_ERR_INVALID_ARG;
+    if (L && (L->cfg.flags & BIGMAC_FLAG_CDAC)) return BIGMAC_OK;             // no shared projections
+    if (!W->w_down || !W->w_up || !aligned(W->w_down, 16) || !aligned(W->w_up, 16)) return BIGMAC_ERR_INVALID_ARG;
     return BIGMAC_OK;
 }
 
@@ -267,7 +272,8 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
     if (cfg->k > cfg->E) return BIGMAC_ERR_INVALID_ARG;
     if (cfg->dtype != BIGMAC_F32 && cfg->dtype != BIGMAC_BF16) return BIGMAC_ERR_INVALID_ARG;
     if (cfg->act < BIGMAC_ACT_RELU || cfg->act > BIGMAC_ACT_IDENTITY) return BIGMAC_ERR_INVALID_ARG;
-    if (cfg->flags & ~BIGMAC_FLAG_SIMT_GEMM) return BIGMAC_ERR_INVALID_ARG;
+    if (cfg->flags & ~(BIGMAC_FLAG_SIMT_GEMM | BIGMAC_FLAG_CDAC)) return BIGMAC_ERR_INVALID_ARG;
+    if ((cfg->flags & BIGMAC_FLAG_CDAC) && cfg->r != cfg->d) return BIGMAC_ERR_INVALID_ARG;
     if (cfg->E > kMaxExperts) return BIGMAC_ERR_UNSUPPORTED;
     if ((int64_t)cfg->max_tokens * cfg->k > (int64_t)1 << 30) return BIGMAC_ERR_UNSUPPORTED;
     const int vec = cfg->dtype == BIGMAC_BF16 ? 8 : 4;     // rows move as 16-byte vectors
@@ -319,7 +325,7 @@ int bigmac_route(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_weigh
                  void* scratch, size_t scratch_bytes, void* stream) {
     BIGMAC_TRY(check_call(L, T));
     if (!out) return BIGMAC_ERR_INVALID_ARG;
-    BIGMAC_TRY(check_weights(W));
+    BIGMAC_TRY(check_weights(L, W));
     if (T == 0) return BIGMAC_OK;
     if (!x || !aligned(x, 16) || !scratch || !aligned(scratch, 256)) return BIGMAC_ERR_INVALID_ARG;
     const Dims m = dims_of(L, T);
@@ -336,7 +342,7 @@ int bigmac_route(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_weigh
 int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_weights_t* W, void* y,
                    bigmac_routing_t* routing_out, void* saved, void* scratch, size_t scratch_bytes, void* stream) {
     BIGMAC_TRY(check_call(L, T));
-    BIGMAC_TRY(check_weights(W));
+    BIGMAC_TRY(check_weights(L, W));
     if (T == 0) return BIGMAC_OK;
     if (!x || !y || !aligned(x, 16) || !aligned(y, 16) || !scratch || !aligned(scratch, 256) ||
         !aligned(saved, 256))
@@ -357,7 +363,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     const bigmac_config_t& c = L->cfg;
 
     // A few tokens, inference: the whole forward in one cooperative kernel (weight streaming, no tensor cores)
-    if (!training && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
+    if (!training && !m.cdac && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
         {
             Stage s(L, S_DECODE, st);
             BIGMAC_CUDA(launch_decode_forward(x, W, y, b.logits, (float*)b.xg, (float*)b.a, (float*)b.u, b.tb.topk_idx,
@@ -372,7 +378,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     }
     // F1 + F4 in one pass over x when the tile grid allows it: [x' | logits] = x [W'_down ; W_gate]^T, logits in fp32
     const int bn_desc = (m.r + m.E) >= 256 ? 256 : 128;
-    const bool fuse_gate = c.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u && m.r % bn_desc == 0;
+    const bool fuse_gate = !m.cdac && c.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u && m.r % bn_desc == 0;
     if (fuse_gate) {
         GemmArgs g;
         g.A = x; g.lda = m.d; g.B = W->w_down; g.ldb = m.d; g.C = b.x_lo; g.ldc = m.r;
@@ -385,7 +391,8 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         BIGMAC_TRY(run_routing(L, m, x, W, b, st));                               // F1-F3
     }
     BIGMAC_TRY(export_routing(m, b, routing_out, st));
-    if (!fuse_gate) {                                                             // F4 descend: x' = x W'_down
+    if (m.cdac) b.x_lo = const_cast<void*>(x);                                    // Eq. 3: experts read the token itself
+    if (!fuse_gate && !m.cdac) {                                                  // F4 descend: x' = x W'_down
         GemmArgs g;
         g.A = x; g.lda = m.d; g.B = W->w_down; g.ldb = m.d; g.C = b.x_lo; g.ldc = m.r;
         g.M = m.T; g.N = m.r; g.K = m.d;
@@ -407,8 +414,9 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
         BIGMAC_TRY(gemm(L, G_EXPERT2, g, st));
     }
+    if (m.cdac) b.y_lo = y;                                                       // Eq. 3: the weighted sum is the output
     { Stage s(L, S_COMBINE, st); BIGMAC_CUDA(launch_combine(b.u, b.y_lo, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st)); }  // F8
-    {                                                                             // F9 ascend: y = y' W'_up
+    if (!m.cdac) {                                                                // F9 ascend: y = y' W'_up
         GemmArgs g;
         g.A = b.y_lo; g.lda = m.r; g.B = W->w_up; g.ldb = m.r; g.C = y; g.ldc = m.d;
         g.M = m.T; g.N = m.d; g.K = m.r;
@@ -421,7 +429,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
                     void* saved, void* dx, const bigmac_grads_t* G, int accumulate, void* scratch,
                     size_t scratch_bytes, void* stream) {
     BIGMAC_TRY(check_call(L, T));
-    BIGMAC_TRY(check_weights(W));
+    BIGMAC_TRY(check_weights(L, W));
     if (!G) return BIGMAC_ERR_INVALID_ARG;
     if (T == 0) return BIGMAC_OK;
     if (!x || !dy || !dx || !saved || !scratch || !aligned(x, 16) || !aligned(dy, 16) || !aligned(dx, 16) ||
@@ -443,15 +451,16 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     const bigmac_config_t& c = L->cfg;
     const bool acc = accumulate != 0;
 
-    {   // dy' = dy W_up                                   [T,d] x [d,r]
+    if (m.cdac) b.dy_lo = const_cast<void*>(dy);
+    if (!m.cdac) {   // dy' = dy W_up                                   [T,d] x [d,r]
         GemmArgs g;
         g.A = dy; g.lda = m.d; g.B = W->w_up; g.ldb = m.r; g.b_kmajor = false; g.C = b.dy_lo; g.ldc = m.r;
         g.M = m.T; g.N = m.r; g.K = m.d;
         BIGMAC_TRY(gemm(L, G_DY_LO, g, st));
     }
     const bool fused = L->cfg.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u;
-    const int ldcat = m.r + m.E64;
-    if (G->dw_up) {   // dW_up[c,c'] = sum_t dy[t,c] y'[t,c']
+    const int ldcat = m.ldcat;
+    if (G->dw_up && !m.cdac) {   // dW_up[c,c'] = sum_t dy[t,c] y'[t,c']
         GemmArgs g;
         g.A = dy; g.lda = m.d; g.a_kmajor = false; g.B = b.y_lo; g.ldb = m.r; g.b_kmajor = false;
         g.C = G->dw_up; g.ldc = m.r; g.M = m.d; g.N = m.r; g.K = m.T; g.accumulate = acc;
@@ -496,6 +505,32 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.C = G->dw1; g.ldc = m.r; g.c_stride = (int64_t)m.h * m.r; g.M = m.h; g.N = m.r; g.K = (int)m.P;
         g.group = GROUP_K; g.num_experts = m.E; g.poffsets = b.tb.poffsets; g.accumulate = acc;
         BIGMAC_TRY(gemm(L, G_DW1, g, st));
+    }
+    if (m.cdac) {
+        // Eq. 3: dx = sum_j dxg[row of slot (t,j)] + dl W_gate; dW_gate = dl^T x
+        { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, dx, nullptr, b.tb.prow_of_slot, m.T, m.k, m.d, m.dtype, st)); }
+        {
+            GemmArgs g;
+            g.A = b.dlogits; g.lda = ldcat; g.B = W->w_gate; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
+            g.M = m.T; g.N = m.d; g.K = m.E; g.accumulate = true;
+            BIGMAC_TRY(gemm(L, G_DX_GATE, g, st));
+        }
+        if (G->dw_gate) {
+            GemmArgs g;
+            g.A = b.dlogits; g.lda = ldcat; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
+            g.M = m.E; g.N = m.d; g.K = m.T;
+            if (fused) {
+                g.C = b.splitk_ws; g.ldc = m.d; g.out_f32 = true; g.M = ldcat; g.split_k = choose_split_k(g.M, g.N, g.K);
+                BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
+                Stage s(L, S_SPLITK_REDUCE, st);
+                BIGMAC_CUDA(launch_splitk_reduce(b.splitk_ws, g.split_k, ldcat, m.d, G->dw_gate, m.E, nullptr, 0, m.dtype, acc, st));
+            } else {
+                g.C = G->dw_gate; g.ldc = m.d; g.accumulate = acc;
+                BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
+            }
+        }
+        if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st)); }
+        return BIGMAC_OK;
     }
     // dx'[t] = sum_j dxg[row of slot (t,j)]   (the transpose of the dispatch gather)
     { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st, ldcat)); }
@@ -646,7 +681,7 @@ int bigmac_route_static(bigmac_layer_t* L, const void* x, int32_t T, const bigma
                         bigmac_routing_t* out, void* stream) {
     BIGMAC_TRY(check_call(L, T));
     if (!out) return BIGMAC_ERR_INVALID_ARG;
-    BIGMAC_TRY(check_weights(W));
+    BIGMAC_TRY(check_weights(L, W));
     if (T == 0) return BIGMAC_OK;
     if (!x || !aligned(x, 16)) return BIGMAC_ERR_INVALID_ARG;
     const Dims m = dims_of(L, T);

@@ -382,22 +382,31 @@ __device__ __forceinline__ void stage_row_bf16(uint8_t* box, int lane, const uin
     for (int j = 0; j < 4; ++j) st_shared_16B(row + ((j ^ sw) << 4), w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
 }
 
-// 32 rows x 32 sigma' bytes for a TMA store without swizzle: row `lane` occupies 32 bytes.
-__device__ __forceinline__ void stage_row_u8(uint8_t* box, int lane, const uint32_t* w /*8 words*/) {
-    uint8_t* row = box + lane * 32;
-    st_shared_16B(row, w[0], w[1], w[2], w[3]);
-    st_shared_16B(row + 16, w[4], w[5], w[6], w[7]);
+// The sigma' bytes of two consecutive 32-column chunks share one box of 32 rows x 64 bytes (64-byte swizzle, like
+// the bf16 box), so that every row segment a TMA copy moves to or from DRAM is 64 bytes: with 32-byte segments
+// the byte tensor ran at well under half the bandwidth of the bf16 one.  `half` = which 32 of the 64 columns.
+__device__ __forceinline__ void stage_row_u8(uint8_t* box, int lane, int half, const uint32_t* w /*8 words*/) {
+    uint8_t* row = box + lane * 64;
+    const int sw = (lane >> 1) & 3;
+    st_shared_16B(row + (((2 * half) ^ sw) << 4), w[0], w[1], w[2], w[3]);
+    st_shared_16B(row + (((2 * half + 1) ^ sw) << 4), w[4], w[5], w[6], w[7]);
+}
+__device__ __forceinline__ void load_row_u8(const uint8_t* box, int lane, int half, uint32_t* w /*8 words*/) {
+    const uint8_t* row = box + lane * 64;
+    const int sw = (lane >> 1) & 3;
+    ld_shared_16B(row + (((2 * half) ^ sw) << 4), w);
+    ld_shared_16B(row + (((2 * half + 1) ^ sw) << 4), w + 4);
 }
 
 // Epilogue of 32 columns through shared memory: v -> (sigma', sigma) or v * Z or v, packed to bf16 into the
 // warp's staging boxes.  Returns nothing; the caller fences and issues the TMA stores.
 __device__ __forceinline__ void stage_row_chunk(const TcParams& p, float* v, uint8_t* box_c, uint8_t* box_z, int lane,
-                                                int64_t row_off, int col0, bool row_ok) {
+                                                int zhalf) {
     uint32_t w[16];
     if (p.epilogue == EPI_ACT) {
         if (p.Z) {
             act_chunk_any<true>(p.act, v, w);
-            stage_row_u8(box_z, lane, w);
+            stage_row_u8(box_z, lane, zhalf, w);
         } else {
             act_chunk_any<false>(p.act, v, nullptr);
         }
@@ -451,7 +460,7 @@ __device__ __forceinline__ Tile get_tile(const TcParams& p, int BN, int t, int t
 
 constexpr int kEpiWarps = 16;
 constexpr uint32_t kBoxBytes = 32 * 64;                  // 32 rows x 32 bf16 columns
-constexpr uint32_t kBoxBytesZ = 32 * 32;                 // 32 rows x 32 sigma' bytes
+constexpr uint32_t kBoxBytesZ = 32 * 64;                 // 32 rows x 64 sigma' bytes (two chunks)
 constexpr int kThreadsV2 = (2 + kEpiWarps) * 32;
 
 
@@ -475,7 +484,7 @@ inline EncodeTiledFn encode_fn() {
 // 2-D bf16 tensor map: `inner` contiguous elements per row, `rows` rows `ld` elements apart.
 // 2-D byte tensor map (the saved sigma'): `inner` bytes per row, rows `ld` bytes apart, no swizzle.
 inline bool make_map_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner,
-                        uint32_t box_rows) {
+                        uint32_t box_rows, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {inner, rows};
@@ -483,7 +492,7 @@ inline bool make_map_u8(CUtensorMap* map, const void* base, uint64_t inner, uint
     const cuuint32_t box[2] = {box_inner, box_rows};
     const cuuint32_t elem[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -30,6 +30,7 @@ import numpy as np
 
 ACT_RELU, ACT_GELU_ERF, ACT_GELU_TANH, ACT_IDENTITY = 0, 1, 2, 3
 DTYPE_F32, DTYPE_BF16 = 0, 1
+FLAG_SIMT_GEMM, FLAG_CDAC = 1, 2
 
 
 @dataclass(frozen=True)
@@ -45,6 +46,7 @@ class Workload:
     act: int
     seed: int
     gate_bias: str = "none"   # "none" | "zipf"  (b_g[e] = ln q_e, q_e ~ (e+1)^-1.1)
+    cdac: bool = False        # the conventional fine-grained layer (Eq. 3): r == d, no w_down / w_up
 
     @property
     def N(self) -> int:
@@ -52,6 +54,13 @@ class Workload:
 
     def with_tokens(self, T: int, seed: Optional[int] = None) -> "Workload":
         return replace(self, T=T, seed=self.seed if seed is None else seed)
+
+    def cdac_twin(self) -> "Workload":
+        """The conventional fine-grained MoE layer with the same E, k, d and the same number of expert
+        parameters: experts d -> m -> d with m = r h / d (the paper's parameter-parity rule), tokens
+        dispatched at width d."""
+        assert not self.cdac and (self.r * self.h) % self.d == 0
+        return replace(self, name=self.name + "_cdac", r=self.d, h=self.r * self.h // self.d, cdac=True)
 
 
 # The five configurations the layer is built and measured on.
@@ -128,15 +137,16 @@ def make_inputs(w: Workload, with_dy: bool = True) -> Dict[str, Optional[np.ndar
 
     x, dy ~ N(0,1); weights ~ N(0, fan_in^-1/2), stored [out_features, in_features]:
     w_gate [E,d], w_down [r,d], w1 [E,h,r], w2 [E,r,h], w_up [d,r].  b_gate is fp32 [E] or None.
+    The projection-free layer (cdac) has r == d and no w_down / w_up (None).
     """
     s, dt = w.seed, w.dtype
     out: Dict[str, Optional[np.ndarray]] = {
         "x": _normal(s, _TAGS["x"], 0, (w.T, w.d), 1.0, dt),
         "w_gate": _normal(s, _TAGS["w_gate"], 0, (w.E, w.d), w.d ** -0.5, dt),
-        "w_down": _normal(s, _TAGS["w_down"], 0, (w.r, w.d), w.d ** -0.5, dt),
+        "w_down": None if w.cdac else _normal(s, _TAGS["w_down"], 0, (w.r, w.d), w.d ** -0.5, dt),
         "w1": _normal(s, _TAGS["w1"], 0, (w.E, w.h, w.r), w.r ** -0.5, dt),
         "w2": _normal(s, _TAGS["w2"], 0, (w.E, w.r, w.h), w.h ** -0.5, dt),
-        "w_up": _normal(s, _TAGS["w_up"], 0, (w.d, w.r), w.r ** -0.5, dt),
+        "w_up": None if w.cdac else _normal(s, _TAGS["w_up"], 0, (w.d, w.r), w.r ** -0.5, dt),
         "b_gate": zipf_log_popularity(w.E) if w.gate_bias == "zipf" else None,
         "dy": _normal(s, _TAGS["dy"], 0, (w.T, w.d), 1.0, dt) if with_dy else None,
     }

@@ -56,7 +56,20 @@ def to_numpy(t):
 def make_layer(w, flags=0, max_tokens=None):
     from paper_2502_16927_b200 import binding
 
+    if w.cdac:
+        flags |= wl.FLAG_CDAC
     return binding.Layer(w.d, w.r, w.h, w.E, w.k, max_tokens or max(w.T, 1), w.dtype, w.act, flags)
+
+
+def oracle_inputs(w, inp):
+    """What the oracle is given for this workload.  The projection-free layer (Eq. 3) is Eq. 2 with identity
+    projections, which is how the oracle evaluates it."""
+    if not w.cdac:
+        return inp
+    out = dict(inp)
+    out["w_down"] = np.eye(w.d, dtype=np.float32)
+    out["w_up"] = np.eye(w.d, dtype=np.float32)
+    return out
 
 
 def empty_grads(w, dev, fill=None):
@@ -65,6 +78,8 @@ def empty_grads(w, dev, fill=None):
     dt = torch.float32 if w.dtype == wl.DTYPE_F32 else torch.bfloat16
     shapes = {"dw_gate": (w.E, w.d), "dw_down": (w.r, w.d), "dw1": (w.E, w.h, w.r), "dw2": (w.E, w.r, w.h),
               "dw_up": (w.d, w.r)}
+    if w.cdac:
+        del shapes["dw_down"], shapes["dw_up"]
     G = {}
     for key, shp in shapes.items():
         G[key] = torch.empty(shp, dtype=dt, device="cuda") if fill is None else torch.full(shp, fill, dtype=dt, device="cuda")

@@ -14,7 +14,7 @@ import oracle
 from oracle import margin
 from paper_2502_16927_b200 import workloads as wl
 
-from helpers import empty_grads, make_layer, to_device, to_numpy
+from helpers import oracle_inputs, empty_grads, make_layer, to_device, to_numpy
 
 pytestmark = pytest.mark.gpu
 
@@ -87,15 +87,18 @@ RELU_DECISION_KEYS = ("dx", "dw1", "dw2", "dw_down", "dw_gate", "db_gate")
 
 
 def compare_full(w, inp, got, tol=None):
+    inp = oracle_inputs(w, inp)
     rt = oracle.route(inp, w.k)
     check_routing(got["routing"], rt)
     ref = oracle.backward_full(inp, rt, w.act, decide_bf16=w.dtype == wl.DTYPE_BF16)
     ref["dw1"] = np.stack([ref["dw1"][e] for e in range(w.E)])
     ref["dw2"] = np.stack([ref["dw2"][e] for e in range(w.E)])
-    keys = ("y", "dx", "dw_up", "dw_down", "dw_gate", "dw1", "dw2", "db_gate")
+    keys = ("y", "dx", "dw_gate", "dw1", "dw2", "db_gate") + (() if w.cdac else ("dw_up", "dw_down"))
     errs = float_errors(w, {key: got[key] for key in keys}, ref)
     if w.dtype == wl.DTYPE_BF16 and w.act == wl.ACT_RELU:
         for key in RELU_DECISION_KEYS:
+            if key not in keys:
+                continue
             assert outlier_fraction(got[key], ref[key], TOL[w.dtype]) <= 1e-3, key
             errs.pop(key)
     assert_within(w, errs)
@@ -193,6 +196,32 @@ def test_bf16_skewed_routing(case):
             ref = got[key] + 0.5
             assert np.max(np.abs(to_numpy(G1[key]) - ref)) <= 2.0 ** -7 * np.max(np.abs(ref)), key
         layer.close()
+
+
+@pytest.mark.parametrize("case", [
+    dict(dtype=wl.DTYPE_F32, act=wl.ACT_GELU_ERF, T=77, d=36, h=20, E=5, k=2),
+    dict(dtype=wl.DTYPE_F32, act=wl.ACT_RELU, T=300, d=64, h=8, E=7, k=3),
+    dict(dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, T=1000, d=256, h=64, E=16, k=4),     # narrow experts: one-CTA kernels
+    dict(dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, T=2048, d=1024, h=256, E=8, k=2),    # CTA pairs, staged stores
+    dict(dtype=wl.DTYPE_BF16, act=wl.ACT_RELU, T=130, d=320, h=128, E=40, k=2),
+])
+def test_projection_free_layer_of_eq3(case):
+    """BIGMAC_FLAG_CDAC: y = sum_i p_i(x) E_i(x) with d -> h -> d experts, dispatched at width d, forward and
+    backward, against the oracle (which evaluates it as Eq. 2 with identity projections)."""
+    case = dict(case)
+    d = case.pop("d")
+    w = wl.Workload("cdac", d=d, r=d, seed=577, cdac=True, **case)
+    inp = conditioned(w)
+    assert inp["w_down"] is None and inp["w_up"] is None
+    compare_full(w, inp, run_full(w, inp))
+
+
+def test_small_cdac_twin_full_config():
+    """The parameter-parity twin of configs[1] (d=1024, E=32, k=4, experts 1024 -> 64 -> 1024) at T=2048."""
+    w = wl.WORKLOADS["small"].cdac_twin().with_tokens(2048)
+    assert (w.r, w.h, w.cdac) == (1024, 64, True)
+    inp = conditioned(w)
+    compare_full(w, inp, run_full(w, inp))
 
 
 def test_route_matches_forward_tables_and_zero_tokens_is_a_noop():

@@ -133,6 +133,31 @@ def test_single_expert_is_a_four_matmul_mlp(act):
     np.testing.assert_allclose(oracle.forward_grouped(inp, rt, act)["y"], _mlp(inp, 0, act), rtol=0, atol=1e-12)
 
 
+def test_identity_projections_give_the_conventional_layer_of_eq3():
+    """Eq. 3 (y = sum_{i in T} p_i(x) E_i(x), experts d -> m -> d) written out token by token with numpy, against
+    the oracle's Eq. 2 evaluated with W_down = W_up = I: the projection-free layer is that special case, and its
+    dx is the sum of the expert path and the gate path."""
+    T, d, m, E, k = 19, 8, 5, 6, 3
+    w = wl.Workload("cdac", T=T, d=d, r=d, h=m, E=E, k=k, dtype=wl.DTYPE_F32, act=wl.ACT_GELU_ERF, seed=41, cdac=True)
+    inp = wl.make_inputs(w)
+    assert inp["w_down"] is None and inp["w_up"] is None and inp["w1"].shape == (E, m, d) and inp["w2"].shape == (E, d, m)
+    x, wg, w1, w2 = (_f64(inp[key]) for key in ("x", "w_gate", "w1", "w2"))
+    y = np.zeros((T, d))
+    for t in range(T):
+        logits = wg @ x[t]
+        chosen = sorted(range(E), key=lambda e: (-logits[e], e))[:k]
+        p = softmax(logits[chosen])
+        for p_i, e in zip(p, chosen):
+            y[t] += p_i * (w2[e] @ _act(w.act, w1[e] @ x[t]))
+    full = dict(inp, w_down=np.eye(d, dtype=np.float32), w_up=np.eye(d, dtype=np.float32))
+    rt = oracle.route(full, k)
+    np.testing.assert_allclose(oracle.forward_tokens(full, rt, w.act)["y"], y, rtol=0, atol=1e-12)
+    # parameter parity of the twin: experts of d -> r -> h -> r -> d and d -> m -> d hold the same number of weights
+    big = wl.WORKLOADS["large"]
+    twin = big.cdac_twin()
+    assert (twin.r, twin.h) == (4096, 256) and 2 * twin.r * twin.h == 2 * big.r * big.h
+
+
 def test_identical_experts_make_the_output_independent_of_routing():
     w, inp = small_workload(T=31, E=5, k=3, act=wl.ACT_GELU_ERF)
     inp["w1"] = np.tile(inp["w1"][:1], (5, 1, 1))
