@@ -11,67 +11,13 @@
 // CTAs.  Accumulators are double-buffered: "tmem_full" is signalled in both CTAs by a multicast commit, and the
 // epilogue warps of both CTAs arrive on the leader's "tmem_empty" when they have read their half.
 // No TMA multicast is used.  Everything else (epilogues, grouping, split contraction) is as in gemm_tc.cu.
-#include "tc_common.cuh"
+#include "tc_pair.cuh"
 
 namespace bigmac {
 
 using namespace tc;
 
 namespace {
-
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(const void* local, uint32_t rank) {
-    uint32_t out;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(smem_u32(local)), "r"(rank));
-    return out;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// TMA load into this CTA's shared memory that completes on a barrier of the pair's leader CTA.
-__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, uint32_t leader_bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(leader_bar)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t* dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// Arrive (when all MMAs issued so far have completed) on the barrier at this offset in both CTAs of the pair.
-__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(smem_u32(bar)), "h"((uint16_t)3)
-        : "memory");
-}
-
-// Instruction descriptor for the pair MMA: M = 256 (128 rows per CTA), N = bn.
-__host__ __device__ constexpr uint32_t instr_desc_pair(int bn, bool a_mn_major, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
-           ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-}
 
 // Work item of one CTA pair: rows m0.. (CTA 0) and m0+128.. (CTA 1) of problem `expert`.
 struct PairTile {
@@ -154,11 +100,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int tiles_n = (p.N + BN - 1) / BN;
     int pairs_m = (p.M + 2 * BM - 1) / (2 * BM);
     if (p.group == GROUP_M) {
+        // the padded offsets come to shared memory in one round trip, then turn into the pair prefix in place
+        for (int e = threadIdx.x; e <= p.num_experts; e += blockDim.x) s_pp[e] = p.poffsets[e];
+        __syncthreads();
         if (threadIdx.x == 0) {
-            int run = 0;
+            int run = 0, lo = s_pp[0];
             for (int e = 0; e < p.num_experts; ++e) {
+                const int hi = s_pp[e + 1];
                 s_pp[e] = run;
-                run += ((p.poffsets[e + 1] - p.poffsets[e]) / kPad + 1) / 2;
+                run += ((hi - lo) / kPad + 1) / 2;
+                lo = hi;
             }
             s_pp[p.num_experts] = run;
         }

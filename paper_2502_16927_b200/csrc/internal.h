@@ -65,6 +65,14 @@ cudaError_t gemm_simt(const GemmArgs& g, int dtype, cudaStream_t stream);
 // tcgen05 / TMEM / TMA GEMM, bf16 inputs, fp32 accumulation.  `status` is the device status word.
 cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream);
 bool gemm_tc_available();
+// Per-expert weight-gradient contraction (GROUP_K, both operands MN-major, bf16 output) with dynamically scheduled
+// work items and long experts cut into parts (gemm_tc_groupk.cu).  ws: gemm_tc_groupk_ws_bytes() bytes, 256-byte
+// aligned; sched: two device ints that are zero between launches (the kernel leaves them so).
+constexpr int kGroupKSlots = 32;
+bool gemm_tc_groupk_supported(const GemmArgs& g);
+size_t gemm_tc_groupk_ws_bytes(int M, int N, int E);
+cudaError_t gemm_tc_groupk(const GemmArgs& g, int* status, int* sched, void* ws, cudaStream_t stream);
+cudaError_t gemm_tc_groupk_finish(const GemmArgs& g, void* ws, cudaStream_t stream);   // always after gemm_tc_groupk
 // CTA-pair variant (tcgen05 cta_group::2) for outputs at least 256 wide.
 bool gemm_tc_pair_supported(const GemmArgs& g);
 bool gemm_tc_pair_preferred(const GemmArgs& g);

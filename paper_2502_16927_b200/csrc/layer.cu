@@ -16,7 +16,8 @@ using namespace bigmac;
 struct bigmac_layer {
     bigmac_config_t cfg;
     int device;
-    int* status;        // device status word; status[1] is the grid-barrier counter of the small-batch kernel
+    int* status;        // device status word; status[1] is the grid-barrier counter of the small-batch kernel,
+                        // status[2..3] the work counters of the per-expert weight-gradient kernel (zero at rest)
     bool use_tc;        // bf16 contractions on tcgen05
     unsigned tc_mask;   // debug: bit i set = contraction i runs on tcgen05 (BIGMAC_TC_MASK)
     // measurement aid
@@ -153,7 +154,10 @@ void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
     b.dlogits = (b.dcat && !m.cdac) ? (char*)b.dcat + (size_t)m.r * es : b.dcat;
     b.dp = cv.take<float>(m.N);
     b.colsum_part = cv.take<float>((size_t)kColsumChunks * m.E);
-    b.splitk_ws = cv.take<float>((size_t)kMaxSplitK * m.ldcat * m.d);
+    // fp32 partial results: of the split dense contractions, and of the parts of long experts in dW1 / dW2
+    const size_t dense_ws = (size_t)kMaxSplitK * m.ldcat * m.d * sizeof(float);
+    const size_t expert_ws = m.dtype == BIGMAC_BF16 ? gemm_tc_groupk_ws_bytes(m.r, m.h, m.E) : 0;
+    b.splitk_ws = (float*)cv.take_bytes(dense_ws > expert_ws ? dense_ws : expert_ws);
 }
 
 size_t forward_scratch_bytes(const Dims& m, bool training) {
@@ -260,6 +264,19 @@ int check_call(const bigmac_layer* L, int32_t T) {
     return BIGMAC_OK;
 }
 
+// Per-expert weight gradient (contraction over the expert's rows): on the tensor-core path the balanced kernel
+// (dynamic work items, long experts in parts), else the generic grouped contraction.
+int expert_weight_grad(const bigmac_layer* L, int id, const GemmArgs& g, const Buffers& b, cudaStream_t st) {
+    static const bool enabled = []() { const char* e = std::getenv("BIGMAC_GROUPK"); return !(e && e[0] == '0'); }();
+    const bool tc = L->cfg.dtype == BIGMAC_BF16 && L->use_tc && ((L->tc_mask >> id) & 1u);
+    if (enabled && tc && gemm_tc_groupk_supported(g)) {
+        { Stage stage(L, id, st); BIGMAC_CUDA(gemm_tc_groupk(g, L->status, L->status + 2, b.splitk_ws, st)); }
+        { Stage stage(L, S_SPLITK_REDUCE, st); BIGMAC_CUDA(gemm_tc_groupk_finish(g, b.splitk_ws, st)); }
+        return BIGMAC_OK;
+    }
+    return gemm(L, id, g, st);
+}
+
 }  // namespace
 
 extern "C" {
@@ -285,8 +302,8 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
     L->use_tc = cfg->dtype == BIGMAC_BF16 && !(cfg->flags & BIGMAC_FLAG_SIMT_GEMM);
     L->tc_mask = ~0u;
     if (const char* env = std::getenv("BIGMAC_TC_MASK")) L->tc_mask = (unsigned)std::strtoul(env, nullptr, 0);
-    if (cudaGetDevice(&L->device) != cudaSuccess || cudaMalloc((void**)&L->status, 2 * sizeof(int)) != cudaSuccess ||
-        cudaMemset(L->status, 0, 2 * sizeof(int)) != cudaSuccess) {
+    if (cudaGetDevice(&L->device) != cudaSuccess || cudaMalloc((void**)&L->status, 4 * sizeof(int)) != cudaSuccess ||
+        cudaMemset(L->status, 0, 4 * sizeof(int)) != cudaSuccess) {
         delete L;
         return BIGMAC_ERR_CUDA;
     }
@@ -490,7 +507,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.A = b.du; g.lda = m.r; g.a_kmajor = false; g.B = b.a; g.ldb = m.h; g.b_kmajor = false;
         g.C = G->dw2; g.ldc = m.h; g.c_stride = (int64_t)m.r * m.h; g.M = m.r; g.N = m.h; g.K = (int)m.P;
         g.group = GROUP_K; g.num_experts = m.E; g.poffsets = b.tb.poffsets; g.accumulate = acc;
-        BIGMAC_TRY(gemm(L, G_DW2, g, st));
+        BIGMAC_TRY(expert_weight_grad(L, G_DW2, g, b, st));
     }
     {   // dxg = dz W1_e
         GemmArgs g;
@@ -504,7 +521,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.A = dz; g.lda = m.h; g.a_kmajor = false; g.B = b.xg; g.ldb = m.r; g.b_kmajor = false;
         g.C = G->dw1; g.ldc = m.r; g.c_stride = (int64_t)m.h * m.r; g.M = m.h; g.N = m.r; g.K = (int)m.P;
         g.group = GROUP_K; g.num_experts = m.E; g.poffsets = b.tb.poffsets; g.accumulate = acc;
-        BIGMAC_TRY(gemm(L, G_DW1, g, st));
+        BIGMAC_TRY(expert_weight_grad(L, G_DW1, g, b, st));
     }
     if (m.cdac) {
         // Eq. 3: dx = sum_j dxg[row of slot (t,j)] + dl W_gate; dW_gate = dl^T x
