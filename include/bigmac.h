@@ -78,6 +78,10 @@ typedef enum {
  * entry points: the like-for-like single-GPU counterpart of the BigMac layer (parameter parity: h = r'h'/d for a
  * BigMac layer with low width r' and expert hidden width h'). */
 #define BIGMAC_FLAG_CDAC 2u
+/* BF16 tensor-core path: run the per-expert weight gradients on the dynamically scheduled kernel (work items handed
+ * out at run time, long experts contracted in parts) whatever the problem size.  Without the flag that kernel is
+ * used when there is enough work per SM pair for it to pay, else the statically scheduled one. */
+#define BIGMAC_FLAG_DYNAMIC_WGRAD 4u
 
 typedef struct {
     int32_t d, r, h, E, k; /* 1 <= k <= E */

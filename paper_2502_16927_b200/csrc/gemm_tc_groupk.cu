@@ -39,38 +39,42 @@ struct Item {
 // experts (their workspace slots).  With `per` output tiles per expert on `pairs` CTA pairs the balanced share
 // is total_kb * per / pairs k slices; parts are at most a quarter of it (at least 8 slices) long, and the
 // length grows until the split experts' parts fit the kGroupKSlots workspace slots.
-// `ss` may alias `poffsets` (entry e is written after entries e and e + 1 have been read).
+// Called by all lanes of one warp (32-bit arithmetic throughout: the plan sits in front of the first load).
 __device__ void groupk_plan(const int32_t* poffsets, int E, int per, int pairs, int32_t* pp, int32_t* ss) {
-    const long long total_kb = poffsets[E] / BK;
-    long long len = total_kb * per / (4LL * pairs);
+    const int lane = threadIdx.x & 31;
+    const int total_kb = poffsets[E] / BK;
+    int len = (int)(((long long)total_kb * per) / (4 * pairs));
     if (len < 8) len = 8;
     for (int iter = 0; iter < 40; ++iter) {
-        long long slots = 0;
-        for (int e = 0; e < E; ++e) {
-            const long long kb = (poffsets[e + 1] - poffsets[e]) / BK;
+        int slots = 0;
+        for (int e = lane; e < E; e += 32) {
+            const int kb = (poffsets[e + 1] - poffsets[e]) / BK;
             if (kb > len) slots += (kb + len - 1) / len;
         }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) slots += __shfl_xor_sync(0xffffffffu, slots, off);
         if (slots <= kGroupKSlots) break;
         len += len / 2;
     }
-    int run = 0, slot = 0;
-    int lo = poffsets[0];
-    for (int e = 0; e < E; ++e) {
-        const int hi = poffsets[e + 1];
-        const long long kb = (hi - lo) / BK;
-        lo = hi;
-        int parts = kb == 0 ? 0 : 1;
-        if (kb > len) {
-            const int want = (int)((kb + len - 1) / len);
-            if (slot + want <= kGroupKSlots) parts = want;
+    if (lane == 0) {
+        int run = 0, slot = 0, lo = poffsets[0];
+        for (int e = 0; e < E; ++e) {
+            const int hi = poffsets[e + 1];
+            const int kb = (hi - lo) / BK;
+            lo = hi;
+            int parts = kb == 0 ? 0 : 1;
+            if (kb > len) {
+                const int want = (kb + len - 1) / len;
+                if (slot + want <= kGroupKSlots) parts = want;
+            }
+            pp[e] = run;
+            ss[e] = slot;
+            run += parts;
+            if (parts > 1) slot += parts;
         }
-        pp[e] = run;
-        ss[e] = slot;
-        run += parts;
-        if (parts > 1) slot += parts;
+        pp[E] = run;
+        ss[E] = slot;
     }
-    pp[E] = run;
-    ss[E] = slot;
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsV2, 1)
@@ -96,6 +100,7 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     volatile int* dead = (volatile int*)(tmem_slot + 1);
     int32_t* s_pp = (int32_t*)(tmem_slot + 4);               // [E + 1] parts before expert e
     int32_t* s_ss = s_pp + p.num_experts + 1;                // [E + 1] workspace slots before expert e
+    int32_t* s_off = s_ss + p.num_experts + 1;               // [E + 1] padded row offsets (a copy: the scheduler reads them per item)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -104,13 +109,11 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     const int tiles_n = (p.N + BN - 1) / BN, pairs_m = (p.M + 2 * BM - 1) / (2 * BM);
     const int per = pairs_m * tiles_n;
 
-    // the offsets come to shared memory in one round trip (s_ss as staging); the plan is then computed from there
-    for (int e = threadIdx.x; e <= p.num_experts; e += blockDim.x) s_ss[e] = p.poffsets[e];
+    // the offsets come to shared memory in one round trip; the plan is computed from there
+    for (int e = threadIdx.x; e <= p.num_experts; e += blockDim.x) s_off[e] = p.poffsets[e];
     __syncthreads();
+    if (warp == 0) groupk_plan(s_off, p.num_experts, per, num_clusters, s_pp, s_ss);
     if (threadIdx.x == 0) {
-        groupk_plan(s_ss, p.num_experts, per, num_clusters, s_pp, s_ss);
-        if (blockIdx.x == 0)
-            for (int e = 0; e <= p.num_experts; ++e) { plan_out[e] = s_pp[e]; plan_out[p.num_experts + 1 + e] = s_ss[e]; }
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], 2 * kEpiWarps); }
         for (int s = 0; s < kRing; ++s) mbar_init(&ring_bar[s], 1);
@@ -125,6 +128,8 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const int total = s_pp[p.num_experts] * per;
+    if (blockIdx.x == 0)     // the plan, for the finishing kernel
+        for (int e = threadIdx.x; e <= p.num_experts; e += blockDim.x) { plan_out[e] = s_pp[e]; plan_out[p.num_experts + 1 + e] = s_ss[e]; }
 
     auto load_stage = [&](const Item& t, int kb, uint32_t it) {
         const int s = it % STAGES;
@@ -159,8 +164,8 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                             if (s_pp[mid] <= pi) lo = mid; else hi = mid;
                         }
                         const int part = pi - s_pp[lo], parts = s_pp[lo + 1] - s_pp[lo];
-                        const int row0 = p.poffsets[lo], kb_e = (p.poffsets[lo + 1] - row0) / BK;
-                        const int kb0 = (int)((long long)part * kb_e / parts), kb1 = (int)((long long)(part + 1) * kb_e / parts);
+                        const int row0 = s_off[lo], kb_e = (s_off[lo + 1] - row0) / BK;
+                        const int kb0 = parts > 1 ? part * kb_e / parts : 0, kb1 = parts > 1 ? (part + 1) * kb_e / parts : kb_e;   // kb_e < 2^24, parts <= 32
                         t.expert = lo;
                         t.m0 = (r / tiles_n) * 2 * BM;
                         t.n0 = (r % tiles_n) * BN;
@@ -344,7 +349,7 @@ cudaError_t gemm_tc_groupk(const GemmArgs& g, int* status, int* sched, void* ws,
     int32_t* plan = (int32_t*)((char*)ws + (((size_t)kGroupKSlots * g.M * g.N * sizeof(float) + 255) & ~(size_t)255));
     constexpr size_t kMaxSmem = 232448;
     const size_t smem = STAGES * (BM * BK * 2 + (BN / 2) * BK * 2) + (2 * STAGES + 4 + kRing) * 8 + kRing * sizeof(Item) + 16 +
-                        2 * (size_t)(E + 1) * 4 + 1024;
+                        3 * (size_t)(E + 1) * 4 + 1024;
     if (smem > kMaxSmem) return cudaErrorInvalidConfiguration;
     static PerDeviceOnce once;
     int dev;

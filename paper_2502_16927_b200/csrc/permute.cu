@@ -194,13 +194,16 @@ __global__ void __launch_bounds__(256) colsum_slots_kernel(const float* __restri
     }
 }
 
+// One warp per column: lane l adds chunks l, l + 32, ... in order, then a fixed shuffle tree adds the lanes.
 __global__ void __launch_bounds__(256) colsum_final_kernel(const float* __restrict__ partial, float* __restrict__ out, int chunks,
                                                            int cols, int accumulate) {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (c >= cols) return;
     float total = 0.0f;
-    for (int i = 0; i < chunks; ++i) total += partial[(int64_t)i * cols + c];
-    out[c] = accumulate ? out[c] + total : total;
+    for (int i = lane; i < chunks; i += 32) total += partial[(int64_t)i * cols + c];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
+    if (lane == 0) out[c] = accumulate ? out[c] + total : total;
 }
 
 template <typename T>
@@ -278,7 +281,7 @@ cudaError_t launch_gate_bwd(float* dp, const Tables& tb, void* dlogits, int T, i
 cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db, float* partial, int64_t N, int E,
                                bool accumulate, cudaStream_t stream) {
     colsum_slots_kernel<<<kColsumChunks, 256, sizeof(float) * 8 * E, stream>>>(dl_slot, tb.topk_idx, partial, N, E);
-    colsum_final_kernel<<<(unsigned)((E + 255) / 256), 256, 0, stream>>>(partial, db, kColsumChunks, E, accumulate);
+    colsum_final_kernel<<<(unsigned)((E + 7) / 8), 256, 0, stream>>>(partial, db, kColsumChunks, E, accumulate);
     return cudaGetLastError();
 }
 

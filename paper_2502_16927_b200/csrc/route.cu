@@ -11,7 +11,9 @@ constexpr unsigned kFull = 0xffffffffu;
 
 // One warp per token.  Lane l holds experts l, l+32, ...  k rounds of warp arg-max under the order
 // (logit descending, expert id ascending); gate values are the softmax over the k winners.
-template <int VPL>
+// KREG: k <= 32, the j-th winner stays in a register of lane j until one coalesced store at the end; otherwise
+// the winners pass through the output arrays.
+template <int VPL, bool KREG>
 __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ logits, const float* __restrict__ b_gate,
                                                    int T, int E, int k, int32_t* __restrict__ topk_idx,
                                                    float* __restrict__ topk_w) {
@@ -27,6 +29,8 @@ __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ log
     }
     int32_t* out_idx = topk_idx + (size_t)t * k;
     float* out_w = topk_w + (size_t)t * k;
+    float my_v = -INFINITY;
+    int my_e = 0;
     for (int j = 0; j < k; ++j) {
         float best = -INFINITY;
         int best_e = 0x7fffffff;
@@ -46,7 +50,24 @@ __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ log
             for (int i = 0; i < VPL; ++i)
                 if (lane + 32 * i == best_e) v[i] = -INFINITY;
         }
-        if (lane == 0) { out_idx[j] = best_e; out_w[j] = best; }   // raw logit for now
+        if (KREG) {
+            if (lane == j) { my_v = best; my_e = best_e; }
+        } else if (lane == 0) {
+            out_idx[j] = best_e;
+            out_w[j] = best;                       // raw logit for now
+        }
+    }
+    if (KREG) {
+        const float top = __shfl_sync(kFull, my_v, 0);
+        const float ex = lane < k ? expf(my_v - top) : 0.0f;
+        float part = ex;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
+        if (lane < k) {
+            out_idx[lane] = my_e;
+            out_w[lane] = ex / part;
+        }
+        return;
     }
     __syncwarp();
     const float top = out_w[0];
@@ -177,7 +198,11 @@ cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, 
     const int warps = 8;
     dim3 grid((T + warps - 1) / warps), block(warps * 32);
     const int vpl = (E + 31) / 32;
-#define BIGMAC_TOPK(V) topk_kernel<V><<<grid, block, 0, stream>>>(logits, b_gate, T, E, k, topk_idx, topk_w)
+#define BIGMAC_TOPK(V)                                                                                   \
+    do {                                                                                                 \
+        if (k <= 32) topk_kernel<V, true><<<grid, block, 0, stream>>>(logits, b_gate, T, E, k, topk_idx, topk_w);  \
+        else topk_kernel<V, false><<<grid, block, 0, stream>>>(logits, b_gate, T, E, k, topk_idx, topk_w);          \
+    } while (0)
     if (vpl <= 1) BIGMAC_TOPK(1);
     else if (vpl <= 2) BIGMAC_TOPK(2);
     else if (vpl <= 4) BIGMAC_TOPK(4);

@@ -30,7 +30,7 @@ import numpy as np
 
 ACT_RELU, ACT_GELU_ERF, ACT_GELU_TANH, ACT_IDENTITY = 0, 1, 2, 3
 DTYPE_F32, DTYPE_BF16 = 0, 1
-FLAG_SIMT_GEMM, FLAG_CDAC = 1, 2
+FLAG_SIMT_GEMM, FLAG_CDAC, FLAG_DYNAMIC_WGRAD = 1, 2, 4
 
 
 @dataclass(frozen=True)

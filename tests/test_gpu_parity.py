@@ -120,6 +120,7 @@ def test_tiny_fp32_forward_backward():
     dict(T=130, d=16, r=8, h=8, E=1, k=1),      # one expert, more than one row tile
     dict(T=5, d=8, r=4, h=4, E=16, k=1),        # fewer slots than experts
     dict(T=300, d=36, r=20, h=44, E=7, k=2),    # nothing a multiple of a tile
+    dict(T=33, d=16, r=8, h=8, E=48, k=40),     # more than 32 experts per token
 ])
 @pytest.mark.parametrize("act", [wl.ACT_RELU, wl.ACT_GELU_ERF, wl.ACT_GELU_TANH])
 def test_fp32_edge_shapes(shape, act):
@@ -168,9 +169,12 @@ def test_bf16_edge_shapes(shape, act):
     # balanced, many row tiles per expert
     dict(shape=dict(T=20000, d=256, r=256, h=256, E=24, k=2), bias=None),
 ])
-def test_bf16_skewed_routing(case):
+@pytest.mark.parametrize("flags", [0, wl.FLAG_DYNAMIC_WGRAD])
+def test_bf16_skewed_routing(case, flags):
     """Expert-load skew (dropless routing keeps every slot, so one expert may hold most rows and others none):
-    results must match the oracle as for balanced routing, also when accumulating into existing gradients."""
+    results must match the oracle as for balanced routing, also when accumulating into existing gradients; with
+    the statically scheduled weight-gradient kernel (the default at these sizes) and the dynamically scheduled one
+    that cuts long experts into parts."""
     import torch
 
     w = wl.Workload("skew", dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=311, **case["shape"])
@@ -182,12 +186,12 @@ def test_bf16_skewed_routing(case):
     elif case["bias"] == "graded":
         inp["b_gate"] = (2.5 * np.linspace(1.0, -1.0, w.E) ** 3).astype(np.float32)
     margin.enforce_margin(w, inp, 1e-3)
-    got = run_full(w, inp)
+    got = run_full(w, inp, flags)
     compare_full(w, inp, got)
     if case["bias"] == "one_hot":
         assert got["routing"]["counts"][3].item() >= 0.9 * w.T
         dev = to_device(w, inp)
-        layer = make_layer(w)
+        layer = make_layer(w, flags)
         layer.forward(dev["x"], dev, training=True)
         G1 = empty_grads(w, "cuda", fill=0.5)
         layer.backward(dev["x"], dev["dy"], dev, G1, accumulate=True)
@@ -222,6 +226,17 @@ def test_small_cdac_twin_full_config():
     assert (w.r, w.h, w.cdac) == (1024, 64, True)
     inp = conditioned(w)
     compare_full(w, inp, run_full(w, inp))
+
+
+@pytest.mark.parametrize("shape", [
+    dict(T=1, d=64, r=256, h=256, E=8, k=3),        # one token: most experts empty (their gradients are zero-filled)
+    dict(T=333, d=128, r=320, h=256, E=5, k=5),     # ragged widths (320 = 256 + 64), k = E
+    dict(T=4096, d=256, r=256, h=1024, E=4, k=1),   # few experts, thousands of rows each: every expert in parts
+])
+def test_bf16_dynamic_weight_gradient_kernel(shape):
+    w = wl.Workload("dyn", dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=733, **shape)
+    inp = conditioned(w)
+    compare_full(w, inp, run_full(w, inp, wl.FLAG_DYNAMIC_WGRAD))
 
 
 def test_route_matches_forward_tables_and_zero_tokens_is_a_noop():
