@@ -71,8 +71,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0;
+            // the next tile is looked up (a global load for grouped rows) before this tile's loads are issued, so
+            // that its latency does not sit between two tiles
+            Tile nxt = get_tile(p, BN, blockIdx.x < total ? blockIdx.x : 0, tiles_m, tiles_n);
             for (int t = blockIdx.x; t < total; t += gridDim.x) {
-                const Tile tl = get_tile(p, BN, t, tiles_m, tiles_n);
+                const Tile tl = nxt;
+                if (t + (int)gridDim.x < total) nxt = get_tile(p, BN, t + gridDim.x, tiles_m, tiles_n);
                 for (int kb = 0; kb < tl.num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, dead, p.status);

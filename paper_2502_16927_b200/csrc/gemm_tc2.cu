@@ -52,14 +52,16 @@ __device__ __forceinline__ PairTile get_pair_tile(const TcParams& p, int BN, int
             const int mid = (lo + hi) >> 1;
             if (s_pp[mid] <= pair) lo = mid; else hi = mid;
         }
-        const int first = p.poffsets[lo] / kPad, count = (p.poffsets[lo + 1] - p.poffsets[lo]) / kPad;
+        const int32_t* s_off = s_pp + p.num_experts + 1;       // the padded offsets, staged beside the prefix
+        const int first = s_off[lo] / kPad, count = (s_off[lo + 1] - s_off[lo]) / kPad;
         const int j = pair - s_pp[lo];
         t.expert = lo;
         t.m0 = (first + 2 * j) * BM;
         t.halves = min(2, count - 2 * j);
     } else if (p.group == GROUP_K) {
-        t.k_row0 = p.poffsets[e];
-        t.num_kb = (p.poffsets[e + 1] - t.k_row0) / BK;
+        const int32_t* s_off = s_pp + p.num_experts + 1;
+        t.k_row0 = s_off[e];
+        t.num_kb = (s_off[e + 1] - t.k_row0) / BK;
         t.c_base = (int64_t)e * p.c_stride;
     }
     return t;
@@ -89,7 +91,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     uint64_t* z_bar = tmem_empty_bar + 2;                    // [kEpiWarps]
     uint32_t* tmem_slot = (uint32_t*)(z_bar + kEpiWarps);
     volatile int* dead = (volatile int*)(tmem_slot + 1);
-    int32_t* s_pp = (int32_t*)(tmem_slot + 4);               // [num_experts + 1] pair prefix (GROUP_M)
+    int32_t* s_pp = (int32_t*)(tmem_slot + 4);               // [E + 1] pair prefix (GROUP_M), then [E + 1] padded offsets:
+                                                             // every role looks tiles up here, not in global memory
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -99,17 +102,15 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ---- work list
     const int tiles_n = (p.N + BN - 1) / BN;
     int pairs_m = (p.M + 2 * BM - 1) / (2 * BM);
-    if (p.group == GROUP_M) {
-        // the padded offsets come to shared memory in one round trip, then turn into the pair prefix in place
-        for (int e = threadIdx.x; e <= p.num_experts; e += blockDim.x) s_pp[e] = p.poffsets[e];
+    if (p.group != GROUP_NONE && p.poffsets) {
+        int32_t* s_off = s_pp + p.num_experts + 1;
+        for (int e = threadIdx.x; e <= p.num_experts; e += blockDim.x) s_off[e] = p.poffsets[e];
         __syncthreads();
-        if (threadIdx.x == 0) {
-            int run = 0, lo = s_pp[0];
+        if (threadIdx.x == 0 && p.group == GROUP_M) {
+            int run = 0;
             for (int e = 0; e < p.num_experts; ++e) {
-                const int hi = s_pp[e + 1];
                 s_pp[e] = run;
-                run += ((hi - lo) / kPad + 1) / 2;
-                lo = hi;
+                run += ((s_off[e + 1] - s_off[e]) / kPad + 1) / 2;
             }
             s_pp[p.num_experts] = run;
         }
@@ -305,7 +306,7 @@ cudaError_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUte
                         const CUtensorMap& mb2, const TcParams& p, int64_t max_items, cudaStream_t stream) {
     constexpr size_t kMaxSmem = 232448;                      // 227 KB: the most a CTA can have on sm_100
     const size_t smem = STAGES * (BM * BK * 2 + (BN / 2) * BK * 2) + (TMA_EPI ? kEpiWarps * 2 * kBoxBytes : 0) +
-                        (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + (size_t)(p.num_experts + 1) * 4 + 1024;
+                        (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + 2 * (size_t)(p.num_experts + 1) * 4 + 1024;
     if (smem > kMaxSmem) return cudaErrorInvalidConfiguration;
     static PerDeviceOnce once;
     auto kernel = gemm_tc_pair_kernel<BN, STAGES, AK, BKM, TMA_EPI>;
@@ -389,10 +390,10 @@ cudaError_t gemm_tc_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
     const bool staged = tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 &&
                         (g.epilogue != EPI_DACT || g.group != GROUP_K);
-    // 32 KB per stage and CTA: 5 stages beside the 64 KB store staging (4 if the expert table is long), 6 without it
+    // 32 KB per stage and CTA: 5 stages beside the 64 KB store staging (4 if the expert tables are long), 6 without it
     if (!staged) return dispatch_pair<256, 6, false>(g, status, stream);
     const int E = g.group == GROUP_NONE ? 1 : g.num_experts;
-    return E <= 256 ? dispatch_pair<256, 5, true>(g, status, stream) : dispatch_pair<256, 4, true>(g, status, stream);
+    return E <= 192 ? dispatch_pair<256, 5, true>(g, status, stream) : dispatch_pair<256, 4, true>(g, status, stream);
 }
 
 }  // namespace bigmac
