@@ -78,6 +78,60 @@ __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ log
     for (int j = lane; j < k; j += 32) out_w[j] = expf(out_w[j] - top) / part;
 }
 
+// Four tokens per warp, eight lanes per token, for k <= 8 and E a multiple of 32 up to 256: lane l of a group
+// holds the experts 4 (l + 8 i) + c (one float4 per i), the arg-max tree has three levels, and the j-th winner
+// stays in lane j of the group until one store.  Same order (logit descending, expert id ascending).
+template <int Q>   // float4 loads per lane: E = 32 Q
+__global__ void __launch_bounds__(256) topk8_kernel(const float* __restrict__ logits, const float* __restrict__ b_gate,
+                                                    int T, int k, int32_t* __restrict__ topk_idx,
+                                                    float* __restrict__ topk_w) {
+    constexpr int E = 32 * Q;
+    const int lane = threadIdx.x & 31, sub = lane & 7;
+    const int t = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 4 + (lane >> 3);
+    const bool live = t < T;
+    const float4* row = reinterpret_cast<const float4*>(logits + (size_t)(live ? t : 0) * E);
+    float v[4 * Q];
+#pragma unroll
+    for (int i = 0; i < Q; ++i) {
+        float4 x = row[sub + 8 * i];
+        if (b_gate) {
+            const float4 b = reinterpret_cast<const float4*>(b_gate)[sub + 8 * i];
+            x.x += b.x; x.y += b.y; x.z += b.z; x.w += b.w;
+        }
+        v[4 * i] = x.x; v[4 * i + 1] = x.y; v[4 * i + 2] = x.z; v[4 * i + 3] = x.w;
+    }
+    float my_v = -INFINITY;
+    int my_e = 0;
+    for (int j = 0; j < k; ++j) {
+        float best = -INFINITY;
+        int best_e = 0x7fffffff;
+#pragma unroll
+        for (int i = 0; i < 4 * Q; ++i) {          // ascending expert id within the lane: strict > keeps the lowest id
+            const int e = 4 * (sub + 8 * (i >> 2)) + (i & 3);
+            if (v[i] > best) { best = v[i]; best_e = e; }
+        }
+#pragma unroll
+        for (int off = 4; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(kFull, best, off);
+            const int oe = __shfl_xor_sync(kFull, best_e, off);
+            if (ov > best || (ov == best && oe < best_e)) { best = ov; best_e = oe; }
+        }
+#pragma unroll
+        for (int i = 0; i < 4 * Q; ++i)
+            if (4 * (sub + 8 * (i >> 2)) + (i & 3) == best_e) v[i] = -INFINITY;
+        if (sub == j) { my_v = best; my_e = best_e; }
+    }
+    const float top = __shfl_sync(kFull, my_v, lane & 24);
+    const float ex = sub < k ? expf(my_v - top) : 0.0f;
+    float part = ex;
+#pragma unroll
+    for (int off = 4; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
+    if (live && sub < k) {
+        topk_idx[(size_t)t * k + sub] = my_e;
+        topk_w[(size_t)t * k + sub] = ex / part;
+    }
+}
+
 // Pass 1 of the counting sort.  Block b owns slots [b*kSortChunk, (b+1)*kSortChunk); it writes, per
 // slot, the number of earlier slots of the same block routed to the same expert, and per expert the
 // block's count.  Warps own consecutive sub-chunks, so the order is the slot order.
@@ -196,6 +250,20 @@ cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, 
                         float* topk_w, cudaStream_t stream) {
     if (T == 0) return cudaSuccess;
     const int warps = 8;
+    if (k <= 8 && E % 32 == 0 && E <= 256 && ((uintptr_t)logits % 16 == 0) && ((uintptr_t)b_gate % 16 == 0)) {
+        const unsigned blocks = (unsigned)((T + 4 * warps - 1) / (4 * warps));
+        switch (E / 32) {
+            case 1: topk8_kernel<1><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
+            case 2: topk8_kernel<2><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
+            case 3: topk8_kernel<3><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
+            case 4: topk8_kernel<4><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
+            case 5: topk8_kernel<5><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
+            case 6: topk8_kernel<6><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
+            case 7: topk8_kernel<7><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
+            default: topk8_kernel<8><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
+        }
+        return cudaGetLastError();
+    }
     dim3 grid((T + warps - 1) / warps), block(warps * 32);
     const int vpl = (E + 31) / 32;
 #define BIGMAC_TOPK(V)                                                                                   \
