@@ -186,23 +186,52 @@ __global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ b
                                                          int32_t* __restrict__ n_tiles) {
     __shared__ int32_t s_cnt[kMaxExperts];
     __shared__ int32_t s_poff[kMaxExperts + 1];
-    for (int e = threadIdx.x; e < E; e += blockDim.x) {
-        int run = 0;
-        int b = 0;
-        for (; b + 8 <= n_blocks; b += 8) {
-            int c[8];
+    __shared__ int32_t s_part[1024];
+    // thread (part, e) owns a contiguous range of blocks of expert e: range sums, then the exclusive scan inside
+    // the range starting from the sum of the ranges before it (two dependent passes instead of one long one)
+    const int parts = E >= (int)blockDim.x ? 1 : min(16, min((int)blockDim.x / E, max(n_blocks, 1)));
+    const int per = (n_blocks + parts - 1) / parts;
+    for (int e0 = 0; e0 < E; e0 += blockDim.x / parts) {
+        const int e = e0 + threadIdx.x % (blockDim.x / parts), part = threadIdx.x / (blockDim.x / parts);
+        const bool mine = e < E && part < parts;
+        const int b0 = min(n_blocks, part * per), b1 = min(n_blocks, b0 + per);
+        int sum = 0;
+        if (mine) {
+            int b = b0;
+            for (; b + 8 <= b1; b += 8) {
+                int c[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) c[i] = block_counts[(size_t)(b + i) * E + e];
+                for (int i = 0; i < 8; ++i) c[i] = block_counts[(size_t)(b + i) * E + e];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) { block_counts[(size_t)(b + i) * E + e] = run; run += c[i]; }
+                for (int i = 0; i < 8; ++i) sum += c[i];
+            }
+            for (; b < b1; ++b) sum += block_counts[(size_t)b * E + e];
         }
-        for (; b < n_blocks; ++b) {
-            const int c = block_counts[(size_t)b * E + e];
-            block_counts[(size_t)b * E + e] = run;
-            run += c;
+        __syncthreads();                            // s_part of the previous round has been read
+        if (part < parts) s_part[part * (blockDim.x / parts) + threadIdx.x % (blockDim.x / parts)] = sum;
+        __syncthreads();
+        if (mine) {
+            int run = 0, total = 0;
+            for (int q = 0; q < parts; ++q) {
+                const int v = s_part[q * (blockDim.x / parts) + threadIdx.x % (blockDim.x / parts)];
+                if (q < part) run += v;
+                total += v;
+            }
+            if (part == 0) { s_cnt[e] = total; counts[e] = total; }
+            int b = b0;
+            for (; b + 8 <= b1; b += 8) {
+                int c[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) c[i] = block_counts[(size_t)(b + i) * E + e];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { block_counts[(size_t)(b + i) * E + e] = run; run += c[i]; }
+            }
+            for (; b < b1; ++b) {
+                const int c = block_counts[(size_t)b * E + e];
+                block_counts[(size_t)b * E + e] = run;
+                run += c;
+            }
         }
-        s_cnt[e] = run;
-        counts[e] = run;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
