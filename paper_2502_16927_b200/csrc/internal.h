@@ -73,6 +73,11 @@ bool gemm_tc_groupk_supported(const GemmArgs& g);
 size_t gemm_tc_groupk_ws_bytes(int M, int N, int E);
 cudaError_t gemm_tc_groupk(const GemmArgs& g, int* status, int* sched, void* ws, cudaStream_t stream);
 cudaError_t gemm_tc_groupk_finish(const GemmArgs& g, void* ws, cudaStream_t stream);   // always after gemm_tc_groupk
+// Inference forward of the experts in one kernel for r <= 256 (gemm_tc_mlp.cu): u = sigma(xg W1_e^T) W2_e^T per
+// 128-row tile, hidden activations kept on the SM.
+bool fused_mlp_supported(int r, int h, int dtype);
+cudaError_t launch_fused_mlp(const void* xg, const void* w1, const void* w2, void* u, int64_t max_rows, int r, int h, int E,
+                             int act, const int32_t* tile_expert, const int32_t* n_tiles, int* status, cudaStream_t stream);
 // CTA-pair variant (tcgen05 cta_group::2) for outputs at least 256 wide.
 bool gemm_tc_pair_supported(const GemmArgs& g);
 bool gemm_tc_pair_preferred(const GemmArgs& g);

@@ -37,6 +37,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return done != 0;
 }
+// Non-blocking test of a phase (try_wait may park the thread for a while before it looks again; a chain of short
+// dependent steps polls with this one instead).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ void mbar_spin(uint64_t* bar, uint32_t parity, volatile int* dead, int* status) {
+    if (*dead) return;
+    for (uint32_t i = 0; i < (kWaitLimit << 4); ++i) {
+        if (mbar_test_wait(bar, parity)) return;
+        if ((i & 4095u) == 4095u && *dead) return;
+    }
+    *dead = 1;
+    atomicExch(status, 1);
+}
 // Bounded wait.  `dead` is a CTA-wide flag in shared memory: once any wait ran out nobody waits again.
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile int* dead, int* status) {
     if (*dead) return;
@@ -123,6 +145,15 @@ __device__ __forceinline__ void tmem_load_32_nowait(uint32_t taddr, uint32_t* v)
           "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
           "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
           "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_load_16_nowait(uint32_t taddr, uint32_t* v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
         : "r"(taddr)
         : "memory");
 }
@@ -292,10 +323,10 @@ __device__ __forceinline__ void mul_by_sig32(float* v, const uint32_t* w) {
 
 // Activation of 32 accumulator values in place; with WITH_G the 32 sigma' values are packed, one byte each, in wg[0..7].
 // The activation is a compile-time constant here so that the switch is taken once per chunk, not per element.
-template <int ACT, bool WITH_G>
+template <int ACT, bool WITH_G, int COUNT = 32>
 __device__ __forceinline__ void act_chunk(float* v, uint32_t* wg) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < COUNT / 4; ++i) {
         float a[4], g[4];
         if (ACT == BIGMAC_ACT_GELU_ERF) {
             gelu_pair2(v[4 * i], v[4 * i + 1], a[0], a[1], g[0], g[1]);
@@ -309,13 +340,13 @@ __device__ __forceinline__ void act_chunk(float* v, uint32_t* wg) {
         if (WITH_G) wg[i] = sig_quant4(g[0], g[1], g[2], g[3]);
     }
 }
-template <bool WITH_G>
+template <bool WITH_G, int COUNT = 32>
 __device__ __forceinline__ void act_chunk_any(int act, float* v, uint32_t* wg) {
     switch (act) {
-        case BIGMAC_ACT_GELU_ERF: act_chunk<BIGMAC_ACT_GELU_ERF, WITH_G>(v, wg); break;
-        case BIGMAC_ACT_RELU: act_chunk<BIGMAC_ACT_RELU, WITH_G>(v, wg); break;
-        case BIGMAC_ACT_GELU_TANH: act_chunk<BIGMAC_ACT_GELU_TANH, WITH_G>(v, wg); break;
-        default: act_chunk<BIGMAC_ACT_IDENTITY, WITH_G>(v, wg); break;
+        case BIGMAC_ACT_GELU_ERF: act_chunk<BIGMAC_ACT_GELU_ERF, WITH_G, COUNT>(v, wg); break;
+        case BIGMAC_ACT_RELU: act_chunk<BIGMAC_ACT_RELU, WITH_G, COUNT>(v, wg); break;
+        case BIGMAC_ACT_GELU_TANH: act_chunk<BIGMAC_ACT_GELU_TANH, WITH_G, COUNT>(v, wg); break;
+        default: act_chunk<BIGMAC_ACT_IDENTITY, WITH_G, COUNT>(v, wg); break;
     }
 }
 

@@ -350,3 +350,34 @@ def test_small_batch_inference_forward(T, shape):
     assert_within(w, float_errors(w, {"y": to_numpy(y)}, {"y": ref}))
     assert torch.equal(y, y2)
     layer.close()
+
+
+@pytest.mark.parametrize("case", [
+    dict(T=300, d=128, r=64, h=192, E=5, k=2, act=wl.ACT_GELU_ERF),      # narrowest width, three hidden chunks, ragged segments
+    dict(T=1000, d=256, r=192, h=320, E=16, k=4, act=wl.ACT_RELU),       # widths that are odd multiples of 64
+    dict(T=2048, d=512, r=256, h=1024, E=8, k=2, act=wl.ACT_GELU_ERF),   # the widest case: all of shared memory, 384 TMEM columns
+    dict(T=700, d=128, r=128, h=64, E=40, k=1, act=wl.ACT_GELU_TANH),    # one hidden chunk per tile, empty experts
+])
+def test_inference_forward_with_the_experts_in_one_kernel(case):
+    """Inference forward above the small-batch limit with r <= 256: expert GEMM1, sigma and GEMM2 run as one kernel
+    whose hidden activations stay on the SM.  y against the oracle, and against the training forward of the same
+    layer (which stores the activations in HBM)."""
+    import torch
+
+    case = dict(case)
+    act = case.pop("act")
+    w = wl.Workload("mlp", dtype=wl.DTYPE_BF16, act=act, seed=911, **case)
+    inp = conditioned(w)
+    dev = to_device(w, inp)
+    layer = make_layer(w)
+    y, R = layer.forward(dev["x"], dev, training=False, want_routing=True)
+    y_train = layer.forward(dev["x"], dev, training=True).clone()
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    rt = oracle.route(inp, w.k)
+    check_routing(R, rt)
+    ref = oracle.forward_tokens(inp, rt, w.act)["y"]
+    assert_within(w, float_errors(w, {"y": to_numpy(y)}, {"y": ref}))
+    # same roundings (bf16 activations, fp32 accumulation), different accumulation grouping only
+    assert oracle.max_rel_err(to_numpy(y), to_numpy(y_train)) <= 2.0 ** -7
+    layer.close()
