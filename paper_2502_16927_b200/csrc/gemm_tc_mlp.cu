@@ -12,12 +12,14 @@
 // r = 256: X 64 KB, W1 and W2 chunks double-buffered 2 x 32 KB each, A2 2 x 16 KB = 224 KB.  After the last chunk
 // the 16 warps store acc2 as bf16 rows of u; the next tile's GEMM1s run meanwhile, only its first GEMM2 waits.
 // All waits are bounded (status word); the tile -> expert table is read one tile ahead.
-// Limit (measured with per-chunk clock stamps): a W2 buffer frees when GEMM2 two chunks back completes and its refill
-// takes about 3 us under load, so a chunk takes 1.5-1.9 us where the tensor pipe needs 0.5: with X and A2 resident
-// there is room for 128 KB of weights in flight per SM, two thirds of what the unfused kernels keep in flight.  The
-// layer therefore uses this kernel only on short tile lists (decode-sized batches), where it saves a launch and the
-// HBM round trip of the activations; the fix for long lists is the same pipeline on CTA pairs (half the weight
-// bytes per SM), not built.
+// Limit (measured with clock stamps around every wait of the MMA warp): a chunk takes about 1.8 us where the
+// tensor pipe needs 0.5.  The waits are short; the time goes into issuing the chunk's 16 + 4 tcgen05.mma
+// instructions, about 100 cycles each whatever their size, and GEMM1's are only N = 64 wide (32-64 cycles of
+// tensor work each).  A variant on CTA pairs (half the weight bytes per SM, four chunks in flight) ran at the same
+// speed, so loads are not what limits it.  A 128-wide chunk would halve the instruction count but leaves no room to
+// double-buffer the activated chunk beside X in shared memory at r = 256.  The layer therefore uses this kernel
+// only on short tile lists (decode-sized batches), where it saves a launch and the HBM round trip of the
+// activations; on long lists the two separate GEMMs (N = 256 instructions) are faster.
 #include "tc_common.cuh"
 
 namespace bigmac {
@@ -134,6 +136,11 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const uint32_t idesc1 = instr_desc(BH, false, false);
         const uint32_t idesc2 = instr_desc(p.r, false, false);
         const uint32_t acc2_tmem = tmem_base + kAcc1 * BH;
+        // Descriptors of the buffers' first bytes; the address field (bits 0-13, in 16-byte units) takes offsets by plain
+        // addition, which keeps the instruction stream of this warp short: it shares its scheduler with four busy
+        // epilogue warps, and with descriptors rebuilt per MMA the issue of one chunk's MMAs took longer than the MMAs.
+        const uint64_t desc_x = smem_desc(smem_u32(s_x), 16, 1024), desc_w1 = smem_desc(smem_u32(s_w1), 16, 1024);
+        const uint64_t desc_w2 = smem_desc(smem_u32(s_w2), 16, 1024), desc_a2 = smem_desc(smem_u32(s_a2), 16, 1024);
         uint32_t g = 0, tl = 0;
         // GEMM2 of global chunk gp (chunk cp of tile number tile_no)
         auto gemm2 = [&](uint32_t gp, int cp, uint32_t tile_no) {
@@ -144,11 +151,10 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (cp == 0) mbar_spin(acc2_empty, (tile_no & 1) ^ 1, dead, p.status);
             tc_fence_after();
             if (lane == 0) {
-                const uint32_t a_addr = smem_u32(s_a2 + s * A2_BYTES), b_addr = smem_u32(s_w2 + s * W2_BYTES);
+                const uint64_t da = desc_a2 + ((s * A2_BYTES) >> 4), db = desc_w2 + ((s * W2_BYTES) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < BH / UMMA_K; ++kk)
-                    umma_bf16(acc2_tmem, smem_desc(a_addr + kk * UMMA_K * 2, 16, 1024), smem_desc(b_addr + kk * UMMA_K * 2, 16, 1024),
-                              idesc2, (cp | kk) != 0);
+                    umma_bf16(acc2_tmem, da + ((kk * UMMA_K * 2) >> 4), db + ((kk * UMMA_K * 2) >> 4), idesc2, (cp | kk) != 0);
                 umma_commit(&a2_empty[s]);
                 umma_commit(&w2_empty[s]);
             }
@@ -163,12 +169,11 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (lane == 0) {
                 const uint32_t d_tmem = tmem_base + a * BH;
                 for (int kb = 0; kb < KB1; ++kb) {
-                    const uint32_t a_addr = smem_u32(s_x + kb * (BM * BK * 2));
-                    const uint32_t b_addr = smem_u32(s_w1 + s * W1_BYTES + kb * (BH * BK * 2));
+                    const uint64_t da = desc_x + ((kb * (BM * BK * 2)) >> 4);
+                    const uint64_t db = desc_w1 + ((s * W1_BYTES + kb * (BH * BK * 2)) >> 4);
 #pragma unroll
                     for (int kk = 0; kk < BK / UMMA_K; ++kk)
-                        umma_bf16(d_tmem, smem_desc(a_addr + kk * UMMA_K * 2, 16, 1024), smem_desc(b_addr + kk * UMMA_K * 2, 16, 1024),
-                                  idesc1, (kb | kk) != 0);
+                        umma_bf16(d_tmem, da + ((kk * UMMA_K * 2) >> 4), db + ((kk * UMMA_K * 2) >> 4), idesc1, (kb | kk) != 0);
                 }
                 umma_commit(&w1_empty[s]);
                 umma_commit(&acc1_full[a]);

@@ -422,12 +422,13 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     }
     { Stage s(L, S_DISPATCH, st); BIGMAC_CUDA(launch_dispatch(b.x_lo, b.xg, b.tb, m.k, m.r, m.dtype, m.P, st)); }  // F5 dispatch at width r
     // Inference, low width r <= 256, up to two row tiles per SM: F6 + F7 in one kernel, the hidden activations stay on
-    // the SM.  With X and the activated chunk resident only 128 KB of weights can be in flight per SM, so on long
-    // tile lists the two separate GEMMs (deeper load pipelines) are faster: measured 0.378 vs 0.329 ms forward at the
-    // medium workload, 0.098 vs 0.106 ms at 512 decode tokens; BIGMAC_FUSED_MLP=0 / =2 force it off / on.
+    // the SM.  On long tile lists the two separate GEMMs are faster (the fused kernel is bound by the issue of its many
+    // narrow MMA instructions): measured 0.375 vs 0.329 ms forward at the medium workload, 0.099 vs 0.106 ms at 512
+    // decode tokens.  BIGMAC_FUSED_MLP=0 / =2 force it off / on.
     static const int fuse_mlp_mode = []() { const char* e = std::getenv("BIGMAC_FUSED_MLP"); return e ? atoi(e) : 1; }();
-    const bool fuse_mlp_enabled = fuse_mlp_mode == 2 || (fuse_mlp_mode == 1 && m.P / kPad <= 2 * (int64_t)gemm_tc_sm_count());
-    if (!training && fuse_mlp_enabled && sigma_as_bytes(L) && fused_mlp_supported(m.r, m.h, m.dtype)) {
+    const bool short_list = m.P / kPad <= 2 * (int64_t)gemm_tc_sm_count();
+    if (!training && (fuse_mlp_mode == 2 || (fuse_mlp_mode == 1 && short_list)) && sigma_as_bytes(L) &&
+        fused_mlp_supported(m.r, m.h, m.dtype)) {
         Stage s(L, S_FUSED_MLP, st);
         BIGMAC_CUDA(launch_fused_mlp(b.xg, W->w1, W->w2, b.u, m.P, m.r, m.h, m.E, c.act, b.tb.tile_expert, b.tb.n_tiles,
                                      L->status, st));
