@@ -624,6 +624,11 @@ int bigmac_device_status(bigmac_layer_t* L, void* stream) {
     if (cudaMemcpyAsync(&word, L->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
         cudaMemsetAsync(L->status, 0, sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
         return BIGMAC_ERR_CUDA;
+    if (word != 0) {
+        // a kernel gave up on a wait: its work counters and the grid-barrier word may be mid-count; back to rest
+        if (cudaMemsetAsync(L->status + 1, 0, 3 * sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+            return BIGMAC_ERR_CUDA;
+    }
     return word == 0 ? BIGMAC_OK : BIGMAC_ERR_TIMEOUT;
 }
 
