@@ -67,6 +67,51 @@ __device__ __forceinline__ PairTile get_pair_tile(const TcParams& p, int BN, int
     return t;
 }
 
+// Walks the work items of one pair, w = cluster_id, cluster_id + num_clusters, ...  For dense and row-grouped
+// problems the (row pair, column tile) indices and the expert are carried along instead of being recomputed from
+// w: the lookup (two integer divisions and a binary search, run by every warp at every tile) took about 1500 of
+// the 8500 cycles an epilogue warp spends per output-heavy tile.
+struct TileWalk {
+    int w, pair, n, lo;
+};
+
+__device__ __forceinline__ void walk_init(TileWalk& tw, int cluster_id, int tiles_n) {
+    tw.w = cluster_id;
+    tw.pair = cluster_id / tiles_n;
+    tw.n = cluster_id - tw.pair * tiles_n;
+    tw.lo = 0;
+}
+
+__device__ __forceinline__ void walk_next(TileWalk& tw, int num_clusters, int step_pair, int step_n, int tiles_n) {
+    tw.w += num_clusters;
+    tw.pair += step_pair;
+    tw.n += step_n;
+    if (tw.n >= tiles_n) { tw.n -= tiles_n; ++tw.pair; }
+}
+
+__device__ __forceinline__ PairTile walk_tile(const TcParams& p, int BN, TileWalk& tw, int pairs_m, int tiles_n, const int32_t* s_pp) {
+    if (p.group == GROUP_K || p.split_k > 1) return get_pair_tile(p, BN, tw.w, pairs_m, tiles_n, s_pp);
+    PairTile t;
+    t.n0 = tw.n * BN;
+    t.m0 = tw.pair * 2 * BM;
+    t.expert = 0;
+    t.k_row0 = 0;
+    t.num_kb = (p.K + BK - 1) / BK;
+    t.m_limit = p.M;
+    t.halves = 2;
+    t.c_base = 0;
+    if (p.group == GROUP_M) {
+        const int32_t* s_off = s_pp + p.num_experts + 1;
+        while (tw.lo + 1 < p.num_experts && s_pp[tw.lo + 1] <= tw.pair) ++tw.lo;     // pairs only grow along the walk
+        const int first = s_off[tw.lo] / kPad, count = (s_off[tw.lo + 1] - s_off[tw.lo]) / kPad;
+        const int j = tw.pair - s_pp[tw.lo];
+        t.expert = tw.lo;
+        t.m0 = (first + 2 * j) * BM;
+        t.halves = min(2, count - 2 * j);
+    }
+    return t;
+}
+
 template <int BN, int STAGES, bool A_KMAJOR, bool B_KMAJOR, bool TMA_EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsV2, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -131,13 +176,15 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t tmem_base = *tmem_slot;
     if (p.group == GROUP_M) pairs_m = s_pp[p.num_experts];
     const int total = pairs_m * tiles_n * (p.group == GROUP_K ? p.num_experts : p.split_k);
+    const int step_pair = num_clusters / tiles_n, step_n = num_clusters - step_pair * tiles_n;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
             uint32_t it = 0;
-            for (int w = cluster_id; w < total; w += num_clusters) {
-                const PairTile tl = get_pair_tile(p, BN, w, pairs_m, tiles_n, s_pp);
+            TileWalk tw;
+            for (walk_init(tw, cluster_id, tiles_n); tw.w < total; walk_next(tw, num_clusters, step_pair, step_n, tiles_n)) {
+                const PairTile tl = walk_tile(p, BN, tw, pairs_m, tiles_n, s_pp);
                 const int my_m0 = tl.m0 + (int)rank * BM;
                 const int my_n0 = tl.n0 + (int)rank * BH;
                 for (int kb = 0; kb < tl.num_kb; ++kb, ++it) {
@@ -171,8 +218,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         if (leader) {
             constexpr uint32_t idesc = instr_desc_pair(BN, !A_KMAJOR, !B_KMAJOR);
             uint32_t it = 0, local = 0;
-            for (int w = cluster_id; w < total; w += num_clusters, ++local) {
-                const PairTile tl = get_pair_tile(p, BN, w, pairs_m, tiles_n, s_pp);
+            TileWalk tw;
+            for (walk_init(tw, cluster_id, tiles_n); tw.w < total; walk_next(tw, num_clusters, step_pair, step_n, tiles_n), ++local) {
+                const PairTile tl = walk_tile(p, BN, tw, pairs_m, tiles_n, s_pp);
                 const uint32_t acc = local & 1;
                 mbar_wait(&tmem_empty_bar[acc], ((local >> 1) & 1) ^ 1, dead, p.status);
                 tc_fence_after();
@@ -229,10 +277,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 tma_load_2d(box_z, &map_z, my_z_bar, tile.n0 + part * COLS_PER_WARP, tile.m0 + (int)rank * BM + quad * 32);
             }
         };
-        if (z_prefetch && cluster_id < total) issue_z(get_pair_tile(p, BN, cluster_id, pairs_m, tiles_n, s_pp));
         uint32_t local = 0;
-        for (int w = cluster_id; w < total; w += num_clusters, ++local) {
-            const PairTile tl = get_pair_tile(p, BN, w, pairs_m, tiles_n, s_pp);
+        TileWalk tw;
+        walk_init(tw, cluster_id, tiles_n);
+        PairTile nxt = tw.w < total ? walk_tile(p, BN, tw, pairs_m, tiles_n, s_pp) : PairTile{};
+        if (z_prefetch && tw.w < total) issue_z(nxt);
+        for (; tw.w < total; ++local) {
+            const PairTile tl = nxt;
+            const int w = tw.w;
+            walk_next(tw, num_clusters, step_pair, step_n, tiles_n);            // tw / nxt now describe the next item
+            if (tw.w < total) nxt = walk_tile(p, BN, tw, pairs_m, tiles_n, s_pp);
             const uint32_t acc = local & 1;
             mbar_wait(&tmem_full_bar[acc], (local >> 1) & 1, dead, p.status);
             tc_fence_after();
@@ -272,7 +326,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         if (c == CHUNKS - 1) {             // box read by every lane: fetch the next tile's
                             fence_async_smem();
                             __syncwarp();
-                            if (w + num_clusters < total) issue_z(get_pair_tile(p, BN, w + num_clusters, pairs_m, tiles_n, s_pp));
+                            if (w + num_clusters < total) issue_z(nxt);
                         }
                         mul_by_sig32(v, wz);
                     }
