@@ -70,16 +70,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t s = 0, phase = 1;                     // stage and the parity its "empty" barrier is waited on with
             // the next tile is looked up (a global load for grouped rows) before this tile's loads are issued, so
             // that its latency does not sit between two tiles
             Tile nxt = get_tile(p, BN, blockIdx.x < total ? blockIdx.x : 0, tiles_m, tiles_n);
             for (int t = blockIdx.x; t < total; t += gridDim.x) {
                 const Tile tl = nxt;
                 if (t + (int)gridDim.x < total) nxt = get_tile(p, BN, t + gridDim.x, tiles_m, tiles_n);
-                for (int kb = 0; kb < tl.num_kb; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, dead, p.status);
+                for (int kb = 0; kb < tl.num_kb; ++kb, s = (s + 1 == STAGES ? 0 : s + 1), phase ^= (s == 0)) {
+                    mbar_wait_lean(&empty_bar[s], phase, dead, p.status);
                     mbar_expect_tx(&full_bar[s], A_BYTES + B_BYTES);
                     const int k0 = tl.k_row0 + kb * BK;
                     uint8_t* a_dst = smem_a + s * A_BYTES;
@@ -106,39 +105,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        constexpr uint32_t idesc = instr_desc(BN, !A_KMAJOR, !B_KMAJOR);
-        uint32_t it = 0, local = 0;
-        for (int t = blockIdx.x; t < total; t += gridDim.x, ++local) {
-            const Tile tl = get_tile(p, BN, t, tiles_m, tiles_n);
-            const uint32_t acc = local & 1;
-            mbar_wait(&tmem_empty_bar[acc], ((local >> 1) & 1) ^ 1, dead, p.status);
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + acc * BN;
-            for (int kb = 0; kb < tl.num_kb; ++kb, ++it) {
-                const int s = it % STAGES;
-                mbar_wait(&full_bar[s], (it / STAGES) & 1, dead, p.status);
+        // ------------------------------------------------------------------ MMA issuer (one thread)
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc(BN, !A_KMAJOR, !B_KMAJOR);
+            // descriptors of stage 0; the address field (16-byte units, bits 0-13) takes stage and k-step offsets by addition
+            const uint64_t da0 = A_KMAJOR ? smem_desc(smem_u32(smem_a), 16, 1024) : smem_desc(smem_u32(smem_a), CHUNK_BYTES, 1024);
+            const uint64_t db0 = B_KMAJOR ? smem_desc(smem_u32(smem_b), 16, 1024) : smem_desc(smem_u32(smem_b), CHUNK_BYTES, 1024);
+            constexpr uint32_t kStepA = (A_KMAJOR ? UMMA_K * 2 : UMMA_K * 128) >> 4, kStepB = (B_KMAJOR ? UMMA_K * 2 : UMMA_K * 128) >> 4;
+            const bool uniform_k = p.group != GROUP_K && p.split_k <= 1;     // every tile contracts over all of K
+            uint32_t stage = 0, phase = 0, local = 0;
+            for (int t = blockIdx.x; t < total; t += gridDim.x, ++local) {
+                const int num_kb = uniform_k ? (p.K + BK - 1) / BK : get_tile(p, BN, t, tiles_m, tiles_n).num_kb;
+                const uint32_t acc = local & 1;
+                mbar_wait_lean(&tmem_empty_bar[acc], ((local >> 1) & 1) ^ 1, dead, p.status);
                 tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t a_addr = smem_u32(smem_a + s * A_BYTES);
-                    const uint32_t b_addr = smem_u32(smem_b + s * B_BYTES);
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    mbar_wait_lean(&full_bar[stage], phase, dead, p.status);
+                    tc_fence_after();
+                    const uint64_t da = da0 + stage * (A_BYTES >> 4), db = db0 + stage * (B_BYTES >> 4);
+                    umma_bf16(d_tmem, da, db, idesc, kb != 0);
 #pragma unroll
-                    for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-                        const uint64_t da = A_KMAJOR ? smem_desc(a_addr + kk * UMMA_K * 2, 16, 1024)
-                                                     : smem_desc(a_addr + kk * UMMA_K * 128, CHUNK_BYTES, 1024);
-                        const uint64_t db = B_KMAJOR ? smem_desc(b_addr + kk * UMMA_K * 2, 16, 1024)
-                                                     : smem_desc(b_addr + kk * UMMA_K * 128, CHUNK_BYTES, 1024);
-                        umma_bf16(d_tmem, da, db, idesc, (kb | kk) != 0);
-                    }
-                    umma_commit(&empty_bar[s]);
+                    for (int kk = 1; kk < BK / UMMA_K; ++kk) umma_bf16(d_tmem, da + kk * kStepA, db + kk * kStepB, idesc, 1);
+                    umma_commit(&empty_bar[stage]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
-                __syncwarp();
-            }
-            if (lane == 0) {
-                if (tl.num_kb > 0) umma_commit(&tmem_full_bar[acc]);
+                if (num_kb > 0) umma_commit(&tmem_full_bar[acc]);
                 else mbar_arrive(&tmem_full_bar[acc]);
             }
-            __syncwarp();
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..17)

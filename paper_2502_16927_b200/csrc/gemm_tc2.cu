@@ -181,15 +181,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t s = 0, phase = 1;                     // stage and the parity its "empty" barrier is waited on with
             TileWalk tw;
             for (walk_init(tw, cluster_id, tiles_n); tw.w < total; walk_next(tw, num_clusters, step_pair, step_n, tiles_n)) {
                 const PairTile tl = walk_tile(p, BN, tw, pairs_m, tiles_n, s_pp);
                 const int my_m0 = tl.m0 + (int)rank * BM;
                 const int my_n0 = tl.n0 + (int)rank * BH;
-                for (int kb = 0; kb < tl.num_kb; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, dead, p.status);
+                for (int kb = 0; kb < tl.num_kb; ++kb, s = (s + 1 == STAGES ? 0 : s + 1), phase ^= (s == 0)) {
+                    mbar_wait_lean(&empty_bar[s], phase, dead, p.status);
                     if (leader) mbar_expect_tx(&full_bar[s], 2 * (A_BYTES + B_BYTES));
                     const uint32_t bar = map_to_cta(&full_bar[s], 0);
                     const int k0 = tl.k_row0 + kb * BK;
@@ -214,45 +213,37 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (leader) {
+        // ------------------------------------------------------------------ MMA issuer (one thread of the leader CTA)
+        if (leader && lane == 0) {
             constexpr uint32_t idesc = instr_desc_pair(BN, !A_KMAJOR, !B_KMAJOR);
-            uint32_t it = 0, local = 0;
+            // descriptors of stage 0; the address field (16-byte units, bits 0-13) takes stage and k-step offsets by addition
+            const uint64_t da0 = A_KMAJOR ? smem_desc(smem_u32(smem_a), 16, 1024) : smem_desc(smem_u32(smem_a), CHUNK_BYTES, 1024);
+            const uint64_t db0 = B_KMAJOR ? smem_desc(smem_u32(smem_b), 16, 1024) : smem_desc(smem_u32(smem_b), CHUNK_BYTES, 1024);
+            constexpr uint32_t kStepA = (A_KMAJOR ? UMMA_K * 2 : UMMA_K * 128) >> 4, kStepB = (B_KMAJOR ? UMMA_K * 2 : UMMA_K * 128) >> 4;
+            uint32_t stage = 0, phase = 0, local = 0;
             TileWalk tw;
             for (walk_init(tw, cluster_id, tiles_n); tw.w < total; walk_next(tw, num_clusters, step_pair, step_n, tiles_n), ++local) {
                 const PairTile tl = walk_tile(p, BN, tw, pairs_m, tiles_n, s_pp);
                 const uint32_t acc = local & 1;
-                mbar_wait(&tmem_empty_bar[acc], ((local >> 1) & 1) ^ 1, dead, p.status);
+                mbar_wait_lean(&tmem_empty_bar[acc], ((local >> 1) & 1) ^ 1, dead, p.status);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < tl.num_kb; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    mbar_wait(&full_bar[s], (it / STAGES) & 1, dead, p.status);
+                for (int kb = 0; kb < tl.num_kb; ++kb) {
+                    mbar_wait_lean(&full_bar[stage], phase, dead, p.status);
                     tc_fence_after();
-                    if (lane == 0) {
-                        const uint32_t a_addr = smem_u32(smem_a + s * A_BYTES);
-                        const uint32_t b_addr = smem_u32(smem_b + s * B_BYTES);
+                    const uint64_t da = da0 + stage * (A_BYTES >> 4), db = db0 + stage * (B_BYTES >> 4);
+                    umma_bf16_pair(d_tmem, da, db, idesc, kb != 0);
 #pragma unroll
-                        for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-                            const uint64_t da = A_KMAJOR ? smem_desc(a_addr + kk * UMMA_K * 2, 16, 1024)
-                                                         : smem_desc(a_addr + kk * UMMA_K * 128, CHUNK_BYTES, 1024);
-                            const uint64_t db = B_KMAJOR ? smem_desc(b_addr + kk * UMMA_K * 2, 16, 1024)
-                                                         : smem_desc(b_addr + kk * UMMA_K * 128, CHUNK_BYTES, 1024);
-                            umma_bf16_pair(d_tmem, da, db, idesc, (kb | kk) != 0);
-                        }
-                        umma_commit_pair(&empty_bar[s]);
-                    }
-                    __syncwarp();
+                    for (int kk = 1; kk < BK / UMMA_K; ++kk) umma_bf16_pair(d_tmem, da + kk * kStepA, db + kk * kStepB, idesc, 1);
+                    umma_commit_pair(&empty_bar[stage]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (lane == 0) {
-                    if (tl.num_kb > 0) {
-                        umma_commit_pair(&tmem_full_bar[acc]);
-                    } else {                                   // nothing to contract: zero accumulators, signal directly
-                        mbar_arrive(&tmem_full_bar[acc]);
-                        mbar_arrive_cluster(map_to_cta(&tmem_full_bar[acc], 1));
-                    }
+                if (tl.num_kb > 0) {
+                    umma_commit_pair(&tmem_full_bar[acc]);
+                } else {                                       // nothing to contract: zero accumulators, signal directly
+                    mbar_arrive(&tmem_full_bar[acc]);
+                    mbar_arrive_cluster(map_to_cta(&tmem_full_bar[acc], 1));
                 }
-                __syncwarp();
             }
         }
     } else {
@@ -433,12 +424,9 @@ bool gemm_tc_pair_supported(const GemmArgs& g) {
     return true;
 }
 
-// Measured on B200 (interleaved A/B at the large workload's shapes): pairs win 5-12 % when B is MN-major (half
-// as many TMA boxes per SM) and on wide, output-heavy problems (expert GEMM1, dz, ascend, dx); the K-major /
-// K-major contraction-heavy GEMMs (expert GEMM2, descend) are 1-2 % faster on single CTAs.
-bool gemm_tc_pair_preferred(const GemmArgs& g) {
-    return gemm_tc_pair_supported(g) && (!g.b_kmajor || g.N >= 1024);
-}
+// Measured on B200 (interleaved A/B at the large workload's shapes, after the MMA-issue thread was made lean): pairs
+// are 3-20 % faster on every shape but the training expert GEMM1 (equal within 2 %): each SM stages half of B.
+bool gemm_tc_pair_preferred(const GemmArgs& g) { return gemm_tc_pair_supported(g); }
 
 cudaError_t gemm_tc_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;

@@ -133,7 +133,7 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 
     auto load_stage = [&](const Item& t, int kb, uint32_t it) {
         const int s = it % STAGES;
-        mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, dead, p.status);
+        mbar_wait_lean(&empty_bar[s], ((it / STAGES) & 1) ^ 1, dead, p.status);
         if (leader) mbar_expect_tx(&full_bar[s], 2 * (A_BYTES + B_BYTES));
         const uint32_t bar = map_to_cta(&full_bar[s], 0);
         const int k0 = t.k_row0 + kb * BK;
@@ -204,37 +204,31 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (leader) {
+        // ------------------------------------------------------------------ MMA issuer (one thread of the leader CTA)
+        if (leader && lane == 0) {
             constexpr uint32_t idesc = instr_desc_pair(BN, true, true);
-            uint32_t it = 0;
+            const uint64_t da0 = smem_desc(smem_u32(smem_a), CHUNK_BYTES, 1024), db0 = smem_desc(smem_u32(smem_b), CHUNK_BYTES, 1024);
+            constexpr uint32_t kStep = (UMMA_K * 128) >> 4;
+            uint32_t stage = 0, phase = 0;
             for (uint32_t local = 0;; ++local) {
                 const uint32_t acc = local & 1;
                 mbar_wait_cluster(&ring_bar[local % kRing], (local / kRing) & 1, dead, p.status);
                 const int num_kb = ring[local % kRing].num_kb;
                 if (num_kb < 0 || *dead) break;
-                mbar_wait(&tmem_empty_bar[acc], ((local >> 1) & 1) ^ 1, dead, p.status);
+                mbar_wait_lean(&tmem_empty_bar[acc], ((local >> 1) & 1) ^ 1, dead, p.status);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    mbar_wait(&full_bar[s], (it / STAGES) & 1, dead, p.status);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    mbar_wait_lean(&full_bar[stage], phase, dead, p.status);
                     tc_fence_after();
-                    if (lane == 0) {
-                        const uint32_t a_addr = smem_u32(smem_a + s * A_BYTES);
-                        const uint32_t b_addr = smem_u32(smem_b + s * B_BYTES);
+                    const uint64_t da = da0 + stage * (A_BYTES >> 4), db = db0 + stage * (B_BYTES >> 4);
+                    umma_bf16_pair(d_tmem, da, db, idesc, kb != 0);
 #pragma unroll
-                        for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-                            const uint64_t da = smem_desc(a_addr + kk * UMMA_K * 128, CHUNK_BYTES, 1024);
-                            const uint64_t db = smem_desc(b_addr + kk * UMMA_K * 128, CHUNK_BYTES, 1024);
-                            umma_bf16_pair(d_tmem, da, db, idesc, (kb | kk) != 0);
-                        }
-                        umma_commit_pair(&empty_bar[s]);
-                    }
-                    __syncwarp();
+                    for (int kk = 1; kk < BK / UMMA_K; ++kk) umma_bf16_pair(d_tmem, da + kk * kStep, db + kk * kStep, idesc, 1);
+                    umma_commit_pair(&empty_bar[stage]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (lane == 0) umma_commit_pair(&tmem_full_bar[acc]);
-                __syncwarp();
+                umma_commit_pair(&tmem_full_bar[acc]);
             }
         }
     } else {
