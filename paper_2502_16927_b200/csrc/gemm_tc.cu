@@ -162,7 +162,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int t = blockIdx.x; t < total; t += gridDim.x, ++local) {
             const Tile tl = get_tile(p, BN, t, tiles_m, tiles_n);
             const uint32_t acc = local & 1;
-            mbar_wait(&tmem_full_bar[acc], (local >> 1) & 1, dead, p.status);
+            mbar_wait_lean(&tmem_full_bar[acc], (local >> 1) & 1, dead, p.status);
             tc_fence_after();
             const int row = tl.m0 + quad * 32 + lane;
             const bool row_ok = row < tl.m_limit;
@@ -190,7 +190,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     __syncwarp();
                     if (z_prefetch) {
                         if (c == 0) {
-                            mbar_wait(my_z_bar, z_count & 1, dead, p.status);
+                            mbar_wait_lean(my_z_bar, z_count & 1, dead, p.status);
                             ++z_count;
                         }
                         uint32_t w[8];

@@ -279,7 +279,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             walk_next(tw, num_clusters, step_pair, step_n, tiles_n);            // tw / nxt now describe the next item
             if (tw.w < total) nxt = walk_tile(p, BN, tw, pairs_m, tiles_n, s_pp);
             const uint32_t acc = local & 1;
-            mbar_wait(&tmem_full_bar[acc], (local >> 1) & 1, dead, p.status);
+            mbar_wait_lean(&tmem_full_bar[acc], (local >> 1) & 1, dead, p.status);
             tc_fence_after();
             const int my_m0 = tl.m0 + (int)rank * BM;
             const int row = my_m0 + quad * 32 + lane;
@@ -309,7 +309,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     __syncwarp();
                     if (z_prefetch) {
                         if (c == 0) {
-                            mbar_wait(my_z_bar, z_count & 1, dead, p.status);
+                            mbar_wait_lean(my_z_bar, z_count & 1, dead, p.status);
                             ++z_count;
                         }
                         uint32_t wz[8];

@@ -244,7 +244,7 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             mbar_wait_cluster(&ring_bar[local % kRing], (local / kRing) & 1, dead, p.status);
             const Item t = ring[local % kRing];
             if (t.num_kb < 0 || *dead) break;
-            mbar_wait(&tmem_full_bar[acc], (local >> 1) & 1, dead, p.status);
+            mbar_wait_lean(&tmem_full_bar[acc], (local >> 1) & 1, dead, p.status);
             tc_fence_after();
             const int row = t.m0 + (int)rank * BM + quad * 32 + lane;
             const bool row_ok = row < p.M;
