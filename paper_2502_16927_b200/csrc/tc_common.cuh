@@ -321,12 +321,18 @@ __device__ __forceinline__ float sig_dequant(uint32_t word) {     // byte I of w
     return (__uint_as_float(bits) - kSigMagic) * kSigStep;
 }
 __device__ __forceinline__ float sig_dequant1(uint8_t q) { return ((float)q - 27.0f) * kSigStep; }
-// v[0..31] *= sigma' from 8 words of 4 bytes
+// v[0..31] *= sigma' from 8 words of 4 bytes: byte -> float bits by a permute, then (f - magic) (exact), * step and
+// the product with v as packed pairs (two elements per issued instruction).
 __device__ __forceinline__ void mul_by_sig32(float* v, const uint32_t* w) {
+    const f32x2_t step = pk2(kSigStep, kSigStep), neg_magic = pk2(-kSigMagic, -kSigMagic);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        v[4 * i] *= sig_dequant<0>(w[i]); v[4 * i + 1] *= sig_dequant<1>(w[i]);
-        v[4 * i + 2] *= sig_dequant<2>(w[i]); v[4 * i + 3] *= sig_dequant<3>(w[i]);
+        const uint32_t b0 = __byte_perm(w[i], 0x4B000000u, 0x7650), b1 = __byte_perm(w[i], 0x4B000000u, 0x7651);
+        const uint32_t b2 = __byte_perm(w[i], 0x4B000000u, 0x7652), b3 = __byte_perm(w[i], 0x4B000000u, 0x7653);
+        const f32x2_t s01 = mul2(add2(pk2(__uint_as_float(b0), __uint_as_float(b1)), neg_magic), step);
+        const f32x2_t s23 = mul2(add2(pk2(__uint_as_float(b2), __uint_as_float(b3)), neg_magic), step);
+        upk2(mul2(pk2(v[4 * i], v[4 * i + 1]), s01), v[4 * i], v[4 * i + 1]);
+        upk2(mul2(pk2(v[4 * i + 2], v[4 * i + 3]), s23), v[4 * i + 2], v[4 * i + 3]);
     }
 }
 
