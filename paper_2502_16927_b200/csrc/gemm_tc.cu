@@ -157,10 +157,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tma_load_2d(box_z, &map_z, my_z_bar, tile.n0 + part * COLS_PER_WARP, tile.m0 + quad * 32);
             }
         };
-        if (z_prefetch && (int)blockIdx.x < total) issue_z(get_tile(p, BN, blockIdx.x, tiles_m, tiles_n));
         uint32_t local = 0;
-        for (int t = blockIdx.x; t < total; t += gridDim.x, ++local) {
-            const Tile tl = get_tile(p, BN, t, tiles_m, tiles_n);
+        const int step_m = (int)gridDim.x / tiles_n, step_n = (int)gridDim.x - step_m * tiles_n;
+        TileWalk1 tw;
+        walk1_init(tw, blockIdx.x, tiles_n);
+        Tile nxt = tw.t < total ? walk1_tile(p, BN, tw, tiles_m, tiles_n) : Tile{};
+        if (z_prefetch && tw.t < total) issue_z(nxt);
+        for (; tw.t < total; ++local) {
+            const Tile tl = nxt;
+            const int t = tw.t;
+            walk1_next(tw, gridDim.x, step_m, step_n, tiles_n);                   // tw / nxt now describe the next tile
+            if (tw.t < total) nxt = walk1_tile(p, BN, tw, tiles_m, tiles_n);
             const uint32_t acc = local & 1;
             mbar_wait_lean(&tmem_full_bar[acc], (local >> 1) & 1, dead, p.status);
             tc_fence_after();
@@ -198,7 +205,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         if (c == CHUNKS - 1) {             // box read by every lane: fetch the next tile's
                             fence_async_smem();
                             __syncwarp();
-                            if (t + (int)gridDim.x < total) issue_z(get_tile(p, BN, t + gridDim.x, tiles_m, tiles_n));
+                            if (t + (int)gridDim.x < total) issue_z(nxt);
                         }
                         mul_by_sig32(v, w);
                     }

@@ -425,8 +425,12 @@ bool gemm_tc_pair_supported(const GemmArgs& g) {
 }
 
 // Measured on B200 (interleaved A/B at the large workload's shapes, after the MMA-issue thread was made lean): pairs
-// are 3-20 % faster on every shape but the training expert GEMM1 (equal within 2 %): each SM stages half of B.
-bool gemm_tc_pair_preferred(const GemmArgs& g) { return gemm_tc_pair_supported(g); }
+// are 3-20 % faster on every shape (each SM stages half of B) but one: the training expert GEMM1, whose epilogue
+// (activation, sigma' quantisation, two output streams) keeps the issue slots so busy that one MMA-issuing thread per
+// SM instead of one per pair is worth 2.5 % (0.615-0.626 vs 0.633-0.642 ms in three interleaved runs).
+bool gemm_tc_pair_preferred(const GemmArgs& g) {
+    return gemm_tc_pair_supported(g) && !(g.epilogue == EPI_ACT && g.Z != nullptr);
+}
 
 cudaError_t gemm_tc_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;

@@ -299,7 +299,9 @@ __device__ __forceinline__ void gelu_pair2(float z0, float z1, float& a0, float&
     float p0, p1;
     upk2(P, p0, p1);
     const f32x2_t cdf = pk2(fma_sat(z0, p0, 0.5f), fma_sat(z1, p1, 0.5f));
-    const f32x2_t e = pk2(fast_ex2(w0 * -0.72134752f), fast_ex2(w1 * -0.72134752f));     // exp(-z^2 / 2)
+    float x0, x1;
+    upk2(mul2(w, pk2(-0.72134752f, -0.72134752f)), x0, x1);
+    const f32x2_t e = pk2(fast_ex2(x0), fast_ex2(x1));                                   // exp(-z^2 / 2)
     upk2(mul2(z, cdf), a0, a1);
     upk2(fma2(mul2(z, e), pk2(0.39894228f, 0.39894228f), cdf), g0, g1);
 }
@@ -310,8 +312,11 @@ __device__ __forceinline__ void gelu_pair2(float z0, float z1, float& a0, float&
 // Rounding uses the 2^23 trick: the low byte of float(2^23 + 27 + 200 g) is q.
 constexpr float kSigScale = 200.0f, kSigMagic = 8388608.0f + 27.0f, kSigStep = 0.005f;
 __device__ __forceinline__ uint32_t sig_quant4(float g0, float g1, float g2, float g3) {
-    const uint32_t b0 = __float_as_uint(fmaf(g0, kSigScale, kSigMagic)), b1 = __float_as_uint(fmaf(g1, kSigScale, kSigMagic));
-    const uint32_t b2 = __float_as_uint(fmaf(g2, kSigScale, kSigMagic)), b3 = __float_as_uint(fmaf(g3, kSigScale, kSigMagic));
+    const f32x2_t scale = pk2(kSigScale, kSigScale), magic = pk2(kSigMagic, kSigMagic);
+    float f0, f1, f2, f3;
+    upk2(fma2(pk2(g0, g1), scale, magic), f0, f1);
+    upk2(fma2(pk2(g2, g3), scale, magic), f2, f3);
+    const uint32_t b0 = __float_as_uint(f0), b1 = __float_as_uint(f1), b2 = __float_as_uint(f2), b3 = __float_as_uint(f3);
     return __byte_perm(__byte_perm(b0, b1, 0x0040), __byte_perm(b2, b3, 0x0040), 0x5410);
 }
 __device__ __forceinline__ uint8_t sig_quant1(float g) { return (uint8_t)(__float_as_uint(fmaf(g, kSigScale, kSigMagic)) & 0xffu); }
@@ -520,6 +525,36 @@ __device__ __forceinline__ Tile get_tile(const TcParams& p, int BN, int t, int t
         tl.num_kb = (p.poffsets[e + 1] - tl.k_row0) / BK;
         tl.c_base = (int64_t)e * p.c_stride;
     }
+    return tl;
+}
+
+// The same for the epilogue warps of the one-CTA kernel, which walk t = first, first + stride, ...: for dense and
+// row-grouped problems (row tile, column tile) are carried along (no divisions per tile) and the tile -> expert
+// table is not read (only the loads need the expert; the outputs of a row-grouped problem are addressed by row).
+struct TileWalk1 {
+    int t, mt, nt;
+};
+__device__ __forceinline__ void walk1_init(TileWalk1& w, int first, int tiles_n) {
+    w.t = first;
+    w.mt = first / tiles_n;
+    w.nt = first - w.mt * tiles_n;
+}
+__device__ __forceinline__ void walk1_next(TileWalk1& w, int stride, int step_m, int step_n, int tiles_n) {
+    w.t += stride;
+    w.mt += step_m;
+    w.nt += step_n;
+    if (w.nt >= tiles_n) { w.nt -= tiles_n; ++w.mt; }
+}
+__device__ __forceinline__ Tile walk1_tile(const TcParams& p, int BN, const TileWalk1& w, int tiles_m, int tiles_n) {
+    if (p.group == GROUP_K || p.split_k > 1) return get_tile(p, BN, w.t, tiles_m, tiles_n);
+    Tile tl;
+    tl.m0 = w.mt * BM;
+    tl.n0 = w.nt * BN;
+    tl.expert = 0;
+    tl.k_row0 = 0;
+    tl.num_kb = (p.K + BK - 1) / BK;
+    tl.m_limit = p.group == GROUP_M ? min(p.M, tiles_m * kPad) : p.M;
+    tl.c_base = 0;
     return tl;
 }
 
