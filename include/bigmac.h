@@ -83,12 +83,28 @@ typedef enum {
  * used when there is enough work per SM pair for it to pay, else the statically scheduled one. */
 #define BIGMAC_FLAG_DYNAMIC_WGRAD 4u
 
+/* The two training-recipe settings of the paper's pre-training configuration (Table 5: capacity factor 1.2,
+ * load-balancing loss with coefficient 0.001).  Both are off (0) in the layer the paper advocates and measures,
+ * which is dropless; the paper prints no formula for either, so the conventional ones are used:
+ *
+ *  capacity_factor f > 0: an expert keeps at most C = ceil(f * T * k / E) rows per call; of the slots that chose
+ *    it, the first C in slot order (token ascending, then choice) are kept, the others are dropped.  A dropped
+ *    slot contributes nothing to y' (its gate value is NOT redistributed: the p of a token are still the softmax
+ *    over its k chosen logits) and receives no gradient.  Conventional implementations pad every expert to C rows;
+ *    here segments stay as long as the kept rows, which gives the same result.
+ *
+ *  aux_loss_coef alpha > 0: L_aux = alpha * E * sum_e f_e P_e, with f_e = (slots that chose e, before dropping)
+ *    / (T k) and P_e the mean over tokens of the softmax of the gate logits over ALL E experts.  The forward
+ *    writes L_aux; the backward adds dL_aux/dl (through P only; f is piecewise constant) to the gate gradient,
+ *    i.e. it returns the gradients of  sum(y * dy) + L_aux. */
 typedef struct {
     int32_t d, r, h, E, k; /* 1 <= k <= E */
     int32_t max_tokens;    /* largest T any call will pass */
     int32_t dtype;         /* bigmac_dtype_t */
     int32_t act;           /* bigmac_act_t */
     uint32_t flags;
+    double capacity_factor; /* 0 = dropless (Eq. 2 as written); else > 0; C = ceil((f * (T k)) / E) in double */
+    double aux_loss_coef;   /* 0 = no load-balancing loss; else > 0 */
 } bigmac_config_t;
 
 typedef struct {
@@ -113,19 +129,26 @@ typedef struct {
  *   counts[e]      rows routed to expert e;  offsets = exclusive prefix sum, offsets[E] = T*k
  *   row_of_slot[s] = offsets[e] + #{s' < s : topk_idx[s'] = e}  (stable counting sort by expert)
  *   slot_of_row    its inverse
+ * With a capacity factor: counts[e] = kept rows = min(chosen, C), offsets[E] = all kept rows, row_of_slot[s] = -1
+ * for a dropped slot, slot_of_row[row] = -1 for row >= offsets[E]; counts_chosen[e] = slots that chose e before
+ * dropping (equal to counts without a capacity factor).
+ *   aux_loss[0]    L_aux of this batch (fp32; 0 when aux_loss_coef = 0)
  * Any member may be NULL if the caller does not want that table. */
 typedef struct {
-    int32_t *topk_idx;    /* [T*k] */
-    float *topk_w;        /* [T*k] */
-    int32_t *counts;      /* [E]   */
-    int32_t *offsets;     /* [E+1] */
-    int32_t *row_of_slot; /* [T*k] */
-    int32_t *slot_of_row; /* [T*k] */
+    int32_t *topk_idx;      /* [T*k] */
+    float *topk_w;          /* [T*k] */
+    int32_t *counts;        /* [E]   */
+    int32_t *offsets;       /* [E+1] */
+    int32_t *row_of_slot;   /* [T*k] */
+    int32_t *slot_of_row;   /* [T*k] */
+    int32_t *counts_chosen; /* [E]   */
+    float *aux_loss;        /* [1]   */
 } bigmac_routing_t;
 
 /* Validate the configuration and create a handle on the current CUDA device.  Allocates one small
  * device status word; no other device memory is owned by the handle.
- * Errors: INVALID_ARG (null pointers, non-positive sizes, k > E, unknown enums), UNSUPPORTED (BF16
+ * Errors: INVALID_ARG (null pointers, non-positive sizes, k > E, unknown enums, a negative or non-finite
+ * capacity_factor or aux_loss_coef), UNSUPPORTED (BF16
  * with d, r or h not a multiple of 64; E > 1024), CUDA. */
 int bigmac_layer_create(const bigmac_config_t *cfg, bigmac_layer_t **out);
 int bigmac_layer_destroy(bigmac_layer_t *L);

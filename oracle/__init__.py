@@ -42,8 +42,10 @@ class Routing:
     topk_p: np.ndarray        # [T,k] f64, softmax over the k selected logits
     counts: np.ndarray        # [E]   int32
     offsets: np.ndarray       # [E+1] int32, exclusive prefix sum of counts
-    row_of_slot: np.ndarray   # [T*k] int32
-    slot_of_row: np.ndarray   # [T*k] int32
+    row_of_slot: np.ndarray   # [T*k] int32 (-1: dropped under a capacity limit)
+    slot_of_row: np.ndarray   # [T*k] int32 (-1 past the kept rows)
+    keep: Optional[np.ndarray] = None            # [T*k] uint8, None = dropless
+    counts_chosen: Optional[np.ndarray] = None   # [E] int32: slots that chose e, before dropping
 
 
 def gate_logits(x, w_gate, b_gate=None) -> np.ndarray:
@@ -78,11 +80,46 @@ def tables(topk_idx: np.ndarray, E: int):
     return counts, offsets, row_of_slot, slot_of_row
 
 
-def route(inp: Dict[str, np.ndarray], k: int) -> Routing:
+def capacity_rows(T: int, k: int, E: int, capacity_factor: float) -> int:
+    """C = ceil(f T k / E) rows per expert (Table 5's capacity factor f), evaluated in double as (f * (T k)) / E."""
+    return int(np.ceil(float(capacity_factor) * float(T * k) / float(E)))
+
+
+def tables_capacity(topk_idx: np.ndarray, E: int, cap: int):
+    topk_idx = np.ascontiguousarray(topk_idx, dtype=np.int32)
+    T, k = topk_idx.shape
+    chosen = np.empty(E, dtype=np.int32)
+    counts = np.empty(E, dtype=np.int32)
+    offsets = np.empty(E + 1, dtype=np.int32)
+    row_of_slot = np.empty(T * k, dtype=np.int32)
+    slot_of_row = np.empty(T * k, dtype=np.int32)
+    keep = np.empty(T * k, dtype=np.uint8)
+    lib().oracle_tables_capacity(_p(topk_idx), C.c_int(T), C.c_int(k), C.c_int(E), C.c_int(cap), _p(chosen),
+                                 _p(counts), _p(offsets), _p(row_of_slot), _p(slot_of_row), _p(keep))
+    return chosen, counts, offsets, row_of_slot, slot_of_row, keep
+
+
+def aux_loss(logits: np.ndarray, topk_idx: np.ndarray, alpha: float, want_grad: bool = True):
+    """Load-balancing loss L_aux (Table 5, coefficient alpha) and dL_aux/dlogits [T,E]."""
+    logits = np.ascontiguousarray(logits, dtype=np.float64)
+    topk_idx = np.ascontiguousarray(topk_idx, dtype=np.int32)
+    T, E = logits.shape
+    loss = C.c_double(0.0)
+    grad = np.empty((T, E), dtype=np.float64) if want_grad else None
+    lib().oracle_aux_loss(_p(logits), _p(topk_idx), C.c_int(T), C.c_int(E), C.c_int(topk_idx.shape[1]),
+                          C.c_double(alpha), C.byref(loss), _p(grad))
+    return loss.value, grad
+
+
+def route(inp: Dict[str, np.ndarray], k: int, capacity_factor: float = 0.0) -> Routing:
     logits = gate_logits(inp["x"], inp["w_gate"], inp.get("b_gate"))
     idx, p = topk(logits, k)
-    counts, offsets, ros, sor = tables(idx, logits.shape[1])
-    return Routing(logits, idx, p, counts, offsets, ros, sor)
+    T, E = logits.shape
+    if capacity_factor > 0:
+        chosen, counts, offsets, ros, sor, keep = tables_capacity(idx, E, capacity_rows(T, k, E, capacity_factor))
+        return Routing(logits, idx, p, counts, offsets, ros, sor, keep, chosen)
+    counts, offsets, ros, sor = tables(idx, E)
+    return Routing(logits, idx, p, counts, offsets, ros, sor, None, counts.copy())
 
 
 def _dims(inp):
@@ -110,7 +147,8 @@ def forward_tokens(inp, routing: Routing, act: int, tokens=None, want_slots: boo
     lib().oracle_forward_tokens(_p(_f32(inp["x"])), _p(_f32(inp["w_down"])), _p(_f32(inp["w1"])),
                                 _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])), _p(routing.topk_idx),
                                 _p(routing.topk_p), _p(tok), C.c_int(n), C.c_int(d), C.c_int(r), C.c_int(h),
-                                C.c_int(E), C.c_int(k), C.c_int(act), _p(x_lo), _p(y_lo), _p(y), _p(z), _p(u))
+                                C.c_int(E), C.c_int(k), C.c_int(act), _p(x_lo), _p(y_lo), _p(y), _p(z), _p(u),
+                                _p(routing.keep))
     out = {"x_lo": x_lo, "y_lo": y_lo, "y": y}
     if want_slots:
         out["z"], out["u"] = z, u
@@ -143,7 +181,8 @@ def backward_tokens(inp, routing: Routing, act: int, tokens=None, decide_bf16: b
                                  _p(_f32(inp["w_down"])), _p(_f32(inp["w1"])), _p(_f32(inp["w2"])),
                                  _p(_f32(inp["w_up"])), _p(routing.topk_idx), _p(routing.topk_p), _p(tok),
                                  C.c_int(n), C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(E), C.c_int(k),
-                                 C.c_int(act), C.c_int(int(decide_bf16)), _p(dx), _p(dx_lo), _p(dlogit), _p(dy_lo))
+                                 C.c_int(act), C.c_int(int(decide_bf16)), _p(dx), _p(dx_lo), _p(dlogit), _p(dy_lo),
+                                 _p(routing.keep))
     return {"dx": dx, "dx_lo": dx_lo, "dlogit": dlogit, "dy_lo": dy_lo}
 
 
@@ -160,8 +199,11 @@ def backward_expert(inp, routing: Routing, act: int, e: int, decide_bf16: bool =
     return dw1, dw2
 
 
-def backward_full(inp, routing: Routing, act: int, experts=None, decide_bf16: bool = False):
-    """All gradients: dx and every weight gradient (dw1/dw2 for `experts`, default all)."""
+def backward_full(inp, routing: Routing, act: int, experts=None, decide_bf16: bool = False, aux_alpha: float = 0.0):
+    """All gradients: dx and every weight gradient (dw1/dw2 for `experts`, default all).
+
+    aux_alpha > 0: gradients of sum(y*dy) + L_aux; the dense gate gradient dL_aux/dl [T,E] reaches dx, dw_gate and
+    db_gate through the linear gate (three matrix products with it)."""
     T, d, r, h, E = _dims(inp)
     k = routing.topk_idx.shape[1]
     fwd = forward_tokens(inp, routing, act)
@@ -186,6 +228,14 @@ def backward_full(inp, routing: Routing, act: int, experts=None, decide_bf16: bo
     out = {"y": fwd["y"], "y_lo": fwd["y_lo"], "x_lo": fwd["x_lo"], "dx": bwd["dx"], "dx_lo": bwd["dx_lo"],
            "dlogit": bwd["dlogit"], "dw_up": dw_up, "dw_down": dw_down, "dw_gate": dw_gate,
            "db_gate": db_gate, "dw1": dw1, "dw2": dw2}
+    if aux_alpha > 0:
+        loss, dl_aux = aux_loss(routing.logits, routing.topk_idx, aux_alpha)
+        x64 = np.asarray(inp["x"], dtype=np.float64)
+        out["aux_loss"] = loss
+        out["dlogit_aux"] = dl_aux
+        out["dx"] = out["dx"] + dl_aux @ np.asarray(inp["w_gate"], dtype=np.float64)    # l = x W_g^T + b_g
+        out["dw_gate"] = dw_gate + dl_aux.T @ x64
+        out["db_gate"] = db_gate + dl_aux.sum(axis=0)
     return out
 
 

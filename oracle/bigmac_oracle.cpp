@@ -17,6 +17,14 @@
 // dropless routing; no biases except the optional gate bias; rows of an expert's segment in
 // ascending slot id (slot s = t*k + j).
 //
+// Training-recipe variants of the pre-training configuration (Table 5: capacity factor 1.2, load-balancing loss
+// with coefficient 0.001), for which the paper prints no formula; the conventional ones are taken:
+//   capacity: an expert keeps the first C = ceil(f T k / E) of the slots that chose it, in slot order; a dropped
+//   slot adds nothing to y' (gate values are not renormalised) and receives no gradient;
+//   load-balancing loss: L_aux = alpha E sum_e f_e P_e, f_e = slots that chose e / (T k) (before dropping),
+//   P_e = mean over tokens of the softmax of the logits over all E experts; gradient through P only.
+// `keep` arguments below are per-slot bytes (1 = kept, 0 = dropped), NULL = every slot kept (dropless).
+//
 // Inputs are float arrays holding values exactly representable in the workload dtype; they are
 // widened to double before any arithmetic and nothing is rounded afterwards.
 //
@@ -24,7 +32,10 @@
 // softmax, tables against a library stable argsort and a brute-force count, E=1/k=1 and
 // shared-expert special cases against a 4-matmul MLP, identity-expert case against the two
 // projections alone, per-token against grouped evaluation, gradients against central finite
-// differences and the adjoint identity.  Float values of y and of the gradients on random data
+// differences and the adjoint identity; capacity tables against a brute-force per-expert list, the dropped
+// forward against the E=1, k=1 case (rows past C are zero, the others a plain MLP) and against the dropless
+// forward minus the dropped slots' terms, the load-balancing loss against its closed forms (equal logits: alpha;
+// collapse onto one expert: alpha E) and its gradient against central differences.  Float values of y and of the gradients on random data
 // have no printed example in the paper: "parity unpinned" by the paper for those, pinned only by
 // the special cases above.
 #include <algorithm>
@@ -181,12 +192,75 @@ void oracle_tables(const int32_t* topk_idx, int T, int k, int E, int32_t* counts
     }
 }
 
+// Dispatch layout under a capacity of `cap` rows per expert (Table 5's capacity factor; cap = ceil(f T k / E) is
+// computed by the caller): the stable counting sort above, except that a slot whose rank among the slots of its
+// expert is >= cap is dropped: keep[s] = 0, row_of_slot[s] = -1.  counts / offsets describe the kept rows,
+// counts_chosen the slots before dropping; slot_of_row[row] = -1 for row >= offsets[E].
+void oracle_tables_capacity(const int32_t* topk_idx, int T, int k, int E, int cap, int32_t* counts_chosen,
+                            int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row,
+                            uint8_t* keep) {
+    const int64_t N = (int64_t)T * k;
+    for (int e = 0; e < E; ++e) counts_chosen[e] = 0;
+    for (int64_t s = 0; s < N; ++s) counts_chosen[topk_idx[s]] += 1;
+    offsets[0] = 0;
+    for (int e = 0; e < E; ++e) {
+        counts[e] = std::min(counts_chosen[e], cap);
+        offsets[e + 1] = offsets[e] + counts[e];
+    }
+    for (int64_t row = 0; row < N; ++row) slot_of_row[row] = -1;
+    std::vector<int32_t> seen(E, 0);
+    for (int64_t s = 0; s < N; ++s) {
+        const int e = topk_idx[s];
+        const int32_t rank = seen[e];
+        seen[e] += 1;
+        keep[s] = rank < cap ? 1 : 0;
+        if (keep[s]) {
+            row_of_slot[s] = offsets[e] + rank;
+            slot_of_row[offsets[e] + rank] = (int32_t)s;
+        } else {
+            row_of_slot[s] = -1;
+        }
+    }
+}
+
+// Load-balancing loss (Table 5, coefficient alpha) and its gradient with respect to the gate logits:
+//   p[t,:] = softmax over all E of l[t,:] ;  P_e = (1/T) sum_t p[t,e] ;  f_e = #{slots with topk_idx = e} / (T k) ;
+//   L_aux = alpha E sum_e f_e P_e ;  dL/dl[t,e] = (alpha E / T) p[t,e] (f_e - sum_j f_j p[t,j])   (f held constant).
+// dlogits [T,E] may be NULL.
+void oracle_aux_loss(const double* logits, const int32_t* topk_idx, int T, int E, int k, double alpha,
+                     double* loss, double* dlogits) {
+    std::vector<double> f(E, 0.0), P(E, 0.0), p((size_t)T * E);
+    for (int64_t s = 0; s < (int64_t)T * k; ++s) f[topk_idx[s]] += 1.0;
+    for (int e = 0; e < E; ++e) f[e] /= (double)T * k;
+    for (int t = 0; t < T; ++t) {
+        const double* l = logits + (size_t)t * E;
+        double m = l[0], denom = 0.0;
+        for (int e = 1; e < E; ++e) m = std::max(m, l[e]);
+        for (int e = 0; e < E; ++e) denom += std::exp(l[e] - m);
+        for (int e = 0; e < E; ++e) {
+            p[(size_t)t * E + e] = std::exp(l[e] - m) / denom;
+            P[e] += p[(size_t)t * E + e] / T;
+        }
+    }
+    double acc = 0.0;
+    for (int e = 0; e < E; ++e) acc += f[e] * P[e];
+    *loss = alpha * E * acc;
+    if (!dlogits) return;
+    for (int t = 0; t < T; ++t) {
+        const double* pt = &p[(size_t)t * E];
+        double fp = 0.0;
+        for (int e = 0; e < E; ++e) fp += f[e] * pt[e];
+        for (int e = 0; e < E; ++e) dlogits[(size_t)t * E + e] = alpha * E / T * pt[e] * (f[e] - fp);
+    }
+}
+
 // Forward, token by token, exactly as Eq. 2 is written.  `tokens` selects n token ids (NULL = 0..n-1).
 // Outputs are indexed by position in `tokens`.  z_out / u_out may be NULL.
 void oracle_forward_tokens(const float* x, const float* w_down, const float* w1, const float* w2,
                            const float* w_up, const int32_t* topk_idx, const double* topk_p,
                            const int32_t* tokens, int n, int d, int r, int h, int E, int k, int act,
-                           double* x_lo_out, double* y_lo_out, double* y_out, double* z_out, double* u_out) {
+                           double* x_lo_out, double* y_lo_out, double* y_out, double* z_out, double* u_out,
+                           const uint8_t* keep) {
     (void)E;
 #pragma omp parallel for schedule(dynamic, 4)
     for (int i = 0; i < n; ++i) {
@@ -199,7 +273,8 @@ void oracle_forward_tokens(const float* x, const float* w_down, const float* w1,
             const double p = topk_p[(size_t)t * k + j];
             expert_forward(x_lo.data(), w1 + (size_t)e * h * r, w2 + (size_t)e * r * h, r, h, act,
                            z.data(), a.data(), u.data());
-            for (int c = 0; c < r; ++c) y_lo[c] += p * u[c];               // p_i(x) E_i(x')
+            if (!keep || keep[(size_t)t * k + j])
+                for (int c = 0; c < r; ++c) y_lo[c] += p * u[c];           // p_i(x) E_i(x'); nothing from a dropped slot
             if (z_out) std::memcpy(z_out + ((size_t)i * k + j) * h, z.data(), sizeof(double) * h);
             if (u_out) std::memcpy(u_out + ((size_t)i * k + j) * r, u.data(), sizeof(double) * r);
         }
@@ -224,7 +299,7 @@ void oracle_forward_grouped(const float* x, const float* w_down, const float* w1
         widen(x + (size_t)t * d, d, xt.data());
         matvec(xt.data(), w_down, r, d, &x_lo[(size_t)t * r]);
     }
-    for (int64_t row = 0; row < N; ++row) {                                 // dispatch
+    for (int64_t row = 0; row < offsets[E]; ++row) {                        // dispatch (offsets[E] = N when dropless)
         const int t = slot_of_row[row] / k;
         std::memcpy(&xg[(size_t)row * r], &x_lo[(size_t)t * r], sizeof(double) * r);
     }
@@ -241,6 +316,7 @@ void oracle_forward_grouped(const float* x, const float* w_down, const float* w1
         for (int j = 0; j < k; ++j) {
             const int64_t s = (int64_t)t * k + j;
             const double p = topk_p[s];
+            if (row_of_slot[s] < 0) continue;                               // dropped under a capacity limit
             const double* u = &ug[(size_t)row_of_slot[s] * r];
             for (int c = 0; c < r; ++c) y_lo[c] += p * u[c];
         }
@@ -260,7 +336,7 @@ void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate
                             const float* w1, const float* w2, const float* w_up, const int32_t* topk_idx,
                             const double* topk_p, const int32_t* tokens, int n, int d, int r, int h, int E,
                             int k, int act, int decide_bf16, double* dx_out, double* dx_lo_out,
-                            double* dlogit_out, double* dy_lo_out) {
+                            double* dlogit_out, double* dy_lo_out, const uint8_t* keep) {
     (void)E;
 #pragma omp parallel for schedule(dynamic, 4)
     for (int i = 0; i < n; ++i) {
@@ -276,6 +352,7 @@ void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate
             const double p = topk_p[(size_t)t * k + j];
             const float* w1_e = w1 + (size_t)e * h * r;
             const float* w2_e = w2 + (size_t)e * r * h;
+            if (keep && !keep[(size_t)t * k + j]) { dp[j] = 0.0; continue; }   // a dropped slot is absent from y'
             expert_forward(x_lo.data(), w1_e, w2_e, r, h, act, z.data(), a.data(), u.data());
             double acc = 0.0;
             for (int c = 0; c < r; ++c) acc += dy_lo[c] * u[c];

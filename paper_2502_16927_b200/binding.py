@@ -21,7 +21,8 @@ BIGMAC_FLAG_SIMT_GEMM = 1
 
 
 class bigmac_config_t(C.Structure):
-    _fields_ = [(n, C.c_int32) for n in ("d", "r", "h", "E", "k", "max_tokens", "dtype", "act")] + [("flags", C.c_uint32)]
+    _fields_ = ([(n, C.c_int32) for n in ("d", "r", "h", "E", "k", "max_tokens", "dtype", "act")] + [("flags", C.c_uint32)] +
+                [("capacity_factor", C.c_double), ("aux_loss_coef", C.c_double)])
 
 
 class bigmac_weights_t(C.Structure):
@@ -32,8 +33,11 @@ class bigmac_grads_t(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("dw_gate", "db_gate", "dw_down", "dw1", "dw2", "dw_up")]
 
 
+_ROUTING_FIELDS = ("topk_idx", "topk_w", "counts", "offsets", "row_of_slot", "slot_of_row", "counts_chosen", "aux_loss")
+
+
 class bigmac_routing_t(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("topk_idx", "topk_w", "counts", "offsets", "row_of_slot", "slot_of_row")]
+    _fields_ = [(n, C.c_void_p) for n in _ROUTING_FIELDS]
 
 
 class bigmac_debug_gemm_t(C.Structure):
@@ -114,8 +118,8 @@ def _stream() -> C.c_void_p:
 
 # ---- the C ABI, name for name -------------------------------------------------------------------------
 
-def bigmac_layer_create(d, r, h, E, k, max_tokens, dtype, act, flags=0) -> C.c_void_p:
-    cfg = bigmac_config_t(d, r, h, E, k, max_tokens, dtype, act, flags)
+def bigmac_layer_create(d, r, h, E, k, max_tokens, dtype, act, flags=0, capacity_factor=0.0, aux_loss_coef=0.0) -> C.c_void_p:
+    cfg = bigmac_config_t(d, r, h, E, k, max_tokens, dtype, act, flags, capacity_factor, aux_loss_coef)
     handle = C.c_void_p()
     _check(lib().bigmac_layer_create(C.byref(cfg), C.byref(handle)), "bigmac_layer_create")
     return handle
@@ -140,8 +144,7 @@ def _weights(W: Dict[str, torch.Tensor]) -> bigmac_weights_t:
 def _routing(R: Optional[Dict[str, torch.Tensor]]):
     if R is None:
         return None
-    return C.byref(bigmac_routing_t(*[_ptr(R.get(n)) for n in ("topk_idx", "topk_w", "counts", "offsets",
-                                                                  "row_of_slot", "slot_of_row")]))
+    return C.byref(bigmac_routing_t(*[_ptr(R.get(n)) for n in _ROUTING_FIELDS]))
 
 
 def bigmac_route(handle, x, T, W, routing, scratch) -> None:
@@ -202,11 +205,12 @@ def bigmac_debug_gemm(handle, q: bigmac_debug_gemm_t, use_tensor_cores) -> None:
 class Layer:
     """One BigMac layer handle plus torch-allocated workspaces.  Marshalling only."""
 
-    def __init__(self, d, r, h, E, k, max_tokens, dtype, act, flags=0, device="cuda"):
-        self.cfg = dict(d=d, r=r, h=h, E=E, k=k, max_tokens=max_tokens, dtype=dtype, act=act, flags=flags)
+    def __init__(self, d, r, h, E, k, max_tokens, dtype, act, flags=0, device="cuda", capacity_factor=0.0, aux_loss_coef=0.0):
+        self.cfg = dict(d=d, r=r, h=h, E=E, k=k, max_tokens=max_tokens, dtype=dtype, act=act, flags=flags,
+                        capacity_factor=capacity_factor, aux_loss_coef=aux_loss_coef)
         self.device = torch.device(device)
         with torch.cuda.device(self.device):
-            self.handle = bigmac_layer_create(d, r, h, E, k, max_tokens, dtype, act, flags)
+            self.handle = bigmac_layer_create(d, r, h, E, k, max_tokens, dtype, act, flags, capacity_factor, aux_loss_coef)
         self.tdtype = torch.bfloat16 if dtype == BIGMAC_BF16 else torch.float32
         self._scratch = None
         self._saved = None
@@ -235,7 +239,8 @@ class Layer:
         i32 = dict(dtype=torch.int32, device=self.device)
         return {"topk_idx": torch.empty(T * k, **i32), "topk_w": torch.empty(T * k, dtype=torch.float32, device=self.device),
                 "counts": torch.empty(E, **i32), "offsets": torch.empty(E + 1, **i32),
-                "row_of_slot": torch.empty(T * k, **i32), "slot_of_row": torch.empty(T * k, **i32)}
+                "row_of_slot": torch.empty(T * k, **i32), "slot_of_row": torch.empty(T * k, **i32),
+                "counts_chosen": torch.empty(E, **i32), "aux_loss": torch.empty(1, dtype=torch.float32, device=self.device)}
 
     def route(self, x, W):
         T = x.shape[0]

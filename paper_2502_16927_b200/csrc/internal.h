@@ -100,6 +100,7 @@ struct Tables {
     int32_t* tile_expert;   // [P/kPad]
     int32_t* n_tiles;       // [1]     number of kPad-row tiles in use
     int32_t* block_counts;  // [n_blocks, E] scratch of the counting sort
+    int32_t* counts_chosen; // [E]     slots that chose the expert, before any dropping (nullable)
 };
 
 // Per-device one-time launch configuration (function attributes are per device; a process may use several).
@@ -122,14 +123,18 @@ inline int sort_blocks(int64_t N) { return (int)((N + kSortChunk - 1) / kSortChu
 // logits [T,E] fp32 (+ b_gate) -> topk_idx, topk_w.
 cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, int k, int32_t* topk_idx,
                         float* topk_w, cudaStream_t stream);
-// topk_idx -> every other table (deterministic stable counting sort of slots by expert).
-cudaError_t launch_tables(const Tables& tb, int T, int E, int k, cudaStream_t stream);
+// topk_idx -> every other table (deterministic stable counting sort of slots by expert).  `cap`: rows an expert
+// keeps at most (the capacity of Table 5's capacity factor; kNoCapacity = dropless); a slot whose rank among the
+// slots of its expert is cap or more gets row_of_slot = prow_of_slot = -1, counts / offsets describe kept rows.
+constexpr int kNoCapacity = 0x7fffffff;
+cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaStream_t stream);
 
 // Row moves.  `width` elements of the dtype per row; all row pointers 16-byte aligned.
 // grouped[prow,:] = src[slot_of_prow[prow]/k,:], zeros on padding rows, for prow < n_tiles*kPad.
 cudaError_t launch_dispatch(const void* src, void* grouped, const Tables& tb, int k, int width, int dtype,
                             int64_t max_prows, cudaStream_t stream);
-// dst[t,:] = sum_j w[t*k+j] * grouped[prow_of_slot[t*k+j],:]   (w == nullptr: unit weights), fp32 accumulation.
+// dst[t,:] = sum_j w[t*k+j] * grouped[prow_of_slot[t*k+j],:]   (w == nullptr: unit weights), fp32 accumulation;
+// slots with prow_of_slot < 0 (dropped under a capacity limit) are left out of the sum.
 // dst rows are `dst_ld` elements apart (0: dense, = width).
 cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const int32_t* prow_of_slot, int T,
                            int k, int width, int dtype, cudaStream_t stream, int dst_ld = 0);
@@ -141,11 +146,22 @@ cudaError_t launch_combine_bwd(const void* dy_lo, const void* u, void* du, float
 // leaves the fp32 dl_j in dp[slot].
 cudaError_t launch_gate_bwd(float* dp, const Tables& tb, void* dlogits, int T, int E, int width, int ld, int k,
                             int dtype, cudaStream_t stream);
+// Load-balancing loss (Table 5; conventional form, the paper prints none):
+//   L_aux = coef * E * sum_e f_e P_e,  f_e = counts_chosen[e] / (T k),  P_e = mean_t softmax_E(logits[t,:] + b_gate)[e].
+// Forward: loss[0] = L_aux; `partial` holds kColsumChunks * E floats of scratch.  Deterministic summation order.
+cudaError_t launch_aux_loss(const float* logits, const float* b_gate, const int32_t* counts_chosen, int T, int E, int k,
+                            float coef, float* partial, float* loss, cudaStream_t stream);
+// launch_gate_bwd plus dL_aux/dl: dlogits[t,e] = (top-k part) + (coef E / T) p[t,e] (f_e - sum_j f_j p[t,j]); the
+// column sums of the second term go to aux_partial [kColsumChunks, E] for launch_gate_colsum.
+cudaError_t launch_gate_bwd_aux(float* dp, const Tables& tb, void* dlogits, const float* logits, const float* b_gate,
+                                float coef, float* aux_partial, int T, int E, int width, int ld, int k, int dtype,
+                                cudaStream_t stream);
 // db[e] (+)= sum over the slots routed to e of dl_slot[slot] (the fp32 per-slot gate gradients launch_gate_bwd
 // leaves in dp); `partial` holds kColsumChunks * E floats of scratch.  Deterministic summation order.
 constexpr int kColsumChunks = 296;
+// aux_partial (nullable): a second [kColsumChunks, E] array of partial column sums added in (launch_gate_bwd_aux).
 cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db, float* partial, int64_t N, int E,
-                               bool accumulate, cudaStream_t stream);
+                               bool accumulate, cudaStream_t stream, const float* aux_partial = nullptr);
 // Sum the `parts` fp32 partial results ws[s][m][n] of a split contraction in the order s = 0, 1, ... and write
 // rows [0, m_split) to dst1 [m_split, N] and rows [m_split, m_split + m2) to dst2 [m2, N] (dst2 may be null),
 // in the dtype, adding to the destination if `accumulate`.

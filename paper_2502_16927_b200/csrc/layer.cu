@@ -2,6 +2,7 @@
 // BigMac DCCA MoE layer (Eq. 2 / Eq. 4), forward and backward.  No device allocation, no stream
 // synchronisation and no host-visible data dependence inside route / forward / backward: segment sizes
 // stay on the device.
+#include <cmath>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -36,12 +37,12 @@ namespace {
 enum { G_LOGITS = 0, G_DESCEND, G_EXPERT1, G_EXPERT2, G_ASCEND, G_DY_LO, G_DW_UP, G_DZ, G_DW2, G_DXG, G_DW1,
        G_DX, G_DX_GATE, G_DW_DOWN, G_DW_GATE,
        S_TOPK, S_TABLES, S_DISPATCH, S_COMBINE, S_COMBINE_BWD, S_GATE_BWD, S_DXLO_GATHER, S_COLSUM, S_SPLITK_REDUCE,
-       S_DECODE, S_FUSED_MLP, S_COUNT };
+       S_DECODE, S_FUSED_MLP, S_AUX_LOSS, S_COUNT };
 const char* const kSlotNames[S_COUNT] = {
     "gemm_logits", "gemm_descend", "gemm_expert1", "gemm_expert2", "gemm_ascend", "gemm_dy_lo", "gemm_dw_up",
     "gemm_dz", "gemm_dw2", "gemm_dxg", "gemm_dw1", "gemm_dx", "gemm_dx_gate", "gemm_dw_down", "gemm_dw_gate",
     "topk", "tables", "dispatch", "combine", "combine_bwd", "gate_bwd", "dxlo_gather", "colsum",
-    "splitk_reduce", "decode_forward", "fused_expert_mlp"};
+    "splitk_reduce", "decode_forward", "fused_expert_mlp", "aux_loss"};
 constexpr size_t kEventPairs = 8192;
 constexpr int kMaxSplitK = 8;
 
@@ -89,7 +90,10 @@ struct Buffers {
     void* dz;            // [P,h]: its own buffer when sigma' is saved as bytes, else written over sigma'
     void* dcat;          // [T, r + E64]: dx' in columns [0, r), the dense gate gradient dl in columns [r, r + E64)
     void *dx_lo, *dlogits;                               // views into dcat (row stride r + E64)
-    float* colsum_part;  // [kColsumChunks, E]
+    float* colsum_part;  // [2, kColsumChunks, E]: partial column sums of the top-k part and of the load-balancing part
+    float* aux_part;     // [kColsumChunks, E] forward scratch of the load-balancing loss
+    float* aux_loss;     // [1] saved: L_aux of the batch
+    float* logits_saved; // [T,E] saved copy of the gate logits (only with a load-balancing loss)
     float* splitk_ws;    // fp32 partial results of the split weight-gradient contractions
 };
 
@@ -100,6 +104,8 @@ struct Dims {
     int z_es;  // bytes per saved sigma'(z) element: 1 on the tensor-core path (quantised), else the dtype's
     bool cdac; // Eq. 3 layer: no descend / ascend projections, r == d
     int ldcat; // row stride of dcat: r + E64, or E64 alone without projections (dx' then goes straight to dx)
+    int cap;   // rows an expert keeps at most (Table 5's capacity factor); kNoCapacity = dropless
+    float aux; // coefficient of the load-balancing loss (Table 5), 0 = none
 };
 
 // The tensor-core kernels save sigma' as one byte per element; that needs expert GEMM1 and dz on the same side.
@@ -113,6 +119,12 @@ Dims dims_of(const bigmac_layer* L, int T) {
     m.z_es = sigma_as_bytes(L) ? 1 : (int)esize(c.dtype);
     m.cdac = (c.flags & BIGMAC_FLAG_CDAC) != 0;
     m.ldcat = m.cdac ? m.E64 : m.r + m.E64;
+    m.cap = kNoCapacity;
+    if (c.capacity_factor > 0) {                     // C = ceil((f * (T k)) / E), evaluated in double in this order
+        const double rows = std::ceil(c.capacity_factor * (double)m.N / (double)c.E);
+        if (rows < (double)m.N) m.cap = (int)rows;
+    }
+    m.aux = (float)c.aux_loss_coef;
     return m;
 }
 
@@ -136,11 +148,15 @@ void carve_saved(Carver& cv, const Dims& m, Buffers& b, bool with_z) {
     b.a = cv.take_bytes((size_t)m.P * m.h * es);
     b.u = cv.take_bytes((size_t)m.P * m.r * es);
     b.y_lo = m.cdac ? nullptr : cv.take_bytes((size_t)m.T * m.r * es);     // ... and y' is y
+    b.tb.counts_chosen = cv.take<int32_t>(m.E);
+    b.aux_loss = cv.take<float>(1);
+    b.logits_saved = (with_z && m.aux > 0) ? cv.take<float>((size_t)m.T * m.E) : nullptr;
 }
 
 void carve_route_scratch(Carver& cv, const Dims& m, Buffers& b) {
     b.logits = cv.take<float>((size_t)m.T * m.E);
     b.tb.block_counts = cv.take<int32_t>((size_t)(sort_blocks(m.N) + 1) * m.E);
+    b.aux_part = m.aux > 0 ? cv.take<float>((size_t)kColsumChunks * m.E) : nullptr;
 }
 
 void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
@@ -153,7 +169,7 @@ void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
     b.dx_lo = m.cdac ? nullptr : b.dcat;
     b.dlogits = (b.dcat && !m.cdac) ? (char*)b.dcat + (size_t)m.r * es : b.dcat;
     b.dp = cv.take<float>(m.N);
-    b.colsum_part = cv.take<float>((size_t)kColsumChunks * m.E);
+    b.colsum_part = cv.take<float>((size_t)2 * kColsumChunks * m.E);
     // fp32 partial results: of the split dense contractions, and of the parts of long experts in dW1 / dW2
     const size_t dense_ws = (size_t)kMaxSplitK * m.ldcat * m.d * sizeof(float);
     const size_t expert_ws = m.dtype == BIGMAC_BF16 ? gemm_tc_groupk_ws_bytes(m.r, m.h, m.E) : 0;
@@ -229,6 +245,20 @@ int choose_split_k(int M, int N, int K) {
         if ((expr) != cudaSuccess) return BIGMAC_ERR_CUDA;  \
     } while (0)
 
+// Steps F2-F3 from the gate logits: top-k with softmax gate values, dispatch layout (under the capacity limit, if
+// any), load-balancing loss.
+int route_from_logits(const bigmac_layer* L, const Dims& m, const bigmac_weights_t* W, Buffers& b, cudaStream_t st) {
+    { Stage s(L, S_TOPK, st); BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st)); }
+    { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st)); }
+    if (m.aux > 0) {
+        Stage s(L, S_AUX_LOSS, st, 2);
+        BIGMAC_CUDA(launch_aux_loss(b.logits, W->b_gate, b.tb.counts_chosen, m.T, m.E, m.k, m.aux, b.aux_part, b.aux_loss, st));
+        if (b.logits_saved)
+            BIGMAC_CUDA(cudaMemcpyAsync(b.logits_saved, b.logits, sizeof(float) * (size_t)m.T * m.E, cudaMemcpyDeviceToDevice, st));
+    }
+    return BIGMAC_OK;
+}
+
 // Steps F1-F3: gate logits on x, top-k with softmax gate values, dispatch layout.
 int run_routing(const bigmac_layer* L, const Dims& m, const void* x, const bigmac_weights_t* W, Buffers& b,
                 cudaStream_t st) {
@@ -236,9 +266,7 @@ int run_routing(const bigmac_layer* L, const Dims& m, const void* x, const bigma
     g.A = x; g.lda = m.d; g.B = W->w_gate; g.ldb = m.d; g.C = b.logits; g.ldc = m.E;
     g.M = m.T; g.N = m.E; g.K = m.d; g.out_f32 = true;
     BIGMAC_TRY(gemm(L, G_LOGITS, g, st));
-    { Stage s(L, S_TOPK, st); BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st)); }
-    { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, st)); }
-    return BIGMAC_OK;
+    return route_from_logits(L, m, W, b, st);
 }
 
 int export_routing(const Dims& m, const Buffers& b, bigmac_routing_t* out, cudaStream_t st) {
@@ -252,6 +280,12 @@ int export_routing(const Dims& m, const Buffers& b, bigmac_routing_t* out, cudaS
         BIGMAC_CUDA(cudaMemcpyAsync(out->row_of_slot, b.tb.row_of_slot, sizeof(int32_t) * m.N, kind, st));
     if (out->slot_of_row)
         BIGMAC_CUDA(cudaMemcpyAsync(out->slot_of_row, b.tb.slot_of_row, sizeof(int32_t) * m.N, kind, st));
+    if (out->counts_chosen)
+        BIGMAC_CUDA(cudaMemcpyAsync(out->counts_chosen, b.tb.counts_chosen, sizeof(int32_t) * m.E, kind, st));
+    if (out->aux_loss) {
+        if (m.aux > 0) BIGMAC_CUDA(cudaMemcpyAsync(out->aux_loss, b.aux_loss, sizeof(float), kind, st));
+        else BIGMAC_CUDA(cudaMemsetAsync(out->aux_loss, 0, sizeof(float), st));
+    }
     return BIGMAC_OK;
 }
 
@@ -296,6 +330,9 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
     if (cfg->act < BIGMAC_ACT_RELU || cfg->act > BIGMAC_ACT_IDENTITY) return BIGMAC_ERR_INVALID_ARG;
     if (cfg->flags & ~(BIGMAC_FLAG_SIMT_GEMM | BIGMAC_FLAG_CDAC | BIGMAC_FLAG_DYNAMIC_WGRAD)) return BIGMAC_ERR_INVALID_ARG;
     if ((cfg->flags & BIGMAC_FLAG_CDAC) && cfg->r != cfg->d) return BIGMAC_ERR_INVALID_ARG;
+    if (!(cfg->capacity_factor >= 0) || !(cfg->aux_loss_coef >= 0) || std::isinf(cfg->capacity_factor) ||
+        std::isinf(cfg->aux_loss_coef))
+        return BIGMAC_ERR_INVALID_ARG;
     if (cfg->E > kMaxExperts) return BIGMAC_ERR_UNSUPPORTED;
     if ((int64_t)cfg->max_tokens * cfg->k > (int64_t)1 << 30) return BIGMAC_ERR_UNSUPPORTED;
     const int vec = cfg->dtype == BIGMAC_BF16 ? 8 : 4;     // rows move as 16-byte vectors
@@ -385,7 +422,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     const bigmac_config_t& c = L->cfg;
 
     // A few tokens, inference: the whole forward in one cooperative kernel (weight streaming, no tensor cores)
-    if (!training && !m.cdac && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
+    if (!training && !m.cdac && m.cap == kNoCapacity && m.aux == 0 && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
         {
             Stage s(L, S_DECODE, st);
             BIGMAC_CUDA(launch_decode_forward(x, W, y, b.logits, (float*)b.xg, (float*)b.a, (float*)b.u, b.tb.topk_idx,
@@ -393,7 +430,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
                                               m.k, c.act, gemm_tc_sm_count(), st));
         }
         if (routing_out) {
-            { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, st)); }
+            { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st)); }
             BIGMAC_TRY(export_routing(m, b, routing_out, st));
         }
         return BIGMAC_OK;
@@ -407,8 +444,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         g.B2 = W->w_gate; g.ldb2 = m.d; g.n_split = m.r; g.C2 = b.logits; g.ldc2 = m.E; g.N2 = m.E;
         g.M = m.T; g.N = m.r + m.E; g.K = m.d;
         BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
-        { Stage s(L, S_TOPK, st); BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st)); }
-        { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, st)); }
+        BIGMAC_TRY(route_from_logits(L, m, W, b, st));
     } else {
         BIGMAC_TRY(run_routing(L, m, x, W, b, st));                               // F1-F3
     }
@@ -509,8 +545,18 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         }
     }
     // du = p dy'[t], dp = <dy'[t], u>; then the softmax-over-k backward
+    if (m.cap != kNoCapacity) BIGMAC_CUDA(cudaMemsetAsync(b.dp, 0, sizeof(float) * m.N, st));   // dropped slots: dp = 0
     { Stage s(L, S_COMBINE_BWD, st); BIGMAC_CUDA(launch_combine_bwd(b.dy_lo, b.u, b.du, b.dp, b.tb, m.k, m.r, m.dtype, m.P, st)); }
-    { Stage s(L, S_GATE_BWD, st); BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, ldcat, m.k, m.dtype, st)); }
+    float* aux_part = nullptr;                                                    // column sums of dL_aux/dl, for db_gate
+    if (m.aux > 0) {
+        aux_part = b.colsum_part + (size_t)kColsumChunks * m.E;
+        Stage s(L, S_GATE_BWD, st);
+        BIGMAC_CUDA(launch_gate_bwd_aux(b.dp, b.tb, b.dlogits, b.logits_saved, W->b_gate, m.aux, aux_part, m.T, m.E, m.E64,
+                                        ldcat, m.k, m.dtype, st));
+    } else {
+        Stage s(L, S_GATE_BWD, st);
+        BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, ldcat, m.k, m.dtype, st));
+    }
     {   // dz = (du W2_e) * sigma'(z); the forward saved sigma'(z) in the z buffer, dz is written over it
         GemmArgs g;
         g.A = b.du; g.lda = m.r; g.B = W->w2; g.ldb = m.h; g.b_kmajor = false; g.b_stride = (int64_t)m.r * m.h;
@@ -564,7 +610,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
                 BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
             }
         }
-        if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st)); }
+        if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st, aux_part)); }
         return BIGMAC_OK;
     }
     // dx'[t] = sum_j dxg[row of slot (t,j)]   (the transpose of the dispatch gather)
@@ -613,7 +659,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
             BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
         }
     }
-    if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st)); }
+    if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st, aux_part)); }
     return BIGMAC_OK;
 }
 
@@ -711,6 +757,8 @@ void carve_route_only(Carver& cv, const Dims& m, Buffers& b) {
     b.tb.slot_of_prow = cv.take<int32_t>(m.P);
     b.tb.tile_expert = cv.take<int32_t>(m.P / kPad);
     b.tb.n_tiles = cv.take<int32_t>(1);
+    b.tb.counts_chosen = cv.take<int32_t>(m.E);
+    b.aux_loss = cv.take<float>(1);
 }
 
 }  // namespace

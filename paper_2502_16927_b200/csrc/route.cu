@@ -183,7 +183,8 @@ __global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ b
                                                          int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                                                          int32_t* __restrict__ poffsets,
                                                          int32_t* __restrict__ tile_expert,
-                                                         int32_t* __restrict__ n_tiles) {
+                                                         int32_t* __restrict__ n_tiles, int cap,
+                                                         int32_t* __restrict__ counts_chosen) {
     __shared__ int32_t s_cnt[kMaxExperts];
     __shared__ int32_t s_poff[kMaxExperts + 1];
     __shared__ int32_t s_part[1024];
@@ -217,7 +218,12 @@ __global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ b
                 if (q < part) run += v;
                 total += v;
             }
-            if (part == 0) { s_cnt[e] = total; counts[e] = total; }
+            if (part == 0) {                        // an expert keeps at most `cap` of the slots that chose it
+                const int kept = min(total, cap);
+                s_cnt[e] = kept;
+                counts[e] = kept;
+                if (counts_chosen) counts_chosen[e] = total;
+            }
             int b = b0;
             for (; b + 8 <= b1; b += 8) {
                 int c[8];
@@ -252,7 +258,7 @@ __global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ b
         for (int tile = s_poff[e] / kPad; tile < s_poff[e + 1] / kPad; ++tile) tile_expert[tile] = e;
 }
 
-// Pass 3: final positions.
+// Pass 3: final positions.  A slot whose rank among the slots of its expert is `cap` or more is dropped (-1).
 __global__ void __launch_bounds__(256) sort_place_kernel(const int32_t* __restrict__ topk_idx, int64_t N, int E,
                                                          const int32_t* __restrict__ block_base,
                                                          const int32_t* __restrict__ offsets,
@@ -260,11 +266,16 @@ __global__ void __launch_bounds__(256) sort_place_kernel(const int32_t* __restri
                                                          int32_t* __restrict__ prow_of_slot /* in: local rank */,
                                                          int32_t* __restrict__ row_of_slot,
                                                          int32_t* __restrict__ slot_of_row,
-                                                         int32_t* __restrict__ slot_of_prow) {
+                                                         int32_t* __restrict__ slot_of_prow, int cap) {
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= N) return;
     const int e = topk_idx[s];
     const int within = block_base[(size_t)(s / kSortChunk) * E + e] + prow_of_slot[s];
+    if (within >= cap) {
+        row_of_slot[s] = -1;
+        prow_of_slot[s] = -1;
+        return;
+    }
     const int row = offsets[e] + within;
     const int prow = poffsets[e] + within;
     row_of_slot[s] = row;
@@ -310,22 +321,26 @@ cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, 
     return cudaGetLastError();
 }
 
-cudaError_t launch_tables(const Tables& tb, int T, int E, int k, cudaStream_t stream) {
+cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaStream_t stream) {
     const int64_t N = (int64_t)T * k;
     const int64_t P = padded_rows_max(N, E);
     cudaError_t err = cudaMemsetAsync(tb.slot_of_prow, 0xff, sizeof(int32_t) * P, stream);
     if (err != cudaSuccess) return err;
+    if (cap < N) {                                   // rows past the kept ones exist only under a capacity limit
+        err = cudaMemsetAsync(tb.slot_of_row, 0xff, sizeof(int32_t) * N, stream);
+        if (err != cudaSuccess) return err;
+    }
     const int nb = sort_blocks(N);
     if (nb > 0)
         sort_local_kernel<<<nb, 256, sizeof(int32_t) * 8 * E, stream>>>(tb.topk_idx, N, E, tb.prow_of_slot,
                                                                       tb.block_counts);
     sort_scan_kernel<<<1, 1024, 0, stream>>>(tb.block_counts, nb, E, tb.counts, tb.offsets, tb.poffsets,
-                                             tb.tile_expert, tb.n_tiles);
+                                             tb.tile_expert, tb.n_tiles, cap, tb.counts_chosen);
     if (N > 0)
         sort_place_kernel<<<(unsigned)((N + 255) / 256), 256, 0, stream>>>(tb.topk_idx, N, E, tb.block_counts,
                                                                           tb.offsets, tb.poffsets, tb.prow_of_slot,
                                                                           tb.row_of_slot, tb.slot_of_row,
-                                                                          tb.slot_of_prow);
+                                                                          tb.slot_of_prow, cap);
     return cudaGetLastError();
 }
 

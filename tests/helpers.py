@@ -53,12 +53,13 @@ def to_numpy(t):
     return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
 
 
-def make_layer(w, flags=0, max_tokens=None):
+def make_layer(w, flags=0, max_tokens=None, capacity_factor=0.0, aux_loss_coef=0.0):
     from paper_2502_16927_b200 import binding
 
     if w.cdac:
         flags |= wl.FLAG_CDAC
-    return binding.Layer(w.d, w.r, w.h, w.E, w.k, max_tokens or max(w.T, 1), w.dtype, w.act, flags)
+    return binding.Layer(w.d, w.r, w.h, w.E, w.k, max_tokens or max(w.T, 1), w.dtype, w.act, flags,
+                         capacity_factor=capacity_factor, aux_loss_coef=aux_loss_coef)
 
 
 def oracle_inputs(w, inp):

@@ -34,21 +34,22 @@ def check_routing(R, rt):
     np.testing.assert_array_equal(to_numpy(R["offsets"]), rt.offsets)
     np.testing.assert_array_equal(to_numpy(R["row_of_slot"]), rt.row_of_slot)
     np.testing.assert_array_equal(to_numpy(R["slot_of_row"]), rt.slot_of_row)
+    np.testing.assert_array_equal(to_numpy(R["counts_chosen"]), rt.counts_chosen)
     np.testing.assert_allclose(to_numpy(R["topk_w"]).reshape(rt.topk_p.shape), rt.topk_p, rtol=0, atol=2e-5)
 
 
-def run_full(w, inp, flags=0):
+def run_full(w, inp, flags=0, capacity_factor=0.0, aux=0.0):
     """Forward (training) + backward on the GPU; returns numpy results keyed like the oracle's."""
     import torch
 
     dev = to_device(w, inp)
-    layer = make_layer(w, flags)
+    layer = make_layer(w, flags, capacity_factor=capacity_factor, aux_loss_coef=aux)
     y, R = layer.forward(dev["x"], dev, training=True, want_routing=True)
     G = empty_grads(w, "cuda", fill=float("nan"))
     dx = layer.backward(dev["x"], dev["dy"], dev, G, accumulate=False)
     torch.cuda.synchronize()
     assert layer.status() == 0
-    out = {"y": to_numpy(y), "dx": to_numpy(dx), "routing": R}
+    out = {"y": to_numpy(y), "dx": to_numpy(dx), "routing": R, "aux_loss": float(R["aux_loss"].item())}
     out.update({key: to_numpy(val) for key, val in G.items()})
     layer.close()
     return out
@@ -86,11 +87,13 @@ def outlier_fraction(a, b, tol):
 RELU_DECISION_KEYS = ("dx", "dw1", "dw2", "dw_down", "dw_gate", "db_gate")
 
 
-def compare_full(w, inp, got, tol=None):
+def compare_full(w, inp, got, tol=None, capacity_factor=0.0, aux=0.0):
     inp = oracle_inputs(w, inp)
-    rt = oracle.route(inp, w.k)
+    rt = oracle.route(inp, w.k, capacity_factor=capacity_factor)
     check_routing(got["routing"], rt)
-    ref = oracle.backward_full(inp, rt, w.act, decide_bf16=w.dtype == wl.DTYPE_BF16)
+    ref = oracle.backward_full(inp, rt, w.act, decide_bf16=w.dtype == wl.DTYPE_BF16, aux_alpha=aux)
+    # the loss is a sum of T*E fp32 terms on the GPU: 1e-5 relative covers its rounding at every size used here
+    assert abs(got["aux_loss"] - ref.get("aux_loss", 0.0)) <= 1e-5 * abs(ref.get("aux_loss", 0.0))
     ref["dw1"] = np.stack([ref["dw1"][e] for e in range(w.E)])
     ref["dw2"] = np.stack([ref["dw2"][e] for e in range(w.E)])
     keys = ("y", "dx", "dw_gate", "dw1", "dw2", "db_gate") + (() if w.cdac else ("dw_up", "dw_down"))
