@@ -189,6 +189,77 @@ int bigmac_device_status(bigmac_layer_t *L, void *stream);
 
 const char *bigmac_status_string(int status);
 
+/* ---- Expert parallelism: the deployment the paper measures (Fig. 2c; Eq. 1 with the row width h replaced by
+ * r h) ------------------------------------------------------------------------------------------------------
+ * `size` ranks, one GPU each.  Every rank holds the shared matrices (w_gate, b_gate, w_down, w_up) in full and
+ * E/size experts: rank q owns experts [q E/size, (q+1) E/size), and its w1 / w2 / dw1 / dw2 hold only those
+ * ([E/size,h,r], [E/size,r,h]).  Every rank brings its own T tokens (T may differ between ranks).  The result is
+ * that of ONE layer applied to all ranks' tokens together (rank 0's first, then rank 1's, ...).
+ *
+ * The two All-to-All exchanges of Fig. 2c are made by the ranks' own kernels over peer memory, at the low width
+ * r: a rank PUTS the r-wide row x' of each of its slots straight into the segment of the owning rank's grouped
+ * buffer, and later GETS the expert output u of that row from there (weighted by its gate value); the backward pass
+ * puts du and gets dxg the same way.  Per rank and direction k T r (size-1)/size elements cross the links, against
+ * k T d (size-1)/size for a layer that exchanges full-width rows (Eq. 1).  Rows land in the owner's local memory
+ * first; its grouped GEMMs read only local memory.  No host-visible sizes, no device allocation, no stream
+ * synchronisation inside the calls.
+ *
+ * Exchange buffers: four per rank (xg, u, du, dxg), bigmac_ep_buffer_bytes() each, caller-owned, 256-byte aligned,
+ * and mapped into every rank's address space (peer access within a process, CUDA IPC or symmetric memory between
+ * processes): entry [q] of each array below is rank q's buffer as THIS rank addresses it.  counts_all is local
+ * memory, [size, E]: bigmac_ep_route writes this rank's row, the caller gathers the other ranks' rows into it (an
+ * all-gather of E integers per rank) before bigmac_ep_dispatch.
+ *
+ * Order of calls on every rank, with a barrier over all ranks' streams wherever "|" stands (each call only
+ * enqueues work on `stream`; the barrier must order that work, e.g. a collective on the same streams):
+ *     route  | (all-gather of counts) dispatch | experts | combine            -> y
+ *     backward_combine | backward_experts | backward_dispatch                -> dx, gradients
+ * `saved` (and, across the three backward calls, `scratch`) must keep their contents between the calls of a step.
+ * The gradients of the shared matrices that the backward returns are this rank's share (the sum over its own
+ * tokens): the caller adds them over the ranks, as for any data-parallel layer; dw1 / dw2 are complete.
+ * Not supported together with a capacity factor, a load-balancing loss or BIGMAC_FLAG_CDAC (BIGMAC_ERR_UNSUPPORTED). */
+#define BIGMAC_EP_MAX_RANKS 8
+typedef struct {
+    int32_t rank, size;                 /* 0 <= rank < size <= BIGMAC_EP_MAX_RANKS, E % size == 0 */
+    int32_t *counts_all;                /* [size, E] device memory of this rank */
+    void *xg[BIGMAC_EP_MAX_RANKS];      /* rows x' received by rank q     [rows, r] */
+    void *u[BIGMAC_EP_MAX_RANKS];       /* expert outputs of rank q       [rows, r] */
+    void *du[BIGMAC_EP_MAX_RANKS];      /* gradients received by rank q   [rows, r] */
+    void *dxg[BIGMAC_EP_MAX_RANKS];     /* input gradients of rank q      [rows, r] */
+} bigmac_ep_t;
+
+/* Bytes of ONE exchange buffer when no rank brings more than the handle's max_tokens tokens (worst case: every
+ * slot of every rank is routed to this rank's experts). */
+int bigmac_ep_buffer_bytes(const bigmac_layer_t *L, int32_t size, size_t *bytes);
+/* Scratch and saved bytes of the expert-parallel calls (both 256-byte aligned, as for bigmac_workspace_bytes). */
+int bigmac_ep_workspace_bytes(const bigmac_layer_t *L, int32_t T, int32_t size, size_t *scratch_bytes,
+                              size_t *saved_bytes);
+/* x' = x W'_down and the gate logits, top-k, gate values, this rank's slots sorted by expert; writes row `rank` of
+ * ep->counts_all.  routing_out (nullable) receives this rank's local tables (counts / offsets / rows local). */
+int bigmac_ep_route(bigmac_layer_t *L, const void *x, int32_t T, const bigmac_weights_t *W, const bigmac_ep_t *ep,
+                    bigmac_routing_t *routing_out, void *saved, void *scratch, size_t scratch_bytes, void *stream);
+/* Layout of every owner's segments from counts_all, zero fill of this rank's padding rows, first exchange: x' rows
+ * of this rank's slots -> xg of the owners. */
+int bigmac_ep_dispatch(bigmac_layer_t *L, int32_t T, const bigmac_ep_t *ep, void *saved, void *stream);
+/* This rank's experts over the rows it received: u = sigma(xg W1_e^T) W2_e^T (Eq. 4).  W->w1 / w2: owned experts. */
+int bigmac_ep_experts(bigmac_layer_t *L, const bigmac_weights_t *W, const bigmac_ep_t *ep, void *saved, void *stream);
+/* Second exchange and the rest of Eq. 2: y' = sum_j p_j u[row of slot j at its owner], y = y' W'_up. */
+int bigmac_ep_combine(bigmac_layer_t *L, int32_t T, const bigmac_weights_t *W, const bigmac_ep_t *ep, void *y,
+                      void *saved, void *stream);
+/* dy' = dy W_up, dW_up; per slot dp = <dy', u at its owner> (get) and du = p dy' -> du of the owner (put); gate
+ * backward.  G members may be NULL. */
+int bigmac_ep_backward_combine(bigmac_layer_t *L, const void *dy, int32_t T, const bigmac_weights_t *W,
+                               const bigmac_ep_t *ep, const bigmac_grads_t *G, int accumulate, void *saved,
+                               void *scratch, size_t scratch_bytes, void *stream);
+/* This rank's experts, backward, over the rows it holds: dz, dW2, dxg, dW1 (G->dw1 / dw2: owned experts). */
+int bigmac_ep_backward_experts(bigmac_layer_t *L, const bigmac_weights_t *W, const bigmac_ep_t *ep,
+                               const bigmac_grads_t *G, int accumulate, void *saved, void *scratch,
+                               size_t scratch_bytes, void *stream);
+/* dx' = sum_j dxg[row of slot j at its owner] (get), dx, dW_down, dW_gate, db_gate (this rank's share). */
+int bigmac_ep_backward_dispatch(bigmac_layer_t *L, const void *x, int32_t T, const bigmac_weights_t *W,
+                                const bigmac_ep_t *ep, void *dx, const bigmac_grads_t *G, int accumulate,
+                                void *saved, void *scratch, size_t scratch_bytes, void *stream);
+
 /* Measurement aid for the dispatch/combine stage (Eq. 1: bytes through the exchange are proportional
  * to the row width): run the standalone dispatch and combine kernels on rows of `width` elements of
  * the layer's dtype.  width = r is BigMac's exchange; width = d is what a fine-grained layer of equal

@@ -56,6 +56,14 @@ class bigmac_profile_t(C.Structure):
                 ("ms", C.c_float * BIGMAC_PROFILE_SLOTS), ("calls", C.c_uint32 * BIGMAC_PROFILE_SLOTS)]
 
 
+BIGMAC_EP_MAX_RANKS = 8
+
+
+class bigmac_ep_t(C.Structure):
+    _fields_ = [("rank", C.c_int32), ("size", C.c_int32), ("counts_all", C.c_void_p)] + \
+               [(n, C.c_void_p * BIGMAC_EP_MAX_RANKS) for n in ("xg", "u", "du", "dxg")]
+
+
 _lib: Optional[C.CDLL] = None
 
 
@@ -86,6 +94,20 @@ def lib() -> C.CDLL:
         L.bigmac_profile_read.argtypes = [vp, vp, C.POINTER(bigmac_profile_t)]
         L.bigmac_profile_slot_name.argtypes = [C.c_int]
         L.bigmac_profile_slot_name.restype = C.c_char_p
+        W, R, G, EP = (C.POINTER(t) for t in (bigmac_weights_t, bigmac_routing_t, bigmac_grads_t, bigmac_ep_t))
+        L.bigmac_ep_buffer_bytes.argtypes = [vp, i32, C.POINTER(sz)]
+        L.bigmac_ep_workspace_bytes.argtypes = [vp, i32, i32, C.POINTER(sz), C.POINTER(sz)]
+        L.bigmac_ep_route.argtypes = [vp, vp, i32, W, EP, R, vp, vp, sz, vp]
+        L.bigmac_ep_dispatch.argtypes = [vp, i32, EP, vp, vp]
+        L.bigmac_ep_experts.argtypes = [vp, W, EP, vp, vp]
+        L.bigmac_ep_combine.argtypes = [vp, i32, W, EP, vp, vp, vp]
+        L.bigmac_ep_backward_combine.argtypes = [vp, vp, i32, W, EP, G, C.c_int, vp, vp, sz, vp]
+        L.bigmac_ep_backward_experts.argtypes = [vp, W, EP, G, C.c_int, vp, vp, sz, vp]
+        L.bigmac_ep_backward_dispatch.argtypes = [vp, vp, i32, W, EP, vp, G, C.c_int, vp, vp, sz, vp]
+        for name in ("bigmac_ep_buffer_bytes", "bigmac_ep_workspace_bytes", "bigmac_ep_route", "bigmac_ep_dispatch",
+                     "bigmac_ep_experts", "bigmac_ep_combine", "bigmac_ep_backward_combine", "bigmac_ep_backward_experts",
+                     "bigmac_ep_backward_dispatch"):
+            getattr(L, name).restype = C.c_int
         for name in ("bigmac_profile_enable", "bigmac_profile_read", "bigmac_layer_create", "bigmac_layer_destroy", "bigmac_workspace_bytes", "bigmac_route",
                      "bigmac_forward", "bigmac_backward", "bigmac_device_status", "bigmac_exchange_rows",
                      "bigmac_debug_gemm"):
@@ -137,8 +159,12 @@ def bigmac_workspace_bytes(handle, T: int, training: bool):
 
 def _weights(W: Dict[str, torch.Tensor]) -> bigmac_weights_t:
     # w_down / w_up are absent for the projection-free layer (BIGMAC_FLAG_CDAC)
-    return bigmac_weights_t(_ptr(W["w_gate"]), _ptr(W.get("b_gate")), _ptr(W.get("w_down")), _ptr(W["w1"]), _ptr(W["w2"]),
-                            _ptr(W.get("w_up")))
+    return bigmac_weights_t(_ptr(W.get("w_gate")), _ptr(W.get("b_gate")), _ptr(W.get("w_down")), _ptr(W.get("w1")),
+                            _ptr(W.get("w2")), _ptr(W.get("w_up")))
+
+
+def _grads(G: Dict[str, torch.Tensor]) -> bigmac_grads_t:
+    return bigmac_grads_t(*[_ptr(G.get(n)) for n in ("dw_gate", "db_gate", "dw_down", "dw1", "dw2", "dw_up")])
 
 
 def _routing(R: Optional[Dict[str, torch.Tensor]]):
@@ -166,9 +192,8 @@ def bigmac_forward(handle, x, T, W, y, routing, saved, scratch) -> None:
 
 
 def bigmac_backward(handle, x, dy, T, W, saved, dx, G, accumulate, scratch) -> None:
-    grads = bigmac_grads_t(*[_ptr(G.get(n)) for n in ("dw_gate", "db_gate", "dw_down", "dw1", "dw2", "dw_up")])
     _check(lib().bigmac_backward(handle, _ptr(x), _ptr(dy), T, C.byref(_weights(W)), _ptr(saved), _ptr(dx),
-                                 C.byref(grads), int(accumulate), _ptr(scratch),
+                                 C.byref(_grads(G)), int(accumulate), _ptr(scratch),
                                  scratch.numel() * scratch.element_size(), _stream()), "bigmac_backward")
 
 
@@ -198,6 +223,71 @@ def bigmac_profile_read(handle) -> Dict[str, object]:
 def bigmac_debug_gemm(handle, q: bigmac_debug_gemm_t, use_tensor_cores) -> None:
     """use_tensor_cores: False/0 plain FMA, True/1 tensor cores, 2 one-CTA kernel, 3 CTA-pair kernel."""
     _check(lib().bigmac_debug_gemm(handle, C.byref(q), int(use_tensor_cores), _stream()), "bigmac_debug_gemm")
+
+
+# ---- expert parallelism: the phase calls, name for name ----------------------------------------------------
+
+def bigmac_ep_buffer_bytes(handle, size: int) -> int:
+    n = C.c_size_t()
+    _check(lib().bigmac_ep_buffer_bytes(handle, size, C.byref(n)), "bigmac_ep_buffer_bytes")
+    return n.value
+
+
+def bigmac_ep_workspace_bytes(handle, T: int, size: int):
+    s, v = C.c_size_t(), C.c_size_t()
+    _check(lib().bigmac_ep_workspace_bytes(handle, T, size, C.byref(s), C.byref(v)), "bigmac_ep_workspace_bytes")
+    return s.value, v.value
+
+
+def make_ep(rank: int, size: int, counts_all: torch.Tensor, ptrs: Dict[str, list]) -> bigmac_ep_t:
+    """ptrs[name][q]: device address (int) of rank q's exchange buffer `name` as this rank addresses it."""
+    ep = bigmac_ep_t()
+    ep.rank, ep.size, ep.counts_all = rank, size, counts_all.data_ptr()
+    for name in ("xg", "u", "du", "dxg"):
+        arr = getattr(ep, name)
+        for q in range(size):
+            arr[q] = ptrs[name][q]
+    return ep
+
+
+def _nbytes(t: torch.Tensor) -> int:
+    return t.numel() * t.element_size()
+
+
+def bigmac_ep_route(handle, x, T, W, ep, routing, saved, scratch) -> None:
+    _check(lib().bigmac_ep_route(handle, _ptr(x), T, C.byref(_weights(W)), C.byref(ep), _routing(routing), _ptr(saved),
+                                 _ptr(scratch), _nbytes(scratch), _stream()), "bigmac_ep_route")
+
+
+def bigmac_ep_dispatch(handle, T, ep, saved) -> None:
+    _check(lib().bigmac_ep_dispatch(handle, T, C.byref(ep), _ptr(saved), _stream()), "bigmac_ep_dispatch")
+
+
+def bigmac_ep_experts(handle, W, ep, saved) -> None:
+    _check(lib().bigmac_ep_experts(handle, C.byref(_weights(W)), C.byref(ep), _ptr(saved), _stream()), "bigmac_ep_experts")
+
+
+def bigmac_ep_combine(handle, T, W, ep, y, saved) -> None:
+    _check(lib().bigmac_ep_combine(handle, T, C.byref(_weights(W)), C.byref(ep), _ptr(y), _ptr(saved), _stream()),
+           "bigmac_ep_combine")
+
+
+def bigmac_ep_backward_combine(handle, dy, T, W, ep, G, accumulate, saved, scratch) -> None:
+    _check(lib().bigmac_ep_backward_combine(handle, _ptr(dy), T, C.byref(_weights(W)), C.byref(ep), C.byref(_grads(G)),
+                                            int(accumulate), _ptr(saved), _ptr(scratch), _nbytes(scratch), _stream()),
+           "bigmac_ep_backward_combine")
+
+
+def bigmac_ep_backward_experts(handle, W, ep, G, accumulate, saved, scratch) -> None:
+    _check(lib().bigmac_ep_backward_experts(handle, C.byref(_weights(W)), C.byref(ep), C.byref(_grads(G)), int(accumulate),
+                                            _ptr(saved), _ptr(scratch), _nbytes(scratch), _stream()),
+           "bigmac_ep_backward_experts")
+
+
+def bigmac_ep_backward_dispatch(handle, x, T, W, ep, dx, G, accumulate, saved, scratch) -> None:
+    _check(lib().bigmac_ep_backward_dispatch(handle, _ptr(x), T, C.byref(_weights(W)), C.byref(ep), _ptr(dx),
+                                             C.byref(_grads(G)), int(accumulate), _ptr(saved), _ptr(scratch),
+                                             _nbytes(scratch), _stream()), "bigmac_ep_backward_dispatch")
 
 
 # ---- a small convenience wrapper: owns the handle and the workspaces ------------------------------------

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbigmac.so")
-SOURCES = ["layer.cu", "route.cu", "permute.cu", "aux_loss.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_tc_groupk.cu", "gemm_tc_mlp.cu", "decode.cu"]
+SOURCES = ["layer.cu", "route.cu", "permute.cu", "aux_loss.cu", "ep.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_tc_groupk.cu", "gemm_tc_mlp.cu", "decode.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

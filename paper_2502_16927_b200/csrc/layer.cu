@@ -9,78 +9,13 @@
 #include <new>
 #include <vector>
 
-#include "internal.h"
-#include "bigmac_debug.h"
+#include "layer_common.h"
 
 using namespace bigmac;
+using namespace bigmac::detail;
 
-struct bigmac_layer {
-    bigmac_config_t cfg;
-    int device;
-    int* status;        // device status word; status[1] is the grid-barrier counter of the small-batch kernel,
-                        // status[2..3] the work counters of the per-expert weight-gradient kernel (zero at rest)
-    bool use_tc;        // bf16 contractions on tcgen05
-    unsigned tc_mask;   // debug: bit i set = contraction i runs on tcgen05 (BIGMAC_TC_MASK)
-    // measurement aid
-    bool prof_on = false;
-    uint64_t launches = 0;
-    uint32_t dropped = 0;
-    std::vector<cudaEvent_t> ev;       // pool of start/stop pairs
-    std::vector<int> ev_slot;          // stage of each recorded pair
-    float ms[BIGMAC_PROFILE_SLOTS] = {};
-    uint32_t calls[BIGMAC_PROFILE_SLOTS] = {};
-};
-
-namespace {
-
-// Contraction ids (bits of tc_mask).
-enum { G_LOGITS = 0, G_DESCEND, G_EXPERT1, G_EXPERT2, G_ASCEND, G_DY_LO, G_DW_UP, G_DZ, G_DW2, G_DXG, G_DW1,
-       G_DX, G_DX_GATE, G_DW_DOWN, G_DW_GATE,
-       S_TOPK, S_TABLES, S_DISPATCH, S_COMBINE, S_COMBINE_BWD, S_GATE_BWD, S_DXLO_GATHER, S_COLSUM, S_SPLITK_REDUCE,
-       S_DECODE, S_FUSED_MLP, S_AUX_LOSS, S_COUNT };
-const char* const kSlotNames[S_COUNT] = {
-    "gemm_logits", "gemm_descend", "gemm_expert1", "gemm_expert2", "gemm_ascend", "gemm_dy_lo", "gemm_dw_up",
-    "gemm_dz", "gemm_dw2", "gemm_dxg", "gemm_dw1", "gemm_dx", "gemm_dx_gate", "gemm_dw_down", "gemm_dw_gate",
-    "topk", "tables", "dispatch", "combine", "combine_bwd", "gate_bwd", "dxlo_gather", "colsum",
-    "splitk_reduce", "decode_forward", "fused_expert_mlp", "aux_loss"};
-constexpr size_t kEventPairs = 8192;
-constexpr int kMaxSplitK = 8;
-
-// Counts the launches of one stage and, while profiling, brackets them with an event pair.
-struct Stage {
-    bigmac_layer* L;
-    cudaStream_t st;
-    cudaEvent_t stop = nullptr;
-    Stage(const bigmac_layer* layer, int slot, cudaStream_t stream, int kernels = 1)
-        : L(const_cast<bigmac_layer*>(layer)), st(stream) {
-        L->launches += kernels;
-        if (!L->prof_on) return;
-        const size_t i = L->ev_slot.size();
-        if (i >= kEventPairs) { L->dropped += kernels; return; }
-        L->ev_slot.push_back(slot);
-        L->calls[slot] += kernels;
-        cudaEventRecord(L->ev[2 * i], st);
-        stop = L->ev[2 * i + 1];
-    }
-    ~Stage() { if (stop) cudaEventRecord(stop, st); }
-};
-
-inline size_t esize(int dtype) { return dtype == BIGMAC_BF16 ? 2 : 4; }
-
-// Hands out 256-byte-aligned regions of one buffer; with base == nullptr it only measures.
-struct Carver {
-    char* base;
-    size_t used = 0;
-    explicit Carver(void* b) : base((char*)b) {}
-    template <typename T> T* take(size_t count) {
-        used = (used + 255) & ~(size_t)255;
-        T* p = base ? (T*)(base + used) : nullptr;
-        used += count * sizeof(T);
-        return p;
-    }
-    void* take_bytes(size_t bytes) { return take<char>(bytes); }
-    size_t total() const { return (used + 255) & ~(size_t)255; }
-};
+namespace bigmac {
+namespace detail {
 
 struct Buffers {
     Tables tb;
@@ -108,8 +43,6 @@ struct Dims {
     float aux; // coefficient of the load-balancing loss (Table 5), 0 = none
 };
 
-// The tensor-core kernels save sigma' as one byte per element; that needs expert GEMM1 and dz on the same side.
-bool sigma_as_bytes(const bigmac_layer* L) { return L->cfg.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u; }
 
 Dims dims_of(const bigmac_layer* L, int T) {
     const bigmac_config_t& c = L->cfg;
@@ -196,7 +129,6 @@ size_t saved_bytes_of(const Dims& m) {
     return cv.total();
 }
 
-bool aligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
 
 int check_weights(const bigmac_layer* L, const bigmac_weights_t* W) {
     if (!W || !W->w_gate || !W->w1 || !W->w2) return BIGMAC_ERR_INVALID_ARG;
@@ -234,16 +166,6 @@ int choose_split_k(int M, int N, int K) {
     }
     return best;
 }
-
-#define BIGMAC_TRY(expr)                        \
-    do {                                        \
-        int _s = (expr);                        \
-        if (_s != BIGMAC_OK) return _s;         \
-    } while (0)
-#define BIGMAC_CUDA(expr)                                   \
-    do {                                                    \
-        if ((expr) != cudaSuccess) return BIGMAC_ERR_CUDA;  \
-    } while (0)
 
 // Steps F2-F3 from the gate logits: top-k with softmax gate values, dispatch layout (under the capacity limit, if
 // any), load-balancing loss.
@@ -300,7 +222,7 @@ int check_call(const bigmac_layer* L, int32_t T) {
 
 // Per-expert weight gradient (contraction over the expert's rows): on the tensor-core path the balanced kernel
 // (dynamic work items, long experts in parts), else the generic grouped contraction.
-int expert_weight_grad(const bigmac_layer* L, int id, const GemmArgs& g, const Buffers& b, cudaStream_t st) {
+int expert_weight_grad(const bigmac_layer* L, int id, const GemmArgs& g, float* splitk_ws, cudaStream_t st) {
     static const bool enabled = []() { const char* e = std::getenv("BIGMAC_GROUPK"); return !(e && e[0] == '0'); }();
     const bool tc = L->cfg.dtype == BIGMAC_BF16 && L->use_tc && ((L->tc_mask >> id) & 1u);
     // below about 16 k slices of work per CTA pair the items are too short for dynamic hand-out to pay (measured:
@@ -309,14 +231,15 @@ int expert_weight_grad(const bigmac_layer* L, int id, const GemmArgs& g, const B
     const bool enough = (L->cfg.flags & BIGMAC_FLAG_DYNAMIC_WGRAD) ||
                         (int64_t)(g.K / 64) * tiles >= 16 * (int64_t)(gemm_tc_sm_count() / 2);
     if (enabled && tc && enough && gemm_tc_groupk_supported(g)) {
-        { Stage stage(L, id, st); BIGMAC_CUDA(gemm_tc_groupk(g, L->status, L->status + 2, b.splitk_ws, st)); }
-        { Stage stage(L, S_SPLITK_REDUCE, st); BIGMAC_CUDA(gemm_tc_groupk_finish(g, b.splitk_ws, st)); }
+        { Stage stage(L, id, st); BIGMAC_CUDA(gemm_tc_groupk(g, L->status, L->status + 2, splitk_ws, st)); }
+        { Stage stage(L, S_SPLITK_REDUCE, st); BIGMAC_CUDA(gemm_tc_groupk_finish(g, splitk_ws, st)); }
         return BIGMAC_OK;
     }
     return gemm(L, id, g, st);
 }
 
-}  // namespace
+}  // namespace detail
+}  // namespace bigmac
 
 extern "C" {
 
@@ -571,7 +494,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.A = b.du; g.lda = m.r; g.a_kmajor = false; g.B = b.a; g.ldb = m.h; g.b_kmajor = false;
         g.C = G->dw2; g.ldc = m.h; g.c_stride = (int64_t)m.r * m.h; g.M = m.r; g.N = m.h; g.K = (int)m.P;
         g.group = GROUP_K; g.num_experts = m.E; g.poffsets = b.tb.poffsets; g.accumulate = acc;
-        BIGMAC_TRY(expert_weight_grad(L, G_DW2, g, b, st));
+        BIGMAC_TRY(expert_weight_grad(L, G_DW2, g, b.splitk_ws, st));
     }
     {   // dxg = dz W1_e
         GemmArgs g;
@@ -585,7 +508,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.A = dz; g.lda = m.h; g.a_kmajor = false; g.B = b.xg; g.ldb = m.r; g.b_kmajor = false;
         g.C = G->dw1; g.ldc = m.r; g.c_stride = (int64_t)m.h * m.r; g.M = m.h; g.N = m.r; g.K = (int)m.P;
         g.group = GROUP_K; g.num_experts = m.E; g.poffsets = b.tb.poffsets; g.accumulate = acc;
-        BIGMAC_TRY(expert_weight_grad(L, G_DW1, g, b, st));
+        BIGMAC_TRY(expert_weight_grad(L, G_DW1, g, b.splitk_ws, st));
     }
     if (m.cdac) {
         // Eq. 3: dx = sum_j dxg[row of slot (t,j)] + dl W_gate; dW_gate = dl^T x

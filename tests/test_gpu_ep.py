@@ -1,0 +1,116 @@
+"""GPU parity of the expert-parallel layer (Fig. 2c): `size` ranks with their own tokens and E/size experts each,
+exchanging r-wide rows through each other's buffers, against the CPU oracle applied to the concatenation of the
+ranks' batches.  The ranks are driven by one process on one GPU (their kernels never wait on one another: every
+phase of every rank is a launch of its own), which exercises the same kernels, tables and addresses as one rank
+per GPU; what differs there is only that the buffer addresses are peer mappings and the barriers collectives."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import margin
+from paper_2502_16927_b200 import binding, ep, workloads as wl
+
+from helpers import to_device, to_numpy
+from test_gpu_parity import TOL, assert_within, float_errors
+
+pytestmark = pytest.mark.gpu
+
+
+def run_group(w, inp, tokens_per_rank, flags=0):
+    """Split the workload's tokens over the ranks, run forward + backward, return per-rank results and the group's sums."""
+    import torch
+
+    size = len(tokens_per_rank)
+    assert sum(tokens_per_rank) == w.T
+    dev = to_device(w, inp)
+    full = {key: dev[key] for key in ("w_gate", "w_down", "w1", "w2", "w_up") if key in dev}
+    if "b_gate" in dev:
+        full["b_gate"] = dev["b_gate"]
+    Ws = [ep.shard_weights(full, q, size) for q in range(size)]
+    bounds = np.concatenate([[0], np.cumsum(tokens_per_rank)])
+    xs = [dev["x"][bounds[q]:bounds[q + 1]].contiguous() for q in range(size)]
+    dys = [dev["dy"][bounds[q]:bounds[q + 1]].contiguous() for q in range(size)]
+    group = ep.EpLocalGroup(w.d, w.r, w.h, w.E, w.k, max(max(tokens_per_rank), 1), w.dtype, w.act, ["cuda"] * size, flags)
+    ys = group.forward(xs, Ws)
+    dt = torch.float32 if w.dtype == wl.DTYPE_F32 else torch.bfloat16
+    per = w.E // size
+    Gs = []
+    for q in range(size):
+        shapes = {"dw_gate": (w.E, w.d), "dw_down": (w.r, w.d), "dw_up": (w.d, w.r), "dw1": (per, w.h, w.r), "dw2": (per, w.r, w.h)}
+        G = {key: torch.full(shp, float("nan"), dtype=dt, device="cuda") for key, shp in shapes.items()}
+        G["db_gate"] = torch.full((w.E,), float("nan"), dtype=torch.float32, device="cuda")
+        Gs.append(G)
+    dxs = group.backward(xs, dys, Ws, Gs)
+    torch.cuda.synchronize()
+    assert group.status() == 0
+    busy = [q for q in range(size) if tokens_per_rank[q] > 0]            # a rank without tokens writes no shared gradients
+    got = {"y": np.concatenate([to_numpy(y) for y in ys]), "dx": np.concatenate([to_numpy(v) for v in dxs]),
+           "dw1": np.concatenate([to_numpy(G["dw1"]) for G in Gs]), "dw2": np.concatenate([to_numpy(G["dw2"]) for G in Gs]),
+           "counts_all": to_numpy(group.ranks[0].counts_all)}
+    for key in ep.SHARED_GRADS:
+        got[key] = sum(to_numpy(Gs[q][key]) for q in busy)
+    group.close()
+    return got
+
+
+def compare(w, inp, got):
+    rt = oracle.route(inp, w.k)
+    np.testing.assert_array_equal(got["counts_all"].sum(axis=0), rt.counts)
+    ref = oracle.backward_full(inp, rt, w.act, decide_bf16=w.dtype == wl.DTYPE_BF16)
+    ref["dw1"] = np.stack([ref["dw1"][e] for e in range(w.E)])
+    ref["dw2"] = np.stack([ref["dw2"][e] for e in range(w.E)])
+    keys = ("y", "dx", "dw_gate", "dw1", "dw2", "db_gate", "dw_up", "dw_down")
+    assert_within(w, float_errors(w, {key: got[key] for key in keys}, ref))
+    for e in range(w.E):
+        if rt.counts[e] == 0:
+            assert not got["dw1"][e].any() and not got["dw2"][e].any()
+
+
+def skewed(w, strength):
+    inp = wl.make_inputs(w)
+    if strength:
+        inp["b_gate"] = (strength * np.linspace(1.0, -1.0, w.E) ** 3).astype(np.float32)
+    margin.enforce_margin(w, inp, 1e-3)
+    return inp
+
+
+@pytest.mark.parametrize("tokens", [[700], [400, 300], [1, 0, 650, 49], [175] * 4, [100, 50, 90, 60, 120, 80, 110, 90]])
+def test_fp32_ranks_together_equal_one_layer(tokens):
+    w = wl.Workload("ep", T=sum(tokens), d=64, r=24, h=40, E=8, k=3, dtype=wl.DTYPE_F32, act=wl.ACT_GELU_ERF, seed=71)
+    inp = skewed(w, 1.5)
+    compare(w, inp, run_group(w, inp, tokens))
+
+
+@pytest.mark.parametrize("case", [
+    dict(shape=dict(d=256, r=128, h=256, E=16, k=4), tokens=[1500, 1500], strength=0.0),
+    dict(shape=dict(d=256, r=256, h=512, E=16, k=2), tokens=[2500, 100, 1400, 2000], strength=3.0),   # one rank's experts take most rows
+    dict(shape=dict(d=128, r=64, h=128, E=24, k=3), tokens=[900, 1100, 1000], strength=2.0),         # some experts without rows
+])
+@pytest.mark.parametrize("flags", [0, wl.FLAG_DYNAMIC_WGRAD])
+def test_bf16_ranks_together_equal_one_layer(case, flags):
+    w = wl.Workload("ep", T=sum(case["tokens"]), dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=73, **case["shape"])
+    inp = skewed(w, case["strength"])
+    compare(w, inp, run_group(w, inp, case["tokens"], flags))
+
+
+def test_small_config_on_four_ranks():
+    w = wl.WORKLOADS["small"]
+    inp = skewed(w, 0.0)
+    compare(w, inp, run_group(w, inp, [1024] * 4))
+
+
+def test_unsupported_combinations_and_bad_arguments():
+    w = wl.WORKLOADS["tiny"]
+    for kw in (dict(capacity_factor=1.2), dict(aux_loss_coef=0.1)):
+        h = binding.bigmac_layer_create(w.d, w.r, w.h, w.E, w.k, 64, w.dtype, w.act, 0, **kw)
+        with pytest.raises(binding.BigmacError) as err:
+            binding.bigmac_ep_buffer_bytes(h, 2)
+        assert err.value.status == -2
+        binding.bigmac_layer_destroy(h)
+    h = binding.bigmac_layer_create(w.d, w.r, w.h, w.E, w.k, 64, w.dtype, w.act)
+    for size in (0, 3, 9):                                   # E = 8: not a divisor, out of range
+        with pytest.raises(binding.BigmacError) as err:
+            binding.bigmac_ep_buffer_bytes(h, size)
+        assert err.value.status == -1
+    assert binding.bigmac_ep_buffer_bytes(h, 2) > 0
+    binding.bigmac_layer_destroy(h)

@@ -1,6 +1,8 @@
-"""The N > 1 path of bench.py on CPU: two gloo ranks.  The layer has no exchange step between ranks (each
-rank runs an independent batch), so what is multi-rank is only the bookkeeping: per-rank seeds, the
-max-over-ranks of the device time, the whole-job throughput, and the reference arm running on rank 0 only."""
+"""The N > 1 paths on CPU: two gloo ranks.  Expert parallelism: the host-side plumbing of the exchange (count
+all-gather, weight sharding, gradient reduction) and the row-placement rule, checked against the oracle's tables
+of the concatenated batch.  bench.py: its ranks run independent batches, so what is multi-rank there is only the
+bookkeeping: per-rank seeds, the max-over-ranks of the device time, the whole-job throughput, and the reference arm
+running on rank 0 only."""
 import json
 import os
 import subprocess
@@ -55,3 +57,67 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+# ---------------------------------------------------------------- expert parallelism: host side
+
+def _ep_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import oracle
+    from paper_2502_16927_b200 import ep
+
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    E, k, T = 6, 2, (37, 20)[rank]
+    g = np.random.default_rng(100 + rank)
+    logits = g.standard_normal((T, E)) + np.linspace(1.5, -1.5, E)
+    idx, _ = oracle.topk(logits, k)
+    counts, offsets, ros, _ = oracle.tables(idx, E)
+    counts_all = torch.zeros((world, E), dtype=torch.int32)
+    counts_all[rank] = torch.from_numpy(counts)
+    ep.gather_counts(counts_all, rank)
+    send_base, poffsets = ep.placement(counts_all.tolist(), rank)
+    dest = [(ep.owner_of_expert(E, int(e), world), send_base[e] + int(ros[s]) - int(offsets[e]))
+            for s, e in enumerate(idx.ravel())]
+    W = {"w_gate": torch.zeros(E, 4), "w1": torch.arange(E * 3 * 2, dtype=torch.float32).reshape(E, 3, 2),
+         "w2": torch.arange(E * 2 * 3, dtype=torch.float32).reshape(E, 2, 3)}
+    mine = ep.shard_weights(W, rank, world)
+    G = {"dw_gate": torch.full((E, 4), float(rank + 1)), "db_gate": torch.full((E,), float(rank + 1)), "dw_down": None,
+         "dw_up": torch.ones(4, 2), "dw1": torch.full((3,), 7.0)}
+    ep.reduce_shared_grads(G)
+    out[rank] = dict(idx=idx, dest=dest, counts_all=counts_all.numpy().copy(), poffsets=poffsets,
+                     w1_first=float(mine["w1"][0, 0, 0]), w1_shape=tuple(mine["w1"].shape),
+                     dw_gate=float(G["dw_gate"][0, 0]), db_gate=float(G["db_gate"][0]), dw1=float(G["dw1"][0]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_expert_parallel_host_side_with_two_ranks():
+    import numpy as np
+    import oracle
+
+    world, port = 2, 30500 + os.getpid() % 1000
+    manager = mp.Manager()
+    out = manager.dict()
+    mp.spawn(_ep_worker, args=(world, port, out), nprocs=world, join=True)
+    E, k, per = 6, 2, 3
+    np.testing.assert_array_equal(out[0]["counts_all"], out[1]["counts_all"])           # the all-gather
+    assert out[0]["poffsets"] == out[1]["poffsets"]
+    # the placement: one layer over the concatenated batch (rank 0's tokens first) sorts every expert's rows the same way
+    idx = np.concatenate([out[0]["idx"], out[1]["idx"]])
+    counts, offsets, ros, _ = oracle.tables(idx, E)
+    np.testing.assert_array_equal(out[0]["counts_all"].sum(axis=0), counts)
+    dest = out[0]["dest"] + out[1]["dest"]
+    seen = set()
+    for s, e in enumerate(idx.ravel()):
+        q, row = dest[s]
+        assert q == e // per
+        assert row == out[0]["poffsets"][q][e % per] + (ros[s] - offsets[e])
+        assert (q, row) not in seen
+        seen.add((q, row))
+    # sharding and gradient reduction
+    assert out[0]["w1_shape"] == out[1]["w1_shape"] == (per, 3, 2)
+    assert out[0]["w1_first"] == 0.0 and out[1]["w1_first"] == float(per * 3 * 2)
+    for r_ in (0, 1):
+        assert out[r_]["dw_gate"] == 3.0 and out[r_]["db_gate"] == 3.0 and out[r_]["dw1"] == 7.0   # experts' gradients stay
