@@ -302,6 +302,61 @@ def run_recipe_variant(w, x, dy, dev, G, y, dx, base_step, steps):
     return out
 
 
+def run_ep_on_one_gpu(w, x, dy, dev, ms_step, steps, esz, size=4):
+    """The expert-parallel layer (Fig. 2c) with `size` ranks driven on this one GPU: every rank brings T/size of the
+    step's tokens and owns E/size experts; rows travel between the ranks' buffers at width r through the same put /
+    get kernels a multi-GPU job runs, here within one memory.  What this measures is the cost of the phase structure
+    and of the exchange kernels against the one-GPU layer on the same tokens; link time it cannot show.  The bytes
+    that would cross the links per rank and exchange are reported for width r and, for comparison, width d (Eq. 1)."""
+    import torch
+    from paper_2502_16927_b200 import binding, ep
+
+    if w.E % size or w.T % size:
+        return None
+    Tq = w.T // size
+    Ws = [ep.shard_weights(dev, q, size) for q in range(size)]
+    xs = [x[q * Tq:(q + 1) * Tq] for q in range(size)]
+    dys = [dy[q * Tq:(q + 1) * Tq] for q in range(size)]
+    ys, dxs = [torch.empty_like(v) for v in xs], [torch.empty_like(v) for v in xs]
+    per = w.E // size
+    Gs = [{"dw_gate": torch.empty_like(dev["w_gate"]), "dw_down": torch.empty_like(dev["w_down"]),
+           "dw_up": torch.empty_like(dev["w_up"]), "dw1": torch.empty_like(Ws[q]["w1"]), "dw2": torch.empty_like(Ws[q]["w2"]),
+           "db_gate": torch.empty(w.E, dtype=torch.float32, device="cuda")} for q in range(size)]
+    group = ep.EpLocalGroup(w.d, w.r, w.h, w.E, w.k, Tq, w.dtype, w.act, ["cuda"] * size)
+
+    def step():
+        group.forward(xs, Ws, ys)
+        group.backward(xs, dys, Ws, Gs, dxs)
+
+    for _ in range(3):
+        step()
+    for rk in group.ranks:
+        binding.bigmac_profile_enable(rk.handle, True)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(steps):
+        step()
+    stop.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(stop) / steps
+    moves = {}
+    for rk in group.ranks:
+        prof = binding.bigmac_profile_read(rk.handle)
+        for name in ("dispatch", "combine", "combine_bwd", "dxlo_gather"):
+            tot, calls = prof["stages"].get(name, (0.0, 1))
+            moves[name] = moves.get(name, 0.0) + tot / steps
+    if group.status() != 0:
+        raise RuntimeError("device status word reports a timed-out wait")
+    group.close()
+    return {"ranks_on_this_gpu": size, "tokens_per_rank": Tq, "experts_per_rank": per, "ms_per_step_all_ranks": ms,
+            "tokens_per_s": w.T / (ms * 1e-3), "over_one_gpu_layer_time": round(ms / ms_step, 3),
+            "exchange_kernels_ms_all_ranks": {name: round(v, 4) for name, v in moves.items()},
+            "link_bytes_per_rank_per_exchange": {"width_r": ep.exchange_bytes_per_rank(Tq, w.k, w.r, size, esz),
+                                                 "width_d": ep.exchange_bytes_per_rank(Tq, w.k, w.d, size, esz)},
+            "note": "ranks share one GPU: no link is crossed; exchanges per step: 2 forward, 2 backward"}
+
+
 # ------------------------------------------------------------------------------------------------ ours
 def run_ours(args, w):
     import torch
@@ -501,6 +556,7 @@ def run_ours(args, w):
     peaks = measured_peaks()
     esz = 2 if w.dtype == wl.DTYPE_BF16 else 4
     twin = run_cdac_twin(w, x, dy, dev, ms_step, ms_fwd, max(3, min(args.steps, 10)), peaks, esz)
+    ep_line = run_ep_on_one_gpu(w, x, dy, dev, ms_step, max(3, min(args.steps, 10)), esz) if w.dtype == wl.DTYPE_BF16 else None
     recipe = run_recipe_variant(w, x, dy, dev, G, y, dx, step, max(3, min(args.steps, 10)))
     stages = {}
     gemm_ms = gemm_flops = 0.0
@@ -556,6 +612,7 @@ def run_ours(args, w):
             "exchange": exchange,
             "cdac_twin": twin,
             "recipe_variant": recipe,
+            "expert_parallel_on_one_gpu": ep_line,
             "stages": stages}
     print(json.dumps(line))
     if world > 1:

@@ -15,7 +15,8 @@ namespace bigmac {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kAuxWarps = 4;
+// Warps per block: 8 where the shared-memory rows of the backward kernel ((2 W + 1) E floats) stay under 48 KB.
+inline int aux_warps(int E) { return E <= 512 ? 8 : 4; }
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
@@ -40,19 +41,20 @@ __device__ __forceinline__ void softmax_stats(const float* __restrict__ l, const
 }
 
 __device__ __forceinline__ void token_range(int T, int warp, int& t0, int& t1) {
-    const int per_warp = (T + (int)gridDim.x * kAuxWarps - 1) / ((int)gridDim.x * kAuxWarps);
-    const int64_t first = ((int64_t)blockIdx.x * kAuxWarps + warp) * per_warp;
+    const int warps = blockDim.x >> 5;
+    const int per_warp = (T + (int)gridDim.x * warps - 1) / ((int)gridDim.x * warps);
+    const int64_t first = ((int64_t)blockIdx.x * warps + warp) * per_warp;
     t0 = (int)(first < T ? first : T);
     t1 = (int)(first + per_warp < T ? first + per_warp : T);
 }
 
 // partial[b][e] = sum over the tokens of block b of p[t,e]
-__global__ void __launch_bounds__(kAuxWarps * 32) aux_prob_sums_kernel(const float* __restrict__ logits,
+__global__ void __launch_bounds__(256) aux_prob_sums_kernel(const float* __restrict__ logits,
                                                                        const float* __restrict__ b_gate, int T, int E,
                                                                        float* __restrict__ partial) {
-    extern __shared__ float acc[];                   // [kAuxWarps][E]
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int i = threadIdx.x; i < kAuxWarps * E; i += blockDim.x) acc[i] = 0.0f;
+    extern __shared__ float acc[];                   // [warps][E]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
+    for (int i = threadIdx.x; i < warps * E; i += blockDim.x) acc[i] = 0.0f;
     __syncthreads();
     float* mine = acc + warp * E;
     int t0, t1;
@@ -66,47 +68,55 @@ __global__ void __launch_bounds__(kAuxWarps * 32) aux_prob_sums_kernel(const flo
     __syncthreads();
     for (int e = threadIdx.x; e < E; e += blockDim.x) {
         float total = 0.0f;
-        for (int w = 0; w < kAuxWarps; ++w) total += acc[w * E + e];
+        for (int w = 0; w < warps; ++w) total += acc[w * E + e];
         partial[(int64_t)blockIdx.x * E + e] = total;
     }
 }
 
-// loss = coef * E * sum_e f_e P_e   (one block; thread e owns expert e, e + 1024 never exists)
+// loss = coef * E * sum_e f_e P_e   (one block).  Thread (g, e) adds the chunks g, g + groups, ... of expert e in order
+// (neighbouring threads read neighbouring experts), thread e then adds its groups in order; a fixed tree over the experts.
 __global__ void __launch_bounds__(1024) aux_loss_final_kernel(const float* __restrict__ partial,
                                                               const int32_t* __restrict__ counts_chosen, int chunks, int T,
                                                               int E, int k, float coef, float* __restrict__ loss) {
+    __shared__ float part[1024];
     __shared__ float term[1024];
-    const int e = threadIdx.x;
-    float v = 0.0f;
-    if (e < E) {
-        float P = 0.0f;
-        for (int i = 0; i < chunks; ++i) P += partial[(int64_t)i * E + e];
-        v = ((float)counts_chosen[e] / ((float)T * (float)k)) * (P / (float)T);
+    const int groups = 1024 / E, g = threadIdx.x / E, e = threadIdx.x - g * E;      // E <= 1024: at least one group
+    if (g < groups) {
+        float acc = 0.0f;
+        for (int i = g; i < chunks; i += groups) acc += partial[(int64_t)i * E + e];
+        part[g * E + e] = acc;
     }
-    term[e] = v;
     __syncthreads();
-    for (int half = 512; half > 0; half >>= 1) {      // fixed tree
-        if (e < half) term[e] += term[e + half];
+    float v = 0.0f;
+    if ((int)threadIdx.x < E) {
+        float P = 0.0f;
+        for (int q = 0; q < groups; ++q) P += part[q * E + threadIdx.x];
+        v = ((float)counts_chosen[threadIdx.x] / ((float)T * (float)k)) * (P / (float)T);
+    }
+    term[threadIdx.x] = v;
+    __syncthreads();
+    for (int half = 512; half > 0; half >>= 1) {
+        if ((int)threadIdx.x < half) term[threadIdx.x] += term[threadIdx.x + half];
         __syncthreads();
     }
-    if (e == 0) loss[0] = coef * (float)E * term[0];
+    if (threadIdx.x == 0) loss[0] = coef * (float)E * term[0];
 }
 
 // Softmax-over-k backward (as in the plain gate backward) plus the gradient of the load-balancing loss.
 template <typename T>
-__global__ void __launch_bounds__(kAuxWarps * 32) gate_bwd_aux_kernel(float* __restrict__ dp, const float* __restrict__ topk_w,
+__global__ void __launch_bounds__(256) gate_bwd_aux_kernel(float* __restrict__ dp, const float* __restrict__ topk_w,
                                                                       const int32_t* __restrict__ topk_idx,
                                                                       const int32_t* __restrict__ counts_chosen,
                                                                       const float* __restrict__ logits,
                                                                       const float* __restrict__ b_gate, float coef,
                                                                       T* __restrict__ dlogits, float* __restrict__ aux_partial,
                                                                       int n_tokens, int E, int width, int ld, int k) {
-    extern __shared__ float smem[];                  // [kAuxWarps][E] column sums, [kAuxWarps][E] the row being built, [E] f
+    extern __shared__ float smem[];                  // [warps][E] column sums, [warps][E] the row being built, [E] f
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
     float* acc = smem;
-    float* rows = smem + kAuxWarps * E;
-    float* f = rows + kAuxWarps * E;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int i = threadIdx.x; i < kAuxWarps * E; i += blockDim.x) acc[i] = 0.0f;
+    float* rows = smem + warps * E;
+    float* f = rows + warps * E;
+    for (int i = threadIdx.x; i < warps * E; i += blockDim.x) acc[i] = 0.0f;
     const float inv_nk = 1.0f / ((float)n_tokens * (float)k);
     for (int e = threadIdx.x; e < E; e += blockDim.x) f[e] = (float)counts_chosen[e] * inv_nk;
     __syncthreads();
@@ -151,7 +161,7 @@ __global__ void __launch_bounds__(kAuxWarps * 32) gate_bwd_aux_kernel(float* __r
     __syncthreads();
     for (int e = threadIdx.x; e < E; e += blockDim.x) {
         float total = 0.0f;
-        for (int w = 0; w < kAuxWarps; ++w) total += acc[w * E + e];
+        for (int w = 0; w < warps; ++w) total += acc[w * E + e];
         aux_partial[(int64_t)blockIdx.x * E + e] = total;
     }
 }
@@ -161,8 +171,9 @@ __global__ void __launch_bounds__(kAuxWarps * 32) gate_bwd_aux_kernel(float* __r
 cudaError_t launch_aux_loss(const float* logits, const float* b_gate, const int32_t* counts_chosen, int T, int E, int k,
                             float coef, float* partial, float* loss, cudaStream_t stream) {
     if (T == 0) return cudaMemsetAsync(loss, 0, sizeof(float), stream);
-    aux_prob_sums_kernel<<<kColsumChunks, kAuxWarps * 32, sizeof(float) * kAuxWarps * E, stream>>>(logits, b_gate, T, E, partial);
-    aux_loss_final_kernel<<<1, 1024, 0, stream>>>(partial, counts_chosen, kColsumChunks, T, E, k, coef, loss);
+    const int warps = aux_warps(E);
+    aux_prob_sums_kernel<<<kAuxChunks, warps * 32, sizeof(float) * warps * E, stream>>>(logits, b_gate, T, E, partial);
+    aux_loss_final_kernel<<<1, 1024, 0, stream>>>(partial, counts_chosen, kAuxChunks, T, E, k, coef, loss);
     return cudaGetLastError();
 }
 
@@ -170,13 +181,14 @@ cudaError_t launch_gate_bwd_aux(float* dp, const Tables& tb, void* dlogits, cons
                                 float coef, float* aux_partial, int T, int E, int width, int ld, int k, int dtype,
                                 cudaStream_t stream) {
     if (T == 0) return cudaSuccess;
-    const size_t smem = sizeof(float) * (2 * kAuxWarps + 1) * E;      // at most 36 KB (E <= 1024)
+    const int warps = aux_warps(E);
+    const size_t smem = sizeof(float) * (2 * warps + 1) * E;          // at most 36 KB (E <= 1024)
     if (dtype == BIGMAC_BF16)
-        gate_bwd_aux_kernel<__nv_bfloat16><<<kColsumChunks, kAuxWarps * 32, smem, stream>>>(
+        gate_bwd_aux_kernel<__nv_bfloat16><<<kAuxChunks, warps * 32, smem, stream>>>(
             dp, tb.topk_w, tb.topk_idx, tb.counts_chosen, logits, b_gate, coef, (__nv_bfloat16*)dlogits, aux_partial, T, E,
             width, ld, k);
     else
-        gate_bwd_aux_kernel<float><<<kColsumChunks, kAuxWarps * 32, smem, stream>>>(
+        gate_bwd_aux_kernel<float><<<kAuxChunks, warps * 32, smem, stream>>>(
             dp, tb.topk_w, tb.topk_idx, tb.counts_chosen, logits, b_gate, coef, (float*)dlogits, aux_partial, T, E, width, ld, k);
     return cudaGetLastError();
 }

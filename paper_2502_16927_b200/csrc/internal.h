@@ -148,18 +148,19 @@ cudaError_t launch_gate_bwd(float* dp, const Tables& tb, void* dlogits, int T, i
                             int dtype, cudaStream_t stream);
 // Load-balancing loss (Table 5; conventional form, the paper prints none):
 //   L_aux = coef * E * sum_e f_e P_e,  f_e = counts_chosen[e] / (T k),  P_e = mean_t softmax_E(logits[t,:] + b_gate)[e].
-// Forward: loss[0] = L_aux; `partial` holds kColsumChunks * E floats of scratch.  Deterministic summation order.
+// Forward: loss[0] = L_aux; `partial` holds kAuxChunks * E floats of scratch.  Deterministic summation order.
+constexpr int kAuxChunks = 1184;
 cudaError_t launch_aux_loss(const float* logits, const float* b_gate, const int32_t* counts_chosen, int T, int E, int k,
                             float coef, float* partial, float* loss, cudaStream_t stream);
 // launch_gate_bwd plus dL_aux/dl: dlogits[t,e] = (top-k part) + (coef E / T) p[t,e] (f_e - sum_j f_j p[t,j]); the
-// column sums of the second term go to aux_partial [kColsumChunks, E] for launch_gate_colsum.
+// column sums of the second term go to aux_partial [kAuxChunks, E] for launch_gate_colsum.
 cudaError_t launch_gate_bwd_aux(float* dp, const Tables& tb, void* dlogits, const float* logits, const float* b_gate,
                                 float coef, float* aux_partial, int T, int E, int width, int ld, int k, int dtype,
                                 cudaStream_t stream);
 // db[e] (+)= sum over the slots routed to e of dl_slot[slot] (the fp32 per-slot gate gradients launch_gate_bwd
 // leaves in dp); `partial` holds kColsumChunks * E floats of scratch.  Deterministic summation order.
 constexpr int kColsumChunks = 296;
-// aux_partial (nullable): a second [kColsumChunks, E] array of partial column sums added in (launch_gate_bwd_aux).
+// aux_partial (nullable): a second array, [kAuxChunks, E], of partial column sums added in (launch_gate_bwd_aux).
 cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db, float* partial, int64_t N, int E,
                                bool accumulate, cudaStream_t stream, const float* aux_partial = nullptr);
 // Sum the `parts` fp32 partial results ws[s][m][n] of a split contraction in the order s = 0, 1, ... and write

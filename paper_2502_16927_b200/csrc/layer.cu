@@ -25,8 +25,8 @@ struct Buffers {
     void* dz;            // [P,h]: its own buffer when sigma' is saved as bytes, else written over sigma'
     void* dcat;          // [T, r + E64]: dx' in columns [0, r), the dense gate gradient dl in columns [r, r + E64)
     void *dx_lo, *dlogits;                               // views into dcat (row stride r + E64)
-    float* colsum_part;  // [2, kColsumChunks, E]: partial column sums of the top-k part and of the load-balancing part
-    float* aux_part;     // [kColsumChunks, E] forward scratch of the load-balancing loss
+    float* colsum_part;  // [kColsumChunks + kAuxChunks, E]: partial column sums of the top-k part, then of the load-balancing part
+    float* aux_part;     // [kAuxChunks, E] forward scratch of the load-balancing loss
     float* aux_loss;     // [1] saved: L_aux of the batch
     float* logits_saved; // [T,E] saved copy of the gate logits (only with a load-balancing loss)
     float* splitk_ws;    // fp32 partial results of the split weight-gradient contractions
@@ -89,7 +89,7 @@ void carve_saved(Carver& cv, const Dims& m, Buffers& b, bool with_z) {
 void carve_route_scratch(Carver& cv, const Dims& m, Buffers& b) {
     b.logits = cv.take<float>((size_t)m.T * m.E);
     b.tb.block_counts = cv.take<int32_t>((size_t)(sort_blocks(m.N) + 1) * m.E);
-    b.aux_part = m.aux > 0 ? cv.take<float>((size_t)kColsumChunks * m.E) : nullptr;
+    b.aux_part = m.aux > 0 ? cv.take<float>((size_t)kAuxChunks * m.E) : nullptr;
 }
 
 void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
@@ -102,7 +102,7 @@ void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
     b.dx_lo = m.cdac ? nullptr : b.dcat;
     b.dlogits = (b.dcat && !m.cdac) ? (char*)b.dcat + (size_t)m.r * es : b.dcat;
     b.dp = cv.take<float>(m.N);
-    b.colsum_part = cv.take<float>((size_t)2 * kColsumChunks * m.E);
+    b.colsum_part = cv.take<float>((size_t)(kColsumChunks + kAuxChunks) * m.E);
     // fp32 partial results: of the split dense contractions, and of the parts of long experts in dW1 / dW2
     const size_t dense_ws = (size_t)kMaxSplitK * m.ldcat * m.d * sizeof(float);
     const size_t expert_ws = m.dtype == BIGMAC_BF16 ? gemm_tc_groupk_ws_bytes(m.r, m.h, m.E) : 0;

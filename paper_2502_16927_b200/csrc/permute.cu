@@ -197,16 +197,16 @@ __global__ void __launch_bounds__(256) colsum_slots_kernel(const float* __restri
 }
 
 // One warp per column: lane l adds chunks l, l + 32, ... in order, then a fixed shuffle tree adds the lanes.
-// `partial2` (nullable): a second array of the same shape, added chunk by chunk.
+// `partial2` (nullable): a second array with chunks2 rows, added after the first.
 __global__ void __launch_bounds__(256) colsum_final_kernel(const float* __restrict__ partial, const float* __restrict__ partial2,
-                                                           float* __restrict__ out, int chunks, int cols, int accumulate) {
+                                                           float* __restrict__ out, int chunks, int chunks2, int cols,
+                                                           int accumulate) {
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (c >= cols) return;
     float total = 0.0f;
-    for (int i = lane; i < chunks; i += 32) {
-        total += partial[(int64_t)i * cols + c];
-        if (partial2) total += partial2[(int64_t)i * cols + c];
-    }
+    for (int i = lane; i < chunks; i += 32) total += partial[(int64_t)i * cols + c];
+    if (partial2)
+        for (int i = lane; i < chunks2; i += 32) total += partial2[(int64_t)i * cols + c];
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
     if (lane == 0) out[c] = accumulate ? out[c] + total : total;
@@ -287,7 +287,7 @@ cudaError_t launch_gate_bwd(float* dp, const Tables& tb, void* dlogits, int T, i
 cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db, float* partial, int64_t N, int E,
                                bool accumulate, cudaStream_t stream, const float* aux_partial) {
     colsum_slots_kernel<<<kColsumChunks, 256, sizeof(float) * 8 * E, stream>>>(dl_slot, tb.topk_idx, partial, N, E);
-    colsum_final_kernel<<<(unsigned)((E + 7) / 8), 256, 0, stream>>>(partial, aux_partial, db, kColsumChunks, E, accumulate);
+    colsum_final_kernel<<<(unsigned)((E + 7) / 8), 256, 0, stream>>>(partial, aux_partial, db, kColsumChunks, kAuxChunks, E, accumulate);
     return cudaGetLastError();
 }
 

@@ -114,3 +114,32 @@ def test_unsupported_combinations_and_bad_arguments():
         assert err.value.status == -1
     assert binding.bigmac_ep_buffer_bytes(h, 2) > 0
     binding.bigmac_layer_destroy(h)
+
+
+def test_one_rank_per_process_plumbing_with_a_group_of_one():
+    """The torch.distributed path (symmetric-memory exchange buffers, all_gather of the counts, collective barriers)
+    with a process group of one rank: the same calls a multi-GPU job makes, here addressing only local memory."""
+    import os
+    import torch
+    import torch.distributed as dist
+
+    w = wl.Workload("ep", T=600, d=128, r=64, h=128, E=8, k=2, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=79)
+    inp = skewed(w, 1.0)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(31500 + os.getpid() % 1000))
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        dev = to_device(w, inp)
+        rank = ep.EpProcessRank(w.d, w.r, w.h, w.E, w.k, w.T, w.dtype, w.act)
+        y = rank.forward(dev["x"], dev)
+        G = {"dw_gate": torch.empty_like(dev["w_gate"]), "dw_down": torch.empty_like(dev["w_down"]),
+             "dw_up": torch.empty_like(dev["w_up"]), "dw1": torch.empty_like(dev["w1"]), "dw2": torch.empty_like(dev["w2"]),
+             "db_gate": torch.empty(w.E, dtype=torch.float32, device="cuda")}
+        dx = rank.backward(dev["x"], dev["dy"], dev, G)
+        torch.cuda.synchronize()
+        assert rank.status() == 0
+        got = {"y": to_numpy(y), "dx": to_numpy(dx), "counts_all": to_numpy(rank.rk.counts_all)}
+        got.update({key: to_numpy(val) for key, val in G.items()})
+        rank.close()
+    finally:
+        dist.destroy_process_group()
+    compare(w, inp, got)
