@@ -201,7 +201,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         for (int c = 0; c < BM / 64; ++c) tma_load_2d_pair(a_dst + c * CHUNK_BYTES, &map_a, bar, my_m0 + 64 * c, k0);
                     }
                     if (B_KMAJOR) {
-                        tma_load_2d_pair(b_dst, &map_b, bar, k0, tl.expert * p.b_rows_per_expert + my_n0);
+                        if (p.n_split >= 0 && tl.n0 >= p.n_split) tma_load_2d_pair(b_dst, &map_b2, bar, k0, my_n0 - p.n_split);
+                        else tma_load_2d_pair(b_dst, &map_b, bar, k0, tl.expert * p.b_rows_per_expert + my_n0);
                     } else {
                         const bool second = p.b2_first_kb >= 0 && kb >= p.b2_first_kb;     // dense only
                         const CUtensorMap* mb = second ? &map_b2 : &map_b;
@@ -331,7 +332,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         tma_store_commit();
                     }
                 } else if (row_ok) {
-                    store_row_chunk(p, v, row_off, col0, vec_ok);
+                    if (p.n_split >= 0 && tl.n0 >= p.n_split) {          // second output: fp32, its own leading dimension
+                        TcParams p2 = p;
+                        p2.C = p.C2; p2.ldc = p.ldc2; p2.N = p.N2; p2.out_f32 = 1; p2.epilogue = EPI_NONE; p2.accumulate = 0;
+                        const bool vec2 = (p.ldc2 % 8 == 0) && (((uintptr_t)p.C2) % 32 == 0);
+                        store_row_chunk(p2, v, (int64_t)row * p.ldc2, col0 - p.n_split, vec2);
+                    } else {
+                        store_row_chunk(p, v, row_off, col0, vec_ok);
+                    }
                 }
             }
         }
@@ -384,11 +392,19 @@ cudaError_t dispatch_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
         ok &= make_map(&mb, g.B, (uint64_t)g.N, g.group == GROUP_M ? rows_per * E : (uint64_t)g.K, (uint64_t)g.ldb, 64, BK);
     CUtensorMap mb2 = mb;
     p.b2_first_kb = -1;
-    if (g.B2) {
+    if (g.B2 && !g.C2) {
         if (g.b_kmajor || g.group != GROUP_NONE || g.b2_first_k % BK) return cudaErrorInvalidValue;
         ok &= make_map(&mb2, g.B2, (uint64_t)g.N, (uint64_t)(g.K - g.b2_first_k), (uint64_t)g.ldb2, 64, BK);
         ok &= make_map(&mb, g.B, (uint64_t)g.N, (uint64_t)g.b2_first_k, (uint64_t)g.ldb, 64, BK);
         p.b2_first_kb = g.b2_first_k / BK;
+    }
+    p.n_split = -1;
+    if (g.C2) {      // second K-major B tensor feeding a second (fp32) output
+        if (!g.b_kmajor || g.group != GROUP_NONE || g.n_split % BN || TMA_EPI || g.B2 == nullptr || g.split_k > 1)
+            return cudaErrorInvalidValue;
+        ok &= make_map(&mb2, g.B2, (uint64_t)g.K, (uint64_t)g.N2, (uint64_t)g.ldb2, BK, BH);
+        ok &= make_map(&mb, g.B, (uint64_t)g.K, (uint64_t)g.n_split, (uint64_t)g.ldb, BK, BH);
+        p.n_split = g.n_split; p.C2 = g.C2; p.ldc2 = g.ldc2; p.N2 = g.N2;
     }
     if (TMA_EPI && !tma_epilogue_possible(g)) return cudaErrorInvalidValue;
     CUtensorMap mc = ma, mz = ma;
@@ -421,6 +437,7 @@ cudaError_t dispatch_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
 bool gemm_tc_pair_supported(const GemmArgs& g) {
     if (g.N < 256) return false;                                  // narrow outputs stay on the one-CTA kernel
     if (g.group == GROUP_M && !g.poffsets) return false;
+    if (g.C2 && (g.n_split % 256 || !g.b_kmajor || !g.a_kmajor)) return false;   // second output: whole tiles of it
     return true;
 }
 
@@ -434,7 +451,7 @@ bool gemm_tc_pair_preferred(const GemmArgs& g) {
 
 cudaError_t gemm_tc_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
-    const bool staged = tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 &&
+    const bool staged = !g.C2 && tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 &&
                         (g.epilogue != EPI_DACT || g.group != GROUP_K);
     // 32 KB per stage and CTA: 5 stages beside the 64 KB store staging (4 if the expert tables are long), 6 without it
     if (!staged) return dispatch_pair<256, 6, false>(g, status, stream);
