@@ -46,6 +46,7 @@ class Routing:
     slot_of_row: np.ndarray   # [T*k] int32 (-1 past the kept rows)
     keep: Optional[np.ndarray] = None            # [T*k] uint8, None = dropless
     counts_chosen: Optional[np.ndarray] = None   # [E] int32: slots that chose e, before dropping
+    gate_low: bool = False                       # the gate read x' (w_gate is [E,r]) instead of x
 
 
 def gate_logits(x, w_gate, b_gate=None) -> np.ndarray:
@@ -55,6 +56,18 @@ def gate_logits(x, w_gate, b_gate=None) -> np.ndarray:
     E = w_gate.shape[0]
     out = np.empty((T, E), dtype=np.float64)
     lib().oracle_gate_logits(_p(x), _p(w_gate), _p(b), C.c_int(T), C.c_int(d), C.c_int(E), _p(out))
+    return out
+
+
+def gate_logits_low(x, w_down, w_gate, b_gate=None, round_x_lo_bf16: bool = False) -> np.ndarray:
+    """Gate logits when the gate reads x' = x W'_down (w_gate [E,r]); x' optionally rounded to bf16 first."""
+    x, w_down, w_gate = _f32(x), _f32(w_down), _f32(w_gate)
+    b = None if b_gate is None else _f32(b_gate)
+    T, d = x.shape
+    E, r = w_gate.shape
+    out = np.empty((T, E), dtype=np.float64)
+    lib().oracle_gate_logits_low(_p(x), _p(w_down), _p(w_gate), _p(b), C.c_int(T), C.c_int(d), C.c_int(r), C.c_int(E),
+                                 C.c_int(int(round_x_lo_bf16)), _p(out))
     return out
 
 
@@ -111,15 +124,19 @@ def aux_loss(logits: np.ndarray, topk_idx: np.ndarray, alpha: float, want_grad: 
     return loss.value, grad
 
 
-def route(inp: Dict[str, np.ndarray], k: int, capacity_factor: float = 0.0) -> Routing:
-    logits = gate_logits(inp["x"], inp["w_gate"], inp.get("b_gate"))
+def route(inp: Dict[str, np.ndarray], k: int, capacity_factor: float = 0.0, gate_low: bool = False,
+          round_x_lo_bf16: bool = False) -> Routing:
+    if gate_low:
+        logits = gate_logits_low(inp["x"], inp["w_down"], inp["w_gate"], inp.get("b_gate"), round_x_lo_bf16)
+    else:
+        logits = gate_logits(inp["x"], inp["w_gate"], inp.get("b_gate"))
     idx, p = topk(logits, k)
     T, E = logits.shape
     if capacity_factor > 0:
         chosen, counts, offsets, ros, sor, keep = tables_capacity(idx, E, capacity_rows(T, k, E, capacity_factor))
-        return Routing(logits, idx, p, counts, offsets, ros, sor, keep, chosen)
+        return Routing(logits, idx, p, counts, offsets, ros, sor, keep, chosen, gate_low)
     counts, offsets, ros, sor = tables(idx, E)
-    return Routing(logits, idx, p, counts, offsets, ros, sor, None, counts.copy())
+    return Routing(logits, idx, p, counts, offsets, ros, sor, None, counts.copy(), gate_low)
 
 
 def _dims(inp):
@@ -182,7 +199,7 @@ def backward_tokens(inp, routing: Routing, act: int, tokens=None, decide_bf16: b
                                  _p(_f32(inp["w_up"])), _p(routing.topk_idx), _p(routing.topk_p), _p(tok),
                                  C.c_int(n), C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(E), C.c_int(k),
                                  C.c_int(act), C.c_int(int(decide_bf16)), _p(dx), _p(dx_lo), _p(dlogit), _p(dy_lo),
-                                 _p(routing.keep))
+                                 _p(routing.keep), C.c_int(int(routing.gate_low)))
     return {"dx": dx, "dx_lo": dx_lo, "dlogit": dlogit, "dy_lo": dy_lo}
 
 
@@ -228,6 +245,13 @@ def backward_full(inp, routing: Routing, act: int, experts=None, decide_bf16: bo
     out = {"y": fwd["y"], "y_lo": fwd["y_lo"], "x_lo": fwd["x_lo"], "dx": bwd["dx"], "dx_lo": bwd["dx_lo"],
            "dlogit": bwd["dlogit"], "dw_up": dw_up, "dw_down": dw_down, "dw_gate": dw_gate,
            "db_gate": db_gate, "dw1": dw1, "dw2": dw2}
+    if routing.gate_low:
+        # the gate read x': dW_g [E,r] = dl^T x' with dl scattered to its dense [T,E] form (a library matmul); dx' above
+        # already holds the gate's share, so dw_down is complete
+        assert aux_alpha == 0
+        dl_dense = np.zeros((T, E))
+        np.put_along_axis(dl_dense, routing.topk_idx.astype(np.int64), bwd["dlogit"], axis=1)
+        out["dw_gate"] = dl_dense.T @ fwd["x_lo"]
     if aux_alpha > 0:
         loss, dl_aux = aux_loss(routing.logits, routing.topk_idx, aux_alpha)
         x64 = np.asarray(inp["x"], dtype=np.float64)

@@ -155,6 +155,24 @@ void oracle_gate_logits(const float* x, const float* w_gate, const float* b_gate
     }
 }
 
+// Variant (the choice the text after Eq. 2 mentions and sets aside): the gate reads the low-width token,
+// l[t,e] = sum_c x'[t,c] W_g[e,c] (+ b_g[e]) with W_g [E,r] and x' = x W'_down.  round_bf16: x' is rounded to bf16
+// first, as the BF16 kernels hold it, so that the discrete top-k choice is taken on the same numbers on both sides.
+void oracle_gate_logits_low(const float* x, const float* w_down, const float* w_gate, const float* b_gate, int T, int d,
+                            int r, int E, int round_x_lo_bf16, double* logits) {
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < T; ++t) {
+        std::vector<double> xt(d), x_lo(r);
+        widen(x + (size_t)t * d, d, xt.data());
+        matvec(xt.data(), w_down, r, d, x_lo.data());
+        if (round_x_lo_bf16)
+            for (int c = 0; c < r; ++c) x_lo[c] = round_bf16(x_lo[c]);
+        matvec(x_lo.data(), w_gate, E, r, logits + (size_t)t * E);
+        if (b_gate)
+            for (int e = 0; e < E; ++e) logits[(size_t)t * E + e] += (double)b_gate[e];
+    }
+}
+
 // Top-k set T of Eq. 2 and the gate values p_i: experts ordered by (logit descending, id ascending),
 // first k kept in that order; p = softmax over the k kept logits (so the p of a token sum to 1).
 void oracle_topk(const double* logits, int T, int E, int k, int32_t* topk_idx, double* topk_p) {
@@ -330,13 +348,13 @@ void oracle_forward_grouped(const float* x, const float* w_down, const float* w1
 // discrete top-k choice carries no gradient, the gate weights do).  Per selected token i (id t):
 //   dy' = dy W_up ; per slot j: dp_j = <dy', u_j>, du_j = p_j dy', da_j = du_j W2, dz_j = da_j * sigma'(z_j),
 //   dx' = sum_j dz_j W1 ; softmax-over-k: g = sum_i p_i dp_i, dl_j = p_j (dp_j - g) ;
-//   dx = dx' W_down + sum_j dl_j W_g[e_j].
+//   dx = dx' W_down + sum_j dl_j W_g[e_j]     (gate on x';  with gate_low: dx = (dx' + sum_j dl_j W_g[e_j]) W_down).
 // Outputs (any may be NULL) are indexed by position in `tokens`.
 void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate, const float* w_down,
                             const float* w1, const float* w2, const float* w_up, const int32_t* topk_idx,
                             const double* topk_p, const int32_t* tokens, int n, int d, int r, int h, int E,
                             int k, int act, int decide_bf16, double* dx_out, double* dx_lo_out,
-                            double* dlogit_out, double* dy_lo_out, const uint8_t* keep) {
+                            double* dlogit_out, double* dy_lo_out, const uint8_t* keep, int gate_low) {
     (void)E;
 #pragma omp parallel for schedule(dynamic, 4)
     for (int i = 0; i < n; ++i) {
@@ -367,12 +385,20 @@ void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate
         double g = 0.0;
         for (int j = 0; j < k; ++j) g += topk_p[(size_t)t * k + j] * dp[j];
         for (int j = 0; j < k; ++j) dl[j] = topk_p[(size_t)t * k + j] * (dp[j] - g);
-        matvec_t(dx_lo.data(), w_down, r, d, dx.data());
-        for (int j = 0; j < k; ++j) {
-            const float* wg = w_gate + (size_t)topk_idx[(size_t)t * k + j] * d;
-            for (int c = 0; c < d; ++c) gate_part[c] += dl[j] * (double)wg[c];
+        if (gate_low) {       // the gate read x' (W_g is [E,r]): its gradient joins dx' before the descend projection
+            for (int j = 0; j < k; ++j) {
+                const float* wg = w_gate + (size_t)topk_idx[(size_t)t * k + j] * r;
+                for (int c = 0; c < r; ++c) dx_lo[c] += dl[j] * (double)wg[c];
+            }
         }
-        for (int c = 0; c < d; ++c) dx[c] += gate_part[c];
+        matvec_t(dx_lo.data(), w_down, r, d, dx.data());
+        if (!gate_low) {
+            for (int j = 0; j < k; ++j) {
+                const float* wg = w_gate + (size_t)topk_idx[(size_t)t * k + j] * d;
+                for (int c = 0; c < d; ++c) gate_part[c] += dl[j] * (double)wg[c];
+            }
+            for (int c = 0; c < d; ++c) dx[c] += gate_part[c];
+        }
         if (dx_out) std::memcpy(dx_out + (size_t)i * d, dx.data(), sizeof(double) * d);
         if (dx_lo_out) std::memcpy(dx_lo_out + (size_t)i * r, dx_lo.data(), sizeof(double) * r);
         if (dlogit_out) std::memcpy(dlogit_out + (size_t)i * k, dl.data(), sizeof(double) * k);

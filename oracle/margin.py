@@ -9,7 +9,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from . import gate_logits
+from . import gate_logits, gate_logits_low
 
 
 def min_topk_gap(logits: np.ndarray, k: int) -> np.ndarray:
@@ -22,15 +22,20 @@ def min_topk_gap(logits: np.ndarray, k: int) -> np.ndarray:
     return np.min(top[:, :-1] - top[:, 1:], axis=1)
 
 
-def enforce_margin(workload, inp, margin: float = 1e-3, max_attempts: int = 64) -> int:
-    """Redraw rows of inp["x"] in place until every token clears the margin; returns rows redrawn."""
+def enforce_margin(workload, inp, margin: float = 1e-3, max_attempts: int = 64, gate_low: bool = False,
+                   round_x_lo_bf16: bool = False) -> int:
+    """Redraw rows of inp["x"] in place until every token clears the margin; returns rows redrawn.
+    gate_low: the logits are those of the gate that reads x' (w_gate [E,r])."""
     from paper_2502_16927_b200.workloads import redraw_rows
 
     x = inp["x"]
     bad = np.arange(x.shape[0])
     total = 0
     for attempt in range(1, max_attempts + 1):
-        logits = gate_logits(x[bad], inp["w_gate"], inp.get("b_gate"))
+        if gate_low:
+            logits = gate_logits_low(x[bad], inp["w_down"], inp["w_gate"], inp.get("b_gate"), round_x_lo_bf16)
+        else:
+            logits = gate_logits(x[bad], inp["w_gate"], inp.get("b_gate"))
         bad = bad[min_topk_gap(logits, workload.k) < margin]
         if bad.size == 0:
             return total
