@@ -82,6 +82,11 @@ typedef enum {
  * out at run time, long experts contracted in parts) whatever the problem size.  Without the flag that kernel is
  * used when there is enough work per SM pair for it to pay, else the statically scheduled one. */
 #define BIGMAC_FLAG_DYNAMIC_WGRAD 4u
+/* The gate reads the low-width token x' = x W'_down instead of x (the alternative the text after Eq. 2 mentions and
+ * sets aside): l = x' w_gate^T (+ b_gate) with w_gate and dw_gate of shape [E,r].  In the backward pass the gate's
+ * gradient joins dx' before the descend projection.  Not together with BIGMAC_FLAG_CDAC (there x' is x:
+ * INVALID_ARG) nor with a load-balancing loss (UNSUPPORTED). */
+#define BIGMAC_FLAG_GATE_LOW 8u
 
 /* The two training-recipe settings of the paper's pre-training configuration (Table 5: capacity factor 1.2,
  * load-balancing loss with coefficient 0.001).  Both are off (0) in the layer the paper advocates and measures,
@@ -108,7 +113,7 @@ typedef struct {
 } bigmac_config_t;
 
 typedef struct {
-    const void *w_gate;   /* [E,d]   */
+    const void *w_gate;   /* [E,d]   ([E,r] with BIGMAC_FLAG_GATE_LOW) */
     const float *b_gate;  /* [E] fp32, or NULL */
     const void *w_down;   /* [r,d]   W'_down of Eq. 2 */
     const void *w1;       /* [E,h,r] W_{i,up} of Eq. 4 */
@@ -217,7 +222,8 @@ const char *bigmac_status_string(int status);
  * `saved` (and, across the three backward calls, `scratch`) must keep their contents between the calls of a step.
  * The gradients of the shared matrices that the backward returns are this rank's share (the sum over its own
  * tokens): the caller adds them over the ranks, as for any data-parallel layer; dw1 / dw2 are complete.
- * Not supported together with a capacity factor, a load-balancing loss or BIGMAC_FLAG_CDAC (BIGMAC_ERR_UNSUPPORTED). */
+ * Not supported together with a capacity factor, a load-balancing loss, BIGMAC_FLAG_CDAC or BIGMAC_FLAG_GATE_LOW
+ * (BIGMAC_ERR_UNSUPPORTED). */
 #define BIGMAC_EP_MAX_RANKS 8
 typedef struct {
     int32_t rank, size;                 /* 0 <= rank < size <= BIGMAC_EP_MAX_RANKS, E % size == 0 */

@@ -39,6 +39,7 @@ struct Dims {
     int z_es;  // bytes per saved sigma'(z) element: 1 on the tensor-core path (quantised), else the dtype's
     bool cdac; // Eq. 3 layer: no descend / ascend projections, r == d
     int ldcat; // row stride of dcat: r + E64, or E64 alone without projections (dx' then goes straight to dx)
+    bool gate_low; // the gate reads x' (w_gate [E,r])
     int cap;   // rows an expert keeps at most (Table 5's capacity factor); kNoCapacity = dropless
     float aux; // coefficient of the load-balancing loss (Table 5), 0 = none
 };
@@ -52,6 +53,7 @@ Dims dims_of(const bigmac_layer* L, int T) {
     m.z_es = sigma_as_bytes(L) ? 1 : (int)esize(c.dtype);
     m.cdac = (c.flags & BIGMAC_FLAG_CDAC) != 0;
     m.ldcat = m.cdac ? m.E64 : m.r + m.E64;
+    m.gate_low = (c.flags & BIGMAC_FLAG_GATE_LOW) != 0;
     m.cap = kNoCapacity;
     if (c.capacity_factor > 0) {                     // C = ceil((f * (T k)) / E), evaluated in double in this order
         const double rows = std::ceil(c.capacity_factor * (double)m.N / (double)c.E);
@@ -185,8 +187,16 @@ int route_from_logits(const bigmac_layer* L, const Dims& m, const bigmac_weights
 int run_routing(const bigmac_layer* L, const Dims& m, const void* x, const bigmac_weights_t* W, Buffers& b,
                 cudaStream_t st) {
     GemmArgs g;
-    g.A = x; g.lda = m.d; g.B = W->w_gate; g.ldb = m.d; g.C = b.logits; g.ldc = m.E;
-    g.M = m.T; g.N = m.E; g.K = m.d; g.out_f32 = true;
+    if (m.gate_low) {                                // the gate reads x': descend first, logits from its stored value
+        GemmArgs q;
+        q.A = x; q.lda = m.d; q.B = W->w_down; q.ldb = m.d; q.C = b.x_lo; q.ldc = m.r;
+        q.M = m.T; q.N = m.r; q.K = m.d;
+        BIGMAC_TRY(gemm(L, G_DESCEND, q, st));
+        g.A = b.x_lo; g.lda = m.r; g.B = W->w_gate; g.ldb = m.r; g.K = m.r;
+    } else {
+        g.A = x; g.lda = m.d; g.B = W->w_gate; g.ldb = m.d; g.K = m.d;
+    }
+    g.C = b.logits; g.ldc = m.E; g.M = m.T; g.N = m.E; g.out_f32 = true;
     BIGMAC_TRY(gemm(L, G_LOGITS, g, st));
     return route_from_logits(L, m, W, b, st);
 }
@@ -251,11 +261,14 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
     if (cfg->k > cfg->E) return BIGMAC_ERR_INVALID_ARG;
     if (cfg->dtype != BIGMAC_F32 && cfg->dtype != BIGMAC_BF16) return BIGMAC_ERR_INVALID_ARG;
     if (cfg->act < BIGMAC_ACT_RELU || cfg->act > BIGMAC_ACT_IDENTITY) return BIGMAC_ERR_INVALID_ARG;
-    if (cfg->flags & ~(BIGMAC_FLAG_SIMT_GEMM | BIGMAC_FLAG_CDAC | BIGMAC_FLAG_DYNAMIC_WGRAD)) return BIGMAC_ERR_INVALID_ARG;
+    if (cfg->flags & ~(BIGMAC_FLAG_SIMT_GEMM | BIGMAC_FLAG_CDAC | BIGMAC_FLAG_DYNAMIC_WGRAD | BIGMAC_FLAG_GATE_LOW))
+        return BIGMAC_ERR_INVALID_ARG;
     if ((cfg->flags & BIGMAC_FLAG_CDAC) && cfg->r != cfg->d) return BIGMAC_ERR_INVALID_ARG;
+    if ((cfg->flags & BIGMAC_FLAG_CDAC) && (cfg->flags & BIGMAC_FLAG_GATE_LOW)) return BIGMAC_ERR_INVALID_ARG;
     if (!(cfg->capacity_factor >= 0) || !(cfg->aux_loss_coef >= 0) || std::isinf(cfg->capacity_factor) ||
         std::isinf(cfg->aux_loss_coef))
         return BIGMAC_ERR_INVALID_ARG;
+    if ((cfg->flags & BIGMAC_FLAG_GATE_LOW) && cfg->aux_loss_coef > 0) return BIGMAC_ERR_UNSUPPORTED;
     if (cfg->E > kMaxExperts) return BIGMAC_ERR_UNSUPPORTED;
     if ((int64_t)cfg->max_tokens * cfg->k > (int64_t)1 << 30) return BIGMAC_ERR_UNSUPPORTED;
     const int vec = cfg->dtype == BIGMAC_BF16 ? 8 : 4;     // rows move as 16-byte vectors
@@ -345,7 +358,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     const bigmac_config_t& c = L->cfg;
 
     // A few tokens, inference: the whole forward in one cooperative kernel (weight streaming, no tensor cores)
-    if (!training && !m.cdac && m.cap == kNoCapacity && m.aux == 0 && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
+    if (!training && !m.cdac && !m.gate_low && m.cap == kNoCapacity && m.aux == 0 && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
         {
             Stage s(L, S_DECODE, st);
             BIGMAC_CUDA(launch_decode_forward(x, W, y, b.logits, (float*)b.xg, (float*)b.a, (float*)b.u, b.tb.topk_idx,
@@ -360,7 +373,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     }
     // F1 + F4 in one pass over x when the tile grid allows it: [x' | logits] = x [W'_down ; W_gate]^T, logits in fp32
     const int bn_desc = (m.r + m.E) >= 256 ? 256 : 128;
-    const bool fuse_gate = !m.cdac && c.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u && m.r % bn_desc == 0;
+    const bool fuse_gate = !m.cdac && !m.gate_low && c.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u && m.r % bn_desc == 0;
     if (fuse_gate) {
         GemmArgs g;
         g.A = x; g.lda = m.d; g.B = W->w_down; g.ldb = m.d; g.C = b.x_lo; g.ldc = m.r;
@@ -373,7 +386,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     }
     BIGMAC_TRY(export_routing(m, b, routing_out, st));
     if (m.cdac) b.x_lo = const_cast<void*>(x);                                    // Eq. 3: experts read the token itself
-    if (!fuse_gate && !m.cdac) {                                                  // F4 descend: x' = x W'_down
+    if (!fuse_gate && !m.cdac && !m.gate_low) {                                   // F4 descend: x' = x W'_down
         GemmArgs g;
         g.A = x; g.lda = m.d; g.B = W->w_down; g.ldb = m.d; g.C = b.x_lo; g.ldc = m.r;
         g.M = m.T; g.N = m.r; g.K = m.d;
@@ -538,6 +551,52 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     }
     // dx'[t] = sum_j dxg[row of slot (t,j)]   (the transpose of the dispatch gather)
     { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st, ldcat)); }
+    if (m.gate_low) {
+        // The gate read x': its gradient joins dx' (dx' += dl W_gate, W_gate [E,r]) before the descend projection;
+        // dW_gate = dl^T x'.
+        {
+            GemmArgs g;
+            g.A = b.dlogits; g.lda = ldcat; g.B = W->w_gate; g.ldb = m.r; g.b_kmajor = false; g.C = b.dx_lo; g.ldc = ldcat;
+            g.M = m.T; g.N = m.r; g.K = m.E; g.accumulate = true;
+            BIGMAC_TRY(gemm(L, G_DX_GATE, g, st));
+        }
+        {   // dx = dx' W_down
+            GemmArgs g;
+            g.A = b.dx_lo; g.lda = ldcat; g.B = W->w_down; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
+            g.M = m.T; g.N = m.d; g.K = m.r;
+            BIGMAC_TRY(gemm(L, G_DX, g, st));
+        }
+        if (G->dw_down) {   // dW_down[c',c] = sum_t dx'[t,c'] x[t,c]
+            GemmArgs g;
+            g.A = b.dx_lo; g.lda = ldcat; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
+            g.M = m.r; g.N = m.d; g.K = m.T;
+            if (fused) {
+                g.C = b.splitk_ws; g.ldc = m.d; g.out_f32 = true; g.split_k = choose_split_k(g.M, g.N, g.K);
+                BIGMAC_TRY(gemm(L, G_DW_DOWN, g, st));
+                Stage s(L, S_SPLITK_REDUCE, st);
+                BIGMAC_CUDA(launch_splitk_reduce(b.splitk_ws, g.split_k, m.r, m.d, G->dw_down, m.r, nullptr, 0, m.dtype, acc, st));
+            } else {
+                g.C = G->dw_down; g.ldc = m.d; g.accumulate = acc;
+                BIGMAC_TRY(gemm(L, G_DW_DOWN, g, st));
+            }
+        }
+        if (G->dw_gate) {   // dW_gate[e,c'] = sum_t dl[t,e] x'[t,c']
+            GemmArgs g;
+            g.A = b.dlogits; g.lda = ldcat; g.a_kmajor = false; g.B = b.x_lo; g.ldb = m.r; g.b_kmajor = false;
+            g.N = m.r; g.K = m.T;
+            if (fused) {
+                g.M = m.E64; g.C = b.splitk_ws; g.ldc = m.r; g.out_f32 = true; g.split_k = choose_split_k(g.M, g.N, g.K);
+                BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
+                Stage s(L, S_SPLITK_REDUCE, st);
+                BIGMAC_CUDA(launch_splitk_reduce(b.splitk_ws, g.split_k, m.E64, m.r, G->dw_gate, m.E, nullptr, 0, m.dtype, acc, st));
+            } else {
+                g.M = m.E; g.C = G->dw_gate; g.ldc = m.r; g.accumulate = acc;
+                BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
+            }
+        }
+        if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st, aux_part)); }
+        return BIGMAC_OK;
+    }
     if (fused) {
         {   // dx = [dx' | dl] [W_down ; W_gate]: one contraction over r + E
             GemmArgs g;
@@ -682,6 +741,7 @@ void carve_route_only(Carver& cv, const Dims& m, Buffers& b) {
     b.tb.n_tiles = cv.take<int32_t>(1);
     b.tb.counts_chosen = cv.take<int32_t>(m.E);
     b.aux_loss = cv.take<float>(1);
+    if (m.gate_low) b.x_lo = cv.take_bytes((size_t)m.T * m.r * esize(m.dtype));   // the gate reads x'
 }
 
 }  // namespace

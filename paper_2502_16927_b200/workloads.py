@@ -30,7 +30,7 @@ import numpy as np
 
 ACT_RELU, ACT_GELU_ERF, ACT_GELU_TANH, ACT_IDENTITY = 0, 1, 2, 3
 DTYPE_F32, DTYPE_BF16 = 0, 1
-FLAG_SIMT_GEMM, FLAG_CDAC, FLAG_DYNAMIC_WGRAD = 1, 2, 4
+FLAG_SIMT_GEMM, FLAG_CDAC, FLAG_DYNAMIC_WGRAD, FLAG_GATE_LOW = 1, 2, 4, 8
 
 
 @dataclass(frozen=True)
@@ -47,6 +47,7 @@ class Workload:
     seed: int
     gate_bias: str = "none"   # "none" | "zipf"  (b_g[e] = ln q_e, q_e ~ (e+1)^-1.1)
     cdac: bool = False        # the conventional fine-grained layer (Eq. 3): r == d, no w_down / w_up
+    gate_low: bool = False    # the gate reads x' (w_gate [E,r]) instead of x
 
     @property
     def N(self) -> int:
@@ -136,13 +137,14 @@ def make_inputs(w: Workload, with_dy: bool = True) -> Dict[str, Optional[np.ndar
     """Draw every tensor of one layer call.
 
     x, dy ~ N(0,1); weights ~ N(0, fan_in^-1/2), stored [out_features, in_features]:
-    w_gate [E,d], w_down [r,d], w1 [E,h,r], w2 [E,r,h], w_up [d,r].  b_gate is fp32 [E] or None.
+    w_gate [E,d] ([E,r] when the gate reads x'), w_down [r,d], w1 [E,h,r], w2 [E,r,h], w_up [d,r].  b_gate is fp32 [E] or None.
     The projection-free layer (cdac) has r == d and no w_down / w_up (None).
     """
     s, dt = w.seed, w.dtype
     out: Dict[str, Optional[np.ndarray]] = {
         "x": _normal(s, _TAGS["x"], 0, (w.T, w.d), 1.0, dt),
-        "w_gate": _normal(s, _TAGS["w_gate"], 0, (w.E, w.d), w.d ** -0.5, dt),
+        "w_gate": (_normal(s, _TAGS["w_gate"], 0, (w.E, w.r), w.r ** -0.5, dt) if w.gate_low
+                   else _normal(s, _TAGS["w_gate"], 0, (w.E, w.d), w.d ** -0.5, dt)),
         "w_down": None if w.cdac else _normal(s, _TAGS["w_down"], 0, (w.r, w.d), w.d ** -0.5, dt),
         "w1": _normal(s, _TAGS["w1"], 0, (w.E, w.h, w.r), w.r ** -0.5, dt),
         "w2": _normal(s, _TAGS["w2"], 0, (w.E, w.r, w.h), w.h ** -0.5, dt),

@@ -58,6 +58,8 @@ def make_layer(w, flags=0, max_tokens=None, capacity_factor=0.0, aux_loss_coef=0
 
     if w.cdac:
         flags |= wl.FLAG_CDAC
+    if w.gate_low:
+        flags |= wl.FLAG_GATE_LOW
     return binding.Layer(w.d, w.r, w.h, w.E, w.k, max_tokens or max(w.T, 1), w.dtype, w.act, flags,
                          capacity_factor=capacity_factor, aux_loss_coef=aux_loss_coef)
 
@@ -77,7 +79,7 @@ def empty_grads(w, dev, fill=None):
     import torch
 
     dt = torch.float32 if w.dtype == wl.DTYPE_F32 else torch.bfloat16
-    shapes = {"dw_gate": (w.E, w.d), "dw_down": (w.r, w.d), "dw1": (w.E, w.h, w.r), "dw2": (w.E, w.r, w.h),
+    shapes = {"dw_gate": (w.E, w.r if w.gate_low else w.d), "dw_down": (w.r, w.d), "dw1": (w.E, w.h, w.r), "dw2": (w.E, w.r, w.h),
               "dw_up": (w.d, w.r)}
     if w.cdac:
         del shapes["dw_down"], shapes["dw_up"]

@@ -28,14 +28,14 @@ def conditioned(w):
     return inp
 
 
-def check_routing(R, rt):
+def check_routing(R, rt, p_atol=2e-5):
     np.testing.assert_array_equal(to_numpy(R["topk_idx"]).reshape(rt.topk_idx.shape), rt.topk_idx)
     np.testing.assert_array_equal(to_numpy(R["counts"]), rt.counts)
     np.testing.assert_array_equal(to_numpy(R["offsets"]), rt.offsets)
     np.testing.assert_array_equal(to_numpy(R["row_of_slot"]), rt.row_of_slot)
     np.testing.assert_array_equal(to_numpy(R["slot_of_row"]), rt.slot_of_row)
     np.testing.assert_array_equal(to_numpy(R["counts_chosen"]), rt.counts_chosen)
-    np.testing.assert_allclose(to_numpy(R["topk_w"]).reshape(rt.topk_p.shape), rt.topk_p, rtol=0, atol=2e-5)
+    np.testing.assert_allclose(to_numpy(R["topk_w"]).reshape(rt.topk_p.shape), rt.topk_p, rtol=0, atol=p_atol)
 
 
 def run_full(w, inp, flags=0, capacity_factor=0.0, aux=0.0):
