@@ -134,10 +134,10 @@ cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaSt
 cudaError_t launch_dispatch(const void* src, void* grouped, const Tables& tb, int k, int width, int dtype,
                             int64_t max_prows, cudaStream_t stream);
 // dst[t,:] = sum_j w[t*k+j] * grouped[prow_of_slot[t*k+j],:]   (w == nullptr: unit weights), fp32 accumulation;
-// slots with prow_of_slot < 0 (dropped under a capacity limit) are left out of the sum.
+// with may_drop, slots with prow_of_slot < 0 (dropped under a capacity limit) are left out of the sum.
 // dst rows are `dst_ld` elements apart (0: dense, = width).
 cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const int32_t* prow_of_slot, int T,
-                           int k, int width, int dtype, cudaStream_t stream, int dst_ld = 0);
+                           int k, int width, int dtype, cudaStream_t stream, int dst_ld = 0, bool may_drop = false);
 // Backward of the combine: du[prow,:] = p[s] * dy_lo[t,:] (zeros on padding), dp[s] = <dy_lo[t,:], u[prow,:]>.
 cudaError_t launch_combine_bwd(const void* dy_lo, const void* u, void* du, float* dp, const Tables& tb, int k,
                                int width, int dtype, int64_t max_prows, cudaStream_t stream);

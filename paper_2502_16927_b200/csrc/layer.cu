@@ -422,7 +422,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         }
     }
     if (m.cdac) b.y_lo = y;                                                       // Eq. 3: the weighted sum is the output
-    { Stage s(L, S_COMBINE, st); BIGMAC_CUDA(launch_combine(b.u, b.y_lo, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st)); }  // F8
+    { Stage s(L, S_COMBINE, st); BIGMAC_CUDA(launch_combine(b.u, b.y_lo, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st, 0, m.cap != kNoCapacity)); }  // F8
     if (!m.cdac) {                                                                // F9 ascend: y = y' W'_up
         GemmArgs g;
         g.A = b.y_lo; g.lda = m.r; g.B = W->w_up; g.ldb = m.r; g.C = y; g.ldc = m.d;
@@ -525,7 +525,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     }
     if (m.cdac) {
         // Eq. 3: dx = sum_j dxg[row of slot (t,j)] + dl W_gate; dW_gate = dl^T x
-        { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, dx, nullptr, b.tb.prow_of_slot, m.T, m.k, m.d, m.dtype, st)); }
+        { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, dx, nullptr, b.tb.prow_of_slot, m.T, m.k, m.d, m.dtype, st, 0, m.cap != kNoCapacity)); }
         {
             GemmArgs g;
             g.A = b.dlogits; g.lda = ldcat; g.B = W->w_gate; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
@@ -550,7 +550,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         return BIGMAC_OK;
     }
     // dx'[t] = sum_j dxg[row of slot (t,j)]   (the transpose of the dispatch gather)
-    { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st, ldcat)); }
+    { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st, ldcat, m.cap != kNoCapacity)); }
     if (m.gate_low) {
         // The gate read x': its gradient joins dx' (dx' += dl W_gate, W_gate [E,r]) before the descend projection;
         // dW_gate = dl^T x'.
@@ -693,7 +693,7 @@ int bigmac_exchange_rows(bigmac_layer_t* L, const void* saved, int32_t T, int32_
     if (which != 1) { Stage s(L, S_DISPATCH, st); BIGMAC_CUDA(launch_dispatch(src, grouped, b.tb, m.k, width, m.dtype, m.P, st)); }
     if (which != 0) {
         Stage s(L, S_COMBINE, st);
-        BIGMAC_CUDA(launch_combine(grouped, dst, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, width, m.dtype, st));
+        BIGMAC_CUDA(launch_combine(grouped, dst, b.tb.topk_w, b.tb.prow_of_slot, m.T, m.k, width, m.dtype, st, 0, m.cap != kNoCapacity));
     }
     return BIGMAC_OK;
 }

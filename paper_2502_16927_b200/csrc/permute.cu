@@ -77,7 +77,9 @@ __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__
     }
 }
 
-template <typename T>
+// MAY_DROP: slots may carry row -1 (dropped under a capacity limit) and are then left out; without it the loop has no
+// branch and the k row loads of a token are issued together.
+template <typename T, bool MAY_DROP>
 __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ grouped, uint4* __restrict__ dst,
                                                       const float* __restrict__ w,
                                                       const int32_t* __restrict__ prow_of_slot, int n_tokens, int k,
@@ -93,7 +95,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
         for (int j = 0; j < k; ++j) {                      // slot order: fixed summation order
             const int64_t s = (int64_t)t * k + j;
             const int prow = prow_of_slot[s];
-            if (prow < 0) continue;                         // dropped under a capacity limit: absent from the sum
+            if (MAY_DROP && prow < 0) continue;             // dropped under a capacity limit: absent from the sum
             const float p = w ? w[s] : 1.0f;
             float f[V];
             Vec<T>::unpack(grouped[(int64_t)prow * vecs_per_row + c], f);
@@ -245,16 +247,19 @@ cudaError_t launch_dispatch(const void* src, void* grouped, const Tables& tb, in
 }
 
 cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const int32_t* prow_of_slot, int T, int k,
-                           int width, int dtype, cudaStream_t stream, int dst_ld) {
+                           int width, int dtype, cudaStream_t stream, int dst_ld, bool may_drop) {
     if (T == 0) return cudaSuccess;
     const int vecs = width * elem_bytes(dtype) / 16;
     const int dvecs = (dst_ld ? dst_ld : width) * elem_bytes(dtype) / 16;
-    if (dtype == BIGMAC_BF16)
-        combine_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, stream>>>((const uint4*)grouped, (uint4*)dst, w,
-                                                                         prow_of_slot, T, k, vecs, dvecs);
-    else
-        combine_kernel<float><<<warp_blocks(T), 256, 0, stream>>>((const uint4*)grouped, (uint4*)dst, w, prow_of_slot,
-                                                                 T, k, vecs, dvecs);
+    const uint4* src = (const uint4*)grouped;
+    uint4* out = (uint4*)dst;
+    if (dtype == BIGMAC_BF16) {
+        if (may_drop) combine_kernel<__nv_bfloat16, true><<<warp_blocks(T), 256, 0, stream>>>(src, out, w, prow_of_slot, T, k, vecs, dvecs);
+        else combine_kernel<__nv_bfloat16, false><<<warp_blocks(T), 256, 0, stream>>>(src, out, w, prow_of_slot, T, k, vecs, dvecs);
+    } else {
+        if (may_drop) combine_kernel<float, true><<<warp_blocks(T), 256, 0, stream>>>(src, out, w, prow_of_slot, T, k, vecs, dvecs);
+        else combine_kernel<float, false><<<warp_blocks(T), 256, 0, stream>>>(src, out, w, prow_of_slot, T, k, vecs, dvecs);
+    }
     return cudaGetLastError();
 }
 
