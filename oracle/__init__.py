@@ -139,6 +139,12 @@ def route(inp: Dict[str, np.ndarray], k: int, capacity_factor: float = 0.0, gate
     return Routing(logits, idx, p, counts, offsets, ros, sor, None, counts.copy(), gate_low)
 
 
+def _bias(inp, key):
+    """Expert bias b1 [E,h] / b2 [E,r] as float32, or None (Eq. 4 has none; they are a variant)."""
+    b = inp.get(key)
+    return None if b is None else _f32(b)
+
+
 def _dims(inp):
     T, d = inp["x"].shape
     E, h, r = inp["w1"].shape
@@ -165,7 +171,7 @@ def forward_tokens(inp, routing: Routing, act: int, tokens=None, want_slots: boo
                                 _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])), _p(routing.topk_idx),
                                 _p(routing.topk_p), _p(tok), C.c_int(n), C.c_int(d), C.c_int(r), C.c_int(h),
                                 C.c_int(E), C.c_int(k), C.c_int(act), _p(x_lo), _p(y_lo), _p(y), _p(z), _p(u),
-                                _p(routing.keep))
+                                _p(routing.keep), _p(_bias(inp, "b1")), _p(_bias(inp, "b2")))
     out = {"x_lo": x_lo, "y_lo": y_lo, "y": y}
     if want_slots:
         out["z"], out["u"] = z, u
@@ -181,7 +187,7 @@ def forward_grouped(inp, routing: Routing, act: int):
                                  _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])), _p(routing.topk_p),
                                  _p(routing.offsets), _p(routing.row_of_slot), _p(routing.slot_of_row),
                                  C.c_int(T), C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(E), C.c_int(k),
-                                 C.c_int(act), _p(xg), _p(y_lo), _p(y))
+                                 C.c_int(act), _p(xg), _p(y_lo), _p(y), _p(_bias(inp, "b1")), _p(_bias(inp, "b2")))
     return {"xg": xg, "y_lo": y_lo, "y": y}
 
 
@@ -199,21 +205,24 @@ def backward_tokens(inp, routing: Routing, act: int, tokens=None, decide_bf16: b
                                  _p(_f32(inp["w_up"])), _p(routing.topk_idx), _p(routing.topk_p), _p(tok),
                                  C.c_int(n), C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(E), C.c_int(k),
                                  C.c_int(act), C.c_int(int(decide_bf16)), _p(dx), _p(dx_lo), _p(dlogit), _p(dy_lo),
-                                 _p(routing.keep), C.c_int(int(routing.gate_low)))
+                                 _p(routing.keep), C.c_int(int(routing.gate_low)), _p(_bias(inp, "b1")),
+                                 _p(_bias(inp, "b2")))
     return {"dx": dx, "dx_lo": dx_lo, "dlogit": dlogit, "dy_lo": dy_lo}
 
 
-def backward_expert(inp, routing: Routing, act: int, e: int, decide_bf16: bool = False):
-    """dW1[e] [h,r] and dW2[e] [r,h], summed over the rows of expert e's segment."""
+def backward_expert(inp, routing: Routing, act: int, e: int, decide_bf16: bool = False, want_bias_grads: bool = False):
+    """dW1[e] [h,r] and dW2[e] [r,h], summed over the rows of expert e's segment (+ db1[e] [h], db2[e] [r])."""
     T, d, r, h, E = _dims(inp)
     k = routing.topk_idx.shape[1]
     dw1 = np.empty((h, r)); dw2 = np.empty((r, h))
+    db1 = np.empty(h) if want_bias_grads else None
+    db2 = np.empty(r) if want_bias_grads else None
     lib().oracle_backward_expert(_p(_f32(inp["x"])), _p(_f32(inp["dy"])), _p(_f32(inp["w_down"])),
                                  _p(_f32(inp["w1"])), _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])),
                                  _p(routing.topk_p), _p(routing.offsets), _p(routing.slot_of_row), C.c_int(e),
                                  C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(k), C.c_int(act), C.c_int(int(decide_bf16)),
-                                 _p(dw1), _p(dw2))
-    return dw1, dw2
+                                 _p(dw1), _p(dw2), _p(_bias(inp, "b1")), _p(_bias(inp, "b2")), _p(db1), _p(db2))
+    return (dw1, dw2, db1, db2) if want_bias_grads else (dw1, dw2)
 
 
 def backward_full(inp, routing: Routing, act: int, experts=None, decide_bf16: bool = False, aux_alpha: float = 0.0):
@@ -230,21 +239,30 @@ def backward_full(inp, routing: Routing, act: int, experts=None, decide_bf16: bo
                                  _p(routing.topk_idx), _p(bwd["dlogit"]), C.c_int(T), C.c_int(d), C.c_int(r),
                                  C.c_int(E), C.c_int(k), _p(dw_up), _p(dw_down), _p(dw_gate), _p(db_gate))
     dw1, dw2 = {}, {}
+    with_bias = inp.get("b1") is not None
+    db1 = np.zeros((E, h)) if with_bias else None
+    db2 = np.zeros((E, r)) if with_bias else None
     if experts is None:
         all1 = np.empty((E, h, r)); all2 = np.empty((E, r, h))
         lib().oracle_backward_all_experts(_p(_f32(inp["x"])), _p(_f32(inp["dy"])), _p(_f32(inp["w_down"])),
                                           _p(_f32(inp["w1"])), _p(_f32(inp["w2"])), _p(_f32(inp["w_up"])),
                                           _p(routing.topk_p), _p(routing.offsets), _p(routing.slot_of_row),
                                           C.c_int(E), C.c_int(d), C.c_int(r), C.c_int(h), C.c_int(k), C.c_int(act),
-                                          C.c_int(int(decide_bf16)), _p(all1), _p(all2))
+                                          C.c_int(int(decide_bf16)), _p(all1), _p(all2), _p(_bias(inp, "b1")),
+                                          _p(_bias(inp, "b2")), _p(db1), _p(db2))
         for e in range(E):
             dw1[e], dw2[e] = all1[e], all2[e]
     else:
         for e in experts:
-            dw1[e], dw2[e] = backward_expert(inp, routing, act, e, decide_bf16)
+            if with_bias:
+                dw1[e], dw2[e], db1[e], db2[e] = backward_expert(inp, routing, act, e, decide_bf16, True)
+            else:
+                dw1[e], dw2[e] = backward_expert(inp, routing, act, e, decide_bf16)
     out = {"y": fwd["y"], "y_lo": fwd["y_lo"], "x_lo": fwd["x_lo"], "dx": bwd["dx"], "dx_lo": bwd["dx_lo"],
            "dlogit": bwd["dlogit"], "dw_up": dw_up, "dw_down": dw_down, "dw_gate": dw_gate,
            "db_gate": db_gate, "dw1": dw1, "dw2": dw2}
+    if with_bias:
+        out["db1"], out["db2"] = db1, db2
     if routing.gate_low:
         # the gate read x': dW_g [E,r] = dl^T x' with dl scattered to its dense [T,E] form (a library matmul); dx' above
         # already holds the gate's share, so dw_down is complete

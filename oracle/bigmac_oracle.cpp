@@ -116,7 +116,7 @@ double round_bf16(double v) {
 // (z > 0): when `decide_bf16` is set it is taken the way the BF16 kernels take it, from x' rounded to
 // bf16, so that both sides decide on the same numbers; every other quantity stays exact.
 void decision_preact(const double* x_lo, const double* z_exact, const float* w1_e, int r, int h, int act,
-                     int decide_bf16, double* z_dec) {
+                     int decide_bf16, double* z_dec, const float* b1_e = nullptr) {
     if (!decide_bf16 || act != ACT_RELU) {
         std::memcpy(z_dec, z_exact, sizeof(double) * h);
         return;
@@ -124,6 +124,8 @@ void decision_preact(const double* x_lo, const double* z_exact, const float* w1_
     std::vector<double> xr(r);
     for (int c = 0; c < r; ++c) xr[c] = round_bf16(x_lo[c]);
     matvec(xr.data(), w1_e, h, r, z_dec);
+    if (b1_e)
+        for (int q = 0; q < h; ++q) z_dec[q] += (double)b1_e[q];
 }
 
 void widen(const float* src, int n, double* dst) {
@@ -131,11 +133,17 @@ void widen(const float* src, int n, double* dst) {
 }
 
 // One routed slot of one token through expert e (Eq. 4):  z = x' W1_e^T, a = sigma(z), u = a W2_e^T.
+// Variant with expert biases (Eq. 4 has none; Table 3's parameter count has a bias-like term): z += b1_e, u += b2_e;
+// b1_e [h] / b2_e [r] are NULL without them.
 void expert_forward(const double* x_lo, const float* w1_e, const float* w2_e, int r, int h, int act,
-                    double* z, double* a, double* u) {
+                    double* z, double* a, double* u, const float* b1_e = nullptr, const float* b2_e = nullptr) {
     matvec(x_lo, w1_e, h, r, z);
+    if (b1_e)
+        for (int q = 0; q < h; ++q) z[q] += (double)b1_e[q];
     for (int q = 0; q < h; ++q) a[q] = act_f(act, z[q]);
     matvec(a, w2_e, r, h, u);
+    if (b2_e)
+        for (int c = 0; c < r; ++c) u[c] += (double)b2_e[c];
 }
 
 }  // namespace
@@ -278,7 +286,7 @@ void oracle_forward_tokens(const float* x, const float* w_down, const float* w1,
                            const float* w_up, const int32_t* topk_idx, const double* topk_p,
                            const int32_t* tokens, int n, int d, int r, int h, int E, int k, int act,
                            double* x_lo_out, double* y_lo_out, double* y_out, double* z_out, double* u_out,
-                           const uint8_t* keep) {
+                           const uint8_t* keep, const float* b1, const float* b2) {
     (void)E;
 #pragma omp parallel for schedule(dynamic, 4)
     for (int i = 0; i < n; ++i) {
@@ -290,7 +298,7 @@ void oracle_forward_tokens(const float* x, const float* w_down, const float* w1,
             const int e = topk_idx[(size_t)t * k + j];
             const double p = topk_p[(size_t)t * k + j];
             expert_forward(x_lo.data(), w1 + (size_t)e * h * r, w2 + (size_t)e * r * h, r, h, act,
-                           z.data(), a.data(), u.data());
+                           z.data(), a.data(), u.data(), b1 ? b1 + (size_t)e * h : nullptr, b2 ? b2 + (size_t)e * r : nullptr);
             if (!keep || keep[(size_t)t * k + j])
                 for (int c = 0; c < r; ++c) y_lo[c] += p * u[c];           // p_i(x) E_i(x'); nothing from a dropped slot
             if (z_out) std::memcpy(z_out + ((size_t)i * k + j) * h, z.data(), sizeof(double) * h);
@@ -308,7 +316,8 @@ void oracle_forward_tokens(const float* x, const float* w_down, const float* w1,
 void oracle_forward_grouped(const float* x, const float* w_down, const float* w1, const float* w2,
                             const float* w_up, const double* topk_p, const int32_t* offsets,
                             const int32_t* row_of_slot, const int32_t* slot_of_row, int T, int d, int r,
-                            int h, int E, int k, int act, double* xg_out, double* y_lo_out, double* y_out) {
+                            int h, int E, int k, int act, double* xg_out, double* y_lo_out, double* y_out,
+                            const float* b1, const float* b2) {
     const int64_t N = (int64_t)T * k;
     std::vector<double> x_lo((size_t)T * r), xg((size_t)N * r), ug((size_t)N * r);
 #pragma omp parallel for schedule(static)
@@ -326,7 +335,8 @@ void oracle_forward_grouped(const float* x, const float* w_down, const float* w1
         std::vector<double> z(h), a(h);
         for (int row = offsets[e]; row < offsets[e + 1]; ++row)
             expert_forward(&xg[(size_t)row * r], w1 + (size_t)e * h * r, w2 + (size_t)e * r * h, r, h, act,
-                           z.data(), a.data(), &ug[(size_t)row * r]);
+                           z.data(), a.data(), &ug[(size_t)row * r], b1 ? b1 + (size_t)e * h : nullptr,
+                           b2 ? b2 + (size_t)e * r : nullptr);
     }
 #pragma omp parallel for schedule(static)
     for (int t = 0; t < T; ++t) {                                           // combine + ascend
@@ -354,7 +364,8 @@ void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate
                             const float* w1, const float* w2, const float* w_up, const int32_t* topk_idx,
                             const double* topk_p, const int32_t* tokens, int n, int d, int r, int h, int E,
                             int k, int act, int decide_bf16, double* dx_out, double* dx_lo_out,
-                            double* dlogit_out, double* dy_lo_out, const uint8_t* keep, int gate_low) {
+                            double* dlogit_out, double* dy_lo_out, const uint8_t* keep, int gate_low,
+                            const float* b1, const float* b2) {
     (void)E;
 #pragma omp parallel for schedule(dynamic, 4)
     for (int i = 0; i < n; ++i) {
@@ -371,13 +382,15 @@ void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate
             const float* w1_e = w1 + (size_t)e * h * r;
             const float* w2_e = w2 + (size_t)e * r * h;
             if (keep && !keep[(size_t)t * k + j]) { dp[j] = 0.0; continue; }   // a dropped slot is absent from y'
-            expert_forward(x_lo.data(), w1_e, w2_e, r, h, act, z.data(), a.data(), u.data());
+            const float* b1_e = b1 ? b1 + (size_t)e * h : nullptr;
+            expert_forward(x_lo.data(), w1_e, w2_e, r, h, act, z.data(), a.data(), u.data(), b1_e,
+                           b2 ? b2 + (size_t)e * r : nullptr);
             double acc = 0.0;
             for (int c = 0; c < r; ++c) acc += dy_lo[c] * u[c];
             dp[j] = acc;
             for (int c = 0; c < r; ++c) du[c] = p * dy_lo[c];
             matvec_t(du.data(), w2_e, r, h, da.data());
-            decision_preact(x_lo.data(), z.data(), w1_e, r, h, act, decide_bf16, zd.data());
+            decision_preact(x_lo.data(), z.data(), w1_e, r, h, act, decide_bf16, zd.data(), b1_e);
             for (int q = 0; q < h; ++q) dz[q] = da[q] * act_df(act, zd[q]);
             matvec_t(dz.data(), w1_e, h, r, tmp.data());
             for (int c = 0; c < r; ++c) dx_lo[c] += tmp[c];
@@ -412,9 +425,14 @@ void oracle_backward_tokens(const float* x, const float* dy, const float* w_gate
 void oracle_backward_expert(const float* x, const float* dy, const float* w_down, const float* w1,
                             const float* w2, const float* w_up, const double* topk_p, const int32_t* offsets,
                             const int32_t* slot_of_row, int e, int d, int r, int h, int k, int act,
-                            int decide_bf16, double* dw1_e, double* dw2_e) {
+                            int decide_bf16, double* dw1_e, double* dw2_e, const float* b1, const float* b2,
+                            double* db1_e, double* db2_e) {
     std::fill(dw1_e, dw1_e + (size_t)h * r, 0.0);
     std::fill(dw2_e, dw2_e + (size_t)r * h, 0.0);
+    if (db1_e) std::fill(db1_e, db1_e + h, 0.0);       // db1_e[q] = sum_rows dz[q] ;  db2_e[c] = sum_rows du[c]
+    if (db2_e) std::fill(db2_e, db2_e + r, 0.0);
+    const float* b1_e = b1 ? b1 + (size_t)e * h : nullptr;
+    const float* b2_e = b2 ? b2 + (size_t)e * r : nullptr;
     const float* w1_e = w1 + (size_t)e * h * r;
     const float* w2_e = w2 + (size_t)e * r * h;
     std::vector<double> xt(d), dyt(d), x_lo(r), dy_lo(r), z(h), zd(h), a(h), u(r), du(r), da(h), dz(h);
@@ -426,11 +444,15 @@ void oracle_backward_expert(const float* x, const float* dy, const float* w_down
         widen(dy + (size_t)t * d, d, dyt.data());
         matvec(xt.data(), w_down, r, d, x_lo.data());
         matvec_t(dyt.data(), w_up, d, r, dy_lo.data());
-        expert_forward(x_lo.data(), w1_e, w2_e, r, h, act, z.data(), a.data(), u.data());
+        expert_forward(x_lo.data(), w1_e, w2_e, r, h, act, z.data(), a.data(), u.data(), b1_e, b2_e);
         for (int c = 0; c < r; ++c) du[c] = p * dy_lo[c];
         matvec_t(du.data(), w2_e, r, h, da.data());
-        decision_preact(x_lo.data(), z.data(), w1_e, r, h, act, decide_bf16, zd.data());
+        decision_preact(x_lo.data(), z.data(), w1_e, r, h, act, decide_bf16, zd.data(), b1_e);
         for (int q = 0; q < h; ++q) dz[q] = da[q] * act_df(act, zd[q]);
+        if (db1_e)
+            for (int q = 0; q < h; ++q) db1_e[q] += dz[q];
+        if (db2_e)
+            for (int c = 0; c < r; ++c) db2_e[c] += du[c];
         for (int c = 0; c < r; ++c)
             for (int q = 0; q < h; ++q) dw2_e[(size_t)c * h + q] += du[c] * a[q];
         for (int q = 0; q < h; ++q)
@@ -442,11 +464,13 @@ void oracle_backward_expert(const float* x, const float* dy, const float* w_down
 void oracle_backward_all_experts(const float* x, const float* dy, const float* w_down, const float* w1,
                                  const float* w2, const float* w_up, const double* topk_p, const int32_t* offsets,
                                  const int32_t* slot_of_row, int E, int d, int r, int h, int k, int act,
-                                 int decide_bf16, double* dw1, double* dw2) {
+                                 int decide_bf16, double* dw1, double* dw2, const float* b1, const float* b2,
+                                 double* db1, double* db2) {
 #pragma omp parallel for schedule(dynamic, 1)
     for (int e = 0; e < E; ++e)
         oracle_backward_expert(x, dy, w_down, w1, w2, w_up, topk_p, offsets, slot_of_row, e, d, r, h, k, act,
-                               decide_bf16, dw1 + (size_t)e * h * r, dw2 + (size_t)e * r * h);
+                               decide_bf16, dw1 + (size_t)e * h * r, dw2 + (size_t)e * r * h, b1, b2,
+                               db1 ? db1 + (size_t)e * h : nullptr, db2 ? db2 + (size_t)e * r : nullptr);
 }
 
 // Gradients of the shared matrices, as sums over all tokens of outer products of per-token vectors
