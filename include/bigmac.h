@@ -87,6 +87,11 @@ typedef enum {
  * gradient joins dx' before the descend projection.  Not together with BIGMAC_FLAG_CDAC (there x' is x:
  * INVALID_ARG) nor with a load-balancing loss (UNSUPPORTED). */
 #define BIGMAC_FLAG_GATE_LOW 8u
+/* Expert biases (Eq. 4 has none; Table 3's parameter count has a bias-like term): E_i(v) = sigma(v W_{i,up} + b1_i)
+ * W_{i,down} + b2_i with fp32 b1 [E,h] and b2 [E,r] in bigmac_weights_t (required with this flag, ignored without)
+ * and fp32 gradients db1 / db2 in bigmac_grads_t (nullable).  The small-batch and fused-expert inference kernels are
+ * bypassed.  Not with expert parallelism (UNSUPPORTED). */
+#define BIGMAC_FLAG_EXPERT_BIAS 16u
 
 /* The two training-recipe settings of the paper's pre-training configuration (Table 5: capacity factor 1.2,
  * load-balancing loss with coefficient 0.001).  Both are off (0) in the layer the paper advocates and measures,
@@ -119,6 +124,8 @@ typedef struct {
     const void *w1;       /* [E,h,r] W_{i,up} of Eq. 4 */
     const void *w2;       /* [E,r,h] W_{i,down} of Eq. 4 */
     const void *w_up;     /* [d,r]   W'_up of Eq. 2 */
+    const float *b1;      /* [E,h] fp32, BIGMAC_FLAG_EXPERT_BIAS only */
+    const float *b2;      /* [E,r] fp32, BIGMAC_FLAG_EXPERT_BIAS only */
 } bigmac_weights_t;
 
 /* Gradient buffers, same shapes and dtype as the weights; db_gate fp32 [E] or NULL. */
@@ -126,6 +133,7 @@ typedef struct {
     void *dw_gate;
     float *db_gate;
     void *dw_down, *dw1, *dw2, *dw_up;
+    float *db1, *db2;     /* [E,h], [E,r] fp32, BIGMAC_FLAG_EXPERT_BIAS only (nullable) */
 } bigmac_grads_t;
 
 /* Routing tables.  Flat slot id s = t*k + j (j-th choice of token t).
@@ -222,8 +230,8 @@ const char *bigmac_status_string(int status);
  * `saved` (and, across the three backward calls, `scratch`) must keep their contents between the calls of a step.
  * The gradients of the shared matrices that the backward returns are this rank's share (the sum over its own
  * tokens): the caller adds them over the ranks, as for any data-parallel layer; dw1 / dw2 are complete.
- * Not supported together with a capacity factor, a load-balancing loss, BIGMAC_FLAG_CDAC or BIGMAC_FLAG_GATE_LOW
- * (BIGMAC_ERR_UNSUPPORTED). */
+ * Not supported together with a capacity factor, a load-balancing loss, BIGMAC_FLAG_CDAC, BIGMAC_FLAG_GATE_LOW or
+ * BIGMAC_FLAG_EXPERT_BIAS (BIGMAC_ERR_UNSUPPORTED). */
 #define BIGMAC_EP_MAX_RANKS 8
 typedef struct {
     int32_t rank, size;                 /* 0 <= rank < size <= BIGMAC_EP_MAX_RANKS, E % size == 0 */

@@ -26,11 +26,11 @@ class bigmac_config_t(C.Structure):
 
 
 class bigmac_weights_t(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("w_gate", "b_gate", "w_down", "w1", "w2", "w_up")]
+    _fields_ = [(n, C.c_void_p) for n in ("w_gate", "b_gate", "w_down", "w1", "w2", "w_up", "b1", "b2")]
 
 
 class bigmac_grads_t(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("dw_gate", "db_gate", "dw_down", "dw1", "dw2", "dw_up")]
+    _fields_ = [(n, C.c_void_p) for n in ("dw_gate", "db_gate", "dw_down", "dw1", "dw2", "dw_up", "db1", "db2")]
 
 
 _ROUTING_FIELDS = ("topk_idx", "topk_w", "counts", "offsets", "row_of_slot", "slot_of_row", "counts_chosen", "aux_loss")
@@ -160,11 +160,11 @@ def bigmac_workspace_bytes(handle, T: int, training: bool):
 def _weights(W: Dict[str, torch.Tensor]) -> bigmac_weights_t:
     # w_down / w_up are absent for the projection-free layer (BIGMAC_FLAG_CDAC)
     return bigmac_weights_t(_ptr(W.get("w_gate")), _ptr(W.get("b_gate")), _ptr(W.get("w_down")), _ptr(W.get("w1")),
-                            _ptr(W.get("w2")), _ptr(W.get("w_up")))
+                            _ptr(W.get("w2")), _ptr(W.get("w_up")), _ptr(W.get("b1")), _ptr(W.get("b2")))
 
 
 def _grads(G: Dict[str, torch.Tensor]) -> bigmac_grads_t:
-    return bigmac_grads_t(*[_ptr(G.get(n)) for n in ("dw_gate", "db_gate", "dw_down", "dw1", "dw2", "dw_up")])
+    return bigmac_grads_t(*[_ptr(G.get(n)) for n in ("dw_gate", "db_gate", "dw_down", "dw1", "dw2", "dw_up", "db1", "db2")])
 
 
 def _routing(R: Optional[Dict[str, torch.Tensor]]):

@@ -209,7 +209,7 @@ int ep_dims(const bigmac_layer* L, int32_t T, int size, int rank, EpDims* out) {
     const bigmac_config_t& c = L->cfg;
     if (size < 1 || size > kMaxRanks || rank < 0 || rank >= size) return BIGMAC_ERR_INVALID_ARG;
     if (c.E % size) return BIGMAC_ERR_INVALID_ARG;
-    if (c.capacity_factor > 0 || c.aux_loss_coef > 0 || (c.flags & (BIGMAC_FLAG_CDAC | BIGMAC_FLAG_GATE_LOW)))
+    if (c.capacity_factor > 0 || c.aux_loss_coef > 0 || (c.flags & (BIGMAC_FLAG_CDAC | BIGMAC_FLAG_GATE_LOW | BIGMAC_FLAG_EXPERT_BIAS)))
         return BIGMAC_ERR_UNSUPPORTED;
     if ((int64_t)size * c.max_tokens * c.k > (int64_t)1 << 30) return BIGMAC_ERR_UNSUPPORTED;
     EpDims m{};

@@ -20,12 +20,14 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
     const T* A = (const T*)g.A;
     const T* B = (const T*)g.B;
     int64_t c_base = 0;
+    const float* bias = nullptr;
     int m_limit = g.M, k_begin = 0, k_end = g.K;
     const int m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
     if (g.group == GROUP_M) {
         const int tile = m0 / kPad;
         if (tile >= *g.n_tiles) return;
         B += (int64_t)g.tile_expert[tile] * g.b_stride;
+        if (g.bias) bias = g.bias + (int64_t)g.tile_expert[tile] * g.bias_stride;
         m_limit = min(g.M, *g.n_tiles * kPad);
     } else if (g.group == GROUP_K) {
         const int e = blockIdx.z;
@@ -81,6 +83,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
             if (gn >= g.N) continue;
             const int64_t off = c_base + (int64_t)gm * g.ldc + gn;
             float v = acc[i][j];
+            if (bias) v += bias[gn];
             if (g.epilogue == EPI_ACT) {
                 if (g.Z) ((T*)g.Z)[off] = (T)act_grad(g.act, v);
                 v = act_apply(g.act, v);

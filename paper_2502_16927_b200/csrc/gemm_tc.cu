@@ -192,6 +192,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 const int col0 = tl.n0 + part * COLS_PER_WARP + c * 32;
                 if (col0 >= p.N) continue;             // uniform across the warp
+                if (p.bias) add_bias32(v, p.bias + (int64_t)tl.expert * p.bias_stride + col0);   // N is a multiple of 32 here
                 if (TMA_EPI) {
                     if (lane == 0) tma_store_wait_read();        // previous boxes of this warp have left smem
                     __syncwarp();
@@ -312,6 +313,8 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
     p.C = g.C; p.Z = g.Z; p.ldc = g.ldc; p.c_stride = g.c_stride; p.M = g.M; p.N = g.N; p.K = g.K;
     p.out_f32 = g.out_f32; p.accumulate = g.accumulate; p.epilogue = g.epilogue; p.act = g.act; p.group = g.group;
     p.num_experts = E; p.tile_expert = g.tile_expert; p.n_tiles = g.n_tiles; p.poffsets = g.poffsets; p.status = status;
+    p.bias = g.group == GROUP_M ? g.bias : nullptr; p.bias_stride = g.bias_stride;
+    if (p.bias && (g.N % 32 || ((uintptr_t)g.bias % 16) || g.bias_stride % 4)) return cudaErrorInvalidValue;
     const int64_t tiles = (int64_t)((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * (g.group == GROUP_K ? E : p.split_k);
     const int max_tiles = tiles > (1 << 30) ? (1 << 30) : (int)tiles;
     if (g.a_kmajor && g.b_kmajor) return launch<BN, STAGES, true, true, TMA_EPI>(ma, mb, mc, mz, mb2, p, max_tiles, stream);

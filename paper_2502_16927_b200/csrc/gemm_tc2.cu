@@ -305,6 +305,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 }
                 const int col0 = tl.n0 + part * COLS_PER_WARP + c * 32;
                 if (col0 >= p.N) continue;             // uniform across the warp
+                if (p.bias) add_bias32(v, p.bias + (int64_t)tl.expert * p.bias_stride + col0);   // N is a multiple of 32 here
                 if (TMA_EPI) {
                     if (lane == 0) tma_store_wait_read();
                     __syncwarp();
@@ -422,6 +423,8 @@ cudaError_t dispatch_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
     p.C = g.C; p.Z = g.Z; p.ldc = g.ldc; p.c_stride = g.c_stride; p.M = g.M; p.N = g.N; p.K = g.K;
     p.out_f32 = g.out_f32; p.accumulate = g.accumulate; p.epilogue = g.epilogue; p.act = g.act; p.group = g.group;
     p.num_experts = E; p.tile_expert = g.tile_expert; p.n_tiles = g.n_tiles; p.poffsets = g.poffsets; p.status = status;
+    p.bias = g.group == GROUP_M ? g.bias : nullptr; p.bias_stride = g.bias_stride;
+    if (p.bias && (g.N % 32 || ((uintptr_t)g.bias % 16) || g.bias_stride % 4)) return cudaErrorInvalidValue;
     // upper bound on work items (the kernel derives the exact count on the device for grouped rows)
     const int64_t pairs = g.group == GROUP_M ? ((g.M + BM - 1) / BM + 1) / 2 + E : (g.M + 2 * BM - 1) / (2 * BM);
     const int64_t items = pairs * ((g.N + BN - 1) / BN) * (g.group == GROUP_K ? E : p.split_k);

@@ -58,6 +58,10 @@ struct GemmArgs {
     int N2 = 0;
     int split_k = 1;                    // > 1: part s of the contraction writes its partial result (fp32) to C + s*M*ldc
     int force_kernel = 0;               // measurement aid: 1 = one-CTA kernel, 2 = CTA-pair kernel, 0 = default choice
+    // GROUP_M only: fp32 bias added to the accumulator before the epilogue, column n of a row of expert e gets
+    // bias[e*bias_stride + n] (16-byte aligned, bias_stride a multiple of 4)
+    const float* bias = nullptr;
+    int64_t bias_stride = 0;
 };
 
 // fp32-FMA GEMM for either dtype (dtype: bigmac_dtype_t of A, B, Z and - unless out_f32 - C).
@@ -163,6 +167,10 @@ constexpr int kColsumChunks = 296;
 // aux_partial (nullable): a second array, [kAuxChunks, E], of partial column sums added in (launch_gate_bwd_aux).
 cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db, float* partial, int64_t N, int E,
                                bool accumulate, cudaStream_t stream, const float* aux_partial = nullptr);
+// Per-expert column sums of a grouped matrix (the expert-bias gradients): out[e, c] (+)= sum over the padded rows of
+// expert e of src[row, c] (padding rows hold zeros), fp32, fixed summation order.  width a multiple of 8 (bf16) / 4.
+cudaError_t launch_grouped_colsum(const void* src, const int32_t* poffsets, float* out, int E, int width, int dtype,
+                                  bool accumulate, cudaStream_t stream);
 // Sum the `parts` fp32 partial results ws[s][m][n] of a split contraction in the order s = 0, 1, ... and write
 // rows [0, m_split) to dst1 [m_split, N] and rows [m_split, m_split + m2) to dst2 [m2, N] (dst2 may be null),
 // in the dtype, adding to the destination if `accumulate`.

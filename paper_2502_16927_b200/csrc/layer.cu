@@ -40,6 +40,7 @@ struct Dims {
     bool cdac; // Eq. 3 layer: no descend / ascend projections, r == d
     int ldcat; // row stride of dcat: r + E64, or E64 alone without projections (dx' then goes straight to dx)
     bool gate_low; // the gate reads x' (w_gate [E,r])
+    bool bias;     // experts have biases b1 [E,h], b2 [E,r]
     int cap;   // rows an expert keeps at most (Table 5's capacity factor); kNoCapacity = dropless
     float aux; // coefficient of the load-balancing loss (Table 5), 0 = none
 };
@@ -54,6 +55,7 @@ Dims dims_of(const bigmac_layer* L, int T) {
     m.cdac = (c.flags & BIGMAC_FLAG_CDAC) != 0;
     m.ldcat = m.cdac ? m.E64 : m.r + m.E64;
     m.gate_low = (c.flags & BIGMAC_FLAG_GATE_LOW) != 0;
+    m.bias = (c.flags & BIGMAC_FLAG_EXPERT_BIAS) != 0;
     m.cap = kNoCapacity;
     if (c.capacity_factor > 0) {                     // C = ceil((f * (T k)) / E), evaluated in double in this order
         const double rows = std::ceil(c.capacity_factor * (double)m.N / (double)c.E);
@@ -135,6 +137,8 @@ size_t saved_bytes_of(const Dims& m) {
 int check_weights(const bigmac_layer* L, const bigmac_weights_t* W) {
     if (!W || !W->w_gate || !W->w1 || !W->w2) return BIGMAC_ERR_INVALID_ARG;
     if (!aligned(W->w_gate, 16) || !aligned(W->w1, 16) || !aligned(W->w2, 16) || !aligned(W->b_gate, 4))
+        return BIGMAC_ERR_INVALID_ARG;
+    if (L && (L->cfg.flags & BIGMAC_FLAG_EXPERT_BIAS) && (!W->b1 || !W->b2 || !aligned(W->b1, 16) || !aligned(W->b2, 16)))
         return BIGMAC_ERR_INVALID_ARG;
     if (L && (L->cfg.flags & BIGMAC_FLAG_CDAC)) return BIGMAC_OK;             // no shared projections
     if (!W->w_down || !W->w_up || !aligned(W->w_down, 16) || !aligned(W->w_up, 16)) return BIGMAC_ERR_INVALID_ARG;
@@ -261,7 +265,8 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
     if (cfg->k > cfg->E) return BIGMAC_ERR_INVALID_ARG;
     if (cfg->dtype != BIGMAC_F32 && cfg->dtype != BIGMAC_BF16) return BIGMAC_ERR_INVALID_ARG;
     if (cfg->act < BIGMAC_ACT_RELU || cfg->act > BIGMAC_ACT_IDENTITY) return BIGMAC_ERR_INVALID_ARG;
-    if (cfg->flags & ~(BIGMAC_FLAG_SIMT_GEMM | BIGMAC_FLAG_CDAC | BIGMAC_FLAG_DYNAMIC_WGRAD | BIGMAC_FLAG_GATE_LOW))
+    if (cfg->flags & ~(BIGMAC_FLAG_SIMT_GEMM | BIGMAC_FLAG_CDAC | BIGMAC_FLAG_DYNAMIC_WGRAD | BIGMAC_FLAG_GATE_LOW |
+                       BIGMAC_FLAG_EXPERT_BIAS))
         return BIGMAC_ERR_INVALID_ARG;
     if ((cfg->flags & BIGMAC_FLAG_CDAC) && cfg->r != cfg->d) return BIGMAC_ERR_INVALID_ARG;
     if ((cfg->flags & BIGMAC_FLAG_CDAC) && (cfg->flags & BIGMAC_FLAG_GATE_LOW)) return BIGMAC_ERR_INVALID_ARG;
@@ -358,7 +363,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     const bigmac_config_t& c = L->cfg;
 
     // A few tokens, inference: the whole forward in one cooperative kernel (weight streaming, no tensor cores)
-    if (!training && !m.cdac && !m.gate_low && m.cap == kNoCapacity && m.aux == 0 && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
+    if (!training && !m.cdac && !m.gate_low && !m.bias && m.cap == kNoCapacity && m.aux == 0 && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
         {
             Stage s(L, S_DECODE, st);
             BIGMAC_CUDA(launch_decode_forward(x, W, y, b.logits, (float*)b.xg, (float*)b.a, (float*)b.u, b.tb.topk_idx,
@@ -399,7 +404,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     // decode tokens.  BIGMAC_FUSED_MLP=0 / =2 force it off / on.
     static const int fuse_mlp_mode = []() { const char* e = std::getenv("BIGMAC_FUSED_MLP"); return e ? atoi(e) : 1; }();
     const bool short_list = m.P / kPad <= 2 * (int64_t)gemm_tc_sm_count();
-    if (!training && (fuse_mlp_mode == 2 || (fuse_mlp_mode == 1 && short_list)) && sigma_as_bytes(L) &&
+    if (!training && !m.bias && (fuse_mlp_mode == 2 || (fuse_mlp_mode == 1 && short_list)) && sigma_as_bytes(L) &&
         fused_mlp_supported(m.r, m.h, m.dtype)) {
         Stage s(L, S_FUSED_MLP, st);
         BIGMAC_CUDA(launch_fused_mlp(b.xg, W->w1, W->w2, b.u, m.P, m.r, m.h, m.E, c.act, b.tb.tile_expert, b.tb.n_tiles,
@@ -411,6 +416,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
             g.C = b.a; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
             g.epilogue = EPI_ACT; g.act = c.act; g.group = GROUP_M; g.num_experts = m.E;
             g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
+            if (m.bias) { g.bias = W->b1; g.bias_stride = m.h; }
             BIGMAC_TRY(gemm(L, G_EXPERT1, g, st));
         }
         {                                                                             // F7 u = a W2_e^T
@@ -418,6 +424,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
             g.A = b.a; g.lda = m.h; g.B = W->w2; g.ldb = m.h; g.b_stride = (int64_t)m.r * m.h;
             g.C = b.u; g.ldc = m.r; g.M = (int)m.P; g.N = m.r; g.K = m.h;
             g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
+            if (m.bias) { g.bias = W->b2; g.bias_stride = m.r; }
             BIGMAC_TRY(gemm(L, G_EXPERT2, g, st));
         }
     }
@@ -502,6 +509,12 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         BIGMAC_TRY(gemm(L, G_DZ, g, st));
     }
     void* dz = b.dz ? b.dz : b.z;
+    if (m.bias) {   // db1_e = sum_rows dz[row,:], db2_e = sum_rows du[row,:]  (padding rows hold zeros)
+        if (!aligned(G->db1, 4) || !aligned(G->db2, 4)) return BIGMAC_ERR_INVALID_ARG;
+        Stage s(L, S_COLSUM, st, (G->db1 ? 1 : 0) + (G->db2 ? 1 : 0));
+        if (G->db1) BIGMAC_CUDA(launch_grouped_colsum(dz, b.tb.poffsets, G->db1, m.E, m.h, m.dtype, acc, st));
+        if (G->db2) BIGMAC_CUDA(launch_grouped_colsum(b.du, b.tb.poffsets, G->db2, m.E, m.r, m.dtype, acc, st));
+    }
     if (G->dw2) {   // dW2_e[c',q] = sum_rows du[row,c'] a[row,q]
         GemmArgs g;
         g.A = b.du; g.lda = m.r; g.a_kmajor = false; g.B = b.a; g.ldb = m.h; g.b_kmajor = false;

@@ -232,6 +232,39 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
     dst[0] = (T)acc.x; dst[1] = (T)acc.y; dst[2] = (T)acc.z; dst[3] = (T)acc.w;
 }
 
+// Per-expert column sums (expert-bias gradients).  Block (cg, e): 32 column-threads x 8 row-lanes; a thread adds rows
+// lane, lane + 8, ... of its 16-byte column vector in order, then the 8 row-lanes are added in order.
+template <typename T>
+__global__ void __launch_bounds__(256) grouped_colsum_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ poffsets,
+                                                             float* __restrict__ out, int vecs_per_row, int accumulate) {
+    constexpr int V = Vec<T>::kElems;
+    __shared__ float part[8][32 * V];
+    const int e = blockIdx.y, ct = threadIdx.x & 31, rl = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + ct;
+    float acc[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] = 0.0f;
+    if (c < vecs_per_row) {
+        for (int64_t row = (int64_t)poffsets[e] + rl; row < poffsets[e + 1]; row += 8) {
+            float f[V];
+            Vec<T>::unpack(src[row * vecs_per_row + c], f);
+#pragma unroll
+            for (int i = 0; i < V; ++i) acc[i] += f[i];
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < V; ++i) part[rl][ct * V + i] = acc[i];
+    __syncthreads();
+    for (int j = threadIdx.x; j < 32 * V; j += blockDim.x) {
+        const int col = blockIdx.x * 32 * V + j;
+        if (col >= vecs_per_row * V) continue;
+        float total = 0.0f;
+        for (int q = 0; q < 8; ++q) total += part[q][j];
+        float* dst = out + (int64_t)e * vecs_per_row * V + col;
+        *dst = accumulate ? *dst + total : total;
+    }
+}
+
 inline int elem_bytes(int dtype) { return dtype == BIGMAC_BF16 ? 2 : 4; }
 inline unsigned warp_blocks(int64_t warps) { return (unsigned)((warps + 7) / 8); }
 
@@ -293,6 +326,18 @@ cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db
                                bool accumulate, cudaStream_t stream, const float* aux_partial) {
     colsum_slots_kernel<<<kColsumChunks, 256, sizeof(float) * 8 * E, stream>>>(dl_slot, tb.topk_idx, partial, N, E);
     colsum_final_kernel<<<(unsigned)((E + 7) / 8), 256, 0, stream>>>(partial, aux_partial, db, kColsumChunks, kAuxChunks, E, accumulate);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_grouped_colsum(const void* src, const int32_t* poffsets, float* out, int E, int width, int dtype,
+                                  bool accumulate, cudaStream_t stream) {
+    if (E == 0 || width == 0) return cudaSuccess;
+    const int vecs = width * elem_bytes(dtype) / 16;
+    dim3 grid((unsigned)((vecs + 31) / 32), (unsigned)E);
+    if (dtype == BIGMAC_BF16)
+        grouped_colsum_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const uint4*)src, poffsets, out, vecs, accumulate ? 1 : 0);
+    else
+        grouped_colsum_kernel<float><<<grid, 256, 0, stream>>>((const uint4*)src, poffsets, out, vecs, accumulate ? 1 : 0);
     return cudaGetLastError();
 }
 

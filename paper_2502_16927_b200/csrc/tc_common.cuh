@@ -211,6 +211,8 @@ struct TcParams {
     int c_rows_per_expert;       // rows of the C tensor map per expert (GROUP_K); 0 otherwise
     int split_k;                 // dense only: the contraction is cut into split_k parts, part s writes C + s*M*ldc
     int b2_first_kb;             // k slices from this one on come from the second B tensor (map_b2); <0: none
+    const float* bias;           // GROUP_M: fp32 bias of expert e at bias + e*bias_stride, added before the epilogue; or null
+    int64_t bias_stride;
     int n_split;                 // output columns from this one on come from map_b2 (K-major) and go to C2 (fp32); <0: none
     float* C2;
     int64_t ldc2;
@@ -367,6 +369,15 @@ __device__ __forceinline__ void act_chunk_any(int act, float* v, uint32_t* wg) {
         case BIGMAC_ACT_RELU: act_chunk<BIGMAC_ACT_RELU, WITH_G, COUNT>(v, wg); break;
         case BIGMAC_ACT_GELU_TANH: act_chunk<BIGMAC_ACT_GELU_TANH, WITH_G, COUNT>(v, wg); break;
         default: act_chunk<BIGMAC_ACT_IDENTITY, WITH_G, COUNT>(v, wg); break;
+    }
+}
+
+// v[0..31] += b[0..31] (32 consecutive fp32 bias values, 16-byte aligned; every lane reads the same addresses).
+__device__ __forceinline__ void add_bias32(float* v, const float* __restrict__ b) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float4 q = __ldg((const float4*)b + i);
+        v[4 * i] += q.x; v[4 * i + 1] += q.y; v[4 * i + 2] += q.z; v[4 * i + 3] += q.w;
     }
 }
 
@@ -550,7 +561,7 @@ __device__ __forceinline__ Tile walk1_tile(const TcParams& p, int BN, const Tile
     Tile tl;
     tl.m0 = w.mt * BM;
     tl.n0 = w.nt * BN;
-    tl.expert = 0;
+    tl.expert = (p.bias && p.group == GROUP_M) ? p.tile_expert[w.mt] : 0;     // only the bias needs the expert here
     tl.k_row0 = 0;
     tl.num_kb = (p.K + BK - 1) / BK;
     tl.m_limit = p.group == GROUP_M ? min(p.M, tiles_m * kPad) : p.M;

@@ -30,7 +30,7 @@ import numpy as np
 
 ACT_RELU, ACT_GELU_ERF, ACT_GELU_TANH, ACT_IDENTITY = 0, 1, 2, 3
 DTYPE_F32, DTYPE_BF16 = 0, 1
-FLAG_SIMT_GEMM, FLAG_CDAC, FLAG_DYNAMIC_WGRAD, FLAG_GATE_LOW = 1, 2, 4, 8
+FLAG_SIMT_GEMM, FLAG_CDAC, FLAG_DYNAMIC_WGRAD, FLAG_GATE_LOW, FLAG_EXPERT_BIAS = 1, 2, 4, 8, 16
 
 
 @dataclass(frozen=True)
@@ -48,6 +48,7 @@ class Workload:
     gate_bias: str = "none"   # "none" | "zipf"  (b_g[e] = ln q_e, q_e ~ (e+1)^-1.1)
     cdac: bool = False        # the conventional fine-grained layer (Eq. 3): r == d, no w_down / w_up
     gate_low: bool = False    # the gate reads x' (w_gate [E,r]) instead of x
+    expert_bias: bool = False # experts have fp32 biases b1 [E,h], b2 [E,r] ~ N(0, 0.25)
 
     @property
     def N(self) -> int:
@@ -79,7 +80,7 @@ WORKLOADS: Dict[str, Workload] = {
 }
 DECODE_TOKEN_COUNTS = (1, 8, 64, 512)
 
-_TAGS = {"x": 1, "dy": 2, "w_gate": 3, "w_down": 4, "w1": 5, "w2": 6, "w_up": 7}
+_TAGS = {"x": 1, "dy": 2, "w_gate": 3, "w_down": 4, "w1": 5, "w2": 6, "w_up": 7, "b1": 8, "b2": 9}
 
 
 def _round_chunk_inplace(bits: np.ndarray) -> None:
@@ -152,6 +153,9 @@ def make_inputs(w: Workload, with_dy: bool = True) -> Dict[str, Optional[np.ndar
         "b_gate": zipf_log_popularity(w.E) if w.gate_bias == "zipf" else None,
         "dy": _normal(s, _TAGS["dy"], 0, (w.T, w.d), 1.0, dt) if with_dy else None,
     }
+    if w.expert_bias:                                # fp32 whatever the workload dtype, like the gate bias
+        out["b1"] = _normal(s, _TAGS["b1"], 0, (w.E, w.h), 0.5, DTYPE_F32)
+        out["b2"] = _normal(s, _TAGS["b2"], 0, (w.E, w.r), 0.5, DTYPE_F32)
     return out
 
 

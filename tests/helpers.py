@@ -36,7 +36,7 @@ def to_device(w, inp, device="cuda"):
     for key, val in inp.items():
         if val is None:
             continue
-        if key == "b_gate" or w.dtype == wl.DTYPE_F32:
+        if key in ("b_gate", "b1", "b2") or w.dtype == wl.DTYPE_F32:
             out[key] = torch.from_numpy(np.ascontiguousarray(val, dtype=np.float32)).to(device)
         else:
             bits = torch.from_numpy(wl.to_bf16_bits(val).view(np.int16)).to(device)
@@ -60,6 +60,8 @@ def make_layer(w, flags=0, max_tokens=None, capacity_factor=0.0, aux_loss_coef=0
         flags |= wl.FLAG_CDAC
     if w.gate_low:
         flags |= wl.FLAG_GATE_LOW
+    if w.expert_bias:
+        flags |= wl.FLAG_EXPERT_BIAS
     return binding.Layer(w.d, w.r, w.h, w.E, w.k, max_tokens or max(w.T, 1), w.dtype, w.act, flags,
                          capacity_factor=capacity_factor, aux_loss_coef=aux_loss_coef)
 
@@ -86,6 +88,10 @@ def empty_grads(w, dev, fill=None):
     G = {}
     for key, shp in shapes.items():
         G[key] = torch.empty(shp, dtype=dt, device="cuda") if fill is None else torch.full(shp, fill, dtype=dt, device="cuda")
-    G["db_gate"] = (torch.empty(w.E, dtype=torch.float32, device="cuda") if fill is None
-                    else torch.full((w.E,), fill, dtype=torch.float32, device="cuda"))
+    f32 = {"db_gate": (w.E,)}
+    if w.expert_bias:
+        f32.update(db1=(w.E, w.h), db2=(w.E, w.r))
+    for key, shp in f32.items():
+        G[key] = (torch.empty(shp, dtype=torch.float32, device="cuda") if fill is None
+                  else torch.full(shp, fill, dtype=torch.float32, device="cuda"))
     return G

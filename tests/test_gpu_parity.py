@@ -84,7 +84,7 @@ def outlier_fraction(a, b, tol):
 # the bf16-rounded x' as well, but a handful of hidden units with |z| inside the accumulation noise still
 # decide differently.  Each such unit changes isolated gradient elements, so for those tensors the
 # elementwise bound is required of all but 1e-3 of the elements and the Frobenius bound of the whole tensor.
-RELU_DECISION_KEYS = ("dx", "dw1", "dw2", "dw_down", "dw_gate", "db_gate")
+RELU_DECISION_KEYS = ("dx", "dw1", "dw2", "dw_down", "dw_gate", "db_gate", "db1")
 
 
 def compare_full(w, inp, got, tol=None, capacity_factor=0.0, aux=0.0):
@@ -96,7 +96,8 @@ def compare_full(w, inp, got, tol=None, capacity_factor=0.0, aux=0.0):
     assert abs(got["aux_loss"] - ref.get("aux_loss", 0.0)) <= 1e-5 * abs(ref.get("aux_loss", 0.0))
     ref["dw1"] = np.stack([ref["dw1"][e] for e in range(w.E)])
     ref["dw2"] = np.stack([ref["dw2"][e] for e in range(w.E)])
-    keys = ("y", "dx", "dw_gate", "dw1", "dw2", "db_gate") + (() if w.cdac else ("dw_up", "dw_down"))
+    keys = (("y", "dx", "dw_gate", "dw1", "dw2", "db_gate") + (() if w.cdac else ("dw_up", "dw_down")) +
+            (("db1", "db2") if w.expert_bias else ()))
     errs = float_errors(w, {key: got[key] for key in keys}, ref)
     if w.dtype == wl.DTYPE_BF16 and w.act == wl.ACT_RELU:
         for key in RELU_DECISION_KEYS:
