@@ -302,6 +302,53 @@ def run_recipe_variant(w, x, dy, dev, G, y, dx, base_step, steps):
     return out
 
 
+def run_small_variants(w, x, dy, dev, G, y, dx, base_step, steps):
+    """The two small variants of the layer on the same inputs, each timed alternately with the plain layer: the gate
+    reading the low-width token x' (w_gate [E,r]) and experts with biases (fp32 b1 [E,h], b2 [E,r])."""
+    import torch
+    from paper_2502_16927_b200 import binding
+
+    def timed(fn):
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(steps):
+            fn()
+        stop.record()
+        torch.cuda.synchronize()
+        return start.elapsed_time(stop) / steps
+
+    gen = torch.Generator(device="cuda").manual_seed(w.seed + 7)
+    out = {}
+    cases = {
+        "gate_on_low_width_token": (wl.FLAG_GATE_LOW,
+                                    {"w_gate": (torch.randn((w.E, w.r), generator=gen, device="cuda") * w.r ** -0.5).to(x.dtype)},
+                                    {"dw_gate": torch.empty((w.E, w.r), dtype=x.dtype, device="cuda")}),
+        "expert_biases": (wl.FLAG_EXPERT_BIAS,
+                          {"b1": torch.randn((w.E, w.h), generator=gen, device="cuda") * 0.5,
+                           "b2": torch.randn((w.E, w.r), generator=gen, device="cuda") * 0.5},
+                          {"db1": torch.empty((w.E, w.h), dtype=torch.float32, device="cuda"),
+                           "db2": torch.empty((w.E, w.r), dtype=torch.float32, device="cuda")}),
+    }
+    for name, (flag, extra_w, extra_g) in cases.items():
+        Wv, Gv = dict(dev, **extra_w), dict(G, **extra_g)
+        layer = binding.Layer(w.d, w.r, w.h, w.E, w.k, w.T, w.dtype, w.act, flag)
+
+        def step():
+            layer.forward(x, Wv, y=y, training=True)
+            layer.backward(x, dy, Wv, Gv, dx=dx)
+
+        for _ in range(3):
+            step()
+        pairs = [(timed(base_step), timed(step)) for _ in range(2)]
+        ms_base, ms = (sum(p[i] for p in pairs) / len(pairs) for i in (0, 1))
+        if layer.status() != 0:
+            raise RuntimeError("device status word reports a timed-out wait")
+        layer.close()
+        out[name] = {"ms_per_step": ms, "plain_layer_ms_per_step_beside_it": ms_base, "over_plain_layer_time": round(ms / ms_base, 3)}
+    return out
+
+
 def run_ep_on_one_gpu(w, x, dy, dev, ms_step, steps, esz, size=4):
     """The expert-parallel layer (Fig. 2c) with `size` ranks driven on this one GPU: every rank brings T/size of the
     step's tokens and owns E/size experts; rows travel between the ranks' buffers at width r through the same put /
@@ -557,6 +604,7 @@ def run_ours(args, w):
     esz = 2 if w.dtype == wl.DTYPE_BF16 else 4
     twin = run_cdac_twin(w, x, dy, dev, ms_step, ms_fwd, max(3, min(args.steps, 10)), peaks, esz)
     ep_line = run_ep_on_one_gpu(w, x, dy, dev, ms_step, max(3, min(args.steps, 10)), esz) if w.dtype == wl.DTYPE_BF16 else None
+    variants = run_small_variants(w, x, dy, dev, G, y, dx, step, max(3, min(args.steps, 10)))
     recipe = run_recipe_variant(w, x, dy, dev, G, y, dx, step, max(3, min(args.steps, 10)))
     stages = {}
     gemm_ms = gemm_flops = 0.0
@@ -612,6 +660,7 @@ def run_ours(args, w):
             "exchange": exchange,
             "cdac_twin": twin,
             "recipe_variant": recipe,
+            "small_variants": variants,
             "expert_parallel_on_one_gpu": ep_line,
             "stages": stages}
     print(json.dumps(line))

@@ -168,9 +168,11 @@ constexpr int kColsumChunks = 296;
 cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db, float* partial, int64_t N, int E,
                                bool accumulate, cudaStream_t stream, const float* aux_partial = nullptr);
 // Per-expert column sums of a grouped matrix (the expert-bias gradients): out[e, c] (+)= sum over the padded rows of
-// expert e of src[row, c] (padding rows hold zeros), fp32, fixed summation order.  width a multiple of 8 (bf16) / 4.
-cudaError_t launch_grouped_colsum(const void* src, const int32_t* poffsets, float* out, int E, int width, int dtype,
-                                  bool accumulate, cudaStream_t stream);
+// expert e of src[row, c] (padding rows hold zeros), fp32, fixed summation order.  width a multiple of 8 (bf16) / 4;
+// partial: E * kColsumSlices * width floats of scratch.
+constexpr int kColsumSlices = 32;
+cudaError_t launch_grouped_colsum(const void* src, const int32_t* poffsets, float* out, float* partial, int E, int width,
+                                  int dtype, bool accumulate, cudaStream_t stream);
 // Sum the `parts` fp32 partial results ws[s][m][n] of a split contraction in the order s = 0, 1, ... and write
 // rows [0, m_split) to dst1 [m_split, N] and rows [m_split, m_split + m2) to dst2 [m2, N] (dst2 may be null),
 // in the dtype, adding to the destination if `accumulate`.

@@ -110,7 +110,10 @@ void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
     // fp32 partial results: of the split dense contractions, and of the parts of long experts in dW1 / dW2
     const size_t dense_ws = (size_t)kMaxSplitK * m.ldcat * m.d * sizeof(float);
     const size_t expert_ws = m.dtype == BIGMAC_BF16 ? gemm_tc_groupk_ws_bytes(m.r, m.h, m.E) : 0;
-    b.splitk_ws = (float*)cv.take_bytes(dense_ws > expert_ws ? dense_ws : expert_ws);
+    const size_t bias_ws = m.bias ? (size_t)m.E * kColsumSlices * (m.h > m.r ? m.h : m.r) * sizeof(float) : 0;
+    size_t ws = dense_ws > expert_ws ? dense_ws : expert_ws;
+    if (bias_ws > ws) ws = bias_ws;
+    b.splitk_ws = (float*)cv.take_bytes(ws);
 }
 
 size_t forward_scratch_bytes(const Dims& m, bool training) {
@@ -511,9 +514,10 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     void* dz = b.dz ? b.dz : b.z;
     if (m.bias) {   // db1_e = sum_rows dz[row,:], db2_e = sum_rows du[row,:]  (padding rows hold zeros)
         if (!aligned(G->db1, 4) || !aligned(G->db2, 4)) return BIGMAC_ERR_INVALID_ARG;
-        Stage s(L, S_COLSUM, st, (G->db1 ? 1 : 0) + (G->db2 ? 1 : 0));
-        if (G->db1) BIGMAC_CUDA(launch_grouped_colsum(dz, b.tb.poffsets, G->db1, m.E, m.h, m.dtype, acc, st));
-        if (G->db2) BIGMAC_CUDA(launch_grouped_colsum(b.du, b.tb.poffsets, G->db2, m.E, m.r, m.dtype, acc, st));
+        Stage s(L, S_COLSUM, st, 2 * ((G->db1 ? 1 : 0) + (G->db2 ? 1 : 0)));
+        // the fp32 workspace is free here: the split dW_up has been reduced, the per-expert weight gradients come later
+        if (G->db1) BIGMAC_CUDA(launch_grouped_colsum(dz, b.tb.poffsets, G->db1, b.splitk_ws, m.E, m.h, m.dtype, acc, st));
+        if (G->db2) BIGMAC_CUDA(launch_grouped_colsum(b.du, b.tb.poffsets, G->db2, b.splitk_ws, m.E, m.r, m.dtype, acc, st));
     }
     if (G->dw2) {   // dW2_e[c',q] = sum_rows du[row,c'] a[row,q]
         GemmArgs g;

@@ -232,20 +232,38 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
     dst[0] = (T)acc.x; dst[1] = (T)acc.y; dst[2] = (T)acc.z; dst[3] = (T)acc.w;
 }
 
-// Per-expert column sums (expert-bias gradients).  Block (cg, e): 32 column-threads x 8 row-lanes; a thread adds rows
-// lane, lane + 8, ... of its 16-byte column vector in order, then the 8 row-lanes are added in order.
+// Per-expert column sums (expert-bias gradients), in two deterministic steps so that one long segment does not
+// serialise.  Step 1, block (cg, e, s): slice s of kColsumSlices equal row ranges of expert e's padded segment; 32
+// column-threads x 8 row-lanes, a thread adds rows lane, lane + 8, ... of its 16-byte column vector in order, then the
+// 8 row-lanes are added in order -> partial[e][s][:].  Step 2 adds the slices in order.
 template <typename T>
 __global__ void __launch_bounds__(256) grouped_colsum_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ poffsets,
-                                                             float* __restrict__ out, int vecs_per_row, int accumulate) {
+                                                             float* __restrict__ partial, int vecs_per_row) {
     constexpr int V = Vec<T>::kElems;
     __shared__ float part[8][32 * V];
-    const int e = blockIdx.y, ct = threadIdx.x & 31, rl = threadIdx.x >> 5;
+    const int e = blockIdx.y, slice = blockIdx.z, ct = threadIdx.x & 31, rl = threadIdx.x >> 5;
     const int c = blockIdx.x * 32 + ct;
+    const int64_t r0 = poffsets[e], rows = poffsets[e + 1] - r0;
+    const int64_t per = (rows + kColsumSlices - 1) / kColsumSlices;
+    const int64_t first = r0 + slice * per, last = min(r0 + rows, first + per);
     float acc[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) acc[i] = 0.0f;
     if (c < vecs_per_row) {
-        for (int64_t row = (int64_t)poffsets[e] + rl; row < poffsets[e + 1]; row += 8) {
+        int64_t row = first + rl;
+        for (; row + 24 < last; row += 32) {           // four rows in flight per thread
+            uint4 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) q[u] = src[(row + 8 * u) * vecs_per_row + c];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float f[V];
+                Vec<T>::unpack(q[u], f);
+#pragma unroll
+                for (int i = 0; i < V; ++i) acc[i] += f[i];
+            }
+        }
+        for (; row < last; row += 8) {
             float f[V];
             Vec<T>::unpack(src[row * vecs_per_row + c], f);
 #pragma unroll
@@ -255,14 +273,23 @@ __global__ void __launch_bounds__(256) grouped_colsum_kernel(const uint4* __rest
 #pragma unroll
     for (int i = 0; i < V; ++i) part[rl][ct * V + i] = acc[i];
     __syncthreads();
+    const int width = vecs_per_row * V;
     for (int j = threadIdx.x; j < 32 * V; j += blockDim.x) {
         const int col = blockIdx.x * 32 * V + j;
-        if (col >= vecs_per_row * V) continue;
+        if (col >= width) continue;
         float total = 0.0f;
         for (int q = 0; q < 8; ++q) total += part[q][j];
-        float* dst = out + (int64_t)e * vecs_per_row * V + col;
-        *dst = accumulate ? *dst + total : total;
+        partial[((int64_t)e * kColsumSlices + slice) * width + col] = total;
     }
+}
+__global__ void __launch_bounds__(256) grouped_colsum_final_kernel(const float* __restrict__ partial, float* __restrict__ out,
+                                                                   int64_t n, int width, int accumulate) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;      // i = e * width + col
+    if (i >= n) return;
+    const int64_t e = i / width, col = i - e * width;
+    float total = 0.0f;
+    for (int s = 0; s < kColsumSlices; ++s) total += partial[(e * kColsumSlices + s) * width + col];
+    out[i] = accumulate ? out[i] + total : total;
 }
 
 inline int elem_bytes(int dtype) { return dtype == BIGMAC_BF16 ? 2 : 4; }
@@ -329,15 +356,17 @@ cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db
     return cudaGetLastError();
 }
 
-cudaError_t launch_grouped_colsum(const void* src, const int32_t* poffsets, float* out, int E, int width, int dtype,
-                                  bool accumulate, cudaStream_t stream) {
+cudaError_t launch_grouped_colsum(const void* src, const int32_t* poffsets, float* out, float* partial, int E, int width,
+                                  int dtype, bool accumulate, cudaStream_t stream) {
     if (E == 0 || width == 0) return cudaSuccess;
     const int vecs = width * elem_bytes(dtype) / 16;
-    dim3 grid((unsigned)((vecs + 31) / 32), (unsigned)E);
+    dim3 grid((unsigned)((vecs + 31) / 32), (unsigned)E, (unsigned)kColsumSlices);
     if (dtype == BIGMAC_BF16)
-        grouped_colsum_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const uint4*)src, poffsets, out, vecs, accumulate ? 1 : 0);
+        grouped_colsum_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const uint4*)src, poffsets, partial, vecs);
     else
-        grouped_colsum_kernel<float><<<grid, 256, 0, stream>>>((const uint4*)src, poffsets, out, vecs, accumulate ? 1 : 0);
+        grouped_colsum_kernel<float><<<grid, 256, 0, stream>>>((const uint4*)src, poffsets, partial, vecs);
+    const int64_t n = (int64_t)E * width;
+    grouped_colsum_final_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(partial, out, n, width, accumulate ? 1 : 0);
     return cudaGetLastError();
 }
 
