@@ -61,6 +61,14 @@ ROW_MOVE_BYTES = {   # per launch, algorithmic: rows read + rows written (+ the 
 }
 
 
+# The two expert contractions whose outputs are larger than their inputs sit nearer to an HBM floor than to the tensor
+# one; algorithmic bytes per launch (b = bytes per element; sigma' is saved as one byte per element on the BF16 path).
+OUTPUT_HEAVY_GEMM_BYTES = {
+    "gemm_expert1": lambda w, b: (w.N * w.r + w.E * w.h * w.r + w.N * w.h) * b + w.N * w.h * (1 if b == 2 else b),
+    "gemm_dz": lambda w, b: (w.N * w.r + w.E * w.h * w.r + w.N * w.h) * b + w.N * w.h * (1 if b == 2 else b),
+}
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -624,6 +632,9 @@ def run_ours(args, w):
             entry["frac_of_measured_sustained"] = round(entry["tflops"] / peaks["tflops_sustained"], 3)
             gemm_ms += ms
             gemm_flops += fl * calls
+            if name in OUTPUT_HEAVY_GEMM_BYTES:
+                entry["hbm_gbs"] = round(OUTPUT_HEAVY_GEMM_BYTES[name](w, esz) / (per * 1e-3) / 1e9, 1)
+                entry["frac_of_measured_hbm"] = round(entry["hbm_gbs"] / peaks["hbm_gbs"], 3)
         elif name in ROW_MOVE_BYTES:
             by = ROW_MOVE_BYTES[name](w, esz)
             entry["gbs"] = round(by / (per * 1e-3) / 1e9, 1)
