@@ -195,9 +195,11 @@ int bigmac_backward(bigmac_layer_t *L, const void *x, const void *dy, int32_t T,
                     void *saved, void *dx, const bigmac_grads_t *G, int accumulate, void *scratch,
                     size_t scratch_bytes, void *stream);
 
-/* Synchronise `stream` and return the device status word (BIGMAC_OK, or BIGMAC_ERR_TIMEOUT if a
- * bounded wait inside a kernel ran out, in which case outputs of that call are undefined).  The word
- * is cleared by the call. */
+/* Synchronise `stream` and return the device status word (BIGMAC_OK; BIGMAC_ERR_TIMEOUT if a
+ * bounded wait inside a kernel ran out, in which case outputs of that call are undefined;
+ * BIGMAC_ERR_STATE if bigmac_ep_dispatch found a count matrix that cannot be right - a negative entry or
+ * more rows than an owner's buffers hold - in which case that step moved and computed nothing and no
+ * memory outside the buffers was touched).  The word is cleared by the call. */
 int bigmac_device_status(bigmac_layer_t *L, void *stream);
 
 const char *bigmac_status_string(int status);

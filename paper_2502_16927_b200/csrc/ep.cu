@@ -58,9 +58,18 @@ template <> struct Row<__nv_bfloat16> {
 
 // One block.  From counts_all [size, E]: where this rank's slots of every expert start at their owner (send_base),
 // and the tables of the segments this rank owns (padded offsets, tile -> local expert, tiles in use).
+// A count matrix that cannot be right (a negative entry, or more rows for one owner than its buffers hold: the caller
+// skipped the all-gather, or passed another step's) must not turn into stores outside the buffers: the kernel then
+// records kBadCounts in the status word and publishes an empty layout (send_base -1, no tiles), which every later
+// kernel of the step treats as "nothing to move".
+constexpr int kBadCounts = 2;
 __global__ void __launch_bounds__(1024) ep_layout_kernel(const int32_t* __restrict__ counts_all, int size, int rank, int E, int El,
+                                                         int64_t max_rows, int* __restrict__ status,
                                                          int32_t* __restrict__ send_base, int32_t* __restrict__ poff_own,
                                                          int32_t* __restrict__ tile_expert_own, int32_t* __restrict__ n_tiles_own) {
+    __shared__ int s_bad;
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
     __shared__ int32_t s_total[kMaxExperts];     // rows of expert e over all ranks
     __shared__ int32_t s_before[kMaxExperts];    // ... of the ranks before this one
     __shared__ int32_t s_poff[kMaxExperts];      // padded offset of expert e in its owner's buffers
@@ -69,7 +78,8 @@ __global__ void __launch_bounds__(1024) ep_layout_kernel(const int32_t* __restri
         int total = 0, before = 0;
         for (int p = 0; p < size; ++p) {
             const int c = counts_all[(size_t)p * E + e];
-            total += c;
+            if (c < 0 || (int64_t)c > max_rows) { s_bad = 1; continue; }
+            total += c;                          // at most size * max_rows: no overflow
             if (p < rank) before += c;
         }
         s_total[e] = total;
@@ -78,14 +88,21 @@ __global__ void __launch_bounds__(1024) ep_layout_kernel(const int32_t* __restri
     __syncthreads();
     if ((int)threadIdx.x < size) {               // owner q: prefix over its experts
         const int q = threadIdx.x;
-        int poff = 0;
+        int64_t poff = 0;
         for (int j = 0; j < El; ++j) {
-            s_poff[q * El + j] = poff;
-            poff += (s_total[q * El + j] + kPad - 1) / kPad * kPad;
+            s_poff[q * El + j] = (int32_t)(poff < max_rows ? poff : max_rows);
+            poff += ((int64_t)s_total[q * El + j] + kPad - 1) / kPad * kPad;
         }
-        s_end[q] = poff;
+        if (poff > max_rows) s_bad = 1;
+        s_end[q] = (int32_t)(poff < max_rows ? poff : max_rows);
     }
     __syncthreads();
+    if (s_bad) {
+        for (int e = threadIdx.x; e < E; e += blockDim.x) send_base[e] = -1;
+        for (int j = threadIdx.x; j <= El; j += blockDim.x) poff_own[j] = 0;
+        if (threadIdx.x == 0) { *n_tiles_own = 0; atomicExch(status, kBadCounts); }
+        return;
+    }
     for (int e = threadIdx.x; e < E; e += blockDim.x) send_base[e] = s_poff[e] + s_before[e];
     for (int j = threadIdx.x; j <= El; j += blockDim.x) poff_own[j] = j < El ? s_poff[rank * El + j] : s_end[rank];
     if (threadIdx.x == 0) *n_tiles_own = s_end[rank] / kPad;
@@ -102,9 +119,14 @@ __global__ void __launch_bounds__(256) ep_zero_padding_kernel(uint4* __restrict_
                                                               const int32_t* __restrict__ counts_all, int size, int rank, int E,
                                                               int El, int vecs) {
     const int j = blockIdx.x;
-    int total = 0;
-    for (int p = 0; p < size; ++p) total += counts_all[(size_t)p * E + rank * El + j];
+    int64_t total = 0;
+    for (int p = 0; p < size; ++p) {
+        const int c = counts_all[(size_t)p * E + rank * El + j];
+        if (c < 0) return;                           // rejected by ep_layout_kernel: the layout is empty
+        total += c;
+    }
     const int64_t first = (int64_t)poff_own[j] + total, last = poff_own[j + 1];
+    if (first >= last) return;                       // no padding rows (or an empty layout)
     const int64_t n = (last - first) * vecs;
     for (int64_t i = threadIdx.x; i < n; i += blockDim.x) {
         buf_a[first * vecs + i] = make_uint4(0, 0, 0, 0);
@@ -121,7 +143,12 @@ __global__ void __launch_bounds__(256) ep_put_rows_kernel(const uint4* __restric
     if (s >= N) return;
     const int lane = threadIdx.x & 31;
     const int e = topk_idx[s];
-    const int dest = send_base[e] + row_of_slot[s] - offsets[e];
+    const int base = send_base[e];
+    if (base < 0) {                                  // empty layout (see ep_layout_kernel): nothing moves
+        if (lane == 0) dest_row[s] = -1;
+        return;
+    }
+    const int dest = base + row_of_slot[s] - offsets[e];
     if (lane == 0) dest_row[s] = dest;
     const uint4* from = src + (s / k) * vecs;
     uint4* to = (uint4*)dst.p[e / El] + (int64_t)dest * vecs;
@@ -145,9 +172,11 @@ __global__ void __launch_bounds__(256) ep_get_combine_kernel(Peers src, uint4* _
         for (int i = 0; i < V; ++i) acc[i] = 0.0f;
         for (int j = 0; j < k; ++j) {
             const int64_t s = (int64_t)t * k + j;
+            const int row = dest_row[s];
+            if (row < 0) continue;                       // empty layout
             const float p = w ? w[s] : 1.0f;
             float f[V];
-            Row<T>::unpack(((const uint4*)src.p[topk_idx[s] / El])[(int64_t)dest_row[s] * vecs + c], f);
+            Row<T>::unpack(((const uint4*)src.p[topk_idx[s] / El])[(int64_t)row * vecs + c], f);
 #pragma unroll
             for (int i = 0; i < V; ++i) acc[i] = fmaf(p, f[i], acc[i]);
         }
@@ -167,6 +196,10 @@ __global__ void __launch_bounds__(256) ep_combine_bwd_kernel(const uint4* __rest
     const int lane = threadIdx.x & 31;
     const int q = topk_idx[s] / El;
     const int64_t row = dest_row[s];
+    if (row < 0) {                                   // empty layout
+        if (lane == 0) dp[s] = 0.0f;
+        return;
+    }
     const float p = topk_w[s];
     const uint4* g = dy_lo + (s / k) * vecs;
     const uint4* ur = (const uint4*)u.p[q] + row * vecs;
@@ -382,8 +415,8 @@ int bigmac_ep_dispatch(bigmac_layer_t* L, int32_t T, const bigmac_ep_t* ep, void
     cudaStream_t st = (cudaStream_t)stream;
     const int vecs = m.r * (int)esize(m.dtype) / 16;
     Stage s(L, S_DISPATCH, st, T > 0 ? 3 : 2);
-    ep_layout_kernel<<<1, 1024, 0, st>>>(ep->counts_all, m.size, m.rank, m.E, m.El, b.send_base, b.poff_own, b.tile_expert_own,
-                                         b.n_tiles_own);
+    ep_layout_kernel<<<1, 1024, 0, st>>>(ep->counts_all, m.size, m.rank, m.E, m.El, m.Pep, L->status, b.send_base, b.poff_own,
+                                         b.tile_expert_own, b.n_tiles_own);
     ep_zero_padding_kernel<<<m.El, 256, 0, st>>>((uint4*)ep->xg[m.rank], (uint4*)ep->du[m.rank], b.poff_own, ep->counts_all, m.size,
                                                  m.rank, m.E, m.El, vecs);
     if (T > 0)

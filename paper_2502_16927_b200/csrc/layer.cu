@@ -674,6 +674,7 @@ int bigmac_device_status(bigmac_layer_t* L, void* stream) {
         if (cudaMemsetAsync(L->status + 1, 0, 3 * sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
             return BIGMAC_ERR_CUDA;
     }
+    if (word == 2) return BIGMAC_ERR_STATE;            // an expert-parallel step was given a count matrix that cannot be right
     return word == 0 ? BIGMAC_OK : BIGMAC_ERR_TIMEOUT;
 }
 
@@ -685,7 +686,7 @@ const char* bigmac_status_string(int status) {
         case BIGMAC_ERR_WORKSPACE: return "workspace too small";
         case BIGMAC_ERR_CUDA: return "CUDA error";
         case BIGMAC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
-        case BIGMAC_ERR_STATE: return "handle used on the wrong device";
+        case BIGMAC_ERR_STATE: return "handle used on the wrong device, or an expert-parallel count matrix that cannot be right";
         case BIGMAC_ERR_TOO_LARGE: return "problem exceeds the fixed scratch array of bigmac_route_static";
         default: return "unknown status";
     }

@@ -143,3 +143,50 @@ def test_one_rank_per_process_plumbing_with_a_group_of_one():
     finally:
         dist.destroy_process_group()
     compare(w, inp, got)
+
+
+@pytest.mark.parametrize("bad", [1 << 30, -5])
+def test_a_count_matrix_that_cannot_be_right_is_refused_on_the_device(bad):
+    """A rank whose count matrix was not gathered properly (here: another rank's row holds impossible values) must not
+    store outside the buffers: its step moves and computes nothing, the status word says so, the handle stays usable."""
+    import torch
+
+    w = wl.Workload("ep", T=400, d=64, r=24, h=40, E=8, k=3, dtype=wl.DTYPE_F32, act=wl.ACT_GELU_ERF, seed=137)
+    inp = skewed(w, 1.0)
+    dev = to_device(w, inp)
+    Ws = [ep.shard_weights(dev, q, 2) for q in range(2)]
+    xs = [dev["x"][:200].contiguous(), dev["x"][200:].contiguous()]
+    dys = [dev["dy"][:200].contiguous(), dev["dy"][200:].contiguous()]
+    group = ep.EpLocalGroup(w.d, w.r, w.h, w.E, w.k, 200, w.dtype, w.act, ["cuda"] * 2)
+    for buf in group.ranks[0].buffers.values():
+        buf.fill_(0)
+    for rk in group.ranks:
+        rk.route(xs[rk.rank], Ws[rk.rank])
+    group.ranks[0].counts_all[1].fill_(bad)               # rank 0 never received rank 1's counts
+    group.ranks[1].counts_all[0].copy_(group.ranks[0].counts_all[0])
+    ys = [torch.full_like(x, float("nan")) for x in xs]
+    rk0 = group.ranks[0]
+    rk0.dispatch()
+    rk0.experts(Ws[0])
+    rk0.combine(Ws[0], ys[0])
+    G = {"dw_gate": torch.empty_like(dev["w_gate"]), "dw_down": torch.empty_like(dev["w_down"]), "dw_up": torch.empty_like(dev["w_up"]),
+         "dw1": torch.empty_like(Ws[0]["w1"]), "dw2": torch.empty_like(Ws[0]["w2"]),
+         "db_gate": torch.empty(w.E, dtype=torch.float32, device="cuda")}
+    dx = torch.empty_like(xs[0])
+    rk0.backward_combine(dys[0], Ws[0], G)
+    rk0.backward_experts(Ws[0], G)
+    rk0.backward_dispatch(xs[0], Ws[0], dx, G)
+    torch.cuda.synchronize()
+    assert rk0.status() == -6                               # BIGMAC_ERR_STATE, and the word is cleared by the read
+    assert rk0.status() == 0
+    assert not bool(ys[0].any())                            # nothing was combined: y' = 0
+    assert not bool(G["dw1"].any()) and not bool(G["dw2"].any())
+    assert not bool(rk0.buffers["xg"].any()) and not bool(rk0.buffers["du"].any())     # its puts went nowhere
+    # the same handles run a proper step afterwards
+    got_y = group.forward(xs, Ws)
+    torch.cuda.synchronize()
+    assert group.status() == 0
+    rt = oracle.route(inp, w.k)
+    ref = oracle.forward_tokens(inp, rt, w.act)["y"]
+    assert oracle.rel_err(np.concatenate([to_numpy(v) for v in got_y]), ref) <= TOL[w.dtype]
+    group.close()
