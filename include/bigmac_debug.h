@@ -32,6 +32,12 @@ typedef struct {
 
 int bigmac_debug_gemm(bigmac_layer_t *L, const bigmac_debug_gemm_t *q, int use_tensor_cores, void *stream);
 
+/* Test aid for the failure path of the device-side waits: launches a one-thread kernel that waits, with the same
+ * bounded wait the TMA / MMA pipelines use but a limit of 4096 polls, on a barrier nobody arrives at.  The wait runs
+ * out, the kernel records it in the handle's status word and returns normally (no trap, no fault): the next
+ * bigmac_device_status returns BIGMAC_ERR_TIMEOUT and the handle and the context stay usable. */
+int bigmac_debug_expire_wait(bigmac_layer_t *L, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -88,6 +88,8 @@ def lib() -> C.CDLL:
         L.bigmac_status_string.restype = C.c_char_p
         L.bigmac_exchange_rows.argtypes = [vp, vp, i32, i32, vp, vp, sz, vp, C.c_int, vp]
         L.bigmac_debug_gemm.argtypes = [vp, C.POINTER(bigmac_debug_gemm_t), C.c_int, vp]
+        L.bigmac_debug_expire_wait.argtypes = [vp, vp]
+        L.bigmac_debug_expire_wait.restype = C.c_int
         L.bigmac_route_static.argtypes = [vp, vp, i32, C.POINTER(bigmac_weights_t), C.POINTER(bigmac_routing_t), vp]
         L.bigmac_route_static.restype = C.c_int
         L.bigmac_profile_enable.argtypes = [vp, C.c_int]
@@ -223,6 +225,11 @@ def bigmac_profile_read(handle) -> Dict[str, object]:
 def bigmac_debug_gemm(handle, q: bigmac_debug_gemm_t, use_tensor_cores) -> None:
     """use_tensor_cores: False/0 plain FMA, True/1 tensor cores, 2 one-CTA kernel, 3 CTA-pair kernel."""
     _check(lib().bigmac_debug_gemm(handle, C.byref(q), int(use_tensor_cores), _stream()), "bigmac_debug_gemm")
+
+
+def bigmac_debug_expire_wait(handle) -> None:
+    """Launch the one-thread kernel whose bounded wait runs out (failure path of the device-side waits)."""
+    _check(lib().bigmac_debug_expire_wait(handle, _stream()), "bigmac_debug_expire_wait")
 
 
 # ---- expert parallelism: the phase calls, name for name ----------------------------------------------------

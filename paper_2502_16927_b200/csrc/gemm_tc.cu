@@ -328,6 +328,26 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
 bool gemm_tc_available() { return encode_fn() != nullptr; }
 int gemm_tc_sm_count() { return sm_count(); }
 
+namespace {
+// One thread waits, with the pipelines' bounded wait and a short limit, on a barrier nobody arrives at: the wait
+// runs out, the status word is set and the kernel returns.
+__global__ void expire_wait_kernel(int* status) {
+    __shared__ uint64_t bar;
+    __shared__ int dead_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        dead_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(&bar, 0, &dead_flag, status, 1u << 12);
+    }
+}
+}  // namespace
+
+cudaError_t launch_expire_wait(int* status, cudaStream_t stream) {
+    expire_wait_kernel<<<1, 32, 0, stream>>>(status);
+    return cudaGetLastError();
+}
+
 cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
     // Where it pays, the problem runs on CTA pairs (each SM stages half of B); BIGMAC_TC_PAIR=0 disables that.

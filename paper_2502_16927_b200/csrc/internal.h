@@ -87,6 +87,8 @@ bool gemm_tc_pair_supported(const GemmArgs& g);
 bool gemm_tc_pair_preferred(const GemmArgs& g);
 cudaError_t gemm_tc_pair(const GemmArgs& g, int* status, cudaStream_t stream);
 int gemm_tc_sm_count();
+// Test aid: a one-thread kernel whose bounded barrier wait runs out after a short limit and records it in `status`.
+cudaError_t launch_expire_wait(int* status, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------------
 // Routing tables held in device memory (internal superset of bigmac_routing_t).

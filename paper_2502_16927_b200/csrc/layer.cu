@@ -840,4 +840,10 @@ int bigmac_debug_gemm(bigmac_layer_t* L, const bigmac_debug_gemm_t* q, int use_t
     return err == cudaSuccess ? BIGMAC_OK : BIGMAC_ERR_CUDA;
 }
 
+int bigmac_debug_expire_wait(bigmac_layer_t* L, void* stream) {
+    if (!L) return BIGMAC_ERR_INVALID_ARG;
+    L->launches += 1;
+    return launch_expire_wait(L->status, (cudaStream_t)stream) == cudaSuccess ? BIGMAC_OK : BIGMAC_ERR_CUDA;
+}
+
 }  // extern "C"

@@ -60,9 +60,10 @@ __device__ __forceinline__ void mbar_spin(uint64_t* bar, uint32_t parity, volati
     atomicExch(status, 1);
 }
 // Bounded wait.  `dead` is a CTA-wide flag in shared memory: once any wait ran out nobody waits again.
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile int* dead, int* status) {
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile int* dead, int* status,
+                                          uint32_t limit = kWaitLimit) {
     if (*dead) return;
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return;
         if ((i & 1023u) == 1023u && *dead) return;
     }

@@ -40,3 +40,30 @@ def test_two_runs_agree_bit_for_bit(case):
             (junk @ junk).sum().item()
     for key, val in runs[0].items():
         assert torch.equal(val.view(torch.uint8), runs[1][key].view(torch.uint8)), key
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_handle_usable():
+    """Failure path of the device-side waits, made without a fault: a one-thread kernel polls, with the pipelines'
+    bounded wait and a short limit, a barrier nobody arrives at; it gives up, records that in the status word and
+    returns.  The host reads BIGMAC_ERR_TIMEOUT once; the same handle then computes a correct step."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_2502_16927_b200 import binding
+    from helpers import to_numpy
+
+    w = wl.Workload("to", T=300, d=128, r=64, h=128, E=8, k=2, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=139)
+    inp = conditioned(w)
+    dev = to_device(w, inp)
+    layer = make_layer(w)
+    assert layer.status() == 0
+    binding.bigmac_debug_expire_wait(layer.handle)
+    assert layer.status() == -5                            # BIGMAC_ERR_TIMEOUT
+    assert layer.status() == 0                             # cleared by the read
+    y = layer.forward(dev["x"], dev, training=False)
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    ref = oracle.forward_tokens(inp, oracle.route(inp, w.k), w.act)["y"]
+    assert oracle.max_rel_err(to_numpy(y), ref) <= 2e-2
+    layer.close()
