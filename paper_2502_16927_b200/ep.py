@@ -157,9 +157,9 @@ class EpRank:
 class EpLocalGroup:
     """`size` ranks driven by this process.  devices[q] is rank q's GPU; the same GPU may appear several times."""
 
-    def __init__(self, d, r, h, E, k, max_tokens, dtype, act, devices: Sequence, flags=0):
+    def __init__(self, d, r, h, E, k, max_tokens, dtype, act, devices: Sequence, flags=0, alloc=None):
         self.size = len(devices)
-        self.ranks = [EpRank(d, r, h, E, k, max_tokens, dtype, act, q, self.size, devices[q], flags)
+        self.ranks = [EpRank(d, r, h, E, k, max_tokens, dtype, act, q, self.size, devices[q], flags, alloc=alloc)
                       for q in range(self.size)]
         distinct = sorted({rk.device.index or 0 for rk in self.ranks})
         for a in distinct:

@@ -67,3 +67,117 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_handle_usable():
     ref = oracle.forward_tokens(inp, oracle.route(inp, w.k), w.act)["y"]
     assert oracle.max_rel_err(to_numpy(y), ref) <= 2e-2
     layer.close()
+
+
+GUARD = 4096
+
+
+def _guarded(nbytes, like=None, shape=None, dtype=None):
+    """A buffer of exactly nbytes with GUARD bytes of 0xA5 on both sides; returns (whole, interior view)."""
+    import torch
+
+    whole = torch.full((GUARD + nbytes + GUARD,), 0xA5, dtype=torch.uint8, device="cuda")
+    inner = whole[GUARD:GUARD + nbytes]
+    if dtype is not None:
+        inner = inner.view(dtype).view(shape)
+    return whole, inner
+
+
+def _intact(whole, nbytes):
+    return bool((whole[:GUARD] == 0xA5).all()) and bool((whole[GUARD + nbytes:] == 0xA5).all())
+
+
+@pytest.mark.parametrize("case", [
+    dict(shape=dict(T=333, d=40, r=12, h=20, E=7, k=3), dtype=wl.DTYPE_F32, kw=dict()),
+    dict(shape=dict(T=1000, d=128, r=64, h=192, E=12, k=5), dtype=wl.DTYPE_BF16, kw=dict()),
+    dict(shape=dict(T=2500, d=256, r=256, h=512, E=16, k=2), dtype=wl.DTYPE_BF16, kw=dict(capacity_factor=1.0, aux_loss_coef=2.0)),
+    dict(shape=dict(T=700, d=128, r=128, h=256, E=8, k=2), dtype=wl.DTYPE_BF16, kw=dict(), bias=True),
+])
+def test_no_kernel_writes_outside_the_buffers_it_was_given(case):
+    """Every buffer of a training forward + backward is given at exactly the size the library asks for, between guard
+    bands; a store past either end of any of them (workspaces, saved state, outputs, gradients, tables) would change a
+    guard byte without necessarily faulting."""
+    import numpy as np
+    import torch
+
+    from paper_2502_16927_b200 import binding
+
+    w = wl.Workload("gb", dtype=case["dtype"], act=wl.ACT_GELU_ERF, seed=149, expert_bias=case.get("bias", False), **case["shape"])
+    inp = conditioned(w)
+    inp["b_gate"] = (2.0 * np.linspace(1.0, -1.0, w.E) ** 3).astype(np.float32)
+    dev = to_device(w, inp)
+    layer = make_layer(w, **case["kw"])
+    tdt = torch.float32 if w.dtype == wl.DTYPE_F32 else torch.bfloat16
+    es = 4 if w.dtype == wl.DTYPE_F32 else 2
+    s_bytes, v_bytes = binding.bigmac_workspace_bytes(layer.handle, w.T, True)
+    held = {}
+
+    def buf(name, nbytes, shape=None, dtype=None):
+        whole, inner = _guarded(nbytes, shape=shape, dtype=dtype)
+        held[name] = (whole, nbytes)
+        return inner
+
+    scratch, saved = buf("scratch", s_bytes), buf("saved", v_bytes)
+    y = buf("y", w.T * w.d * es, (w.T, w.d), tdt)
+    dx = buf("dx", w.T * w.d * es, (w.T, w.d), tdt)
+    N = w.T * w.k
+    R = {"topk_idx": buf("topk_idx", 4 * N, (N,), torch.int32), "topk_w": buf("topk_w", 4 * N, (N,), torch.float32),
+         "counts": buf("counts", 4 * w.E, (w.E,), torch.int32), "offsets": buf("offsets", 4 * (w.E + 1), (w.E + 1,), torch.int32),
+         "row_of_slot": buf("row_of_slot", 4 * N, (N,), torch.int32), "slot_of_row": buf("slot_of_row", 4 * N, (N,), torch.int32),
+         "counts_chosen": buf("counts_chosen", 4 * w.E, (w.E,), torch.int32), "aux_loss": buf("aux_loss", 4, (1,), torch.float32)}
+    shapes = {"dw_gate": (w.E, w.d), "dw_down": (w.r, w.d), "dw1": (w.E, w.h, w.r), "dw2": (w.E, w.r, w.h), "dw_up": (w.d, w.r)}
+    G = {key: buf(key, int(np.prod(shp)) * es, shp, tdt) for key, shp in shapes.items()}
+    G["db_gate"] = buf("db_gate", 4 * w.E, (w.E,), torch.float32)
+    if w.expert_bias:
+        G["db1"] = buf("db1", 4 * w.E * w.h, (w.E, w.h), torch.float32)
+        G["db2"] = buf("db2", 4 * w.E * w.r, (w.E, w.r), torch.float32)
+    binding.bigmac_forward(layer.handle, dev["x"], w.T, dev, y, R, saved, scratch)
+    binding.bigmac_backward(layer.handle, dev["x"], dev["dy"], w.T, dev, saved, dx, G, False, scratch)
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    for name, (whole, nbytes) in held.items():
+        assert _intact(whole, nbytes), name
+    assert bool(torch.isfinite(y.float()).all()) and bool(torch.isfinite(dx.float()).all())
+    layer.close()
+
+
+def test_expert_parallel_exchange_stays_inside_the_exchange_buffers():
+    """The puts of every rank land inside the owners' buffers of exactly bigmac_ep_buffer_bytes, also when one rank's
+    experts receive nearly all rows: guard bands around all sixteen buffers stay intact."""
+    import numpy as np
+    import torch
+
+    from paper_2502_16927_b200 import ep
+
+    w = wl.Workload("gb", T=1200, d=128, r=64, h=128, E=8, k=2, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=151)
+    inp = conditioned(w)
+    b = np.full(w.E, -6.0, dtype=np.float32)
+    b[:2] = 6.0                                             # everybody's two choices are rank 0's experts
+    inp["b_gate"] = b
+    dev = to_device(w, inp)
+    size, Tq = 4, 300
+    held = []
+
+    def alloc(nbytes):
+        whole, inner = _guarded(nbytes)
+        held.append((whole, nbytes))
+        return inner
+
+    group = ep.EpLocalGroup(w.d, w.r, w.h, w.E, w.k, Tq, w.dtype, w.act, ["cuda"] * size, alloc=alloc)
+    Ws = [ep.shard_weights(dev, q, size) for q in range(size)]
+    xs = [dev["x"][q * Tq:(q + 1) * Tq].contiguous() for q in range(size)]
+    dys = [dev["dy"][q * Tq:(q + 1) * Tq].contiguous() for q in range(size)]
+    ys = group.forward(xs, Ws)
+    Gs = [{"dw_gate": torch.empty_like(dev["w_gate"]), "dw_down": torch.empty_like(dev["w_down"]), "dw_up": torch.empty_like(dev["w_up"]),
+           "dw1": torch.empty_like(Ws[q]["w1"]), "dw2": torch.empty_like(Ws[q]["w2"]),
+           "db_gate": torch.empty(w.E, dtype=torch.float32, device="cuda")} for q in range(size)]
+    group.backward(xs, dys, Ws, Gs)
+    torch.cuda.synchronize()
+    assert group.status() == 0
+    assert len(held) == 4 * size
+    for whole, nbytes in held:
+        assert _intact(whole, nbytes)
+    counts = group.ranks[0].counts_all.sum(dim=0)
+    assert int(counts[:2].sum()) == w.T * w.k               # all rows went to rank 0's first two experts
+    assert bool(torch.isfinite(torch.cat(ys).float()).all())
+    group.close()
