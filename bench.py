@@ -640,6 +640,17 @@ def run_ours(args, w):
             entry["gbs"] = round(by / (per * 1e-3) / 1e9, 1)
             entry["frac_of_measured_hbm"] = round(entry["gbs"] / peaks["hbm_gbs"], 3)
         stages[name] = entry
+    # the two groups the target names: the per-expert (grouped) contractions together, the row-move kernels together
+    grouped = [n for n in ("gemm_expert1", "gemm_expert2", "gemm_dz", "gemm_dw2", "gemm_dxg", "gemm_dw1") if n in stages]
+    g_ms = sum(stages[n]["ms"] for n in grouped)
+    g_tf = sum(flops_of[n] for n in grouped) / (g_ms * 1e-3) / 1e12 if g_ms > 0 else 0.0
+    moves = [n for n in ROW_MOVE_BYTES if n in stages]
+    m_ms = sum(stages[n]["ms"] for n in moves)
+    m_gbs = sum(ROW_MOVE_BYTES[n](w, esz) for n in moves) / (m_ms * 1e-3) / 1e9 if m_ms > 0 else 0.0
+    groups = {"grouped_expert_gemms": {"ms": round(g_ms, 4), "tflops": round(g_tf, 1),
+                                       "frac_of_measured_sustained": round(g_tf / peaks["tflops_sustained"], 3)},
+              "dispatch_combine_and_their_backward": {"ms": round(m_ms, 4), "gbs": round(m_gbs, 1),
+                                                      "frac_of_measured_hbm": round(m_gbs / peaks["hbm_gbs"], 3)}}
     achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
     fwd_fl = forward_flops(w)
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (tcgen05 contractions, all launches of a step)",
@@ -673,6 +684,7 @@ def run_ours(args, w):
             "recipe_variant": recipe,
             "small_variants": variants,
             "expert_parallel_on_one_gpu": ep_line,
+            "groups": groups,
             "stages": stages}
     print(json.dumps(line))
     if world > 1:
