@@ -9,7 +9,7 @@ from oracle import margin
 from paper_2502_16927_b200 import binding, workloads as wl
 
 from helpers import make_layer, to_device, to_numpy
-from test_gpu_parity import TOL, assert_within, check_routing, float_errors, run_full
+from test_gpu_parity import RELU_DECISION_KEYS, TOL, assert_within, check_routing, float_errors, outlier_fraction, run_full
 
 pytestmark = pytest.mark.gpu
 
@@ -39,7 +39,13 @@ def compare(w, inp, got, capacity_factor=0.0):
     ref["dw2"] = np.stack([ref["dw2"][e] for e in range(w.E)])
     keys = ("y", "dx", "dw_gate", "dw1", "dw2", "db_gate", "dw_up", "dw_down")
     assert got["dw_gate"].shape == (w.E, w.r)
-    assert_within(w, float_errors(w, {key: got[key] for key in keys}, ref))
+    errs = float_errors(w, {key: got[key] for key in keys}, ref)
+    if bf16 and w.act == wl.ACT_RELU:                  # isolated ReLU' decisions inside the accumulation noise (see test_gpu_parity)
+        for key in RELU_DECISION_KEYS:
+            if key in keys:
+                assert outlier_fraction(got[key], ref[key], TOL[w.dtype]) <= 1e-3, key
+                errs.pop(key)
+    assert_within(w, errs)
 
 
 @pytest.mark.parametrize("shape", [
@@ -59,8 +65,9 @@ def test_fp32_gate_on_the_low_width_token(shape, act):
     dict(T=1500, d=128, r=64, h=128, E=24, k=3),
 ])
 @pytest.mark.parametrize("flags", [0, wl.FLAG_SIMT_GEMM])
-def test_bf16_gate_on_the_low_width_token(shape, flags):
-    w = wl.Workload("gl", dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=89, gate_low=True, **shape)
+@pytest.mark.parametrize("act", [wl.ACT_GELU_ERF, wl.ACT_RELU])
+def test_bf16_gate_on_the_low_width_token(shape, flags, act):
+    w = wl.Workload("gl", dtype=wl.DTYPE_BF16, act=act, seed=89, gate_low=True, **shape)
     inp = conditioned(w, 1.0)
     compare(w, inp, run_full(w, inp, flags))
 
