@@ -392,7 +392,7 @@ int bigmac_ep_route(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_we
         BIGMAC_TRY(gemm(L, G_DESCEND, q, st));
     }
     { Stage s(L, S_TOPK, st); BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st)); }
-    { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, kNoCapacity, st)); }
+    { Stage s(L, S_TABLES, st, tables_kernel_count(m.N, m.E)); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, kNoCapacity, st)); }
     BIGMAC_CUDA(cudaMemcpyAsync(my_counts, b.tb.counts, sizeof(int32_t) * m.E, cudaMemcpyDeviceToDevice, st));
     if (routing_out) {
         const cudaMemcpyKind kind = cudaMemcpyDeviceToDevice;

@@ -180,7 +180,7 @@ int choose_split_k(int M, int N, int K) {
 // any), load-balancing loss.
 int route_from_logits(const bigmac_layer* L, const Dims& m, const bigmac_weights_t* W, Buffers& b, cudaStream_t st) {
     { Stage s(L, S_TOPK, st); BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st)); }
-    { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st)); }
+    { Stage s(L, S_TABLES, st, tables_kernel_count(m.N, m.E)); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st)); }
     if (m.aux > 0) {
         Stage s(L, S_AUX_LOSS, st, 2);
         BIGMAC_CUDA(launch_aux_loss(b.logits, W->b_gate, b.tb.counts_chosen, m.T, m.E, m.k, m.aux, b.aux_part, b.aux_loss, st));
@@ -374,7 +374,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
                                               m.k, c.act, gemm_tc_sm_count(), st));
         }
         if (routing_out) {
-            { Stage s(L, S_TABLES, st, 3); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st)); }
+            { Stage s(L, S_TABLES, st, tables_kernel_count(m.N, m.E)); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st)); }
             BIGMAC_TRY(export_routing(m, b, routing_out, st));
         }
         return BIGMAC_OK;

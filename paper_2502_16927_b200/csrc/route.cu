@@ -284,6 +284,91 @@ __global__ void __launch_bounds__(256) sort_place_kernel(const int32_t* __restri
     slot_of_prow[prow] = (int32_t)s;
 }
 
+// All three passes (and the fill of slot_of_prow) in ONE block, for the few thousand slots of decode-shaped batches,
+// where four launches cost more than the work.  1024 threads; chunk c holds slots [1024 c, 1024 (c + 1)), warp w of
+// it the 32 slots from 1024 c + 32 w: ranks inside a warp by match_any, across the warps of a chunk by a scan over the
+// per-warp counts, across chunks by the running per-expert totals - the same stable order as the three-pass sort.
+__global__ void __launch_bounds__(1024) tables_small_kernel(const int32_t* __restrict__ topk_idx, int N, int E, int cap, int P,
+                                                            int32_t* __restrict__ counts, int32_t* __restrict__ counts_chosen,
+                                                            int32_t* __restrict__ offsets, int32_t* __restrict__ poffsets,
+                                                            int32_t* __restrict__ tile_expert, int32_t* __restrict__ n_tiles,
+                                                            int32_t* __restrict__ prow_of_slot, int32_t* __restrict__ row_of_slot,
+                                                            int32_t* __restrict__ slot_of_row, int32_t* __restrict__ slot_of_prow) {
+    extern __shared__ int32_t sm[];                  // [32][E] per-warp counts of the chunk, [E] totals so far, 2 x [E+1]: 35 E + 2 ints
+    int32_t* warp_run = sm;
+    int32_t* total = sm + 32 * E;
+    int32_t* s_off = total + E;
+    int32_t* s_poff = s_off + E + 1;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < P; i += blockDim.x) slot_of_prow[i] = -1;
+    if (cap < N)
+        for (int i = threadIdx.x; i < N; i += blockDim.x) slot_of_row[i] = -1;
+    for (int e = threadIdx.x; e < E; e += blockDim.x) total[e] = 0;
+    const int chunks = (N + 1023) / 1024;
+    int32_t rank_of[kSmallTablesMaxSlots / 1024];    // this thread's slot of every chunk: rank among its expert's slots
+#pragma unroll
+    for (int c = 0; c < kSmallTablesMaxSlots / 1024; ++c) {
+        if (c >= chunks) break;                      // uniform
+        for (int i = threadIdx.x; i < 32 * E; i += blockDim.x) warp_run[i] = 0;
+        __syncthreads();
+        const int s = c * 1024 + threadIdx.x;
+        const int e = s < N ? topk_idx[s] : -1;
+        const unsigned peers = __match_any_sync(kFull, e);
+        if (e >= 0 && lane == __ffs(peers) - 1) warp_run[warp * E + e] = __popc(peers);
+        const int in_warp = __popc(peers & ((1u << lane) - 1u));
+        __syncthreads();
+        for (int x = threadIdx.x; x < E; x += blockDim.x) {      // exclusive scan over the warps, on top of the earlier chunks
+            int run = total[x];
+            for (int w = 0; w < 32; ++w) {
+                const int n = warp_run[w * E + x];
+                warp_run[w * E + x] = run;
+                run += n;
+            }
+            total[x] = run;
+        }
+        __syncthreads();
+        rank_of[c] = e >= 0 ? warp_run[warp * E + e] + in_warp : 0;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int off = 0, poff = 0;
+        for (int e = 0; e < E; ++e) {
+            const int kept = min(total[e], cap);
+            s_off[e] = off;
+            s_poff[e] = poff;
+            off += kept;
+            poff += (kept + kPad - 1) / kPad * kPad;
+        }
+        s_off[E] = off;
+        s_poff[E] = poff;
+        *n_tiles = poff / kPad;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e <= E; e += blockDim.x) { offsets[e] = s_off[e]; poffsets[e] = s_poff[e]; }
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        counts[e] = min(total[e], cap);
+        if (counts_chosen) counts_chosen[e] = total[e];
+        for (int tile = s_poff[e] / kPad; tile < s_poff[e + 1] / kPad; ++tile) tile_expert[tile] = e;
+    }
+#pragma unroll
+    for (int c = 0; c < kSmallTablesMaxSlots / 1024; ++c) {
+        if (c >= chunks) break;
+        const int s = c * 1024 + threadIdx.x;
+        if (s >= N) continue;
+        const int e = topk_idx[s], within = rank_of[c];
+        if (within >= cap) {
+            row_of_slot[s] = -1;
+            prow_of_slot[s] = -1;
+            continue;
+        }
+        const int row = s_off[e] + within, prow = s_poff[e] + within;
+        row_of_slot[s] = row;
+        slot_of_row[row] = s;
+        prow_of_slot[s] = prow;
+        slot_of_prow[prow] = s;
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, int k, int32_t* topk_idx,
@@ -324,6 +409,12 @@ cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, 
 cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaStream_t stream) {
     const int64_t N = (int64_t)T * k;
     const int64_t P = padded_rows_max(N, E);
+    if (tables_kernel_count(N, E) == 1) {
+        tables_small_kernel<<<1, 1024, sizeof(int32_t) * (35 * E + 2), stream>>>(
+            tb.topk_idx, (int)N, E, cap, (int)P, tb.counts, tb.counts_chosen, tb.offsets, tb.poffsets, tb.tile_expert, tb.n_tiles,
+            tb.prow_of_slot, tb.row_of_slot, tb.slot_of_row, tb.slot_of_prow);
+        return cudaGetLastError();
+    }
     cudaError_t err = cudaMemsetAsync(tb.slot_of_prow, 0xff, sizeof(int32_t) * P, stream);
     if (err != cudaSuccess) return err;
     if (cap < N) {                                   // rows past the kept ones exist only under a capacity limit

@@ -385,3 +385,24 @@ def test_inference_forward_with_the_experts_in_one_kernel(case):
     # same roundings (bf16 activations, fp32 accumulation), different accumulation grouping only
     assert oracle.max_rel_err(to_numpy(y), to_numpy(y_train)) <= 2.0 ** -7
     layer.close()
+
+
+@pytest.mark.parametrize("T,E,k", [(1, 1, 1), (31, 7, 1), (128, 256, 8), (1024, 5, 1), (205, 64, 5), (256, 256, 8),
+                                   (2048, 3, 1), (257, 16, 8), (683, 40, 3), (300, 300, 7)])
+@pytest.mark.parametrize("f", [0.0, 0.7])
+def test_routing_tables_around_the_single_block_limit(T, E, k, f):
+    """Up to 2048 slots and 256 experts the tables come from one single-block kernel (one or two chunks of 1024
+    slots), beyond from the three-pass sort: both sides of both limits, with and without a capacity limit."""
+    import torch
+
+    w = wl.Workload("tb", T=T, d=32, r=8, h=8, E=E, k=k, dtype=wl.DTYPE_F32, act=wl.ACT_RELU, seed=157)
+    inp = conditioned(w)
+    inp["b_gate"] = (2.0 * np.linspace(1.0, -1.0, E) ** 3).astype(np.float32)
+    margin.enforce_margin(w, inp, 1e-3)
+    dev = to_device(w, inp)
+    layer = make_layer(w, capacity_factor=f)
+    R = layer.route(dev["x"], dev)
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    check_routing(R, oracle.route(inp, w.k, capacity_factor=f))
+    layer.close()
