@@ -132,6 +132,8 @@ def test_one_rank_per_process_plumbing_with_a_group_of_one():
         try:
             rank = ep.EpProcessRank(w.d, w.r, w.h, w.E, w.k, w.T, w.dtype, w.act)
         except (RuntimeError, NotImplementedError) as err:       # torch's symmetric memory is not available on this host
+            if isinstance(err, binding.BigmacError):
+                raise
             pytest.skip(f"torch symmetric memory unavailable: {err}")
         y = rank.forward(dev["x"], dev)
         G = {"dw_gate": torch.empty_like(dev["w_gate"]), "dw_down": torch.empty_like(dev["w_down"]),
