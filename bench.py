@@ -361,23 +361,38 @@ def run_ep_on_one_gpu(w, x, dy, dev, ms_step, steps, esz, size=4):
     """The expert-parallel layer (Fig. 2c) with `size` ranks driven on this one GPU: every rank brings T/size of the
     step's tokens and owns E/size experts; rows travel between the ranks' buffers at width r through the same put /
     get kernels a multi-GPU job runs, here within one memory.  What this measures is the cost of the phase structure
-    and of the exchange kernels against the one-GPU layer on the same tokens; link time it cannot show.  The bytes
-    that would cross the links per rank and exchange are reported for width r and, for comparison, width d (Eq. 1)."""
+    and of the exchange kernels against the one-GPU layer on the same tokens; link time it cannot show.  Beside it the
+    conventional layer of Eq. 3 with equal E, k and expert parameters runs the same way, its rows travelling at width d:
+    the exchange kernels' times and the bytes that would cross the links per rank and exchange (Eq. 1) are set against
+    each other."""
     import torch
     from paper_2502_16927_b200 import binding, ep
 
     if w.E % size or w.T % size:
         return None
+    if not w.cdac:                                   # beside it: the parameter-parity twin of Eq. 3, rows at width d
+        twin = None
+        if w.dtype == wl.DTYPE_BF16 and (w.r * w.h) % w.d == 0 and (w.r * w.h // w.d) % 64 == 0:
+            t = w.cdac_twin()
+            gen = torch.Generator(device="cuda").manual_seed(w.seed + 11)
+            tw = {"w_gate": dev["w_gate"],
+                  "w1": (torch.randn((t.E, t.h, t.d), generator=gen, device="cuda") * t.d ** -0.5).to(torch.bfloat16),
+                  "w2": (torch.randn((t.E, t.d, t.h), generator=gen, device="cuda") * t.h ** -0.5).to(torch.bfloat16)}
+            if "b_gate" in dev:
+                tw["b_gate"] = dev["b_gate"]
+            twin = run_ep_on_one_gpu(t, x, dy, tw, None, steps, esz, size)
     Tq = w.T // size
     Ws = [ep.shard_weights(dev, q, size) for q in range(size)]
     xs = [x[q * Tq:(q + 1) * Tq] for q in range(size)]
     dys = [dy[q * Tq:(q + 1) * Tq] for q in range(size)]
     ys, dxs = [torch.empty_like(v) for v in xs], [torch.empty_like(v) for v in xs]
     per = w.E // size
-    Gs = [{"dw_gate": torch.empty_like(dev["w_gate"]), "dw_down": torch.empty_like(dev["w_down"]),
-           "dw_up": torch.empty_like(dev["w_up"]), "dw1": torch.empty_like(Ws[q]["w1"]), "dw2": torch.empty_like(Ws[q]["w2"]),
+    Gs = [{"dw_gate": torch.empty_like(dev["w_gate"]), "dw1": torch.empty_like(Ws[q]["w1"]), "dw2": torch.empty_like(Ws[q]["w2"]),
            "db_gate": torch.empty(w.E, dtype=torch.float32, device="cuda")} for q in range(size)]
-    group = ep.EpLocalGroup(w.d, w.r, w.h, w.E, w.k, Tq, w.dtype, w.act, ["cuda"] * size)
+    if not w.cdac:
+        for G in Gs:
+            G.update(dw_down=torch.empty_like(dev["w_down"]), dw_up=torch.empty_like(dev["w_up"]))
+    group = ep.EpLocalGroup(w.d, w.r, w.h, w.E, w.k, Tq, w.dtype, w.act, ["cuda"] * size, wl.FLAG_CDAC if w.cdac else 0)
 
     def step():
         group.forward(xs, Ws, ys)
@@ -404,12 +419,21 @@ def run_ep_on_one_gpu(w, x, dy, dev, ms_step, steps, esz, size=4):
     if group.status() != 0:
         raise RuntimeError("device status word reports a timed-out wait")
     group.close()
-    return {"ranks_on_this_gpu": size, "tokens_per_rank": Tq, "experts_per_rank": per, "ms_per_step_all_ranks": ms,
-            "tokens_per_s": w.T / (ms * 1e-3), "over_one_gpu_layer_time": round(ms / ms_step, 3),
-            "exchange_kernels_ms_all_ranks": {name: round(v, 4) for name, v in moves.items()},
-            "link_bytes_per_rank_per_exchange": {"width_r": ep.exchange_bytes_per_rank(Tq, w.k, w.r, size, esz),
-                                                 "width_d": ep.exchange_bytes_per_rank(Tq, w.k, w.d, size, esz)},
-            "note": "ranks share one GPU: no link is crossed; exchanges per step: 2 forward, 2 backward"}
+    out = {"ranks_on_this_gpu": size, "tokens_per_rank": Tq, "experts_per_rank": per, "row_width": w.r, "ms_per_step_all_ranks": ms,
+           "tokens_per_s": w.T / (ms * 1e-3),
+           "exchange_kernels_ms_all_ranks": {name: round(v, 4) for name, v in moves.items()},
+           "exchange_kernels_ms_total": round(sum(moves.values()), 4),
+           "link_bytes_per_rank_per_exchange": ep.exchange_bytes_per_rank(Tq, w.k, w.r, size, esz)}
+    if w.cdac:
+        return out
+    out["over_one_gpu_layer_time"] = round(ms / ms_step, 3)
+    out["eq3_twin_rows_at_width_d"] = twin
+    if twin:
+        out["bigmac_over_twin"] = {"step_time": round(ms / twin["ms_per_step_all_ranks"], 3),
+                                   "exchange_kernel_time": round(out["exchange_kernels_ms_total"] / twin["exchange_kernels_ms_total"], 3),
+                                   "link_bytes": round(out["link_bytes_per_rank_per_exchange"] / twin["link_bytes_per_rank_per_exchange"], 4)}
+    out["note"] = "ranks share one GPU: no link is crossed; exchanges per step: 2 forward, 2 backward"
+    return out
 
 
 # ------------------------------------------------------------------------------------------------ ours

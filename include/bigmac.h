@@ -232,7 +232,10 @@ const char *bigmac_status_string(int status);
  * `saved` (and, across the three backward calls, `scratch`) must keep their contents between the calls of a step.
  * The gradients of the shared matrices that the backward returns are this rank's share (the sum over its own
  * tokens): the caller adds them over the ranks, as for any data-parallel layer; dw1 / dw2 are complete.
- * Not supported together with a capacity factor, a load-balancing loss, BIGMAC_FLAG_CDAC, BIGMAC_FLAG_GATE_LOW or
+ * With BIGMAC_FLAG_CDAC the same calls run the conventional layer of Eq. 3 under expert parallelism: no shared
+ * projections, the rows that travel are the tokens themselves at the full width d (Eq. 1 as written), w1 / w2 of the
+ * owned experts are [E/size,h,d] / [E/size,d,h], w_down / w_up and their gradients are ignored.
+ * Not supported together with a capacity factor, a load-balancing loss, BIGMAC_FLAG_GATE_LOW or
  * BIGMAC_FLAG_EXPERT_BIAS (BIGMAC_ERR_UNSUPPORTED). */
 #define BIGMAC_EP_MAX_RANKS 8
 typedef struct {

@@ -226,6 +226,7 @@ struct EpDims {
     int T, d, r, h, E, El, k, dtype, size, rank;
     int64_t N, P, Pep;   // this rank's slots, its local padded bound (tables), the bound on rows it can receive
     int E64, z_es, ldcat;
+    bool cdac;           // Eq. 3 layer: no shared projections, rows travel at the full width d (r == d)
 };
 
 struct EpBuffers {
@@ -242,7 +243,7 @@ int ep_dims(const bigmac_layer* L, int32_t T, int size, int rank, EpDims* out) {
     const bigmac_config_t& c = L->cfg;
     if (size < 1 || size > kMaxRanks || rank < 0 || rank >= size) return BIGMAC_ERR_INVALID_ARG;
     if (c.E % size) return BIGMAC_ERR_INVALID_ARG;
-    if (c.capacity_factor > 0 || c.aux_loss_coef > 0 || (c.flags & (BIGMAC_FLAG_CDAC | BIGMAC_FLAG_GATE_LOW | BIGMAC_FLAG_EXPERT_BIAS)))
+    if (c.capacity_factor > 0 || c.aux_loss_coef > 0 || (c.flags & (BIGMAC_FLAG_GATE_LOW | BIGMAC_FLAG_EXPERT_BIAS)))
         return BIGMAC_ERR_UNSUPPORTED;
     if ((int64_t)size * c.max_tokens * c.k > (int64_t)1 << 30) return BIGMAC_ERR_UNSUPPORTED;
     EpDims m{};
@@ -253,7 +254,8 @@ int ep_dims(const bigmac_layer* L, int32_t T, int size, int rank, EpDims* out) {
     m.Pep = padded_rows_max((int64_t)size * c.max_tokens * c.k, m.El);
     m.E64 = (c.E + 63) / 64 * 64;
     m.z_es = sigma_as_bytes(L) ? 1 : (int)esize(c.dtype);
-    m.ldcat = m.r + m.E64;
+    m.cdac = (c.flags & BIGMAC_FLAG_CDAC) != 0;
+    m.ldcat = m.cdac ? m.E64 : m.r + m.E64;
     *out = m;
     return BIGMAC_OK;
 }
@@ -295,8 +297,8 @@ void carve_ep_scratch(Carver& cv, const EpDims& m, EpBuffers& b) {
     b.tb.block_counts = cv.take<int32_t>((size_t)(sort_blocks(m.N) + 1) * m.E);
     b.dy_lo = cv.take_bytes((size_t)m.T * m.r * es);
     b.dcat = cv.take_bytes((size_t)m.T * m.ldcat * es);
-    b.dx_lo = b.dcat;
-    b.dlogits = (char*)b.dcat + (size_t)m.r * es;
+    b.dx_lo = m.cdac ? nullptr : b.dcat;                              // Eq. 3: dx' is dx itself
+    b.dlogits = m.cdac ? b.dcat : (char*)b.dcat + (size_t)m.r * es;
     b.dp = cv.take<float>(m.N);
 }
 
@@ -330,12 +332,12 @@ Peers peers_of(void* const* bufs, int size) {
     return p;
 }
 
-int check_shared_weights(const bigmac_weights_t* W, bool experts) {
+int check_shared_weights(const bigmac_weights_t* W, bool experts, bool cdac = false) {
     if (!W) return BIGMAC_ERR_INVALID_ARG;
     if (experts) return (W->w1 && W->w2 && aligned(W->w1, 16) && aligned(W->w2, 16)) ? BIGMAC_OK : BIGMAC_ERR_INVALID_ARG;
-    if (!W->w_gate || !W->w_down || !W->w_up || !aligned(W->w_gate, 16) || !aligned(W->w_down, 16) || !aligned(W->w_up, 16) ||
-        !aligned(W->b_gate, 4))
-        return BIGMAC_ERR_INVALID_ARG;
+    if (!W->w_gate || !aligned(W->w_gate, 16) || !aligned(W->b_gate, 4)) return BIGMAC_ERR_INVALID_ARG;
+    if (cdac) return BIGMAC_OK;
+    if (!W->w_down || !W->w_up || !aligned(W->w_down, 16) || !aligned(W->w_up, 16)) return BIGMAC_ERR_INVALID_ARG;
     return BIGMAC_OK;
 }
 
@@ -366,7 +368,7 @@ int bigmac_ep_route(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_we
     EpDims m;
     EpBuffers b{};
     BIGMAC_TRY(ep_enter(L, T, ep, saved, scratch, scratch_bytes, true, &m, &b));
-    BIGMAC_TRY(check_shared_weights(W, false));
+    BIGMAC_TRY(check_shared_weights(W, false, m.cdac));
     cudaStream_t st = (cudaStream_t)stream;
     int32_t* my_counts = ep->counts_all + (size_t)m.rank * m.E;
     if (T == 0) {                                    // this rank brings nothing: its row of the count matrix is zero
@@ -375,7 +377,13 @@ int bigmac_ep_route(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_we
     }
     if (!x || !aligned(x, 16)) return BIGMAC_ERR_INVALID_ARG;
     const int bn_desc = (m.r + m.E) >= 256 ? 256 : 128;
-    if (m.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u && m.r % bn_desc == 0) {
+    if (m.cdac) {                                    // Eq. 3: logits only; the rows that travel are the tokens themselves,
+        GemmArgs g;                                  // kept in `saved` so that the dispatch phase needs no x
+        g.A = x; g.lda = m.d; g.B = W->w_gate; g.ldb = m.d; g.C = b.logits; g.ldc = m.E;
+        g.M = m.T; g.N = m.E; g.K = m.d; g.out_f32 = true;
+        BIGMAC_TRY(gemm(L, G_LOGITS, g, st));
+        BIGMAC_CUDA(cudaMemcpyAsync(b.x_lo, x, (size_t)m.T * m.d * esize(m.dtype), cudaMemcpyDeviceToDevice, st));
+    } else if (m.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u && m.r % bn_desc == 0) {
         GemmArgs g;                                  // [x' | logits] = x [W'_down ; W_gate]^T in one pass over x
         g.A = x; g.lda = m.d; g.B = W->w_down; g.ldb = m.d; g.C = b.x_lo; g.ldc = m.r;
         g.B2 = W->w_gate; g.ldb2 = m.d; g.n_split = m.r; g.C2 = b.logits; g.ldc2 = m.E; g.N2 = m.E;
@@ -456,21 +464,23 @@ int bigmac_ep_combine(bigmac_layer_t* L, int32_t T, const bigmac_weights_t* W, c
     EpDims m;
     EpBuffers b{};
     BIGMAC_TRY(ep_enter(L, T, ep, saved, nullptr, 0, false, &m, &b));
-    BIGMAC_TRY(check_shared_weights(W, false));
+    BIGMAC_TRY(check_shared_weights(W, false, m.cdac));
     if (T == 0) return BIGMAC_OK;
     if (!y || !aligned(y, 16)) return BIGMAC_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int vecs = m.r * (int)esize(m.dtype) / 16;
+    uint4* y_lo = (uint4*)(m.cdac ? y : b.y_lo);     // Eq. 3: the weighted sum is the output
     {
         Stage s(L, S_COMBINE, st);
         if (m.dtype == BIGMAC_BF16)
-            ep_get_combine_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, st>>>(peers_of(ep->u, m.size), (uint4*)b.y_lo, b.tb.topk_w,
+            ep_get_combine_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, st>>>(peers_of(ep->u, m.size), y_lo, b.tb.topk_w,
                                                                                 b.tb.topk_idx, b.dest_row, T, m.k, m.El, vecs, vecs);
         else
-            ep_get_combine_kernel<float><<<warp_blocks(T), 256, 0, st>>>(peers_of(ep->u, m.size), (uint4*)b.y_lo, b.tb.topk_w,
+            ep_get_combine_kernel<float><<<warp_blocks(T), 256, 0, st>>>(peers_of(ep->u, m.size), y_lo, b.tb.topk_w,
                                                                         b.tb.topk_idx, b.dest_row, T, m.k, m.El, vecs, vecs);
         BIGMAC_CUDA(cudaGetLastError());
     }
+    if (m.cdac) return BIGMAC_OK;
     GemmArgs g;                                      // y = y' W'_up
     g.A = b.y_lo; g.lda = m.r; g.B = W->w_up; g.ldb = m.r; g.C = y; g.ldc = m.d;
     g.M = m.T; g.N = m.d; g.K = m.r;
@@ -483,20 +493,21 @@ int bigmac_ep_backward_combine(bigmac_layer_t* L, const void* dy, int32_t T, con
     EpDims m;
     EpBuffers b{};
     BIGMAC_TRY(ep_enter(L, T, ep, saved, scratch, scratch_bytes, true, &m, &b));
-    BIGMAC_TRY(check_shared_weights(W, false));
+    BIGMAC_TRY(check_shared_weights(W, false, m.cdac));
     if (!G) return BIGMAC_ERR_INVALID_ARG;
     if (T == 0) return BIGMAC_OK;
     if (!dy || !aligned(dy, 16) || !aligned(G->dw_up, 16)) return BIGMAC_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const bool acc = accumulate != 0;
     const bool fused = m.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u;
-    {   // dy' = dy W_up
+    const void* dy_lo = m.cdac ? dy : b.dy_lo;       // Eq. 3: dy' is dy
+    if (!m.cdac) {   // dy' = dy W_up
         GemmArgs g;
         g.A = dy; g.lda = m.d; g.B = W->w_up; g.ldb = m.r; g.b_kmajor = false; g.C = b.dy_lo; g.ldc = m.r;
         g.M = m.T; g.N = m.r; g.K = m.d;
         BIGMAC_TRY(gemm(L, G_DY_LO, g, st));
     }
-    if (G->dw_up) {   // dW_up[c,c'] = sum_t dy[t,c] y'[t,c']   (this rank's tokens)
+    if (G->dw_up && !m.cdac) {   // dW_up[c,c'] = sum_t dy[t,c] y'[t,c']   (this rank's tokens)
         GemmArgs g;
         g.A = dy; g.lda = m.d; g.a_kmajor = false; g.B = b.y_lo; g.ldb = m.r; g.b_kmajor = false;
         g.C = G->dw_up; g.ldc = m.r; g.M = m.d; g.N = m.r; g.K = m.T; g.accumulate = acc;
@@ -513,11 +524,11 @@ int bigmac_ep_backward_combine(bigmac_layer_t* L, const void* dy, int32_t T, con
     {
         Stage s(L, S_COMBINE_BWD, st);
         if (m.dtype == BIGMAC_BF16)
-            ep_combine_bwd_kernel<__nv_bfloat16><<<warp_blocks(m.N), 256, 0, st>>>((const uint4*)b.dy_lo, peers_of(ep->u, m.size),
+            ep_combine_bwd_kernel<__nv_bfloat16><<<warp_blocks(m.N), 256, 0, st>>>((const uint4*)dy_lo, peers_of(ep->u, m.size),
                                                                                   peers_of(ep->du, m.size), b.dp, b.tb.topk_w,
                                                                                   b.tb.topk_idx, b.dest_row, m.N, m.k, m.El, vecs);
         else
-            ep_combine_bwd_kernel<float><<<warp_blocks(m.N), 256, 0, st>>>((const uint4*)b.dy_lo, peers_of(ep->u, m.size),
+            ep_combine_bwd_kernel<float><<<warp_blocks(m.N), 256, 0, st>>>((const uint4*)dy_lo, peers_of(ep->u, m.size),
                                                                           peers_of(ep->du, m.size), b.dp, b.tb.topk_w, b.tb.topk_idx,
                                                                           b.dest_row, m.N, m.k, m.El, vecs);
         BIGMAC_CUDA(cudaGetLastError());
@@ -575,7 +586,7 @@ int bigmac_ep_backward_dispatch(bigmac_layer_t* L, const void* x, int32_t T, con
     EpDims m;
     EpBuffers b{};
     BIGMAC_TRY(ep_enter(L, T, ep, saved, scratch, scratch_bytes, true, &m, &b));
-    BIGMAC_TRY(check_shared_weights(W, false));
+    BIGMAC_TRY(check_shared_weights(W, false, m.cdac));
     if (!G) return BIGMAC_ERR_INVALID_ARG;
     if (T == 0) return BIGMAC_OK;
     if (!x || !dx || !aligned(x, 16) || !aligned(dx, 16) || !aligned(G->dw_gate, 16) || !aligned(G->dw_down, 16) ||
@@ -585,15 +596,41 @@ int bigmac_ep_backward_dispatch(bigmac_layer_t* L, const void* x, int32_t T, con
     const bool acc = accumulate != 0;
     const bool fused = m.dtype == BIGMAC_BF16 && L->use_tc && L->tc_mask == ~0u;
     const int vecs = m.r * (int)esize(m.dtype) / 16, dvecs = m.ldcat * (int)esize(m.dtype) / 16;
+    uint4* gather_to = (uint4*)(m.cdac ? dx : b.dx_lo);          // Eq. 3: the gathered rows are dx (before the gate's share)
+    const int gather_ld = m.cdac ? vecs : dvecs;
     {   // dx'[t] = sum_j dxg[row of slot (t,j) at its owner]
         Stage s(L, S_DXLO_GATHER, st);
         if (m.dtype == BIGMAC_BF16)
-            ep_get_combine_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, st>>>(peers_of(ep->dxg, m.size), (uint4*)b.dx_lo, nullptr,
-                                                                                b.tb.topk_idx, b.dest_row, T, m.k, m.El, vecs, dvecs);
+            ep_get_combine_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, st>>>(peers_of(ep->dxg, m.size), gather_to, nullptr,
+                                                                                b.tb.topk_idx, b.dest_row, T, m.k, m.El, vecs, gather_ld);
         else
-            ep_get_combine_kernel<float><<<warp_blocks(T), 256, 0, st>>>(peers_of(ep->dxg, m.size), (uint4*)b.dx_lo, nullptr,
-                                                                        b.tb.topk_idx, b.dest_row, T, m.k, m.El, vecs, dvecs);
+            ep_get_combine_kernel<float><<<warp_blocks(T), 256, 0, st>>>(peers_of(ep->dxg, m.size), gather_to, nullptr,
+                                                                        b.tb.topk_idx, b.dest_row, T, m.k, m.El, vecs, gather_ld);
         BIGMAC_CUDA(cudaGetLastError());
+    }
+    if (m.cdac) {
+        {   // dx += dl W_gate
+            GemmArgs g;
+            g.A = b.dlogits; g.lda = m.ldcat; g.B = W->w_gate; g.ldb = m.d; g.b_kmajor = false; g.C = dx; g.ldc = m.d;
+            g.M = m.T; g.N = m.d; g.K = m.E; g.accumulate = true;
+            BIGMAC_TRY(gemm(L, G_DX_GATE, g, st));
+        }
+        if (G->dw_gate) {   // dW_gate = dl^T x
+            GemmArgs g;
+            g.A = b.dlogits; g.lda = m.ldcat; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
+            g.M = m.E; g.N = m.d; g.K = m.T;
+            if (fused) {
+                g.C = b.splitk_ws; g.ldc = m.d; g.out_f32 = true; g.M = m.ldcat; g.split_k = choose_split_k(g.M, g.N, g.K);
+                BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
+                Stage s(L, S_SPLITK_REDUCE, st);
+                BIGMAC_CUDA(launch_splitk_reduce(b.splitk_ws, g.split_k, m.ldcat, m.d, G->dw_gate, m.E, nullptr, 0, m.dtype, acc, st));
+            } else {
+                g.C = G->dw_gate; g.ldc = m.d; g.accumulate = acc;
+                BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
+            }
+        }
+        if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st)); }
+        return BIGMAC_OK;
     }
     if (fused) {
         {   // dx = [dx' | dl] [W_down ; W_gate]

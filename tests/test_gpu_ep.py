@@ -10,7 +10,7 @@ import oracle
 from oracle import margin
 from paper_2502_16927_b200 import binding, ep, workloads as wl
 
-from helpers import to_device, to_numpy
+from helpers import oracle_inputs, to_device, to_numpy
 from test_gpu_parity import TOL, assert_within, float_errors
 
 pytestmark = pytest.mark.gpu
@@ -30,6 +30,8 @@ def run_group(w, inp, tokens_per_rank, flags=0):
     bounds = np.concatenate([[0], np.cumsum(tokens_per_rank)])
     xs = [dev["x"][bounds[q]:bounds[q + 1]].contiguous() for q in range(size)]
     dys = [dev["dy"][bounds[q]:bounds[q + 1]].contiguous() for q in range(size)]
+    if w.cdac:
+        flags |= wl.FLAG_CDAC
     group = ep.EpLocalGroup(w.d, w.r, w.h, w.E, w.k, max(max(tokens_per_rank), 1), w.dtype, w.act, ["cuda"] * size, flags)
     ys = group.forward(xs, Ws)
     dt = torch.float32 if w.dtype == wl.DTYPE_F32 else torch.bfloat16
@@ -37,6 +39,8 @@ def run_group(w, inp, tokens_per_rank, flags=0):
     Gs = []
     for q in range(size):
         shapes = {"dw_gate": (w.E, w.d), "dw_down": (w.r, w.d), "dw_up": (w.d, w.r), "dw1": (per, w.h, w.r), "dw2": (per, w.r, w.h)}
+        if w.cdac:
+            del shapes["dw_down"], shapes["dw_up"]
         G = {key: torch.full(shp, float("nan"), dtype=dt, device="cuda") for key, shp in shapes.items()}
         G["db_gate"] = torch.full((w.E,), float("nan"), dtype=torch.float32, device="cuda")
         Gs.append(G)
@@ -48,18 +52,20 @@ def run_group(w, inp, tokens_per_rank, flags=0):
            "dw1": np.concatenate([to_numpy(G["dw1"]) for G in Gs]), "dw2": np.concatenate([to_numpy(G["dw2"]) for G in Gs]),
            "counts_all": to_numpy(group.ranks[0].counts_all)}
     for key in ep.SHARED_GRADS:
-        got[key] = sum(to_numpy(Gs[q][key]) for q in busy)
+        if key in Gs[0]:
+            got[key] = sum(to_numpy(Gs[q][key]) for q in busy)
     group.close()
     return got
 
 
 def compare(w, inp, got):
+    inp = oracle_inputs(w, inp)                     # Eq. 3 is Eq. 2 with identity projections for the oracle
     rt = oracle.route(inp, w.k)
     np.testing.assert_array_equal(got["counts_all"].sum(axis=0), rt.counts)
     ref = oracle.backward_full(inp, rt, w.act, decide_bf16=w.dtype == wl.DTYPE_BF16)
     ref["dw1"] = np.stack([ref["dw1"][e] for e in range(w.E)])
     ref["dw2"] = np.stack([ref["dw2"][e] for e in range(w.E)])
-    keys = ("y", "dx", "dw_gate", "dw1", "dw2", "db_gate", "dw_up", "dw_down")
+    keys = ("y", "dx", "dw_gate", "dw1", "dw2", "db_gate") + (() if w.cdac else ("dw_up", "dw_down"))
     assert_within(w, float_errors(w, {key: got[key] for key in keys}, ref))
     for e in range(w.E):
         if rt.counts[e] == 0:
@@ -91,6 +97,18 @@ def test_bf16_ranks_together_equal_one_layer(case, flags):
     w = wl.Workload("ep", T=sum(case["tokens"]), dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=73, **case["shape"])
     inp = skewed(w, case["strength"])
     compare(w, inp, run_group(w, inp, case["tokens"], flags))
+
+
+@pytest.mark.parametrize("case", [
+    dict(shape=dict(d=48, r=48, h=20, E=8, k=3), dtype=wl.DTYPE_F32, tokens=[150, 0, 200, 77]),
+    dict(shape=dict(d=128, r=128, h=64, E=8, k=2), dtype=wl.DTYPE_BF16, tokens=[900, 1100]),
+    dict(shape=dict(d=256, r=256, h=128, E=12, k=4), dtype=wl.DTYPE_BF16, tokens=[700, 500, 800]),
+])
+def test_conventional_layer_of_eq3_on_expert_parallel_ranks(case):
+    """BIGMAC_FLAG_CDAC under expert parallelism: the rows that travel are the tokens themselves at width d."""
+    w = wl.Workload("ep", T=sum(case["tokens"]), dtype=case["dtype"], act=wl.ACT_GELU_ERF, seed=163, cdac=True, **case["shape"])
+    inp = skewed(w, 1.5)
+    compare(w, inp, run_group(w, inp, case["tokens"]))
 
 
 def test_small_config_on_four_ranks():
