@@ -242,8 +242,9 @@ def run_cdac_twin(w, x, dy, dev, ms_step, ms_fwd, steps, peaks, esz):
 
     for _ in range(3):
         step()
-    binding.bigmac_profile_enable(layer.handle, True)
     ms = timed(step, steps)
+    binding.bigmac_profile_enable(layer.handle, True)       # a second pass with per-stage events, for the stage rates
+    timed(step, steps)
     prof = binding.bigmac_profile_read(layer.handle)
     binding.bigmac_profile_enable(layer.handle, False)
     fwd = lambda: layer.forward(x, tw, y=y, training=False)
@@ -400,16 +401,21 @@ def run_ep_on_one_gpu(w, x, dy, dev, ms_step, steps, esz, size=4):
 
     for _ in range(3):
         step()
-    for rk in group.ranks:
+
+    def timed_steps():
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(steps):
+            step()
+        stop.record()
+        torch.cuda.synchronize()
+        return start.elapsed_time(stop) / steps
+
+    ms = timed_steps()
+    for rk in group.ranks:                                   # a second pass with per-stage events, for the exchange kernels
         binding.bigmac_profile_enable(rk.handle, True)
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    start.record()
-    for _ in range(steps):
-        step()
-    stop.record()
-    torch.cuda.synchronize()
-    ms = start.elapsed_time(stop) / steps
+    timed_steps()
     moves = {}
     for rk in group.ranks:
         prof = binding.bigmac_profile_read(rk.handle)
@@ -519,16 +525,20 @@ def run_ours(args, w):
         step()
         torch.cuda.synchronize()
 
-    # ---- timed region: K steps, device-timed, max over ranks; per-stage events recorded inside it
-    binding.bigmac_profile_enable(layer.handle, True)
+    # ---- timed region: K steps as a caller runs them, device-timed, max over ranks
     t0 = time.time()
     ms_total = timed(step, args.steps)
     t1 = time.time()
-    prof = binding.bigmac_profile_read(layer.handle)
-    binding.bigmac_profile_enable(layer.handle, False)
     clocks = sampler.stop(t0, t1) if sampler else None
     ms_step = ms_total / args.steps
     value = whole_job_tokens_per_s(w.T, world, ms_step)
+    # ---- the same K steps again with a CUDA-event pair around every stage (what the roofline and the per-stage rates
+    # below come from).  The events cost time of their own (27 pairs per step), and while they are recorded the
+    # backward pass keeps all launches on one stream so that a stage's time is its own.
+    binding.bigmac_profile_enable(layer.handle, True)
+    ms_step_events = timed(step, args.steps) / args.steps
+    prof = binding.bigmac_profile_read(layer.handle)
+    binding.bigmac_profile_enable(layer.handle, False)
 
     # forward only (inference forward: nothing saved)
     def fwd_only():
@@ -696,6 +706,7 @@ def run_ours(args, w):
             "e2e": {"value": world * w.T / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": bytes_io,
                     "d2h_bytes_per_step": bytes_io, "ms_per_step": ms_e2e},
             "gpu_launches": prof["launches"],
+            "with_stage_events": {"ms_per_step": ms_step_events, "value": whole_job_tokens_per_s(w.T, world, ms_step_events), "unit": UNIT},
             "forward_only": {"tokens_per_s": world * w.T / (ms_fwd * 1e-3), "ms": ms_fwd,
                              "frac_of_tensor_roofline": round(fwd_fl / (ms_fwd * 1e-3) / 1e12 / peaks["tflops_sustained"], 4),
                              "cuda_graph_ms": ms_fwd_graph},

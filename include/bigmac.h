@@ -29,8 +29,12 @@
  *    chosen by (logit descending, expert id ascending); p is the softmax over the k chosen logits,
  *    so the p of one token sum to 1; there are no biases other than the optional gate bias.
  *  - The library never allocates device memory in route/forward/backward, never synchronises the
- *    stream (bigmac_device_status excepted) and launches everything on the stream passed in
- *    (a cudaStream_t as void*).  One handle serves one stream at a time.
+ *    stream (bigmac_device_status excepted) and orders everything after the work already on the stream
+ *    passed in (a cudaStream_t as void*) and before whatever the caller puts there next.  bigmac_backward
+ *    runs a few launches that do not depend on each other on a second stream owned by the handle, forked
+ *    from and joined back into the caller's stream with events (stream capture sees an ordinary fork and
+ *    join; BIGMAC_OVERLAP=0 in the environment keeps everything on the one stream).  One handle serves one
+ *    stream at a time.
  *  - Return value: BIGMAC_OK (0) or a negative bigmac_status_t.  On an argument error nothing is
  *    launched.  Nothing throws, aborts or traps; problems detected on the device (a bounded wait that
  *    ran out) are recorded in a status word read by bigmac_device_status.
@@ -159,7 +163,7 @@ typedef struct {
 } bigmac_routing_t;
 
 /* Validate the configuration and create a handle on the current CUDA device.  Allocates one small
- * device status word; no other device memory is owned by the handle.
+ * device status word (no other device memory is owned by the handle), one stream and six events.
  * Errors: INVALID_ARG (null pointers, non-positive sizes, k > E, unknown enums, a negative or non-finite
  * capacity_factor or aux_loss_coef), UNSUPPORTED (BF16
  * with d, r or h not a multiple of 64; E > 1024), CUDA. */

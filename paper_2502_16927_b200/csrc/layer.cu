@@ -298,6 +298,16 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
         delete L;
         return BIGMAC_ERR_UNSUPPORTED;
     }
+    // the backward pass's second stream and its fork / join events; without them the pass runs on one stream
+    bool side_ok = cudaStreamCreateWithFlags(&L->side, cudaStreamNonBlocking) == cudaSuccess;
+    for (cudaEvent_t& e : L->fork_join)
+        side_ok = side_ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+    if (!side_ok) {
+        for (cudaEvent_t& e : L->fork_join)
+            if (e) { cudaEventDestroy(e); e = nullptr; }
+        if (L->side) { cudaStreamDestroy(L->side); L->side = nullptr; }
+        cudaGetLastError();
+    }
     *out = L;
     return BIGMAC_OK;
 }
@@ -305,6 +315,9 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
 int bigmac_layer_destroy(bigmac_layer_t* L) {
     if (!L) return BIGMAC_ERR_INVALID_ARG;
     for (cudaEvent_t e : L->ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : L->fork_join)
+        if (e) cudaEventDestroy(e);
+    if (L->side) cudaStreamDestroy(L->side);
     cudaFree(L->status);
     delete L;
     return BIGMAC_OK;
@@ -468,6 +481,18 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     const bigmac_config_t& c = L->cfg;
     const bool acc = accumulate != 0;
 
+    // Overlap (BIGMAC_OVERLAP=0 turns it off): dW_up, the bias-gradient column sums and the dx' gather go to a second
+    // stream, forked from and joined back into the caller's stream with events, so that they run beside launches they
+    // do not depend on.  Everything that shares the fp32 workspace stays ordered.
+    static const bool overlap_on = []() { const char* e = std::getenv("BIGMAC_OVERLAP"); return !(e && e[0] == '0'); }();
+    // (not while per-stage events are recorded: a stage timed beside another stream's launches would not be its own time)
+    const bool overlap = overlap_on && L->side && !L->prof_on && !m.cdac && !m.gate_low;
+    cudaStream_t sd = st;
+    if (overlap) {
+        sd = L->side;
+        BIGMAC_CUDA(cudaEventRecord(L->fork_join[0], st));
+        BIGMAC_CUDA(cudaStreamWaitEvent(sd, L->fork_join[0], 0));
+    }
     if (m.cdac) b.dy_lo = const_cast<void*>(dy);
     if (!m.cdac) {   // dy' = dy W_up                                   [T,d] x [d,r]
         GemmArgs g;
@@ -483,13 +508,14 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.C = G->dw_up; g.ldc = m.r; g.M = m.d; g.N = m.r; g.K = m.T; g.accumulate = acc;
         if (fused) {   // contraction over all tokens, few output tiles: split it, reduce the parts in order
             g.split_k = choose_split_k(g.M, g.N, g.K); g.C = b.splitk_ws; g.out_f32 = true; g.accumulate = false;
-            BIGMAC_TRY(gemm(L, G_DW_UP, g, st));
-            Stage s(L, S_SPLITK_REDUCE, st);
-            BIGMAC_CUDA(launch_splitk_reduce(b.splitk_ws, g.split_k, m.d, m.r, G->dw_up, m.d, nullptr, 0, m.dtype, acc, st));
+            BIGMAC_TRY(gemm(L, G_DW_UP, g, sd));
+            Stage s(L, S_SPLITK_REDUCE, sd);
+            BIGMAC_CUDA(launch_splitk_reduce(b.splitk_ws, g.split_k, m.d, m.r, G->dw_up, m.d, nullptr, 0, m.dtype, acc, sd));
         } else {
-            BIGMAC_TRY(gemm(L, G_DW_UP, g, st));
+            BIGMAC_TRY(gemm(L, G_DW_UP, g, sd));
         }
     }
+    if (overlap) BIGMAC_CUDA(cudaEventRecord(L->fork_join[1], sd));          // dW_up done: the fp32 workspace is free again
     // du = p dy'[t], dp = <dy'[t], u>; then the softmax-over-k backward
     if (m.cap != kNoCapacity) BIGMAC_CUDA(cudaMemsetAsync(b.dp, 0, sizeof(float) * m.N, st));   // dropped slots: dp = 0
     { Stage s(L, S_COMBINE_BWD, st); BIGMAC_CUDA(launch_combine_bwd(b.dy_lo, b.u, b.du, b.dp, b.tb, m.k, m.r, m.dtype, m.P, st)); }
@@ -503,6 +529,14 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         Stage s(L, S_GATE_BWD, st);
         BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, ldcat, m.k, m.dtype, st));
     }
+    bool colsum_done = false;
+    if (overlap && G->db_gate) {   // the gate-bias gradient needs only the per-slot dl: beside the expert contractions
+        BIGMAC_CUDA(cudaEventRecord(L->fork_join[2], st));
+        BIGMAC_CUDA(cudaStreamWaitEvent(sd, L->fork_join[2], 0));
+        { Stage s(L, S_COLSUM, sd, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, sd, aux_part)); }
+        BIGMAC_CUDA(cudaEventRecord(L->fork_join[3], sd));
+        colsum_done = true;
+    }
     {   // dz = (du W2_e) * sigma'(z); the forward saved sigma'(z) in the z buffer, dz is written over it
         GemmArgs g;
         g.A = b.du; g.lda = m.r; g.B = W->w2; g.ldb = m.h; g.b_kmajor = false; g.b_stride = (int64_t)m.r * m.h;
@@ -512,6 +546,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         BIGMAC_TRY(gemm(L, G_DZ, g, st));
     }
     void* dz = b.dz ? b.dz : b.z;
+    if (overlap) BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[1], 0));    // from here on the fp32 workspace is used again
     if (m.bias) {   // db1_e = sum_rows dz[row,:], db2_e = sum_rows du[row,:]  (padding rows hold zeros)
         if (!aligned(G->db1, 4) || !aligned(G->db2, 4)) return BIGMAC_ERR_INVALID_ARG;
         Stage s(L, S_COLSUM, st, 2 * ((G->db1 ? 1 : 0) + (G->db2 ? 1 : 0)));
@@ -532,6 +567,12 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         g.C = b.dxg; g.ldc = m.r; g.M = (int)m.P; g.N = m.r; g.K = m.h;
         g.group = GROUP_M; g.num_experts = m.E; g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
         BIGMAC_TRY(gemm(L, G_DXG, g, st));
+    }
+    if (overlap) {   // dx'[t] = sum_j dxg[row of slot (t,j)]: an HBM-bound gather beside the tensor-bound dW1
+        BIGMAC_CUDA(cudaEventRecord(L->fork_join[4], st));
+        BIGMAC_CUDA(cudaStreamWaitEvent(sd, L->fork_join[4], 0));
+        { Stage s(L, S_DXLO_GATHER, sd); BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, sd, ldcat, m.cap != kNoCapacity)); }
+        BIGMAC_CUDA(cudaEventRecord(L->fork_join[5], sd));
     }
     if (G->dw1) {   // dW1_e[q,c'] = sum_rows dz[row,q] xg[row,c']
         GemmArgs g;
@@ -567,7 +608,12 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         return BIGMAC_OK;
     }
     // dx'[t] = sum_j dxg[row of slot (t,j)]   (the transpose of the dispatch gather)
-    { Stage s(L, S_DXLO_GATHER, st); BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st, ldcat, m.cap != kNoCapacity)); }
+    if (overlap) {
+        BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[5], 0));
+    } else {
+        Stage s(L, S_DXLO_GATHER, st);
+        BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st, ldcat, m.cap != kNoCapacity));
+    }
     if (m.gate_low) {
         // The gate read x': its gradient joins dx' (dx' += dl W_gate, W_gate [E,r]) before the descend projection;
         // dW_gate = dl^T x'.
@@ -658,7 +704,12 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
             BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
         }
     }
-    if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st, aux_part)); }
+    if (colsum_done) {
+        BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[3], 0));              // join
+    } else if (G->db_gate) {
+        Stage s(L, S_COLSUM, st, 2);
+        BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st, aux_part));
+    }
     return BIGMAC_OK;
 }
 

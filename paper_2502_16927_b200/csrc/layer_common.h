@@ -15,6 +15,10 @@ struct bigmac_layer {
                         // status[2..3] the work counters of the per-expert weight-gradient kernel (zero at rest)
     bool use_tc;        // bf16 contractions on tcgen05
     unsigned tc_mask;   // debug: bit i set = contraction i runs on tcgen05 (BIGMAC_TC_MASK)
+    // second stream of the backward pass (created on first use): launches that do not depend on each other and lean
+    // on different units (a tensor-bound weight gradient beside an HBM-bound row move) run side by side
+    cudaStream_t side = nullptr;
+    cudaEvent_t fork_join[6] = {};
     // measurement aid
     bool prof_on = false;
     uint64_t launches = 0;

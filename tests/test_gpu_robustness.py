@@ -181,3 +181,67 @@ def test_expert_parallel_exchange_stays_inside_the_exchange_buffers():
     assert int(counts[:2].sum()) == w.T * w.k               # all rows went to rank 0's first two experts
     assert bool(torch.isfinite(torch.cat(ys).float()).all())
     group.close()
+
+
+def test_backward_on_two_streams_equals_backward_on_one_and_can_be_captured():
+    """bigmac_backward forks a few independent launches to the handle's second stream and joins them back: the
+    results are bit for bit those of the one-stream order (run in a child process with BIGMAC_OVERLAP=0), and a
+    captured forward + backward replays to the same bits."""
+    import os
+    import subprocess
+    import sys
+    import tempfile
+
+    import numpy as np
+    import torch
+
+    w = wl.Workload("ov", T=3000, d=256, r=128, h=256, E=16, k=4, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=167)
+    inp = conditioned(w)
+    dev = to_device(w, inp)
+    layer = make_layer(w)
+    y = layer.forward(dev["x"], dev, training=True)
+    G = empty_grads(w, "cuda", fill=float("nan"))
+    dx = layer.backward(dev["x"], dev["dy"], dev, G)
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    eager = {key: val.clone() for key, val in dict(G, y=y, dx=dx).items()}
+
+    # the same step captured into a CUDA graph and replayed
+    side = torch.cuda.Stream()
+    G2 = empty_grads(w, "cuda", fill=float("nan"))
+    y2, dx2 = torch.empty_like(y), torch.empty_like(dx)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        layer.forward(dev["x"], dev, y=y2, training=True)             # warm-up on the capture stream
+        layer.backward(dev["x"], dev["dy"], dev, G2, dx=dx2)
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            layer.forward(dev["x"], dev, y=y2, training=True)
+            layer.backward(dev["x"], dev["dy"], dev, G2, dx=dx2)
+    for t in list(G2.values()) + [y2, dx2]:
+        t.fill_(float("nan")) if t.is_floating_point() else None
+    graph.replay()
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    for key, val in dict(G2, y=y2, dx=dx2).items():
+        assert torch.equal(val.view(torch.uint8), eager[key].view(torch.uint8)), key
+    layer.close()
+
+    # one-stream order in a child process: the environment switch is read once per process
+    with tempfile.TemporaryDirectory() as tmp:
+        out = os.path.join(tmp, "one_stream.pt")
+        code = (
+            "import sys, torch; sys.path.insert(0, %r); sys.path.insert(0, %r)\n"
+            "from paper_2502_16927_b200 import workloads as wl\n"
+            "from helpers import empty_grads, make_layer, to_device\n"
+            "from test_gpu_parity import conditioned\n"
+            "w = wl.Workload('ov', T=3000, d=256, r=128, h=256, E=16, k=4, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=167)\n"
+            "inp = conditioned(w); dev = to_device(w, inp); layer = make_layer(w)\n"
+            "y = layer.forward(dev['x'], dev, training=True); G = empty_grads(w, 'cuda', fill=float('nan'))\n"
+            "dx = layer.backward(dev['x'], dev['dy'], dev, G); torch.cuda.synchronize(); assert layer.status() == 0\n"
+            "torch.save({k: v.cpu() for k, v in dict(G, y=y, dx=dx).items()}, %r)\n"
+        ) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)), out)
+        subprocess.run([sys.executable, "-c", code], check=True, env=dict(os.environ, BIGMAC_OVERLAP="0"), timeout=600)
+        one = torch.load(out)
+    for key, val in eager.items():
+        assert torch.equal(val.cpu().view(torch.uint8), one[key].view(torch.uint8)), key
