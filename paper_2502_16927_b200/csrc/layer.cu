@@ -519,21 +519,28 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     // du = p dy'[t], dp = <dy'[t], u>; then the softmax-over-k backward
     if (m.cap != kNoCapacity) BIGMAC_CUDA(cudaMemsetAsync(b.dp, 0, sizeof(float) * m.N, st));   // dropped slots: dp = 0
     { Stage s(L, S_COMBINE_BWD, st); BIGMAC_CUDA(launch_combine_bwd(b.dy_lo, b.u, b.du, b.dp, b.tb, m.k, m.r, m.dtype, m.P, st)); }
+    // The gate backward (dp -> dl) and the gate-bias column sums feed only dx, dW_gate and db_gate at the end of the pass:
+    // with the second stream they run beside the expert contractions instead of in front of them.
+    if (overlap) {
+        BIGMAC_CUDA(cudaEventRecord(L->fork_join[2], st));
+        BIGMAC_CUDA(cudaStreamWaitEvent(sd, L->fork_join[2], 0));
+    }
     float* aux_part = nullptr;                                                    // column sums of dL_aux/dl, for db_gate
     if (m.aux > 0) {
         aux_part = b.colsum_part + (size_t)kColsumChunks * m.E;
-        Stage s(L, S_GATE_BWD, st);
+        Stage s(L, S_GATE_BWD, sd);
         BIGMAC_CUDA(launch_gate_bwd_aux(b.dp, b.tb, b.dlogits, b.logits_saved, W->b_gate, m.aux, aux_part, m.T, m.E, m.E64,
-                                        ldcat, m.k, m.dtype, st));
+                                        ldcat, m.k, m.dtype, sd));
     } else {
-        Stage s(L, S_GATE_BWD, st);
-        BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, ldcat, m.k, m.dtype, st));
+        Stage s(L, S_GATE_BWD, sd);
+        BIGMAC_CUDA(launch_gate_bwd(b.dp, b.tb, b.dlogits, m.T, m.E, m.E64, ldcat, m.k, m.dtype, sd));
     }
     bool colsum_done = false;
-    if (overlap && G->db_gate) {   // the gate-bias gradient needs only the per-slot dl: beside the expert contractions
-        BIGMAC_CUDA(cudaEventRecord(L->fork_join[2], st));
-        BIGMAC_CUDA(cudaStreamWaitEvent(sd, L->fork_join[2], 0));
-        { Stage s(L, S_COLSUM, sd, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, sd, aux_part)); }
+    if (overlap) {
+        if (G->db_gate) {
+            Stage s(L, S_COLSUM, sd, 2);
+            BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, sd, aux_part));
+        }
         BIGMAC_CUDA(cudaEventRecord(L->fork_join[3], sd));
         colsum_done = true;
     }
@@ -609,7 +616,8 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     }
     // dx'[t] = sum_j dxg[row of slot (t,j)]   (the transpose of the dispatch gather)
     if (overlap) {
-        BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[5], 0));
+        BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[5], 0));             // join: the gather ...
+        BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[3], 0));             // ... and the gate backward with its column sums
     } else {
         Stage s(L, S_DXLO_GATHER, st);
         BIGMAC_CUDA(launch_combine(b.dxg, b.dx_lo, nullptr, b.tb.prow_of_slot, m.T, m.k, m.r, m.dtype, st, ldcat, m.cap != kNoCapacity));
@@ -704,9 +712,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
             BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
         }
     }
-    if (colsum_done) {
-        BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[3], 0));              // join
-    } else if (G->db_gate) {
+    if (!colsum_done && G->db_gate) {
         Stage s(L, S_COLSUM, st, 2);
         BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st, aux_part));
     }
