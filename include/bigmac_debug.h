@@ -10,8 +10,9 @@
  *   epilogue 0: none; 1: Z = sigma'(acc) (if Z), C = sigma(acc); 2: C = acc * Z.  On the tensor-core kernels Z holds
  *   sigma' as one byte per element, q = round(200 sigma' + 27); on the plain FMA kernel Z has the layer's dtype.
  * All pointers are device memory (tables included), 16-byte aligned.  use_tensor_cores: 0 = plain FMA kernel,
- * 1 = tensor cores (default kernel choice), 2 = force the one-CTA kernel, 3 = force the CTA-pair kernel; non-zero
- * values require a BF16 handle.  Returns a bigmac_status_t.
+ * 1 = tensor cores (default kernel choice), 2 = force the one-CTA kernel, 3 / 4 / 5 = force the CTA-pair kernel with
+ * four / two / one working epilogue warps per lane quadrant (plain epilogues only; the default choice is two);
+ * non-zero values require a BF16 handle.  Returns a bigmac_status_t.
  */
 #ifndef BIGMAC_DEBUG_H_
 #define BIGMAC_DEBUG_H_

@@ -223,7 +223,8 @@ def bigmac_profile_read(handle) -> Dict[str, object]:
 
 
 def bigmac_debug_gemm(handle, q: bigmac_debug_gemm_t, use_tensor_cores) -> None:
-    """use_tensor_cores: False/0 plain FMA, True/1 tensor cores, 2 one-CTA kernel, 3 CTA-pair kernel."""
+    """use_tensor_cores: False/0 plain FMA, True/1 tensor cores, 2 one-CTA kernel, 3/4/5 CTA-pair kernel with 4/2/1 working
+    epilogue warps per lane quadrant."""
     _check(lib().bigmac_debug_gemm(handle, C.byref(q), int(use_tensor_cores), _stream()), "bigmac_debug_gemm")
 
 

@@ -11,6 +11,8 @@
 // CTAs.  Accumulators are double-buffered: "tmem_full" is signalled in both CTAs by a multicast commit, and the
 // epilogue warps of both CTAs arrive on the leader's "tmem_empty" when they have read their half.
 // No TMA multicast is used.  Everything else (epilogues, grouping, split contraction) is as in gemm_tc.cu.
+#include <cstdlib>
+
 #include "tc_pair.cuh"
 
 namespace bigmac {
@@ -274,6 +276,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         walk_init(tw, cluster_id, tiles_n);
         PairTile nxt = tw.w < total ? walk_tile(p, BN, tw, pairs_m, tiles_n, s_pp) : PairTile{};
         if (z_prefetch && tw.w < total) issue_z(nxt);
+        // Plain epilogues have time to spare: two of the four warps of a lane quadrant do all its columns and the other
+        // two stay out of the MMA thread's way (expert GEMM2 / dxg -3 %, ascend -6 %, a plain K = 512 grouped GEMM -9 %;
+        // with one warp per quadrant the short-K launches become epilogue-bound, with an activation two are too few).
+        const int part_step = p.epilogue == EPI_NONE ? p.epi_parts : 4;
+        if (part < part_step)
         for (; tw.w < total; ++local) {
             const PairTile tl = nxt;
             const int w = tw.w;
@@ -287,7 +294,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             const bool half_ok = (int)rank < tl.halves;
             const bool row_ok = half_ok && row < tl.m_limit;
             const int64_t row_off = tl.c_base + (int64_t)row * p.ldc;
-            const uint32_t t_addr = tmem_base + acc * BN + ((uint32_t)(quad * 32) << 16) + (uint32_t)(part * COLS_PER_WARP);
+            for (int pp = part; pp < 4; pp += part_step) {
+            const uint32_t t_addr = tmem_base + acc * BN + ((uint32_t)(quad * 32) << 16) + (uint32_t)(pp * COLS_PER_WARP);
 #pragma unroll 1
             for (int c = 0; c < CHUNKS; ++c) {
                 float v[32];
@@ -303,7 +311,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(leader_tmem_empty[acc]);
                 }
-                const int col0 = tl.n0 + part * COLS_PER_WARP + c * 32;
+                const int col0 = tl.n0 + pp * COLS_PER_WARP + c * 32;
                 if (col0 >= p.N) continue;             // uniform across the warp
                 if (p.bias) add_bias32(v, p.bias + (int64_t)tl.expert * p.bias_stride + col0);   // N is a multiple of 32 here
                 if (TMA_EPI) {
@@ -342,6 +350,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         store_row_chunk(p, v, row_off, col0, vec_ok);
                     }
                 }
+            }
             }
         }
         if (TMA_EPI && lane == 0) tma_store_wait_all();
@@ -423,6 +432,7 @@ cudaError_t dispatch_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
     p.C = g.C; p.Z = g.Z; p.ldc = g.ldc; p.c_stride = g.c_stride; p.M = g.M; p.N = g.N; p.K = g.K;
     p.out_f32 = g.out_f32; p.accumulate = g.accumulate; p.epilogue = g.epilogue; p.act = g.act; p.group = g.group;
     p.num_experts = E; p.tile_expert = g.tile_expert; p.n_tiles = g.n_tiles; p.poffsets = g.poffsets; p.status = status;
+    p.epi_parts = epi_parts_default(g.epi_parts);
     p.bias = g.group == GROUP_M ? g.bias : nullptr; p.bias_stride = g.bias_stride;
     if (p.bias && (g.N % 32 || ((uintptr_t)g.bias % 16) || g.bias_stride % 4)) return cudaErrorInvalidValue;
     // upper bound on work items (the kernel derives the exact count on the device for grouped rows)

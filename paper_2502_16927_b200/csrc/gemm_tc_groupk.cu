@@ -239,6 +239,9 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         const int part = (warp - 2) >> 2;
         const bool vec_ok = (p.ldc % 16 == 0) && ((p.c_stride * 2) % 32 == 0) && (((uintptr_t)p.C) % 32 == 0);
         const uint32_t leader_tmem_empty[2] = {map_to_cta(&tmem_empty_bar[0], 0), map_to_cta(&tmem_empty_bar[1], 0)};
+        // as in the pair kernel: p.epi_parts of the four warps of a lane quadrant do all its columns, the others leave
+        const int part_step = p.epi_parts;
+        if (part < part_step)
         for (uint32_t local = 0;; ++local) {
             const uint32_t acc = local & 1;
             mbar_wait_cluster(&ring_bar[local % kRing], (local / kRing) & 1, dead, p.status);
@@ -250,7 +253,8 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             const bool row_ok = row < p.M;
             // whole contraction: the expert's gradient; one part of it: the part's fp32 slot in the workspace
             const int64_t row_off = (t.slot >= 0 ? (int64_t)t.slot * p.M * p.ldc : (int64_t)t.expert * p.c_stride) + (int64_t)row * p.ldc;
-            const uint32_t t_addr = tmem_base + acc * BN + ((uint32_t)(quad * 32) << 16) + (uint32_t)(part * COLS_PER_WARP);
+            for (int pp = part; pp < 4; pp += part_step) {
+            const uint32_t t_addr = tmem_base + acc * BN + ((uint32_t)(quad * 32) << 16) + (uint32_t)(pp * COLS_PER_WARP);
 #pragma unroll 1
             for (int c = 0; c < CHUNKS; ++c) {
                 float v[32];
@@ -261,7 +265,7 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(leader_tmem_empty[acc]);
                 }
-                const int col0 = t.n0 + part * COLS_PER_WARP + c * 32;
+                const int col0 = t.n0 + pp * COLS_PER_WARP + c * 32;
                 if (col0 < p.N && row_ok) {
                     if (t.slot >= 0) {
                         TcParams p2 = p;
@@ -271,6 +275,7 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                         store_row_chunk(p, v, row_off, col0, vec_ok);
                     }
                 }
+            }
             }
         }
     }
@@ -338,7 +343,7 @@ cudaError_t gemm_tc_groupk(const GemmArgs& g, int* status, int* sched, void* ws,
     TcParams p{};
     p.C = g.C; p.ldc = g.ldc; p.c_stride = g.c_stride; p.M = g.M; p.N = g.N; p.K = g.K;
     p.accumulate = g.accumulate; p.epilogue = EPI_NONE; p.group = GROUP_K; p.num_experts = E; p.poffsets = g.poffsets;
-    p.status = status; p.split_k = 1; p.b2_first_kb = -1; p.n_split = -1;
+    p.status = status; p.split_k = 1; p.b2_first_kb = -1; p.n_split = -1; p.epi_parts = epi_parts_default(g.epi_parts);
     float* slots = (float*)ws;
     int32_t* plan = (int32_t*)((char*)ws + (((size_t)kGroupKSlots * g.M * g.N * sizeof(float) + 255) & ~(size_t)255));
     constexpr size_t kMaxSmem = 232448;

@@ -58,6 +58,7 @@ struct GemmArgs {
     int N2 = 0;
     int split_k = 1;                    // > 1: part s of the contraction writes its partial result (fp32) to C + s*M*ldc
     int force_kernel = 0;               // measurement aid: 1 = one-CTA kernel, 2 = CTA-pair kernel, 0 = default choice
+    int epi_parts = 0;                  // measurement aid: epilogue warps per lane quadrant that work (1, 2 or 4); 0 = default choice
     // GROUP_M only: fp32 bias added to the accumulator before the epilogue, column n of a row of expert e gets
     // bias[e*bias_stride + n] (16-byte aligned, bias_stride a multiple of 4)
     const float* bias = nullptr;

@@ -891,7 +891,8 @@ int bigmac_debug_gemm(bigmac_layer_t* L, const bigmac_debug_gemm_t* q, int use_t
     g.group = q->group; g.num_experts = q->num_experts; g.b_stride = q->b_stride; g.c_stride = q->c_stride;
     g.tile_expert = q->tile_expert; g.n_tiles = q->n_tiles; g.poffsets = q->poffsets;
     L->launches += 1;
-    g.force_kernel = use_tensor_cores == 2 ? 1 : use_tensor_cores == 3 ? 2 : 0;
+    g.force_kernel = use_tensor_cores == 2 ? 1 : use_tensor_cores >= 3 ? 2 : 0;
+    g.epi_parts = use_tensor_cores == 4 ? 2 : use_tensor_cores == 5 ? 1 : use_tensor_cores == 3 ? 4 : 0;
     cudaError_t err = use_tensor_cores ? gemm_tc(g, L->status, (cudaStream_t)stream)
                                        : gemm_simt(g, L->cfg.dtype, (cudaStream_t)stream);
     return err == cudaSuccess ? BIGMAC_OK : BIGMAC_ERR_CUDA;

@@ -3,6 +3,8 @@
 #pragma once
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "internal.h"
 #include "act.cuh"
 
@@ -212,6 +214,7 @@ struct TcParams {
     int c_rows_per_expert;       // rows of the C tensor map per expert (GROUP_K); 0 otherwise
     int split_k;                 // dense only: the contraction is cut into split_k parts, part s writes C + s*M*ldc
     int b2_first_kb;             // k slices from this one on come from the second B tensor (map_b2); <0: none
+    int epi_parts;               // plain epilogues: this many (1, 2 or 4) of the four epilogue warps of a lane quadrant work
     const float* bias;           // GROUP_M: fp32 bias of expert e at bias + e*bias_stride, added before the epilogue; or null
     int64_t bias_stride;
     int n_split;                 // output columns from this one on come from map_b2 (K-major) and go to C2 (fp32); <0: none
@@ -577,6 +580,13 @@ constexpr int kThreadsV2 = (2 + kEpiWarps) * 32;
 
 
 // ------------------------------------------------------------------------------------------ host side
+// Working epilogue warps per lane quadrant for plain epilogues: the request, else BIGMAC_EPI_PARTS, else 2.
+inline int epi_parts_default(int requested) {
+    static const int env = []() { const char* e = std::getenv("BIGMAC_EPI_PARTS"); return e ? atoi(e) : 0; }();
+    const int v = requested ? requested : env ? env : 2;
+    return (v == 1 || v == 2) ? v : 4;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);

@@ -75,6 +75,24 @@ def test_dense_kmajor_kmajor(M, N, K):
     _close(_np(C), A.astype(np.float64) @ B.astype(np.float64).T)
 
 
+@pytest.mark.parametrize("M,N,K", [(1000, 1024, 192), (777, 320, 512), (300, 2048, 64)])
+def test_pair_kernel_gives_the_same_bits_with_four_two_or_one_working_epilogue_warps(M, N, K):
+    """Plain epilogues let two of the four epilogue warps of a lane quadrant do all its columns (the default) so that
+    fewer warps compete with the MMA-issuing thread; who drains a column does not change its value."""
+    import torch
+    A, B = _rand((M, K), 5), _rand((N, K), 6, K ** -0.5)
+    dA, dB = _dev_bf16(A), _dev_bf16(B)
+    layer = _layer()
+    outs = []
+    for mode in (3, 4, 5, 1):                      # 4, 2, 1 working warps per quadrant, then the default choice
+        C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        _run(layer, _q(A=dA, B=dB, C=C, lda=K, ldb=K, ldc=N, M=M, N=N, K=K, a_kmajor=1, b_kmajor=1), mode)
+        outs.append(C)
+    _close(_np(outs[0]), A.astype(np.float64) @ B.astype(np.float64).T)
+    for other in outs[1:]:
+        assert torch.equal(outs[0].view(torch.int16), other.view(torch.int16))
+
+
 def test_gelu_epilogue_error_bound_over_a_sweep_of_z():
     """z = A I through the expert-GEMM1 epilogue for z across [-6, 6]: sigma(z) within one bf16 rounding plus the
     stated absolute bound of the Phi polynomial, sigma'(z) within half a quantisation step."""
