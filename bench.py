@@ -525,20 +525,43 @@ def run_ours(args, w):
         step()
         torch.cuda.synchronize()
 
-    # ---- timed region: K steps as a caller runs them, device-timed, max over ranks
+    # ---- timed region: K steps as a caller runs them, device-timed, max over ranks; and the same K steps with a
+    # CUDA-event pair around every stage (what the roofline and the per-stage rates below come from).  The events cost
+    # time of their own (27 pairs per step), and while they are recorded the backward pass keeps all launches on one
+    # stream so that a stage's time is its own.  Under the power cap the clocks drift over the first seconds of load, so
+    # the two kinds of steps alternate in halves (K/2 plain, K/2 with events, the rest plain, the rest with events) and
+    # see the same clocks; each half is bracketed by barrier + synchronize like a whole region.
+    halves = [args.steps // 2, args.steps - args.steps // 2]
+    ms_total = ms_events_total = 0.0
+    prof = {"launches": 0, "dropped": 0, "stages": {}}
     t0 = time.time()
-    ms_total = timed(step, args.steps)
+    def plain_half(n):
+        nonlocal ms_total
+        ms_total += timed(step, n)
+
+    def events_half(n):
+        nonlocal ms_events_total
+        binding.bigmac_profile_enable(layer.handle, True)
+        ms_events_total += timed(step, n)
+        part = binding.bigmac_profile_read(layer.handle)
+        binding.bigmac_profile_enable(layer.handle, False)
+        prof["launches"] += part["launches"]
+        prof["dropped"] += part["dropped"]
+        for name, (ms, calls) in part["stages"].items():
+            old_ms, old_calls = prof["stages"].get(name, (0.0, 0))
+            prof["stages"][name] = (old_ms + ms, old_calls + calls)
+
+    # plain, events, events, plain: whichever kind follows a pause (reading the events back) meets a rested GPU
+    for i, n in enumerate(halves):
+        if n == 0:
+            continue
+        for half in ((plain_half, events_half) if i == 0 else (events_half, plain_half)):
+            half(n)
     t1 = time.time()
     clocks = sampler.stop(t0, t1) if sampler else None
     ms_step = ms_total / args.steps
+    ms_step_events = ms_events_total / args.steps
     value = whole_job_tokens_per_s(w.T, world, ms_step)
-    # ---- the same K steps again with a CUDA-event pair around every stage (what the roofline and the per-stage rates
-    # below come from).  The events cost time of their own (27 pairs per step), and while they are recorded the
-    # backward pass keeps all launches on one stream so that a stage's time is its own.
-    binding.bigmac_profile_enable(layer.handle, True)
-    ms_step_events = timed(step, args.steps) / args.steps
-    prof = binding.bigmac_profile_read(layer.handle)
-    binding.bigmac_profile_enable(layer.handle, False)
 
     # forward only (inference forward: nothing saved)
     def fwd_only():
