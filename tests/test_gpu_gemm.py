@@ -75,10 +75,11 @@ def test_dense_kmajor_kmajor(M, N, K):
     _close(_np(C), A.astype(np.float64) @ B.astype(np.float64).T)
 
 
-@pytest.mark.parametrize("M,N,K", [(1000, 1024, 192), (777, 320, 512), (300, 2048, 64)])
+@pytest.mark.parametrize("M,N,K", [(1000, 1024, 192), (777, 320, 512), (300, 2048, 64), (500, 384, 256), (260, 400, 128)])
 def test_pair_kernel_gives_the_same_bits_with_four_two_or_one_working_epilogue_warps(M, N, K):
     """Plain epilogues let two of the four epilogue warps of a lane quadrant do all its columns (the default) so that
-    fewer warps compete with the MMA-issuing thread; who drains a column does not change its value."""
+    fewer warps compete with the MMA-issuing thread; who drains a column does not change its value.  N = 320, 384 and
+    400 end in a partly filled column tile."""
     import torch
     A, B = _rand((M, K), 5), _rand((N, K), 6, K ** -0.5)
     dA, dB = _dev_bf16(A), _dev_bf16(B)
