@@ -715,7 +715,7 @@ def run_ours(args, w):
                 "frac": round(achieved / peaks["tflops_sustained"], 4),
                 # DRAM bytes of those launches per step from a one-pass ncu capture of this workload
                 # (profiles/gemm_dram_traffic_large.md); not captured for the other workloads
-                "traffic": 12.757e9 if (w.name == "large" and w.T == 32768) else None,
+                "traffic": 12.791e9 if (w.name == "large" and w.T == 32768) else None,
                 "peak_source": f"{peaks['source']}: sustained bf16 (kernels timed inside a long step)",
                 "frac_of_burst_peak": round(achieved / peaks["tflops_burst"], 4),
                 "step_frac": round(3.0 * fwd_fl / (ms_step * 1e-3) / 1e12 / peaks["tflops_sustained"], 4)}
