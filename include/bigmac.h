@@ -163,7 +163,7 @@ typedef struct {
 } bigmac_routing_t;
 
 /* Validate the configuration and create a handle on the current CUDA device.  Allocates one small
- * device status word (no other device memory is owned by the handle), one stream and six events.
+ * device status word (no other device memory is owned by the handle), one stream and eight events.
  * Errors: INVALID_ARG (null pointers, non-positive sizes, k > E, unknown enums, a negative or non-finite
  * capacity_factor or aux_loss_coef), UNSUPPORTED (BF16
  * with d, r or h not a multiple of 64; E > 1024), CUDA. */

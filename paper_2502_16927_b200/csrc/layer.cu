@@ -481,8 +481,8 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     const bigmac_config_t& c = L->cfg;
     const bool acc = accumulate != 0;
 
-    // Overlap (BIGMAC_OVERLAP=0 turns it off): dW_up, the bias-gradient column sums and the dx' gather go to a second
-    // stream, forked from and joined back into the caller's stream with events, so that they run beside launches they
+    // Overlap (BIGMAC_OVERLAP=0 turns it off): dW_up, the gate backward with the bias-gradient column sums, the dx' gather
+    // and [dW_down ; dW_gate] go to a second stream, forked from and joined back into the caller's stream with events, so that they run beside launches they
     // do not depend on.  Everything that shares the fp32 workspace stays ordered.
     static const bool overlap_on = []() { const char* e = std::getenv("BIGMAC_OVERLAP"); return !(e && e[0] == '0'); }();
     // (not while per-stage events are recorded: a stage timed beside another stream's launches would not be its own time)
@@ -669,6 +669,14 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         return BIGMAC_OK;
     }
     if (fused) {
+        // dx and [dW_down ; dW_gate] share only their input [dx' | dl]: with the second stream the weight gradient's CTAs
+        // move in as those of dx leave.  The caller's stream has finished dW1 here, so the fp32 workspace is free.
+        cudaStream_t sw = st;
+        if (overlap && (G->dw_down || G->dw_gate)) {
+            BIGMAC_CUDA(cudaEventRecord(L->fork_join[6], st));
+            BIGMAC_CUDA(cudaStreamWaitEvent(sd, L->fork_join[6], 0));
+            sw = sd;
+        }
         {   // dx = [dx' | dl] [W_down ; W_gate]: one contraction over r + E
             GemmArgs g;
             g.A = b.dcat; g.lda = ldcat; g.B = W->w_down; g.ldb = m.d; g.b_kmajor = false;
@@ -681,10 +689,14 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
             g.A = b.dcat; g.lda = ldcat; g.a_kmajor = false; g.B = x; g.ldb = m.d; g.b_kmajor = false;
             g.C = b.splitk_ws; g.ldc = m.d; g.out_f32 = true; g.M = ldcat; g.N = m.d; g.K = m.T;
             g.split_k = choose_split_k(g.M, g.N, g.K);
-            BIGMAC_TRY(gemm(L, G_DW_DOWN, g, st));
-            Stage s(L, S_SPLITK_REDUCE, st);
+            BIGMAC_TRY(gemm(L, G_DW_DOWN, g, sw));
+            Stage s(L, S_SPLITK_REDUCE, sw);
             BIGMAC_CUDA(launch_splitk_reduce(b.splitk_ws, g.split_k, ldcat, m.d, G->dw_down, m.r, G->dw_gate, m.E, m.dtype,
-                                             acc, st));
+                                             acc, sw));
+        }
+        if (sw != st) {
+            BIGMAC_CUDA(cudaEventRecord(L->fork_join[7], sd));
+            BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[7], 0));
         }
     } else {
         {   // dx = dx' W_down
