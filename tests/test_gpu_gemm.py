@@ -64,7 +64,9 @@ def _run(layer, q, tc=True):
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 128, 64), (300, 192, 256), (1000, 64, 4096), (77, 320, 128), (333, 1024, 192),
-                                   (20000, 2048, 64)])
+                                   (20000, 2048, 64),
+                                   # long contractions at least 512 wide
+                                   (700, 512, 2048), (1300, 640, 2112), (520, 896, 4096), (300, 1100, 2048)])
 def test_dense_kmajor_kmajor(M, N, K):
     import torch
     A, B = _rand((M, K), 1), _rand((N, K), 2, K ** -0.5)
@@ -131,7 +133,7 @@ def test_dense_fp32_output_with_narrow_n(N):
     _close(_np(C), A.astype(np.float64) @ B.astype(np.float64).T, out_bf16=False)
 
 
-@pytest.mark.parametrize("M,N,K", [(256, 128, 192), (130, 256, 64), (200, 192, 32)])
+@pytest.mark.parametrize("M,N,K", [(256, 128, 192), (130, 256, 64), (200, 192, 32), (900, 512, 2048), (270, 768, 2304)])
 def test_dense_kmajor_mnmajor_with_accumulate(M, N, K):
     import torch
     A, Bt = _rand((M, K), 5), _rand((K, N), 6, K ** -0.5)       # B(n,k) = Bt[k,n]
