@@ -111,6 +111,17 @@ def test_conventional_layer_of_eq3_on_expert_parallel_ranks(case):
     compare(w, inp, run_group(w, inp, case["tokens"]))
 
 
+@pytest.mark.parametrize("case", [
+    dict(shape=dict(d=16, r=8, h=8, E=1024, k=3), dtype=wl.DTYPE_F32, tokens=[90, 70, 0, 110, 60, 80, 100, 90]),
+    dict(shape=dict(d=64, r=64, h=64, E=1024, k=2), dtype=wl.DTYPE_BF16, tokens=[800, 700, 900, 600]),
+])
+def test_the_largest_expert_count_on_expert_parallel_ranks(case):
+    """E = 1024, the most the library takes: 128 or 256 experts per rank, most of them with a handful of rows or none."""
+    w = wl.Workload("ep", T=sum(case["tokens"]), dtype=case["dtype"], act=wl.ACT_GELU_ERF, seed=167, **case["shape"])
+    inp = skewed(w, 0.3)
+    compare(w, inp, run_group(w, inp, case["tokens"]))
+
+
 def test_small_config_on_four_ranks():
     w = wl.WORKLOADS["small"]
     inp = skewed(w, 0.0)

@@ -125,6 +125,7 @@ def test_tiny_fp32_forward_backward():
     dict(T=5, d=8, r=4, h=4, E=16, k=1),        # fewer slots than experts
     dict(T=300, d=36, r=20, h=44, E=7, k=2),    # nothing a multiple of a tile
     dict(T=33, d=16, r=8, h=8, E=48, k=40),     # more than 32 experts per token
+    dict(T=700, d=16, r=8, h=8, E=1024, k=3),   # the largest expert count the library takes; most experts empty
 ])
 @pytest.mark.parametrize("act", [wl.ACT_RELU, wl.ACT_GELU_ERF, wl.ACT_GELU_TANH])
 def test_fp32_edge_shapes(shape, act):
@@ -155,6 +156,7 @@ def test_small_bf16_full_config():
     dict(T=130, d=64, r=128, h=64, E=1, k=1),      # one expert
     dict(T=300, d=192, r=64, h=128, E=40, k=2),    # E between tile sizes
     dict(T=1000, d=256, r=192, h=320, E=16, k=4),  # widths that are odd multiples of 64
+    dict(T=3000, d=64, r=64, h=64, E=1024, k=2),   # the largest expert count: a few rows per expert, 1024 padded tiles
 ])
 @pytest.mark.parametrize("act", [wl.ACT_RELU, wl.ACT_GELU_ERF])
 def test_bf16_edge_shapes(shape, act):
