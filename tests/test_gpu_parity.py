@@ -167,6 +167,15 @@ def test_bf16_edge_shapes(shape, act):
     compare_full(w, inp, run_full(w, inp))
 
 
+def test_bf16_widths_beyond_the_large_workload():
+    """d = 8192, r = 1024, h = 2048: contractions twice as long and outputs twice as wide as the large workload's, on a
+    batch small enough for the oracle (300 tokens, 4 experts)."""
+    w = wl.Workload("wide", dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=211, T=300, d=8192, r=1024, h=2048, E=4, k=2)
+    inp = conditioned(w)
+    margin.enforce_margin(w, inp, 1e-3)
+    compare_full(w, inp, run_full(w, inp))
+
+
 @pytest.mark.parametrize("case", [
     # one expert takes a slot of nearly every token
     dict(shape=dict(T=6000, d=256, r=256, h=512, E=16, k=2), bias="one_hot"),
