@@ -399,11 +399,13 @@ def test_inference_forward_with_the_experts_in_one_kernel(case):
 
 
 @pytest.mark.parametrize("T,E,k", [(1, 1, 1), (31, 7, 1), (128, 256, 8), (1024, 5, 1), (205, 64, 5), (256, 256, 8),
-                                   (2048, 3, 1), (257, 16, 8), (683, 40, 3), (300, 300, 7)])
+                                   (2048, 3, 1), (257, 16, 8), (683, 40, 3), (300, 300, 7),
+                                   (150000, 64, 8), (70000, 1024, 4)])
 @pytest.mark.parametrize("f", [0.0, 0.7])
 def test_routing_tables_around_the_single_block_limit(T, E, k, f):
     """Up to 2048 slots and 256 experts the tables come from one single-block kernel (one or two chunks of 1024
-    slots), beyond from the three-pass sort: both sides of both limits, with and without a capacity limit."""
+    slots), beyond from the three-pass sort: both sides of both limits, with and without a capacity limit; and two
+    batches well beyond the large workload's (1.2 million slots; 1024 experts), every table bit for bit."""
     import torch
 
     w = wl.Workload("tb", T=T, d=32, r=8, h=8, E=E, k=k, dtype=wl.DTYPE_F32, act=wl.ACT_RELU, seed=157)
