@@ -27,3 +27,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_library():
+    """On a machine with a GPU the CUDA library is compiled first if it is absent or older than its sources (a fresh
+    checkout holds sources only); the tests themselves never run without it."""
+    if _has_gpu():
+        from paper_2502_16927_b200 import build
+
+        build.build()
