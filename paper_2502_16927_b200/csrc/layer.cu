@@ -30,6 +30,7 @@ struct Buffers {
     float* aux_loss;     // [1] saved: L_aux of the batch
     float* logits_saved; // [T,E] saved copy of the gate logits (only with a load-balancing loss)
     float* splitk_ws;    // fp32 partial results of the split weight-gradient contractions
+    float* bias_ws;      // fp32 row-slice sums of the expert-bias gradients (a region of their own: they run on the second stream)
 };
 
 struct Dims {
@@ -111,9 +112,8 @@ void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
     const size_t dense_ws = (size_t)kMaxSplitK * m.ldcat * m.d * sizeof(float);
     const size_t expert_ws = m.dtype == BIGMAC_BF16 ? gemm_tc_groupk_ws_bytes(m.r, m.h, m.E) : 0;
     const size_t bias_ws = m.bias ? (size_t)m.E * kColsumSlices * (m.h > m.r ? m.h : m.r) * sizeof(float) : 0;
-    size_t ws = dense_ws > expert_ws ? dense_ws : expert_ws;
-    if (bias_ws > ws) ws = bias_ws;
-    b.splitk_ws = (float*)cv.take_bytes(ws);
+    b.splitk_ws = (float*)cv.take_bytes(dense_ws > expert_ws ? dense_ws : expert_ws);
+    b.bias_ws = bias_ws ? (float*)cv.take_bytes(bias_ws) : nullptr;
 }
 
 size_t forward_scratch_bytes(const Dims& m, bool training) {
@@ -556,10 +556,17 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     if (overlap) BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[1], 0));    // from here on the fp32 workspace is used again
     if (m.bias) {   // db1_e = sum_rows dz[row,:], db2_e = sum_rows du[row,:]  (padding rows hold zeros)
         if (!aligned(G->db1, 4) || !aligned(G->db2, 4)) return BIGMAC_ERR_INVALID_ARG;
-        Stage s(L, S_COLSUM, st, 2 * ((G->db1 ? 1 : 0) + (G->db2 ? 1 : 0)));
-        // the fp32 workspace is free here: the split dW_up has been reduced, the per-expert weight gradients come later
-        if (G->db1) BIGMAC_CUDA(launch_grouped_colsum(dz, b.tb.poffsets, G->db1, b.splitk_ws, m.E, m.h, m.dtype, acc, st));
-        if (G->db2) BIGMAC_CUDA(launch_grouped_colsum(b.du, b.tb.poffsets, G->db2, b.splitk_ws, m.E, m.r, m.dtype, acc, st));
+        // Two HBM-bound passes over dz and du that nothing later in the pass reads: with the second stream they run
+        // beside the tensor-bound dW2 / dxg (joined with the dx' gather), on slice sums in a region of their own.
+        cudaStream_t sb = st;
+        if (overlap) {
+            BIGMAC_CUDA(cudaEventRecord(L->fork_join[8], st));
+            BIGMAC_CUDA(cudaStreamWaitEvent(sd, L->fork_join[8], 0));
+            sb = sd;
+        }
+        Stage s(L, S_COLSUM, sb, 2 * ((G->db1 ? 1 : 0) + (G->db2 ? 1 : 0)));
+        if (G->db1) BIGMAC_CUDA(launch_grouped_colsum(dz, b.tb.poffsets, G->db1, b.bias_ws, m.E, m.h, m.dtype, acc, sb));
+        if (G->db2) BIGMAC_CUDA(launch_grouped_colsum(b.du, b.tb.poffsets, G->db2, b.bias_ws, m.E, m.r, m.dtype, acc, sb));
     }
     if (G->dw2) {   // dW2_e[c',q] = sum_rows du[row,c'] a[row,q]
         GemmArgs g;

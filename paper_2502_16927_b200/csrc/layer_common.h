@@ -18,7 +18,7 @@ struct bigmac_layer {
     // second stream of the backward pass (created on first use): launches that do not depend on each other and lean
     // on different units (a tensor-bound weight gradient beside an HBM-bound row move) run side by side
     cudaStream_t side = nullptr;
-    cudaEvent_t fork_join[8] = {};
+    cudaEvent_t fork_join[9] = {};
     // measurement aid
     bool prof_on = false;
     uint64_t launches = 0;
