@@ -486,7 +486,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     // do not depend on.  Everything that shares the fp32 workspace stays ordered.
     static const bool overlap_on = []() { const char* e = std::getenv("BIGMAC_OVERLAP"); return !(e && e[0] == '0'); }();
     // (not while per-stage events are recorded: a stage timed beside another stream's launches would not be its own time)
-    const bool overlap = overlap_on && L->side && !L->prof_on && !m.cdac && !m.gate_low;
+    const bool overlap = overlap_on && L->side && !L->prof_on && !m.cdac;
     cudaStream_t sd = st;
     if (overlap) {
         sd = L->side;
@@ -672,7 +672,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
                 BIGMAC_TRY(gemm(L, G_DW_GATE, g, st));
             }
         }
-        if (G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st, aux_part)); }
+        if (!colsum_done && G->db_gate) { Stage s(L, S_COLSUM, st, 2); BIGMAC_CUDA(launch_gate_colsum(b.dp, b.tb, G->db_gate, b.colsum_part, m.N, m.E, acc, st, aux_part)); }
         return BIGMAC_OK;
     }
     if (fused) {

@@ -183,10 +183,12 @@ def test_expert_parallel_exchange_stays_inside_the_exchange_buffers():
     group.close()
 
 
-def test_backward_on_two_streams_equals_backward_on_one_and_can_be_captured():
+@pytest.mark.parametrize("variant", [{}, {"gate_low": True}, {"expert_bias": True}], ids=["plain", "gate_low", "expert_bias"])
+def test_backward_on_two_streams_equals_backward_on_one_and_can_be_captured(variant):
     """bigmac_backward forks a few independent launches to the handle's second stream and joins them back: the
-    results are bit for bit those of the one-stream order (run in a child process with BIGMAC_OVERLAP=0), and a
-    captured forward + backward replays to the same bits."""
+    results are bit for bit those of the one-stream order (run in a child process with BIGMAC_OVERLAP=0), a
+    captured forward + backward replays to the same bits, and a pass that accumulates adds each gradient once.
+    The variants put more on the second stream (the expert-bias column sums) or join it elsewhere (gate on x')."""
     import os
     import subprocess
     import sys
@@ -195,8 +197,9 @@ def test_backward_on_two_streams_equals_backward_on_one_and_can_be_captured():
     import numpy as np
     import torch
 
-    w = wl.Workload("ov", T=3000, d=256, r=128, h=256, E=16, k=4, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=167)
-    inp = conditioned(w)
+    w = wl.Workload("ov", T=3000, d=256, r=128, h=256, E=16, k=4, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=167,
+                    **variant)
+    inp = wl.make_inputs(w) if variant else conditioned(w)
     dev = to_device(w, inp)
     layer = make_layer(w)
     y = layer.forward(dev["x"], dev, training=True)
@@ -205,6 +208,17 @@ def test_backward_on_two_streams_equals_backward_on_one_and_can_be_captured():
     torch.cuda.synchronize()
     assert layer.status() == 0
     eager = {key: val.clone() for key, val in dict(G, y=y, dx=dx).items()}
+
+    # accumulation on top of 0.5: every gradient is added exactly once (fp32 ones to rounding, BF16 ones to a BF16 step)
+    G3 = empty_grads(w, "cuda", fill=0.5)
+    layer.forward(dev["x"], dev, training=True)
+    layer.backward(dev["x"], dev["dy"], dev, G3, accumulate=True)
+    torch.cuda.synchronize()
+    for key, val in G3.items():
+        want = eager[key].double() + 0.5
+        tol = (1e-5 if val.dtype == torch.float32 else 1e-2) * (1.0 + want.abs())
+        assert bool(((val.double() - want).abs() <= tol).all()), key
+        assert float(eager[key].double().abs().max()) > 0.05, key          # large enough for a second addition to show
 
     # the same step captured into a CUDA graph and replayed
     side = torch.cuda.Stream()
@@ -235,12 +249,13 @@ def test_backward_on_two_streams_equals_backward_on_one_and_can_be_captured():
             "from paper_2502_16927_b200 import workloads as wl\n"
             "from helpers import empty_grads, make_layer, to_device\n"
             "from test_gpu_parity import conditioned\n"
-            "w = wl.Workload('ov', T=3000, d=256, r=128, h=256, E=16, k=4, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=167)\n"
-            "inp = conditioned(w); dev = to_device(w, inp); layer = make_layer(w)\n"
+            "variant = %r\n"
+            "w = wl.Workload('ov', T=3000, d=256, r=128, h=256, E=16, k=4, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=167, **variant)\n"
+            "inp = wl.make_inputs(w) if variant else conditioned(w); dev = to_device(w, inp); layer = make_layer(w)\n"
             "y = layer.forward(dev['x'], dev, training=True); G = empty_grads(w, 'cuda', fill=float('nan'))\n"
             "dx = layer.backward(dev['x'], dev['dy'], dev, G); torch.cuda.synchronize(); assert layer.status() == 0\n"
             "torch.save({k: v.cpu() for k, v in dict(G, y=y, dx=dx).items()}, %r)\n"
-        ) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)), out)
+        ) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)), variant, out)
         subprocess.run([sys.executable, "-c", code], check=True, env=dict(os.environ, BIGMAC_OVERLAP="0"), timeout=600)
         one = torch.load(out)
     for key, val in eager.items():
