@@ -735,6 +735,11 @@ def run_ours(args, w):
                 "frac_of_burst_peak": round(achieved / peaks["tflops_burst"], 4),
                 "step_frac": round(3.0 * fwd_fl / (ms_step * 1e-3) / 1e12 / peaks["tflops_sustained"], 4)}
 
+    gemm_stages = [n for n in stages if n in GEMM_FLOPS]
+    if gemm_stages:     # the single launch that takes the most time of a step, with its own rates
+        top = max(gemm_stages, key=lambda n: stages[n]["ms"])
+        roofline["longest_launch"] = dict(stages[top], stage=top)
+
     rate, dt, S_used, cores = oracle_sample_rate(w, inp, args.ref_tokens or sample_size_for(w, inp, 15.0))
     bytes_io = 2 * w.T * w.d * esz
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
