@@ -61,12 +61,44 @@ ROW_MOVE_BYTES = {   # per launch, algorithmic: rows read + rows written (+ the 
 }
 
 
-# The two expert contractions whose outputs are larger than their inputs sit nearer to an HBM floor than to the tensor
-# one; algorithmic bytes per launch (b = bytes per element; sigma' is saved as one byte per element on the BF16 path).
-OUTPUT_HEAVY_GEMM_BYTES = {
+def _e64(w):
+    return (w.E + 63) // 64 * 64
+
+
+# Algorithmic operand + output bytes per launch of every contraction (b = bytes per element; the saved sigma' is one
+# byte per element on the BF16 path, logits are fp32): what the launch has to read and write once, with no re-reads.
+GEMM_BYTES = {
+    "gemm_logits": lambda w, b: (w.T * w.d + w.E * w.d) * b + 4.0 * w.T * w.E,
+    "gemm_descend": lambda w, b: (w.T * w.d + w.r * w.d + w.T * w.r) * b,
     "gemm_expert1": lambda w, b: (w.N * w.r + w.E * w.h * w.r + w.N * w.h) * b + w.N * w.h * (1 if b == 2 else b),
+    "gemm_expert2": lambda w, b: (w.N * w.h + w.E * w.h * w.r + w.N * w.r) * b,
+    "gemm_ascend": lambda w, b: (w.T * w.r + w.r * w.d + w.T * w.d) * b,
+    "gemm_dy_lo": lambda w, b: (w.T * w.d + w.r * w.d + w.T * w.r) * b,
+    "gemm_dw_up": lambda w, b: (w.T * w.d + w.T * w.r + w.r * w.d) * b,
     "gemm_dz": lambda w, b: (w.N * w.r + w.E * w.h * w.r + w.N * w.h) * b + w.N * w.h * (1 if b == 2 else b),
+    "gemm_dw2": lambda w, b: (w.N * w.r + w.N * w.h + w.E * w.h * w.r) * b,
+    "gemm_dxg": lambda w, b: (w.N * w.h + w.E * w.h * w.r + w.N * w.r) * b,
+    "gemm_dw1": lambda w, b: (w.N * w.h + w.N * w.r + w.E * w.h * w.r) * b,
+    "gemm_dx": lambda w, b: (w.T * w.r + w.r * w.d + w.T * w.d) * b,
+    "gemm_dx_gate": lambda w, b: (w.T * _e64(w) + w.E * w.d) * b,
+    "gemm_dw_down": lambda w, b: (w.T * w.r + w.T * w.d + w.r * w.d) * b,
+    "gemm_dw_gate": lambda w, b: (w.T * _e64(w) + w.E * w.d) * b,
 }
+
+# DRAM bytes per launch of the two output-heavy contractions as ncu counted them (dram__bytes_read.sum +
+# dram__bytes_write.sum) on a SMALL case of the large workload's widths (T = 8192, one launch per capture:
+# profiles/expert_gemm1_dz_dram_small_case.md), as bytes that do not depend on the batch (the experts' weights) plus
+# bytes per routed row.  A full launch is scaled from that by its rows.  None until a capture of this build exists.
+MEASURED_DRAM = {
+}
+
+
+def measured_traffic(stage, w):
+    key = (stage, w.d, w.r, w.h, w.E, w.k)
+    if key not in MEASURED_DRAM:
+        return None
+    fixed, per_row = MEASURED_DRAM[key]
+    return fixed + per_row * w.N
 
 
 def measured_peaks():
@@ -81,50 +113,92 @@ def measured_peaks():
 
 # ------------------------------------------------------------------------------------------------ clocks
 class ClockSampler:
-    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and throttle reasons of one GPU while the timed regions run (reading only: no
+    setting of the GPU is touched).  NVML is polled every 5 ms from a thread, so that a region of a few tens of
+    milliseconds still gets samples; without the NVML module nvidia-smi is polled every 100 ms instead."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20), ("sw_power_cap", 0x4))
 
-    def __init__(self, index: int):
-        self.rows, self.proc, self.thread = [], None, None
+    def __init__(self, index: int, uuid: str = ""):
+        self.rows, self.proc, self.thread, self.nvml, self.max_mhz = [], None, None, None, None   # rows: (time, mhz, watts, reasons)
+        self._stop = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            try:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid if uuid.startswith("GPU-") else "GPU-" + uuid) if uuid else None
+            except Exception:
+                self.handle = None
+            if self.handle is None:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.nvml = pynvml
+            self.thread = threading.Thread(target=self._poll_nvml, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
                                           "--format=csv,noheader,nounits", "-lms", "100"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread = threading.Thread(target=self._read_smi, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
 
-    def _read(self):
+    def _poll_nvml(self):
+        n = self.nvml
+        while not self._stop.is_set():
+            try:
+                mhz = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+                watts = n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0
+                mask = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                self.rows.append((time.time(), mhz, watts, {name for name, bit in self.REASONS if mask & bit}))
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def _read_smi(self):
         for line in self.proc.stdout:
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) >= 7:
-                self.rows.append((time.time(), parts))
+            if len(parts) < 7:
+                continue
+            try:
+                mhz, self.max_mhz, watts = float(parts[0]), float(parts[1]), float(parts[2])
+            except ValueError:
+                continue
+            names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+            self.rows.append((time.time(), mhz, watts, {n for n, v in zip(names, parts[3:7]) if v.lower().startswith("active")}))
+
+    def window(self, t0, t1):
+        """Median SM MHz (and the rest) of the samples taken between two host times."""
+        inside = [r for r in self.rows if t0 <= r[0] <= t1 + 0.01]
+        if not inside:
+            return None
+        reasons = set()
+        for r in inside:
+            reasons |= r[3]
+        return {"sm_mhz": float(np.median([r[1] for r in inside])), "watts": float(np.median([r[2] for r in inside])),
+                "reasons": sorted(reasons), "samples": len(inside)}
 
     def stop(self, t0=None, t1=None):
+        self._stop.set()
         if self.proc is not None:
             self.proc.terminate()
             try:
                 self.proc.wait(timeout=5)
             except subprocess.TimeoutExpired:
                 self.proc.kill()
-        inside = [r for t, r in self.rows if t0 is None or (t0 <= t <= t1 + 0.15)]
-        window = "timed region"
-        if not inside:                      # region shorter than the sampling period: use the loaded run
-            inside, window = [r for _, r in self.rows], "warm-up and timed region"
-        sm, mx, reasons = [], 0.0, set()
-        for r in inside:
-            try:
-                sm.append(float(r[0])); mx = max(mx, float(r[1]))
-            except ValueError:
-                continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None,
-                "reasons": sorted(reasons), "samples": len(sm), "window": window}
+        win, label = (self.window(t0, t1) if t0 is not None else None), "timed region"
+        if win is None and self.rows:                    # region shorter than the sampling period: use the loaded run
+            win, label = self.window(self.rows[0][0], self.rows[-1][0]), "warm-up and timed region"
+        if win is None:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "window": label}
+        return {"sm_mhz": win["sm_mhz"], "sm_max_mhz": self.max_mhz, "reasons": win["reasons"], "samples": win["samples"],
+                "power_w": round(win["watts"], 1), "window": label, "source": "nvml" if self.nvml else "nvidia-smi"}
 
 
 # ------------------------------------------------------------------------------------------------ oracle leg
@@ -501,7 +575,13 @@ def run_ours(args, w):
     if rank != 0:
         del inp
 
+    # the decode-shaped configuration is an inference forward (no backward exists for it in the metric)
+    forward_only_workload = w.name == "decode"
+
     def step():
+        if forward_only_workload:
+            layer.forward(x, dev, y=y, training=False)
+            return
         layer.forward(x, dev, y=y, training=True)
         layer.backward(x, dy, dev, G, dx=dx)
 
@@ -522,6 +602,7 @@ def run_ours(args, w):
         return slowest_rank_ms(start.elapsed_time(stop), device="cuda")
 
     if args.profile_run:                    # bare loop for a profiler: warm-up and K steps, nothing else
+        binding.bigmac_debug_set("overlap", 0)   # one stream: launches reach the profiler in program order
         for _ in range(args.warmup + args.steps):
             step()
         torch.cuda.synchronize()
@@ -530,7 +611,7 @@ def run_ours(args, w):
         print(json.dumps({"profile_run": True, "config": config_dict(w, args), "steps": args.steps,
                           "warmup": args.warmup}))
         return
-    sampler = ClockSampler(local) if rank == 0 else None
+    sampler = ClockSampler(local, str(torch.cuda.get_device_properties(local).uuid)) if rank == 0 else None
     t_warm = time.time()
     for _ in range(max(args.warmup, 3)):
         step()
@@ -573,10 +654,30 @@ def run_ours(args, w):
         for half in ((plain_half, events_half) if i == 0 else (events_half, plain_half)):
             half(n)
     t1 = time.time()
-    clocks = sampler.stop(t0, t1) if sampler else None
     ms_step = ms_total / args.steps
     ms_step_events = ms_events_total / args.steps
     value = whole_job_tokens_per_s(w.T, world, ms_step)
+
+    # ---- the same K plain steps again as separate regions, each with the SM clock seen while it ran: median and
+    # minimum over the regions, and time x clock (million SM cycles per step), which tells a faster kernel from a
+    # GPU that happened to clock higher under the power cap.  The headline stays the region above.
+    n_regions = 5 if ms_step * args.steps < 2000.0 else 2
+    regions = []
+    for _ in range(n_regions):
+        ta = time.time()
+        ms_r = timed(step, args.steps) / args.steps
+        tb = time.time()
+        win = sampler.window(ta, tb) if sampler else None
+        regions.append({"ms_per_step": round(ms_r, 4), "sm_mhz": win["sm_mhz"] if win else None,
+                        "mcycles_per_step": round(ms_r * win["sm_mhz"] / 1e3, 3) if win else None})
+    clocks = sampler.stop(t0, t1) if sampler else None
+    r_ms = [r["ms_per_step"] for r in regions]
+    r_mc = [r["mcycles_per_step"] for r in regions if r["mcycles_per_step"] is not None]
+    repeats = {"regions": n_regions, "steps_per_region": args.steps, "ms_per_step_median": float(np.median(r_ms)),
+               "ms_per_step_min": float(np.min(r_ms)),
+               "mcycles_per_step_median": float(np.median(r_mc)) if r_mc else None, "each": regions}
+    if clocks and clocks.get("sm_mhz"):
+        clocks["mcycles_per_step"] = round(ms_step * clocks["sm_mhz"] / 1e3, 3)
 
     # forward only (inference forward: nothing saved)
     def fwd_only():
@@ -605,7 +706,14 @@ def run_ours(args, w):
     # ---- the exchange stage alone at width r (BigMac) and at width d (a fine-grained CDAC layer of equal E, k
     # dispatches and combines full-width rows, Eq. 1): same kernels, same routing, rank 0's GPU only
     exchange = None
-    if rank == 0:
+    touched_bytes, n_distinct = None, None
+    if forward_only_workload:
+        _, Rt = layer.forward(x, dev, y=y, training=False, want_routing=True)
+        torch.cuda.synchronize()
+        n_distinct = int((Rt["counts"] > 0).sum().item())
+        esz_ = 2 if w.dtype == wl.DTYPE_BF16 else 4
+        touched_bytes = float((2 * w.T * w.d + w.E * w.d + 2 * w.r * w.d + 2 * n_distinct * w.r * w.h) * esz_)
+    if rank == 0 and not forward_only_workload:
         layer.forward(x, dev, y=y, training=True)                  # leaves the routing tables in `saved`
         P = ((w.N + 127) // 128 + w.E) * 128
         exchange = {}
@@ -647,17 +755,22 @@ def run_ours(args, w):
             s_in.wait_event(ev_comp[i & 1])                 # the step that last read these input buffers is done
             with torch.cuda.stream(s_in):
                 bx.copy_(hx, non_blocking=True)
-                bdy.copy_(hdy, non_blocking=True)
+                if not forward_only_workload:
+                    bdy.copy_(hdy, non_blocking=True)
                 ev_in[i & 1].record(s_in)
             main.wait_event(ev_in[i & 1])
             main.wait_event(ev_out[i & 1])                  # ... and its outputs have left the output buffers
-            layer.forward(bx, dev, y=by, training=True)
-            layer.backward(bx, bdy, dev, G, dx=bdx)
+            if forward_only_workload:
+                layer.forward(bx, dev, y=by, training=False)
+            else:
+                layer.forward(bx, dev, y=by, training=True)
+                layer.backward(bx, bdy, dev, G, dx=bdx)
             ev_comp[i & 1].record(main)
             s_out.wait_event(ev_comp[i & 1])
             with torch.cuda.stream(s_out):
                 hy.copy_(by, non_blocking=True)
-                hdx.copy_(bdx, non_blocking=True)
+                if not forward_only_workload:
+                    hdx.copy_(bdx, non_blocking=True)
                 ev_out[i & 1].record(s_out)
         main.wait_event(ev_out[0])
         main.wait_event(ev_out[1])
@@ -682,10 +795,12 @@ def run_ours(args, w):
 
     peaks = measured_peaks()
     esz = 2 if w.dtype == wl.DTYPE_BF16 else 4
-    twin = run_cdac_twin(w, x, dy, dev, ms_step, ms_fwd, max(3, min(args.steps, 10)), peaks, esz)
-    ep_line = run_ep_on_one_gpu(w, x, dy, dev, ms_step, max(3, min(args.steps, 10)), esz) if w.dtype == wl.DTYPE_BF16 else None
-    variants = run_small_variants(w, x, dy, dev, G, y, dx, step, max(3, min(args.steps, 10)))
-    recipe = run_recipe_variant(w, x, dy, dev, G, y, dx, step, max(3, min(args.steps, 10)))
+    twin = ep_line = variants = recipe = None
+    if not forward_only_workload and not args.headline_only:
+        twin = run_cdac_twin(w, x, dy, dev, ms_step, ms_fwd, max(3, min(args.steps, 10)), peaks, esz)
+        ep_line = run_ep_on_one_gpu(w, x, dy, dev, ms_step, max(3, min(args.steps, 10)), esz) if w.dtype == wl.DTYPE_BF16 else None
+        variants = run_small_variants(w, x, dy, dev, G, y, dx, step, max(3, min(args.steps, 10)))
+        recipe = run_recipe_variant(w, x, dy, dev, G, y, dx, step, max(3, min(args.steps, 10)))
     stages = {}
     gemm_ms = gemm_flops = 0.0
     flops_of = {name: fn(w) for name, fn in GEMM_FLOPS.items()}
@@ -695,6 +810,14 @@ def run_ours(args, w):
         flops_of["gemm_dx"] += flops_of["gemm_dx_gate"]
     if "gemm_dw_gate" not in prof["stages"]:        # dW_gate computed together with dW_down
         flops_of["gemm_dw_down"] += flops_of["gemm_dw_gate"]
+    bytes_of = {name: fn(w, esz) for name, fn in GEMM_BYTES.items()}
+    if "gemm_logits" not in prof["stages"]:
+        bytes_of["gemm_descend"] += esz * w.E * w.d + 4.0 * w.T * w.E
+    if "gemm_dx_gate" not in prof["stages"]:
+        bytes_of["gemm_dx"] += bytes_of["gemm_dx_gate"]
+    if "gemm_dw_gate" not in prof["stages"]:
+        bytes_of["gemm_dw_down"] += bytes_of["gemm_dw_gate"]
+    gemm_bytes = 0.0
     for name, (ms, calls) in prof["stages"].items():
         per = ms / calls
         entry = {"ms": round(per, 4), "launches_per_step": calls // args.steps}
@@ -704,9 +827,10 @@ def run_ours(args, w):
             entry["frac_of_measured_sustained"] = round(entry["tflops"] / peaks["tflops_sustained"], 3)
             gemm_ms += ms
             gemm_flops += fl * calls
-            if name in OUTPUT_HEAVY_GEMM_BYTES:
-                entry["hbm_gbs"] = round(OUTPUT_HEAVY_GEMM_BYTES[name](w, esz) / (per * 1e-3) / 1e9, 1)
-                entry["frac_of_measured_hbm"] = round(entry["hbm_gbs"] / peaks["hbm_gbs"], 3)
+            gemm_bytes += bytes_of[name] * calls
+            entry["algorithmic_bytes"] = bytes_of[name]
+            entry["hbm_gbs"] = round(bytes_of[name] / (per * 1e-3) / 1e9, 1)
+            entry["frac_of_measured_hbm"] = round(entry["hbm_gbs"] / peaks["hbm_gbs"], 3)
         elif name in ROW_MOVE_BYTES:
             by = ROW_MOVE_BYTES[name](w, esz)
             entry["gbs"] = round(by / (per * 1e-3) / 1e9, 1)
@@ -720,35 +844,54 @@ def run_ours(args, w):
     m_ms = sum(stages[n]["ms"] for n in moves)
     m_gbs = sum(ROW_MOVE_BYTES[n](w, esz) for n in moves) / (m_ms * 1e-3) / 1e9 if m_ms > 0 else 0.0
     groups = {"grouped_expert_gemms": {"ms": round(g_ms, 4), "tflops": round(g_tf, 1),
-                                       "frac_of_measured_sustained": round(g_tf / peaks["tflops_sustained"], 3)},
+                                       "frac_of_measured_sustained": round(g_tf / peaks["tflops_sustained"], 3),
+                                       "frac_of_measured_burst": round(g_tf / peaks["tflops_burst"], 3)},
               "dispatch_combine_and_their_backward": {"ms": round(m_ms, 4), "gbs": round(m_gbs, 1),
                                                       "frac_of_measured_hbm": round(m_gbs / peaks["hbm_gbs"], 3)}}
     achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
     fwd_fl = forward_flops(w)
-    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (tcgen05 contractions, all launches of a step)",
-                "achieved": round(achieved, 1), "peak": peaks["tflops_sustained"], "unit": "TFLOP/s",
-                "frac": round(achieved / peaks["tflops_sustained"], 4),
-                # DRAM bytes of those launches per step from a one-pass ncu capture of this workload
-                # (profiles/gemm_dram_traffic_large.md); not captured for the other workloads
-                "traffic": 12.791e9 if (w.name == "large" and w.T == 32768) else None,
-                "peak_source": f"{peaks['source']}: sustained bf16 (kernels timed inside a long step)",
-                "frac_of_burst_peak": round(achieved / peaks["tflops_burst"], 4),
-                "step_frac": round(3.0 * fwd_fl / (ms_step * 1e-3) / 1e12 / peaks["tflops_sustained"], 4)}
-
+    all_gemms = {"kernels": "every tcgen05 contraction launch of a step", "launches_per_step": sum(stages[n]["launches_per_step"] for n in stages if n in GEMM_FLOPS),
+                 "achieved": round(achieved, 1), "unit": "TFLOP/s", "frac": round(achieved / peaks["tflops_sustained"], 4),
+                 "frac_of_burst_peak": round(achieved / peaks["tflops_burst"], 4), "ms_per_step": round(gemm_ms / args.steps, 4),
+                 "algorithmic_bytes_per_step": gemm_bytes / args.steps}
     gemm_stages = [n for n in stages if n in GEMM_FLOPS]
-    if gemm_stages:     # the single launch that takes the most time of a step, with its own rates
+    if forward_only_workload:
+        # decode-shaped batches stream the touched weights once: the bound is HBM, not the tensor pipe
+        roofline = {"bound": "hbm", "kernel": "inference forward (every launch of a call)",
+                    "achieved": round(touched_bytes / (ms_fwd * 1e-3) / 1e9, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": round(touched_bytes / (ms_fwd * 1e-3) / 1e9 / peaks["hbm_gbs"], 4), "traffic": None,
+                    "algorithmic_bytes": touched_bytes, "distinct_experts": n_distinct,
+                    "peak_source": f"{peaks['source']}: copy bandwidth", "floor_us": round(touched_bytes / peaks["hbm_gbs"] / 1e3, 2)}
+    elif gemm_stages:
+        # the dominant kernel = the single launch that takes the most time of a step; all contractions together follow
         top = max(gemm_stages, key=lambda n: stages[n]["ms"])
-        roofline["longest_launch"] = dict(stages[top], stage=top)
+        t = stages[top]
+        roofline = {"bound": "tensor", "kernel": f"{top}: the longest launch of a step (tcgen05 contraction)",
+                    "achieved": t["tflops"], "peak": peaks["tflops_sustained"], "unit": "TFLOP/s",
+                    "frac": round(t["tflops"] / peaks["tflops_sustained"], 4),
+                    "traffic": measured_traffic(top, w),
+                    "traffic_source": ("ncu dram bytes of one launch on a small case of the same widths, scaled by rows"
+                                       if measured_traffic(top, w) else None),
+                    "algorithmic_bytes": t["algorithmic_bytes"], "ms": t["ms"], "hbm_gbs": t["hbm_gbs"],
+                    "frac_of_measured_hbm": t["frac_of_measured_hbm"],
+                    "peak_source": f"{peaks['source']}: sustained bf16 (kernels timed inside a long step)",
+                    "frac_of_burst_peak": round(t["tflops"] / peaks["tflops_burst"], 4),
+                    "all_gemm_launches": all_gemms,
+                    "step_frac": round(3.0 * fwd_fl / (ms_step * 1e-3) / 1e12 / peaks["tflops_sustained"], 4)}
+    else:
+        roofline = {"bound": "alu", "kernel": "fp32 FMA path (correctness configuration, not a performance point)",
+                    "achieved": None, "peak": None, "unit": "TFLOP/s", "frac": None, "traffic": None}
 
     rate, dt, S_used, cores = oracle_sample_rate(w, inp, args.ref_tokens or sample_size_for(w, inp, 15.0))
-    bytes_io = 2 * w.T * w.d * esz
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+    bytes_io = (1 if forward_only_workload else 2) * w.T * w.d * esz
+    line = {"metric": "bigmac_layer_fwd_tokens_per_s" if forward_only_workload else METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == wl.DTYPE_BF16 else "f32", "data": "synthetic",
             "config": config_dict(w, args), "clocks": clocks,
             "e2e": {"value": world * w.T / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": bytes_io,
                     "d2h_bytes_per_step": bytes_io, "ms_per_step": ms_e2e},
             "gpu_launches": prof["launches"],
+            "repeats": repeats,
             "with_stage_events": {"ms_per_step": ms_step_events, "value": whole_job_tokens_per_s(w.T, world, ms_step_events), "unit": UNIT},
             "forward_only": {"tokens_per_s": world * w.T / (ms_fwd * 1e-3), "ms": ms_fwd,
                              "frac_of_tensor_roofline": round(fwd_fl / (ms_fwd * 1e-3) / 1e12 / peaks["tflops_sustained"], 4),
@@ -777,6 +920,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="large", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0, help="override T (per GPU)")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="skip the side measurements (Eq. 3 twin, expert-parallel ranks on one GPU, variants, recipe)")
     ap.add_argument("--profile-run", action="store_true",
                     help="only run warm-up + K steps (for a kernel-list or counter capture); prints no bench line")
     ap.add_argument("--ref-tokens", type=int, default=0,

@@ -33,8 +33,14 @@
  *    passed in (a cudaStream_t as void*) and before whatever the caller puts there next.  bigmac_backward
  *    runs a few launches that do not depend on each other on a second stream owned by the handle, forked
  *    from and joined back into the caller's stream with events (stream capture sees an ordinary fork and
- *    join; BIGMAC_OVERLAP=0 in the environment keeps everything on the one stream).  One handle serves one
- *    stream at a time.
+ *    join; if a launch fails after the fork the second stream is joined back before the error is returned).
+ *    One handle serves one stream at a time.
+ *  - Behaviour does not depend on the environment: the library reads no environment variable.  Measurement and
+ *    debugging aids (per-stage timing, single contractions, kernel-choice switches) are declared in
+ *    bigmac_debug.h and are not part of this interface.
+ *  - Non-finite values are not trapped and propagate as in any matrix product, with one guarantee: routing never
+ *    writes an expert id outside [0, E).  A NaN gate logit is ordered as -inf; when only -inf logits are left among
+ *    the experts not yet chosen the lowest such id is taken (its gate value is 0, or 1/k if all k are -inf).
  *  - Return value: BIGMAC_OK (0) or a negative bigmac_status_t.  On an argument error nothing is
  *    launched.  Nothing throws, aborts or traps; problems detected on the device (a bounded wait that
  *    ran out) are recorded in a status word read by bigmac_device_status.
@@ -163,7 +169,7 @@ typedef struct {
 } bigmac_routing_t;
 
 /* Validate the configuration and create a handle on the current CUDA device.  Allocates one small
- * device status word (no other device memory is owned by the handle), one stream and eight events.
+ * device status word (no other device memory is owned by the handle), one stream and ten events.
  * Errors: INVALID_ARG (null pointers, non-positive sizes, k > E, unknown enums, a negative or non-finite
  * capacity_factor or aux_loss_coef), UNSUPPORTED (BF16
  * with d, r or h not a multiple of 64; E > 1024), CUDA. */
@@ -283,15 +289,6 @@ int bigmac_ep_backward_dispatch(bigmac_layer_t *L, const void *x, int32_t T, con
                                 const bigmac_ep_t *ep, void *dx, const bigmac_grads_t *G, int accumulate,
                                 void *saved, void *scratch, size_t scratch_bytes, void *stream);
 
-/* Measurement aid for the dispatch/combine stage (Eq. 1: bytes through the exchange are proportional
- * to the row width): run the standalone dispatch and combine kernels on rows of `width` elements of
- * the layer's dtype.  width = r is BigMac's exchange; width = d is what a fine-grained layer of equal
- * E and k moves.  src [T,width] -> grouped [rows_padded,width] -> dst [T,width] with the gate values
- * of the routing held in `saved` (from a training forward of the same T).  which: 0 = dispatch only,
- * 1 = combine only (grouped must hold data), 2 = both. */
-int bigmac_exchange_rows(bigmac_layer_t *L, const void *saved, int32_t T, int32_t width, const void *src,
-                         void *grouped, size_t grouped_bytes, void *dst, int which, void *stream);
-
 /* bigmac_route for callers that cannot provide scratch memory.  (The paper has no counterpart: this is
  * a deployment variant of the routing step, not part of the method.)
  *
@@ -305,34 +302,18 @@ int bigmac_exchange_rows(bigmac_layer_t *L, const void *saved, int32_t T, int32_
  *
  *  - It allocates nothing: no cudaMalloc / cudaFree, no allocating library routine.  The caller still passes
  *    x, the weights and the output tables (device memory, as for bigmac_route).
- *  - Limit: the routing intermediates of (T, E, k) must fit the array, roughly
- *    4*T*E + 20*T*k + 5*E*(T*k/1024 + 130) bytes; a larger problem is rejected with BIGMAC_ERR_TOO_LARGE and
- *    nothing is launched.
+ *  - Limit: the routing intermediates of (T, E, k) must fit the array: about
+ *    4*T*E + 24*T*k + 4*E*(T*k/1024) + 1.2 KB * E bytes, plus 4.8 KB * E with a load-balancing loss and T*r
+ *    elements with BIGMAC_FLAG_GATE_LOW (the return code is the authority: the exact carve includes 256-byte
+ *    alignment of every region); a larger problem is rejected with BIGMAC_ERR_TOO_LARGE and nothing is launched.
  *  - The first call on a device resolves the array's device address (once per device, with that device
- *    current); make that first call before any stream capture.
+ *    current); that first call should come before any stream capture.
  *  - All calls share the one array, and it keeps the previous call's contents (everything a call reads it
  *    has written itself first).  Two calls that overlap on the GPU - different streams, or different
  *    handles - race on it: serialise them. */
 #define BIGMAC_STATIC_SCRATCH_BYTES (8u << 20)
 int bigmac_route_static(bigmac_layer_t *L, const void *x, int32_t T, const bigmac_weights_t *W,
                         bigmac_routing_t *out, void *stream);
-
-/* Measurement aid: per-stage device timing and a launch counter.  While enabled, every kernel the
- * library launches is bracketed by a pair of CUDA events on the caller's stream (no synchronisation) and
- * counted.  bigmac_profile_read synchronises `stream`, adds the elapsed time of every bracket recorded
- * since the last read to its stage's slot and returns the totals; the bracket pool holds 8192 launches
- * between reads, later ones are counted in `dropped` and not timed.  The paper has no counterpart. */
-#define BIGMAC_PROFILE_SLOTS 32
-typedef struct {
-    uint64_t launches;                      /* kernels launched since enable */
-    uint32_t dropped;                       /* launches not timed because the pool was full */
-    int32_t n_slots;                        /* slots in use */
-    float ms[BIGMAC_PROFILE_SLOTS];         /* summed device time per stage */
-    uint32_t calls[BIGMAC_PROFILE_SLOTS];   /* launches per stage */
-} bigmac_profile_t;
-int bigmac_profile_enable(bigmac_layer_t *L, int on);
-int bigmac_profile_read(bigmac_layer_t *L, void *stream, bigmac_profile_t *out);
-const char *bigmac_profile_slot_name(int slot);
 
 #ifdef __cplusplus
 }

@@ -183,18 +183,24 @@ void oracle_gate_logits_low(const float* x, const float* w_down, const float* w_
 
 // Top-k set T of Eq. 2 and the gate values p_i: experts ordered by (logit descending, id ascending),
 // first k kept in that order; p = softmax over the k kept logits (so the p of a token sum to 1).
+// Non-finite logits (the paper is silent; a diverging run produces them): NaN is ordered as -inf, so that the order
+// is total and ties among -inf fall to the lower id; a token whose k kept logits are all -inf gets p = 1/k each.
+// Every id written lies in [0, E).
 void oracle_topk(const double* logits, int T, int E, int k, int32_t* topk_idx, double* topk_p) {
 #pragma omp parallel for schedule(static)
     for (int t = 0; t < T; ++t) {
-        const double* l = logits + (size_t)t * E;
+        std::vector<double> l(logits + (size_t)t * E, logits + (size_t)(t + 1) * E);
+        for (int e = 0; e < E; ++e)
+            if (std::isnan(l[e])) l[e] = -INFINITY;
         std::vector<int> order(E);
         std::iota(order.begin(), order.end(), 0);
-        std::stable_sort(order.begin(), order.end(), [l](int a, int b) { return l[a] > l[b]; });
-        double m = l[order[0]], denom = 0.0;
-        for (int j = 0; j < k; ++j) denom += std::exp(l[order[j]] - m);
+        std::stable_sort(order.begin(), order.end(), [&l](int a, int b) { return l[a] > l[b]; });
+        const double m = l[order[0]];
+        double denom = 0.0;
+        for (int j = 0; j < k; ++j) denom += std::isinf(m) && m < 0 ? 1.0 : std::exp(l[order[j]] - m);
         for (int j = 0; j < k; ++j) {
             topk_idx[(size_t)t * k + j] = order[j];
-            topk_p[(size_t)t * k + j] = std::exp(l[order[j]] - m) / denom;
+            topk_p[(size_t)t * k + j] = (std::isinf(m) && m < 0 ? 1.0 : std::exp(l[order[j]] - m)) / denom;
         }
     }
 }

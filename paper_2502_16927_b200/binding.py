@@ -90,6 +90,8 @@ def lib() -> C.CDLL:
         L.bigmac_debug_gemm.argtypes = [vp, C.POINTER(bigmac_debug_gemm_t), C.c_int, vp]
         L.bigmac_debug_expire_wait.argtypes = [vp, vp]
         L.bigmac_debug_expire_wait.restype = C.c_int
+        L.bigmac_debug_set.argtypes = [C.c_char_p, C.c_int]
+        L.bigmac_debug_set.restype = C.c_int
         L.bigmac_route_static.argtypes = [vp, vp, i32, C.POINTER(bigmac_weights_t), C.POINTER(bigmac_routing_t), vp]
         L.bigmac_route_static.restype = C.c_int
         L.bigmac_profile_enable.argtypes = [vp, C.c_int]
@@ -226,6 +228,12 @@ def bigmac_debug_gemm(handle, q: bigmac_debug_gemm_t, use_tensor_cores) -> None:
     """use_tensor_cores: False/0 plain FMA, True/1 tensor cores, 2 one-CTA kernel, 3/4/5 CTA-pair kernel with 4/2/1 working
     epilogue warps per lane quadrant."""
     _check(lib().bigmac_debug_gemm(handle, C.byref(q), int(use_tensor_cores), _stream()), "bigmac_debug_gemm")
+
+
+def bigmac_debug_set(name: str, value: int = 0) -> None:
+    """Process-wide measurement / debugging switch ("overlap", "tc_pair", "groupk", "fused_mlp", "epi_parts",
+    "fuse_dispatch", "tc_mask"; "defaults" restores all).  The defaults are the product."""
+    _check(lib().bigmac_debug_set(name.encode(), int(value)), "bigmac_debug_set")
 
 
 def bigmac_debug_expire_wait(handle) -> None:

@@ -150,7 +150,8 @@ __global__ void __launch_bounds__(256) gate_bwd_aux_kernel(float* __restrict__ d
         __syncwarp();
         for (int j = lane; j < k; j += 32) {
             const float dl = pw[j] * (gp[j] - part);
-            row[topk_idx[(int64_t)t * k + j]] += dl;  // the k experts of a token are distinct
+            const int e = topk_idx[(int64_t)t * k + j];
+            if ((unsigned)e < (unsigned)E) row[e] += dl;  // the k experts of a token are distinct
             gp[j] = dl;                               // fp32 copy per slot, for the bias gradient
         }
         __syncwarp();

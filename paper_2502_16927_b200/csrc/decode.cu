@@ -166,18 +166,21 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_forward_kernel(const
         float top = 0.0f, part = 0.0f;
         for (int j = 0; j < p.k; ++j) {
             float best = -INFINITY;
-            int best_e = 0x7fffffff;
-            for (int i = 0, e = lane; e < p.E; ++i, e += 32)
-                if (!((taken >> i) & 1u) && l[e] > best) { best = l[e]; best_e = e; }
+            int best_e = 0x7fffffff;                         // "no candidate yet"; k <= E, so every round ends with a real id
+            for (int i = 0, e = lane; e < p.E; ++i, e += 32) {
+                float v = l[e];
+                v = v == v ? v : -INFINITY;                  // NaN is ordered as -inf
+                if (!((taken >> i) & 1u) && (best_e == 0x7fffffff || v > best)) { best = v; best_e = e; }
+            }
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
                 const float ov = __shfl_xor_sync(kFull, best, off);
                 const int oe = __shfl_xor_sync(kFull, best_e, off);
                 if (ov > best || (ov == best && oe < best_e)) { best = ov; best_e = oe; }
             }
-            if ((best_e & 31) == lane) taken |= 1u << (best_e >> 5);
+            if (best_e != 0x7fffffff && (best_e & 31) == lane) taken |= 1u << (best_e >> 5);
             if (j == 0) top = best;
-            const float ex = expf(best - top);
+            const float ex = top == -INFINITY ? 1.0f : expf(best - top);   // only -inf logits kept: 1/k each
             part += ex;
             if (lane == 0) { p.topk_idx[t * p.k + j] = best_e; p.topk_w[t * p.k + j] = ex; }
         }

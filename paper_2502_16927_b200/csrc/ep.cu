@@ -138,12 +138,12 @@ __global__ void __launch_bounds__(256) ep_zero_padding_kernel(uint4* __restrict_
 __global__ void __launch_bounds__(256) ep_put_rows_kernel(const uint4* __restrict__ src, Peers dst, const int32_t* __restrict__ topk_idx,
                                                           const int32_t* __restrict__ row_of_slot, const int32_t* __restrict__ offsets,
                                                           const int32_t* __restrict__ send_base, int32_t* __restrict__ dest_row,
-                                                          int64_t N, int k, int El, int vecs) {
+                                                          int64_t N, int k, int El, int vecs, int E) {
     const int64_t s = warp_global_id();
     if (s >= N) return;
     const int lane = threadIdx.x & 31;
     const int e = topk_idx[s];
-    const int base = send_base[e];
+    const int base = (unsigned)e < (unsigned)E ? send_base[e] : -1;   // an id outside [0, E): treated like an empty layout
     if (base < 0) {                                  // empty layout (see ep_layout_kernel): nothing moves
         if (lane == 0) dest_row[s] = -1;
         return;
@@ -400,7 +400,7 @@ int bigmac_ep_route(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_we
         BIGMAC_TRY(gemm(L, G_DESCEND, q, st));
     }
     { Stage s(L, S_TOPK, st); BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st)); }
-    { Stage s(L, S_TABLES, st, tables_kernel_count(m.N, m.E)); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, kNoCapacity, st)); }
+    { Stage s(L, S_TABLES, st, tables_kernel_count(m.N, m.E)); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, kNoCapacity, st, L->status)); }
     BIGMAC_CUDA(cudaMemcpyAsync(my_counts, b.tb.counts, sizeof(int32_t) * m.E, cudaMemcpyDeviceToDevice, st));
     if (routing_out) {
         const cudaMemcpyKind kind = cudaMemcpyDeviceToDevice;
@@ -430,7 +430,7 @@ int bigmac_ep_dispatch(bigmac_layer_t* L, int32_t T, const bigmac_ep_t* ep, void
     if (T > 0)
         ep_put_rows_kernel<<<warp_blocks(m.N), 256, 0, st>>>((const uint4*)b.x_lo, peers_of(ep->xg, m.size), b.tb.topk_idx,
                                                             b.tb.row_of_slot, b.tb.offsets, b.send_base, b.dest_row, m.N, m.k, m.El,
-                                                            vecs);
+                                                            vecs, m.E);
     BIGMAC_CUDA(cudaGetLastError());
     return BIGMAC_OK;
 }

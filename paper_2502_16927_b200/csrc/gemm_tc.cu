@@ -351,8 +351,8 @@ cudaError_t launch_expire_wait(int* status, cudaStream_t stream) {
 
 cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
-    // Where it pays, the problem runs on CTA pairs (each SM stages half of B); BIGMAC_TC_PAIR=0 disables that.
-    static const bool pair_enabled = []() { const char* e = std::getenv("BIGMAC_TC_PAIR"); return !(e && e[0] == '0'); }();
+    // Where it pays, the problem runs on CTA pairs (each SM stages half of B); the tc_pair debug switch disables that.
+    const bool pair_enabled = switches().tc_pair != 0;
     const bool want_pair = g.force_kernel == 2 ? gemm_tc_pair_supported(g)
                            : g.force_kernel == 1 ? false : (pair_enabled && gemm_tc_pair_preferred(g));
     if (want_pair) return gemm_tc_pair(g, status, stream);

@@ -140,7 +140,9 @@ constexpr int kSmallTablesMaxSlots = 2048, kSmallTablesMaxExperts = 256;
 inline int tables_kernel_count(int64_t N, int E) {
     return (N > 0 && N <= kSmallTablesMaxSlots && E <= kSmallTablesMaxExperts) ? 1 : 3;
 }
-cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaStream_t stream);
+// `status` (nullable): the handle's status word; an expert id outside [0, E) - which the top-k kernels never write -
+// is placed nowhere (row -1) and recorded there as 2.
+cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaStream_t stream, int* status = nullptr);
 
 // Row moves.  `width` elements of the dtype per row; all row pointers 16-byte aligned.
 // grouped[prow,:] = src[slot_of_prow[prow]/k,:], zeros on padding rows, for prow < n_tiles*kPad.

@@ -10,6 +10,14 @@
 #include <vector>
 
 #include "layer_common.h"
+#include "switches.h"
+
+namespace bigmac {
+Switches& switches() {
+    static Switches s;
+    return s;
+}
+}  // namespace bigmac
 
 using namespace bigmac;
 using namespace bigmac::detail;
@@ -180,7 +188,7 @@ int choose_split_k(int M, int N, int K) {
 // any), load-balancing loss.
 int route_from_logits(const bigmac_layer* L, const Dims& m, const bigmac_weights_t* W, Buffers& b, cudaStream_t st) {
     { Stage s(L, S_TOPK, st); BIGMAC_CUDA(launch_topk(b.logits, W->b_gate, m.T, m.E, m.k, b.tb.topk_idx, b.tb.topk_w, st)); }
-    { Stage s(L, S_TABLES, st, tables_kernel_count(m.N, m.E)); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st)); }
+    { Stage s(L, S_TABLES, st, tables_kernel_count(m.N, m.E)); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st, L->status)); }
     if (m.aux > 0) {
         Stage s(L, S_AUX_LOSS, st, 2);
         BIGMAC_CUDA(launch_aux_loss(b.logits, W->b_gate, b.tb.counts_chosen, m.T, m.E, m.k, m.aux, b.aux_part, b.aux_loss, st));
@@ -208,22 +216,40 @@ int run_routing(const bigmac_layer* L, const Dims& m, const void* x, const bigma
     return route_from_logits(L, m, W, b, st);
 }
 
+// Calls that keep no saved state (bigmac_route, the inference forward): the tables the caller asked for are produced
+// in the caller's arrays themselves (same element types and layouts as the internal ones), so nothing is copied.
+void alias_routing(Buffers& b, const bigmac_routing_t* out) {
+    if (!out) return;
+    if (out->topk_idx) b.tb.topk_idx = out->topk_idx;
+    if (out->topk_w) b.tb.topk_w = out->topk_w;
+    if (out->counts) b.tb.counts = out->counts;
+    if (out->offsets) b.tb.offsets = out->offsets;
+    if (out->row_of_slot) b.tb.row_of_slot = out->row_of_slot;
+    if (out->slot_of_row) b.tb.slot_of_row = out->slot_of_row;
+    if (out->counts_chosen) b.tb.counts_chosen = out->counts_chosen;
+    if (out->aux_loss) b.aux_loss = out->aux_loss;
+}
+
+// Copies the tables into the caller's arrays (a training forward keeps its own copy in `saved` for the backward);
+// members that alias_routing pointed at the caller's arrays are already in place.
 int export_routing(const Dims& m, const Buffers& b, bigmac_routing_t* out, cudaStream_t st) {
     if (!out) return BIGMAC_OK;
     const cudaMemcpyKind kind = cudaMemcpyDeviceToDevice;
-    if (out->topk_idx) BIGMAC_CUDA(cudaMemcpyAsync(out->topk_idx, b.tb.topk_idx, sizeof(int32_t) * m.N, kind, st));
-    if (out->topk_w) BIGMAC_CUDA(cudaMemcpyAsync(out->topk_w, b.tb.topk_w, sizeof(float) * m.N, kind, st));
-    if (out->counts) BIGMAC_CUDA(cudaMemcpyAsync(out->counts, b.tb.counts, sizeof(int32_t) * m.E, kind, st));
-    if (out->offsets) BIGMAC_CUDA(cudaMemcpyAsync(out->offsets, b.tb.offsets, sizeof(int32_t) * (m.E + 1), kind, st));
-    if (out->row_of_slot)
+    if (out->topk_idx && out->topk_idx != b.tb.topk_idx)
+        BIGMAC_CUDA(cudaMemcpyAsync(out->topk_idx, b.tb.topk_idx, sizeof(int32_t) * m.N, kind, st));
+    if (out->topk_w && out->topk_w != b.tb.topk_w) BIGMAC_CUDA(cudaMemcpyAsync(out->topk_w, b.tb.topk_w, sizeof(float) * m.N, kind, st));
+    if (out->counts && out->counts != b.tb.counts) BIGMAC_CUDA(cudaMemcpyAsync(out->counts, b.tb.counts, sizeof(int32_t) * m.E, kind, st));
+    if (out->offsets && out->offsets != b.tb.offsets)
+        BIGMAC_CUDA(cudaMemcpyAsync(out->offsets, b.tb.offsets, sizeof(int32_t) * (m.E + 1), kind, st));
+    if (out->row_of_slot && out->row_of_slot != b.tb.row_of_slot)
         BIGMAC_CUDA(cudaMemcpyAsync(out->row_of_slot, b.tb.row_of_slot, sizeof(int32_t) * m.N, kind, st));
-    if (out->slot_of_row)
+    if (out->slot_of_row && out->slot_of_row != b.tb.slot_of_row)
         BIGMAC_CUDA(cudaMemcpyAsync(out->slot_of_row, b.tb.slot_of_row, sizeof(int32_t) * m.N, kind, st));
-    if (out->counts_chosen)
+    if (out->counts_chosen && out->counts_chosen != b.tb.counts_chosen)
         BIGMAC_CUDA(cudaMemcpyAsync(out->counts_chosen, b.tb.counts_chosen, sizeof(int32_t) * m.E, kind, st));
     if (out->aux_loss) {
-        if (m.aux > 0) BIGMAC_CUDA(cudaMemcpyAsync(out->aux_loss, b.aux_loss, sizeof(float), kind, st));
-        else BIGMAC_CUDA(cudaMemsetAsync(out->aux_loss, 0, sizeof(float), st));
+        if (m.aux <= 0) BIGMAC_CUDA(cudaMemsetAsync(out->aux_loss, 0, sizeof(float), st));
+        else if (out->aux_loss != b.aux_loss) BIGMAC_CUDA(cudaMemcpyAsync(out->aux_loss, b.aux_loss, sizeof(float), kind, st));
     }
     return BIGMAC_OK;
 }
@@ -240,7 +266,7 @@ int check_call(const bigmac_layer* L, int32_t T) {
 // Per-expert weight gradient (contraction over the expert's rows): on the tensor-core path the balanced kernel
 // (dynamic work items, long experts in parts), else the generic grouped contraction.
 int expert_weight_grad(const bigmac_layer* L, int id, const GemmArgs& g, float* splitk_ws, cudaStream_t st) {
-    static const bool enabled = []() { const char* e = std::getenv("BIGMAC_GROUPK"); return !(e && e[0] == '0'); }();
+    const bool enabled = switches().groupk != 0;
     const bool tc = L->cfg.dtype == BIGMAC_BF16 && L->use_tc && ((L->tc_mask >> id) & 1u);
     // below about 16 k slices of work per CTA pair the items are too short for dynamic hand-out to pay (measured:
     // +10 us per launch at 1024 tokens of the medium shape, -31 % at 16384 tokens with Zipf loads)
@@ -286,8 +312,7 @@ int bigmac_layer_create(const bigmac_config_t* cfg, bigmac_layer_t** out) {
     if (!L) return BIGMAC_ERR_CUDA;
     L->cfg = *cfg;
     L->use_tc = cfg->dtype == BIGMAC_BF16 && !(cfg->flags & BIGMAC_FLAG_SIMT_GEMM);
-    L->tc_mask = ~0u;
-    if (const char* env = std::getenv("BIGMAC_TC_MASK")) L->tc_mask = (unsigned)std::strtoul(env, nullptr, 0);
+    L->tc_mask = switches().tc_mask;
     if (cudaGetDevice(&L->device) != cudaSuccess || cudaMalloc((void**)&L->status, 4 * sizeof(int)) != cudaSuccess ||
         cudaMemset(L->status, 0, 4 * sizeof(int)) != cudaSuccess) {
         delete L;
@@ -350,6 +375,7 @@ int bigmac_route(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_weigh
     Buffers b{};
     carve_route_scratch(cv, m, b);
     carve_saved(cv, m, b, false);
+    alias_routing(b, out);
     cudaStream_t st = (cudaStream_t)stream;
     BIGMAC_TRY(run_routing(L, m, x, W, b, st));
     return export_routing(m, b, out, st);
@@ -374,6 +400,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         carve_saved(cv, m, b, true);
     } else {
         carve_saved(cs, m, b, false);
+        alias_routing(b, routing_out);
     }
     cudaStream_t st = (cudaStream_t)stream;
     const bigmac_config_t& c = L->cfg;
@@ -387,7 +414,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
                                               m.k, c.act, gemm_tc_sm_count(), st));
         }
         if (routing_out) {
-            { Stage s(L, S_TABLES, st, tables_kernel_count(m.N, m.E)); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st)); }
+            { Stage s(L, S_TABLES, st, tables_kernel_count(m.N, m.E)); BIGMAC_CUDA(launch_tables(b.tb, m.T, m.E, m.k, m.cap, st, L->status)); }
             BIGMAC_TRY(export_routing(m, b, routing_out, st));
         }
         return BIGMAC_OK;
@@ -417,8 +444,8 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     // Inference, low width r <= 256, up to two row tiles per SM: F6 + F7 in one kernel, the hidden activations stay on
     // the SM.  On long tile lists the two separate GEMMs are faster (the fused kernel is bound by the issue of its many
     // narrow MMA instructions): measured 0.375 vs 0.329 ms forward at the medium workload, 0.099 vs 0.106 ms at 512
-    // decode tokens.  BIGMAC_FUSED_MLP=0 / =2 force it off / on.
-    static const int fuse_mlp_mode = []() { const char* e = std::getenv("BIGMAC_FUSED_MLP"); return e ? atoi(e) : 1; }();
+    // decode tokens.  The fused_mlp debug switch forces it off (0) / on (2).
+    const int fuse_mlp_mode = switches().fused_mlp;
     const bool short_list = m.P / kPad <= 2 * (int64_t)gemm_tc_sm_count();
     if (!training && !m.bias && (fuse_mlp_mode == 2 || (fuse_mlp_mode == 1 && short_list)) && sigma_as_bytes(L) &&
         fused_mlp_supported(m.r, m.h, m.dtype)) {
@@ -455,9 +482,26 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     return BIGMAC_OK;
 }
 
+static int backward_launches(bigmac_layer_t* L, const void* x, const void* dy, int32_t T, const bigmac_weights_t* W,
+                             void* saved, void* dx, const bigmac_grads_t* G, int accumulate, void* scratch,
+                             size_t scratch_bytes, void* stream);
+
 int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T, const bigmac_weights_t* W,
                     void* saved, void* dx, const bigmac_grads_t* G, int accumulate, void* scratch,
                     size_t scratch_bytes, void* stream) {
+    if (L) L->side_forked = false;
+    const int rc = backward_launches(L, x, dy, T, W, saved, dx, G, accumulate, scratch, scratch_bytes, stream);
+    if (rc != BIGMAC_OK && L && L->side_forked) {
+        // a launch failed after work was forked to the second stream: join it, so that the caller's stream (and a
+        // capture in progress) is not left with an open fork and nothing of this call outlives its return unordered
+        if (cudaEventRecord(L->fork_join[9], L->side) == cudaSuccess) cudaStreamWaitEvent((cudaStream_t)stream, L->fork_join[9], 0);
+    }
+    return rc;
+}
+
+static int backward_launches(bigmac_layer_t* L, const void* x, const void* dy, int32_t T, const bigmac_weights_t* W,
+                             void* saved, void* dx, const bigmac_grads_t* G, int accumulate, void* scratch,
+                             size_t scratch_bytes, void* stream) {
     BIGMAC_TRY(check_call(L, T));
     BIGMAC_TRY(check_weights(L, W));
     if (!G) return BIGMAC_ERR_INVALID_ARG;
@@ -468,6 +512,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     if (!aligned(G->dw_gate, 16) || !aligned(G->dw_down, 16) || !aligned(G->dw1, 16) || !aligned(G->dw2, 16) ||
         !aligned(G->dw_up, 16) || !aligned(G->db_gate, 4))
         return BIGMAC_ERR_INVALID_ARG;
+    if ((L->cfg.flags & BIGMAC_FLAG_EXPERT_BIAS) && (!aligned(G->db1, 4) || !aligned(G->db2, 4))) return BIGMAC_ERR_INVALID_ARG;
     const Dims m = dims_of(L, T);
     if (scratch_bytes < backward_scratch_bytes(m)) return BIGMAC_ERR_WORKSPACE;
     Buffers b{};
@@ -481,10 +526,10 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     const bigmac_config_t& c = L->cfg;
     const bool acc = accumulate != 0;
 
-    // Overlap (BIGMAC_OVERLAP=0 turns it off): dW_up, the gate backward with the bias-gradient column sums, the dx' gather
+    // Overlap (the overlap debug switch turns it off): dW_up, the gate backward with the bias-gradient column sums, the dx' gather
     // and [dW_down ; dW_gate] go to a second stream, forked from and joined back into the caller's stream with events, so that they run beside launches they
     // do not depend on.  Everything that shares the fp32 workspace stays ordered.
-    static const bool overlap_on = []() { const char* e = std::getenv("BIGMAC_OVERLAP"); return !(e && e[0] == '0'); }();
+    const bool overlap_on = switches().overlap != 0;
     // (not while per-stage events are recorded: a stage timed beside another stream's launches would not be its own time)
     const bool overlap = overlap_on && L->side && !L->prof_on && !m.cdac;
     cudaStream_t sd = st;
@@ -492,6 +537,7 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
         sd = L->side;
         BIGMAC_CUDA(cudaEventRecord(L->fork_join[0], st));
         BIGMAC_CUDA(cudaStreamWaitEvent(sd, L->fork_join[0], 0));
+        L->side_forked = true;
     }
     if (m.cdac) b.dy_lo = const_cast<void*>(dy);
     if (!m.cdac) {   // dy' = dy W_up                                   [T,d] x [d,r]
@@ -555,7 +601,6 @@ int bigmac_backward(bigmac_layer_t* L, const void* x, const void* dy, int32_t T,
     void* dz = b.dz ? b.dz : b.z;
     if (overlap) BIGMAC_CUDA(cudaStreamWaitEvent(st, L->fork_join[1], 0));    // from here on the fp32 workspace is used again
     if (m.bias) {   // db1_e = sum_rows dz[row,:], db2_e = sum_rows du[row,:]  (padding rows hold zeros)
-        if (!aligned(G->db1, 4) || !aligned(G->db2, 4)) return BIGMAC_ERR_INVALID_ARG;
         // Two HBM-bound passes over dz and du that nothing later in the pass reads: with the second stream they run
         // beside the tensor-bound dW2 / dxg (joined with the dx' gather), on slice sums in a region of their own.
         cudaStream_t sb = st;
@@ -750,7 +795,7 @@ int bigmac_device_status(bigmac_layer_t* L, void* stream) {
         if (cudaMemsetAsync(L->status + 1, 0, 3 * sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
             return BIGMAC_ERR_CUDA;
     }
-    if (word == 2) return BIGMAC_ERR_STATE;            // an expert-parallel step was given a count matrix that cannot be right
+    if (word == 2) return BIGMAC_ERR_STATE;            // an expert-parallel count matrix that cannot be right, or an expert id outside [0, E)
     return word == 0 ? BIGMAC_OK : BIGMAC_ERR_TIMEOUT;
 }
 
@@ -762,7 +807,7 @@ const char* bigmac_status_string(int status) {
         case BIGMAC_ERR_WORKSPACE: return "workspace too small";
         case BIGMAC_ERR_CUDA: return "CUDA error";
         case BIGMAC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
-        case BIGMAC_ERR_STATE: return "handle used on the wrong device, or an expert-parallel count matrix that cannot be right";
+        case BIGMAC_ERR_STATE: return "handle used on the wrong device, an expert-parallel count matrix that cannot be right, or an expert id outside [0, E) in the routing tables";
         case BIGMAC_ERR_TOO_LARGE: return "problem exceeds the fixed scratch array of bigmac_route_static";
         default: return "unknown status";
     }
@@ -861,6 +906,7 @@ int bigmac_route_static(bigmac_layer_t* L, const void* x, int32_t T, const bigma
     Carver cv(base);
     Buffers b{};
     carve_route_only(cv, m, b);
+    alias_routing(b, out);
     cudaStream_t st = (cudaStream_t)stream;
     BIGMAC_TRY(run_routing(L, m, x, W, b, st));
     return export_routing(m, b, out, st);
@@ -915,6 +961,21 @@ int bigmac_debug_gemm(bigmac_layer_t* L, const bigmac_debug_gemm_t* q, int use_t
     cudaError_t err = use_tensor_cores ? gemm_tc(g, L->status, (cudaStream_t)stream)
                                        : gemm_simt(g, L->cfg.dtype, (cudaStream_t)stream);
     return err == cudaSuccess ? BIGMAC_OK : BIGMAC_ERR_CUDA;
+}
+
+int bigmac_debug_set(const char* name, int value) {
+    if (!name) return BIGMAC_ERR_INVALID_ARG;
+    Switches& sw = switches();
+    if (!std::strcmp(name, "overlap")) sw.overlap = value;
+    else if (!std::strcmp(name, "tc_pair")) sw.tc_pair = value;
+    else if (!std::strcmp(name, "groupk")) sw.groupk = value;
+    else if (!std::strcmp(name, "fused_mlp")) sw.fused_mlp = value;
+    else if (!std::strcmp(name, "epi_parts")) sw.epi_parts = value;
+    else if (!std::strcmp(name, "fuse_dispatch")) sw.fuse_dispatch = value;
+    else if (!std::strcmp(name, "tc_mask")) sw.tc_mask = (unsigned)value;
+    else if (!std::strcmp(name, "defaults")) sw = Switches();
+    else return BIGMAC_ERR_INVALID_ARG;
+    return BIGMAC_OK;
 }
 
 int bigmac_debug_expire_wait(bigmac_layer_t* L, void* stream) {

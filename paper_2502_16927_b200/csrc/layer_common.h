@@ -14,11 +14,12 @@ struct bigmac_layer {
     int* status;        // device status word; status[1] is the grid-barrier counter of the small-batch kernel,
                         // status[2..3] the work counters of the per-expert weight-gradient kernel (zero at rest)
     bool use_tc;        // bf16 contractions on tcgen05
-    unsigned tc_mask;   // debug: bit i set = contraction i runs on tcgen05 (BIGMAC_TC_MASK)
+    unsigned tc_mask;   // debug: bit i set = contraction i runs on tcgen05 (the tc_mask switch at creation)
     // second stream of the backward pass (created on first use): launches that do not depend on each other and lean
     // on different units (a tensor-bound weight gradient beside an HBM-bound row move) run side by side
     cudaStream_t side = nullptr;
-    cudaEvent_t fork_join[9] = {};
+    cudaEvent_t fork_join[10] = {};     // [9]: joins the second stream back when a call fails after its fork
+    bool side_forked = false;          // the running bigmac_backward has put work on `side`
     // measurement aid
     bool prof_on = false;
     uint64_t launches = 0;

@@ -94,8 +94,9 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
         for (int i = 0; i < V; ++i) acc[i] = 0.0f;
         for (int j = 0; j < k; ++j) {                      // slot order: fixed summation order
             const int64_t s = (int64_t)t * k + j;
-            const int prow = prow_of_slot[s];
+            int prow = prow_of_slot[s];
             if (MAY_DROP && prow < 0) continue;             // dropped under a capacity limit: absent from the sum
+            if (!MAY_DROP) prow = max(prow, 0);             // dropless rows are never negative; keeps the address in range if one were
             const float p = w ? w[s] : 1.0f;
             float f[V];
             Vec<T>::unpack(grouped[(int64_t)prow * vecs_per_row + c], f);
@@ -160,7 +161,8 @@ __global__ void __launch_bounds__(256) gate_bwd_kernel(float* __restrict__ dp, c
     __syncwarp();
     for (int j = lane; j < k; j += 32) {
         const float dl = p[j] * (g[j] - part);
-        row[topk_idx[(int64_t)t * k + j]] = (T)dl;
+        const int e = topk_idx[(int64_t)t * k + j];
+        if ((unsigned)e < (unsigned)E) row[e] = (T)dl;
         g[j] = dl;                                   // fp32 copy per slot, for the bias gradient
     }
 }

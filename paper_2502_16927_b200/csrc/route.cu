@@ -8,11 +8,15 @@ namespace bigmac {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kNoExpert = 0x7fffffff;          // "no candidate yet" in the arg-max rounds; never written out
 
 // One warp per token.  Lane l holds experts l, l+32, ...  k rounds of warp arg-max under the order
 // (logit descending, expert id ascending); gate values are the softmax over the k winners.
 // KREG: k <= 32, the j-th winner stays in a register of lane j until one coalesced store at the end; otherwise
 // the winners pass through the output arrays.
+// Non-finite logits: NaN is ordered as -inf, and a round that finds only -inf among the experts not yet chosen takes
+// the lowest such id, so every id written lies in [0, E) whatever the logits hold (k <= E).  A token whose kept
+// logits are all -inf gets the gate value 1/k on each.
 template <int VPL, bool KREG>
 __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ logits, const float* __restrict__ b_gate,
                                                    int T, int E, int k, int32_t* __restrict__ topk_idx,
@@ -25,19 +29,21 @@ __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ log
 #pragma unroll
     for (int i = 0; i < VPL; ++i) {
         const int e = lane + 32 * i;
-        v[i] = e < E ? row[e] + (b_gate ? b_gate[e] : 0.0f) : -INFINITY;
+        const float x = e < E ? row[e] + (b_gate ? b_gate[e] : 0.0f) : -INFINITY;
+        v[i] = x == x ? x : -INFINITY;             // NaN is ordered as -inf
     }
     int32_t* out_idx = topk_idx + (size_t)t * k;
     float* out_w = topk_w + (size_t)t * k;
     float my_v = -INFINITY;
     int my_e = 0;
+    uint32_t taken = 0;                            // bit i: expert lane + 32 i already chosen
     for (int j = 0; j < k; ++j) {
         float best = -INFINITY;
-        int best_e = 0x7fffffff;
+        int best_e = kNoExpert;
 #pragma unroll
         for (int i = 0; i < VPL; ++i) {            // ascending expert id within the lane: strict > keeps the lowest id
             const int e = lane + 32 * i;
-            if (e < E && v[i] > best) { best = v[i]; best_e = e; }
+            if (e < E && !((taken >> i) & 1u) && (best_e == kNoExpert || v[i] > best)) { best = v[i]; best_e = e; }
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
@@ -45,11 +51,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ log
             const int oe = __shfl_xor_sync(kFull, best_e, off);
             if (ov > best || (ov == best && oe < best_e)) { best = ov; best_e = oe; }
         }
-        if ((best_e & 31) == lane) {
-#pragma unroll
-            for (int i = 0; i < VPL; ++i)
-                if (lane + 32 * i == best_e) v[i] = -INFINITY;
-        }
+        if (best_e != kNoExpert && (best_e & 31) == lane) taken |= 1u << (best_e >> 5);
         if (KREG) {
             if (lane == j) { my_v = best; my_e = best_e; }
         } else if (lane == 0) {
@@ -59,7 +61,7 @@ __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ log
     }
     if (KREG) {
         const float top = __shfl_sync(kFull, my_v, 0);
-        const float ex = lane < k ? expf(my_v - top) : 0.0f;
+        const float ex = lane < k ? (top == -INFINITY ? 1.0f : expf(my_v - top)) : 0.0f;
         float part = ex;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
@@ -71,11 +73,12 @@ __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ log
     }
     __syncwarp();
     const float top = out_w[0];
+    const bool none = top == -INFINITY;
     float part = 0.0f;
-    for (int j = lane; j < k; j += 32) part += expf(out_w[j] - top);
+    for (int j = lane; j < k; j += 32) part += none ? 1.0f : expf(out_w[j] - top);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
-    for (int j = lane; j < k; j += 32) out_w[j] = expf(out_w[j] - top) / part;
+    for (int j = lane; j < k; j += 32) out_w[j] = (none ? 1.0f : expf(out_w[j] - top)) / part;
 }
 
 // Four tokens per warp, eight lanes per token, for k <= 8 and E a multiple of 32 up to 256: lane l of a group
@@ -100,15 +103,18 @@ __global__ void __launch_bounds__(256) topk8_kernel(const float* __restrict__ lo
         }
         v[4 * i] = x.x; v[4 * i + 1] = x.y; v[4 * i + 2] = x.z; v[4 * i + 3] = x.w;
     }
+#pragma unroll
+    for (int i = 0; i < 4 * Q; ++i) v[i] = v[i] == v[i] ? v[i] : -INFINITY;     // NaN is ordered as -inf
     float my_v = -INFINITY;
     int my_e = 0;
+    uint32_t taken = 0;                            // bit i: this lane's i-th expert already chosen
     for (int j = 0; j < k; ++j) {
         float best = -INFINITY;
-        int best_e = 0x7fffffff;
+        int best_e = kNoExpert;
 #pragma unroll
         for (int i = 0; i < 4 * Q; ++i) {          // ascending expert id within the lane: strict > keeps the lowest id
             const int e = 4 * (sub + 8 * (i >> 2)) + (i & 3);
-            if (v[i] > best) { best = v[i]; best_e = e; }
+            if (!((taken >> i) & 1u) && (best_e == kNoExpert || v[i] > best)) { best = v[i]; best_e = e; }
         }
 #pragma unroll
         for (int off = 4; off > 0; off >>= 1) {
@@ -118,11 +124,11 @@ __global__ void __launch_bounds__(256) topk8_kernel(const float* __restrict__ lo
         }
 #pragma unroll
         for (int i = 0; i < 4 * Q; ++i)
-            if (4 * (sub + 8 * (i >> 2)) + (i & 3) == best_e) v[i] = -INFINITY;
+            if (4 * (sub + 8 * (i >> 2)) + (i & 3) == best_e) taken |= 1u << i;
         if (sub == j) { my_v = best; my_e = best_e; }
     }
     const float top = __shfl_sync(kFull, my_v, lane & 24);
-    const float ex = sub < k ? expf(my_v - top) : 0.0f;
+    const float ex = sub < k ? (top == -INFINITY ? 1.0f : expf(my_v - top)) : 0.0f;
     float part = ex;
 #pragma unroll
     for (int off = 4; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
@@ -147,7 +153,8 @@ __global__ void __launch_bounds__(256) sort_local_kernel(const int32_t* __restri
 #pragma unroll
     for (int it = 0; it < kSortChunk / 256; ++it) {
         const int64_t s = base + it * 32 + lane;
-        const int e = s < N ? topk_idx[s] : -1;
+        int e = s < N ? topk_idx[s] : -1;
+        if ((unsigned)e >= (unsigned)E) e = -1;      // an id outside [0, E) (never written by the top-k kernels) counts nowhere
         const unsigned peers = __match_any_sync(kFull, e);
         const int leader = __ffs(peers) - 1;
         int old = 0;
@@ -173,7 +180,9 @@ __global__ void __launch_bounds__(256) sort_local_kernel(const int32_t* __restri
 #pragma unroll
     for (int it = 0; it < kSortChunk / 256; ++it) {
         const int64_t s = base + it * 32 + lane;
-        if (s < N) local_rank[s] = warp_run[warp * E + topk_idx[s]] + my_rank[it];
+        if (s >= N) continue;
+        const int e = topk_idx[s];
+        local_rank[s] = (unsigned)e < (unsigned)E ? warp_run[warp * E + e] + my_rank[it] : 0;
     }
 }
 
@@ -266,10 +275,17 @@ __global__ void __launch_bounds__(256) sort_place_kernel(const int32_t* __restri
                                                          int32_t* __restrict__ prow_of_slot /* in: local rank */,
                                                          int32_t* __restrict__ row_of_slot,
                                                          int32_t* __restrict__ slot_of_row,
-                                                         int32_t* __restrict__ slot_of_prow, int cap) {
+                                                         int32_t* __restrict__ slot_of_prow, int cap,
+                                                         int* __restrict__ status) {
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= N) return;
     const int e = topk_idx[s];
+    if ((unsigned)e >= (unsigned)E) {               // second line of defence: the slot goes nowhere, the call reports it
+        row_of_slot[s] = -1;
+        prow_of_slot[s] = -1;
+        if (status) atomicExch(status, 2);
+        return;
+    }
     const int within = block_base[(size_t)(s / kSortChunk) * E + e] + prow_of_slot[s];
     if (within >= cap) {
         row_of_slot[s] = -1;
@@ -293,7 +309,8 @@ __global__ void __launch_bounds__(1024) tables_small_kernel(const int32_t* __res
                                                             int32_t* __restrict__ offsets, int32_t* __restrict__ poffsets,
                                                             int32_t* __restrict__ tile_expert, int32_t* __restrict__ n_tiles,
                                                             int32_t* __restrict__ prow_of_slot, int32_t* __restrict__ row_of_slot,
-                                                            int32_t* __restrict__ slot_of_row, int32_t* __restrict__ slot_of_prow) {
+                                                            int32_t* __restrict__ slot_of_row, int32_t* __restrict__ slot_of_prow,
+                                                            int* __restrict__ status) {
     extern __shared__ int32_t sm[];                  // [32][E] per-warp counts of the chunk, [E] totals so far, 2 x [E+1]: 35 E + 2 ints
     int32_t* warp_run = sm;
     int32_t* total = sm + 32 * E;
@@ -312,7 +329,8 @@ __global__ void __launch_bounds__(1024) tables_small_kernel(const int32_t* __res
         for (int i = threadIdx.x; i < 32 * E; i += blockDim.x) warp_run[i] = 0;
         __syncthreads();
         const int s = c * 1024 + threadIdx.x;
-        const int e = s < N ? topk_idx[s] : -1;
+        int e = s < N ? topk_idx[s] : -1;
+        if ((unsigned)e >= (unsigned)E) e = -1;      // an id outside [0, E) counts nowhere
         const unsigned peers = __match_any_sync(kFull, e);
         if (e >= 0 && lane == __ffs(peers) - 1) warp_run[warp * E + e] = __popc(peers);
         const int in_warp = __popc(peers & ((1u << lane) - 1u));
@@ -356,7 +374,9 @@ __global__ void __launch_bounds__(1024) tables_small_kernel(const int32_t* __res
         const int s = c * 1024 + threadIdx.x;
         if (s >= N) continue;
         const int e = topk_idx[s], within = rank_of[c];
-        if (within >= cap) {
+        const bool bad = (unsigned)e >= (unsigned)E;
+        if (bad && status) atomicExch(status, 2);
+        if (bad || within >= cap) {
             row_of_slot[s] = -1;
             prow_of_slot[s] = -1;
             continue;
@@ -406,13 +426,13 @@ cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, 
     return cudaGetLastError();
 }
 
-cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaStream_t stream) {
+cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaStream_t stream, int* status) {
     const int64_t N = (int64_t)T * k;
     const int64_t P = padded_rows_max(N, E);
     if (tables_kernel_count(N, E) == 1) {
         tables_small_kernel<<<1, 1024, sizeof(int32_t) * (35 * E + 2), stream>>>(
             tb.topk_idx, (int)N, E, cap, (int)P, tb.counts, tb.counts_chosen, tb.offsets, tb.poffsets, tb.tile_expert, tb.n_tiles,
-            tb.prow_of_slot, tb.row_of_slot, tb.slot_of_row, tb.slot_of_prow);
+            tb.prow_of_slot, tb.row_of_slot, tb.slot_of_row, tb.slot_of_prow, status);
         return cudaGetLastError();
     }
     cudaError_t err = cudaMemsetAsync(tb.slot_of_prow, 0xff, sizeof(int32_t) * P, stream);
@@ -431,7 +451,7 @@ cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaSt
         sort_place_kernel<<<(unsigned)((N + 255) / 256), 256, 0, stream>>>(tb.topk_idx, N, E, tb.block_counts,
                                                                           tb.offsets, tb.poffsets, tb.prow_of_slot,
                                                                           tb.row_of_slot, tb.slot_of_row,
-                                                                          tb.slot_of_prow, cap);
+                                                                          tb.slot_of_prow, cap, status);
     return cudaGetLastError();
 }
 

@@ -1,0 +1,19 @@
+// Process-wide measurement and debugging switches of libbigmac.  The defaults are the product; they change only
+// through bigmac_debug_set (bigmac_debug.h).  The library never reads the environment.
+#pragma once
+
+namespace bigmac {
+
+struct Switches {
+    int overlap = 1;        // backward pass: independent launches on the handle's second stream (0: one stream)
+    int tc_pair = 1;        // CTA-pair tcgen05 kernel where it is the faster one (0: one-CTA kernel everywhere)
+    int groupk = 1;         // dynamically scheduled per-expert weight-gradient kernel where it pays (0: never)
+    int fused_mlp = 1;      // inference: expert GEMM1 + sigma + GEMM2 in one kernel on short tile lists (0: never, 2: always)
+    int epi_parts = 0;      // working epilogue warps per lane quadrant of plain epilogues (1, 2, 4; 0: the default, 2)
+    int fuse_dispatch = 1;  // expert GEMM1 gathers its rows from x' itself where supported (0: standalone dispatch kernel)
+    unsigned tc_mask = ~0u; // bit i: contraction i runs on tcgen05 (read when a handle is created)
+};
+
+Switches& switches();
+
+}  // namespace bigmac

@@ -7,6 +7,7 @@
 
 #include "internal.h"
 #include "act.cuh"
+#include "switches.h"
 
 namespace bigmac {
 namespace tc {
@@ -581,10 +582,10 @@ constexpr int kThreadsV2 = (2 + kEpiWarps) * 32;
 
 
 // ------------------------------------------------------------------------------------------ host side
-// Working epilogue warps per lane quadrant for plain epilogues: the request, else BIGMAC_EPI_PARTS, else 2.
+// Working epilogue warps per lane quadrant for plain epilogues: the request, else the debug switch, else 2.
 inline int epi_parts_default(int requested) {
-    static const int env = []() { const char* e = std::getenv("BIGMAC_EPI_PARTS"); return e ? atoi(e) : 0; }();
-    const int v = requested ? requested : env ? env : 2;
+    const int sw = switches().epi_parts;
+    const int v = requested ? requested : sw ? sw : 2;
     return (v == 1 || v == 2) ? v : 4;
 }
 

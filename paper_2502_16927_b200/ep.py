@@ -226,7 +226,53 @@ class EpLocalGroup:
 
 # ---- one rank per process ------------------------------------------------------------------------------------------
 
-class EpProcessRank:
+class EpStepOrder:
+    """Order of the phase calls of one step and of the barriers between them, for one rank per process (Fig. 2c):
+
+        route | all-gather of counts | dispatch | experts | combine
+        backward_combine | backward_experts | backward_dispatch | (sum of the shared gradients)
+
+    "|" is a barrier over all ranks' streams: what follows reads rows that peers wrote in what precedes (experts read
+    the rows every rank put; combine gets the outputs of every owner; ...).  The all-gather doubles as the barrier
+    that orders a step after the previous one.  A subclass provides `rk` (the phase calls of this rank), `barrier()`,
+    `gather()` (fill every row of the count matrix) and `reduce(G)` (sum the shared matrices' gradients)."""
+
+    rk = None
+
+    def barrier(self):
+        raise NotImplementedError
+
+    def gather(self):
+        raise NotImplementedError
+
+    def reduce(self, G):
+        raise NotImplementedError
+
+    def forward(self, x, W, y=None, routing=None):
+        y = torch.empty_like(x) if y is None else y
+        self.rk.route(x, W, routing)
+        self.gather()                                # also orders this step after the last one
+        self.rk.dispatch()
+        self.barrier()
+        self.rk.experts(W)
+        self.barrier()
+        self.rk.combine(W, y)
+        return y
+
+    def backward(self, x, dy, W, G, dx=None, accumulate=False, reduce_shared=True):
+        dx = torch.empty_like(x) if dx is None else dx
+        self.barrier()
+        self.rk.backward_combine(dy, W, G, accumulate)
+        self.barrier()
+        self.rk.backward_experts(W, G, accumulate)
+        self.barrier()
+        self.rk.backward_dispatch(x, W, dx, G, accumulate)
+        if reduce_shared:
+            self.reduce(G)
+        return dx
+
+
+class EpProcessRank(EpStepOrder):
     """This process's rank of a torch.distributed group (NCCL): exchange buffers in symmetric memory, so that every
     rank can address every other rank's; counts by all_gather; barriers as one-element all_reduces on the ranks'
     streams.  Plain peer loads and stores only."""
@@ -256,28 +302,11 @@ class EpProcessRank:
 
         dist.all_reduce(self._flag, group=self.group)
 
-    def forward(self, x, W, y=None, routing=None):
-        y = torch.empty_like(x) if y is None else y
-        self.rk.route(x, W, routing)
-        gather_counts(self.rk.counts_all, self.rk.rank, self.group)     # also orders this step after the last one
-        self.rk.dispatch()
-        self.barrier()
-        self.rk.experts(W)
-        self.barrier()
-        self.rk.combine(W, y)
-        return y
+    def gather(self):
+        gather_counts(self.rk.counts_all, self.rk.rank, self.group)
 
-    def backward(self, x, dy, W, G, dx=None, accumulate=False, reduce_shared=True):
-        dx = torch.empty_like(x) if dx is None else dx
-        self.barrier()
-        self.rk.backward_combine(dy, W, G, accumulate)
-        self.barrier()
-        self.rk.backward_experts(W, G, accumulate)
-        self.barrier()
-        self.rk.backward_dispatch(x, W, dx, G, accumulate)
-        if reduce_shared:
-            reduce_shared_grads(G, self.group)
-        return dx
+    def reduce(self, G):
+        reduce_shared_grads(G, self.group)
 
     def status(self) -> int:
         return self.rk.status()

@@ -222,5 +222,5 @@ def test_a_count_matrix_that_cannot_be_right_is_refused_on_the_device(bad):
     assert group.status() == 0
     rt = oracle.route(inp, w.k)
     ref = oracle.forward_tokens(inp, rt, w.act)["y"]
-    assert oracle.rel_err(np.concatenate([to_numpy(v) for v in got_y]), ref) <= TOL[w.dtype]
+    assert_within(w, float_errors(w, {"y": np.concatenate([to_numpy(v) for v in got_y])}, {"y": ref}))
     group.close()

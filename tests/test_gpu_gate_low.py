@@ -45,6 +45,7 @@ def compare(w, inp, got, capacity_factor=0.0):
             if key in keys:
                 assert outlier_fraction(got[key], ref[key], TOL[w.dtype]) <= 1e-3, key
                 errs.pop(key)
+                errs.pop(key + ":rms")
     assert_within(w, errs)
 
 
@@ -90,7 +91,7 @@ def test_gate_on_the_low_width_token_with_a_capacity_limit_and_the_other_entry_p
     assert layer.status() == 0
     for tables in (R, R2, R3):
         check_routing(tables, rt)
-    assert oracle.rel_err(to_numpy(y), ref) <= TOL[w.dtype]
+    assert_within(w, float_errors(w, {"y": to_numpy(y)}, {"y": ref}))
     layer.close()
 
 

@@ -1,12 +1,18 @@
 """GPU parity: the CUDA layer, called through the C ABI, against the CPU oracle on the same seeded
-inputs.  Integer tables must match bit for bit.  Floats:
+inputs.  Integer tables must match bit for bit.  Floats, per output tensor:
   fp32 path  max_i |a_i-b_i| / max(|b_i|, rms(b)) <= 1e-4   (every element, denominator floored at the RMS);
-  BF16 path  max_i |a_i-b_i| / max_i |b_i| <= 2e-2  and  ||a-b||_F / ||b||_F <= 2e-2.
+  BF16 path  max_i |a_i-b_i| / max_i |b_i| <= 1e-2,  ||a-b||_F / ||b||_F <= 8e-3,  and the RMS-floored metric of
+             the fp32 path <= 6e-2 (per expert for the stacked per-expert gradients).
 The BF16 layer stores five (forward) to eight (gradients) intermediates per output in bf16 (unit roundoff
 2^-8): each storage adds noise of about 0.165 % of the tensor's RMS, so the extreme element of 10^6..10^8
 outputs sits at 2-2.5 % of the RMS even with exact accumulation (test_precision_model.py shows this with an
-emulation), which is why the BF16 bound is taken relative to the largest magnitude and backed by the
-Frobenius bound rather than floored at the RMS."""
+emulation: per-element noise of 0.47 % of the RMS after eight storages, whose extreme over 10^8 elements lies near
+seven standard deviations), and where the rows of a tensor differ in scale (skewed routing, dropped slots) the
+storage noise of the large rows reaches elements that sit at the floor: measured up to 5.0e-2 (dx under a capacity
+limit), so the RMS-floored metric is reported and bounded at 6e-2 only, and the two bounds
+that do the discriminating are set at about twice what the kernels deliver: the largest error relative to the
+largest magnitude (measured 0.35-0.5 %) and the Frobenius error (measured 0.35-0.6 %), so that an error of a
+few per cent of the RMS in isolated elements, or a per-cent-level systematic one, fails."""
 import numpy as np
 import pytest
 
@@ -18,7 +24,15 @@ from helpers import oracle_inputs, empty_grads, make_layer, to_device, to_numpy
 
 pytestmark = pytest.mark.gpu
 
-TOL = {wl.DTYPE_F32: 1e-4, wl.DTYPE_BF16: 2e-2}
+BF16_MAX, BF16_FRO, BF16_RMS = 1e-2, 8e-3, 6e-2
+# Tensors with bounds of their own (max-norm, Frobenius), measured worst values in brackets:
+#   dw1, dw2   a per-expert gradient is a sum over that expert's rows only; with a handful of rows (the sampled
+#              full-size checks, nearly empty experts) the storage error of the terms does not average out and the
+#              largest elements carry it whole (0.92 % of max|b| at the large workload, Frobenius 0.48 %);
+#   db_gate    a sum of terms of both signs that cancels to a small difference of large parts under skewed routing;
+#              the bf16 storage of dy' and u behind every term is then a larger share of the result (1.6 % / 1.0 %).
+BF16_OWN = {"dw1": (1.5e-2, BF16_FRO), "dw2": (1.5e-2, BF16_FRO), "db_gate": (2e-2, 1.5e-2)}
+TOL = {wl.DTYPE_F32: 1e-4, wl.DTYPE_BF16: BF16_MAX}
 SIMT = 1
 
 
@@ -56,7 +70,8 @@ def run_full(w, inp, flags=0, capacity_factor=0.0, aux=0.0):
 
 
 def float_errors(w, got, ref):
-    """Per output tensor: the gate metric of the workload's dtype (and the Frobenius error for BF16)."""
+    """Per output tensor: the gate metric of the workload's dtype; for BF16 also the Frobenius error (":fro") and the
+    RMS-floored elementwise metric (":rms")."""
     metric = oracle.rel_err if w.dtype == wl.DTYPE_F32 else oracle.max_rel_err
     out = {}
     for key in got:
@@ -64,13 +79,44 @@ def float_errors(w, got, ref):
             out[key] = metric(got[key], ref[key])
             if w.dtype == wl.DTYPE_BF16:
                 out[key + ":fro"] = oracle.fro_rel_err(got[key], ref[key])
+                a, b = np.asarray(got[key]), np.asarray(ref[key])
+                if key in ("dw1", "dw2") and b.ndim == 3:      # one RMS floor per expert: their scales differ with their loads
+                    out[key + ":rms"] = max(oracle.rel_err(a[e], b[e]) for e in range(b.shape[0]))
+                else:
+                    out[key + ":rms"] = oracle.rel_err(a, b)
     return out
 
 
+def tolerance_of(w, key):
+    if w.dtype == wl.DTYPE_F32:
+        return TOL[wl.DTYPE_F32]
+    base, _, suffix = key.partition(":")
+    own_max, own_fro = BF16_OWN.get(base, (BF16_MAX, BF16_FRO))
+    return own_fro if suffix == "fro" else BF16_RMS if suffix == "rms" else own_max
+
+
 def assert_within(w, errs):
-    tol = TOL[w.dtype]
-    bad = {key: val for key, val in errs.items() if not val <= tol}
+    record_errors(w, errs)
+    bad = {key: val for key, val in errs.items() if not val <= tolerance_of(w, key)}
     assert not bad, (bad, errs)
+
+
+# Worst value of every metric seen per workload name during the run, written next to the test log so that the
+# measured margins can be quoted (tests never read it back).
+_WORST = {}
+
+
+def record_errors(w, errs):
+    import json
+    import os
+
+    slot = _WORST.setdefault(w.name, {})
+    for key, val in errs.items():
+        slot[key] = max(slot.get(key, 0.0), float(val))
+    out = os.environ.get("BIGMAC_ERROR_REPORT")
+    if out:
+        with open(out, "w") as f:
+            json.dump(_WORST, f, indent=1, sort_keys=True)
 
 
 def outlier_fraction(a, b, tol):
@@ -105,6 +151,7 @@ def compare_full(w, inp, got, tol=None, capacity_factor=0.0, aux=0.0):
                 continue
             assert outlier_fraction(got[key], ref[key], TOL[w.dtype]) <= 1e-3, key
             errs.pop(key)
+            errs.pop(key + ":rms")
     assert_within(w, errs)
     for e in range(w.E):                                   # experts without tokens: exactly zero gradients
         if rt.counts[e] == 0:

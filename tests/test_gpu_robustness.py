@@ -65,7 +65,7 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_handle_usable():
     torch.cuda.synchronize()
     assert layer.status() == 0
     ref = oracle.forward_tokens(inp, oracle.route(inp, w.k), w.act)["y"]
-    assert oracle.max_rel_err(to_numpy(y), ref) <= 2e-2
+    assert oracle.max_rel_err(to_numpy(y), ref) <= 1e-2
     layer.close()
 
 
@@ -186,14 +186,9 @@ def test_expert_parallel_exchange_stays_inside_the_exchange_buffers():
 @pytest.mark.parametrize("variant", [{}, {"gate_low": True}, {"expert_bias": True}], ids=["plain", "gate_low", "expert_bias"])
 def test_backward_on_two_streams_equals_backward_on_one_and_can_be_captured(variant):
     """bigmac_backward forks a few independent launches to the handle's second stream and joins them back: the
-    results are bit for bit those of the one-stream order (run in a child process with BIGMAC_OVERLAP=0), a
+    results are bit for bit those of the one-stream order (the "overlap" debug switch off), a
     captured forward + backward replays to the same bits, and a pass that accumulates adds each gradient once.
     The variants put more on the second stream (the expert-bias column sums) or join it elsewhere (gate on x')."""
-    import os
-    import subprocess
-    import sys
-    import tempfile
-
     import numpy as np
     import torch
 
@@ -241,22 +236,78 @@ def test_backward_on_two_streams_equals_backward_on_one_and_can_be_captured(vari
         assert torch.equal(val.view(torch.uint8), eager[key].view(torch.uint8)), key
     layer.close()
 
-    # one-stream order in a child process: the environment switch is read once per process
-    with tempfile.TemporaryDirectory() as tmp:
-        out = os.path.join(tmp, "one_stream.pt")
-        code = (
-            "import sys, torch; sys.path.insert(0, %r); sys.path.insert(0, %r)\n"
-            "from paper_2502_16927_b200 import workloads as wl\n"
-            "from helpers import empty_grads, make_layer, to_device\n"
-            "from test_gpu_parity import conditioned\n"
-            "variant = %r\n"
-            "w = wl.Workload('ov', T=3000, d=256, r=128, h=256, E=16, k=4, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=167, **variant)\n"
-            "inp = wl.make_inputs(w) if variant else conditioned(w); dev = to_device(w, inp); layer = make_layer(w)\n"
-            "y = layer.forward(dev['x'], dev, training=True); G = empty_grads(w, 'cuda', fill=float('nan'))\n"
-            "dx = layer.backward(dev['x'], dev['dy'], dev, G); torch.cuda.synchronize(); assert layer.status() == 0\n"
-            "torch.save({k: v.cpu() for k, v in dict(G, y=y, dx=dx).items()}, %r)\n"
-        ) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)), variant, out)
-        subprocess.run([sys.executable, "-c", code], check=True, env=dict(os.environ, BIGMAC_OVERLAP="0"), timeout=600)
-        one = torch.load(out)
+    # one-stream order: the same step with the overlap switch off
+    from paper_2502_16927_b200 import binding
+
+    binding.bigmac_debug_set("overlap", 0)
+    try:
+        layer = make_layer(w)
+        y1 = layer.forward(dev["x"], dev, training=True)
+        G1 = empty_grads(w, "cuda", fill=float("nan"))
+        dx1 = layer.backward(dev["x"], dev["dy"], dev, G1)
+        torch.cuda.synchronize()
+        assert layer.status() == 0
+        one = {key: val.cpu() for key, val in dict(G1, y=y1, dx=dx1).items()}
+        layer.close()
+    finally:
+        binding.bigmac_debug_set("defaults")
     for key, val in eager.items():
         assert torch.equal(val.cpu().view(torch.uint8), one[key].view(torch.uint8)), key
+
+
+@pytest.mark.parametrize("case", [
+    dict(dtype=wl.DTYPE_F32, shape=dict(T=200, d=32, r=16, h=24, E=8, k=3)),               # generic top-k kernel
+    dict(dtype=wl.DTYPE_BF16, shape=dict(T=700, d=128, r=64, h=128, E=64, k=8)),            # four-tokens-per-warp kernel, three-pass sort
+    dict(dtype=wl.DTYPE_BF16, shape=dict(T=9, d=128, r=64, h=128, E=32, k=4), decode=True), # one-kernel small-batch forward
+])
+def test_non_finite_logits_keep_every_expert_id_in_range(case):
+    """A NaN token and a gate bias that masks all but k - 1 experts with -inf: every id the routing writes lies in
+    [0, E) (NaN ordered as -inf, lowest id not yet chosen when only -inf is left), the tables equal the oracle's bit
+    for bit, masked experts get the gate value 0, the NaN token 1/k, the status word stays clean and the other tokens'
+    outputs are the oracle's."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from helpers import to_numpy
+    from test_gpu_parity import check_routing
+
+    w = wl.Workload("nf", dtype=case["dtype"], act=wl.ACT_GELU_ERF, seed=151, **case["shape"])
+    inp = wl.make_inputs(w)
+    finite = np.arange(w.E - w.k + 1, w.E)                                   # k - 1 experts stay finite
+    b = np.full(w.E, -np.inf, dtype=np.float32)
+    b[finite] = 40.0 * np.arange(1, finite.size + 1, dtype=np.float32)      # far apart: their order is the bias order
+    inp["b_gate"] = b
+    bad = min(3, w.T - 1)
+    inp["x"][bad, :] = np.nan
+    dev = to_device(w, inp)
+    layer = make_layer(w)
+    if case.get("decode"):
+        y, R = layer.forward(dev["x"], dev, training=False, want_routing=True)
+    else:
+        y, R = layer.forward(dev["x"], dev, training=True, want_routing=True)
+        G = empty_grads(w, "cuda", fill=float("nan"))
+        layer.backward(dev["x"], dev["dy"], dev, G)
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    idx = to_numpy(R["topk_idx"]).reshape(w.T, w.k)
+    assert idx.min() >= 0 and idx.max() < w.E
+    for name in ("row_of_slot", "slot_of_row"):
+        t = to_numpy(R[name])
+        assert t.min() >= 0 and t.max() < w.T * w.k
+    rt = oracle.route(inp, w.k)
+    check_routing(R, rt)
+    p = to_numpy(R["topk_w"]).reshape(w.T, w.k)
+    np.testing.assert_array_equal(idx[bad], np.arange(w.k))                 # the NaN token: lowest ids, equal shares
+    np.testing.assert_allclose(p[bad], 1.0 / w.k, rtol=0, atol=1e-6)
+    good = np.array([t for t in range(w.T) if t != bad])
+    np.testing.assert_array_equal(idx[good, -1], 0)                          # last slot: the lowest masked id, weight 0
+    np.testing.assert_array_equal(p[good, -1], 0.0)
+    got = to_numpy(y)
+    assert np.isnan(got[bad]).all() and not np.isnan(got[good]).any()
+    ref = oracle.forward_tokens(inp, rt, w.act, tokens=good)["y"]
+    if w.dtype == wl.DTYPE_F32:
+        assert oracle.rel_err(got[good], ref) <= 1e-4
+    else:
+        assert oracle.max_rel_err(got[good], ref) <= 1e-2 and oracle.fro_rel_err(got[good], ref) <= 8e-3
+    layer.close()

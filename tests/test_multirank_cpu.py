@@ -121,3 +121,91 @@ def test_expert_parallel_host_side_with_two_ranks():
     assert out[0]["w1_first"] == 0.0 and out[1]["w1_first"] == float(per * 3 * 2)
     for r_ in (0, 1):
         assert out[r_]["dw_gate"] == 3.0 and out[r_]["db_gate"] == 3.0 and out[r_]["dw1"] == 7.0   # experts' gradients stay
+
+
+# ---------------------------------------------------------------- expert parallelism: order of phases and barriers
+
+# what a phase reads from its peers: every rank must have finished these before any rank starts the phase
+_NEEDS_FROM_ALL = {"dispatch": ("route",), "experts": ("dispatch",), "combine": ("experts",),
+                   "backward_combine": ("combine",), "backward_experts": ("backward_combine",),
+                   "backward_dispatch": ("backward_experts",)}
+
+
+def _order_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    from paper_2502_16927_b200 import ep
+
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    store = dist.distributed_c10d._get_default_store()
+    log, violations = [], []
+
+    class StubRank:
+        """Phase calls that do no arithmetic: each records that this rank ran it (in the store every rank sees) after
+        checking that every rank has finished what the phase reads from its peers."""
+        counts_all = torch.zeros((world, 4), dtype=torch.int32)
+
+        def __init__(self):
+            self.rank, self.step = rank, 0
+
+        def _run(self, name):
+            import time
+            for need in _NEEDS_FROM_ALL.get(name, ()):
+                for q in range(world):
+                    if store.add(f"{self.step}/{need}/{q}", 0) != 1:
+                        violations.append((self.step, name, need, q))
+            time.sleep(0.02 * (rank + 1) if name in ("dispatch", "experts", "backward_experts") else 0.0)   # ranks drift apart
+            store.add(f"{self.step}/{name}/{rank}", 1)
+            log.append(name)
+
+        def route(self, x, W, routing=None): self._run("route"); self.counts_all[rank] = rank + 1
+        def dispatch(self): self._run("dispatch")
+        def experts(self, W): self._run("experts")
+        def combine(self, W, y): self._run("combine")
+        def backward_combine(self, dy, W, G, accumulate=False): self._run("backward_combine")
+        def backward_experts(self, W, G, accumulate=False): self._run("backward_experts")
+        def backward_dispatch(self, x, W, dx, G, accumulate=False): self._run("backward_dispatch"); self.step += 1
+
+    class Order(ep.EpStepOrder):
+        def __init__(self):
+            self.rk = StubRank()
+            self._flag = torch.zeros(1, dtype=torch.int32)
+
+        def barrier(self):
+            log.append("|")
+            dist.all_reduce(self._flag)
+
+        def gather(self):
+            log.append("gather")
+            ep.gather_counts(self.rk.counts_all, rank)
+
+        def reduce(self, G):
+            log.append("reduce")
+            ep.reduce_shared_grads(G)
+
+    order = Order()
+    x = torch.zeros(3, 4)
+    G = {"dw_gate": torch.full((2,), float(rank + 1)), "db_gate": None, "dw_down": None, "dw_up": None}
+    for _ in range(2):
+        order.forward(x, {})
+        order.backward(x, x, {}, G)
+    out[rank] = dict(log=log, violations=violations, counts=order.rk.counts_all.tolist(), dw_gate=float(G["dw_gate"][0]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_expert_parallel_phase_order_and_barriers_with_two_ranks():
+    """EpStepOrder (what EpProcessRank runs) over two gloo ranks with stub phase calls: the order of the calls, a
+    barrier in front of every phase that reads what peers wrote, the count all-gather between route and dispatch, and
+    the shared-gradient reduction at the end of the backward."""
+    world, port = 2, 31500 + os.getpid() % 1000
+    manager = mp.Manager()
+    out = manager.dict()
+    mp.spawn(_order_worker, args=(world, port, out), nprocs=world, join=True)
+    step = ["route", "gather", "dispatch", "|", "experts", "|", "combine",
+            "|", "backward_combine", "|", "backward_experts", "|", "backward_dispatch", "reduce"]
+    for r_ in range(world):
+        assert out[r_]["log"] == step + step
+        assert out[r_]["violations"] == []                      # no phase ran before its inputs existed on every rank
+        assert out[r_]["counts"] == [[1, 1, 1, 1], [2, 2, 2, 2]]
+        assert out[r_]["dw_gate"] == 6.0                          # (1 + 2) after the first step's reduction, doubled by the second

@@ -364,3 +364,82 @@ def test_margin_conditioning_reaches_the_requested_gap():
     inp2 = wl.make_inputs(w)
     margin.enforce_margin(w, inp2, 1e-3)
     np.testing.assert_array_equal(inp["x"], inp2["x"])                    # seeded: reproducible
+
+
+# ---------------------------------------------------------------- non-finite logits; the bf16 ReLU' decision
+
+def test_topk_with_non_finite_logits_stays_in_range():
+    """NaN is ordered as -inf; a round that finds only -inf takes the lowest id not yet chosen; gate values are the
+    softmax of what was kept (exp(-inf) = 0), and 1/k each when nothing finite was kept.  Expected values by hand."""
+    ninf, nan = -np.inf, np.nan
+    logits = np.array([
+        [0.5, ninf, 2.0, ninf, ninf],      # two finite experts, k = 3: 2, 0, then the lowest masked id 1
+        [nan, nan, nan, nan, nan],         # a NaN token: experts 0, 1, 2 at 1/3 each
+        [nan, 1.0, ninf, 1.0, 3.0],        # NaN behind every finite value; the tie 1 = 1 goes to the lower id
+        [ninf, ninf, ninf, ninf, 7.0],     # one finite expert: it takes all the weight
+    ])
+    idx, p = oracle.topk(logits, 3)
+    np.testing.assert_array_equal(idx, [[2, 0, 1], [0, 1, 2], [4, 1, 3], [4, 0, 1]])
+    a = np.exp(-1.5)
+    b = np.exp(-2.0)
+    np.testing.assert_allclose(p[0], [1 / (1 + a), a / (1 + a), 0.0], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(p[1], [1 / 3, 1 / 3, 1 / 3], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(p[2], [1 / (1 + 2 * b), b / (1 + 2 * b), b / (1 + 2 * b)], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(p[3], [1.0, 0.0, 0.0], rtol=0, atol=0)
+    idx5, p5 = oracle.topk(logits, 5)                      # k = E: a permutation of all experts, whatever the values
+    assert all(sorted(row) == [0, 1, 2, 3, 4] for row in idx5.tolist())
+    np.testing.assert_array_equal(idx5[0], [2, 0, 1, 3, 4])
+    # finite rows are untouched by the rule
+    g = np.random.default_rng(5)
+    fin = g.standard_normal((20, 9))
+    np.testing.assert_array_equal(oracle.topk(fin, 4)[0], np.argsort(-fin, axis=1, kind="stable")[:, :4].astype(np.int32))
+
+
+def test_relu_decision_from_bf16_rounded_low_width_token():
+    """decide_bf16: ReLU' = [z > 0] is taken from z = bf16(x') W1^T (the numbers a BF16 kernel holds), everything
+    else stays exact.  E = 1, k = 1, identity descend projection, so x' = x; the first token is built so that one
+    hidden unit's exact z is 2^-10 > 0 while the rounded x' gives z = 0: its decision flips.  Checked against a numpy
+    restatement (library matmuls, the mask written out) and against the exact decision."""
+    d = r = 4
+    h, T = 5, 6
+    g = np.random.default_rng(11)
+    x = np.round(g.standard_normal((T, d)) * 64) / 64                      # exact in bf16 except the engineered row
+    x[0] = [1.0 + 2.0 ** -10, -1.0, 0.25, -0.5]
+    w1 = np.round(g.standard_normal((1, h, r)) * 8) / 8
+    w1[0, 0] = [1.0, 1.0, 0.0, 0.0]                                          # z = 2^-10 exactly; 0 from bf16(x')
+    w1[0, 1] = [1.0, -1.0, 0.0, 0.0]                                         # z = 2 + 2^-10: positive either way
+    inp = {"x": x.astype(np.float32), "dy": g.standard_normal((T, d)).astype(np.float32),
+           "w_gate": np.zeros((1, d), np.float32), "b_gate": None, "w_down": np.eye(r, d, dtype=np.float32),
+           "w1": w1.astype(np.float32), "w2": g.standard_normal((1, r, h)).astype(np.float32),
+           "w_up": g.standard_normal((d, r)).astype(np.float32)}
+    rt = oracle.route(inp, 1)
+    np.testing.assert_array_equal(rt.topk_p, 1.0)
+
+    def restated(x_for_decision):
+        X, W1, W2, Wup = _f64(inp["x"]), _f64(inp["w1"][0]), _f64(inp["w2"][0]), _f64(inp["w_up"])
+        mask = (x_for_decision @ W1.T > 0).astype(np.float64)               # [T,h]
+        dy_lo = _f64(inp["dy"]) @ Wup                                         # [T,r]
+        dz = (dy_lo @ W2) * mask                                              # du = dy' (p = 1); da = du W2
+        dx = dz @ W1                                                          # dx' = dz W1, dx = dx' I
+        dw1 = dz.T @ X                                                        # x' = x
+        a = np.maximum(X @ W1.T, 0.0)
+        dw2 = dy_lo.T @ a
+        return mask, dx, dw1, dw2
+
+    x_rounded = _f64(wl.bf16_round(inp["x"]))
+    mask_r, dx_r, dw1_r, dw2_r = restated(x_rounded)
+    mask_e, dx_e, dw1_e, dw2_e = restated(_f64(inp["x"]))
+    assert mask_e[0, 0] == 1.0 and mask_r[0, 0] == 0.0                       # the engineered unit flips
+    assert (mask_e != mask_r).sum() == 1 and mask_e[0, 1] == mask_r[0, 1] == 1.0
+    got_r = oracle.backward_full(inp, rt, wl.ACT_RELU, decide_bf16=True)
+    got_e = oracle.backward_full(inp, rt, wl.ACT_RELU, decide_bf16=False)
+    for got, (dx, dw1, dw2) in ((got_r, (dx_r, dw1_r, dw2_r)), (got_e, (dx_e, dw1_e, dw2_e))):
+        np.testing.assert_allclose(got["dx"], dx, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(got["dw1"][0], dw1, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(got["dw2"][0], dw2, rtol=0, atol=1e-12)
+    assert np.abs(got_r["dx"][0] - got_e["dx"][0]).max() > 1e-3              # the flip is visible in the gradient
+    np.testing.assert_array_equal(got_r["dw2"][0], got_e["dw2"][0])          # sigma itself is never rounded
+    # other activations ignore the switch
+    a1 = oracle.backward_full(inp, rt, wl.ACT_GELU_ERF, decide_bf16=True)
+    a0 = oracle.backward_full(inp, rt, wl.ACT_GELU_ERF, decide_bf16=False)
+    np.testing.assert_array_equal(a1["dx"], a0["dx"])

@@ -4,8 +4,10 @@ that only receives input and output pointers).  Its intermediates live in a fixe
 library instead of a caller-provided scratch buffer.
 
 The check: through the C ABI, on the same inputs, it must return exactly the tables bigmac_route returns -
-twice in a row, because the array keeps the previous call's contents - and it must refuse a problem that does
-not fit the array.  Collected last on purpose, and independent of what ran before it."""
+twice in a row, because the array keeps the previous call's contents - it must leave the device's free memory
+as it found it, and it must refuse a problem that does not fit the array.  The variants whose routing needs more
+intermediates (a load-balancing loss, a gate that reads x') go through the same comparison.  Collected last on
+purpose, and independent of what ran before it."""
 import numpy as np
 import pytest
 
@@ -23,15 +25,23 @@ def _same(a, b):
         np.testing.assert_array_equal(a[key].cpu().numpy(), b[key].cpu().numpy(), err_msg=key)
 
 
-@pytest.mark.parametrize("name,T", [("tiny", 256), ("small", 2048)])
-def test_route_static_matches_route_twice_in_a_row(name, T):
+@pytest.mark.parametrize("name,T,variant", [("tiny", 256, {}), ("small", 2048, {}), ("tiny", 200, {"aux_loss_coef": 0.01}),
+                                            ("tiny", 200, {"gate_low": True})])
+def test_route_static_matches_route_twice_in_a_row(name, T, variant):
+    import dataclasses
+
     import torch
     from paper_2502_16927_b200 import binding
 
     w = wl.WORKLOADS[name].with_tokens(T)
+    kw = {}
+    if variant.get("gate_low"):
+        w = dataclasses.replace(w, gate_low=True)
+    if "aux_loss_coef" in variant:
+        kw["aux_loss_coef"] = variant["aux_loss_coef"]
     inp = wl.make_inputs(w)
     dev = to_device(w, inp)
-    layer = make_layer(w)
+    layer = make_layer(w, **kw)
     expected = layer.route(dev["x"], dev)                       # existing entry point, caller-provided scratch
     torch.cuda.synchronize()
     other = to_device(w, wl.make_inputs(w.with_tokens(T, seed=w.seed + 7)))
@@ -39,9 +49,15 @@ def test_route_static_matches_route_twice_in_a_row(name, T):
         got = layer.empty_routing(T)
         for t in got.values():
             t.fill_(-1)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0] if call == 1 else None
         binding.bigmac_route_static(layer.handle, dev["x"], T, dev, got)
         torch.cuda.synchronize()
+        if call == 1:                                           # the set-up call is behind us: free memory does not move
+            assert torch.cuda.mem_get_info()[0] == free_before
         _same(got, expected)
+        if "aux_loss_coef" in variant:
+            assert got["aux_loss"].item() == expected["aux_loss"].item() > 0
         if call == 0:                                           # leave different contents behind in the array
             junk = layer.empty_routing(T)
             binding.bigmac_route_static(layer.handle, other["x"], T, other, junk)
