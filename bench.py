@@ -531,6 +531,89 @@ def run_ep_on_one_gpu(w, x, dy, dev, ms_step, steps, esz, size=4):
     return out
 
 
+def run_expert_parallel_ranks(w, x, dy, dev, steps, esz, rank, world, timed):
+    """One expert-parallel rank per process (Fig. 2c) over the job's NCCL group: every rank keeps its batch of T tokens
+    and owns E / N experts; rows cross the links at width r through the library's put / get kernels over symmetric
+    memory (plain peer loads and stores).  Beside it the Eq. 3 twin with equal E, k and expert parameters, whose rows
+    travel at width d.  Returns, on every rank, the whole-job tokens/s, the slowest rank's step time, this rank's
+    exchange-kernel times and the bytes a rank sends per exchange (Eq. 1).  Called after the headline number is final."""
+    import torch
+    from paper_2502_16927_b200 import binding, ep
+
+    if w.E % world:
+        return {"skipped": f"E = {w.E} is not a multiple of {world} ranks"}
+
+    def one(wv, Wfull, flags):
+        Ws = ep.shard_weights(Wfull, rank, world)
+        G = {"dw_gate": torch.empty_like(Wfull["w_gate"]), "dw1": torch.empty_like(Ws["w1"]), "dw2": torch.empty_like(Ws["w2"]),
+             "db_gate": torch.empty(wv.E, dtype=torch.float32, device="cuda")}
+        if not wv.cdac:
+            G.update(dw_down=torch.empty_like(Wfull["w_down"]), dw_up=torch.empty_like(Wfull["w_up"]))
+        epr = ep.EpProcessRank(wv.d, wv.r, wv.h, wv.E, wv.k, wv.T, wv.dtype, wv.act, flags=flags)
+        y, dx = torch.empty_like(x), torch.empty_like(x)
+
+        def step():
+            epr.forward(x, Ws, y=y)
+            epr.backward(x, dy, Ws, G, dx=dx)
+
+        for _ in range(3):
+            step()
+        ms = timed(step, steps) / steps
+        binding.bigmac_profile_enable(epr.rk.handle, True)
+        timed(step, steps)
+        prof = binding.bigmac_profile_read(epr.rk.handle)
+        binding.bigmac_profile_enable(epr.rk.handle, False)
+        status = epr.status()
+        epr.close()
+        if status != 0:
+            raise RuntimeError(f"device status word: {status}")
+        moves = {name: round(prof["stages"].get(name, (0.0, 1))[0] / steps, 4)
+                 for name in ("dispatch", "combine", "combine_bwd", "dxlo_gather")}
+        nbytes = ep.exchange_bytes_per_rank(wv.T, wv.k, wv.r, world, esz)
+        return {"row_width": wv.r, "ms_per_step": ms, "tokens_per_s": world * wv.T / (ms * 1e-3),
+                "exchange_kernels_ms_this_rank": moves, "exchange_kernels_ms_total": round(sum(moves.values()), 4),
+                "link_bytes_per_rank_per_exchange": nbytes,
+                "exchange_gbs_per_direction": {name: round(nbytes / (v * 1e-3) / 1e9, 1) for name, v in moves.items() if v > 0}}
+
+    out = {"ranks": world, "tokens_per_rank": w.T, "experts_per_rank": w.E // world,
+           "exchanges_per_step": "2 forward, 2 backward; peer puts / gets of rows, NCCL only for the count all-gather, "
+                                 "the barriers and the shared-gradient sums"}
+    out["bigmac_rows_at_width_r"] = one(w, dev, 0)
+    if w.dtype == wl.DTYPE_BF16 and (w.r * w.h) % w.d == 0 and (w.r * w.h // w.d) % 64 == 0:
+        t = w.cdac_twin()
+        need = 4 * world * t.T * t.k * t.r * esz                       # the four exchange buffers, worst case
+        if need < 0.5 * torch.cuda.mem_get_info()[0]:
+            gen = torch.Generator(device="cuda").manual_seed(w.seed + 11)
+            tw = {"w_gate": dev["w_gate"],
+                  "w1": (torch.randn((t.E, t.h, t.d), generator=gen, device="cuda") * t.d ** -0.5).to(torch.bfloat16),
+                  "w2": (torch.randn((t.E, t.d, t.h), generator=gen, device="cuda") * t.h ** -0.5).to(torch.bfloat16)}
+            if "b_gate" in dev:
+                tw["b_gate"] = dev["b_gate"]
+            out["eq3_twin_rows_at_width_d"] = one(t, tw, wl.FLAG_CDAC)
+            a, b = out["bigmac_rows_at_width_r"], out["eq3_twin_rows_at_width_d"]
+            out["bigmac_over_twin"] = {"step_time": round(a["ms_per_step"] / b["ms_per_step"], 3),
+                                       "exchange_kernel_time": round(a["exchange_kernels_ms_total"] / max(b["exchange_kernels_ms_total"], 1e-9), 3),
+                                       "link_bytes": round(a["link_bytes_per_rank_per_exchange"] / b["link_bytes_per_rank_per_exchange"], 4)}
+        else:
+            out["eq3_twin_rows_at_width_d"] = {"skipped": "exchange buffers at width d would not fit beside the rest"}
+    return out
+
+
+def nccl_communicator_line(path_pattern: str):
+    """The line of NCCL's own log that names the communicator's rank count (evidence of how many ranks took part)."""
+    import glob
+    import re
+
+    for path in sorted(glob.glob(path_pattern)):
+        try:
+            for line in open(path, errors="replace"):
+                if re.search(r"nranks\s+\d+", line):
+                    return line.strip()[-240:]
+        except OSError:
+            continue
+    return None
+
+
 # ------------------------------------------------------------------------------------------------ ours
 def run_ours(args, w):
     import torch
@@ -543,8 +626,22 @@ def run_ours(args, w):
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the layer has no CPU path")
     torch.cuda.set_device(local)
+    want_ep = world > 1 or args.expert_parallel
+    nccl_log = None
+    if want_ep:
+        # NCCL's communicator log goes to a file of its own (its default, stdout, would break the one-line contract)
+        import tempfile
+        nccl_dir = tempfile.mkdtemp(prefix="bigmac_nccl_")
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        os.environ.setdefault("NCCL_DEBUG_FILE", os.path.join(nccl_dir, "rank%p.log"))
+        nccl_log = os.environ["NCCL_DEBUG_FILE"].replace("%p", "*").replace("%h", "*")
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    elif want_ep:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", str(29600 + os.getpid() % 1000))
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", local))
     if rank == 0:
         build.build()
     if world > 1:
@@ -788,9 +885,45 @@ def run_ours(args, w):
     if layer.status() != 0:
         raise RuntimeError("device status word reports a timed-out wait")
 
+    # ---- expert parallelism over the job's ranks (N > 1, or on request with a group of one): after everything the
+    # headline needs, on all ranks together.  A failure here is recorded, not raised; should a rank hang in a
+    # collective, rank 0's watchdog prints the headline without this section before the process group's own time-out
+    # can take the process down.
+    ep_ranks = None
+    if want_ep and w.dtype == wl.DTYPE_BF16 and not forward_only_workload:
+        esz_ep = 2
+        bytes_io_ep = 2 * w.T * w.d * esz_ep
+        minimal = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                   "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                   "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config_dict(w, args), "clocks": clocks,
+                   "e2e": {"value": world * w.T / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": bytes_io_ep,
+                           "d2h_bytes_per_step": bytes_io_ep, "ms_per_step": ms_e2e},
+                   "gpu_launches": prof["launches"], "repeats": repeats,
+                   "expert_parallel": {"error": "timed out: a rank did not reach a collective; side measurements skipped"}}
+
+        def print_minimal_and_leave():
+            print(json.dumps(minimal), flush=True)
+            os._exit(0)
+
+        watchdog = None
+        if rank == 0:
+            watchdog = threading.Timer(300.0, print_minimal_and_leave)
+            watchdog.daemon = True
+            watchdog.start()
+        try:
+            ep_ranks = run_expert_parallel_ranks(w, x, dy, dev, max(3, min(args.steps, 10)), esz_ep, rank, world, timed)
+            ep_ranks["nccl_communicator"] = nccl_communicator_line(nccl_log) if nccl_log else None
+        except Exception as err:                       # the headline must survive whatever happens here
+            ep_ranks = {"error": f"{type(err).__name__}: {err}"[:300]}
+        if watchdog:
+            watchdog.cancel()
+
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        if dist.is_initialized():
+            try:
+                dist.destroy_process_group()
+            except Exception:
+                pass
         return
 
     peaks = measured_peaks()
@@ -907,9 +1040,14 @@ def run_ours(args, w):
             "expert_parallel_on_one_gpu": ep_line,
             "groups": groups,
             "stages": stages}
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    if ep_ranks is not None:
+        line["expert_parallel"] = ep_ranks
+    print(json.dumps(line), flush=True)
+    if dist.is_initialized():
+        try:
+            dist.destroy_process_group()
+        except Exception:
+            pass
 
 
 def main():
@@ -920,6 +1058,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="large", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0, help="override T (per GPU)")
+    ap.add_argument("--expert-parallel", action="store_true",
+                    help="also run the expert-parallel layer over the job's ranks when there is only one (N > 1: always)")
     ap.add_argument("--headline-only", action="store_true",
                     help="skip the side measurements (Eq. 3 twin, expert-parallel ranks on one GPU, variants, recipe)")
     ap.add_argument("--profile-run", action="store_true",

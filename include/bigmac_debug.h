@@ -76,6 +76,7 @@ const char *bigmac_profile_slot_name(int slot);
  *   "groupk" 0/1         never / where it pays: the dynamically scheduled per-expert weight-gradient kernel (default 1)
  *   "fused_mlp" 0/1/2    inference expert GEMM1 + sigma + GEMM2 in one kernel never / on short tile lists / always (default 1)
  *   "epi_parts" 0/1/2/4  working epilogue warps per lane quadrant of plain epilogues (0 = default choice, 2)
+ *   "staged_stores" 0/1  wide bf16 outputs by 32-byte direct stores / through shared-memory boxes and TMA stores (default 1)
  *   "fuse_dispatch" 0/1  standalone dispatch kernel / expert GEMM1 gathers its rows itself where supported (default 1)
  *   "tc_mask" bits       bit i: contraction i runs on tcgen05, else on the FMA kernel; read when a handle is created
  *   "defaults"           every switch back to its default (value ignored)

@@ -232,7 +232,7 @@ def bigmac_debug_gemm(handle, q: bigmac_debug_gemm_t, use_tensor_cores) -> None:
 
 def bigmac_debug_set(name: str, value: int = 0) -> None:
     """Process-wide measurement / debugging switch ("overlap", "tc_pair", "groupk", "fused_mlp", "epi_parts",
-    "fuse_dispatch", "tc_mask"; "defaults" restores all).  The defaults are the product."""
+    "staged_stores", "fuse_dispatch", "tc_mask"; "defaults" restores all).  The defaults are the product."""
     _check(lib().bigmac_debug_set(name.encode(), int(value)), "bigmac_debug_set")
 
 

@@ -25,7 +25,10 @@ namespace {
 // Persistent kernel: gridDim.x CTAs (one per SM) walk the tile list with stride gridDim.x.  The
 // accumulator is double-buffered in tensor memory (2 x BN columns), so the epilogue of tile i overlaps
 // the MMAs of tile i+1.
-template <int BN, int STAGES, bool A_KMAJOR, bool B_KMAJOR, bool TMA_EPI>
+// GATHER: the rows of the (K-major) A tile are gathered by the producer warp with 16-byte asynchronous copies
+// (TcParams::gather_rows) instead of one TMA box per k slice; a slice is handed to the MMA warp once its copies have
+// landed and the proxy fence is behind them, kGatherLag slices after it was issued.
+template <int BN, int STAGES, bool A_KMAJOR, bool B_KMAJOR, bool TMA_EPI, bool GATHER = false>
 __global__ void __launch_bounds__(kThreadsV2, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_z,
@@ -48,13 +51,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint64_t* z_bar = tmem_empty_bar + 2;                    // [kEpiWarps]: sigma' boxes prefetched by TMA (EPI_DACT)
     uint32_t* tmem_slot = (uint32_t*)(z_bar + kEpiWarps);
     volatile int* dead = (volatile int*)(tmem_slot + 1);
+    int32_t* row_tok = (int32_t*)(tmem_slot + 4);            // [BM] source row of every row of the tile being gathered (GATHER)
+    static_assert(!GATHER || A_KMAJOR, "gathered rows: K-major A");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int tiles_m, tiles_n;
     const int total = total_tiles(p, BN, tiles_m, tiles_n);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        // a gathered slice completes on the B box's bytes and on the producer warp's arrival for the A rows
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 2 : 1); mbar_init(&empty_bar[s], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], kEpiWarps); }
         for (int s = 0; s < kEpiWarps; ++s) mbar_init(&z_bar[s], 1);
         *dead = 0;
@@ -67,7 +73,43 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0) {
+    if (warp == 0 && GATHER) {
+        // ------------------------------------------------------------------ producer, gathered A rows (whole warp)
+        uint32_t s = 0, phase = 1, issued = 0, sig = 0;    // sig: stage of the oldest slice not yet handed over
+        const uint8_t* src = (const uint8_t*)p.gather_src;
+        const int64_t ld_bytes = p.gather_ld * 2;
+        auto hand_over = [&]() {                           // the copies of the oldest slice in flight have landed
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[sig]);
+            sig = sig + 1 == STAGES ? 0 : sig + 1;
+        };
+        for (int t = blockIdx.x; t < total; t += gridDim.x) {
+            const Tile tl = get_tile(p, BN, t, tiles_m, tiles_n);
+            __syncwarp();
+            for (int q = lane; q < BM; q += 32) {
+                const int g = p.gather_rows[tl.m0 + q];
+                row_tok[q] = g < 0 ? -1 : g / p.gather_div;
+            }
+            __syncwarp();
+            for (int kb = 0; kb < tl.num_kb; ++kb, s = (s + 1 == STAGES ? 0 : s + 1), phase ^= (s == 0)) {
+                mbar_wait_lean(&empty_bar[s], phase, dead, p.status);
+                const int k0 = kb * BK;
+                if (lane == 0) {
+                    mbar_expect_tx(&full_bar[s], B_BYTES);
+                    tma_load_2d(smem_b + s * B_BYTES, &map_b, &full_bar[s], k0, tl.expert * p.b_rows_per_expert + tl.n0);
+                }
+                gather_kmajor_slice(smem_a + s * A_BYTES, src, ld_bytes, k0 * 2, row_tok, lane);
+                cp_async_commit();
+                if (++issued > kGatherLag) {
+                    cp_async_wait<kGatherLag>();
+                    hand_over();
+                }
+            }
+        }
+        cp_async_wait<0>();
+        for (uint32_t left = issued < kGatherLag ? issued : kGatherLag; left > 0; --left) hand_over();
+    } else if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t s = 0, phase = 1;                     // stage and the parity its "empty" barrier is waited on with
@@ -241,13 +283,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 }
 
-template <int BN, int STAGES, bool AK, bool BKM, bool TMA_EPI>
+template <int BN, int STAGES, bool AK, bool BKM, bool TMA_EPI, bool GATHER = false>
 cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mz,
                    const CUtensorMap& mb2, const TcParams& p, int max_tiles, cudaStream_t stream) {
     constexpr size_t smem = STAGES * (BM * BK * 2 + BN * BK * 2) + (TMA_EPI ? kEpiWarps * 2 * kBoxBytes : 0) +
-                            (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + 1024;
+                            (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + (GATHER ? BM * 4 : 0) + 1024;
     static PerDeviceOnce once;
-    auto kernel = gemm_tc_kernel<BN, STAGES, AK, BKM, TMA_EPI>;
+    auto kernel = gemm_tc_kernel<BN, STAGES, AK, BKM, TMA_EPI, GATHER>;
     int dev;
     if (once.needed(&dev)) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -266,7 +308,12 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
     bool ok = true;
     TcParams p{};
     // A: [M,K] (K-major) or [K,M] (MN-major).  In GROUP_K, K is the row extent of the padded grouped buffers.
-    if (g.a_kmajor) ok &= make_map(&ma, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.lda, BK, BM);
+    const bool gather = g.gather_rows != nullptr;           // A's rows are gathered by the producer warp: no tensor map for A
+    if (gather && (!g.a_kmajor || !g.b_kmajor || g.group != GROUP_M || g.B2 || g.C2 || g.split_k > 1 || g.K % BK ||
+                   (g.lda * 2) % 16 || (uintptr_t)g.A % 16))
+        return cudaErrorInvalidValue;
+    if (gather) ok &= make_map(&ma, g.A, (uint64_t)g.K, 1, (uint64_t)g.lda, BK, 1);       // placeholder, never used
+    else if (g.a_kmajor) ok &= make_map(&ma, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.lda, BK, BM);
     else ok &= make_map(&ma, g.A, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.lda, 64, BK);
     // B: dense [N,K] / [K,N]; grouped weights are E consecutive such matrices (b_stride elements apart).
     const uint64_t rows_per = g.group == GROUP_M ? (uint64_t)(g.b_stride / g.ldb) : 0;
@@ -316,8 +363,10 @@ cudaError_t dispatch(const GemmArgs& g, int* status, cudaStream_t stream) {
     p.epi_parts = 4;
     p.bias = g.group == GROUP_M ? g.bias : nullptr; p.bias_stride = g.bias_stride;
     if (p.bias && (g.N % 32 || ((uintptr_t)g.bias % 16) || g.bias_stride % 4)) return cudaErrorInvalidValue;
+    p.gather_rows = g.gather_rows; p.gather_src = g.A; p.gather_ld = g.lda; p.gather_div = g.gather_div > 0 ? g.gather_div : 1;
     const int64_t tiles = (int64_t)((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * (g.group == GROUP_K ? E : p.split_k);
     const int max_tiles = tiles > (1 << 30) ? (1 << 30) : (int)tiles;
+    if (gather) return launch<BN, STAGES, true, true, TMA_EPI, true>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
     if (g.a_kmajor && g.b_kmajor) return launch<BN, STAGES, true, true, TMA_EPI>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
     if (g.a_kmajor && !g.b_kmajor) return launch<BN, STAGES, true, false, TMA_EPI>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
     if (!g.a_kmajor && !g.b_kmajor) return launch<BN, STAGES, false, false, TMA_EPI>(ma, mb, mc, mz, mb2, p, max_tiles, stream);
@@ -353,12 +402,14 @@ cudaError_t gemm_tc(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
     // Where it pays, the problem runs on CTA pairs (each SM stages half of B); the tc_pair debug switch disables that.
     const bool pair_enabled = switches().tc_pair != 0;
-    const bool want_pair = g.force_kernel == 2 ? gemm_tc_pair_supported(g)
+    const bool want_pair = g.gather_rows ? false          // gathered rows: the one-CTA kernel
+                           : g.force_kernel == 2 ? gemm_tc_pair_supported(g)
                            : g.force_kernel == 1 ? false : (pair_enabled && gemm_tc_pair_preferred(g));
     if (want_pair) return gemm_tc_pair(g, status, stream);
     // Output-heavy problems (wide rows: activations, ascend, dx) stage their stores through shared memory and
     // TMA, which costs one pipeline stage; contraction-heavy ones keep the deeper pipeline and store directly.
-    const bool staged = !g.C2 && tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 && (g.epilogue != EPI_DACT || g.group != GROUP_K);
+    const bool staged = switches().staged_stores && !g.C2 && tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 &&
+                        (g.epilogue != EPI_DACT || g.group != GROUP_K);
     if (g.N >= 256) return staged ? dispatch<256, 3, true>(g, status, stream) : dispatch<256, 4, false>(g, status, stream);
     return dispatch<128, 6, false>(g, status, stream);
 }

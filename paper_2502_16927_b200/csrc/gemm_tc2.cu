@@ -464,7 +464,7 @@ bool gemm_tc_pair_preferred(const GemmArgs& g) {
 
 cudaError_t gemm_tc_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
-    const bool staged = !g.C2 && tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 &&
+    const bool staged = switches().staged_stores && !g.C2 && tma_epilogue_possible(g) && g.N >= 1024 && g.N % 256 == 0 &&
                         (g.epilogue != EPI_DACT || g.group != GROUP_K);
     // 32 KB per stage and CTA: 5 stages beside the 64 KB store staging (4 if the expert tables are long), 6 without it
     if (!staged) return dispatch_pair<256, 6, false>(g, status, stream);

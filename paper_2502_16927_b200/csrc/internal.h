@@ -59,6 +59,11 @@ struct GemmArgs {
     int split_k = 1;                    // > 1: part s of the contraction writes its partial result (fp32) to C + s*M*ldc
     int force_kernel = 0;               // measurement aid: 1 = one-CTA kernel, 2 = CTA-pair kernel, 0 = default choice
     int epi_parts = 0;                  // measurement aid: epilogue warps per lane quadrant that work (1, 2 or 4); 0 = default choice
+    // Tensor-core path, GROUP_M with K-major A: the rows of A are gathered (the dispatch fused into the operand load):
+    // row m of A is row gather_rows[m] / gather_div of A itself (which then is the ungrouped matrix, lda its row
+    // stride), zeros where gather_rows[m] < 0.  Null: A holds the grouped rows.
+    const int32_t* gather_rows = nullptr;
+    int gather_div = 1;
     // GROUP_M only: fp32 bias added to the accumulator before the epilogue, column n of a row of expert e gets
     // bias[e*bias_stride + n] (16-byte aligned, bias_stride a multiple of 4)
     const float* bias = nullptr;

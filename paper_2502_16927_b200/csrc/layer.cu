@@ -440,15 +440,20 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         g.M = m.T; g.N = m.r; g.K = m.d;
         BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
     }
-    { Stage s(L, S_DISPATCH, st); BIGMAC_CUDA(launch_dispatch(b.x_lo, b.xg, b.tb, m.k, m.r, m.dtype, m.P, st)); }  // F5 dispatch at width r
+    // F5 dispatch at width r.  Inference on the tensor-core path with the two expert GEMMs as separate launches: the
+    // dispatch is fused into expert GEMM1, whose producer warp gathers the rows of x' itself (slot_of_prow names the
+    // token of every grouped row, -1 the zero padding rows), so the grouped copy xg is never written.  A training
+    // forward keeps xg: the per-expert weight gradient dW1 contracts over it.
+    const bool short_list = m.P / kPad <= 2 * (int64_t)gemm_tc_sm_count();
+    const bool mlp_fused_ = !training && !m.bias && (switches().fused_mlp == 2 || (switches().fused_mlp == 1 && short_list)) &&
+                            sigma_as_bytes(L) && fused_mlp_supported(m.r, m.h, m.dtype);
+    const bool gather_dispatch = switches().fuse_dispatch && !training && !mlp_fused_ && sigma_as_bytes(L) && m.r % 64 == 0;
+    if (!gather_dispatch) { Stage s(L, S_DISPATCH, st); BIGMAC_CUDA(launch_dispatch(b.x_lo, b.xg, b.tb, m.k, m.r, m.dtype, m.P, st)); }
     // Inference, low width r <= 256, up to two row tiles per SM: F6 + F7 in one kernel, the hidden activations stay on
     // the SM.  On long tile lists the two separate GEMMs are faster (the fused kernel is bound by the issue of its many
     // narrow MMA instructions): measured 0.375 vs 0.329 ms forward at the medium workload, 0.099 vs 0.106 ms at 512
     // decode tokens.  The fused_mlp debug switch forces it off (0) / on (2).
-    const int fuse_mlp_mode = switches().fused_mlp;
-    const bool short_list = m.P / kPad <= 2 * (int64_t)gemm_tc_sm_count();
-    if (!training && !m.bias && (fuse_mlp_mode == 2 || (fuse_mlp_mode == 1 && short_list)) && sigma_as_bytes(L) &&
-        fused_mlp_supported(m.r, m.h, m.dtype)) {
+    if (mlp_fused_) {
         Stage s(L, S_FUSED_MLP, st);
         BIGMAC_CUDA(launch_fused_mlp(b.xg, W->w1, W->w2, b.u, m.P, m.r, m.h, m.E, c.act, b.tb.tile_expert, b.tb.n_tiles,
                                      L->status, st));
@@ -456,6 +461,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         {                                                                             // F6 a = sigma(xg W1_e^T); saves sigma'(z)
             GemmArgs g;
             g.A = b.xg; g.lda = m.r; g.B = W->w1; g.ldb = m.r; g.b_stride = (int64_t)m.h * m.r;
+            if (gather_dispatch) { g.A = b.x_lo; g.gather_rows = b.tb.slot_of_prow; g.gather_div = m.k; }
             g.C = b.a; g.Z = b.z; g.ldc = m.h; g.M = (int)m.P; g.N = m.h; g.K = m.r;
             g.epilogue = EPI_ACT; g.act = c.act; g.group = GROUP_M; g.num_experts = m.E;
             g.tile_expert = b.tb.tile_expert; g.n_tiles = b.tb.n_tiles; g.poffsets = b.tb.poffsets;
@@ -971,6 +977,7 @@ int bigmac_debug_set(const char* name, int value) {
     else if (!std::strcmp(name, "groupk")) sw.groupk = value;
     else if (!std::strcmp(name, "fused_mlp")) sw.fused_mlp = value;
     else if (!std::strcmp(name, "epi_parts")) sw.epi_parts = value;
+    else if (!std::strcmp(name, "staged_stores")) sw.staged_stores = value;
     else if (!std::strcmp(name, "fuse_dispatch")) sw.fuse_dispatch = value;
     else if (!std::strcmp(name, "tc_mask")) sw.tc_mask = (unsigned)value;
     else if (!std::strcmp(name, "defaults")) sw = Switches();

@@ -10,6 +10,7 @@ struct Switches {
     int groupk = 1;         // dynamically scheduled per-expert weight-gradient kernel where it pays (0: never)
     int fused_mlp = 1;      // inference: expert GEMM1 + sigma + GEMM2 in one kernel on short tile lists (0: never, 2: always)
     int epi_parts = 0;      // working epilogue warps per lane quadrant of plain epilogues (1, 2, 4; 0: the default, 2)
+    int staged_stores = 1;  // wide bf16 outputs leave through shared-memory boxes and TMA stores (0: always 32-byte direct stores)
     int fuse_dispatch = 1;  // expert GEMM1 gathers its rows from x' itself where supported (0: standalone dispatch kernel)
     unsigned tc_mask = ~0u; // bit i: contraction i runs on tcgen05 (read when a handle is created)
 };

@@ -125,6 +125,33 @@ __device__ __forceinline__ void st_shared_16B(void* ptr, uint32_t a, uint32_t b,
     asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(smem_u32(ptr)), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// ---- gathered operand rows (dispatch fused into a contraction's operand load)
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros (the source is not read).
+__device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+constexpr int kGatherLag = 2;       // gathered k slices in flight behind the newest before the oldest is handed to the MMA warp
+
+// One 64-deep k slice of a K-major operand tile whose rows are gathered: row i of the 128-row tile is row tok[i] of
+// the source matrix (row stride ld_bytes; zeros where tok[i] < 0), written in the 128-byte-swizzled layout a TMA
+// load of the same box would produce (16-byte piece j of row i at piece j ^ (i & 7)).  Called by all lanes of a warp:
+// lane l moves piece l & 7 of rows (l >> 3) + 4 j, j = 0..31.
+__device__ __forceinline__ void gather_kmajor_slice(uint8_t* stage, const uint8_t* src, int64_t ld_bytes, int k0_bytes,
+                                                    const int32_t* tok, int lane) {
+    const int piece = lane & 7, r0 = lane >> 3;
+    const uint32_t base = smem_u32(stage);
+#pragma unroll 8
+    for (int j = 0; j < BM / 4; ++j) {
+        const int row = r0 + 4 * j;
+        const int t = tok[row];
+        const uint8_t* from = src + (int64_t)(t < 0 ? 0 : t) * ld_bytes + k0_bytes + piece * 16;
+        cp_async_16(base + row * 128 + ((piece ^ (row & 7)) << 4), from, t < 0 ? 0u : 16u);
+    }
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
                  : "memory");
@@ -225,6 +252,13 @@ struct TcParams {
     const int32_t* tile_expert;
     const int32_t* n_tiles;
     const int32_t* poffsets;
+    // gathered A rows (dispatch fused into the operand load; K-major A, GROUP_M): row m of A is row
+    // gather_rows[m] / gather_div of the matrix at gather_src (row stride gather_ld elements), zeros where
+    // gather_rows[m] < 0 (padding rows); null = A is read as it lies
+    const int32_t* gather_rows;
+    const void* gather_src;
+    int64_t gather_ld;
+    int gather_div;
     int* status;
 };
 

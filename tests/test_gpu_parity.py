@@ -30,8 +30,16 @@ BF16_MAX, BF16_FRO, BF16_RMS = 1e-2, 8e-3, 6e-2
 #              full-size checks, nearly empty experts) the storage error of the terms does not average out and the
 #              largest elements carry it whole (0.92 % of max|b| at the large workload, Frobenius 0.48 %);
 #   db_gate    a sum of terms of both signs that cancels to a small difference of large parts under skewed routing;
-#              the bf16 storage of dy' and u behind every term is then a larger share of the result (1.6 % / 1.0 %).
-BF16_OWN = {"dw1": (1.5e-2, BF16_FRO), "dw2": (1.5e-2, BF16_FRO), "db_gate": (2e-2, 1.5e-2)}
+#              the bf16 storage of dy' and u behind every term is then a larger share of the result (1.6 % / 1.0 %);
+#   dw_gate    its rows are dl_j x: every dl_j = p_j (dp_j - g) is itself a difference of dot products of bf16-stored
+#              rows, and with a handful of tokens nothing averages that out (Frobenius 1.2 % for a single token).
+#   Their RMS-floored metric (one floor per expert) is bounded at 1e-1: an element of a per-expert gradient is a sum of
+#   products of two Gaussian-like factors, and where one large term dominates a small sum its storage error is several
+#   per cent of the expert's RMS (measured up to 8.0e-2 on the medium workload's sampled check).
+BF16_OWN = {"dw1": (1.5e-2, BF16_FRO, 1e-1), "dw2": (1.5e-2, BF16_FRO, 1e-1), "db_gate": (2e-2, 1.5e-2, BF16_RMS),
+            "dw_gate": (1.5e-2, 1.5e-2, BF16_RMS)}
+# ReLU' flips (see RELU_DECISION_KEYS below) are counted against twice the max-norm bound.
+RELU_OUTLIER = 2 * BF16_MAX
 TOL = {wl.DTYPE_F32: 1e-4, wl.DTYPE_BF16: BF16_MAX}
 SIMT = 1
 
@@ -91,8 +99,8 @@ def tolerance_of(w, key):
     if w.dtype == wl.DTYPE_F32:
         return TOL[wl.DTYPE_F32]
     base, _, suffix = key.partition(":")
-    own_max, own_fro = BF16_OWN.get(base, (BF16_MAX, BF16_FRO))
-    return own_fro if suffix == "fro" else BF16_RMS if suffix == "rms" else own_max
+    own_max, own_fro, own_rms = BF16_OWN.get(base, (BF16_MAX, BF16_FRO, BF16_RMS))
+    return own_fro if suffix == "fro" else own_rms if suffix == "rms" else own_max
 
 
 def assert_within(w, errs):
@@ -128,8 +136,9 @@ def outlier_fraction(a, b, tol):
 # Gradients that pass through sigma'.  With ReLU in BF16, sigma'(z) = [z > 0] is a discrete decision taken
 # on z values that carry the rounding of x' (and its fp32 accumulation order): the oracle takes it from
 # the bf16-rounded x' as well, but a handful of hidden units with |z| inside the accumulation noise still
-# decide differently.  Each such unit changes isolated gradient elements, so for those tensors the
-# elementwise bound is required of all but 1e-3 of the elements and the Frobenius bound of the whole tensor.
+# decide differently.  Each such unit changes isolated gradient elements, so for those tensors an elementwise
+# bound (2e-2 of the largest magnitude) is required of all but 1e-3 of the elements and the Frobenius bound of the
+# whole tensor.
 RELU_DECISION_KEYS = ("dx", "dw1", "dw2", "dw_down", "dw_gate", "db_gate", "db1")
 
 
@@ -149,7 +158,7 @@ def compare_full(w, inp, got, tol=None, capacity_factor=0.0, aux=0.0):
         for key in RELU_DECISION_KEYS:
             if key not in keys:
                 continue
-            assert outlier_fraction(got[key], ref[key], TOL[w.dtype]) <= 1e-3, key
+            assert outlier_fraction(got[key], ref[key], RELU_OUTLIER) <= 1e-3, key
             errs.pop(key)
             errs.pop(key + ":rms")
     assert_within(w, errs)
@@ -466,3 +475,40 @@ def test_routing_tables_around_the_single_block_limit(T, E, k, f):
     assert layer.status() == 0
     check_routing(R, oracle.route(inp, w.k, capacity_factor=f))
     layer.close()
+
+
+@pytest.mark.parametrize("case", [
+    dict(T=300, d=128, r=64, h=192, E=5, k=2, act=wl.ACT_GELU_ERF),       # one k slice per tile, ragged segments, narrow outputs
+    dict(T=1000, d=256, r=320, h=1024, E=16, k=4, act=wl.ACT_RELU),       # five k slices: more than the gather's lag, staged stores
+    dict(T=5000, d=512, r=512, h=2048, E=8, k=2, act=wl.ACT_GELU_ERF),    # the large workload's widths, many row tiles per SM
+    dict(T=700, d=128, r=128, h=64, E=40, k=1, act=wl.ACT_GELU_TANH),     # empty experts, 128-wide tiles
+    dict(T=2, d=64, r=64, h=256, E=8, k=3, act=wl.ACT_GELU_ERF),          # nearly all padding rows
+])
+def test_inference_forward_with_the_dispatch_fused_into_expert_gemm1(case):
+    """Inference forward with the two expert GEMMs as separate launches: expert GEMM1 gathers the rows of x' itself
+    (no grouped copy is written).  y against the oracle, and bit for bit against the same forward with the standalone
+    dispatch kernel in front (same operands, same arithmetic order)."""
+    import torch
+    from paper_2502_16927_b200 import binding
+
+    case = dict(case)
+    act = case.pop("act")
+    w = wl.Workload("fd", dtype=wl.DTYPE_BF16, act=act, seed=977, **case)
+    inp = conditioned(w)
+    dev = to_device(w, inp)
+    binding.bigmac_debug_set("fused_mlp", 0)
+    try:
+        layer = make_layer(w)
+        y, R = layer.forward(dev["x"], dev, training=False, want_routing=True)
+        y = y.clone()
+        binding.bigmac_debug_set("fuse_dispatch", 0)
+        y_plain = layer.forward(dev["x"], dev, training=False).clone()
+        torch.cuda.synchronize()
+        assert layer.status() == 0
+        layer.close()
+    finally:
+        binding.bigmac_debug_set("defaults")
+    rt = oracle.route(inp, w.k)
+    check_routing(R, rt)
+    assert_within(w, float_errors(w, {"y": to_numpy(y)}, {"y": oracle.forward_tokens(inp, rt, w.act)["y"]}))
+    assert torch.equal(y.view(torch.int16), y_plain.view(torch.int16))
