@@ -591,9 +591,10 @@ def run_expert_parallel_ranks(w, x, dy, dev, steps, esz, rank, world, timed):
                 tw["b_gate"] = dev["b_gate"]
             out["eq3_twin_rows_at_width_d"] = one(t, tw, wl.FLAG_CDAC)
             a, b = out["bigmac_rows_at_width_r"], out["eq3_twin_rows_at_width_d"]
-            out["bigmac_over_twin"] = {"step_time": round(a["ms_per_step"] / b["ms_per_step"], 3),
-                                       "exchange_kernel_time": round(a["exchange_kernels_ms_total"] / max(b["exchange_kernels_ms_total"], 1e-9), 3),
-                                       "link_bytes": round(a["link_bytes_per_rank_per_exchange"] / b["link_bytes_per_rank_per_exchange"], 4)}
+            ratio = lambda u, v, nd: round(u / v, nd) if v else None
+            out["bigmac_over_twin"] = {"step_time": ratio(a["ms_per_step"], b["ms_per_step"], 3),
+                                       "exchange_kernel_time": ratio(a["exchange_kernels_ms_total"], b["exchange_kernels_ms_total"], 3),
+                                       "link_bytes": ratio(a["link_bytes_per_rank_per_exchange"], b["link_bytes_per_rank_per_exchange"], 4)}
         else:
             out["eq3_twin_rows_at_width_d"] = {"skipped": "exchange buffers at width d would not fit beside the rest"}
     return out
@@ -646,6 +647,9 @@ def run_ours(args, w):
         build.build()
     if world > 1:
         dist.barrier()
+    for item in args.debug_set:
+        name, _, val = item.partition("=")
+        binding.bigmac_debug_set(name, int(val or 0))
 
     wr = w.with_tokens(w.T, seed=rank_seed(w.seed, rank))
     inp = wl.make_inputs(wr)
@@ -1058,6 +1062,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="large", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0, help="override T (per GPU)")
+    ap.add_argument("--debug-set", action="append", default=[], metavar="NAME=VALUE",
+                    help="measurement aid: set a kernel-choice switch of the library (bigmac_debug_set) before anything runs")
     ap.add_argument("--expert-parallel", action="store_true",
                     help="also run the expert-parallel layer over the job's ranks when there is only one (N > 1: always)")
     ap.add_argument("--headline-only", action="store_true",

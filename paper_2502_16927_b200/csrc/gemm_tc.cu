@@ -25,11 +25,12 @@ namespace {
 // Persistent kernel: gridDim.x CTAs (one per SM) walk the tile list with stride gridDim.x.  The
 // accumulator is double-buffered in tensor memory (2 x BN columns), so the epilogue of tile i overlaps
 // the MMAs of tile i+1.
-// GATHER: the rows of the (K-major) A tile are gathered by the producer warp with 16-byte asynchronous copies
-// (TcParams::gather_rows) instead of one TMA box per k slice; a slice is handed to the MMA warp once its copies have
-// landed and the proxy fence is behind them, kGatherLag slices after it was issued.
+// GATHER: the rows of the (K-major) A tile are gathered (TcParams::gather_rows) by two extra warps with 16-byte
+// asynchronous copies into the layout a TMA box would have, instead of one TMA box per k slice: warp g of them owns
+// rows 64 g .. 64 g + 63 of the tile, lane l piece l & 7 of rows (l >> 3) + 4 j; every thread arrives on the stage's
+// "full" barrier when its copies have landed.
 template <int BN, int STAGES, bool A_KMAJOR, bool B_KMAJOR, bool TMA_EPI, bool GATHER = false>
-__global__ void __launch_bounds__(kThreadsV2, 1)
+__global__ void __launch_bounds__(GATHER ? kThreadsGather : kThreadsV2, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_z,
                const __grid_constant__ CUtensorMap map_b2, const TcParams p) {
@@ -51,7 +52,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint64_t* z_bar = tmem_empty_bar + 2;                    // [kEpiWarps]: sigma' boxes prefetched by TMA (EPI_DACT)
     uint32_t* tmem_slot = (uint32_t*)(z_bar + kEpiWarps);
     volatile int* dead = (volatile int*)(tmem_slot + 1);
-    int32_t* row_tok = (int32_t*)(tmem_slot + 4);            // [BM] source row of every row of the tile being gathered (GATHER)
     static_assert(!GATHER || A_KMAJOR, "gathered rows: K-major A");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -59,8 +59,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int total = total_tiles(p, BN, tiles_m, tiles_n);
 
     if (threadIdx.x == 0) {
-        // a gathered slice completes on the B box's bytes and on the producer warp's arrival for the A rows
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 2 : 1); mbar_init(&empty_bar[s], 1); }
+        // a gathered slice completes on the B box's bytes and on the arrival of every gathering thread
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 1 + kGatherWarps * 32 : 1); mbar_init(&empty_bar[s], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], kEpiWarps); }
         for (int s = 0; s < kEpiWarps; ++s) mbar_init(&z_bar[s], 1);
         *dead = 0;
@@ -73,42 +73,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0 && GATHER) {
-        // ------------------------------------------------------------------ producer, gathered A rows (whole warp)
-        uint32_t s = 0, phase = 1, issued = 0, sig = 0;    // sig: stage of the oldest slice not yet handed over
-        const uint8_t* src = (const uint8_t*)p.gather_src;
+    if (GATHER && warp >= 2 + kEpiWarps) {
+        // ------------------------------------------------------------------ gathered A rows (two warps)
+        const int piece = lane & 7;
+        const int row0 = (warp - 2 - kEpiWarps) * (BM / kGatherWarps) + (lane >> 3);
+        constexpr int ROWS = BM / kGatherWarps / 4;          // rows per lane: row0 + 4 j
+        const uint8_t* src = (const uint8_t*)p.gather_src + piece * 16;
         const int64_t ld_bytes = p.gather_ld * 2;
-        auto hand_over = [&]() {                           // the copies of the oldest slice in flight have landed
-            fence_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&full_bar[sig]);
-            sig = sig + 1 == STAGES ? 0 : sig + 1;
-        };
+        uint32_t s = 0, phase = 1;
         for (int t = blockIdx.x; t < total; t += gridDim.x) {
             const Tile tl = get_tile(p, BN, t, tiles_m, tiles_n);
-            __syncwarp();
-            for (int q = lane; q < BM; q += 32) {
-                const int g = p.gather_rows[tl.m0 + q];
-                row_tok[q] = g < 0 ? -1 : g / p.gather_div;
+            const uint8_t* from[ROWS];                       // this tile's source rows (null: a zero row)
+#pragma unroll
+            for (int j = 0; j < ROWS; ++j) {
+                const int g = p.gather_rows[tl.m0 + row0 + 4 * j];
+                from[j] = g < 0 ? nullptr : src + (int64_t)(g / p.gather_div) * ld_bytes;
             }
-            __syncwarp();
             for (int kb = 0; kb < tl.num_kb; ++kb, s = (s + 1 == STAGES ? 0 : s + 1), phase ^= (s == 0)) {
                 mbar_wait_lean(&empty_bar[s], phase, dead, p.status);
-                const int k0 = kb * BK;
-                if (lane == 0) {
-                    mbar_expect_tx(&full_bar[s], B_BYTES);
-                    tma_load_2d(smem_b + s * B_BYTES, &map_b, &full_bar[s], k0, tl.expert * p.b_rows_per_expert + tl.n0);
+                const uint32_t base = smem_u32(smem_a + s * A_BYTES);
+                const int k0_bytes = kb * BK * 2;
+#pragma unroll
+                for (int j = 0; j < ROWS; ++j) {
+                    const int row = row0 + 4 * j;
+                    cp_async_16(base + row * 128 + ((piece ^ (row & 7)) << 4), from[j] ? from[j] + k0_bytes : src, from[j] ? 16u : 0u);
                 }
-                gather_kmajor_slice(smem_a + s * A_BYTES, src, ld_bytes, k0 * 2, row_tok, lane);
-                cp_async_commit();
-                if (++issued > kGatherLag) {
-                    cp_async_wait<kGatherLag>();
-                    hand_over();
+                cp_async_arrive(&full_bar[s]);
+            }
+        }
+    } else if (warp == 0 && GATHER) {
+        // ------------------------------------------------------------------ TMA producer of B beside the gathered A rows
+        if (lane == 0) {
+            uint32_t s = 0, phase = 1;
+            for (int t = blockIdx.x; t < total; t += gridDim.x) {
+                const Tile tl = get_tile(p, BN, t, tiles_m, tiles_n);
+                for (int kb = 0; kb < tl.num_kb; ++kb, s = (s + 1 == STAGES ? 0 : s + 1), phase ^= (s == 0)) {
+                    mbar_wait_lean(&empty_bar[s], phase, dead, p.status);
+                    mbar_expect_tx(&full_bar[s], B_BYTES);
+                    tma_load_2d(smem_b + s * B_BYTES, &map_b, &full_bar[s], kb * BK, tl.expert * p.b_rows_per_expert + tl.n0);
                 }
             }
         }
-        cp_async_wait<0>();
-        for (uint32_t left = issued < kGatherLag ? issued : kGatherLag; left > 0; --left) hand_over();
     } else if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -164,6 +169,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     mbar_wait_lean(&full_bar[stage], phase, dead, p.status);
+                    if (GATHER) fence_async_smem();        // the gathered rows were written through the generic proxy
                     tc_fence_after();
                     const uint64_t da = da0 + stage * (A_BYTES >> 4), db = db0 + stage * (B_BYTES >> 4);
                     umma_bf16(d_tmem, da, db, idesc, kb != 0);
@@ -176,7 +182,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 else mbar_arrive(&tmem_full_bar[acc]);
             }
         }
-    } else {
+    } else if (warp < 2 + kEpiWarps) {
         // ------------------------------------------------------------------ epilogue (warps 2..17)
         const int quad = warp & 3;                     // TMEM lanes 32*quad .. 32*quad+31
         constexpr int COLS_PER_WARP = BN / (kEpiWarps / 4);
@@ -287,7 +293,7 @@ template <int BN, int STAGES, bool AK, bool BKM, bool TMA_EPI, bool GATHER = fal
 cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mz,
                    const CUtensorMap& mb2, const TcParams& p, int max_tiles, cudaStream_t stream) {
     constexpr size_t smem = STAGES * (BM * BK * 2 + BN * BK * 2) + (TMA_EPI ? kEpiWarps * 2 * kBoxBytes : 0) +
-                            (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + (GATHER ? BM * 4 : 0) + 1024;
+                            (2 * STAGES + 4 + kEpiWarps) * 8 + 16 + 1024;
     static PerDeviceOnce once;
     auto kernel = gemm_tc_kernel<BN, STAGES, AK, BKM, TMA_EPI, GATHER>;
     int dev;
@@ -297,7 +303,7 @@ cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorM
         once.mark(dev);
     }
     const int grid = max_tiles < sm_count() ? max_tiles : sm_count();
-    kernel<<<grid, kThreadsV2, smem, stream>>>(ma, mb, mc, mz, mb2, p);
+    kernel<<<grid, GATHER ? kThreadsGather : kThreadsV2, smem, stream>>>(ma, mb, mc, mz, mb2, p);
     return cudaGetLastError();
 }
 

@@ -18,6 +18,15 @@
 // runs at most two accumulators ahead of the epilogue: kRing = 16 entries are never overwritten while in use.
 // The counter is left at zero by the last pair to finish, ready for the next launch on the stream.
 // Mainloop, barriers and accumulator double-buffering are those of gemm_tc2.cu (both operands MN-major).
+//
+// GATHER: the rows of B are not read from a grouped copy but gathered (the dispatch fused into this operand load: for
+// dW1 the rows of B are rows of x', row k of the grouped order being row gather_rows[k] / gather_div of x', zeros on
+// padding rows).  The producer thread of each CTA then issues the TMA boxes of A only, and two extra warps per CTA
+// follow the item ring and copy this CTA's 128 columns of the 64 gathered rows of every k slice with 16-byte
+// asynchronous copies into the swizzled MN-major layout.  Each copying thread arrives on the stage's barrier when its
+// copies have landed: in the leader CTA on the "full" barrier itself, in the peer on a barrier of its own that a relay
+// thread (the peer's otherwise idle MMA-warp thread) waits on before it passes a proxy fence and arrives, with release
+// at cluster scope, on the leader's "full" barrier; the MMA thread acquires at cluster scope and passes a proxy fence.
 #include "tc_pair.cuh"
 
 namespace bigmac {
@@ -77,7 +86,8 @@ __device__ void groupk_plan(const int32_t* poffsets, int E, int per, int pairs, 
     }
 }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsV2, 1)
+template <bool GATHER>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GATHER ? kThreadsGather : kThreadsV2, 1)
 gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p,
                       int* __restrict__ sched, float* __restrict__ ws, int32_t* __restrict__ plan_out) {
     constexpr int BH = BN / 2;
@@ -101,6 +111,7 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     int32_t* s_pp = (int32_t*)(tmem_slot + 4);               // [E + 1] parts before expert e
     int32_t* s_ss = s_pp + p.num_experts + 1;                // [E + 1] workspace slots before expert e
     int32_t* s_off = s_ss + p.num_experts + 1;               // [E + 1] padded row offsets (a copy: the scheduler reads them per item)
+    uint64_t* gfull_bar = (uint64_t*)(((uintptr_t)(s_off + p.num_experts + 1) + 7) & ~(uintptr_t)7);   // [STAGES] peer CTA: its gathered rows landed (GATHER)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -114,7 +125,10 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     __syncthreads();
     if (warp == 0) groupk_plan(s_off, p.num_experts, per, num_clusters, s_pp, s_ss);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        // a gathered slice completes on the A boxes' bytes, on the leader's copying threads and on the peer's relay thread
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 2 + kGatherWarps * 32 : 1); mbar_init(&empty_bar[s], 1); }
+        if (GATHER)
+            for (int s = 0; s < STAGES; ++s) mbar_init(&gfull_bar[s], kGatherWarps * 32);
         for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], 2 * kEpiWarps); }
         for (int s = 0; s < kRing; ++s) mbar_init(&ring_bar[s], 1);
         *dead = 0;
@@ -134,7 +148,7 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     auto load_stage = [&](const Item& t, int kb, uint32_t it) {
         const int s = it % STAGES;
         mbar_wait_lean(&empty_bar[s], ((it / STAGES) & 1) ^ 1, dead, p.status);
-        if (leader) mbar_expect_tx(&full_bar[s], 2 * (A_BYTES + B_BYTES));
+        if (leader) mbar_expect_tx(&full_bar[s], GATHER ? 2 * A_BYTES : 2 * (A_BYTES + B_BYTES));
         const uint32_t bar = map_to_cta(&full_bar[s], 0);
         const int k0 = t.k_row0 + kb * BK;
         const int my_m0 = t.m0 + (int)rank * BM, my_n0 = t.n0 + (int)rank * BH;
@@ -142,11 +156,57 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         uint8_t* b_dst = smem_b + s * B_BYTES;
 #pragma unroll
         for (int c = 0; c < BM / 64; ++c) tma_load_2d_pair(a_dst + c * CHUNK_BYTES, &map_a, bar, my_m0 + 64 * c, k0);
+        if (GATHER) return;                                  // the rows of B are gathered by the copying warps
 #pragma unroll
         for (int c = 0; c < BH / 64; ++c) tma_load_2d_pair(b_dst + c * CHUNK_BYTES, &map_b, bar, my_n0 + 64 * c, k0);
     };
 
-    if (warp == 0) {
+    if (GATHER && warp >= 2 + kEpiWarps) {
+        // ---------------------------------------------------------- gathered B rows (two warps per CTA)
+        const int gw = warp - 2 - kEpiWarps;                    // rows 32 gw .. 32 gw + 31 of every slice
+        const int piece = lane & 7, chunk = (lane >> 3) & 1, r0 = lane >> 4;
+        const uint8_t* src = (const uint8_t*)p.gather_src + chunk * 128 + piece * 16;
+        const int64_t ld_bytes = p.gather_ld * 2;
+        uint32_t it = 0;
+        for (uint32_t i = 0;; ++i) {
+            mbar_wait_cluster(&ring_bar[i % kRing], (i / kRing) & 1, dead, p.status);
+            const Item t = ring[i % kRing];
+            if (t.num_kb < 0 || *dead) break;
+            const uint8_t* col = src + (int64_t)(t.n0 + (int)rank * BH) * 2;
+            int idx = p.gather_rows[t.k_row0 + 32 * gw + lane];     // lane j: the source of row 32 gw + j of the slice
+            for (int kb = 0; kb < t.num_kb; ++kb, ++it) {
+                const int s = it % STAGES;
+                const int tok = idx < 0 ? -1 : idx / p.gather_div;
+                if (kb + 1 < t.num_kb) idx = p.gather_rows[t.k_row0 + (kb + 1) * BK + 32 * gw + lane];   // one slice ahead
+                mbar_wait_lean(&empty_bar[s], ((it / STAGES) & 1) ^ 1, dead, p.status);
+                const uint32_t base = smem_u32(smem_b + s * B_BYTES) + chunk * CHUNK_BYTES;
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    const int j = r0 + 2 * q, kr = 32 * gw + j;
+                    const int tk = __shfl_sync(0xffffffffu, tok, j);
+                    cp_async_16(base + kr * 128 + ((piece ^ (kr & 7)) << 4), tk < 0 ? col : col + (int64_t)tk * ld_bytes, tk < 0 ? 0u : 16u);
+                }
+                cp_async_arrive(leader ? &full_bar[s] : &gfull_bar[s]);
+            }
+        }
+    } else if (GATHER && warp == 1 && !leader) {
+        // ---------------------------------------------------------- relay (peer CTA): gathered rows landed -> leader's barrier
+        if (lane == 0) {
+            const uint32_t leader_full = map_to_cta(full_bar, 0);
+            uint32_t it = 0;
+            for (uint32_t i = 0;; ++i) {
+                mbar_wait_cluster(&ring_bar[i % kRing], (i / kRing) & 1, dead, p.status);
+                const int num_kb = ring[i % kRing].num_kb;
+                if (num_kb < 0 || *dead) break;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const uint32_t s = it % STAGES;
+                    mbar_wait_lean(&gfull_bar[s], (it / STAGES) & 1, dead, p.status);
+                    fence_async_smem();
+                    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(leader_full + s * 8u) : "memory");
+                }
+            }
+        }
+    } else if (warp == 0) {
         if (lane == 0) {
             uint32_t it = 0;
             if (leader) {
@@ -219,7 +279,12 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    mbar_wait_lean(&full_bar[stage], phase, dead, p.status);
+                    if (GATHER) {                      // the peer's relay releases at cluster scope; gathered rows are generic-proxy writes
+                        mbar_wait_cluster(&full_bar[stage], phase, dead, p.status);
+                        fence_async_smem();
+                    } else {
+                        mbar_wait_lean(&full_bar[stage], phase, dead, p.status);
+                    }
                     tc_fence_after();
                     const uint64_t da = da0 + stage * (A_BYTES >> 4), db = db0 + stage * (B_BYTES >> 4);
                     umma_bf16_pair(d_tmem, da, db, idesc, kb != 0);
@@ -231,7 +296,7 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 umma_commit_pair(&tmem_full_bar[acc]);
             }
         }
-    } else {
+    } else if (warp < 2 + kEpiWarps) {
         // ------------------------------------------------------------------ epilogue (warps 2..17, both CTAs)
         const int quad = warp & 3;
         constexpr int COLS_PER_WARP = BN / (kEpiWarps / 4);
@@ -337,28 +402,34 @@ cudaError_t gemm_tc_groupk(const GemmArgs& g, int* status, int* sched, void* ws,
     if (g.M <= 0 || g.N <= 0 || g.num_experts <= 0) return cudaSuccess;
     const int E = g.num_experts;
     CUtensorMap ma, mb;
+    const bool gather = g.gather_rows != nullptr;            // B's rows are gathered by the producer warps: no tensor map for B
+    if (gather && ((g.ldb * 2) % 16 || (uintptr_t)g.B % 16 || g.N % 128)) return cudaErrorInvalidValue;
     bool ok = make_map(&ma, g.A, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.lda, 64, BK);
-    ok &= make_map(&mb, g.B, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.ldb, 64, BK);
+    ok &= gather ? make_map(&mb, g.B, (uint64_t)g.N, 1, (uint64_t)g.ldb, 64, 1)         // placeholder, never used
+                 : make_map(&mb, g.B, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.ldb, 64, BK);
     if (!ok) return cudaErrorInvalidValue;
     TcParams p{};
     p.C = g.C; p.ldc = g.ldc; p.c_stride = g.c_stride; p.M = g.M; p.N = g.N; p.K = g.K;
     p.accumulate = g.accumulate; p.epilogue = EPI_NONE; p.group = GROUP_K; p.num_experts = E; p.poffsets = g.poffsets;
     p.status = status; p.split_k = 1; p.b2_first_kb = -1; p.n_split = -1; p.epi_parts = epi_parts_default(g.epi_parts);
+    p.gather_rows = g.gather_rows; p.gather_src = g.B; p.gather_ld = g.ldb; p.gather_div = g.gather_div > 0 ? g.gather_div : 1;
     float* slots = (float*)ws;
     int32_t* plan = (int32_t*)((char*)ws + (((size_t)kGroupKSlots * g.M * g.N * sizeof(float) + 255) & ~(size_t)255));
     constexpr size_t kMaxSmem = 232448;
     const size_t smem = STAGES * (BM * BK * 2 + (BN / 2) * BK * 2) + (2 * STAGES + 4 + kRing) * 8 + kRing * sizeof(Item) + 16 +
-                        3 * (size_t)(E + 1) * 4 + 1024;
+                        3 * (size_t)(E + 1) * 4 + 8 + STAGES * 8 + 1024;
     if (smem > kMaxSmem) return cudaErrorInvalidConfiguration;
     static PerDeviceOnce once;
     int dev;
     if (once.needed(&dev)) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_groupk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_groupk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_groupk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem);
         if (e != cudaSuccess) return e;
         once.mark(dev);
     }
     const int clusters = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
-    gemm_tc_groupk_kernel<<<2 * clusters, kThreadsV2, smem, stream>>>(ma, mb, p, sched, slots, plan);
+    if (gather) gemm_tc_groupk_kernel<true><<<2 * clusters, kThreadsGather, smem, stream>>>(ma, mb, p, sched, slots, plan);
+    else gemm_tc_groupk_kernel<false><<<2 * clusters, kThreadsV2, smem, stream>>>(ma, mb, p, sched, slots, plan);
     return cudaGetLastError();
 }
 

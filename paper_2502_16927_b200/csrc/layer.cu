@@ -263,9 +263,8 @@ int check_call(const bigmac_layer* L, int32_t T) {
     return BIGMAC_OK;
 }
 
-// Per-expert weight gradient (contraction over the expert's rows): on the tensor-core path the balanced kernel
-// (dynamic work items, long experts in parts), else the generic grouped contraction.
-int expert_weight_grad(const bigmac_layer* L, int id, const GemmArgs& g, float* splitk_ws, cudaStream_t st) {
+// Does the per-expert weight gradient run on the balanced kernel (dynamic work items, long experts in parts)?
+bool uses_groupk(const bigmac_layer* L, int id, const GemmArgs& g) {
     const bool enabled = switches().groupk != 0;
     const bool tc = L->cfg.dtype == BIGMAC_BF16 && L->use_tc && ((L->tc_mask >> id) & 1u);
     // below about 16 k slices of work per CTA pair the items are too short for dynamic hand-out to pay (measured:
@@ -273,7 +272,43 @@ int expert_weight_grad(const bigmac_layer* L, int id, const GemmArgs& g, float* 
     const int64_t tiles = (int64_t)((g.M + 255) / 256) * ((g.N + 255) / 256);
     const bool enough = (L->cfg.flags & BIGMAC_FLAG_DYNAMIC_WGRAD) ||
                         (int64_t)(g.K / 64) * tiles >= 16 * (int64_t)(gemm_tc_sm_count() / 2);
-    if (enabled && tc && enough && gemm_tc_groupk_supported(g)) {
+    return enabled && tc && enough && gemm_tc_groupk_supported(g);
+}
+
+// dW1_e[q,c'] = sum over the rows of expert e of dz[row,q] xg[row,c'] as a contraction request (xg: the grouped rows,
+// or with gather_rows the ungrouped matrix they are copies of).
+GemmArgs dw1_request(const Dims& m, const void* dz, const void* rows, const Tables& tb, void* dw1, bool acc) {
+    GemmArgs g;
+    g.A = dz; g.lda = m.h; g.a_kmajor = false; g.B = rows; g.ldb = m.r; g.b_kmajor = false;
+    g.C = dw1; g.ldc = m.r; g.c_stride = (int64_t)m.h * m.r; g.M = m.h; g.N = m.r; g.K = (int)m.P;
+    g.group = GROUP_K; g.num_experts = m.E; g.poffsets = tb.poffsets; g.accumulate = acc;
+    return g;
+}
+
+// Is the dispatch fused into its consumers' operand loads (F5 of the forward disappears as a launch, the grouped
+// copy xg of x' is never written)?  Inference: expert GEMM1 gathers the rows of x' itself.  Training: so does the
+// weight gradient dW1, when it runs on the balanced kernel (the statically scheduled kernels read a grouped copy).
+// A pure function of the handle, T and the debug switches: a training forward and its backward must see the same
+// switches.
+bool dispatch_is_fused(const bigmac_layer* L, const Dims& m, bool training) {
+    if (!switches().fuse_dispatch || !sigma_as_bytes(L) || m.r % 64) return false;
+    if (!training) {
+        const bool short_list = m.P / kPad <= 2 * (int64_t)gemm_tc_sm_count();
+        const bool mlp_fused = !m.bias && (switches().fused_mlp == 2 || (switches().fused_mlp == 1 && short_list)) &&
+                               fused_mlp_supported(m.r, m.h, m.dtype);
+        return !mlp_fused;
+    }
+    if (m.r % 128) return false;
+    Tables shape_only{};                                     // the kernel choice depends on shapes and alignment only:
+    void* const somewhere = (void*)(uintptr_t)256;           // stand-ins that are tested for presence and alignment, never read
+    shape_only.poffsets = (int32_t*)somewhere;
+    return uses_groupk(L, G_DW1, dw1_request(m, somewhere, somewhere, shape_only, somewhere, false));
+}
+
+// Per-expert weight gradient (contraction over the expert's rows): on the tensor-core path the balanced kernel
+// (dynamic work items, long experts in parts), else the generic grouped contraction.
+int expert_weight_grad(const bigmac_layer* L, int id, const GemmArgs& g, float* splitk_ws, cudaStream_t st) {
+    if (uses_groupk(L, id, g)) {
         { Stage stage(L, id, st); BIGMAC_CUDA(gemm_tc_groupk(g, L->status, L->status + 2, splitk_ws, st)); }
         { Stage stage(L, S_SPLITK_REDUCE, st); BIGMAC_CUDA(gemm_tc_groupk_finish(g, splitk_ws, st)); }
         return BIGMAC_OK;
@@ -406,7 +441,8 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     const bigmac_config_t& c = L->cfg;
 
     // A few tokens, inference: the whole forward in one cooperative kernel (weight streaming, no tensor cores)
-    if (!training && !m.cdac && !m.gate_low && !m.bias && m.cap == kNoCapacity && m.aux == 0 && sigma_as_bytes(L) && decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
+    if (!training && !m.cdac && !m.gate_low && !m.bias && m.cap == kNoCapacity && m.aux == 0 && sigma_as_bytes(L) &&
+        decode_forward_supported(m.T, m.d, m.r, m.h, m.E, m.k, m.dtype)) {
         {
             Stage s(L, S_DECODE, st);
             BIGMAC_CUDA(launch_decode_forward(x, W, y, b.logits, (float*)b.xg, (float*)b.a, (float*)b.u, b.tb.topk_idx,
@@ -440,14 +476,13 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         g.M = m.T; g.N = m.r; g.K = m.d;
         BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
     }
-    // F5 dispatch at width r.  Inference on the tensor-core path with the two expert GEMMs as separate launches: the
-    // dispatch is fused into expert GEMM1, whose producer warp gathers the rows of x' itself (slot_of_prow names the
-    // token of every grouped row, -1 the zero padding rows), so the grouped copy xg is never written.  A training
-    // forward keeps xg: the per-expert weight gradient dW1 contracts over it.
+    // F5 dispatch at width r - unless it is fused into its consumers: expert GEMM1's producer warp then gathers the
+    // rows of x' itself (slot_of_prow names the token of every grouped row, -1 the zero padding rows) and the grouped
+    // copy xg is never written.
     const bool short_list = m.P / kPad <= 2 * (int64_t)gemm_tc_sm_count();
     const bool mlp_fused_ = !training && !m.bias && (switches().fused_mlp == 2 || (switches().fused_mlp == 1 && short_list)) &&
                             sigma_as_bytes(L) && fused_mlp_supported(m.r, m.h, m.dtype);
-    const bool gather_dispatch = switches().fuse_dispatch && !training && !mlp_fused_ && sigma_as_bytes(L) && m.r % 64 == 0;
+    const bool gather_dispatch = dispatch_is_fused(L, m, training);
     if (!gather_dispatch) { Stage s(L, S_DISPATCH, st); BIGMAC_CUDA(launch_dispatch(b.x_lo, b.xg, b.tb, m.k, m.r, m.dtype, m.P, st)); }
     // Inference, low width r <= 256, up to two row tiles per SM: F6 + F7 in one kernel, the hidden activations stay on
     // the SM.  On long tile lists the two separate GEMMs are faster (the fused kernel is bound by the issue of its many
@@ -640,10 +675,12 @@ static int backward_launches(bigmac_layer_t* L, const void* x, const void* dy, i
         BIGMAC_CUDA(cudaEventRecord(L->fork_join[5], sd));
     }
     if (G->dw1) {   // dW1_e[q,c'] = sum_rows dz[row,q] xg[row,c']
-        GemmArgs g;
-        g.A = dz; g.lda = m.h; g.a_kmajor = false; g.B = b.xg; g.ldb = m.r; g.b_kmajor = false;
-        g.C = G->dw1; g.ldc = m.r; g.c_stride = (int64_t)m.h * m.r; g.M = m.h; g.N = m.r; g.K = (int)m.P;
-        g.group = GROUP_K; g.num_experts = m.E; g.poffsets = b.tb.poffsets; g.accumulate = acc;
+        GemmArgs g = dw1_request(m, dz, b.xg, b.tb, G->dw1, acc);
+        if (dispatch_is_fused(L, m, true)) {     // no grouped copy exists: the contraction gathers the rows of x' (Eq. 3: of x)
+            g.B = m.cdac ? x : b.x_lo;
+            g.gather_rows = b.tb.slot_of_prow;
+            g.gather_div = m.k;
+        }
         BIGMAC_TRY(expert_weight_grad(L, G_DW1, g, b.splitk_ws, st));
     }
     if (m.cdac) {

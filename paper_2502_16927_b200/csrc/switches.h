@@ -11,7 +11,10 @@ struct Switches {
     int fused_mlp = 1;      // inference: expert GEMM1 + sigma + GEMM2 in one kernel on short tile lists (0: never, 2: always)
     int epi_parts = 0;      // working epilogue warps per lane quadrant of plain epilogues (1, 2, 4; 0: the default, 2)
     int staged_stores = 1;  // wide bf16 outputs leave through shared-memory boxes and TMA stores (0: always 32-byte direct stores)
-    int fuse_dispatch = 1;  // expert GEMM1 gathers its rows from x' itself where supported (0: standalone dispatch kernel)
+    int fuse_dispatch = 0;  // 1: expert GEMM1 (and dW1) gather the rows of x' themselves, no dispatch launch, no grouped copy.
+                            // Off by default: the gathered operand loads (16-byte asynchronous copies by two extra warps)
+                            // feed the mainloop at half the rate of TMA boxes (large workload: expert GEMM1 1.08 ms against
+                            // 0.73 + 0.07 ms for the dispatch, dW1 1.20 against 0.47 ms)
     unsigned tc_mask = ~0u; // bit i: contraction i runs on tcgen05 (read when a handle is created)
 };
 

@@ -12,6 +12,10 @@
 namespace bigmac {
 namespace tc {
 
+constexpr int kEpiWarps = 16;
+constexpr uint32_t kBoxBytes = 32 * 64;                  // 32 rows x 32 bf16 columns
+constexpr uint32_t kBoxBytesZ = 32 * 64;                 // 32 rows x 64 sigma' bytes (two chunks)
+constexpr int kThreadsV2 = (2 + kEpiWarps) * 32;
 constexpr int BM = 128;          // UMMA M
 constexpr int BK = 64;           // bf16 elements per k slice = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
@@ -133,24 +137,16 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src, 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-constexpr int kGatherLag = 2;       // gathered k slices in flight behind the newest before the oldest is handed to the MMA warp
-
-// One 64-deep k slice of a K-major operand tile whose rows are gathered: row i of the 128-row tile is row tok[i] of
-// the source matrix (row stride ld_bytes; zeros where tok[i] < 0), written in the 128-byte-swizzled layout a TMA
-// load of the same box would produce (16-byte piece j of row i at piece j ^ (i & 7)).  Called by all lanes of a warp:
-// lane l moves piece l & 7 of rows (l >> 3) + 4 j, j = 0..31.
-__device__ __forceinline__ void gather_kmajor_slice(uint8_t* stage, const uint8_t* src, int64_t ld_bytes, int k0_bytes,
-                                                    const int32_t* tok, int lane) {
-    const int piece = lane & 7, r0 = lane >> 3;
-    const uint32_t base = smem_u32(stage);
-#pragma unroll 8
-    for (int j = 0; j < BM / 4; ++j) {
-        const int row = r0 + 4 * j;
-        const int t = tok[row];
-        const uint8_t* from = src + (int64_t)(t < 0 ? 0 : t) * ld_bytes + k0_bytes + piece * 16;
-        cp_async_16(base + row * 128 + ((piece ^ (row & 7)) << 4), from, t < 0 ? 0u : 16u);
-    }
+// Arrive on an mbarrier of this CTA once all asynchronous copies this thread has issued so far have landed (the
+// arrival is counted in the barrier's expected count: .noinc).
+__device__ __forceinline__ void cp_async_arrive(uint64_t* bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// Gathered operand rows are copied by kGatherWarps extra warps (the last warps of the CTA), 64 threads that each
+// arrive on the stage's "full" barrier when their copies have landed; the MMA thread passes a proxy fence between
+// that barrier and its first MMA on the stage (the copies are generic-proxy writes, the MMA reads through the async one).
+constexpr int kGatherWarps = 2;
+constexpr int kThreadsGather = kThreadsV2 + kGatherWarps * 32;
 
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
@@ -609,10 +605,6 @@ __device__ __forceinline__ Tile walk1_tile(const TcParams& p, int BN, const Tile
     return tl;
 }
 
-constexpr int kEpiWarps = 16;
-constexpr uint32_t kBoxBytes = 32 * 64;                  // 32 rows x 32 bf16 columns
-constexpr uint32_t kBoxBytesZ = 32 * 64;                 // 32 rows x 64 sigma' bytes (two chunks)
-constexpr int kThreadsV2 = (2 + kEpiWarps) * 32;
 
 
 // ------------------------------------------------------------------------------------------ host side

@@ -497,6 +497,7 @@ def test_inference_forward_with_the_dispatch_fused_into_expert_gemm1(case):
     inp = conditioned(w)
     dev = to_device(w, inp)
     binding.bigmac_debug_set("fused_mlp", 0)
+    binding.bigmac_debug_set("fuse_dispatch", 1)
     try:
         layer = make_layer(w)
         y, R = layer.forward(dev["x"], dev, training=False, want_routing=True)
@@ -512,3 +513,40 @@ def test_inference_forward_with_the_dispatch_fused_into_expert_gemm1(case):
     check_routing(R, rt)
     assert_within(w, float_errors(w, {"y": to_numpy(y)}, {"y": oracle.forward_tokens(inp, rt, w.act)["y"]}))
     assert torch.equal(y.view(torch.int16), y_plain.view(torch.int16))
+
+
+@pytest.mark.parametrize("case", [
+    dict(shape=dict(T=6000, d=256, r=256, h=512, E=16, k=2), bias="graded", flags=wl.FLAG_DYNAMIC_WGRAD),   # long and empty experts, parts
+    dict(shape=dict(T=333, d=128, r=384, h=256, E=5, k=5), bias=None, flags=wl.FLAG_DYNAMIC_WGRAD),         # ragged widths (384 = 256 + 128), k = E
+    dict(shape=dict(T=20000, d=256, r=256, h=256, E=24, k=2), bias=None, flags=wl.FLAG_DYNAMIC_WGRAD),      # balanced, many row tiles per expert
+    dict(shape=dict(T=9000, d=512, r=512, h=1024, E=8, k=4), bias=None, flags=0),                           # enough work for the balanced kernel by size
+])
+def test_training_step_with_the_dispatch_fused_into_its_consumers(case):
+    """Training forward + backward without a grouped copy of x': expert GEMM1 and the weight gradient dW1 gather the
+    rows of x' themselves.  Every output against the oracle, and bit for bit against the same step with the standalone
+    dispatch kernel (same operands, same arithmetic order)."""
+    import torch
+    from paper_2502_16927_b200 import binding
+
+    w = wl.Workload("fdt", dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=983, **case["shape"])
+    inp = conditioned(w)
+    if case["bias"] == "graded":
+        inp["b_gate"] = (2.5 * np.linspace(1.0, -1.0, w.E) ** 3).astype(np.float32)
+        margin.enforce_margin(w, inp, 1e-3)
+    binding.bigmac_debug_set("fuse_dispatch", 1)
+    try:
+        got = run_full(w, inp, case["flags"])
+        compare_full(w, inp, got)
+        prof_layer = make_layer(w, case["flags"])
+        dev = to_device(w, inp)
+        binding.bigmac_profile_enable(prof_layer.handle, True)
+        prof_layer.forward(dev["x"], dev, training=True)
+        stages = binding.bigmac_profile_read(prof_layer.handle)["stages"]
+        binding.bigmac_profile_enable(prof_layer.handle, False)
+        prof_layer.close()
+        assert "dispatch" not in stages, stages            # the fused path ran: no dispatch launch in the forward
+    finally:
+        binding.bigmac_debug_set("defaults")
+    plain = run_full(w, inp, case["flags"])
+    for key in ("y", "dx", "dw1", "dw2", "dw_up", "dw_down", "dw_gate", "db_gate"):
+        np.testing.assert_array_equal(got[key], plain[key], err_msg=key)
