@@ -307,7 +307,7 @@ int bigmac_ep_backward_dispatch(bigmac_layer_t *L, const void *x, int32_t T, con
  *    elements with BIGMAC_FLAG_GATE_LOW (the return code is the authority: the exact carve includes 256-byte
  *    alignment of every region); a larger problem is rejected with BIGMAC_ERR_TOO_LARGE and nothing is launched.
  *  - The first call on a device resolves the array's device address (once per device, with that device
- *    current); that first call should come before any stream capture.
+ *    current) and keeps it for the later ones.
  *  - All calls share the one array, and it keeps the previous call's contents (everything a call reads it
  *    has written itself first).  Two calls that overlap on the GPU - different streams, or different
  *    handles - race on it: serialise them. */
