@@ -345,7 +345,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         TcParams p2 = p;
                         p2.C = p.C2; p2.ldc = p.ldc2; p2.N = p.N2; p2.out_f32 = 1; p2.epilogue = EPI_NONE; p2.accumulate = 0;
                         const bool vec2 = (p.ldc2 % 8 == 0) && (((uintptr_t)p.C2) % 32 == 0);
-                        store_row_chunk(p2, v, (int64_t)row * p.ldc2, col0 - p.n_split, vec2);
+                        // a split contraction writes partial results: both outputs then share one fp32 matrix (ldc2 == ldc)
+                        const int64_t part2 = p.split_k > 1 ? tl.c_base : 0;
+                        store_row_chunk(p2, v, part2 + (int64_t)row * p.ldc2, col0 - p.n_split, vec2);
                     } else {
                         store_row_chunk(p, v, row_off, col0, vec_ok);
                     }
@@ -410,7 +412,8 @@ cudaError_t dispatch_pair(const GemmArgs& g, int* status, cudaStream_t stream) {
     }
     p.n_split = -1;
     if (g.C2) {      // second K-major B tensor feeding a second (fp32) output
-        if (!g.b_kmajor || g.group != GROUP_NONE || g.n_split % BN || TMA_EPI || g.B2 == nullptr || g.split_k > 1)
+        if (!g.b_kmajor || g.group != GROUP_NONE || g.n_split % BN || TMA_EPI || g.B2 == nullptr ||
+            (g.split_k > 1 && (!g.out_f32 || g.ldc2 != g.ldc)))
             return cudaErrorInvalidValue;
         ok &= make_map(&mb2, g.B2, (uint64_t)g.K, (uint64_t)g.N2, (uint64_t)g.ldb2, BK, BH);
         ok &= make_map(&mb, g.B, (uint64_t)g.K, (uint64_t)g.n_split, (uint64_t)g.ldb, BK, BH);

@@ -194,6 +194,9 @@ cudaError_t launch_grouped_colsum(const void* src, const int32_t* poffsets, floa
 // in the dtype, adding to the destination if `accumulate`.
 cudaError_t launch_splitk_reduce(const float* ws, int parts, int M, int N, void* dst1, int m_split, void* dst2, int m2,
                                  int dtype, bool accumulate, cudaStream_t stream);
+// [x' (bf16) | logits (fp32)] from the [parts][T][r + E] fp32 partial results of a split descend launch (r, E % 4 == 0).
+cudaError_t launch_descend_reduce(const float* ws, int parts, int T, int r, int E, void* x_lo, float* logits,
+                                  cudaStream_t stream);
 
 // Small-batch inference forward in one cooperative kernel (bf16, T <= 16): scratch logits [T,E], x_lo [T,r],
 // a [T*k,h], u [T*k,r] fp32; writes y, topk_idx, topk_w.  `barrier` is one device word owned by the handle.

@@ -38,6 +38,7 @@ struct Buffers {
     float* aux_loss;     // [1] saved: L_aux of the batch
     float* logits_saved; // [T,E] saved copy of the gate logits (only with a load-balancing loss)
     float* splitk_ws;    // fp32 partial results of the split weight-gradient contractions
+    float* descend_ws;   // few tokens: fp32 partial results [parts][T][r + E] of the split descend + logits launch
     float* bias_ws;      // fp32 row-slice sums of the expert-bias gradients (a region of their own: they run on the second stream)
 };
 
@@ -124,10 +125,23 @@ void carve_backward_scratch(Carver& cv, const Dims& m, Buffers& b) {
     b.bias_ws = bias_ws ? (float*)cv.take_bytes(bias_ws) : nullptr;
 }
 
+// Few tokens: the descend + gate-logits launch has a handful of output tiles, each walking all of d; its contraction
+// is then cut into parts (fp32 partial results, added by a small kernel) so that the SMs share the weight streaming.
+// A function of the shape only: every call of a handle with the same T takes the same path.
+int descend_split_parts(const Dims& m) {
+    if (m.T > 1024 || m.E % 4 || m.dtype != BIGMAC_BF16) return 1;
+    return choose_split_k(m.T, m.r + m.E, m.d);
+}
+void carve_descend_split(Carver& cv, const Dims& m, Buffers& b) {
+    const int parts = descend_split_parts(m);
+    b.descend_ws = parts > 1 ? cv.take<float>((size_t)parts * m.T * (m.r + m.E)) : nullptr;
+}
+
 size_t forward_scratch_bytes(const Dims& m, bool training) {
     Carver cv(nullptr);
     Buffers b{};
     carve_route_scratch(cv, m, b);
+    carve_descend_split(cv, m, b);
     if (!training) carve_saved(cv, m, b, false);
     return cv.total();
 }
@@ -430,6 +444,7 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
     Buffers b{};
     Carver cs(scratch);
     carve_route_scratch(cs, m, b);
+    carve_descend_split(cs, m, b);
     if (training) {
         Carver cv(saved);
         carve_saved(cv, m, b, true);
@@ -463,7 +478,15 @@ int bigmac_forward(bigmac_layer_t* L, const void* x, int32_t T, const bigmac_wei
         g.A = x; g.lda = m.d; g.B = W->w_down; g.ldb = m.d; g.C = b.x_lo; g.ldc = m.r;
         g.B2 = W->w_gate; g.ldb2 = m.d; g.n_split = m.r; g.C2 = b.logits; g.ldc2 = m.E; g.N2 = m.E;
         g.M = m.T; g.N = m.r + m.E; g.K = m.d;
-        BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
+        if (b.descend_ws) {                                   // few tokens: contraction in parts, then [x' | logits] from them
+            g.split_k = descend_split_parts(m); g.out_f32 = true;
+            g.C = b.descend_ws; g.ldc = m.r + m.E; g.C2 = b.descend_ws + m.r; g.ldc2 = m.r + m.E;
+            BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
+            Stage s(L, S_SPLITK_REDUCE, st);
+            BIGMAC_CUDA(launch_descend_reduce(b.descend_ws, g.split_k, m.T, m.r, m.E, b.x_lo, b.logits, st));
+        } else {
+            BIGMAC_TRY(gemm(L, G_DESCEND, g, st));
+        }
         BIGMAC_TRY(route_from_logits(L, m, W, b, st));
     } else {
         BIGMAC_TRY(run_routing(L, m, x, W, b, st));                               // F1-F3

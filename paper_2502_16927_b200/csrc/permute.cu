@@ -234,6 +234,29 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
     dst[0] = (T)acc.x; dst[1] = (T)acc.y; dst[2] = (T)acc.z; dst[3] = (T)acc.w;
 }
 
+// [x' | logits] from the fp32 partial results of a descend launch whose contraction was cut into parts (few tokens:
+// the launch has too few output tiles to fill the SMs otherwise).  ws is [parts][T][r + E]; the first r columns of a
+// row are added in part order and rounded to bf16 (x'), the other E stay fp32 (the gate logits).  r, E multiples of 4.
+__global__ void __launch_bounds__(256) descend_reduce_kernel(const float* __restrict__ ws, int parts, int T, int r, int E,
+                                                             __nv_bfloat16* __restrict__ x_lo, float* __restrict__ logits) {
+    const int n = r + E;
+    const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= (int64_t)T * n) return;
+    const int t = (int)(i / n), c = (int)(i - (int64_t)t * n);
+    float4 acc = *(const float4*)(ws + i);
+    for (int s = 1; s < parts; ++s) {
+        const float4 v = *(const float4*)(ws + (int64_t)s * T * n + i);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    if (c < r) {
+        __nv_bfloat162* dst = (__nv_bfloat162*)(x_lo + (int64_t)t * r + c);
+        dst[0] = __floats2bfloat162_rn(acc.x, acc.y);
+        dst[1] = __floats2bfloat162_rn(acc.z, acc.w);
+    } else {
+        *(float4*)(logits + (int64_t)t * E + (c - r)) = acc;
+    }
+}
+
 // Per-expert column sums (expert-bias gradients), in two deterministic steps so that one long segment does not
 // serialise.  Step 1, block (cg, e, s): slice s of kColsumSlices equal row ranges of expert e's padded segment; 32
 // column-threads x 8 row-lanes, a thread adds rows lane, lane + 8, ... of its 16-byte column vector in order, then the
@@ -369,6 +392,14 @@ cudaError_t launch_grouped_colsum(const void* src, const int32_t* poffsets, floa
         grouped_colsum_kernel<float><<<grid, 256, 0, stream>>>((const uint4*)src, poffsets, partial, vecs);
     const int64_t n = (int64_t)E * width;
     grouped_colsum_final_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(partial, out, n, width, accumulate ? 1 : 0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_descend_reduce(const float* ws, int parts, int T, int r, int E, void* x_lo, float* logits,
+                                  cudaStream_t stream) {
+    const int64_t quads = (int64_t)T * (r + E) / 4;
+    if (quads == 0) return cudaSuccess;
+    descend_reduce_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, stream>>>(ws, parts, T, r, E, (__nv_bfloat16*)x_lo, logits);
     return cudaGetLastError();
 }
 
