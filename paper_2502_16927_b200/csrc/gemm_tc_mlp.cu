@@ -20,7 +20,7 @@
 // double-buffer the activated chunk beside X in shared memory at r = 256.  The layer therefore uses this kernel
 // only on short tile lists (decode-sized batches), where it saves a launch and the HBM round trip of the
 // activations; on long lists the two separate GEMMs (N = 256 instructions) are faster.
-#include "tc_common.cuh"
+#include "tc_pair.cuh"
 
 namespace bigmac {
 
@@ -45,9 +45,23 @@ struct MlpParams {
     int* status;
 };
 
-__global__ void __launch_bounds__(kMlpThreads, 1)
-fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w1,
-                 const __grid_constant__ CUtensorMap map_w2, const MlpParams p) {
+// Arrive on a barrier of another CTA of the cluster, making this thread's earlier stores into that CTA visible to
+// whoever acquires the barrier at cluster scope.
+__device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_cluster_16B(uint32_t cluster_addr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+// SPLIT: a pair of CTAs (a cluster) shares every tile: CTA 0 walks the first half of the hidden chunks, CTA 1 the
+// second, so that a short tile list (a few hundred tokens: one tile per expert, far fewer tiles than SMs) streams
+// its weights through twice as many SMs.  CTA 1 hands its 128 x r fp32 partial result to CTA 0 through CTA 0's
+// shared memory (the X and W1 buffers, free once CTA 0's last GEMM1 of the tile is done: 128 r 2 + 2 x 64 r 2 bytes
+// = 128 r 4), CTA 0 adds it to its own and stores the tile.
+template <bool SPLIT>
+__device__ __forceinline__ void fused_mlp_body(const CUtensorMap& map_x, const CUtensorMap& map_w1, const CUtensorMap& map_w2,
+                                               const MlpParams& p) {
     const int KB1 = p.r / BK;                            // 64-deep k slices of GEMM1
     const uint32_t X_BYTES = (uint32_t)KB1 * BM * BK * 2;
     const uint32_t W1_BYTES = (uint32_t)KB1 * BH * BK * 2;
@@ -68,7 +82,10 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     uint64_t* acc1_full = bars + 10;    uint64_t* acc1_empty = bars + 14;      // [kAcc1] each
     uint64_t* a2_full = bars + 18;      uint64_t* a2_empty = bars + 20;
     uint64_t* acc2_full = bars + 22;    uint64_t* acc2_empty = bars + 23;
-    uint32_t* tmem_slot = (uint32_t*)(bars + 24);
+    uint64_t* peer_free = bars + 24;                     // SPLIT, in CTA 1: CTA 0's X and W1 buffers may be written
+    uint64_t* partial_full = bars + 25;                  // SPLIT, in CTA 0: CTA 1's partial result has arrived
+    uint64_t* tile_done = bars + 26;                     // SPLIT, in CTA 0: the partial result has been read
+    uint32_t* tmem_slot = (uint32_t*)(bars + 27);
     volatile int* dead = (volatile int*)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -81,6 +98,7 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         }
         for (int s = 0; s < kAcc1; ++s) { mbar_init(&acc1_full[s], 1); mbar_init(&acc1_empty[s], kMlpEpiWarps); }
         mbar_init(acc2_full, 1); mbar_init(acc2_empty, kMlpEpiWarps);
+        mbar_init(peer_free, 1); mbar_init(partial_full, kMlpEpiWarps); mbar_init(tile_done, kMlpEpiWarps);
         *dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -89,19 +107,25 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (SPLIT) cluster_sync_all();                        // the peer's barriers exist before anything signals them
     const uint32_t tmem_base = *tmem_slot;
     const int total = min(*p.n_tiles, p.max_tiles);
-    const int chunks = p.h / BH;
+    const uint32_t crank = SPLIT ? cluster_ctarank() : 0u;
+    const int first = SPLIT ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, stride = SPLIT ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int chunks = SPLIT ? p.h / BH / 2 : p.h / BH;   // this CTA's chunks of a tile: cbase, cbase + 1, ...
+    const int cbase = SPLIT ? (int)crank * chunks : 0;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: X and the W1 chunks
         if (lane == 0) {
             uint32_t g = 0, tl = 0;
-            int next_e = (int)blockIdx.x < total ? p.tile_expert[blockIdx.x] : 0;
-            for (int t = blockIdx.x; t < total; t += gridDim.x, ++tl) {
+            int next_e = first < total ? p.tile_expert[first] : 0;
+            for (int t = first; t < total; t += stride, ++tl) {
                 const int e = next_e;
-                if (t + (int)gridDim.x < total) next_e = p.tile_expert[t + gridDim.x];
+                if (t + stride < total) next_e = p.tile_expert[t + stride];
                 mbar_wait(x_empty, (tl & 1) ^ 1, dead, p.status);
+                // CTA 0 of a pair: X and W1 buffers hold the peer's partial result until the epilogue has read it
+                if (SPLIT && crank == 0 && tl > 0) mbar_wait(tile_done, (tl - 1) & 1, dead, p.status);
                 mbar_expect_tx(x_full, X_BYTES);
                 for (int kb = 0; kb < KB1; ++kb) tma_load_2d(s_x + kb * (BM * BK * 2), &map_x, x_full, kb * BK, t * BM);
                 for (int c = 0; c < chunks; ++c, ++g) {
@@ -110,7 +134,7 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_expect_tx(&w1_full[s], W1_BYTES);
                     for (int kb = 0; kb < KB1; ++kb)
                         tma_load_2d(s_w1 + s * W1_BYTES + kb * (BH * BK * 2), &map_w1, &w1_full[s], kb * BK,
-                                    e * p.b1_rows_per_expert + c * BH);
+                                    e * p.b1_rows_per_expert + (cbase + c) * BH);
                 }
             }
         }
@@ -119,15 +143,15 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         // thread: a W2 buffer frees only when GEMM2 two chunks back is done, and the W1 loads must not queue behind that)
         if (lane == 0) {
             uint32_t g = 0;
-            int next_e = (int)blockIdx.x < total ? p.tile_expert[blockIdx.x] : 0;
-            for (int t = blockIdx.x; t < total; t += gridDim.x) {
+            int next_e = first < total ? p.tile_expert[first] : 0;
+            for (int t = first; t < total; t += stride) {
                 const int e = next_e;
-                if (t + (int)gridDim.x < total) next_e = p.tile_expert[t + gridDim.x];
+                if (t + stride < total) next_e = p.tile_expert[t + stride];
                 for (int c = 0; c < chunks; ++c, ++g) {
                     const int s = g & 1;
                     mbar_wait(&w2_empty[s], ((g >> 1) & 1) ^ 1, dead, p.status);
                     mbar_expect_tx(&w2_full[s], W2_BYTES);
-                    tma_load_2d(s_w2 + s * W2_BYTES, &map_w2, &w2_full[s], c * BH, e * p.b2_rows_per_expert);
+                    tma_load_2d(s_w2 + s * W2_BYTES, &map_w2, &w2_full[s], (cbase + c) * BH, e * p.b2_rows_per_expert);
                 }
             }
         }
@@ -181,7 +205,7 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             }
             __syncwarp();
         };
-        for (int t = blockIdx.x; t < total; t += gridDim.x, ++tl) {
+        for (int t = first; t < total; t += stride, ++tl) {
             mbar_spin(x_full, tl & 1, dead, p.status);
             for (int c = 0; c < kAhead && c < chunks; ++c) gemm1(g + c, c);
             for (int c = 0; c < chunks; ++c, ++g) {
@@ -197,12 +221,15 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const int cpart = (warp - kFirstEpiWarp) >> 2;   // 16 of the chunk's 64 columns
         const int row_in_tile = quad * 32 + lane;
         uint32_t g = 0, tl = 0;
-        for (int t = blockIdx.x; t < total; t += gridDim.x, ++tl) {
+        for (int t = first; t < total; t += stride, ++tl) {
             for (int c = 0; c < chunks; ++c, ++g) {
                 const int s = g & 1, a = g & (kAcc1 - 1);
                 const uint32_t ph = (g >> 1) & 1;
                 mbar_spin(&acc1_full[a], (g / kAcc1) & 1, dead, p.status);
                 tc_fence_after();
+                // the tile's last GEMM1 is done: nothing reads this CTA's X and W1 buffers any more, the peer may write
+                if (SPLIT && crank == 0 && c == chunks - 1 && warp == kFirstEpiWarp && lane == 0)
+                    mbar_arrive_cluster(map_to_cta(peer_free, 1));
                 float v[16];
                 tmem_load_16_nowait(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a * BH + cpart * 16), (uint32_t*)v);
                 tmem_load_wait();
@@ -228,14 +255,46 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             const int cols = p.r / 4;                                   // per warp: 16, 32, 48 or 64
             __nv_bfloat16* out = (__nv_bfloat16*)p.U + ((int64_t)t * BM + row_in_tile) * p.r + cpart * cols;
             const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(kAcc1 * BH + cpart * cols);
-            for (int j = 0; j < cols; j += 16) {
-                float v[16];
-                tmem_load_16_nowait(t_addr + j, (uint32_t*)v);
-                tmem_load_wait();
-                uint32_t w[8];
+            // SPLIT: the partial result sits in CTA 0's X / W1 buffers as 16-byte pieces [column / 4][row] (neighbouring
+            // lanes, i.e. rows, at neighbouring addresses)
+            const int piece0 = cpart * (cols / 4);
+            if (SPLIT && crank == 1) {
+                mbar_wait_cluster(peer_free, tl & 1, dead, p.status);
+                const uint32_t dst = map_to_cta(s_x, 0);
+                for (int j = 0; j < cols; j += 16) {
+                    float v[16];
+                    tmem_load_16_nowait(t_addr + j, (uint32_t*)v);
+                    tmem_load_wait();
 #pragma unroll
-                for (int i = 0; i < 8; ++i) w[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
-                st_global_32B(out + j, w);
+                    for (int q = 0; q < 4; ++q)
+                        st_cluster_16B(dst + (uint32_t)(((piece0 + j / 4 + q) * BM + row_in_tile) * 16), v[4 * q], v[4 * q + 1],
+                                       v[4 * q + 2], v[4 * q + 3]);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive_release_cluster(map_to_cta(partial_full, 0));
+            } else {
+                if (SPLIT) mbar_wait_cluster(partial_full, tl & 1, dead, p.status);
+                for (int j = 0; j < cols; j += 16) {
+                    float v[16];
+                    tmem_load_16_nowait(t_addr + j, (uint32_t*)v);
+                    tmem_load_wait();
+                    if (SPLIT) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float4 o = *(const float4*)(s_x + ((piece0 + j / 4 + q) * BM + row_in_tile) * 16);
+                            v[4 * q] += o.x; v[4 * q + 1] += o.y; v[4 * q + 2] += o.z; v[4 * q + 3] += o.w;
+                        }
+                    }
+                    uint32_t w[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) w[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+                    st_global_32B(out + j, w);
+                }
+                if (SPLIT) {                                 // these reads come before the next tile's TMA writes
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tile_done);
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -244,10 +303,22 @@ fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     }
     tc_fence_before();
     __syncthreads();
+    if (SPLIT) cluster_sync_all();                        // nobody leaves while the peer may still signal or write here
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
+}
+
+__global__ void __launch_bounds__(kMlpThreads, 1)
+fused_mlp_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w1,
+                 const __grid_constant__ CUtensorMap map_w2, const MlpParams p) {
+    fused_mlp_body<false>(map_x, map_w1, map_w2, p);
+}
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMlpThreads, 1)
+fused_mlp_split_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w1,
+                       const __grid_constant__ CUtensorMap map_w2, const MlpParams p) {
+    fused_mlp_body<true>(map_x, map_w1, map_w2, p);
 }
 
 }  // namespace
@@ -271,17 +342,24 @@ cudaError_t launch_fused_mlp(const void* xg, const void* w1, const void* w2, voi
     p.tile_expert = tile_expert; p.n_tiles = n_tiles; p.max_tiles = (int)(max_rows / BM); p.status = status;
     const int kb1 = r / BK;
     const size_t smem = (size_t)kb1 * BM * BK * 2 + 2 * (size_t)kb1 * BH * BK * 2 + 2 * (size_t)r * BH * 2 + 2 * (size_t)BM * BH * 2 +
-                        24 * 8 + 16 + 1024;
+                        27 * 8 + 16 + 1024;
     static PerDeviceOnce once;
     int dev;
     if (once.needed(&dev)) {
         cudaError_t e = cudaFuncSetAttribute(fused_mlp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(fused_mlp_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
         if (e != cudaSuccess) return e;
         once.mark(dev);
     }
-    const int grid = p.max_tiles < sm_count() ? p.max_tiles : sm_count();
-    if (grid <= 0) return cudaSuccess;
-    fused_mlp_kernel<<<grid, kMlpThreads, smem, stream>>>(mx, m1, m2, p);
+    if (p.max_tiles <= 0) return cudaSuccess;
+    // at most one tile per SM and an even number of hidden chunks: two SMs per tile, half of the chunks each
+    if (p.max_tiles <= sm_count() && (h / BH) % 2 == 0) {
+        const int pairs = p.max_tiles < sm_count() / 2 ? p.max_tiles : sm_count() / 2;
+        fused_mlp_split_kernel<<<2 * pairs, kMlpThreads, smem, stream>>>(mx, m1, m2, p);
+    } else {
+        const int grid = p.max_tiles < sm_count() ? p.max_tiles : sm_count();
+        fused_mlp_kernel<<<grid, kMlpThreads, smem, stream>>>(mx, m1, m2, p);
+    }
     return cudaGetLastError();
 }
 

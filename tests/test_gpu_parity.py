@@ -423,6 +423,35 @@ def test_small_batch_inference_forward(T, shape):
     layer.close()
 
 
+@pytest.mark.parametrize("T", [17, 64, 200, 512, 1024])
+@pytest.mark.parametrize("shape", [
+    dict(d=2048, r=256, h=1024, E=64, k=8),        # the decode configuration
+    dict(d=512, r=128, h=256, E=12, k=3),          # four hidden chunks, two per CTA of a pair
+])
+def test_inference_forward_of_a_few_hundred_tokens(T, shape):
+    """Inference forward above the one-kernel limit at decode-like sizes: the descend + logits contraction runs in
+    parts (fp32 partial results, added by a small kernel) and the experts run on CTA pairs that share a tile's hidden
+    chunks.  y and the routing tables against the oracle; two calls agree bit for bit."""
+    import torch
+
+    w = wl.Workload("decode", T=T, dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=700 + T, **shape)
+    inp = conditioned(w)
+    inp["b_gate"] = (np.linspace(-0.2, 0.2, w.E)).astype(np.float32)
+    margin.enforce_margin(w, inp, 1e-3)
+    dev = to_device(w, inp)
+    layer = make_layer(w)
+    y, R = layer.forward(dev["x"], dev, training=False, want_routing=True)
+    y2 = layer.forward(dev["x"], dev, training=False)
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    rt = oracle.route(inp, w.k)
+    check_routing(R, rt)
+    ref = oracle.forward_tokens(inp, rt, w.act)["y"]
+    assert_within(w, float_errors(w, {"y": to_numpy(y)}, {"y": ref}))
+    assert torch.equal(y, y2)
+    layer.close()
+
+
 @pytest.mark.parametrize("case", [
     dict(T=300, d=128, r=64, h=192, E=5, k=2, act=wl.ACT_GELU_ERF),      # narrowest width, three hidden chunks, ragged segments
     dict(T=1000, d=256, r=192, h=320, E=16, k=4, act=wl.ACT_RELU),       # widths that are odd multiples of 64
