@@ -76,6 +76,7 @@ const char *bigmac_profile_slot_name(int slot);
  *   "groupk" 0/1         never / where it pays: the dynamically scheduled per-expert weight-gradient kernel (default 1)
  *   "fused_mlp" 0/1/2    inference expert GEMM1 + sigma + GEMM2 in one kernel never / on short tile lists / always (default 1)
  *   "epi_parts" 0/1/2/4  working epilogue warps per lane quadrant of plain epilogues (0 = default choice, 2)
+ *   "chain" 0/1          kernels launched with programmatic stream serialisation (set-up overlaps the predecessor) (default 1)
  *   "staged_stores" 0/1  wide bf16 outputs by 32-byte direct stores / through shared-memory boxes and TMA stores (default 1)
  *   "fuse_dispatch" 0/1  standalone dispatch kernel / the dispatch fused into its consumers: expert GEMM1 and the weight
  *                        gradient dW1 gather the rows of x' themselves, no grouped copy is written (default 0: measured slower)

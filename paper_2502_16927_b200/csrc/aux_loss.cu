@@ -52,6 +52,8 @@ __device__ __forceinline__ void token_range(int T, int warp, int& t0, int& t1) {
 __global__ void __launch_bounds__(256) aux_prob_sums_kernel(const float* __restrict__ logits,
                                                                        const float* __restrict__ b_gate, int T, int E,
                                                                        float* __restrict__ partial) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     extern __shared__ float acc[];                   // [warps][E]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
     for (int i = threadIdx.x; i < warps * E; i += blockDim.x) acc[i] = 0.0f;
@@ -78,6 +80,8 @@ __global__ void __launch_bounds__(256) aux_prob_sums_kernel(const float* __restr
 __global__ void __launch_bounds__(1024) aux_loss_final_kernel(const float* __restrict__ partial,
                                                               const int32_t* __restrict__ counts_chosen, int chunks, int T,
                                                               int E, int k, float coef, float* __restrict__ loss) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     __shared__ float part[1024];
     __shared__ float term[1024];
     const int groups = 1024 / E, g = threadIdx.x / E, e = threadIdx.x - g * E;      // E <= 1024: at least one group
@@ -111,6 +115,8 @@ __global__ void __launch_bounds__(256) gate_bwd_aux_kernel(float* __restrict__ d
                                                                       const float* __restrict__ b_gate, float coef,
                                                                       T* __restrict__ dlogits, float* __restrict__ aux_partial,
                                                                       int n_tokens, int E, int width, int ld, int k) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     extern __shared__ float smem[];                  // [warps][E] column sums, [warps][E] the row being built, [E] f
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
     float* acc = smem;
@@ -173,8 +179,8 @@ cudaError_t launch_aux_loss(const float* logits, const float* b_gate, const int3
                             float coef, float* partial, float* loss, cudaStream_t stream) {
     if (T == 0) return cudaMemsetAsync(loss, 0, sizeof(float), stream);
     const int warps = aux_warps(E);
-    aux_prob_sums_kernel<<<kAuxChunks, warps * 32, sizeof(float) * warps * E, stream>>>(logits, b_gate, T, E, partial);
-    aux_loss_final_kernel<<<1, 1024, 0, stream>>>(partial, counts_chosen, kAuxChunks, T, E, k, coef, loss);
+    (void)launch_chained(aux_prob_sums_kernel, kAuxChunks, warps * 32, sizeof(float) * warps * E, stream, logits, b_gate, T, E, partial);
+    (void)launch_chained(aux_loss_final_kernel, 1, 1024, 0, stream, partial, counts_chosen, kAuxChunks, T, E, k, coef, loss);
     return cudaGetLastError();
 }
 
@@ -185,11 +191,11 @@ cudaError_t launch_gate_bwd_aux(float* dp, const Tables& tb, void* dlogits, cons
     const int warps = aux_warps(E);
     const size_t smem = sizeof(float) * (2 * warps + 1) * E;          // at most 36 KB (E <= 1024)
     if (dtype == BIGMAC_BF16)
-        gate_bwd_aux_kernel<__nv_bfloat16><<<kAuxChunks, warps * 32, smem, stream>>>(
+        (void)launch_chained(gate_bwd_aux_kernel<__nv_bfloat16>, kAuxChunks, warps * 32, smem, stream, 
             dp, tb.topk_w, tb.topk_idx, tb.counts_chosen, logits, b_gate, coef, (__nv_bfloat16*)dlogits, aux_partial, T, E,
             width, ld, k);
     else
-        gate_bwd_aux_kernel<float><<<kAuxChunks, warps * 32, smem, stream>>>(
+        (void)launch_chained(gate_bwd_aux_kernel<float>, kAuxChunks, warps * 32, smem, stream, 
             dp, tb.topk_w, tb.topk_idx, tb.counts_chosen, logits, b_gate, coef, (float*)dlogits, aux_partial, T, E, width, ld, k);
     return cudaGetLastError();
 }

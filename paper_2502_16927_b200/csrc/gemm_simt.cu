@@ -15,6 +15,8 @@ template <typename T> __device__ __forceinline__ float ld(const T* p) { return (
 
 template <typename T>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     __shared__ float As[TK][TM + 4];
     __shared__ float Bs[TK][TN + 4];
     const T* A = (const T*)g.A;
@@ -107,9 +109,9 @@ cudaError_t gemm_simt(const GemmArgs& g, int dtype, cudaStream_t stream) {
     if (g.M <= 0 || g.N <= 0) return cudaSuccess;
     dim3 grid((g.M + TM - 1) / TM, (g.N + TN - 1) / TN, g.group == GROUP_K ? g.num_experts : 1);
     if (dtype == BIGMAC_BF16)
-        gemm_simt_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(g);
+        (void)launch_chained(gemm_simt_kernel<__nv_bfloat16>, grid, 256, 0, stream, g);
     else
-        gemm_simt_kernel<float><<<grid, 256, 0, stream>>>(g);
+        (void)launch_chained(gemm_simt_kernel<float>, grid, 256, 0, stream, g);
     return cudaGetLastError();
 }
 

@@ -55,8 +55,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     static_assert(!GATHER || A_KMAJOR, "gathered rows: K-major A");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int tiles_m, tiles_n;
-    const int total = total_tiles(p, BN, tiles_m, tiles_n);
+    if (threadIdx.x == 32) {                                 // the maps are on their way while the barriers are set up
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+        prefetch_tensormap(&map_c);
+        prefetch_tensormap(&map_z);
+        prefetch_tensormap(&map_b2);
+    }
 
     if (threadIdx.x == 0) {
         // a gathered slice completes on the B box's bytes and on the arrival of every gathering thread
@@ -70,8 +75,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
+    // Chained launch: everything above touched no global memory and may have run while the kernel before this one in
+    // the stream was still working.  Tensor memory is held, so the next kernel of the stream may be set up in turn;
+    // from the wait on, the predecessor's results are complete.
+    grid_dependency_launch();
+    grid_dependency_wait();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    int tiles_m, tiles_n;
+    const int total = total_tiles(p, BN, tiles_m, tiles_n);
 
     if (GATHER && warp >= 2 + kEpiWarps) {
         // ------------------------------------------------------------------ gathered A rows (two warps)
@@ -281,7 +293,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
             }
         }
-        if (TMA_EPI && lane == 0) tma_store_wait_all();
+        if (TMA_EPI && lane == 0) tma_store_wait_read();          // the boxes have left shared memory; the writes land before the grid ends
     }
     tc_fence_before();
     __syncthreads();
@@ -305,8 +317,7 @@ cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorM
         once.mark(dev);
     }
     const int grid = max_tiles < sm_count() ? max_tiles : sm_count();
-    kernel<<<grid, GATHER ? kThreadsGather : kThreadsV2, smem, stream>>>(ma, mb, mc, mz, mb2, p);
-    return cudaGetLastError();
+    return launch_chained(kernel, grid, GATHER ? kThreadsGather : kThreadsV2, smem, stream, ma, mb, mc, mz, mb2, p);
 }
 
 template <int BN, int STAGES, bool TMA_EPI>

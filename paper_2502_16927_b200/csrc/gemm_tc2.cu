@@ -143,9 +143,36 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
+    if (threadIdx.x == 32) {                                 // the maps are on their way while the barriers are set up
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+        prefetch_tensormap(&map_c);
+        prefetch_tensormap(&map_z);
+        prefetch_tensormap(&map_b2);
+    }
+
     const bool leader = rank == 0;
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
 
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], 2 * kEpiWarps); }
+        for (int s = 0; s < kEpiWarps; ++s) mbar_init(&z_bar[s], 1);
+        *dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(tmem_slot, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                      // the peer's barriers exist before anything signals them
+    // Chained launch: everything above touched no global memory and may have run while the kernel before this one in
+    // the stream was still working.  Tensor memory is held, so the next kernel of the stream may be set up in turn;
+    // from the wait on, the predecessor's results are complete.
+    grid_dependency_launch();
+    grid_dependency_wait();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
     // ---- work list
     const int tiles_n = (p.N + BN - 1) / BN;
     int pairs_m = (p.M + 2 * BM - 1) / (2 * BM);
@@ -162,20 +189,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             s_pp[p.num_experts] = run;
         }
     }
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], 2 * kEpiWarps); }
-        for (int s = 0; s < kEpiWarps; ++s) mbar_init(&z_bar[s], 1);
-        *dead = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (warp == 1) tmem_alloc_pair(tmem_slot, TMEM_COLS);
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                                      // the peer's barriers exist before anything signals them
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    __syncthreads();                                         // the pair prefix is in shared memory
     if (p.group == GROUP_M) pairs_m = s_pp[p.num_experts];
     const int total = pairs_m * tiles_n * (p.group == GROUP_K ? p.num_experts : p.split_k);
     const int step_pair = num_clusters / tiles_n, step_n = num_clusters - step_pair * tiles_n;
@@ -355,7 +369,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             }
         }
-        if (TMA_EPI && lane == 0) tma_store_wait_all();
+        if (TMA_EPI && lane == 0) tma_store_wait_read();          // the boxes have left shared memory; the writes land before the grid ends
     }
     tc_fence_before();
     __syncthreads();
@@ -384,8 +398,7 @@ cudaError_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUte
     int64_t clusters = sm_count() / 2;
     if (max_items < clusters) clusters = max_items;
     if (clusters < 1) clusters = 1;
-    kernel<<<(unsigned)(2 * clusters), kThreadsV2, smem, stream>>>(ma, mb, mc, mz, mb2, p);
-    return cudaGetLastError();
+    return launch_chained(kernel, (unsigned)(2 * clusters), kThreadsV2, smem, stream, ma, mb, mc, mz, mb2, p);
 }
 
 template <int BN, int STAGES, bool TMA_EPI>

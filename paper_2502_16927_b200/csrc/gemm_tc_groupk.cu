@@ -115,15 +115,15 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
+    if (threadIdx.x == 32) {                                 // the maps are on their way while the barriers are set up
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+    }
     const bool leader = rank == 0;
     const int num_clusters = gridDim.x >> 1;
     const int tiles_n = (p.N + BN - 1) / BN, pairs_m = (p.M + 2 * BM - 1) / (2 * BM);
     const int per = pairs_m * tiles_n;
 
-    // the offsets come to shared memory in one round trip; the plan is computed from there
-    for (int e = threadIdx.x; e <= p.num_experts; e += blockDim.x) s_off[e] = p.poffsets[e];
-    __syncthreads();
-    if (warp == 0) groupk_plan(s_off, p.num_experts, per, num_clusters, s_pp, s_ss);
     if (threadIdx.x == 0) {
         // a gathered slice completes on the A boxes' bytes, on the leader's copying threads and on the peer's relay thread
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 2 + kGatherWarps * 32 : 1); mbar_init(&empty_bar[s], 1); }
@@ -139,8 +139,18 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();
+    // Chained launch: everything above touched no global memory and may have run while the kernel before this one in
+    // the stream was still working.  Tensor memory is held, so the next kernel of the stream may be set up in turn;
+    // from the wait on, the predecessor's results are complete.
+    grid_dependency_launch();
+    grid_dependency_wait();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // the offsets come to shared memory in one round trip; the plan is computed from there
+    for (int e = threadIdx.x; e <= p.num_experts; e += blockDim.x) s_off[e] = p.poffsets[e];
+    __syncthreads();
+    if (warp == 0) groupk_plan(s_off, p.num_experts, per, num_clusters, s_pp, s_ss);
+    __syncthreads();
     const int total = s_pp[p.num_experts] * per;
     if (blockIdx.x == 0)     // the plan, for the finishing kernel
         for (int e = threadIdx.x; e <= p.num_experts; e += blockDim.x) { plan_out[e] = s_pp[e]; plan_out[p.num_experts + 1 + e] = s_ss[e]; }
@@ -358,6 +368,8 @@ gemm_tc_groupk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 __global__ void __launch_bounds__(256) groupk_finish_kernel(const float* __restrict__ ws, const int32_t* __restrict__ plan,
                                                             __nv_bfloat16* __restrict__ C, int64_t c_stride, int64_t mn,
                                                             int E, int accumulate) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const int e = blockIdx.y;
     const int parts = plan[e + 1] - plan[e];
     if (parts == 1 || (parts == 0 && accumulate)) return;
@@ -428,9 +440,8 @@ cudaError_t gemm_tc_groupk(const GemmArgs& g, int* status, int* sched, void* ws,
         once.mark(dev);
     }
     const int clusters = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
-    if (gather) gemm_tc_groupk_kernel<true><<<2 * clusters, kThreadsGather, smem, stream>>>(ma, mb, p, sched, slots, plan);
-    else gemm_tc_groupk_kernel<false><<<2 * clusters, kThreadsV2, smem, stream>>>(ma, mb, p, sched, slots, plan);
-    return cudaGetLastError();
+    if (gather) return launch_chained(gemm_tc_groupk_kernel<true>, 2 * clusters, kThreadsGather, smem, stream, ma, mb, p, sched, slots, plan);
+    return launch_chained(gemm_tc_groupk_kernel<false>, 2 * clusters, kThreadsV2, smem, stream, ma, mb, p, sched, slots, plan);
 }
 
 // Second step of gemm_tc_groupk (same g, same ws, same stream): adds the parts of split experts, zero-fills the
@@ -442,8 +453,7 @@ cudaError_t gemm_tc_groupk_finish(const GemmArgs& g, void* ws, cudaStream_t stre
     int32_t* plan = (int32_t*)((char*)ws + (((size_t)kGroupKSlots * g.M * g.N * sizeof(float) + 255) & ~(size_t)255));
     const int64_t mn = (int64_t)g.M * g.N;
     dim3 grid((unsigned)((mn / 8 + 255) / 256 < 64 ? (mn / 8 + 255) / 256 : 64), (unsigned)E);
-    groupk_finish_kernel<<<grid, 256, 0, stream>>>(slots, plan, (__nv_bfloat16*)g.C, g.c_stride, mn, E, g.accumulate ? 1 : 0);
-    return cudaGetLastError();
+    return launch_chained(groupk_finish_kernel, grid, 256, 0, stream, slots, plan, (__nv_bfloat16*)g.C, g.c_stride, mn, E, g.accumulate ? 1 : 0);
 }
 
 }  // namespace bigmac

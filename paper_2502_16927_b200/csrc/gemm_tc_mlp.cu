@@ -89,6 +89,12 @@ __device__ __forceinline__ void fused_mlp_body(const CUtensorMap& map_x, const C
     volatile int* dead = (volatile int*)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 32) {                                 // the maps are on their way while the barriers are set up
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_w1);
+        prefetch_tensormap(&map_w2);
+    }
+
     if (threadIdx.x == 0) {
         mbar_init(x_full, 1); mbar_init(x_empty, 1);
         for (int s = 0; s < 2; ++s) {
@@ -108,6 +114,11 @@ __device__ __forceinline__ void fused_mlp_body(const CUtensorMap& map_x, const C
     __syncthreads();
     tc_fence_after();
     if (SPLIT) cluster_sync_all();                        // the peer's barriers exist before anything signals them
+    // Chained launch: everything above touched no global memory and may have run while the kernel before this one in
+    // the stream was still working.  Tensor memory is held, so the next kernel of the stream may be set up in turn;
+    // from the wait on, the predecessor's results are complete.
+    grid_dependency_launch();
+    grid_dependency_wait();
     const uint32_t tmem_base = *tmem_slot;
     const int total = min(*p.n_tiles, p.max_tiles);
     const uint32_t crank = SPLIT ? cluster_ctarank() : 0u;
@@ -355,12 +366,10 @@ cudaError_t launch_fused_mlp(const void* xg, const void* w1, const void* w2, voi
     // at most one tile per SM and an even number of hidden chunks: two SMs per tile, half of the chunks each
     if (p.max_tiles <= sm_count() && (h / BH) % 2 == 0) {
         const int pairs = p.max_tiles < sm_count() / 2 ? p.max_tiles : sm_count() / 2;
-        fused_mlp_split_kernel<<<2 * pairs, kMlpThreads, smem, stream>>>(mx, m1, m2, p);
-    } else {
-        const int grid = p.max_tiles < sm_count() ? p.max_tiles : sm_count();
-        fused_mlp_kernel<<<grid, kMlpThreads, smem, stream>>>(mx, m1, m2, p);
+        return launch_chained(fused_mlp_split_kernel, 2 * pairs, kMlpThreads, smem, stream, mx, m1, m2, p);
     }
-    return cudaGetLastError();
+    const int grid = p.max_tiles < sm_count() ? p.max_tiles : sm_count();
+    return launch_chained(fused_mlp_kernel, grid, kMlpThreads, smem, stream, mx, m1, m2, p);
 }
 
 }  // namespace bigmac

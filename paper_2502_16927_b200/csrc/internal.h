@@ -6,8 +6,31 @@
 #include <stddef.h>
 
 #include "bigmac.h"
+#include "switches.h"
 
 namespace bigmac {
+
+// Chained launches.  A kernel launched through launch_chained may be set up (its CTAs placed, their prologue run)
+// while the kernel before it in the stream is still running; it must call grid_dependency_wait() before it reads
+// or writes any global memory - that call returns once the predecessor has completed and its writes are visible.
+// grid_dependency_launch() lets the successor's set-up begin; a kernel that allocates tensor memory calls it only
+// after its allocation (a successor's CTA on the same SM could otherwise take the columns first and then wait for
+// this kernel for ever).  Launched plainly, both calls do nothing.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                  Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = switches().chain ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
 
 constexpr int kPad = 128;          // expert segments are padded to multiples of this many rows internally
 constexpr int kMaxExperts = 1024;

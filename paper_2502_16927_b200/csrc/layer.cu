@@ -1038,6 +1038,7 @@ int bigmac_debug_set(const char* name, int value) {
     else if (!std::strcmp(name, "fused_mlp")) sw.fused_mlp = value;
     else if (!std::strcmp(name, "epi_parts")) sw.epi_parts = value;
     else if (!std::strcmp(name, "staged_stores")) sw.staged_stores = value;
+    else if (!std::strcmp(name, "chain")) sw.chain = value;
     else if (!std::strcmp(name, "fuse_dispatch")) sw.fuse_dispatch = value;
     else if (!std::strcmp(name, "tc_mask")) sw.tc_mask = (unsigned)value;
     else if (!std::strcmp(name, "defaults")) sw = Switches();

@@ -50,6 +50,8 @@ __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__
                                                        const int32_t* __restrict__ slot_of_prow,
                                                        const int32_t* __restrict__ n_tiles, int k, int vecs_per_row,
                                                        int64_t max_prows) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const int64_t prow0 = (int64_t)warp_global_id() * kDispatchRows;
     int64_t live = (int64_t)(*n_tiles) * kPad;              // a multiple of kDispatchRows
     if (live > max_prows) live = max_prows;
@@ -84,6 +86,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
                                                       const float* __restrict__ w,
                                                       const int32_t* __restrict__ prow_of_slot, int n_tokens, int k,
                                                       int vecs_per_row, int dst_vecs_per_row) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     constexpr int V = Vec<T>::kElems;
     const int t = warp_global_id();
     if (t >= n_tokens) return;
@@ -114,6 +118,8 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const uint4* __restric
                                                           const float* __restrict__ topk_w,
                                                           const int32_t* __restrict__ n_tiles, int k, int vecs_per_row,
                                                           int64_t max_prows) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     constexpr int V = Vec<T>::kElems;
     const int64_t prow = warp_global_id();
     int64_t live = (int64_t)(*n_tiles) * kPad;
@@ -147,6 +153,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) gate_bwd_kernel(float* __restrict__ dp, const float* __restrict__ topk_w,
                                                        const int32_t* __restrict__ topk_idx, T* __restrict__ dlogits,
                                                        int n_tokens, int E, int width, int ld, int k) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const int t = warp_global_id();
     if (t >= n_tokens) return;
     const int lane = threadIdx.x & 31;
@@ -173,6 +181,8 @@ __global__ void __launch_bounds__(256) gate_bwd_kernel(float* __restrict__ dp, c
 // the warp's row of shared memory.  The block then adds its warps' rows in order.
 __global__ void __launch_bounds__(256) colsum_slots_kernel(const float* __restrict__ dl, const int32_t* __restrict__ topk_idx,
                                                            float* __restrict__ partial, int64_t N, int E) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     extern __shared__ float warp_acc[];              // [8][E]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int i = threadIdx.x; i < 8 * E; i += blockDim.x) warp_acc[i] = 0.0f;
@@ -205,6 +215,8 @@ __global__ void __launch_bounds__(256) colsum_slots_kernel(const float* __restri
 __global__ void __launch_bounds__(256) colsum_final_kernel(const float* __restrict__ partial, const float* __restrict__ partial2,
                                                            float* __restrict__ out, int chunks, int chunks2, int cols,
                                                            int accumulate) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (c >= cols) return;
     float total = 0.0f;
@@ -220,6 +232,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ ws, int parts, int M, int N,
                                                             T* __restrict__ dst1, int m_split, T* __restrict__ dst2, int m2,
                                                             int accumulate) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;     // N is a multiple of 4
     if (i >= (int64_t)(m_split + m2) * N) return;
     const int m = (int)(i / N);
@@ -239,6 +253,8 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
 // row are added in part order and rounded to bf16 (x'), the other E stay fp32 (the gate logits).  r, E multiples of 4.
 __global__ void __launch_bounds__(256) descend_reduce_kernel(const float* __restrict__ ws, int parts, int T, int r, int E,
                                                              __nv_bfloat16* __restrict__ x_lo, float* __restrict__ logits) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const int n = r + E;
     const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= (int64_t)T * n) return;
@@ -264,6 +280,8 @@ __global__ void __launch_bounds__(256) descend_reduce_kernel(const float* __rest
 template <typename T>
 __global__ void __launch_bounds__(256) grouped_colsum_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ poffsets,
                                                              float* __restrict__ partial, int vecs_per_row) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     constexpr int V = Vec<T>::kElems;
     __shared__ float part[8][32 * V];
     const int e = blockIdx.y, slice = blockIdx.z, ct = threadIdx.x & 31, rl = threadIdx.x >> 5;
@@ -309,6 +327,8 @@ __global__ void __launch_bounds__(256) grouped_colsum_kernel(const uint4* __rest
 }
 __global__ void __launch_bounds__(256) grouped_colsum_final_kernel(const float* __restrict__ partial, float* __restrict__ out,
                                                                    int64_t n, int width, int accumulate) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;      // i = e * width + col
     if (i >= n) return;
     const int64_t e = i / width, col = i - e * width;
@@ -326,9 +346,8 @@ cudaError_t launch_dispatch(const void* src, void* grouped, const Tables& tb, in
                             int64_t max_prows, cudaStream_t stream) {
     if (max_prows == 0) return cudaSuccess;
     const int vecs = width * elem_bytes(dtype) / 16;
-    dispatch_kernel<<<warp_blocks((max_prows + kDispatchRows - 1) / kDispatchRows), 256, 0, stream>>>((const uint4*)src, (uint4*)grouped, tb.slot_of_prow,
-                                                                tb.n_tiles, k, vecs, max_prows);
-    return cudaGetLastError();
+    return launch_chained(dispatch_kernel, warp_blocks((max_prows + kDispatchRows - 1) / kDispatchRows), 256, 0, stream, (const uint4*)src, (uint4*)grouped, tb.slot_of_prow,
+                          tb.n_tiles, k, vecs, max_prows);
 }
 
 cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const int32_t* prow_of_slot, int T, int k,
@@ -339,11 +358,11 @@ cudaError_t launch_combine(const void* grouped, void* dst, const float* w, const
     const uint4* src = (const uint4*)grouped;
     uint4* out = (uint4*)dst;
     if (dtype == BIGMAC_BF16) {
-        if (may_drop) combine_kernel<__nv_bfloat16, true><<<warp_blocks(T), 256, 0, stream>>>(src, out, w, prow_of_slot, T, k, vecs, dvecs);
-        else combine_kernel<__nv_bfloat16, false><<<warp_blocks(T), 256, 0, stream>>>(src, out, w, prow_of_slot, T, k, vecs, dvecs);
+        if (may_drop) return launch_chained(combine_kernel<__nv_bfloat16, true>, warp_blocks(T), 256, 0, stream, src, out, w, prow_of_slot, T, k, vecs, dvecs);
+        return launch_chained(combine_kernel<__nv_bfloat16, false>, warp_blocks(T), 256, 0, stream, src, out, w, prow_of_slot, T, k, vecs, dvecs);
     } else {
-        if (may_drop) combine_kernel<float, true><<<warp_blocks(T), 256, 0, stream>>>(src, out, w, prow_of_slot, T, k, vecs, dvecs);
-        else combine_kernel<float, false><<<warp_blocks(T), 256, 0, stream>>>(src, out, w, prow_of_slot, T, k, vecs, dvecs);
+        if (may_drop) return launch_chained(combine_kernel<float, true>, warp_blocks(T), 256, 0, stream, src, out, w, prow_of_slot, T, k, vecs, dvecs);
+        return launch_chained(combine_kernel<float, false>, warp_blocks(T), 256, 0, stream, src, out, w, prow_of_slot, T, k, vecs, dvecs);
     }
     return cudaGetLastError();
 }
@@ -353,11 +372,11 @@ cudaError_t launch_combine_bwd(const void* dy_lo, const void* u, void* du, float
     if (max_prows == 0) return cudaSuccess;
     const int vecs = width * elem_bytes(dtype) / 16;
     if (dtype == BIGMAC_BF16)
-        combine_bwd_kernel<__nv_bfloat16><<<warp_blocks(max_prows), 256, 0, stream>>>(
+        (void)launch_chained(combine_bwd_kernel<__nv_bfloat16>, warp_blocks(max_prows), 256, 0, stream, 
             (const uint4*)dy_lo, (const uint4*)u, (uint4*)du, dp, tb.slot_of_prow, tb.topk_w, tb.n_tiles, k, vecs,
             max_prows);
     else
-        combine_bwd_kernel<float><<<warp_blocks(max_prows), 256, 0, stream>>>(
+        (void)launch_chained(combine_bwd_kernel<float>, warp_blocks(max_prows), 256, 0, stream, 
             (const uint4*)dy_lo, (const uint4*)u, (uint4*)du, dp, tb.slot_of_prow, tb.topk_w, tb.n_tiles, k, vecs,
             max_prows);
     return cudaGetLastError();
@@ -367,17 +386,17 @@ cudaError_t launch_gate_bwd(float* dp, const Tables& tb, void* dlogits, int T, i
                             int dtype, cudaStream_t stream) {
     if (T == 0) return cudaSuccess;
     if (dtype == BIGMAC_BF16)
-        gate_bwd_kernel<__nv_bfloat16><<<warp_blocks(T), 256, 0, stream>>>(dp, tb.topk_w, tb.topk_idx,
+        (void)launch_chained(gate_bwd_kernel<__nv_bfloat16>, warp_blocks(T), 256, 0, stream, dp, tb.topk_w, tb.topk_idx,
                                                                           (__nv_bfloat16*)dlogits, T, E, width, ld, k);
     else
-        gate_bwd_kernel<float><<<warp_blocks(T), 256, 0, stream>>>(dp, tb.topk_w, tb.topk_idx, (float*)dlogits, T, E, width, ld, k);
+        (void)launch_chained(gate_bwd_kernel<float>, warp_blocks(T), 256, 0, stream, dp, tb.topk_w, tb.topk_idx, (float*)dlogits, T, E, width, ld, k);
     return cudaGetLastError();
 }
 
 cudaError_t launch_gate_colsum(const float* dl_slot, const Tables& tb, float* db, float* partial, int64_t N, int E,
                                bool accumulate, cudaStream_t stream, const float* aux_partial) {
-    colsum_slots_kernel<<<kColsumChunks, 256, sizeof(float) * 8 * E, stream>>>(dl_slot, tb.topk_idx, partial, N, E);
-    colsum_final_kernel<<<(unsigned)((E + 7) / 8), 256, 0, stream>>>(partial, aux_partial, db, kColsumChunks, kAuxChunks, E, accumulate);
+    (void)launch_chained(colsum_slots_kernel, kColsumChunks, 256, sizeof(float) * 8 * E, stream, dl_slot, tb.topk_idx, partial, N, E);
+    (void)launch_chained(colsum_final_kernel, (unsigned)((E + 7) / 8), 256, 0, stream, partial, aux_partial, db, kColsumChunks, kAuxChunks, E, accumulate);
     return cudaGetLastError();
 }
 
@@ -387,11 +406,11 @@ cudaError_t launch_grouped_colsum(const void* src, const int32_t* poffsets, floa
     const int vecs = width * elem_bytes(dtype) / 16;
     dim3 grid((unsigned)((vecs + 31) / 32), (unsigned)E, (unsigned)kColsumSlices);
     if (dtype == BIGMAC_BF16)
-        grouped_colsum_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const uint4*)src, poffsets, partial, vecs);
+        (void)launch_chained(grouped_colsum_kernel<__nv_bfloat16>, grid, 256, 0, stream, (const uint4*)src, poffsets, partial, vecs);
     else
-        grouped_colsum_kernel<float><<<grid, 256, 0, stream>>>((const uint4*)src, poffsets, partial, vecs);
+        (void)launch_chained(grouped_colsum_kernel<float>, grid, 256, 0, stream, (const uint4*)src, poffsets, partial, vecs);
     const int64_t n = (int64_t)E * width;
-    grouped_colsum_final_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(partial, out, n, width, accumulate ? 1 : 0);
+    (void)launch_chained(grouped_colsum_final_kernel, (unsigned)((n + 255) / 256), 256, 0, stream, partial, out, n, width, accumulate ? 1 : 0);
     return cudaGetLastError();
 }
 
@@ -399,8 +418,7 @@ cudaError_t launch_descend_reduce(const float* ws, int parts, int T, int r, int 
                                   cudaStream_t stream) {
     const int64_t quads = (int64_t)T * (r + E) / 4;
     if (quads == 0) return cudaSuccess;
-    descend_reduce_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, stream>>>(ws, parts, T, r, E, (__nv_bfloat16*)x_lo, logits);
-    return cudaGetLastError();
+    return launch_chained(descend_reduce_kernel, (unsigned)((quads + 255) / 256), 256, 0, stream, ws, parts, T, r, E, (__nv_bfloat16*)x_lo, logits);
 }
 
 cudaError_t launch_splitk_reduce(const float* ws, int parts, int M, int N, void* dst1, int m_split, void* dst2, int m2,
@@ -409,10 +427,10 @@ cudaError_t launch_splitk_reduce(const float* ws, int parts, int M, int N, void*
     if (quads == 0) return cudaSuccess;
     const unsigned blocks = (unsigned)((quads + 255) / 256);
     if (dtype == BIGMAC_BF16)
-        splitk_reduce_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(ws, parts, M, N, (__nv_bfloat16*)dst1, m_split,
+        (void)launch_chained(splitk_reduce_kernel<__nv_bfloat16>, blocks, 256, 0, stream, ws, parts, M, N, (__nv_bfloat16*)dst1, m_split,
                                                                       (__nv_bfloat16*)dst2, m2, accumulate);
     else
-        splitk_reduce_kernel<float><<<blocks, 256, 0, stream>>>(ws, parts, M, N, (float*)dst1, m_split, (float*)dst2, m2,
+        (void)launch_chained(splitk_reduce_kernel<float>, blocks, 256, 0, stream, ws, parts, M, N, (float*)dst1, m_split, (float*)dst2, m2,
                                                                accumulate);
     return cudaGetLastError();
 }

@@ -21,6 +21,8 @@ template <int VPL, bool KREG>
 __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ logits, const float* __restrict__ b_gate,
                                                    int T, int E, int k, int32_t* __restrict__ topk_idx,
                                                    float* __restrict__ topk_w) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (t >= T) return;
@@ -88,6 +90,8 @@ template <int Q>   // float4 loads per lane: E = 32 Q
 __global__ void __launch_bounds__(256) topk8_kernel(const float* __restrict__ logits, const float* __restrict__ b_gate,
                                                     int T, int k, int32_t* __restrict__ topk_idx,
                                                     float* __restrict__ topk_w) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     constexpr int E = 32 * Q;
     const int lane = threadIdx.x & 31, sub = lane & 7;
     const int t = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 4 + (lane >> 3);
@@ -144,6 +148,8 @@ __global__ void __launch_bounds__(256) topk8_kernel(const float* __restrict__ lo
 __global__ void __launch_bounds__(256) sort_local_kernel(const int32_t* __restrict__ topk_idx, int64_t N, int E,
                                                          int32_t* __restrict__ local_rank,
                                                          int32_t* __restrict__ block_counts) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     extern __shared__ int32_t warp_run[];            // [8][E]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int i = threadIdx.x; i < 8 * E; i += blockDim.x) warp_run[i] = 0;
@@ -194,6 +200,8 @@ __global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ b
                                                          int32_t* __restrict__ tile_expert,
                                                          int32_t* __restrict__ n_tiles, int cap,
                                                          int32_t* __restrict__ counts_chosen) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     __shared__ int32_t s_cnt[kMaxExperts];
     __shared__ int32_t s_poff[kMaxExperts + 1];
     __shared__ int32_t s_part[1024];
@@ -277,6 +285,8 @@ __global__ void __launch_bounds__(256) sort_place_kernel(const int32_t* __restri
                                                          int32_t* __restrict__ slot_of_row,
                                                          int32_t* __restrict__ slot_of_prow, int cap,
                                                          int* __restrict__ status) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= N) return;
     const int e = topk_idx[s];
@@ -311,6 +321,8 @@ __global__ void __launch_bounds__(1024) tables_small_kernel(const int32_t* __res
                                                             int32_t* __restrict__ prow_of_slot, int32_t* __restrict__ row_of_slot,
                                                             int32_t* __restrict__ slot_of_row, int32_t* __restrict__ slot_of_prow,
                                                             int* __restrict__ status) {
+    grid_dependency_wait();
+    grid_dependency_launch();
     extern __shared__ int32_t sm[];                  // [32][E] per-warp counts of the chunk, [E] totals so far, 2 x [E+1]: 35 E + 2 ints
     int32_t* warp_run = sm;
     int32_t* total = sm + 32 * E;
@@ -398,14 +410,14 @@ cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, 
     if (k <= 8 && E % 32 == 0 && E <= 256 && ((uintptr_t)logits % 16 == 0) && ((uintptr_t)b_gate % 16 == 0)) {
         const unsigned blocks = (unsigned)((T + 4 * warps - 1) / (4 * warps));
         switch (E / 32) {
-            case 1: topk8_kernel<1><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
-            case 2: topk8_kernel<2><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
-            case 3: topk8_kernel<3><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
-            case 4: topk8_kernel<4><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
-            case 5: topk8_kernel<5><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
-            case 6: topk8_kernel<6><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
-            case 7: topk8_kernel<7><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
-            default: topk8_kernel<8><<<blocks, warps * 32, 0, stream>>>(logits, b_gate, T, k, topk_idx, topk_w); break;
+            case 1: return launch_chained(topk8_kernel<1>, blocks, warps * 32, 0, stream, logits, b_gate, T, k, topk_idx, topk_w);
+            case 2: return launch_chained(topk8_kernel<2>, blocks, warps * 32, 0, stream, logits, b_gate, T, k, topk_idx, topk_w);
+            case 3: return launch_chained(topk8_kernel<3>, blocks, warps * 32, 0, stream, logits, b_gate, T, k, topk_idx, topk_w);
+            case 4: return launch_chained(topk8_kernel<4>, blocks, warps * 32, 0, stream, logits, b_gate, T, k, topk_idx, topk_w);
+            case 5: return launch_chained(topk8_kernel<5>, blocks, warps * 32, 0, stream, logits, b_gate, T, k, topk_idx, topk_w);
+            case 6: return launch_chained(topk8_kernel<6>, blocks, warps * 32, 0, stream, logits, b_gate, T, k, topk_idx, topk_w);
+            case 7: return launch_chained(topk8_kernel<7>, blocks, warps * 32, 0, stream, logits, b_gate, T, k, topk_idx, topk_w);
+            default: return launch_chained(topk8_kernel<8>, blocks, warps * 32, 0, stream, logits, b_gate, T, k, topk_idx, topk_w);
         }
         return cudaGetLastError();
     }
@@ -413,8 +425,8 @@ cudaError_t launch_topk(const float* logits, const float* b_gate, int T, int E, 
     const int vpl = (E + 31) / 32;
 #define BIGMAC_TOPK(V)                                                                                   \
     do {                                                                                                 \
-        if (k <= 32) topk_kernel<V, true><<<grid, block, 0, stream>>>(logits, b_gate, T, E, k, topk_idx, topk_w);  \
-        else topk_kernel<V, false><<<grid, block, 0, stream>>>(logits, b_gate, T, E, k, topk_idx, topk_w);          \
+        if (k <= 32) return launch_chained(topk_kernel<V, true>, grid, block, 0, stream, logits, b_gate, T, E, k, topk_idx, topk_w);  \
+        else return launch_chained(topk_kernel<V, false>, grid, block, 0, stream, logits, b_gate, T, E, k, topk_idx, topk_w);          \
     } while (0)
     if (vpl <= 1) BIGMAC_TOPK(1);
     else if (vpl <= 2) BIGMAC_TOPK(2);
@@ -430,10 +442,9 @@ cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaSt
     const int64_t N = (int64_t)T * k;
     const int64_t P = padded_rows_max(N, E);
     if (tables_kernel_count(N, E) == 1) {
-        tables_small_kernel<<<1, 1024, sizeof(int32_t) * (35 * E + 2), stream>>>(
-            tb.topk_idx, (int)N, E, cap, (int)P, tb.counts, tb.counts_chosen, tb.offsets, tb.poffsets, tb.tile_expert, tb.n_tiles,
-            tb.prow_of_slot, tb.row_of_slot, tb.slot_of_row, tb.slot_of_prow, status);
-        return cudaGetLastError();
+        return launch_chained(tables_small_kernel, 1, 1024, sizeof(int32_t) * (35 * E + 2), stream, tb.topk_idx, (int)N, E, cap,
+                              (int)P, tb.counts, tb.counts_chosen, tb.offsets, tb.poffsets, tb.tile_expert, tb.n_tiles,
+                              tb.prow_of_slot, tb.row_of_slot, tb.slot_of_row, tb.slot_of_prow, status);
     }
     cudaError_t err = cudaMemsetAsync(tb.slot_of_prow, 0xff, sizeof(int32_t) * P, stream);
     if (err != cudaSuccess) return err;
@@ -442,17 +453,19 @@ cudaError_t launch_tables(const Tables& tb, int T, int E, int k, int cap, cudaSt
         if (err != cudaSuccess) return err;
     }
     const int nb = sort_blocks(N);
-    if (nb > 0)
-        sort_local_kernel<<<nb, 256, sizeof(int32_t) * 8 * E, stream>>>(tb.topk_idx, N, E, tb.prow_of_slot,
-                                                                      tb.block_counts);
-    sort_scan_kernel<<<1, 1024, 0, stream>>>(tb.block_counts, nb, E, tb.counts, tb.offsets, tb.poffsets,
-                                             tb.tile_expert, tb.n_tiles, cap, tb.counts_chosen);
+    if (nb > 0) {
+        err = launch_chained(sort_local_kernel, nb, 256, sizeof(int32_t) * 8 * E, stream, tb.topk_idx, N, E, tb.prow_of_slot,
+                             tb.block_counts);
+        if (err != cudaSuccess) return err;
+    }
+    err = launch_chained(sort_scan_kernel, 1, 1024, 0, stream, tb.block_counts, nb, E, tb.counts, tb.offsets, tb.poffsets,
+                         tb.tile_expert, tb.n_tiles, cap, tb.counts_chosen);
+    if (err != cudaSuccess) return err;
     if (N > 0)
-        sort_place_kernel<<<(unsigned)((N + 255) / 256), 256, 0, stream>>>(tb.topk_idx, N, E, tb.block_counts,
-                                                                          tb.offsets, tb.poffsets, tb.prow_of_slot,
-                                                                          tb.row_of_slot, tb.slot_of_row,
-                                                                          tb.slot_of_prow, cap, status);
-    return cudaGetLastError();
+        err = launch_chained(sort_place_kernel, (unsigned)((N + 255) / 256), 256, 0, stream, tb.topk_idx, N, E, tb.block_counts,
+                             tb.offsets, tb.poffsets, tb.prow_of_slot, tb.row_of_slot, tb.slot_of_row, tb.slot_of_prow, cap,
+                             status);
+    return err;
 }
 
 }  // namespace bigmac

@@ -15,6 +15,8 @@ struct Switches {
                             // Off by default: the gathered operand loads (16-byte asynchronous copies by two extra warps)
                             // feed the mainloop at half the rate of TMA boxes (large workload: expert GEMM1 1.08 ms against
                             // 0.73 + 0.07 ms for the dispatch, dW1 1.20 against 0.47 ms)
+    int chain = 1;          // kernels of a call are launched with programmatic stream serialisation: a grid is set up while
+                            // its predecessor still runs and waits (griddepcontrol.wait) before it touches memory (0: plain launches)
     unsigned tc_mask = ~0u; // bit i: contraction i runs on tcgen05 (read when a handle is created)
 };
 
