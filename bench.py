@@ -451,6 +451,53 @@ def run_small_variants(w, x, dy, dev, G, y, dx, base_step, steps):
     return out
 
 
+def run_decode_latencies(peaks, tokens=(1, 8, 16, 64, 512), calls=200):
+    """Inference forward at the decode-shaped configuration for a few batch sizes: latency per call (CUDA events over
+    `calls` back-to-back calls after 20 warm-up calls; the 70 MB a call touches stay in L2, so a warm number), next to
+    the time the touched weights would take from HBM at the measured copy bandwidth."""
+    import torch
+    from paper_2502_16927_b200 import binding
+
+    base = wl.WORKLOADS["decode"]
+    out = {}
+    for T in tokens:
+        w = base.with_tokens(T)
+        inp = wl.make_inputs(w)
+
+        def dev_of(a):
+            return torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).view(torch.bfloat16).cuda()
+
+        dev = {k: dev_of(inp[k]) for k in ("w_gate", "w_down", "w1", "w2", "w_up")}
+        if inp["b_gate"] is not None:
+            dev["b_gate"] = torch.from_numpy(inp["b_gate"]).cuda()
+        x = dev_of(inp["x"])
+        y = torch.empty_like(x)
+        layer = binding.Layer(w.d, w.r, w.h, w.E, w.k, w.T, w.dtype, w.act)
+        for _ in range(20):
+            layer.forward(x, dev, y=y, training=False)
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(calls):
+            layer.forward(x, dev, y=y, training=False)
+        stop.record()
+        torch.cuda.synchronize()
+        us = start.elapsed_time(stop) * 1e3 / calls
+        # touched weights: both projections, the gate, and the experts at least one token chose (expected number for a
+        # uniform gate: E (1 - (1 - k/E)^T))
+        experts = w.E * (1.0 - (1.0 - w.k / w.E) ** T)
+        weight_bytes = 2.0 * (2 * w.d * w.r + w.E * w.d + experts * 2 * w.r * w.h)
+        floor_us = weight_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6
+        out[str(T)] = {"us_per_call": round(us, 1), "weight_streaming_floor_us": round(floor_us, 1),
+                       "times_floor": round(us / floor_us, 1), "tokens_per_s": round(T / (us * 1e-6))}
+        if layer.status() != 0:
+            raise RuntimeError("device status word reports a timed-out wait")
+        layer.close()
+        del dev, x, y
+    return {"workload": "decode (d 2048, r 256, h 1024, E 64, k 8), inference forward", "l2": "warm: a call's 70 MB fit L2",
+            "by_tokens": out}
+
+
 def run_ep_on_one_gpu(w, x, dy, dev, ms_step, steps, esz, size=4):
     """The expert-parallel layer (Fig. 2c) with `size` ranks driven on this one GPU: every rank brings T/size of the
     step's tokens and owns E/size experts; rows travel between the ranks' buffers at width r through the same put /
@@ -942,6 +989,8 @@ def run_ours(args, w):
         ep_line = run_ep_on_one_gpu(w, x, dy, dev, ms_step, max(3, min(args.steps, 10)), esz) if w.dtype == wl.DTYPE_BF16 else None
         variants = run_small_variants(w, x, dy, dev, G, y, dx, step, max(3, min(args.steps, 10)))
         recipe = run_recipe_variant(w, x, dy, dev, G, y, dx, step, max(3, min(args.steps, 10)))
+    decode_lat = run_decode_latencies(peaks) if (rank == 0 and not args.headline_only and w.dtype == wl.DTYPE_BF16
+                                                 and not forward_only_workload) else None
     stages = {}
     gemm_ms = gemm_flops = 0.0
     flops_of = {name: fn(w) for name, fn in GEMM_FLOPS.items()}
@@ -1045,6 +1094,7 @@ def run_ours(args, w):
             "cdac_twin": twin,
             "recipe_variant": recipe,
             "small_variants": variants,
+            "decode_forward": decode_lat,
             "expert_parallel_on_one_gpu": ep_line,
             "groups": groups,
             "stages": stages}
