@@ -34,7 +34,9 @@
  *    runs a few launches that do not depend on each other on a second stream owned by the handle, forked
  *    from and joined back into the caller's stream with events (stream capture sees an ordinary fork and
  *    join; if a launch fails after the fork the second stream is joined back before the error is returned).
- *    One handle serves one stream at a time.
+ *    One handle serves one stream at a time.  The kernels of a call are launched with programmatic stream
+ *    serialisation (each is set up while its predecessor still runs and waits for it before it touches memory):
+ *    results and ordering against other work on the stream are those of plain launches.
  *  - Behaviour does not depend on the environment: the library reads no environment variable.  Measurement and
  *    debugging aids (per-stage timing, single contractions, kernel-choice switches) are declared in
  *    bigmac_debug.h and are not part of this interface.
