@@ -49,20 +49,20 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
     }
 }
 
-// All CTAs of the (cooperative) grid meet here; `phase` counts the barriers passed so far.
+// All CTAs of the (cooperative) grid meet here; `phase` counts the barriers passed so far.  One thread per CTA arrives
+// with a release at GPU scope (the block barrier before it makes the CTA's writes part of what is released) and
+// spins with acquire loads; the block barrier after it hands what was acquired to the other threads.
 __device__ __forceinline__ void grid_barrier(unsigned* counter, unsigned phase, int* status) {
     __syncthreads();
     if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(counter, 1u);
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
         const unsigned target = (phase + 1) * gridDim.x;
         unsigned seen = 0;
         for (uint32_t i = 0; i < (1u << 24); ++i) {
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter));
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
             if (seen >= target) break;
         }
         if (seen < target) atomicExch(status, 1);
-        __threadfence();
     }
     __syncthreads();
 }
