@@ -256,6 +256,51 @@ def test_backward_on_two_streams_equals_backward_on_one_and_can_be_captured(vari
 
 
 @pytest.mark.parametrize("case", [
+    dict(T=3000, d=256, r=128, h=256, E=16, k=4, training=True),      # a training step: every kernel of both passes
+    dict(T=300, d=512, r=128, h=256, E=12, k=3, training=False),      # inference: split descend, experts on CTA pairs
+])
+def test_chained_launches_equal_plain_launches(case):
+    """Every kernel of a call is launched with programmatic stream serialisation (it may be set up while its
+    predecessor still runs and waits for it before touching memory).  Results are bit for bit those of plain
+    launches (the "chain" debug switch off), also when the call is repeated back to back without a synchronisation
+    in between (the next call's first kernels are then set up while this call's last ones run)."""
+    import torch
+    from paper_2502_16927_b200 import binding
+
+    case = dict(case)
+    training = case.pop("training")
+    w = wl.Workload("chain", dtype=wl.DTYPE_BF16, act=wl.ACT_GELU_ERF, seed=421, **case)
+    inp = conditioned(w)
+    dev = to_device(w, inp)
+
+    def run(repeats):
+        layer = make_layer(w)
+        out = None
+        for _ in range(repeats):
+            if training:
+                y = layer.forward(dev["x"], dev, training=True)
+                G = empty_grads(w, "cuda", fill=float("nan"))
+                dx = layer.backward(dev["x"], dev["dy"], dev, G)
+                out = dict(G, y=y, dx=dx)
+            else:
+                out = {"y": layer.forward(dev["x"], dev, training=False)}
+        torch.cuda.synchronize()
+        assert layer.status() == 0
+        out = {key: val.cpu() for key, val in out.items()}
+        layer.close()
+        return out
+
+    chained = run(3)
+    binding.bigmac_debug_set("chain", 0)
+    try:
+        plain = run(1)
+    finally:
+        binding.bigmac_debug_set("defaults")
+    for key, val in chained.items():
+        assert torch.equal(val.view(torch.uint8), plain[key].view(torch.uint8)), key
+
+
+@pytest.mark.parametrize("case", [
     dict(dtype=wl.DTYPE_F32, shape=dict(T=200, d=32, r=16, h=24, E=8, k=3)),               # generic top-k kernel
     dict(dtype=wl.DTYPE_BF16, shape=dict(T=700, d=128, r=64, h=128, E=64, k=8)),            # four-tokens-per-warp kernel, three-pass sort
     dict(dtype=wl.DTYPE_BF16, shape=dict(T=9, d=128, r=64, h=128, E=32, k=4), decode=True), # one-kernel small-batch forward
