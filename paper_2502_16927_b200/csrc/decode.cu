@@ -2,7 +2,7 @@
 //
 // For a handful of tokens the layer is a chain of matrix-vector products that is bound by streaming the touched
 // weights once (W'_down, W_gate, the selected experts' W1/W2, W'_up) and by launch latency; ten separate launches
-// cost far more than the arithmetic.  All SMs walk five phases, four of them separated by grid-wide barriers:
+// cost far more than the arithmetic.  All SMs walk five phases with three grid-wide barriers (after A, C and D):
 //   A  [x' | logits] = x [W'_down ; W_gate]^T           a CTA owns a few weight rows, its sixteen warps a sixteenth of
 //                                                        the contraction each, tokens four at a time
 //   B  top-k + softmax gate values                       one warp per token, repeated by every CTA into its own
