@@ -87,7 +87,7 @@ GEMM_BYTES = {
 
 # DRAM bytes per launch of the two output-heavy contractions as ncu counted them (dram__bytes_read.sum +
 # dram__bytes_write.sum) on a SMALL case of the large workload's widths (T = 8192, N = 65536 routed rows, one launch
-# each: profiles/step_launches_dram_large_widths_T8192.md): expert GEMM1 343.17 MB read + 393.99 MB written, dz
+# each; the capture's summary is kept with the other profiler summaries): expert GEMM1 343.17 MB read + 393.99 MB written, dz
 # 492.26 MB + 264.03 MB.  Split into the bytes that do not depend on the batch (the experts' weights, E h r
 # elements of bf16 = 268.44 MB) and bytes per routed row (the rest / 65536); a full launch is scaled from that by
 # its rows (traffic grows in proportion: operands and outputs are far larger than L2 at both sizes).
